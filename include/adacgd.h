@@ -1,0 +1,202 @@
+/*
+ * adacgd.h -- C ABI of the B200 (sm_100a) implementation of one AdaCGD iteration
+ * (Makarenko, Gasanov, Islamov, Sadiev, Richtarik: "Adaptive Compression for
+ * Communication-Efficient Distributed Training", arXiv 2211.00188).
+ *
+ * The n workers of the paper's problem statement (Eq. 1) are simulated as n rows
+ * of row-major [n x d] binary32 arrays on ONE GPU.  One iteration is, in the
+ * order of Algorithm 1 (with the three-point arguments of Algorithm 2):
+ *
+ *   a0  x <- x - gamma * g                                   (Alg. 1, x-update)
+ *   a1  X_i = grad f_i(x) for every worker i                 (Alg. 1, worker step; Section 6 objective)
+ *   a2  v_i = X_i - g_i,  D_i = ||X_i - Y_i||^2              (Eq. 7 shift; right side of Eq. 10)
+ *   a3  error ||v_i - C_j(v_i)||^2 of every candidate C_j    (left side of Eq. 10)
+ *   a4  level_i = first j whose trigger holds, g_i update    (Eq. 11)
+ *   a5  g~ = (1/n) sum_i g_i, master compression g           (Alg. 1 aggregation; Alg. 2 master step)
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host
+ *     memory.  The library never frees or reallocates a caller's buffer.
+ *   - All device work is enqueued on the stream given to adacgd_init.  A call
+ *     that returns results to the host synchronises that stream; the others
+ *     return as soon as the work is enqueued.
+ *   - Every entry point returns an adacgd_status and never aborts; a message for
+ *     the last failure is available from adacgd_last_error.
+ *   - Arithmetic: every elementwise operation is one IEEE binary32 operation
+ *     (round to nearest even, no fused multiply-add, subnormals kept).  Squared
+ *     norms that feed the trigger are exact sums rounded once to binary64.
+ *     Top-K keeps the first K entries in the order (|v| descending, index
+ *     ascending), |v| compared on its bit pattern (so -0 == +0).
+ */
+#ifndef ADACGD_H
+#define ADACGD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adacgd_ctx adacgd_ctx; /* opaque; created by adacgd_init, released by adacgd_destroy */
+
+typedef enum {
+  ADACGD_OK = 0,
+  ADACGD_ERR_INVALID_ARG = 1, /* null pointer, size out of range, misaligned pointer */
+  ADACGD_ERR_BAD_ORDER = 2,   /* candidate list not ordered strongest compression first */
+  ADACGD_ERR_NONFINITE = 3,   /* an input held Inf/NaN; the estimators of that call are left unchanged */
+  ADACGD_ERR_WORKSPACE = 4,   /* workspace smaller than adacgd_workspace_bytes reports */
+  ADACGD_ERR_CUDA = 5,        /* a CUDA runtime call failed (no device, launch failure, ...) */
+  ADACGD_ERR_UNSUPPORTED = 6  /* valid request that this build does not implement */
+} adacgd_status;
+
+#define ADACGD_MAX_CANDS 8
+
+/* Candidate kinds of the user's compressor set (Section 4.3: "a set of m EF21
+ * compressors sorted from the highest compression level to the lowest"). */
+#define ADACGD_TOPK 0  /* param = K >= 1; K >= d is the identity (Section 2.1) */
+#define ADACGD_QUANT 1 /* param = bits in [2,16]; deterministic uniform quantiser, 2^(bits-1)-1 positive levels */
+
+typedef struct {
+  int32_t kind;
+  int32_t reserved; /* must be 0 */
+  int64_t param;
+} adacgd_cand;
+
+/* A compressor set: m candidates in the order they are tried, and the trigger
+ * zeta >= 0 of Eq. 10.  m = 0 is the identity compressor (no trigger).  Host memory;
+ * copied by the call that receives it.  Top-K parameters must be strictly
+ * increasing along the list and quantiser widths strictly increasing. */
+typedef struct {
+  const adacgd_cand* cands;
+  int32_t m;
+  float zeta;
+} adacgd_cset;
+
+/* Objectives f_i (Eq. 1). m_rows samples per worker, features a_l, targets t_l. */
+#define ADACGD_LOSS_LOGISTIC_NCVX 0 /* (1/m) sum log(1+exp(-t a.x)) + lambda sum x_j^2/(1+x_j^2)  (Section 6) */
+#define ADACGD_LOSS_LOGISTIC_L2 1   /* (1/m) sum log(1+exp(-t a.x)) + (lambda/2) ||x||^2 */
+#define ADACGD_LOSS_LEAST_SQUARES 2 /* ||A x - t||^2 / (2m) */
+#define ADACGD_LOSS_NONE 3          /* no data: the context only serves adacgd_compress */
+
+#define ADACGD_LAYOUT_DENSE 0 /* A: [n][m_rows][d] row-major binary32 */
+#define ADACGD_LAYOUT_CSR 1   /* per worker i: rowptr[i*(m_rows+1) ..], entries of worker i stored from
+                                 nnz_offset = sum of the previous workers' nnz; columns ascending in a row */
+
+typedef struct {
+  int32_t loss;
+  float lambda;
+  int32_t n;          /* workers, 1 <= n <= 65535 */
+  int32_t layout;
+  int64_t d;          /* 1 <= d < 2^31 */
+  int64_t m_rows;     /* samples per worker */
+  const float* A;           /* dev, dense layout */
+  const float* target;      /* dev, [n][m_rows]: labels in {-1,+1} or least-squares targets */
+  const int64_t* csr_rowptr;/* dev, [n][m_rows+1], offsets into csr_col/csr_val, global (not per worker) */
+  const int32_t* csr_col;   /* dev */
+  const float* csr_val;     /* dev */
+} adacgd_problem; /* device arrays are BORROWED for the lifetime of the context */
+
+#define ADACGD_FLAG_HOST_STAGING 1 /* reserve device staging so that adacgd_compress_host can be used */
+
+/* Bytes of device workspace adacgd_init needs for this problem and these sets.
+ * adacgd_compress later accepts any shape with rows <= n and d <= problem->d.
+ * Returns ADACGD_ERR_INVALID_ARG / ADACGD_ERR_BAD_ORDER for bad descriptors. */
+adacgd_status adacgd_workspace_bytes(const adacgd_problem* problem, const adacgd_cset* worker,
+                                     const adacgd_cset* master, int32_t flags, size_t* bytes_out);
+
+/* Inputs of Algorithm 1: x^0, the estimators g_i^0 (g0_mode 0: zero; 1: grad f_i(x^0);
+ * 2: C^1(grad f_i(x^0)) with the first candidate, the CLAG start of Section 2.3),
+ * g~^0 = mean, g^0 = g~^0; step size gamma > 0.
+ *   master = NULL or m = 0: identity master (the setting of the paper's experiments).
+ *   x0_dev: dev [d], copied.  workspace_dev: dev, 256-byte aligned, caller-owned, must
+ *   outlive the context.  cuda_stream: a cudaStream_t (NULL = default stream).
+ * On success *ctx_out owns host-side bookkeeping only. */
+adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem,
+                          const adacgd_cset* worker, const adacgd_cset* master,
+                          const float* x0_dev, float gamma, int32_t g0_mode, int32_t flags,
+                          void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+
+/* Per-iteration record written by adacgd_step. */
+typedef struct {
+  double loss;           /* f(x^{t+1}) = (1/n) sum_i f_i, by-product of a1 */
+  uint64_t bits_up;      /* sum over workers of the bits of the chosen level (this iteration) */
+  uint64_t bits_down;    /* bits of the master's chosen level (32 d for the identity) */
+  int32_t master_level;  /* 0 = skip, j = j-th master candidate; 0 for the identity */
+  int32_t exact_rechecks;/* trigger comparisons that had to be re-evaluated in exact integer arithmetic */
+} adacgd_step_report;
+
+/* n_steps iterations a0..a5 of Algorithm 1 / Algorithm 2.
+ *   report_host: NULL or host array of n_steps records.
+ *   levels_host: NULL or host int32 [n_steps][n], the level each worker chose (Eq. 11:
+ *                0 = skip, j = j-th candidate).
+ * Synchronises the stream iff a host pointer is given. */
+adacgd_status adacgd_step(adacgd_ctx* ctx, int32_t n_steps, adacgd_step_report* report_host,
+                          int32_t* levels_host);
+
+/* Stages a2-a4 (and the mean of a5) on caller arrays: for every row i
+ *     G_i <- AdaCGD_{h=G_i, y=Y_i}(X_i)      (Eq. 11 with EF21 candidates, Eq. 7)
+ * and, if mean_out_dev != NULL, mean_out = (1/rows) sum_i G_i (binary32, summed in row
+ * order, one division).  The master step of Algorithm 2 is the same call with rows = 1,
+ * X = g~^{t+1}, G = g^t, Y = g~^t.
+ *   X_dev, Y_dev: dev [rows][d], read only.  G_dev: dev [rows][d], updated in place.
+ *   cset: host; m = 0 copies X into G.  rows*d must fit the shape given at init.
+ *   Outputs, all dev, each may be NULL:
+ *     level_dev int32[rows]; bits_dev uint64[rows]; err_dev double[rows][m+1] (||v||^2 then
+ *     one value per candidate); D_dev double[rows];
+ *     kept_idx_dev int32[rows][kept_stride]: indices written by a Top-K level, in no
+ *     particular order, kept_cnt_dev int64[rows] their number (0 for other levels).
+ * Returns ADACGD_ERR_NONFINITE only from the _host variant and from adacgd_step (the
+ * device-side flag is read where the stream is synchronised anyway); see
+ * adacgd_get_state(ADACGD_STATE_FLAGS). */
+adacgd_status adacgd_compress(adacgd_ctx* ctx, const float* X_dev, float* G_dev, const float* Y_dev,
+                              int32_t rows, int64_t d, const adacgd_cset* cset, float* mean_out_dev,
+                              int32_t* level_dev, uint64_t* bits_dev, double* err_dev, double* D_dev,
+                              int32_t* kept_idx_dev, int64_t kept_stride, int64_t* kept_cnt_dev);
+
+/* The same operation on HOST arrays: copies X, G, Y to the context's staging area
+ * (requires ADACGD_FLAG_HOST_STAGING), runs adacgd_compress, copies G (and the mean,
+ * levels, bits if requested) back, and synchronises.  Pinned host memory makes the
+ * copies asynchronous but is not required. */
+adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* G_host,
+                                   const float* Y_host, int32_t rows, int64_t d,
+                                   const adacgd_cset* cset, float* mean_out_host,
+                                   int32_t* level_host, uint64_t* bits_host);
+
+/* Stage a1 alone: grads_out_dev [n][d] = grad f_i(x_dev); loss_out_host (may be NULL,
+ * synchronises) = (1/n) sum_i f_i(x). */
+adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_out_dev,
+                              double* loss_out_host);
+
+/* State of Algorithm 1 (its inputs line) plus what the three-point arguments of
+ * Algorithm 2 need.  get/set copy `bytes` bytes (must equal the item's size). */
+#define ADACGD_STATE_X 0        /* x^t            float [d] */
+#define ADACGD_STATE_G 1        /* g~_i^t         float [n][d] */
+#define ADACGD_STATE_GRAD 2     /* grad f_i(x^t)  float [n][d]  (the y of the next worker step) */
+#define ADACGD_STATE_GT 3       /* g~^t           float [d] */
+#define ADACGD_STATE_GM 4       /* g^t            float [d] */
+#define ADACGD_STATE_STEP 5     /* t              int64 */
+#define ADACGD_STATE_BITS_UP 6  /* cumulative     uint64 */
+#define ADACGD_STATE_BITS_DOWN 7/* cumulative     uint64 */
+#define ADACGD_STATE_LEVELS 8   /* last step      int32 [n] */
+#define ADACGD_STATE_FLAGS 9    /* uint32: bit 0 = a non-finite input was seen since init (get only) */
+#define ADACGD_STATE_RECHECKS 10/* uint32: trigger comparisons redone in exact arithmetic since init (get only) */
+adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,
+                               int32_t dst_is_device);
+adacgd_status adacgd_set_state(adacgd_ctx* ctx, int32_t which, const void* src, size_t bytes,
+                               int32_t src_is_device);
+
+/* Message of the last failure on this context (ctx = NULL: of the last failed
+ * adacgd_init / adacgd_workspace_bytes on this thread).  Never NULL. */
+const char* adacgd_last_error(const adacgd_ctx* ctx);
+
+/* Releases host bookkeeping.  Device memory belongs to the caller. */
+void adacgd_destroy(adacgd_ctx* ctx);
+
+/* Number of kernels this library has launched on behalf of ctx since init. */
+int64_t adacgd_launch_count(const adacgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADACGD_H */

@@ -1,0 +1,10 @@
+"""B200 (sm_100a) implementation of one AdaCGD iteration behind a C ABI.
+
+The Python layer only marshals arguments: every step of the path runs in the CUDA
+kernels of libadacgd.so.  Importing this package does not need a GPU; calling it does,
+and there is no CPU fallback.
+"""
+from .binding import (  # noqa: F401
+    AdaCGD, Cand, TOPK, QUANT, LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE,
+    AdacgdError, load_library, EXPORTED_SYMBOLS,
+)

@@ -1,0 +1,503 @@
+// C ABI of libadacgd: context, workspace carving and the iteration driver
+// (Algorithm 1 with the three-point arguments of Algorithm 2).
+#include <new>
+#include <string>
+#include <vector>
+
+#include "adacgd_internal.cuh"
+
+using namespace adacgd;
+
+namespace {
+
+constexpr int LOG_CAP = 256;  // iterations logged on the device between two host reads
+
+struct StepLog {  // one record per iteration, device resident
+  double loss;
+  unsigned long long bits_up, bits_down;
+  int master_level, rechecks;
+};
+
+struct Counters {  // device resident, cumulative
+  long long step;
+  unsigned long long bits_up, bits_down;
+  unsigned int rechecks_seen;
+  unsigned int pad;
+};
+
+thread_local std::string g_err = "";
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct WsLayout {
+  size_t scratch, grad, x, G, gradA, gradB, gtA, gtB, gm, levels, bits, mlevel, mbits, counters, log,
+      loglevels, stage, total;
+};
+
+WsLayout ws_layout(const adacgd_problem& p, bool master_compresses, int flags) {
+  WsLayout L;
+  size_t o = 0;
+  const size_t nd = (size_t)p.n * (size_t)p.d * 4, dd = (size_t)p.d * 4;
+  L.scratch = o; o = align_up(o + scratch_bytes(p.n, p.d), 256);
+  L.grad = o; o = align_up(o + grad_scratch_bytes(p), 256);
+  L.levels = o; o = align_up(o + (size_t)p.n * 4, 256);
+  L.bits = o; o = align_up(o + (size_t)p.n * 8, 256);
+  L.mlevel = o; o = align_up(o + 4, 256);
+  L.mbits = o; o = align_up(o + 8, 256);
+  L.counters = o; o = align_up(o + sizeof(Counters), 256);
+  L.log = o; o = align_up(o + sizeof(StepLog) * LOG_CAP, 256);
+  L.loglevels = o; o = align_up(o + (size_t)LOG_CAP * p.n * 4, 256);
+  L.x = L.G = L.gradA = L.gradB = L.gtA = L.gtB = L.gm = o;
+  if (p.loss != ADACGD_LOSS_NONE) {
+    L.x = o; o = align_up(o + dd, 256);
+    L.G = o; o = align_up(o + nd, 256);
+    L.gradA = o; o = align_up(o + nd, 256);
+    L.gradB = o; o = align_up(o + nd, 256);
+    L.gtA = o; o = align_up(o + dd, 256);
+    L.gtB = o; o = align_up(o + dd, 256);
+    L.gm = o;
+    if (master_compresses) o = align_up(o + dd, 256);
+  }
+  L.stage = o;
+  if (flags & ADACGD_FLAG_HOST_STAGING) o = align_up(o + 3 * nd + dd, 256);
+  L.total = o;
+  return L;
+}
+
+adacgd_status check_problem(const adacgd_problem* p, const char** msg) {
+  if (!p) { *msg = "problem is NULL"; return ADACGD_ERR_INVALID_ARG; }
+  if (p->n < 1 || p->n > 65535) { *msg = "n must be in [1, 65535]"; return ADACGD_ERR_INVALID_ARG; }
+  if (p->d < 1 || p->d >= (1ll << 31)) { *msg = "d must be in [1, 2^31)"; return ADACGD_ERR_INVALID_ARG; }
+  if (p->loss < 0 || p->loss > ADACGD_LOSS_NONE) { *msg = "unknown loss"; return ADACGD_ERR_INVALID_ARG; }
+  if (p->loss != ADACGD_LOSS_NONE) {
+    if (p->m_rows < 1) { *msg = "m_rows must be >= 1"; return ADACGD_ERR_INVALID_ARG; }
+    if (p->layout == ADACGD_LAYOUT_DENSE) {
+      if (!p->A || !p->target) { *msg = "dense layout needs A and target"; return ADACGD_ERR_INVALID_ARG; }
+    } else if (p->layout == ADACGD_LAYOUT_CSR) {
+      *msg = "CSR layout is not implemented in this build";
+      return ADACGD_ERR_UNSUPPORTED;
+    } else {
+      *msg = "unknown layout";
+      return ADACGD_ERR_INVALID_ARG;
+    }
+    if (!(p->lambda >= 0.f)) { *msg = "lambda must be >= 0"; return ADACGD_ERR_INVALID_ARG; }
+  }
+  return ADACGD_OK;
+}
+
+__global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned long long* __restrict__ bits,
+                           const int* __restrict__ mlevel, const unsigned long long* __restrict__ mbits,
+                           const double* __restrict__ loss, const unsigned int* __restrict__ flags,
+                           Counters* cnt, StepLog* log, int* loglevels, int slot) {
+  __shared__ unsigned long long sh[32];
+  unsigned long long a = 0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    a += bits[i];
+    loglevels[(long long)slot * n + i] = levels[i];
+  }
+  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long up = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) up += sh[w];
+    StepLog r;
+    r.loss = loss ? *loss : 0.0;
+    r.bits_up = up;
+    r.bits_down = *mbits;
+    r.master_level = *mlevel;
+    r.rechecks = (int)(flags[1] - cnt->rechecks_seen);
+    cnt->rechecks_seen = flags[1];
+    cnt->step += 1;
+    cnt->bits_up += up;
+    cnt->bits_down += r.bits_down;
+    log[slot] = r;
+  }
+}
+
+__global__ void k_set_master_identity(int* mlevel, unsigned long long* mbits, long long d) {
+  *mlevel = 0;
+  *mbits = 32ull * (unsigned long long)d;
+}
+
+}  // namespace
+
+struct adacgd_ctx {
+  adacgd_problem p;
+  CsetDev wcs, mcs;
+  bool master_compresses;
+  float gamma;
+  int flags;
+  cudaStream_t stream;
+  Scratch scr;
+  GradScratch gs;
+  float *x, *G, *grad_cur, *grad_nxt, *gt_cur, *gt_nxt, *gm, *gm_buf;
+  int* levels;
+  unsigned long long* bits;
+  int* mlevel;
+  unsigned long long* mbits;
+  Counters* counters;
+  StepLog* log;
+  int* loglevels;
+  float* stage;
+  long long launches;
+  std::string err;
+};
+
+namespace {
+
+adacgd_status fail(adacgd_ctx* c, adacgd_status s, const std::string& m) {
+  if (c) c->err = m;
+  else g_err = m;
+  return s;
+}
+
+adacgd_status cuda_fail(adacgd_ctx* c, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  return fail(c, ADACGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+// Worker side + mean, then master side, on the context's own state.
+adacgd_status run_server_and_master(adacgd_ctx* c) {
+  CompressOut mo;
+  memset(&mo, 0, sizeof(mo));
+  if (c->master_compresses) {
+    mo.level = c->mlevel;
+    mo.bits = (uint64_t*)c->mbits;
+    int r = launch_compress(c->scr, c->mcs, c->gt_nxt, c->gm_buf, c->gt_cur, 1, c->p.d, mo, c->stream);
+    if (r < 0) return cuda_fail(c, "master compression");
+    c->launches += r;
+    c->gm = c->gm_buf;
+  } else {
+    c->gm = c->gt_nxt;
+  }
+  float* t = c->gt_cur;
+  c->gt_cur = c->gt_nxt;
+  c->gt_nxt = t;
+  return ADACGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+adacgd_status adacgd_workspace_bytes(const adacgd_problem* problem, const adacgd_cset* worker,
+                                     const adacgd_cset* master, int32_t flags, size_t* bytes_out) {
+  const char* msg = "";
+  adacgd_status s = check_problem(problem, &msg);
+  if (s != ADACGD_OK) return fail(nullptr, s, msg);
+  if (!bytes_out) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "bytes_out is NULL");
+  CsetDev tmp;
+  if ((s = make_cset(worker, problem->d, &tmp, &msg)) != ADACGD_OK) return fail(nullptr, s, msg);
+  if ((s = make_cset(master, problem->d, &tmp, &msg)) != ADACGD_OK) return fail(nullptr, s, msg);
+  const bool mc = master && master->m > 0;
+  *bytes_out = ws_layout(*problem, mc, flags).total;
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, const adacgd_cset* worker,
+                          const adacgd_cset* master, const float* x0_dev, float gamma, int32_t g0_mode,
+                          int32_t flags, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+  const char* msg = "";
+  if (!ctx_out) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx_out is NULL");
+  *ctx_out = nullptr;
+  adacgd_status s = check_problem(problem, &msg);
+  if (s != ADACGD_OK) return fail(nullptr, s, msg);
+  adacgd_ctx* c = new (std::nothrow) adacgd_ctx();
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "out of host memory");
+  c->p = *problem;
+  if ((s = make_cset(worker, problem->d, &c->wcs, &msg)) != ADACGD_OK ||
+      (s = make_cset(master, problem->d, &c->mcs, &msg)) != ADACGD_OK) {
+    delete c;
+    return fail(nullptr, s, msg);
+  }
+  c->master_compresses = master && master->m > 0;
+  c->gamma = gamma;
+  c->flags = flags;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->launches = 0;
+  const bool has_loss = problem->loss != ADACGD_LOSS_NONE;
+  if (has_loss && (!x0_dev || !(gamma > 0.f) || g0_mode < 0 || g0_mode > 2)) {
+    delete c;
+    return fail(nullptr, ADACGD_ERR_INVALID_ARG, "x0_dev must be non-NULL, gamma > 0, g0_mode in {0,1,2}");
+  }
+  if (has_loss && g0_mode == 2 && c->wcs.m == 0) {
+    delete c;
+    return fail(nullptr, ADACGD_ERR_INVALID_ARG, "g0_mode 2 needs a worker candidate");
+  }
+  const WsLayout L = ws_layout(*problem, c->master_compresses, flags);
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255)) {
+    delete c;
+    return fail(nullptr, ADACGD_ERR_INVALID_ARG, "workspace_dev must be non-NULL and 256-byte aligned");
+  }
+  if (workspace_bytes < L.total) {
+    delete c;
+    return fail(nullptr, ADACGD_ERR_WORKSPACE, "workspace smaller than adacgd_workspace_bytes reports");
+  }
+  char* b = (char*)workspace_dev;
+  carve_scratch(&c->scr, b + L.scratch, problem->n, problem->d);
+  c->levels = (int*)(b + L.levels);
+  c->bits = (unsigned long long*)(b + L.bits);
+  c->mlevel = (int*)(b + L.mlevel);
+  c->mbits = (unsigned long long*)(b + L.mbits);
+  c->counters = (Counters*)(b + L.counters);
+  c->log = (StepLog*)(b + L.log);
+  c->loglevels = (int*)(b + L.loglevels);
+  c->stage = (flags & ADACGD_FLAG_HOST_STAGING) ? (float*)(b + L.stage) : nullptr;
+  c->x = c->G = c->grad_cur = c->grad_nxt = c->gt_cur = c->gt_nxt = c->gm = c->gm_buf = nullptr;
+
+  if (cudaMemsetAsync(c->scr.flags, 0, 16, c->stream) != cudaSuccess ||
+      cudaMemsetAsync(c->counters, 0, sizeof(Counters), c->stream) != cudaSuccess) {
+    adacgd_status st = cuda_fail(nullptr, "adacgd_init (memset)");
+    delete c;
+    return st;
+  }
+  if (has_loss) {
+    carve_grad_scratch(&c->gs, b + L.grad, *problem);
+    c->x = (float*)(b + L.x);
+    c->G = (float*)(b + L.G);
+    c->grad_cur = (float*)(b + L.gradA);
+    c->grad_nxt = (float*)(b + L.gradB);
+    c->gt_cur = (float*)(b + L.gtA);
+    c->gt_nxt = (float*)(b + L.gtB);
+    c->gm_buf = c->master_compresses ? (float*)(b + L.gm) : nullptr;
+    const size_t nd = (size_t)problem->n * problem->d * 4, dd = (size_t)problem->d * 4;
+    cudaMemcpyAsync(c->x, x0_dev, dd, cudaMemcpyDeviceToDevice, c->stream);
+    int r = launch_gradient(c->p, c->gs, c->x, c->grad_cur, c->stream);
+    if (r < 0) {
+      adacgd_status st = (r == -2) ? fail(nullptr, ADACGD_ERR_UNSUPPORTED, "layout not implemented")
+                                   : cuda_fail(nullptr, "adacgd_init (gradient)");
+      delete c;
+      return st;
+    }
+    c->launches += r;
+    if (g0_mode == 0) {
+      cudaMemsetAsync(c->G, 0, nd, c->stream);
+    } else if (g0_mode == 1) {
+      cudaMemcpyAsync(c->G, c->grad_cur, nd, cudaMemcpyDeviceToDevice, c->stream);
+    } else {
+      cudaMemsetAsync(c->G, 0, nd, c->stream);
+      adacgd_cand first = worker->cands[0];
+      adacgd_cset one = {&first, 1, 0.f};
+      CsetDev cs1;
+      make_cset(&one, problem->d, &cs1, &msg);
+      CompressOut o;
+      memset(&o, 0, sizeof(o));
+      r = launch_compress(c->scr, cs1, c->grad_cur, c->G, c->grad_cur, problem->n, problem->d, o, c->stream);
+      if (r < 0) { adacgd_status st = cuda_fail(nullptr, "adacgd_init (g0)"); delete c; return st; }
+      c->launches += r;
+    }
+    r = launch_mean_rows(c->G, problem->n, problem->d, c->gt_cur, c->stream);
+    if (r < 0) { adacgd_status st = cuda_fail(nullptr, "adacgd_init (mean)"); delete c; return st; }
+    c->launches += r;
+    if (c->master_compresses) {
+      cudaMemcpyAsync(c->gm_buf, c->gt_cur, dd, cudaMemcpyDeviceToDevice, c->stream);
+      c->gm = c->gm_buf;
+    } else {
+      c->gm = c->gt_cur;
+      k_set_master_identity<<<1, 1, 0, c->stream>>>(c->mlevel, c->mbits, problem->d);
+      c->launches += 1;
+    }
+  }
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+    adacgd_status st = cuda_fail(nullptr, "adacgd_init");
+    delete c;
+    return st;
+  }
+  *ctx_out = c;
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_compress(adacgd_ctx* ctx, const float* X_dev, float* G_dev, const float* Y_dev, int32_t rows,
+                              int64_t d, const adacgd_cset* cset, float* mean_out_dev, int32_t* level_dev,
+                              uint64_t* bits_dev, double* err_dev, double* D_dev, int32_t* kept_idx_dev,
+                              int64_t kept_stride, int64_t* kept_cnt_dev) {
+  if (!ctx) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!X_dev || !G_dev || !Y_dev) return fail(ctx, ADACGD_ERR_INVALID_ARG, "X, G, Y must be non-NULL");
+  if (rows < 1 || rows > ctx->p.n || d < 1 || d > ctx->p.d)
+    return fail(ctx, ADACGD_ERR_INVALID_ARG, "rows/d exceed the shape given at init");
+  if ((kept_idx_dev != nullptr) != (kept_cnt_dev != nullptr) || (kept_idx_dev && kept_stride < 1))
+    return fail(ctx, ADACGD_ERR_INVALID_ARG, "kept_idx_dev and kept_cnt_dev go together, kept_stride >= 1");
+  const char* msg = "";
+  CsetDev cs;
+  adacgd_status s = make_cset(cset, d, &cs, &msg);
+  if (s != ADACGD_OK) return fail(ctx, s, msg);
+  CompressOut o;
+  o.mean_out = mean_out_dev; o.level = level_dev; o.bits = bits_dev; o.err = err_dev; o.D = D_dev;
+  o.kept_idx = kept_idx_dev; o.kept_stride = kept_stride; o.kept_cnt = (long long*)kept_cnt_dev;
+  int r = launch_compress(ctx->scr, cs, X_dev, G_dev, Y_dev, rows, d, o, ctx->stream);
+  if (r < 0) return cuda_fail(ctx, "adacgd_compress");
+  ctx->launches += r;
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* G_host, const float* Y_host,
+                                   int32_t rows, int64_t d, const adacgd_cset* cset, float* mean_out_host,
+                                   int32_t* level_host, uint64_t* bits_host) {
+  if (!ctx) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!ctx->stage) return fail(ctx, ADACGD_ERR_INVALID_ARG, "context was created without ADACGD_FLAG_HOST_STAGING");
+  if (!X_host || !G_host || !Y_host) return fail(ctx, ADACGD_ERR_INVALID_ARG, "X, G, Y must be non-NULL");
+  if (rows < 1 || rows > ctx->p.n || d < 1 || d > ctx->p.d)
+    return fail(ctx, ADACGD_ERR_INVALID_ARG, "rows/d exceed the shape given at init");
+  const size_t nd = (size_t)rows * (size_t)d * 4;
+  const size_t cap = (size_t)ctx->p.n * (size_t)ctx->p.d;
+  float* Xs = ctx->stage;
+  float* Gs = Xs + cap;
+  float* Ys = Gs + cap;
+  float* Ms = Ys + cap;
+  unsigned int flags_before = 0, flags_after = 0;
+  cudaMemcpyAsync(&flags_before, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
+  cudaMemcpyAsync(Xs, X_host, nd, cudaMemcpyHostToDevice, ctx->stream);
+  cudaMemcpyAsync(Gs, G_host, nd, cudaMemcpyHostToDevice, ctx->stream);
+  cudaMemcpyAsync(Ys, Y_host, nd, cudaMemcpyHostToDevice, ctx->stream);
+  adacgd_status s = adacgd_compress(ctx, Xs, Gs, Ys, rows, d, cset, mean_out_host ? Ms : nullptr,
+                                    level_host ? ctx->levels : nullptr, bits_host ? (uint64_t*)ctx->bits : nullptr,
+                                    nullptr, nullptr, nullptr, 0, nullptr);
+  if (s != ADACGD_OK) return s;
+  cudaMemcpyAsync(G_host, Gs, nd, cudaMemcpyDeviceToHost, ctx->stream);
+  if (mean_out_host) cudaMemcpyAsync(mean_out_host, Ms, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (level_host) cudaMemcpyAsync(level_host, ctx->levels, (size_t)rows * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (bits_host) cudaMemcpyAsync(bits_host, ctx->bits, (size_t)rows * 8, cudaMemcpyDeviceToHost, ctx->stream);
+  cudaMemcpyAsync(&flags_after, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_compress_host");
+  if ((flags_after & 1u) && !(flags_before & 1u))
+    return fail(ctx, ADACGD_ERR_NONFINITE, "an input row held Inf or NaN; its estimator was left unchanged");
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_out_dev, double* loss_out_host) {
+  if (!ctx) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (ctx->p.loss == ADACGD_LOSS_NONE) return fail(ctx, ADACGD_ERR_INVALID_ARG, "context has no objective");
+  if (!x_dev || !grads_out_dev) return fail(ctx, ADACGD_ERR_INVALID_ARG, "x_dev and grads_out_dev must be non-NULL");
+  int r = launch_gradient(ctx->p, ctx->gs, x_dev, grads_out_dev, ctx->stream);
+  if (r < 0) return cuda_fail(ctx, "adacgd_gradient");
+  ctx->launches += r;
+  if (loss_out_host) {
+    cudaMemcpyAsync(loss_out_host, ctx->gs.loss, 8, cudaMemcpyDeviceToHost, ctx->stream);
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_gradient");
+  }
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* report_host, int32_t* levels_host) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (c->p.loss == ADACGD_LOSS_NONE) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective");
+  if (n_steps < 0) return fail(c, ADACGD_ERR_INVALID_ARG, "n_steps must be >= 0");
+  const int n = c->p.n;
+  const long long d = c->p.d;
+  std::vector<StepLog> hostlog;
+  for (int done = 0; done < n_steps;) {
+    const int batch = (n_steps - done < LOG_CAP) ? (n_steps - done) : LOG_CAP;
+    for (int t = 0; t < batch; ++t) {
+      // a0: x^{t+1} = x^t - gamma g^t
+      int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream);
+      if (r < 0) return cuda_fail(c, "x update");
+      c->launches += r;
+      // a1: X_i = grad f_i(x^{t+1})
+      r = launch_gradient(c->p, c->gs, c->x, c->grad_nxt, c->stream);
+      if (r < 0) return cuda_fail(c, "gradient");
+      c->launches += r;
+      // a2-a4 and the mean of a5: h = g~_i^t, y = grad f_i(x^t), x = grad f_i(x^{t+1})
+      CompressOut o;
+      memset(&o, 0, sizeof(o));
+      o.mean_out = c->gt_nxt;
+      o.level = c->levels;
+      o.bits = (uint64_t*)c->bits;
+      r = launch_compress(c->scr, c->wcs, c->grad_nxt, c->G, c->grad_cur, n, d, o, c->stream);
+      if (r < 0) return cuda_fail(c, "worker compression");
+      c->launches += r;
+      // a5: master step h = g^t, y = g~^t, x = g~^{t+1}
+      adacgd_status s = run_server_and_master(c);
+      if (s != ADACGD_OK) return s;
+      float* t2 = c->grad_cur;
+      c->grad_cur = c->grad_nxt;
+      c->grad_nxt = t2;
+      k_log_step<<<1, 256, 0, c->stream>>>(n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
+                                           c->counters, c->log, c->loglevels, t);
+      c->launches += 1;
+    }
+    if (report_host || levels_host) {
+      hostlog.resize(batch);
+      cudaMemcpyAsync(hostlog.data(), c->log, sizeof(StepLog) * batch, cudaMemcpyDeviceToHost, c->stream);
+      if (levels_host)
+        cudaMemcpyAsync(levels_host + (size_t)done * n, c->loglevels, (size_t)batch * n * 4,
+                        cudaMemcpyDeviceToHost, c->stream);
+      if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
+      if (report_host)
+        for (int t = 0; t < batch; ++t) {
+          adacgd_step_report& rr = report_host[done + t];
+          rr.loss = hostlog[t].loss;
+          rr.bits_up = hostlog[t].bits_up;
+          rr.bits_down = hostlog[t].bits_down;
+          rr.master_level = hostlog[t].master_level;
+          rr.exact_rechecks = hostlog[t].rechecks;
+        }
+    }
+    done += batch;
+  }
+  if (report_host || levels_host) {
+    unsigned int fl = 0;
+    cudaMemcpyAsync(&fl, c->scr.flags, 4, cudaMemcpyDeviceToHost, c->stream);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
+    if (fl & 1u) return fail(c, ADACGD_ERR_NONFINITE, "a gradient or estimator held Inf or NaN");
+  }
+  if (cudaGetLastError() != cudaSuccess) return cuda_fail(c, "adacgd_step");
+  return ADACGD_OK;
+}
+
+static adacgd_status state_ptr(adacgd_ctx* c, int32_t which, void** p, size_t* bytes) {
+  const size_t nd = (size_t)c->p.n * c->p.d * 4, dd = (size_t)c->p.d * 4;
+  const bool has = c->p.loss != ADACGD_LOSS_NONE;
+  switch (which) {
+    case ADACGD_STATE_X: *p = c->x; *bytes = dd; break;
+    case ADACGD_STATE_G: *p = c->G; *bytes = nd; break;
+    case ADACGD_STATE_GRAD: *p = c->grad_cur; *bytes = nd; break;
+    case ADACGD_STATE_GT: *p = c->gt_cur; *bytes = dd; break;
+    case ADACGD_STATE_GM: *p = c->gm; *bytes = dd; break;
+    case ADACGD_STATE_STEP: *p = &c->counters->step; *bytes = 8; return ADACGD_OK;
+    case ADACGD_STATE_BITS_UP: *p = &c->counters->bits_up; *bytes = 8; return ADACGD_OK;
+    case ADACGD_STATE_BITS_DOWN: *p = &c->counters->bits_down; *bytes = 8; return ADACGD_OK;
+    case ADACGD_STATE_LEVELS: *p = c->levels; *bytes = (size_t)c->p.n * 4; return ADACGD_OK;
+    case ADACGD_STATE_FLAGS: *p = c->scr.flags; *bytes = 4; return ADACGD_OK;
+    case ADACGD_STATE_RECHECKS: *p = c->scr.flags + 1; *bytes = 4; return ADACGD_OK;
+    default: return fail(c, ADACGD_ERR_INVALID_ARG, "unknown state item");
+  }
+  if (!has) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective, hence no iterate state");
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_get_state(adacgd_ctx* c, int32_t which, void* dst, size_t bytes, int32_t dst_is_device) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!dst) return fail(c, ADACGD_ERR_INVALID_ARG, "dst is NULL");
+  void* p;
+  size_t want;
+  adacgd_status s = state_ptr(c, which, &p, &want);
+  if (s != ADACGD_OK) return s;
+  if (bytes != want) return fail(c, ADACGD_ERR_INVALID_ARG, "bytes does not match the item's size");
+  cudaMemcpyAsync(dst, p, bytes, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream);
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_get_state");
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, size_t bytes, int32_t src_is_device) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!src) return fail(c, ADACGD_ERR_INVALID_ARG, "src is NULL");
+  if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS)
+    return fail(c, ADACGD_ERR_INVALID_ARG, "this item is read-only");
+  void* p;
+  size_t want;
+  adacgd_status s = state_ptr(c, which, &p, &want);
+  if (s != ADACGD_OK) return s;
+  if (bytes != want) return fail(c, ADACGD_ERR_INVALID_ARG, "bytes does not match the item's size");
+  cudaMemcpyAsync(p, src, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream);
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_set_state");
+  return ADACGD_OK;
+}
+
+const char* adacgd_last_error(const adacgd_ctx* ctx) { return ctx ? ctx->err.c_str() : g_err.c_str(); }
+
+void adacgd_destroy(adacgd_ctx* ctx) { delete ctx; }
+
+int64_t adacgd_launch_count(const adacgd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,923 @@
+// Stages a2-a4 of one AdaCGD iteration and the server mean of a5:
+//   v = X - G (EF21 shift, Eq. 7), D = ||X - Y||^2 and the error of every candidate
+//   (both sides of the trigger, Eq. 10), the adaptive level choice and the
+//   estimator update (Eq. 11), and g~ = (1/n) sum_i g_i (Algorithm 1).
+//
+// Selection is an exact three-pass radix select on the bit pattern of |v|
+// (11 + 11 + 9 bits), shared by all Top-K candidates of a row.  Energies are
+// summed in binary64 from non-negative exact terms; a comparison whose margin is
+// below the worst-case summation error is redone in exact integer arithmetic.
+#include "adacgd_internal.cuh"
+
+namespace adacgd {
+
+// --------------------------------------------------------------------------
+// small helpers
+// --------------------------------------------------------------------------
+__device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+template <bool ALIGNED>
+__device__ __forceinline__ void load4(const float* __restrict__ row, long long c0, long long d, float (&o)[4]) {
+  if (ALIGNED) {
+    float4 t = *reinterpret_cast<const float4*>(row + c0);
+    o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o[k] = (c0 + k < d) ? row[c0 + k] : 0.f;
+  }
+}
+
+template <bool ALIGNED>
+__device__ __forceinline__ void store4(float* __restrict__ row, long long c0, long long d, const float (&o)[4]) {
+  if (ALIGNED) {
+    *reinterpret_cast<float4*>(row + c0) = make_float4(o[0], o[1], o[2], o[3]);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (c0 + k < d) row[c0 + k] = o[k];
+  }
+}
+
+__device__ __forceinline__ u32 warp_sum_u32(u32 v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Exclusive prefix sum of one u32 per thread over the CTA (TPB threads); also returns the total.
+__device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
+  __shared__ u32 wsum[TPB / 32];
+  __shared__ u32 wtot;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  u32 inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  __syncthreads();  // protects wsum against the previous call
+  if (lane == 31) wsum[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    u32 w = (lane < TPB / 32) ? wsum[lane] : 0;
+    u32 winc = w;
+#pragma unroll
+    for (int o = 1; o < TPB / 32; o <<= 1) {
+      u32 t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    if (lane < TPB / 32) wsum[lane] = winc - w;
+    if (lane == TPB / 32 - 1) wtot = winc;
+  }
+  __syncthreads();
+  if (total) *total = wtot;
+  return wsum[wid] + inc - v;
+}
+
+// Finds, in a histogram of nb bins ordered by key, the bin that holds the krem-th
+// largest key: out[0] = bin, out[1] = number of keys in higher bins.  All TPB threads call.
+__device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 krem, u32* out) {
+  const int per = nb / TPB;  // 8 or 2
+  u32 loc[8];
+  u32 sum = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    loc[k] = (k < per) ? hist[nb - 1 - (threadIdx.x * per + k)] : 0;
+    sum += loc[k];
+  }
+  u32 excl = block_excl_scan(sum, nullptr);
+  if (krem > excl && krem <= excl + sum) {
+    u32 run = excl;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (k < per) {
+        if (krem <= run + loc[k]) {
+          out[0] = nb - 1 - (threadIdx.x * per + k);
+          out[1] = run;
+          break;
+        }
+        run += loc[k];
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// --------------------------------------------------------------------------
+// radix-select passes
+// --------------------------------------------------------------------------
+// PASS 1: histogram of key[30:20] (one table per row) and the row maximum.
+// PASS 2: for every selecting candidate, histogram of key[19:9] over the keys in its pass-1 bin.
+// PASS 3: histogram of key[8:0] over the keys that share its 22-bit prefix.
+template <int PASS, bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const float* __restrict__ G,
+                                              long long d, int nsel, const SelRow* __restrict__ sel,
+                                              u32* __restrict__ hist, u32* __restrict__ maxkey,
+                                              const RowDec* __restrict__ only_flagged) {
+  extern __shared__ u32 sh[];
+  const int row = blockIdx.y;
+  if (only_flagged && !only_flagged[row].need_exact) return;
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  const int ntab = (PASS == 1) ? 1 : nsel;
+  for (int i = threadIdx.x; i < ntab * NB; i += TPB) sh[i] = 0;
+  u32 pref[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    pref[j] = 0xffffffffu;
+    if (PASS == 2 && j < nsel) pref[j] = sel[row].b1[j];
+    if (PASS == 3 && j < nsel) pref[j] = sel[row].p2[j];
+  }
+  __syncthreads();
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  u32 mx = 0;
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    if (c0 >= d) continue;
+    float x[4], g[4];
+    load4<ALIGNED>(xr, c0, d, x);
+    load4<ALIGNED>(gr, c0, d, g);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (!ALIGNED && c0 + k >= d) break;
+      const u32 key = key_of(__fsub_rn(x[k], g[k]));
+      if (PASS == 1) {
+        mx = max(mx, key);
+        atomicAdd(&sh[key >> 20], 1u);
+      } else if (PASS == 2) {
+#pragma unroll
+        for (int j = 0; j < MAXC; ++j)
+          if (j < nsel && (key >> 20) == pref[j]) atomicAdd(&sh[j * NB + ((key >> 9) & 0x7ffu)], 1u);
+      } else {
+#pragma unroll
+        for (int j = 0; j < MAXC; ++j)
+          if (j < nsel && (key >> 9) == pref[j]) atomicAdd(&sh[j * NB + (key & 0x1ffu)], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  u32* gh = hist + (long long)row * ((PASS == 1) ? NB : MAXC * NB);
+  for (int i = threadIdx.x; i < ntab * NB; i += TPB)
+    if (sh[i]) atomicAdd(&gh[i], sh[i]);
+  if (PASS == 1) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((threadIdx.x & 31) == 0 && mx) atomicMax(&maxkey[row], mx);
+  }
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict__ hist, SelRow* __restrict__ sel,
+                                              const RowDec* __restrict__ only_flagged) {
+  __shared__ u32 res[2];
+  const int row = blockIdx.x;
+  if (only_flagged && !only_flagged[row].need_exact) return;
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  SelRow* s = sel + row;
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 K = (u32)cs.param[cs.sel[j]];
+    const u32* h = hist + (long long)row * ((PASS == 1) ? NB : MAXC * NB) + ((PASS == 1) ? 0 : j * NB);
+    const u32 before = (PASS == 1) ? 0u : (PASS == 2 ? s->above1[j] : s->above2[j]);
+    block_find_kth_desc(h, NB, K - before, res);
+    if (threadIdx.x == 0) {
+      if (PASS == 1) {
+        s->b1[j] = res[0];
+        s->above1[j] = res[1];
+      } else if (PASS == 2) {
+        s->p2[j] = (s->b1[j] << 11) | res[0];
+        s->above2[j] = before + res[1];
+      } else {
+        s->T[j] = (s->p2[j] << 9) | res[0];
+        s->above[j] = before + res[1];
+        s->ntie[j] = h[res[0]];
+        s->q[j] = K - (before + res[1]);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// --------------------------------------------------------------------------
+// energies (binary64, non-negative exact terms)
+// --------------------------------------------------------------------------
+// slot 0: D = sum (x-y)^2; slot 1: sum v^2; slot 2+c (Top-K candidate c with a
+// threshold): sum of v^2 over keys strictly below its threshold.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, const float* __restrict__ G,
+                                                const float* __restrict__ Y, long long d, CsetDev cs,
+                                                const SelRow* __restrict__ sel, double* __restrict__ partial) {
+  const int row = blockIdx.y;
+  u32 T[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) T[j] = (j < cs.nsel) ? sel[row].T[j] : 0u;
+  double aD = 0, aE = 0, aB[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) aB[j] = 0;
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  const float* yr = Y + (long long)row * d;
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    if (c0 >= d) continue;
+    float x[4], g[4], y[4];
+    load4<ALIGNED>(xr, c0, d, x);
+    load4<ALIGNED>(gr, c0, d, g);
+    load4<ALIGNED>(yr, c0, d, y);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (!ALIGNED && c0 + k >= d) break;
+      const float v = __fsub_rn(x[k], g[k]);
+      const float w = __fsub_rn(x[k], y[k]);
+      const double dv = (double)v, dw = (double)w;
+      const double sq = __dmul_rn(dv, dv);
+      aD = __dadd_rn(aD, __dmul_rn(dw, dw));
+      aE = __dadd_rn(aE, sq);
+      const u32 key = key_of(v);
+#pragma unroll
+      for (int j = 0; j < MAXC; ++j)
+        if (j < cs.nsel && key < T[j]) aB[j] = __dadd_rn(aB[j], sq);
+    }
+  }
+  __shared__ double red[NSLOT][TPB / 32];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  double v0 = warp_sum_f64(aD), v1 = warp_sum_f64(aE);
+  if (lane == 0) { red[0][wid] = v0; red[1][wid] = v1; }
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    if (j < cs.nsel) {
+      double vb = warp_sum_f64(aB[j]);
+      if (lane == 0) red[2 + cs.sel[j]][wid] = vb;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < NSLOT) {
+    const int s = threadIdx.x;
+    bool used = (s < 2);
+    for (int j = 0; j < cs.nsel; ++j) used |= (s == 2 + cs.sel[j]);
+    if (used) {
+      double acc = 0;
+      for (int w = 0; w < TPB / 32; ++w) acc += red[s][w];
+      partial[((long long)row * MAX_BLK_PER_ROW + blockIdx.x) * NSLOT + s] = acc;
+    }
+  }
+}
+
+__device__ __forceinline__ float quant_value(float v, float L, float inv, float step) {
+  const float code = fminf(L, rintf(__fmul_rn(fabsf(v), inv)));
+  return copysignf(__fmul_rn(code, step), v);
+}
+
+// slot 2+c for quantiser candidate c: sum (v - Q_c(v))^2 with the row scale s = max|v|.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_quant_err(const float* __restrict__ X, const float* __restrict__ G,
+                                                   long long d, CsetDev cs, const u32* __restrict__ maxkey,
+                                                   double* __restrict__ partial) {
+  const int row = blockIdx.y;
+  const float s = __uint_as_float(maxkey[row]);
+  float L[MAXC], inv[MAXC], step[MAXC];
+  double acc[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    acc[j] = 0;
+    L[j] = inv[j] = step[j] = 0.f;
+    if (j < cs.nquant) {
+      L[j] = (float)((1 << ((int)cs.param[cs.qsel[j]] - 1)) - 1);
+      if (s > 0.f) { inv[j] = __fdiv_rn(L[j], s); step[j] = __fdiv_rn(s, L[j]); }
+    }
+  }
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    if (c0 >= d) continue;
+    float x[4], g[4];
+    load4<ALIGNED>(xr, c0, d, x);
+    load4<ALIGNED>(gr, c0, d, g);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (!ALIGNED && c0 + k >= d) break;
+      const float v = __fsub_rn(x[k], g[k]);
+#pragma unroll
+      for (int j = 0; j < MAXC; ++j) {
+        if (j < cs.nquant) {
+          const double r = (double)__fsub_rn(v, quant_value(v, L[j], inv[j], step[j]));
+          acc[j] = __dadd_rn(acc[j], __dmul_rn(r, r));
+        }
+      }
+    }
+  }
+  __shared__ double red[MAXC][TPB / 32];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    if (j < cs.nquant) {
+      double vb = warp_sum_f64(acc[j]);
+      if (lane == 0) red[j][wid] = vb;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < cs.nquant) {
+    double a = 0;
+    for (int w = 0; w < TPB / 32; ++w) a += red[threadIdx.x][w];
+    partial[((long long)row * MAX_BLK_PER_ROW + blockIdx.x) * NSLOT + 2 + cs.qsel[threadIdx.x]] = a;
+  }
+}
+
+// --------------------------------------------------------------------------
+// level choice (Eq. 11)
+// --------------------------------------------------------------------------
+__device__ uint64_t level_bits(const CsetDev& cs, int level, long long d) {
+  if (level == 0) return 0;
+  const int c = level - 1;
+  if (cs.kind[c] == ADACGD_TOPK) {
+    if (cs.param[c] >= d) return 32ull * (uint64_t)d;
+    int idx_bits = 64 - __clzll((unsigned long long)(d - 1));
+    if (d == 1) idx_bits = 1;
+    if (idx_bits < 1) idx_bits = 1;
+    return (uint64_t)cs.param[c] * (uint64_t)(32 + idx_bits);
+  }
+  return 32ull + (uint64_t)cs.param[c] * (uint64_t)d;
+}
+
+// Fills the decision record of a row once its level is known.
+__device__ void finalize_row(const CsetDev& cs, int row, int level, long long d, const SelRow* sel,
+                             const u32* maxkey, RowDec* dec, const CompressOut& out, const double* e,
+                             double D) {
+  RowDec r;
+  r.level = level; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 0;
+  r.qL = r.qinv = r.qstep = 0.f; r.pad = 0;
+  if (level > 0) {
+    const int c = level - 1;
+    if (cs.kind[c] == ADACGD_TOPK) {
+      if (cs.param[c] >= d) {
+        r.mode = 2;
+      } else {
+        int j = 0;
+        for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
+        r.mode = 1; r.T = sel[row].T[j]; r.q = sel[row].q[j];
+        r.need_tie = (sel[row].q[j] < sel[row].ntie[j]) ? 1 : 0;
+      }
+    } else {
+      r.mode = 3;
+      const float s = __uint_as_float(maxkey[row]);
+      r.qL = (float)((1 << ((int)cs.param[c] - 1)) - 1);
+      if (s > 0.f) { r.qinv = __fdiv_rn(r.qL, s); r.qstep = __fdiv_rn(s, r.qL); }
+    }
+  }
+  dec[row] = r;
+  if (out.level) out.level[row] = level;
+  if (out.bits) out.bits[row] = level_bits(cs, level, d);
+  if (out.D) out.D[row] = D;
+  if (out.err)
+    for (int j = 0; j <= cs.m; ++j) out.err[(long long)row * (cs.m + 1) + j] = e[j];
+}
+
+__global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk, const double* __restrict__ partial,
+                                             const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                                             RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out) {
+  const int row = blockIdx.x, lane = threadIdx.x;
+  double sum[NSLOT];
+#pragma unroll
+  for (int s = 0; s < NSLOT; ++s) {
+    double a = 0;
+    if (s < 2 + cs.m)
+      for (int b = lane; b < nblk; b += 32) a += partial[((long long)row * MAX_BLK_PER_ROW + b) * NSLOT + s];
+    sum[s] = warp_sum_f64(a);
+  }
+  if (lane != 0) return;
+  const double D = sum[0];
+  double e[MAXC + 1];
+  e[0] = sum[1];
+  for (int c = 0; c < cs.m; ++c) {
+    if (cs.kind[c] == ADACGD_TOPK) {
+      if (cs.param[c] >= d) { e[c + 1] = 0.0; continue; }
+      int j = 0;
+      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
+      const double tv = (double)__uint_as_float(sel[row].T[j]);
+      e[c + 1] = sum[2 + c] + (double)(sel[row].ntie[j] - sel[row].q[j]) * (tv * tv);
+    } else {
+      e[c + 1] = sum[2 + c];
+    }
+  }
+  bool finite = (D <= 1.7e308) && (e[0] <= 1.7e308) && (maxkey[row] < 0x7f800000u);
+  if (!finite) {
+    atomicOr(&flags[0], 1u);
+    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, e, D);
+    return;
+  }
+  // worst-case relative error of a binary64 sum of <= d non-negative exact terms, any order,
+  // plus the few roundings of the tie term and of zeta*D on either side
+  const double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;
+  const double rhs = (double)cs.zeta * D;
+  int level = cs.m;
+  bool unsure = false;
+  for (int j = 0; j <= cs.m; ++j) {
+    const double E = e[j];
+    int verdict;  // 1 true, 0 false, -1 unsure
+    if (E == 0.0) verdict = 1;
+    else if (rhs == 0.0) verdict = 0;
+    else if (E * (1.0 + tol) < rhs * (1.0 - tol)) verdict = 1;
+    else if (E * (1.0 - tol) > rhs * (1.0 + tol)) verdict = 0;
+    else verdict = -1;
+    if (verdict == 1) { level = j; break; }
+    if (verdict < 0) { unsure = true; break; }
+  }
+  if (unsure) {
+    RowDec r;
+    r.level = -1; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 1;
+    r.qL = r.qinv = r.qstep = 0.f; r.pad = 0;
+    dec[row] = r;
+    atomicAdd(&flags[1], 1u);
+    return;
+  }
+  finalize_row(cs, row, level, d, sel, maxkey, dec, out, e, D);
+}
+
+// --------------------------------------------------------------------------
+// exact re-evaluation of a row whose comparison could not be certified
+// --------------------------------------------------------------------------
+// A square of a binary32 value is mant^2 * 2^(2*eff-2) units of 2^-298; it is added as
+// three 32-bit pieces into 64-bit limbs (radix 2^32, carries resolved at the end).
+__device__ __forceinline__ void sq_pieces(float w, int* k, u32 (&p)[3]) {
+  const u32 b = key_of(w);
+  const u32 ex = b >> 23, fr = b & 0x7fffffu;
+  const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
+  const int off = 2 * (int)(ex ? ex : 1u) - 2;
+  const unsigned __int128 t = (unsigned __int128)(m * m) << (off & 31);
+  *k = off >> 5;
+  p[0] = (u32)t; p[1] = (u32)(t >> 32); p[2] = (u32)(t >> 64);
+}
+__device__ __forceinline__ void limb_add(u64* limbs, int k, const u32 (&p)[3]) {
+  if (p[0]) atomicAdd(&limbs[k], (u64)p[0]);
+  if (p[1]) atomicAdd(&limbs[k + 1], (u64)p[1]);
+  if (p[2]) atomicAdd(&limbs[k + 2], (u64)p[2]);
+}
+
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X, const float* __restrict__ G,
+                                                    const float* __restrict__ Y, long long d, CsetDev cs,
+                                                    const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                                                    const RowDec* __restrict__ dec, u64* __restrict__ limbs) {
+  const int row = blockIdx.y;
+  if (!dec[row].need_exact) return;
+  __shared__ u64 sh[NSLOT * NLIMB];
+  for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) sh[i] = 0;
+  __syncthreads();
+  const float s = __uint_as_float(maxkey[row]);
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  const float* yr = Y + (long long)row * d;
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    if (c0 >= d) continue;
+    float x[4], g[4], y[4];
+    load4<ALIGNED>(xr, c0, d, x);
+    load4<ALIGNED>(gr, c0, d, g);
+    load4<ALIGNED>(yr, c0, d, y);
+    for (int k = 0; k < 4; ++k) {
+      if (!ALIGNED && c0 + k >= d) break;
+      const float v = __fsub_rn(x[k], g[k]);
+      int kk; u32 p[3];
+      sq_pieces(__fsub_rn(x[k], y[k]), &kk, p);
+      limb_add(sh + 0 * NLIMB, kk, p);
+      sq_pieces(v, &kk, p);
+      limb_add(sh + 1 * NLIMB, kk, p);
+      const u32 key = key_of(v);
+      for (int j = 0; j < cs.nsel; ++j)
+        if (key < sel[row].T[j]) limb_add(sh + (2 + cs.sel[j]) * NLIMB, kk, p);
+      for (int j = 0; j < cs.nquant; ++j) {
+        const int c = cs.qsel[j];
+        const float L = (float)((1 << ((int)cs.param[c] - 1)) - 1);
+        float inv = 0.f, step = 0.f;
+        if (s > 0.f) { inv = __fdiv_rn(L, s); step = __fdiv_rn(s, L); }
+        int k2; u32 p2[3];
+        sq_pieces(__fsub_rn(v, quant_value(v, L, inv, step)), &k2, p2);
+        limb_add(sh + (2 + c) * NLIMB, k2, p2);
+      }
+    }
+  }
+  __syncthreads();
+  u64* gl = limbs + (long long)row * NSLOT * NLIMB;
+  for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) {
+    // split so that the global limb stays below 2^63 for any row length < 2^31
+    const u64 vlo = sh[i] & 0xffffffffull, vhi = sh[i] >> 32;
+    if (vlo) atomicAdd(&gl[i], vlo);
+    if (vhi && (i % NLIMB) + 1 < NLIMB) atomicAdd(&gl[i + 1], vhi);
+  }
+}
+
+// Normalised radix-2^32 digits -> nearest binary64 (ties to even); value = digits * 2^-298.
+__device__ double digits_to_double(const u32* dig) {
+  int t = NLIMB - 1;
+  while (t >= 0 && dig[t] == 0) --t;
+  if (t < 0) return 0.0;
+  const u32 hi = dig[t], mid = (t >= 1) ? dig[t - 1] : 0u, lo = (t >= 2) ? dig[t - 2] : 0u;
+  bool sticky = false;
+  for (int i = 0; i < t - 2; ++i) sticky |= (dig[i] != 0);
+  const unsigned __int128 W = ((unsigned __int128)hi << 64) | ((unsigned __int128)mid << 32) | lo;
+  const int nb = 32 - __clz(hi);         // significant bits of hi
+  const int sh = nb + 11;                // keep 53 of the 64+nb bits
+  u64 mant = (u64)(W >> sh);
+  const bool rnd = (W >> (sh - 1)) & 1;
+  sticky |= (W & (((unsigned __int128)1 << (sh - 1)) - 1)) != 0;
+  if (rnd && (sticky || (mant & 1))) ++mant;
+  return ldexp((double)mant, sh + 32 * (t - 2) - 298);
+}
+
+__global__ void k_pick_exact(CsetDev cs, long long d, const u64* __restrict__ limbs, const SelRow* __restrict__ sel,
+                             const u32* __restrict__ maxkey, RowDec* __restrict__ dec, CompressOut out) {
+  const int row = blockIdx.x;
+  if (threadIdx.x != 0 || !dec[row].need_exact) return;
+  double val[NSLOT];
+  for (int s = 0; s < 2 + cs.m; ++s) {
+    u32 dig[NLIMB];
+    const u64* l = limbs + ((long long)row * NSLOT + s) * NLIMB;
+    unsigned __int128 tie = 0;
+    int tk = 0;
+    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
+      int j = 0;
+      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
+      const u32 T = sel[row].T[j];
+      const u32 ex = T >> 23, fr = T & 0x7fffffu;
+      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
+      const int off = 2 * (int)(ex ? ex : 1u) - 2;
+      tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
+      tk = off >> 5;
+    }
+    u64 carry = 0;
+    for (int k = 0; k < NLIMB; ++k) {
+      u64 add = 0;
+      if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
+      const unsigned __int128 tsum = (unsigned __int128)l[k] + carry + add;
+      dig[k] = (u32)tsum;
+      carry = (u64)(tsum >> 32);
+    }
+    val[s] = digits_to_double(dig);
+    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) val[s] = 0.0;
+  }
+  const double D = val[0];
+  const double rhs = (double)cs.zeta * D;
+  int level = cs.m;
+  for (int j = 0; j <= cs.m; ++j)
+    if (val[1 + j] <= rhs) { level = j; break; }
+  finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
+}
+
+// --------------------------------------------------------------------------
+// tie order, estimator update, server mean
+// --------------------------------------------------------------------------
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, const float* __restrict__ G,
+                                                  long long d, const RowDec* __restrict__ dec,
+                                                  u32* __restrict__ tiecnt, long long nchunk) {
+  const int row = blockIdx.y;
+  if (!dec[row].need_tie) return;
+  const u32 T = dec[row].T;
+  const long long c0 = (long long)blockIdx.x * UPD_COLS + threadIdx.x * 4;
+  u32 cnt = 0;
+  if (c0 < d) {
+    float x[4], g[4];
+    load4<ALIGNED>(X + (long long)row * d, c0, d, x);
+    load4<ALIGNED>(G + (long long)row * d, c0, d, g);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if ((ALIGNED || c0 + k < d) && key_of(__fsub_rn(x[k], g[k])) == T) ++cnt;
+  }
+  u32 total;
+  block_excl_scan(cnt, &total);
+  if (threadIdx.x == 0) tiecnt[(long long)row * nchunk + blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(TPB) k_tiescan(const RowDec* __restrict__ dec, u32* __restrict__ tiecnt,
+                                                 long long nchunk) {
+  const int row = blockIdx.x;
+  if (!dec[row].need_tie) return;
+  u32* t = tiecnt + (long long)row * nchunk;
+  u32 carry = 0;
+  for (long long base = 0; base < nchunk; base += TPB) {
+    const long long i = base + threadIdx.x;
+    const u32 v = (i < nchunk) ? t[i] : 0u;
+    u32 total;
+    const u32 ex = block_excl_scan(v, &total);
+    if (i < nchunk) t[i] = carry + ex;
+    carry += total;
+  }
+}
+
+// Thread owns 4 consecutive columns and walks the rows in order, so that the mean is
+// summed in worker order.  Row i: G_i <- G_i + C_level(X_i - G_i) (EF21, Eq. 7).
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
+                                                long long d, const RowDec* __restrict__ dec,
+                                                const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
+                                                CompressOut out) {
+  const long long c0 = (long long)blockIdx.x * UPD_COLS + threadIdx.x * 4;
+  const bool live = c0 < d;
+  const int lane = threadIdx.x & 31;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int i = 0; i < rows; ++i) {
+    const int mode = copy_mode ? 4 : dec[i].mode;
+    float* grow = G + (long long)i * d;
+    float g[4] = {0.f, 0.f, 0.f, 0.f};
+    if (live && mode != 4) load4<ALIGNED>(grow, c0, d, g);
+    if (mode != 0) {
+      float x[4] = {0.f, 0.f, 0.f, 0.f};
+      if (live) load4<ALIGNED>(X + (long long)i * d, c0, d, x);
+      bool kept[4] = {false, false, false, false};
+      bool any = false;
+      if (mode == 4) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[k] = x[k];
+        any = live;
+      } else if (mode == 1) {
+        const u32 T = dec[i].T, q = dec[i].q;
+        const int need_tie = dec[i].need_tie;
+        u32 key[4];
+        float v[4];
+        u32 nt = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const bool ok = live && (ALIGNED || c0 + k < d);
+          v[k] = __fsub_rn(x[k], g[k]);
+          key[k] = ok ? key_of(v[k]) : 0xffffffffu;  // never equal to T, handled below
+          if (ok && key[k] == T) ++nt;
+        }
+        u32 before = 0;
+        if (need_tie) before = tiepref[(long long)i * nchunk + blockIdx.x] + block_excl_scan(nt, nullptr);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const bool ok = live && (ALIGNED || c0 + k < d);
+          if (!ok) continue;
+          if (key[k] > T) kept[k] = true;
+          else if (key[k] == T) {
+            kept[k] = need_tie ? (before < q) : true;
+            ++before;
+          }
+          if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
+        }
+      } else if (mode == 2) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
+          kept[k] = live && (ALIGNED || c0 + k < d);
+        }
+        any = live;
+      } else {  // quantiser
+        const float L = dec[i].qL, inv = dec[i].qinv, step = dec[i].qstep;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float v = __fsub_rn(x[k], g[k]);
+          g[k] = __fadd_rn(g[k], quant_value(v, L, inv, step));
+        }
+        any = live;
+      }
+      if (any) store4<ALIGNED>(grow, c0, d, g);
+      if (out.kept_idx && (mode == 1 || mode == 2)) {
+        int mine = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mine += kept[k] ? 1 : 0;
+        int inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += t;
+        }
+        const int wtotal = __shfl_sync(0xffffffffu, inc, 31);
+        long long base = 0;
+        if (lane == 31 && wtotal) base = (long long)atomicAdd((u64*)&out.kept_cnt[i], (u64)wtotal);
+        base = __shfl_sync(0xffffffffu, base, 31);
+        long long pos = base + inc - mine;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (kept[k]) {
+            if (pos < out.kept_stride) out.kept_idx[(long long)i * out.kept_stride + pos] = (int32_t)(c0 + k);
+            ++pos;
+          }
+      }
+    }
+    if (out.mean_out) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[k] = (i == 0) ? g[k] : __fadd_rn(acc[k], g[k]);
+    }
+  }
+  if (out.mean_out && live) {
+    const float n = (float)rows;
+    float r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) r[k] = __fdiv_rn(acc[k], n);
+    store4<ALIGNED>(out.mean_out, c0, d, r);
+  }
+}
+
+__global__ void k_copy_report(int rows, long long d, int m, CompressOut out) {
+  // identity compressor: level 0, bits 32 d, no error values
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  if (out.level) out.level[row] = 0;
+  if (out.bits) out.bits[row] = 32ull * (uint64_t)d;
+  if (out.D) out.D[row] = 0.0;
+  if (out.err) out.err[row] = 0.0;
+}
+
+// --------------------------------------------------------------------------
+// host side
+// --------------------------------------------------------------------------
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; }
+
+struct Layout {
+  size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
+};
+
+static Layout layout_of(int rows, long long d) {
+  Layout L;
+  size_t o = 0;
+  L.hist1 = o; o = align_up(o + (size_t)rows * BINS1 * 4, 256);
+  L.hist2 = o; o = align_up(o + (size_t)rows * MAXC * BINS2 * 4, 256);
+  L.hist3 = o; o = align_up(o + (size_t)rows * MAXC * BINS3 * 4, 256);
+  L.maxkey = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.limbs = o; o = align_up(o + (size_t)rows * NSLOT * NLIMB * 8, 256);
+  L.flags = o; o = align_up(o + 16, 256);
+  L.zero_end = o;
+  L.sel = o; o = align_up(o + (size_t)rows * sizeof(SelRow), 256);
+  L.dec = o; o = align_up(o + (size_t)rows * sizeof(RowDec), 256);
+  L.partial = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * NSLOT * 8, 256);
+  L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
+  L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
+  L.total = o;
+  return L;
+}
+
+size_t scratch_bytes(int rows, long long d) { return layout_of(rows, d).total; }
+
+void carve_scratch(Scratch* s, void* base, int rows, long long d) {
+  const Layout L = layout_of(rows, d);
+  char* b = (char*)base;
+  s->hist1 = (u32*)(b + L.hist1);
+  s->hist2 = (u32*)(b + L.hist2);
+  s->hist3 = (u32*)(b + L.hist3);
+  s->maxkey = (u32*)(b + L.maxkey);
+  s->limbs = (u64*)(b + L.limbs);
+  s->flags = (u32*)(b + L.flags);
+  s->zero_begin = b;
+  s->zero_bytes = L.zero_end;
+  s->sel = (SelRow*)(b + L.sel);
+  s->dec = (RowDec*)(b + L.dec);
+  s->partial = (double*)(b + L.partial);
+  s->energy = (double*)(b + L.energy);
+  s->tiecnt = (u32*)(b + L.tiecnt);
+  s->rows_cap = rows;
+  s->d_cap = d;
+  s->nchunk_cap = nchunk_of(d);
+}
+
+adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const char** msg) {
+  CsetDev cs;
+  memset(&cs, 0, sizeof(cs));
+  if (!in || in->m == 0) { *out = cs; return ADACGD_OK; }
+  if (in->m < 0 || in->m > MAXC || !in->cands) { *msg = "candidate count must be in [0, ADACGD_MAX_CANDS] with a non-null list"; return ADACGD_ERR_INVALID_ARG; }
+  if (!(in->zeta >= 0.f) || !(in->zeta <= 3.0e38f)) { *msg = "zeta must be finite and >= 0"; return ADACGD_ERR_INVALID_ARG; }
+  cs.m = in->m;
+  cs.zeta = in->zeta;
+  long long lastK = 0, lastB = 0;
+  for (int c = 0; c < in->m; ++c) {
+    const adacgd_cand& a = in->cands[c];
+    if (a.reserved != 0) { *msg = "candidate.reserved must be 0"; return ADACGD_ERR_INVALID_ARG; }
+    cs.kind[c] = a.kind;
+    cs.param[c] = a.param;
+    if (a.kind == ADACGD_TOPK) {
+      if (a.param < 1) { *msg = "Top-K needs K >= 1"; return ADACGD_ERR_INVALID_ARG; }
+      if (a.param <= lastK) { *msg = "Top-K candidates must have strictly increasing K (strongest compression first)"; return ADACGD_ERR_BAD_ORDER; }
+      if (lastK >= d) { *msg = "only the last Top-K candidate may have K >= d"; return ADACGD_ERR_BAD_ORDER; }
+      lastK = a.param;
+      if (a.param < d) cs.sel[cs.nsel++] = c;
+    } else if (a.kind == ADACGD_QUANT) {
+      if (a.param < 2 || a.param > 16) { *msg = "quantiser width must be in [2,16] bits"; return ADACGD_ERR_INVALID_ARG; }
+      if (a.param <= lastB) { *msg = "quantiser candidates must have strictly increasing width"; return ADACGD_ERR_BAD_ORDER; }
+      lastB = a.param;
+      cs.qsel[cs.nquant++] = c;
+    } else {
+      *msg = "unknown candidate kind";
+      return ADACGD_ERR_INVALID_ARG;
+    }
+  }
+  *out = cs;
+  return ADACGD_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
+                    long long d, const CompressOut& out, cudaStream_t stream) {
+  int launches = 0;
+  static bool attr_done = false;
+  if (!attr_done) {  // tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory
+    cudaFuncSetAttribute(k_hist<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+    cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+    attr_done = true;
+  }
+  const bool al = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y) &&
+                  (!out.mean_out || aligned16(out.mean_out));
+  const long long nchunk = nchunk_of(d);
+  const dim3 ugrid((unsigned)nchunk);
+  if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
+  if (cs.m == 0) {
+    k_copy_report<<<(rows + 127) / 128, 128, 0, stream>>>(rows, d, 0, out);
+    if (al) k_update<true><<<ugrid, TPB, 0, stream>>>(X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
+    else k_update<false><<<ugrid, TPB, 0, stream>>>(X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
+    launches += 2;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+  }
+  // zero the per-call accumulators; the tail of the region depends on rows_cap, so clear by piece
+  cudaMemsetAsync(s.hist1, 0, (size_t)rows * BINS1 * 4, stream);
+  if (cs.nsel) {
+    cudaMemsetAsync(s.hist2, 0, (size_t)rows * MAXC * BINS2 * 4, stream);
+    cudaMemsetAsync(s.hist3, 0, (size_t)rows * MAXC * BINS3 * 4, stream);
+  }
+  cudaMemsetAsync(s.maxkey, 0, (size_t)rows * 4, stream);
+  cudaMemsetAsync(s.limbs, 0, (size_t)rows * NSLOT * NLIMB * 8, stream);
+
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  long long want = (148 * 8 + rows - 1) / rows;
+  if (want > ntile) want = ntile;
+  if (want > MAX_BLK_PER_ROW) want = MAX_BLK_PER_ROW;
+  if (want < 1) want = 1;
+  const int nblk = (int)want;
+  const dim3 sgrid(nblk, rows);
+
+#define LAUNCH_AL(kern, grid, shm, ...)                                          \
+  do {                                                                           \
+    if (al) kern<true><<<grid, TPB, shm, stream>>>(__VA_ARGS__);                 \
+    else kern<false><<<grid, TPB, shm, stream>>>(__VA_ARGS__);                   \
+    ++launches;                                                                  \
+  } while (0)
+#define LAUNCH_HIST(PASS, shm, hist)                                                              \
+  do {                                                                                            \
+    if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr);  \
+    else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr);    \
+    ++launches;                                                                                   \
+  } while (0)
+
+  if (cs.nsel || cs.nquant) {
+    LAUNCH_HIST(1, BINS1 * 4, s.hist1);
+  }
+  if (cs.nsel) {
+    k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, nullptr);
+    LAUNCH_HIST(2, cs.nsel * BINS2 * 4, s.hist2);
+    k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, nullptr);
+    LAUNCH_HIST(3, cs.nsel * BINS3 * 4, s.hist3);
+    k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, nullptr);
+    launches += 3;
+  }
+  LAUNCH_AL(k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial);
+  if (cs.nquant) LAUNCH_AL(k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
+  k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out);
+  LAUNCH_AL(k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs);
+  k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out);
+  launches += 2;
+  if (cs.nsel) {
+    LAUNCH_AL(k_tiecount, dim3((unsigned)nchunk, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
+    k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk);
+    ++launches;
+  }
+  LAUNCH_AL(k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+#undef LAUNCH_AL
+#undef LAUNCH_HIST
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+// --------------------------------------------------------------------------
+// small vector kernels of the loop
+// --------------------------------------------------------------------------
+__global__ void k_axpy(float* __restrict__ x, const float* __restrict__ g, float gamma, long long d) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));
+}
+int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream) {
+  k_axpy<<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(x, g, gamma, d);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+__global__ void k_mean_rows(const float* __restrict__ G, int rows, long long d, float* __restrict__ out) {
+  const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d) return;
+  float acc = G[c];
+  for (int i = 1; i < rows; ++i) acc = __fadd_rn(acc, G[(long long)i * d + c]);
+  out[c] = __fdiv_rn(acc, (float)rows);
+}
+int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStream_t stream) {
+  k_mean_rows<<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(G, rows, d, out);
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace adacgd

@@ -1,0 +1,106 @@
+// Internal declarations shared by the translation units of libadacgd.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "adacgd.h"
+
+namespace adacgd {
+
+typedef uint32_t u32;
+typedef unsigned long long u64;
+
+constexpr int TPB = 256;            // threads per CTA of the streaming kernels
+constexpr int MAXC = ADACGD_MAX_CANDS;
+constexpr int NSLOT = 2 + MAXC;     // energy slots: D, ||v||^2, then one per candidate
+constexpr int NLIMB = 20;           // 32-bit digits of the exact accumulator (covers 2^-298 .. 2^342)
+constexpr int BINS1 = 2048;         // key bits [30:20]
+constexpr int BINS2 = 2048;         // key bits [19:9]
+constexpr int BINS3 = 512;          // key bits [8:0]
+constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (also the tie-order chunk)
+constexpr int MAX_BLK_PER_ROW = 2048;
+
+// Candidate set as the kernels see it (passed by value).
+struct CsetDev {
+  int m;                 // candidates
+  float zeta;
+  int kind[MAXC];
+  long long param[MAXC]; // K or bits
+  int nsel;              // Top-K candidates with K < d: they need a threshold
+  int sel[MAXC];         // their candidate indices, K ascending
+  int nquant;
+  int qsel[MAXC];
+};
+
+// Result of the selection for one row: per selecting candidate (index in CsetDev::sel)
+struct SelRow {
+  u32 b1[MAXC], above1[MAXC];   // pass 1: bin of key[30:20], #keys in higher bins
+  u32 p2[MAXC], above2[MAXC];   // pass 2: key[30:9] prefix, #keys with a higher prefix
+  u32 T[MAXC];                  // threshold key: the K-th largest |v| bit pattern
+  u32 above[MAXC];              // #keys  > T
+  u32 ntie[MAXC];               // #keys == T
+  u32 q[MAXC];                  // how many of the ties are kept (lowest indices first)
+};
+
+// Decision for one row, consumed by the update kernel.
+struct RowDec {
+  int level;       // 0 = skip, j = j-th candidate
+  int mode;        // 0 none, 1 Top-K with threshold, 2 identity (K >= d), 3 quantiser
+  u32 T, q;
+  int need_tie;    // q < ntie: ties must be ranked by index
+  int need_exact;  // the fast comparison could not be certified
+  float qL, qinv, qstep;
+  int pad;
+};
+
+struct Scratch {
+  // carved from the caller's workspace by carve_scratch(); all device pointers
+  u32* hist1;      // [rows][BINS1]
+  u32* hist2;      // [rows][MAXC][BINS2]
+  u32* hist3;      // [rows][MAXC][BINS3]
+  u32* maxkey;     // [rows]
+  u64* limbs;      // [rows][NSLOT][NLIMB] exact accumulators
+  u32* flags;      // [4]: 0 nonfinite seen, 1 #exact rechecks
+  void* zero_begin; size_t zero_bytes;  // region cleared at the start of every call
+  SelRow* sel;     // [rows]
+  RowDec* dec;     // [rows]
+  double* partial; // [rows][MAX_BLK_PER_ROW][NSLOT]
+  double* energy;  // [rows][NSLOT]
+  u32* tiecnt;     // [rows][nchunk]  (exclusive prefix after the scan)
+  int rows_cap; long long d_cap; long long nchunk_cap;
+};
+
+size_t scratch_bytes(int rows, long long d);
+void carve_scratch(Scratch* s, void* base, int rows, long long d);
+
+// Validates and converts a host candidate set. Returns ADACGD_OK / error and a message.
+adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const char** msg);
+
+struct CompressOut {
+  float* mean_out; int32_t* level; uint64_t* bits; double* err; double* D;
+  int32_t* kept_idx; long long kept_stride; long long* kept_cnt;
+};
+
+// Enqueues stages a2-a4 (+ mean) on `stream`; returns the number of kernels launched (<0: CUDA error).
+int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y,
+                    int rows, long long d, const CompressOut& out, cudaStream_t stream);
+
+// ---- gradient stage (a1) ----
+struct GradScratch {
+  float* r;         // [n][m_rows] residuals scaled by 1/m
+  float* part;      // [split][n][d] partial column sums (split > 1 only)
+  double* losspart; // [n][loss_blocks]
+  double* loss;     // [1]
+  int split; int loss_blocks;
+};
+size_t grad_scratch_bytes(const adacgd_problem& p);
+void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p);
+int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
+                    cudaStream_t stream);
+
+// x <- x - gamma * g  (two binary32 roundings: the product, then the difference)
+int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream);
+int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStream_t stream);
+
+}  // namespace adacgd

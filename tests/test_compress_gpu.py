@@ -1,0 +1,234 @@
+"""Parity of stages a2-a4 (+ the server mean) between the CUDA path, called through
+the C ABI, and the CPU oracle on identical binary32 inputs.  Integer results (levels,
+bits, kept index sets) and the estimators must agree bit for bit."""
+import numpy as np
+import pytest
+
+import synthetic_inputs as S
+from oracle import adacgd_oracle as O
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+TOPK, QUANT = 0, 1
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+    return t
+
+
+def gpu_compress(torch, X, G, Y, cands, zeta, want_mean=True, engine=None):
+    import paper_2211_00188_b200 as pkg
+    rows, d = X.shape
+    dev = torch.device("cuda:0")
+    eng = engine or pkg.AdaCGD(rows, d, cands, zeta)
+    Xd, Gd, Yd = (torch.from_numpy(np.ascontiguousarray(a)).to(dev) for a in (X, G, Y))
+    m = len(cands)
+    level = torch.full((rows,), -7, dtype=torch.int32, device=dev)
+    bits = torch.zeros(rows, dtype=torch.int64, device=dev)
+    err = torch.zeros(rows, m + 1, dtype=torch.float64, device=dev)
+    D = torch.zeros(rows, dtype=torch.float64, device=dev)
+    stride = d
+    kept_idx = torch.full((rows, stride), -1, dtype=torch.int32, device=dev)
+    kept_cnt = torch.zeros(rows, dtype=torch.int64, device=dev)
+    mean = torch.zeros(d, dtype=torch.float32, device=dev) if want_mean else None
+    eng.compress(Xd, Gd, Yd, cands, zeta, mean_out=mean, level=level, bits=bits, err=err, D=D,
+                 kept_idx=kept_idx, kept_cnt=kept_cnt)
+    torch.cuda.synchronize()
+    cnt = kept_cnt.cpu().numpy()
+    idx = kept_idx.cpu().numpy()
+    return dict(G=Gd.cpu().numpy(), level=level.cpu().numpy(), bits=bits.cpu().numpy(), err=err.cpu().numpy(),
+                D=D.cpu().numpy(), kept=[np.sort(idx[i, :cnt[i]]) for i in range(rows)],
+                mean=mean.cpu().numpy() if want_mean else None, rechecks=eng.get_state("rechecks"),
+                flags=eng.get_state("flags"), engine=eng)
+
+
+def assert_bitwise(a, b, what):
+    a, b = np.ascontiguousarray(a, F32), np.ascontiguousarray(b, F32)
+    bad = np.nonzero(a.view(np.uint32) != b.view(np.uint32))
+    assert bad[0].size == 0, f"{what}: {bad[0].size} mismatches, first at {tuple(x[0] for x in bad)}"
+
+
+def check_against_oracle(torch, X, G, Y, cands, zeta):
+    got = gpu_compress(torch, X, G, Y, cands, zeta)
+    G_ref, res = O.compress_rows(X, G, Y, cands, zeta)
+    rows, d = X.shape
+    for i, r in enumerate(res):
+        assert got["level"][i] == r["level"], (i, got["level"][i], r["level"], r["err"], r["D"])
+        assert got["bits"][i] == r["bits"], i
+        assert np.allclose(got["err"][i], r["err"], rtol=1e-9, atol=0), (i, got["err"][i], r["err"])
+        assert np.isclose(got["D"][i], r["D"], rtol=1e-9, atol=0)
+        if r["kept"] is not None:
+            assert np.array_equal(got["kept"][i], r["kept"]), (i, r["level"])
+        else:
+            assert got["kept"][i].size == 0
+    assert_bitwise(got["G"], G_ref, "G")
+    assert_bitwise(got["mean"], O.server_mean(G_ref), "mean")
+    assert got["flags"] == 0
+    return got, res
+
+
+CANDS3 = [(TOPK, 3), (TOPK, 30), (TOPK, 300)]
+
+
+@pytest.mark.parametrize("d", [1, 2, 3, 5, 17, 1000, 1023, 1024, 1025, 4096, 5000, 70001])
+@pytest.mark.parametrize("rows", [1, 3])
+def test_topk_gaussian_shapes(torch, rows, d):
+    X, G, Y = S.gaussian_rows(rows, d, seed=d + rows)
+    cands = [(TOPK, k) for k in sorted({1, max(1, d // 100), max(1, d // 10), max(1, d // 2)})]
+    for zeta in (0.0, 1.0, 4.0):
+        check_against_oracle(torch, X, G, Y, cands, zeta)
+
+
+@pytest.mark.parametrize("zeta", [0.0, 0.25, 1.0, 4.0, 1e30])
+def test_zeta_sweep_reaches_every_level(torch, zeta):
+    X, G, Y = S.gaussian_rows(8, 20000, seed=1, drift=0.4, move=0.5)
+    got, res = check_against_oracle(torch, X, G, Y, [(TOPK, 20), (TOPK, 2000), (TOPK, 10000), (TOPK, 20000)], zeta)
+    if zeta == 0.0:
+        assert set(got["level"].tolist()) == {4}      # EF21 with the last candidate (Section 4.3)
+    if zeta == 1e30:
+        assert set(got["level"].tolist()) == {0}      # every worker skips
+
+
+def test_levels_differ_across_rows(torch):
+    # rows with different staleness pick different levels in one call
+    rows, d = 6, 30000
+    X, G, Y = S.gaussian_rows(rows, d, seed=2)
+    rng = np.random.Generator(np.random.PCG64(5))
+    for i, drift in enumerate([0.05, 0.1004, 0.11, 0.12, 0.2, 0.5]):
+        G[i] = (X[i] + drift * rng.standard_normal(d)).astype(F32)
+    got, _ = check_against_oracle(torch, X, G, Y, [(TOPK, 30), (TOPK, 3000), (TOPK, 15000)], 1.0)
+    assert len(set(got["level"].tolist())) >= 3
+
+
+@pytest.mark.parametrize("d", [7, 1000, 4099, 50000])
+def test_ties_and_equalities_use_the_exact_path(torch, d):
+    # small integers: many equal magnitudes (lowest index wins), signed zeros, and
+    # trigger comparisons that hold with equality, which only exact sums decide
+    X, G, Y = S.tie_vectors(4, d, seed=d)
+    total = 0
+    for zeta in (0.0, 0.5, 1.0, 2.0):
+        cands = [(TOPK, k) for k in sorted({1, max(2, d // 7), max(3, d // 2), d - 1 if d > 4 else d})]
+        got, _ = check_against_oracle(torch, X, G, Y, cands, zeta)
+        total += got["rechecks"]
+    # and a row built so that ||v - C(v)||^2 == zeta * D exactly
+    x = np.zeros(d, F32); x[: min(d, 6)] = [3, -1, 2, 0.5, 0, 0][: min(d, 6)]
+    y = x.copy(); y[0] -= 1.0
+    h = np.zeros(d, F32)
+    got, res = check_against_oracle(torch, x[None], h[None], y[None], [(TOPK, 1), (TOPK, 2), (TOPK, 3)], 0.25)
+    if d >= 6:
+        assert res[0]["level"] == 3 and got["rechecks"] >= 1
+
+
+def test_degenerate_rows(torch):
+    d = 3000
+    z = np.zeros((1, d), F32)
+    one = np.ones((1, d), F32)
+    cands = [(TOPK, 5), (TOPK, 500)]
+    check_against_oracle(torch, z, z, z, cands, 1.0)                 # v = 0, D = 0: skip
+    check_against_oracle(torch, one, z, one, cands, 1.0)             # D = 0, all |v| equal: last candidate, ties by index
+    check_against_oracle(torch, one, z, z, cands, 0.5)               # all equal magnitudes
+    check_against_oracle(torch, one, z, z, cands, 1.0)               # ||v||^2 == D: skip by equality
+    neg = -one
+    check_against_oracle(torch, neg, z, one, [(TOPK, 1), (TOPK, d)], 0.1)   # identity last
+    check_against_oracle(torch, neg, z, one, [(TOPK, d + 5)], 0.0)          # K > d
+    tiny = np.full((2, d), 1e-42, F32)                                # subnormal differences
+    tiny[1, ::3] = 3e-45
+    check_against_oracle(torch, tiny, z[[0, 0]], z[[0, 0]], cands, 0.3)
+    big = np.full((1, d), 1e18, F32); big[0, 5] = 3e19                # squares near the top of binary32 range
+    check_against_oracle(torch, big, z, (big * F32(0.5)).astype(F32), cands, 0.2)
+
+
+def test_heavy_tailed_block_scaled_rows(torch):
+    Xs, G0 = S.stress_vectors(3, 120000, blocks=10, period=4, seed=3, device="cpu")
+    X, Y, G = Xs[1].numpy(), Xs[0].numpy(), G0.numpy()
+    for zeta in (0.0, 1.0):
+        check_against_oracle(torch, X, G, Y, [(TOPK, 120), (TOPK, 1200), (TOPK, 12000)], zeta)
+
+
+@pytest.mark.parametrize("d", [9, 1000, 12345])
+def test_quantiser_and_mixed_candidates(torch, d):
+    X, G, Y = S.gaussian_rows(3, d, seed=d)
+    for zeta in (0.0, 0.05, 0.5, 2.0):
+        check_against_oracle(torch, X, G, Y, [(QUANT, 2), (QUANT, 4), (QUANT, 8)], zeta)
+        check_against_oracle(torch, X, G, Y, [(TOPK, 1), (TOPK, max(2, d // 100)), (QUANT, 2), (QUANT, 4),
+                                              (TOPK, max(3, d // 10)), (QUANT, 8)], zeta)
+
+
+def test_identity_set_copies(torch):
+    X, G, Y = S.gaussian_rows(3, 2049, seed=4)
+    got = gpu_compress(torch, X, G, Y, [], 0.0)
+    assert_bitwise(got["G"], X, "G")
+    assert_bitwise(got["mean"], O.server_mean(X), "mean")
+    assert got["level"].tolist() == [0, 0, 0] and got["bits"].tolist() == [32 * 2049] * 3
+
+
+def test_master_step_is_the_same_call_with_one_row(torch):
+    # Algorithm 2: g^{t+1} = C^M_{g^t, g~^t}(g~^{t+1})
+    n, d = 5, 40000
+    X, G, Y = S.gaussian_rows(n, d, seed=6)
+    wc, mc = [(TOPK, 40), (TOPK, 4000)], [(TOPK, 400), (TOPK, 20000)]
+    got = gpu_compress(torch, X, G, Y, wc, 1.0)
+    G_ref, _ = O.compress_rows(X, G, Y, wc, 1.0)
+    gt_new = O.server_mean(G_ref)
+    rng = np.random.Generator(np.random.PCG64(9))
+    gt_old = (gt_new + 0.2 * rng.standard_normal(d)).astype(F32)
+    gm = (gt_old + 0.1 * rng.standard_normal(d)).astype(F32)
+    got_m = gpu_compress(torch, got["mean"][None], gm[None], gt_old[None], mc, 0.5, engine=got["engine"])
+    ref_m = O.adacgd(gm, gt_old, gt_new, mc, 0.5)
+    assert got_m["level"][0] == ref_m["level"] and got_m["bits"][0] == ref_m["bits"]
+    assert_bitwise(got_m["G"][0], ref_m["out"], "gm")
+
+
+def test_repeated_calls_are_deterministic_and_reuse_the_context(torch):
+    X, G, Y = S.gaussian_rows(4, 33333, seed=7)
+    a = gpu_compress(torch, X, G, Y, CANDS3, 1.0)
+    b = gpu_compress(torch, X, G, Y, CANDS3, 1.0, engine=a["engine"])
+    c = gpu_compress(torch, X[:2, :1000].copy(), G[:2, :1000].copy(), Y[:2, :1000].copy(), CANDS3, 1.0, engine=a["engine"])
+    assert_bitwise(a["G"], b["G"], "G")
+    assert np.array_equal(a["err"], b["err"]) and np.array_equal(a["level"], b["level"])
+    G_ref, res = O.compress_rows(X[:2, :1000], G[:2, :1000], Y[:2, :1000], CANDS3, 1.0)
+    assert_bitwise(c["G"], G_ref, "G small")
+
+
+def test_nonfinite_rows_are_flagged_and_left_unchanged(torch):
+    X, G, Y = S.gaussian_rows(3, 5000, seed=8)
+    X[1, 77] = np.inf
+    got = gpu_compress(torch, X, G, Y, CANDS3, 0.0)
+    assert got["flags"] & 1
+    assert got["level"][1] == 0
+    assert_bitwise(got["G"][1], G[1], "flagged row")
+    G_ref, res = O.compress_rows(X[[0, 2]], G[[0, 2]], Y[[0, 2]], CANDS3, 0.0)
+    assert_bitwise(got["G"][[0, 2]], G_ref, "other rows")
+
+
+def test_argument_errors(torch):
+    import paper_2211_00188_b200 as pkg
+    eng = pkg.AdaCGD(2, 100, CANDS3[:1], 1.0)
+    X = torch.zeros(3, 100, device="cuda:0")
+    with pytest.raises(pkg.AdacgdError) as e:
+        eng.compress(X, X.clone(), X)
+    assert e.value.status == 1
+    X = torch.zeros(2, 100, device="cuda:0")
+    with pytest.raises(pkg.AdacgdError) as e:
+        eng.compress(X, X.clone(), X, [(TOPK, 9), (TOPK, 3)], 1.0)
+    assert e.value.status == 2
+    with pytest.raises(pkg.AdacgdError):
+        eng.step(1)
+
+
+def test_host_entry_point(torch):
+    import paper_2211_00188_b200 as pkg
+    n, d = 3, 10000
+    X, G, Y = S.gaussian_rows(n, d, seed=10)
+    eng = pkg.AdaCGD(n, d, CANDS3, 1.0, host_staging=True)
+    Xh, Gh, Yh = (torch.from_numpy(a.copy()).pin_memory() for a in (X, G, Y))
+    mean = torch.zeros(d).pin_memory()
+    level = torch.zeros(n, dtype=torch.int32).pin_memory()
+    bits = torch.zeros(n, dtype=torch.int64).pin_memory()
+    eng.compress_host(Xh, Gh, Yh, mean_out=mean, level=level, bits=bits)
+    G_ref, res = O.compress_rows(X, G, Y, CANDS3, 1.0)
+    assert_bitwise(Gh.numpy(), G_ref, "G")
+    assert_bitwise(mean.numpy(), O.server_mean(G_ref), "mean")
+    assert level.tolist() == [r["level"] for r in res] and bits.tolist() == [r["bits"] for r in res]
