@@ -163,3 +163,26 @@ def gaussian_rows(rows, d, seed=0, drift=0.3, move=0.1):
     G = (X + drift * rng.standard_normal((rows, d))).astype(F32)
     Y = (X + move * rng.standard_normal((rows, d))).astype(F32)
     return X, G, Y
+
+
+def smoothness_estimate(A, loss: int, lam: float, iters: int = 30, seed: int = 0) -> float:
+    """Upper estimate of the smoothness constant of f = (1/n) sum f_i by power iteration
+    (binary64, host): lambda_max of (1/(n m)) sum_i A_i^T A_i, times 1/4 for the logistic
+    losses, plus the regulariser's curvature bound (2 lam for x^2/(1+x^2), lam for l2).
+    Used only to pick a step size gamma for the workloads."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    n, m, d = A.shape
+    v = rng.standard_normal(d)
+    v /= np.linalg.norm(v)
+    lam_max = 0.0
+    for _ in range(iters):
+        w = np.zeros(d)
+        for i in range(n):
+            Ai = A[i].astype(np.float64)
+            w += Ai.T @ (Ai @ v)
+        w /= n * m
+        lam_max = float(np.linalg.norm(w))
+        v = w / max(lam_max, 1e-300)
+    if loss == 2:
+        return lam_max
+    return 0.25 * lam_max + (2.0 * lam if loss == 0 else lam)

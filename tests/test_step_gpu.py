@@ -1,0 +1,190 @@
+"""Parity of the full iteration (stages a0-a5, Algorithm 1 / Algorithm 2) between the
+CUDA path and the CPU oracle: gradients and iterates to rel 1e-5 in lock-step,
+selections bit-exact on identical inputs, loss to rel 1e-3 free-running."""
+import numpy as np
+import pytest
+
+import synthetic_inputs as S
+from oracle import adacgd_oracle as O
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+TOPK, QUANT = 0, 1
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+    return t
+
+
+def relerr(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def make_engine(torch, A, target, loss, lam, x0, gamma, wc, wz, mc=(), mz=0.0, g0_mode=1):
+    import paper_2211_00188_b200 as pkg
+    dev = torch.device("cuda:0")
+    n, m, d = A.shape
+    Ad = torch.from_numpy(A).to(dev)
+    td = torch.from_numpy(target).to(dev)
+    xd = torch.from_numpy(x0).to(dev)
+    return pkg.AdaCGD(n, d, wc, wz, mc, mz, loss=loss, lam=lam, A=Ad, target=td, x0=xd, gamma=gamma, g0_mode=g0_mode)
+
+
+def oracle_problem(A, target, loss, lam):
+    return dict(A=[A[i] for i in range(A.shape[0])], target=[target[i] for i in range(A.shape[0])], loss=loss, lam=lam)
+
+
+@pytest.mark.parametrize("loss,n,m,d", [(0, 3, 50, 1000), (0, 2, 37, 1001), (1, 2, 64, 4096), (2, 3, 40, 777),
+                                        (2, 2, 16, 40000), (0, 2, 9, 33001), (0, 20, 300, 800)])
+def test_gradient_and_loss(torch, loss, n, m, d):
+    if loss == 2:
+        A, t, _ = S.least_squares_problem(n, d, m, seed=d)
+    else:
+        A, t = S.logistic_problem(n, d, m, seed=d)
+    lam = 0.1 if loss != 2 else 0.0
+    x = (0.3 * np.random.Generator(np.random.PCG64(1)).standard_normal(d)).astype(F32)
+    eng = make_engine(torch, A, t, loss, lam, x, 1.0, [(TOPK, 1)], 0.0)
+    xd = torch.from_numpy(x).cuda()
+    out = torch.zeros(n, d, device="cuda:0")
+    f = eng.gradient(xd, out, want_loss=True)
+    prob = oracle_problem(A, t, loss, lam)
+    want = O.all_gradients(prob, x)
+    got = out.cpu().numpy()
+    for i in range(n):
+        assert relerr(got[i], want[i]) <= 1e-5, (i, relerr(got[i], want[i]))
+    assert abs(f - O.global_loss(prob, x)) <= 1e-6 * abs(O.global_loss(prob, x))
+    # the state after init holds the same gradients (g0_mode 1: G = grad)
+    assert relerr(eng.get_state("grad").cpu().numpy(), want) <= 1e-5
+    assert np.array_equal(eng.get_state("G").cpu().numpy(), eng.get_state("grad").cpu().numpy())
+
+
+def push_state(eng, torch, st):
+    for k_gpu, k_or in (("x", "x"), ("G", "G"), ("grad", "X"), ("gt", "gt"), ("gm", "gm")):
+        eng.set_state(k_gpu, torch.from_numpy(np.ascontiguousarray(st[k_or])))
+
+
+def lockstep(torch, A, t, loss, lam, gamma, wc, wz, mc, mz, T, g0_mode=1):
+    n, m, d = A.shape
+    x0 = np.zeros(d, F32)
+    prob = oracle_problem(A, t, loss, lam)
+    st = O.init_state(prob, x0, wc, g0_mode)
+    eng = make_engine(torch, A, t, loss, lam, x0, gamma, wc, wz, mc, mz, g0_mode)
+    # init parity: same estimators up to the gradient tolerance
+    assert relerr(eng.get_state("G").cpu().numpy(), st["G"]) <= 1e-5 or g0_mode != 1
+    levels_seen = set()
+    for it in range(T):
+        push_state(eng, torch, st)
+        before = {k: np.copy(v) for k, v in st.items() if isinstance(v, np.ndarray)}
+        recs, levels = eng.step(1, report=True)
+        O.step(st, prob, gamma, wc, wz, mc, mz)
+        gx = eng.get_state("x").cpu().numpy()
+        ggrad = eng.get_state("grad").cpu().numpy()
+        assert np.array_equal(gx.view(np.uint32), st["x"].view(np.uint32)), it       # same two roundings
+        assert relerr(ggrad, st["X"]) <= 1e-5, (it, relerr(ggrad, st["X"]))
+        assert np.abs(ggrad - st["X"]).max() <= 1e-5 * np.abs(st["X"]).max()
+        f_ref = O.global_loss(prob, st["x"])
+        assert abs(recs[0]["loss"] - f_ref) <= 1e-5 * abs(f_ref)
+        # selections: run the oracle's compressor on the GPU's own gradients
+        G_ref, res = O.compress_rows(ggrad, before["G"], before["X"], wc, wz)
+        assert levels[0] == [r["level"] for r in res], it
+        assert recs[0]["bits_up"] == sum(r["bits"] for r in res)
+        gG = eng.get_state("G").cpu().numpy()
+        assert np.array_equal(gG.view(np.uint32), G_ref.view(np.uint32)), it
+        gt_ref = O.server_mean(G_ref)
+        assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), gt_ref.view(np.uint32))
+        mres = O.adacgd(before["gm"], before["gt"], gt_ref, list(mc), mz)
+        assert np.array_equal(eng.get_state("gm").cpu().numpy().view(np.uint32), mres["out"].view(np.uint32)), it
+        assert recs[0]["master_level"] == mres["level"] and recs[0]["bits_down"] == mres["bits"]
+        levels_seen.update(levels[0])
+    return levels_seen
+
+
+def test_lockstep_c1_shape(torch):
+    # workload c1: n=4, d=1000, m=100, logistic + non-convex regulariser, Top-K {10,50,100,500}
+    W = S.WORKLOADS["c1"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"])
+    seen = lockstep(torch, A, t, W["loss"], W["lam"], gamma, W["worker"], 1.0, [], 0.0, T=40)
+    assert len(seen) >= 2
+
+
+def test_lockstep_bidirectional_small_c2_shape(torch):
+    A, t = S.logistic_problem(5, 800, 200, seed=1)
+    gamma = 0.5 / S.smoothness_estimate(A, 0, 0.1)
+    cands = [(TOPK, 1), (TOPK, 8), (TOPK, 80), (TOPK, 800)]
+    lockstep(torch, A, t, 0, 0.1, gamma, cands, 1.0, cands, 1.0, T=25)
+
+
+def test_lockstep_least_squares_and_quantisers(torch):
+    A, t, _ = S.least_squares_problem(4, 3000, 64, seed=2)
+    gamma = 0.5 / S.smoothness_estimate(A, 2, 0.0)
+    lockstep(torch, A, t, 2, 0.0, gamma, [(TOPK, 3), (QUANT, 2), (TOPK, 300), (QUANT, 8)], 0.5,
+             [(QUANT, 4), (TOPK, 1500)], 0.25, T=15, g0_mode=0)
+    lockstep(torch, A, t, 2, 0.0, gamma, [(TOPK, 30), (TOPK, 300)], 2.0, [], 0.0, T=10, g0_mode=2)
+
+
+def free_run(torch, A, t, loss, lam, gamma, wc, wz, mc, mz, T):
+    n, m, d = A.shape
+    x0 = np.zeros(d, F32)
+    prob = oracle_problem(A, t, loss, lam)
+    st = O.init_state(prob, x0, wc)
+    eng = make_engine(torch, A, t, loss, lam, x0, gamma, wc, wz, mc, mz)
+    recs, levels = eng.step(T, report=True)
+    for it in range(T):
+        O.step(st, prob, gamma, wc, wz, mc, mz)
+    return recs, levels, O.global_loss(prob, st["x"]), O.global_loss(prob, x0), st, eng
+
+
+def test_free_running_c1_loss_trajectory(torch):
+    W = S.WORKLOADS["c1"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"])
+    recs, levels, f_ref, f0, st, eng = free_run(torch, A, t, W["loss"], W["lam"], gamma, W["worker"], 1.0, [], 0.0,
+                                                W["iters"])
+    assert abs(recs[-1]["loss"] - f_ref) <= 1e-3 * abs(f_ref)
+    assert f_ref < 0.9 * f0                                      # the run makes progress
+    assert eng.get_state("step") == W["iters"]
+    assert eng.get_state("bits_up") == sum(r["bits_up"] for r in recs)
+    assert eng.get_state("bits_down") == sum(r["bits_down"] for r in recs)
+    assert relerr(eng.get_state("x").cpu().numpy(), st["x"]) <= 1e-2
+
+
+def test_free_running_gd_special_case_matches_closed_form(torch):
+    # Top-d, zeta = 0, identity master: plain gradient descent (Eq. 2)
+    A, t, _ = S.least_squares_problem(3, 64, 40, seed=3)
+    n, m, d = A.shape
+    H = sum(A[i].astype(np.float64).T @ A[i].astype(np.float64) for i in range(n)) / (n * m)
+    c = sum(A[i].astype(np.float64).T @ t[i].astype(np.float64) for i in range(n)) / (n * m)
+    x_star = np.linalg.solve(H, c)
+    gamma = 1.0 / np.linalg.eigvalsh(H).max()
+    T = 50
+    eng = make_engine(torch, A, t, 2, 0.0, np.ones(d, F32), gamma, [(TOPK, d)], 0.0)
+    recs, levels = eng.step(T, report=True)
+    want = x_star + np.linalg.matrix_power(np.eye(d) - np.float64(F32(gamma)) * H, T) @ (np.ones(d) - x_star)
+    assert np.allclose(eng.get_state("x").cpu().numpy(), want, rtol=0, atol=5e-5 * np.abs(want).max())
+    losses = [r["loss"] for r in recs]
+    assert all(b <= a * (1 + 1e-6) for a, b in zip(losses, losses[1:]))
+    assert all(lv == [1] * n for lv in levels)
+
+
+def test_state_roundtrip_and_errors(torch):
+    import paper_2211_00188_b200 as pkg
+    A, t = S.logistic_problem(2, 100, 10, seed=4)
+    eng = make_engine(torch, A, t, 0, 0.1, np.zeros(100, F32), 0.1, [(TOPK, 5)], 1.0)
+    x = torch.arange(100, dtype=torch.float32)
+    eng.set_state("x", x)
+    assert torch.equal(eng.get_state("x").cpu(), x)
+    G = torch.randn(2, 100)
+    eng.set_state("G", G)
+    assert torch.equal(eng.get_state("G").cpu(), G)
+    eng.set_state("step", 41)
+    eng.step(1)
+    assert eng.get_state("step") == 42
+    with pytest.raises(pkg.AdacgdError):
+        eng.set_state("x", torch.zeros(99))
+    with pytest.raises(pkg.AdacgdError):
+        pkg.AdaCGD(2, 100, [(TOPK, 5)], 1.0, loss=0, lam=0.1, A=torch.zeros(2, 10, 100, device="cuda"),
+                   target=torch.zeros(2, 10, device="cuda"), x0=torch.zeros(100, device="cuda"), gamma=-1.0)
