@@ -196,6 +196,17 @@ void adacgd_destroy(adacgd_ctx* ctx);
 /* Number of kernels this library has launched on behalf of ctx since init. */
 int64_t adacgd_launch_count(const adacgd_ctx* ctx);
 
+/* Per-kernel timing with CUDA events recorded on the context's stream around every
+ * launch (measurement aid; the paper has no counterpart).  adacgd_profile_enable
+ * reserves max_records event pairs (<= 0 switches timing off); records beyond that are
+ * dropped.  adacgd_profile_read synchronises the stream, writes for every kernel id in
+ * [0, adacgd_profile_kernel_count()) the summed device time in milliseconds and the
+ * number of timed launches, and clears the records. */
+int32_t adacgd_profile_kernel_count(void);
+const char* adacgd_profile_kernel_name(int32_t id);
+adacgd_status adacgd_profile_enable(adacgd_ctx* ctx, int32_t max_records);
+adacgd_status adacgd_profile_read(adacgd_ctx* ctx, double* ms_out, int64_t* records_out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,7 +18,8 @@ STATUS = {0: "OK", 1: "INVALID_ARG", 2: "BAD_ORDER", 3: "NONFINITE", 4: "WORKSPA
 EXPORTED_SYMBOLS = [
     "adacgd_workspace_bytes", "adacgd_init", "adacgd_step", "adacgd_compress", "adacgd_compress_host",
     "adacgd_gradient", "adacgd_get_state", "adacgd_set_state", "adacgd_last_error", "adacgd_destroy",
-    "adacgd_launch_count",
+    "adacgd_launch_count", "adacgd_profile_kernel_count", "adacgd_profile_kernel_name", "adacgd_profile_enable",
+    "adacgd_profile_read",
 ]
 
 Cand = Tuple[int, int]
@@ -82,8 +83,14 @@ def load_library():
     lib.adacgd_destroy.restype = None
     lib.adacgd_launch_count.argtypes = [vp]
     lib.adacgd_launch_count.restype = i64
+    lib.adacgd_profile_kernel_count.argtypes = []
+    lib.adacgd_profile_kernel_name.argtypes = [i32]
+    lib.adacgd_profile_kernel_name.restype = C.c_char_p
+    lib.adacgd_profile_enable.argtypes = [vp, i32]
+    lib.adacgd_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     for name in EXPORTED_SYMBOLS:
-        if name not in ("adacgd_last_error", "adacgd_destroy", "adacgd_launch_count"):
+        if name not in ("adacgd_last_error", "adacgd_destroy", "adacgd_launch_count",
+                        "adacgd_profile_kernel_name"):
             getattr(lib, name).restype = i32
     _LIB = lib
     return lib
@@ -222,6 +229,17 @@ class AdaCGD:
         else:
             buf = C.c_uint64(int(value))
             self._check(self.lib.adacgd_set_state(self.ctx, STATE[which], C.byref(buf), 8, 0), self.ctx)
+
+    def profile_enable(self, max_records: int):
+        self._check(self.lib.adacgd_profile_enable(self.ctx, int(max_records)), self.ctx)
+
+    def profile_read(self):
+        """Returns {kernel name: (total ms, timed launches)} and clears the records."""
+        k = self.lib.adacgd_profile_kernel_count()
+        ms = (C.c_double * k)()
+        cnt = (C.c_int64 * k)()
+        self._check(self.lib.adacgd_profile_read(self.ctx, ms, cnt), self.ctx)
+        return {self.lib.adacgd_profile_kernel_name(i).decode(): (ms[i], int(cnt[i])) for i in range(k) if cnt[i]}
 
     def launch_count(self) -> int:
         return int(self.lib.adacgd_launch_count(self.ctx))

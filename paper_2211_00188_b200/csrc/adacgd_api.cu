@@ -141,6 +141,10 @@ struct adacgd_ctx {
   int* loglevels;
   float* stage;
   long long launches;
+  Prof* prof;
+  Prof prof_store;
+  std::vector<cudaEvent_t> ev_beg, ev_end;
+  std::vector<int> ev_id;
   std::string err;
 };
 
@@ -216,6 +220,7 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   c->flags = flags;
   c->stream = (cudaStream_t)cuda_stream;
   c->launches = 0;
+  c->prof = nullptr;
   const bool has_loss = problem->loss != ADACGD_LOSS_NONE;
   if (has_loss && (!x0_dev || !(gamma > 0.f) || g0_mode < 0 || g0_mode > 2)) {
     delete c;
@@ -390,7 +395,7 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
     const int batch = (n_steps - done < LOG_CAP) ? (n_steps - done) : LOG_CAP;
     for (int t = 0; t < batch; ++t) {
       // a0: x^{t+1} = x^t - gamma g^t
-      int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream);
+      int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream, c->prof);
       if (r < 0) return cuda_fail(c, "x update");
       c->launches += r;
       // a1: X_i = grad f_i(x^{t+1})
@@ -412,8 +417,10 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
       float* t2 = c->grad_cur;
       c->grad_cur = c->grad_nxt;
       c->grad_nxt = t2;
+      prof_begin(c->prof, KID_LOG, c->stream);
       k_log_step<<<1, 256, 0, c->stream>>>(n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
                                            c->counters, c->log, c->loglevels, t);
+      prof_end(c->prof, c->stream);
       c->launches += 1;
     }
     if (report_host || levels_host) {
@@ -496,7 +503,65 @@ adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, si
 
 const char* adacgd_last_error(const adacgd_ctx* ctx) { return ctx ? ctx->err.c_str() : g_err.c_str(); }
 
-void adacgd_destroy(adacgd_ctx* ctx) { delete ctx; }
+void adacgd_destroy(adacgd_ctx* ctx) {
+  if (!ctx) return;
+  for (cudaEvent_t e : ctx->ev_beg) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->ev_end) cudaEventDestroy(e);
+  delete ctx;
+}
+
+static const char* const kKernelNames[KID_COUNT] = {
+    "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
+    "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
+    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step"};
+
+int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
+
+const char* adacgd_profile_kernel_name(int32_t id) { return (id >= 0 && id < KID_COUNT) ? kKernelNames[id] : ""; }
+
+adacgd_status adacgd_profile_enable(adacgd_ctx* c, int32_t max_records) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (max_records <= 0) {
+    c->prof = nullptr;
+    c->scr.prof = nullptr;
+    c->gs.prof = nullptr;
+    return ADACGD_OK;
+  }
+  while ((int)c->ev_beg.size() < max_records) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess)
+      return cuda_fail(c, "adacgd_profile_enable");
+    c->ev_beg.push_back(a);
+    c->ev_end.push_back(b);
+  }
+  c->ev_id.assign(c->ev_beg.size(), 0);
+  c->prof_store.cap = max_records;
+  c->prof_store.used = 0;
+  c->prof_store.beg = c->ev_beg.data();
+  c->prof_store.end = c->ev_end.data();
+  c->prof_store.id = c->ev_id.data();
+  c->prof = &c->prof_store;
+  c->scr.prof = c->prof;
+  c->gs.prof = c->prof;
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_profile_read(adacgd_ctx* c, double* ms_out, int64_t* records_out) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!ms_out || !records_out) return fail(c, ADACGD_ERR_INVALID_ARG, "output arrays must be non-NULL");
+  for (int i = 0; i < KID_COUNT; ++i) { ms_out[i] = 0.0; records_out[i] = 0; }
+  if (!c->prof) return ADACGD_OK;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_profile_read");
+  for (int i = 0; i < c->prof->used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof->beg[i], c->prof->end[i]) != cudaSuccess)
+      return cuda_fail(c, "adacgd_profile_read");
+    ms_out[c->prof->id[i]] += (double)ms;
+    records_out[c->prof->id[i]] += 1;
+  }
+  c->prof->used = 0;
+  return ADACGD_OK;
+}
 
 int64_t adacgd_launch_count(const adacgd_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

@@ -779,6 +779,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d) {
   s->rows_cap = rows;
   s->d_cap = d;
   s->nchunk_cap = nchunk_of(d);
+  s->prof = nullptr;
 }
 
 adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const char** msg) {
@@ -830,15 +831,29 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                   (!out.mean_out || aligned16(out.mean_out));
   const long long nchunk = nchunk_of(d);
   const dim3 ugrid((unsigned)nchunk);
-  if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
+  Prof* pf = s.prof;
+#define TIMED(id, ...)             \
+  do {                             \
+    prof_begin(pf, id, stream);    \
+    __VA_ARGS__;                   \
+    prof_end(pf, stream);          \
+    ++launches;                    \
+  } while (0)
+#define TIMED_AL(id, kern, grid, shm, ...)                                  \
+  TIMED(id, if (al) kern<true><<<grid, TPB, shm, stream>>>(__VA_ARGS__);    \
+            else kern<false><<<grid, TPB, shm, stream>>>(__VA_ARGS__))
+
   if (cs.m == 0) {
-    k_copy_report<<<(rows + 127) / 128, 128, 0, stream>>>(rows, d, 0, out);
-    if (al) k_update<true><<<ugrid, TPB, 0, stream>>>(X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
-    else k_update<false><<<ugrid, TPB, 0, stream>>>(X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
-    launches += 2;
+    prof_begin(pf, KID_MEMSET, stream);
+    if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
+    prof_end(pf, stream);
+    TIMED(KID_PICK, (k_copy_report<<<(rows + 127) / 128, 128, 0, stream>>>(rows, d, 0, out)));
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
-  // zero the per-call accumulators; the tail of the region depends on rows_cap, so clear by piece
+  // clear the per-call accumulators
+  prof_begin(pf, KID_MEMSET, stream);
+  if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
   cudaMemsetAsync(s.hist1, 0, (size_t)rows * BINS1 * 4, stream);
   if (cs.nsel) {
     cudaMemsetAsync(s.hist2, 0, (size_t)rows * MAXC * BINS2 * 4, stream);
@@ -846,6 +861,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   }
   cudaMemsetAsync(s.maxkey, 0, (size_t)rows * 4, stream);
   cudaMemsetAsync(s.limbs, 0, (size_t)rows * NSLOT * NLIMB * 8, stream);
+  prof_end(pf, stream);
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
   long long want = (148 * 8 + rows - 1) / rows;
@@ -855,44 +871,31 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const int nblk = (int)want;
   const dim3 sgrid(nblk, rows);
 
-#define LAUNCH_AL(kern, grid, shm, ...)                                          \
-  do {                                                                           \
-    if (al) kern<true><<<grid, TPB, shm, stream>>>(__VA_ARGS__);                 \
-    else kern<false><<<grid, TPB, shm, stream>>>(__VA_ARGS__);                   \
-    ++launches;                                                                  \
-  } while (0)
-#define LAUNCH_HIST(PASS, shm, hist)                                                              \
-  do {                                                                                            \
-    if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr);  \
-    else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr);    \
-    ++launches;                                                                                   \
-  } while (0)
+#define TIMED_HIST(id, PASS, shm, hist)                                                                              \
+  TIMED(id, if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr); \
+            else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr))
 
-  if (cs.nsel || cs.nquant) {
-    LAUNCH_HIST(1, BINS1 * 4, s.hist1);
-  }
+  if (cs.nsel || cs.nquant) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
   if (cs.nsel) {
-    k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, nullptr);
-    LAUNCH_HIST(2, cs.nsel * BINS2 * 4, s.hist2);
-    k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, nullptr);
-    LAUNCH_HIST(3, cs.nsel * BINS3 * 4, s.hist3);
-    k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, nullptr);
-    launches += 3;
+    TIMED(KID_SCAN, (k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, nullptr)));
+    TIMED_HIST(KID_HIST2, 2, cs.nsel * BINS2 * 4, s.hist2);
+    TIMED(KID_SCAN, (k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, nullptr)));
+    TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
+    TIMED(KID_SCAN, (k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, nullptr)));
   }
-  LAUNCH_AL(k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial);
-  if (cs.nquant) LAUNCH_AL(k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
-  k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out);
-  LAUNCH_AL(k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs);
-  k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out);
-  launches += 2;
+  TIMED_AL(KID_ENERGY, k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial);
+  if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
+  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out)));
+  TIMED_AL(KID_EXACT, k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs);
+  TIMED(KID_EXACT, (k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out)));
   if (cs.nsel) {
-    LAUNCH_AL(k_tiecount, dim3((unsigned)nchunk, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
-    k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk);
-    ++launches;
+    TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)nchunk, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
+    TIMED(KID_TIE, (k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk)));
   }
-  LAUNCH_AL(k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
-#undef LAUNCH_AL
-#undef LAUNCH_HIST
+  TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+#undef TIMED_HIST
+#undef TIMED_AL
+#undef TIMED
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
@@ -903,8 +906,10 @@ __global__ void k_axpy(float* __restrict__ x, const float* __restrict__ g, float
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));
 }
-int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream) {
+int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof) {
+  prof_begin(prof, KID_AXPY, stream);
   k_axpy<<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(x, g, gamma, d);
+  prof_end(prof, stream);
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -237,6 +237,7 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p) {
   if (g->split > 1) { g->part = (float*)(b + o); o = align_up(o + (size_t)g->split * p.n * p.d * 4, 256); }
   g->losspart = (double*)(b + o); o = align_up(o + (size_t)p.n * g->loss_blocks * 8, 256);
   g->loss = (double*)(b + o);
+  g->prof = nullptr;
 }
 
 int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
@@ -244,6 +245,7 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
   if (p.layout != ADACGD_LAYOUT_DENSE) return -2;
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
+  prof_begin(g.prof, KID_GRAD_FWD, stream);
   if (cta_row_mode(p)) {
     const dim3 grid((unsigned)p.m_rows, p.n);
     if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
@@ -253,16 +255,23 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
     if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
     else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
   }
+  prof_end(g.prof, stream);
   ++launches;
   const dim3 bgrid((unsigned)((p.d + TPB * 4 - 1) / (TPB * 4)), p.n * g.split);
+  prof_begin(g.prof, KID_GRAD_BWD, stream);
   if (al) k_dense_bwd<true><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n);
   else k_dense_bwd<false><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n);
+  prof_end(g.prof, stream);
   ++launches;
   if (g.split > 1) {
+    prof_begin(g.prof, KID_GRAD_REDUCE, stream);
     k_grad_reduce<<<dim3((unsigned)((p.d + 255) / 256), p.n), 256, 0, stream>>>(g.part, x, p.d, p.n, g.split, p.loss, p.lambda, grads);
+    prof_end(g.prof, stream);
     ++launches;
   }
+  prof_begin(g.prof, KID_LOSS, stream);
   k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, g.loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+  prof_end(g.prof, stream);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

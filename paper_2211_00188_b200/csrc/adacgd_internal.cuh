@@ -21,6 +21,25 @@ constexpr int BINS3 = 512;          // key bits [8:0]
 constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (also the tie-order chunk)
 constexpr int MAX_BLK_PER_ROW = 2048;
 
+// Optional per-kernel timing with CUDA events on the launching stream.
+enum KernelId {
+  KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
+  KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
+  KID_LOG, KID_COUNT
+};
+struct Prof {
+  int cap, used;
+  cudaEvent_t* beg;
+  cudaEvent_t* end;
+  int* id;
+};
+inline void prof_begin(Prof* p, int id, cudaStream_t s) {
+  if (p && p->used < p->cap) { p->id[p->used] = id; cudaEventRecord(p->beg[p->used], s); }
+}
+inline void prof_end(Prof* p, cudaStream_t s) {
+  if (p && p->used < p->cap) { cudaEventRecord(p->end[p->used], s); ++p->used; }
+}
+
 // Candidate set as the kernels see it (passed by value).
 struct CsetDev {
   int m;                 // candidates
@@ -69,6 +88,7 @@ struct Scratch {
   double* energy;  // [rows][NSLOT]
   u32* tiecnt;     // [rows][nchunk]  (exclusive prefix after the scan)
   int rows_cap; long long d_cap; long long nchunk_cap;
+  Prof* prof;      // host pointer, may be null
 };
 
 size_t scratch_bytes(int rows, long long d);
@@ -93,6 +113,7 @@ struct GradScratch {
   double* losspart; // [n][loss_blocks]
   double* loss;     // [1]
   int split; int loss_blocks;
+  Prof* prof;
 };
 size_t grad_scratch_bytes(const adacgd_problem& p);
 void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p);
@@ -100,7 +121,7 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
                     cudaStream_t stream);
 
 // x <- x - gamma * g  (two binary32 roundings: the product, then the difference)
-int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream);
+int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof);
 int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStream_t stream);
 
 }  // namespace adacgd
