@@ -163,6 +163,36 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
                                    const adacgd_cset* cset, float* mean_out_host,
                                    int32_t* level_host, uint64_t* bits_host);
 
+/* adacgd_compress for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of the same kernels).  Meant for code that is
+ * only ever handed buffers: a plug-in inside a host application whose own allocator has
+ * claimed the whole device, so that cudaMalloc would fail; a control loop that cannot
+ * afford the device-wide synchronisation an allocation implies; a component running
+ * under a policy that forbids it to grow the process's device footprint.  There is no
+ * context and no workspace: the histograms, accumulators and per-row records live in a
+ * 2 MiB array that is compiled into the library, so every GPU that loads the library
+ * holds those 2 MiB until the process exits.  The call itself allocates nothing on the
+ * host or the device and frees nothing.
+ *   Limits: rows <= ADACGD_NOALLOC_MAX_ROWS, d <= ADACGD_NOALLOC_MAX_D; larger shapes
+ *   return ADACGD_ERR_INVALID_ARG (message via adacgd_last_error(NULL)).
+ *   X_dev, G_dev, Y_dev, cset, mean_out_dev, level_dev, bits_dev: as in adacgd_compress
+ *   (the last three may be NULL); results are identical to adacgd_compress.
+ *   cuda_stream: the cudaStream_t the work is enqueued on (NULL = default stream); the
+ *   call does not synchronise.
+ *   The first call on each device looks up the array's device address, with the current
+ *   device being the one that owns the buffers; make that first call before any stream
+ *   capture is started.
+ *   All calls on a device share the one array and it keeps the previous call's
+ *   contents (the call clears what has to start from zero).  Two calls whose kernels can
+ *   overlap on the GPU -- different streams without an ordering between them, or two
+ *   host threads -- race on it and give wrong results: serialise them. */
+#define ADACGD_NOALLOC_MAX_ROWS 4
+#define ADACGD_NOALLOC_MAX_D 4194304
+adacgd_status adacgd_compress_noalloc(const float* X_dev, float* G_dev, const float* Y_dev,
+                                      int32_t rows, int64_t d, const adacgd_cset* cset,
+                                      float* mean_out_dev, int32_t* level_dev, uint64_t* bits_dev,
+                                      void* cuda_stream);
+
 /* Stage a1 alone: grads_out_dev [n][d] = grad f_i(x_dev); loss_out_host (may be NULL,
  * synchronises) = (1/n) sum_i f_i(x). */
 adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_out_dev,

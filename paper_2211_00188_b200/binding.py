@@ -19,7 +19,7 @@ EXPORTED_SYMBOLS = [
     "adacgd_workspace_bytes", "adacgd_init", "adacgd_step", "adacgd_compress", "adacgd_compress_host",
     "adacgd_gradient", "adacgd_get_state", "adacgd_set_state", "adacgd_last_error", "adacgd_destroy",
     "adacgd_launch_count", "adacgd_profile_kernel_count", "adacgd_profile_kernel_name", "adacgd_profile_enable",
-    "adacgd_profile_read",
+    "adacgd_profile_read", "adacgd_compress_noalloc",
 ]
 
 Cand = Tuple[int, int]
@@ -83,6 +83,7 @@ def load_library():
     lib.adacgd_destroy.restype = None
     lib.adacgd_launch_count.argtypes = [vp]
     lib.adacgd_launch_count.restype = i64
+    lib.adacgd_compress_noalloc.argtypes = [vp, vp, vp, i32, i64, C.POINTER(_Cset), vp, vp, vp, vp]
     lib.adacgd_profile_kernel_count.argtypes = []
     lib.adacgd_profile_kernel_name.argtypes = [i32]
     lib.adacgd_profile_kernel_name.restype = C.c_char_p
@@ -243,3 +244,27 @@ class AdaCGD:
 
     def launch_count(self) -> int:
         return int(self.lib.adacgd_launch_count(self.ctx))
+
+
+NOALLOC_MAX_ROWS = 4
+NOALLOC_MAX_D = 4194304
+
+
+def compress_noalloc(X, G, Y, cands: Sequence[Cand], zeta: float, *, mean_out=None, level=None, bits=None,
+                     stream=None):
+    """adacgd_compress_noalloc on device tensors: the same result as AdaCGD.compress for
+    callers that may not allocate device memory.  Needs no context and no workspace (the
+    library's built-in 2 MiB scratch is used), accepts at most NOALLOC_MAX_ROWS rows of at
+    most NOALLOC_MAX_D columns, enqueues on `stream` (default: torch's current stream) and
+    must not run concurrently with another call on the same GPU."""
+    import torch
+
+    lib = load_library()
+    rows, d = X.shape
+    cs, keep = _cset(cands, zeta)
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    with torch.cuda.device(X.device):
+        status = lib.adacgd_compress_noalloc(_ptr(X), _ptr(G), _ptr(Y), rows, d, C.byref(cs), _ptr(mean_out),
+                                             _ptr(level), _ptr(bits), C.c_void_p(st.cuda_stream))
+    if status != 0:
+        raise AdacgdError(status, lib.adacgd_last_error(None).decode())

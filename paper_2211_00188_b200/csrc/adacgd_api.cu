@@ -122,6 +122,10 @@ __global__ void k_set_master_identity(int* mlevel, unsigned long long* mbits, lo
 
 }  // namespace
 
+namespace adacgd {
+void set_thread_error(const char* msg) { g_err = msg ? msg : ""; }
+}  // namespace adacgd
+
 struct adacgd_ctx {
   adacgd_problem p;
   CsetDev wcs, mcs;

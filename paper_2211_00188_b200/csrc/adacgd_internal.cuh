@@ -124,4 +124,7 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
 int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof);
 int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStream_t stream);
 
+// Stores the message that adacgd_last_error(NULL) returns on this thread.
+void set_thread_error(const char* msg);
+
 }  // namespace adacgd
