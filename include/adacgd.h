@@ -143,7 +143,8 @@ adacgd_status adacgd_step(adacgd_ctx* ctx, int32_t n_steps, adacgd_step_report* 
  *   cset: host; m = 0 copies X into G.  rows*d must fit the shape given at init.
  *   Outputs, all dev, each may be NULL:
  *     level_dev int32[rows]; bits_dev uint64[rows]; err_dev double[rows][m+1] (||v||^2 then
- *     one value per candidate); D_dev double[rows];
+ *     one value per candidate); D_dev double[rows]; these two are diagnostics accurate to a
+ *     relative 4e-6 (the level choice itself is exact);
  *     kept_idx_dev int32[rows][kept_stride]: indices written by a Top-K level, in no
  *     particular order, kept_cnt_dev int64[rows] their number (0 for other levels).
  * Returns ADACGD_ERR_NONFINITE only from the _host variant and from adacgd_step (the
@@ -211,6 +212,8 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
 #define ADACGD_STATE_LEVELS 8   /* last step      int32 [n] */
 #define ADACGD_STATE_FLAGS 9    /* uint32: bit 0 = a non-finite input was seen since init (get only) */
 #define ADACGD_STATE_RECHECKS 10/* uint32: trigger comparisons redone in exact arithmetic since init (get only) */
+#define ADACGD_STATE_FALLBACKS 11/* uint32: rows whose sampled threshold bracket failed and that took the full
+                                   three-pass radix select instead, since init (get only) */
 adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,
                                int32_t dst_is_device);
 adacgd_status adacgd_set_state(adacgd_ctx* ctx, int32_t which, const void* src, size_t bytes,

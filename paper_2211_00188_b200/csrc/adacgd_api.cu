@@ -38,7 +38,7 @@ WsLayout ws_layout(const adacgd_problem& p, bool master_compresses, int flags) {
   WsLayout L;
   size_t o = 0;
   const size_t nd = (size_t)p.n * (size_t)p.d * 4, dd = (size_t)p.d * 4;
-  L.scratch = o; o = align_up(o + scratch_bytes(p.n, p.d), 256);
+  L.scratch = o; o = align_up(o + scratch_bytes(p.n, p.d, true), 256);
   L.grad = o; o = align_up(o + grad_scratch_bytes(p), 256);
   L.levels = o; o = align_up(o + (size_t)p.n * 4, 256);
   L.bits = o; o = align_up(o + (size_t)p.n * 8, 256);
@@ -244,7 +244,7 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
     return fail(nullptr, ADACGD_ERR_WORKSPACE, "workspace smaller than adacgd_workspace_bytes reports");
   }
   char* b = (char*)workspace_dev;
-  carve_scratch(&c->scr, b + L.scratch, problem->n, problem->d);
+  carve_scratch(&c->scr, b + L.scratch, problem->n, problem->d, true);
   c->levels = (int*)(b + L.levels);
   c->bits = (unsigned long long*)(b + L.bits);
   c->mlevel = (int*)(b + L.mlevel);
@@ -471,6 +471,7 @@ static adacgd_status state_ptr(adacgd_ctx* c, int32_t which, void** p, size_t* b
     case ADACGD_STATE_LEVELS: *p = c->levels; *bytes = (size_t)c->p.n * 4; return ADACGD_OK;
     case ADACGD_STATE_FLAGS: *p = c->scr.flags; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_RECHECKS: *p = c->scr.flags + 1; *bytes = 4; return ADACGD_OK;
+    case ADACGD_STATE_FALLBACKS: *p = c->scr.flags + 2; *bytes = 4; return ADACGD_OK;
     default: return fail(c, ADACGD_ERR_INVALID_ARG, "unknown state item");
   }
   if (!has) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective, hence no iterate state");
@@ -493,7 +494,8 @@ adacgd_status adacgd_get_state(adacgd_ctx* c, int32_t which, void* dst, size_t b
 adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, size_t bytes, int32_t src_is_device) {
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (!src) return fail(c, ADACGD_ERR_INVALID_ARG, "src is NULL");
-  if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS)
+  if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS ||
+      which == ADACGD_STATE_FALLBACKS)
     return fail(c, ADACGD_ERR_INVALID_ARG, "this item is read-only");
   void* p;
   size_t want;
@@ -517,7 +519,7 @@ void adacgd_destroy(adacgd_ctx* ctx) {
 static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
-    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step"};
+    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lscan"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
 

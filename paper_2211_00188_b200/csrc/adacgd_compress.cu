@@ -118,10 +118,10 @@ template <int PASS, bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const float* __restrict__ G,
                                               long long d, int nsel, const SelRow* __restrict__ sel,
                                               u32* __restrict__ hist, u32* __restrict__ maxkey,
-                                              const RowDec* __restrict__ only_flagged) {
+                                              const u32* __restrict__ rowflag) {
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
-  if (only_flagged && !only_flagged[row].need_exact) return;
+  if (rowflag && !rowflag[row]) return;  // single-pass mode: only rows whose bracket failed
   constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
   const int ntab = (PASS == 1) ? 1 : nsel;
   for (int i = threadIdx.x; i < ntab * NB; i += TPB) sh[i] = 0;
@@ -174,10 +174,11 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
 
 template <int PASS>
 __global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict__ hist, SelRow* __restrict__ sel,
-                                              const RowDec* __restrict__ only_flagged) {
+                                              const u32* __restrict__ rowflag, u32* __restrict__ flags) {
   __shared__ u32 res[2];
   const int row = blockIdx.x;
-  if (only_flagged && !only_flagged[row].need_exact) return;
+  if (rowflag && !rowflag[row]) return;
+  if (PASS == 1 && rowflag && threadIdx.x == 0) atomicAdd(&flags[2], 1u);  // rows sent through the full select
   constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
   SelRow* s = sel + row;
   for (int j = 0; j < cs.nsel; ++j) {
@@ -197,6 +198,7 @@ __global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict_
         s->above[j] = before + res[1];
         s->ntie[j] = h[res[0]];
         s->q[j] = K - (before + res[1]);
+        s->extraE[j] = 0.0;
       }
     }
     __syncthreads();
@@ -211,12 +213,15 @@ __global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict_
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, const float* __restrict__ G,
                                                 const float* __restrict__ Y, long long d, CsetDev cs,
-                                                const SelRow* __restrict__ sel, double* __restrict__ partial) {
+                                                const SelRow* __restrict__ sel, double* __restrict__ partial,
+                                                const u32* __restrict__ rowflag, u32* __restrict__ diffflag) {
   const int row = blockIdx.y;
+  if (rowflag && !rowflag[row]) return;
   u32 T[MAXC];
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) T[j] = (j < cs.nsel) ? sel[row].T[j] : 0u;
   double aD = 0, aE = 0, aB[MAXC];
+  u32 mxw = 0;
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) aB[j] = 0;
   const float* xr = X + (long long)row * d;
@@ -236,6 +241,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
       const float v = __fsub_rn(x[k], g[k]);
       const float w = __fsub_rn(x[k], y[k]);
       const double dv = (double)v, dw = (double)w;
+      mxw = max(mxw, key_of(w));
       const double sq = __dmul_rn(dv, dv);
       aD = __dadd_rn(aD, __dmul_rn(dw, dw));
       aE = __dadd_rn(aE, sq);
@@ -245,6 +251,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
         if (j < cs.nsel && key < T[j]) aB[j] = __dadd_rn(aB[j], sq);
     }
   }
+  if (mxw >= 0x7f800000u) atomicOr(&diffflag[row], 0x80000000u);
   __shared__ double red[NSLOT][TPB / 32];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   double v0 = warp_sum_f64(aD), v1 = warp_sum_f64(aE);
@@ -382,7 +389,8 @@ __device__ void finalize_row(const CsetDev& cs, int row, int level, long long d,
 
 __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk, const double* __restrict__ partial,
                                              const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                                             RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out) {
+                                             RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
+                                             const u32* __restrict__ diffflag, int single_pass, double tol) {
   const int row = blockIdx.x, lane = threadIdx.x;
   double sum[NSLOT];
 #pragma unroll
@@ -402,28 +410,35 @@ __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk, 
       int j = 0;
       for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
       const double tv = (double)__uint_as_float(sel[row].T[j]);
-      e[c + 1] = sum[2 + c] + (double)(sel[row].ntie[j] - sel[row].q[j]) * (tv * tv);
+      e[c + 1] = (sum[2 + c] + sel[row].extraE[j]) + (double)(sel[row].ntie[j] - sel[row].q[j]) * (tv * tv);
     } else {
       e[c + 1] = sum[2 + c];
     }
   }
-  bool finite = (D <= 1.7e308) && (e[0] <= 1.7e308) && (maxkey[row] < 0x7f800000u);
-  if (!finite) {
+  if (maxkey[row] >= 0x7f800000u || (diffflag[row] & 0x80000000u)) {  // Inf/NaN in X - G or X - Y: estimator kept
     atomicOr(&flags[0], 1u);
     finalize_row(cs, row, 0, d, sel, maxkey, dec, out, e, D);
     return;
   }
-  // worst-case relative error of a binary64 sum of <= d non-negative exact terms, any order,
-  // plus the few roundings of the tie term and of zeta*D on either side
-  const double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;
+  // `tol` bounds the relative error of every sum above (non-negative terms).  A sum is only
+  // trusted inside [2^-90, inf): below, binary32 squares may have underflowed; above, a chain
+  // overflowed (or X - Y is not finite, which the exact pass reports).
+  const double tiny = 8.0e-28;
   const double rhs = (double)cs.zeta * D;
+  const bool d_ok = (D >= tiny && D <= 1.7e308);
   int level = cs.m;
   bool unsure = false;
   for (int j = 0; j <= cs.m; ++j) {
     const double E = e[j];
+    const bool by_def = (j > 0 && cs.kind[j - 1] == ADACGD_TOPK && cs.param[j - 1] >= d);  // identity: error 0
+    const bool e_ok = (E >= tiny && E <= 1.7e308);
     int verdict;  // 1 true, 0 false, -1 unsure
-    if (E == 0.0) verdict = 1;
-    else if (rhs == 0.0) verdict = 0;
+    if (by_def) verdict = 1;
+    else if (j == 0 && single_pass && (diffflag[row] & 0x7fffffffu) == 0 && d_ok)
+      verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
+    else if (!e_ok) verdict = -1;
+    else if (cs.zeta == 0.f) verdict = 0;  // E > 0 for certain, right side is 0
+    else if (!d_ok) verdict = -1;
     else if (E * (1.0 + tol) < rhs * (1.0 - tol)) verdict = 1;
     else if (E * (1.0 - tol) > rhs * (1.0 + tol)) verdict = 0;
     else verdict = -1;
@@ -465,7 +480,8 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X, const float* __restrict__ G,
                                                     const float* __restrict__ Y, long long d, CsetDev cs,
                                                     const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                                                    const RowDec* __restrict__ dec, u64* __restrict__ limbs) {
+                                                    const RowDec* __restrict__ dec, u64* __restrict__ limbs,
+                                                    u32* __restrict__ diffflag) {
   const int row = blockIdx.y;
   if (!dec[row].need_exact) return;
   __shared__ u64 sh[NSLOT * NLIMB];
@@ -487,6 +503,7 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
       if (!ALIGNED && c0 + k >= d) break;
       const float v = __fsub_rn(x[k], g[k]);
       int kk; u32 p[3];
+      if (key_of(__fsub_rn(x[k], y[k])) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
       sq_pieces(__fsub_rn(x[k], y[k]), &kk, p);
       limb_add(sh + 0 * NLIMB, kk, p);
       sq_pieces(v, &kk, p);
@@ -534,10 +551,17 @@ __device__ double digits_to_double(const u32* dig) {
 }
 
 __global__ void k_pick_exact(CsetDev cs, long long d, const u64* __restrict__ limbs, const SelRow* __restrict__ sel,
-                             const u32* __restrict__ maxkey, RowDec* __restrict__ dec, CompressOut out) {
+                             const u32* __restrict__ maxkey, RowDec* __restrict__ dec, CompressOut out,
+                             const u32* __restrict__ diffflag, u32* __restrict__ flags) {
   const int row = blockIdx.x;
   if (threadIdx.x != 0 || !dec[row].need_exact) return;
   double val[NSLOT];
+  if (diffflag[row] & 0x80000000u) {  // X - Y is not finite
+    for (int s = 0; s < NSLOT; ++s) val[s] = 0.0;
+    atomicOr(&flags[0], 1u);
+    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, val + 1, 0.0);
+    return;
+  }
   for (int s = 0; s < 2 + cs.m; ++s) {
     u32 dig[NLIMB];
     const u64* l = limbs + ((long long)row * NSLOT + s) * NLIMB;
@@ -729,6 +753,367 @@ __global__ void k_copy_report(int rows, long long d, int m, CompressOut out) {
 }
 
 // --------------------------------------------------------------------------
+// single-pass path: brackets from a sample, one streaming pass, selection on short lists
+// --------------------------------------------------------------------------
+// Every `stride`-th tile of a row is sampled; the histogram has one bin per value of
+// key[30:15].  Per-CTA counts are 16 bit (two bins per shared word), so a CTA takes at most
+// 63 tiles.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
+                                                long long d, long long nsamp, long long stride,
+                                                u32* __restrict__ shist) {
+  extern __shared__ u32 sh[];  // SBINS / 2 words
+  const int row = blockIdx.y;
+  for (int i = threadIdx.x; i < SBINS / 2; i += TPB) sh[i] = 0;
+  __syncthreads();
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  for (long long sidx = blockIdx.x; sidx < nsamp; sidx += gridDim.x) {
+    const long long t = sidx * stride + (stride >> 1);
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    if (c0 >= d) continue;
+    float x[4], g[4];
+    load4<ALIGNED>(xr, c0, d, x);
+    load4<ALIGNED>(gr, c0, d, g);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (!ALIGNED && c0 + k >= d) break;
+      const u32 bin = key_of(__fsub_rn(x[k], g[k])) >> 15;
+      atomicAdd(&sh[bin >> 1], (bin & 1u) ? 0x10000u : 1u);
+    }
+  }
+  __syncthreads();
+  u32* gh = shist + (long long)row * SBINS;
+  for (int i = threadIdx.x; i < SBINS / 2; i += TPB) {
+    const u32 w = sh[i];
+    if (w & 0xffffu) atomicAdd(&gh[2 * i], w & 0xffffu);
+    if (w >> 16) atomicAdd(&gh[2 * i + 1], w >> 16);
+  }
+}
+
+// Finds the bin holding the r-th largest sampled key (1-based); all TPB threads call.
+// `excl`/`sum` are this thread's exclusive prefix and count over its 256 bins (descending order).
+__device__ void sample_rank_bin(const u32* __restrict__ h, u32 excl, u32 sum, u32 r, u32* out) {
+  if (r > excl && r <= excl + sum) {
+    u32 run = excl;
+    for (int k = 0; k < SBINS / TPB; ++k) {
+      const int bin = SBINS - 1 - (threadIdx.x * (SBINS / TPB) + k);
+      const u32 c = h[bin];
+      if (r <= run + c) { *out = (u32)bin; break; }
+      run += c;
+    }
+  }
+  __syncthreads();
+}
+
+// Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
+// holds the K-th largest key with overwhelming probability (checked exactly afterwards).
+__global__ void __launch_bounds__(TPB) k_bracket(CsetDev cs, long long d, int full_sample,
+                                                 const u32* __restrict__ shist, SelRow* __restrict__ sel) {
+  __shared__ u32 res;
+  const int row = blockIdx.x;
+  const u32* h = shist + (long long)row * SBINS;
+  u32 sum = 0;
+  for (int k = 0; k < SBINS / TPB; ++k) sum += h[SBINS - 1 - (threadIdx.x * (SBINS / TPB) + k)];
+  u32 S;
+  const u32 excl = block_excl_scan(sum, &S);
+  for (int j = 0; j < cs.nsel; ++j) {
+    const double K = (double)cs.param[cs.sel[j]];
+    const double r = K * (double)S / (double)d;
+    const double dev = full_sample ? 0.0 : 6.0 * sqrt(r * (1.0 - K / (double)d)) + 8.0;
+    const double r_hi = floor(r - dev), r_lo = ceil(r + dev) + 1.0;
+    u32 hi = 0x80000000u, lo = 0u;
+    if (r_hi >= 1.0) {
+      sample_rank_bin(h, excl, sum, (u32)r_hi, &res);
+      hi = (res + 1u) << 15;
+      __syncthreads();
+    }
+    if (r_lo <= (double)S) {
+      sample_rank_bin(h, excl, sum, (u32)r_lo, &res);
+      lo = res << 15;
+    }
+    if (threadIdx.x == 0) { sel[row].lo[j] = lo; sel[row].hi[j] = hi; }
+    __syncthreads();
+  }
+}
+
+// The streaming pass: D, ||v||^2, per bracket the count of keys >= hi and the energy of keys
+// < lo, the row maximum, and the keys inside a bracket appended to this CTA's list segment.
+// Sums run in binary32 chains of at most 4*FLUSH_TILES fused multiply-adds (relative error
+// <= (4*FLUSH_TILES + 1) 2^-24 for non-negative terms), folded into binary64.
+template <int NSEL, bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
+                                               const float* __restrict__ Y, long long d, CsetDev cs,
+                                               const SelRow* __restrict__ sel, double* __restrict__ partial,
+                                               u32* __restrict__ cntpart, u64* __restrict__ list,
+                                               u32* __restrict__ lcount, long long list_row, u32 segcap,
+                                               u32* __restrict__ maxkey, u32* __restrict__ rowflag,
+                                               u32* __restrict__ diffflag) {
+  constexpr int NS = NSEL > 0 ? NSEL : 1;
+  const int row = blockIdx.y;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  __shared__ u32 sh_cnt;
+  if (threadIdx.x == 0) sh_cnt = 0;
+  u32 lo[NS], hi[NS], cnt[NS];
+  float fB[NS];
+  double dB[NS];
+#pragma unroll
+  for (int j = 0; j < NS; ++j) {
+    lo[j] = (j < NSEL) ? sel[row].lo[j] : 0u;
+    hi[j] = (j < NSEL) ? sel[row].hi[j] : 0u;
+    cnt[j] = 0; fB[j] = 0.f; dB[j] = 0.0;
+  }
+  float fD = 0.f, fE = 0.f;
+  double dD = 0.0, dE = 0.0;
+  u32 mx = 0, mxw = 0, df = 0;
+  __syncthreads();
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  const float* yr = Y + (long long)row * d;
+  u64* seg = list + (long long)row * list_row + (long long)blockIdx.x * segcap;
+  const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  int it = 0;
+  for (long long t = blockIdx.x; t < ntile; t += gridDim.x, ++it) {
+    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
+    const bool live = c0 < d;
+    float x[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f}, y[4] = {0.f, 0.f, 0.f, 0.f};
+    if (live) {
+      load4<ALIGNED>(xr, c0, d, x);
+      load4<ALIGNED>(gr, c0, d, g);
+      load4<ALIGNED>(yr, c0, d, y);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const bool ok = live && (ALIGNED || c0 + k < d);
+      const float v = __fsub_rn(x[k], g[k]);
+      const float w = __fsub_rn(x[k], y[k]);
+      fE = fmaf(v, v, fE);
+      fD = fmaf(w, w, fD);
+      const u32 key = key_of(v), keyw = key_of(w);
+      mx = max(mx, key);
+      mxw = max(mxw, keyw);
+      df |= key ^ keyw;
+      if (NSEL > 0) {
+        bool inb = false;
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+          const bool ge = key >= hi[j];
+          const bool below = key < lo[j];
+          cnt[j] += ge ? 1u : 0u;
+          fB[j] = below ? fmaf(v, v, fB[j]) : fB[j];
+          inb = inb || (!ge && !below);
+        }
+        inb = inb && ok;
+        const u32 mask = __ballot_sync(0xffffffffu, inb);
+        if (mask) {
+          const int leader = __ffs(mask) - 1;
+          u32 base = 0;
+          if (lane == leader) base = atomicAdd(&sh_cnt, (u32)__popc(mask));
+          base = __shfl_sync(0xffffffffu, base, leader);
+          if (inb) {
+            const u32 pos = base + (u32)__popc(mask & ((1u << lane) - 1u));
+            if (pos < segcap) seg[pos] = ((u64)key << 32) | (u64)(u32)(c0 + k);
+          }
+        }
+      }
+    }
+    if ((it & (FLUSH_TILES - 1)) == FLUSH_TILES - 1) {
+      dD += (double)fD; fD = 0.f;
+      dE += (double)fE; fE = 0.f;
+#pragma unroll
+      for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; fB[j] = 0.f; }
+    }
+  }
+  dD += (double)fD;
+  dE += (double)fE;
+#pragma unroll
+  for (int j = 0; j < NS; ++j) dB[j] += (double)fB[j];
+
+  __shared__ double red[2 + NS][TPB / 32];
+  __shared__ u32 redc[NS][TPB / 32];
+  double v0 = warp_sum_f64(dD), v1 = warp_sum_f64(dE);
+  if (lane == 0) { red[0][wid] = v0; red[1][wid] = v1; }
+#pragma unroll
+  for (int j = 0; j < NS; ++j) {
+    const double vb = warp_sum_f64(dB[j]);
+    const u32 vc = warp_sum_u32(cnt[j]);
+    if (lane == 0) { red[2 + j][wid] = vb; redc[j][wid] = vc; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mxw = max(mxw, __shfl_xor_sync(0xffffffffu, mxw, o));
+    df |= __shfl_xor_sync(0xffffffffu, df, o);
+  }
+  if (lane == 0) {
+    if (mx) atomicMax(&maxkey[row], mx);
+    df &= 0x7fffffffu;
+    if (mxw >= 0x7f800000u) df |= 0x80000000u;
+    if (df) atomicOr(&diffflag[row], df);
+  }
+  __syncthreads();
+  const long long pbase = ((long long)row * MAX_BLK_PER_ROW + blockIdx.x);
+  if (threadIdx.x < 2 + NSEL) {
+    const int s = threadIdx.x;
+    double acc = 0;
+    for (int w = 0; w < TPB / 32; ++w) acc += red[s][w];
+    const int slot = (s < 2) ? s : 2 + cs.sel[s - 2];
+    partial[pbase * NSLOT + slot] = acc;
+  }
+  if (threadIdx.x >= 32 && threadIdx.x < 32 + NSEL) {
+    const int j = threadIdx.x - 32;
+    u32 acc = 0;
+    for (int w = 0; w < TPB / 32; ++w) acc += redc[j][w];
+    cntpart[pbase * MAXC + j] = acc;
+  }
+  if (threadIdx.x == 0 && NSEL > 0) {
+    const u32 n = sh_cnt;
+    lcount[pbase] = n < segcap ? n : segcap;
+    if (n > segcap) atomicOr(&rowflag[row], 1u);
+  }
+}
+
+// Passes over the listed keys.  PASS 1: per bracket, histogram of key[30:20];
+// PASS 2: key[19:9] of the keys in the bracket's first-digit bin; PASS 3: key[8:0] of the keys
+// sharing the 22-bit prefix, plus the energy of the bracket's keys below that prefix.
+template <int PASS>
+__global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow* __restrict__ sel,
+                                               const u64* __restrict__ list, const u32* __restrict__ lcount,
+                                               long long list_row, u32 segcap, u32* __restrict__ hist,
+                                               double* __restrict__ lepart, const u32* __restrict__ rowflag) {
+  extern __shared__ u32 sh[];
+  const int row = blockIdx.y;
+  if (rowflag[row]) return;
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  for (int i = threadIdx.x; i < nsel * NB; i += TPB) sh[i] = 0;
+  u32 lo[MAXC], hi[MAXC], pref[MAXC];
+  double en[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    lo[j] = (j < nsel) ? sel[row].lo[j] : 1u;
+    hi[j] = (j < nsel) ? sel[row].hi[j] : 0u;
+    pref[j] = 0;
+    if (PASS == 2 && j < nsel) pref[j] = sel[row].b1[j];
+    if (PASS == 3 && j < nsel) pref[j] = sel[row].p2[j];
+    en[j] = 0.0;
+  }
+  __syncthreads();
+  for (int sg = blockIdx.x; sg < nseg; sg += gridDim.x) {
+    const u32 n = lcount[(long long)row * MAX_BLK_PER_ROW + sg];
+    const u64* seg = list + (long long)row * list_row + (long long)sg * segcap;
+    for (u32 i = threadIdx.x; i < n; i += TPB) {
+      const u32 key = (u32)(seg[i] >> 32);
+#pragma unroll
+      for (int j = 0; j < MAXC; ++j) {
+        if (j < nsel && key >= lo[j] && key < hi[j]) {
+          if (PASS == 1) atomicAdd(&sh[j * NB + (key >> 20)], 1u);
+          if (PASS == 2 && (key >> 20) == pref[j]) atomicAdd(&sh[j * NB + ((key >> 9) & 0x7ffu)], 1u);
+          if (PASS == 3) {
+            if ((key >> 9) == pref[j]) atomicAdd(&sh[j * NB + (key & 0x1ffu)], 1u);
+            else if ((key >> 9) < pref[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  u32* gh = hist + (long long)row * MAXC * NB;
+  for (int i = threadIdx.x; i < nsel * NB; i += TPB)
+    if (sh[i]) atomicAdd(&gh[i], sh[i]);
+  if (PASS == 3) {
+    __shared__ double red[MAXC][TPB / 32];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < MAXC; ++j) {
+      const double vb = warp_sum_f64(en[j]);
+      if (lane == 0) red[j][wid] = vb;
+    }
+    __syncthreads();
+    if (threadIdx.x < MAXC) {
+      double a = 0;
+      for (int w = 0; w < TPB / 32; ++w) a += red[threadIdx.x][w];
+      lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
+    }
+  }
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, const u32* __restrict__ hist,
+                                               const u32* __restrict__ cntpart, const double* __restrict__ lepart,
+                                               SelRow* __restrict__ sel, u32* __restrict__ rowflag) {
+  __shared__ u32 res[2];
+  __shared__ u32 bad;
+  const int row = blockIdx.x;
+  if (rowflag[row]) return;  // uniform: written by earlier kernels only
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  SelRow* s = sel + row;
+  if (PASS == 1) {
+    // exact check of every bracket: the K-th largest key must be one of the listed keys
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    for (int j = 0; j < cs.nsel; ++j) {
+      u32 a = 0, tot = 0;
+      for (int b = threadIdx.x; b < nblk; b += TPB) a += cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j];
+      const u32* h = hist + ((long long)row * MAXC + j) * NB;
+      for (int b = threadIdx.x; b < NB; b += TPB) tot += h[b];
+      u32 above, total;
+      block_excl_scan(a, &above);
+      block_excl_scan(tot, &total);
+      if (threadIdx.x == 0) {
+        const long long K = cs.param[cs.sel[j]];
+        s->above_hi[j] = above;
+        if (K <= (long long)above || K > (long long)above + (long long)total) bad = 1;
+      }
+    }
+    __syncthreads();
+    if (bad) {
+      if (threadIdx.x == 0) rowflag[row] = 1;
+      return;
+    }
+  }
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 K = (u32)cs.param[cs.sel[j]];
+    const u32* h = hist + ((long long)row * MAXC + j) * NB;
+    const u32 before = (PASS == 1) ? s->above_hi[j] : (PASS == 2 ? s->above1[j] : s->above2[j]);
+    block_find_kth_desc(h, NB, K - before, res);
+    if (PASS == 3) {
+      // energy of the keys that share the 22-bit prefix and lie below the threshold: each bin is one key value
+      double a = 0.0;
+      for (int b = threadIdx.x; b < (int)res[0]; b += TPB) {
+        const double kv = (double)__uint_as_float((s->p2[j] << 9) | (u32)b);
+        a += (double)h[b] * (kv * kv);
+      }
+      __shared__ double redd[TPB / 32];
+      a = warp_sum_f64(a);
+      __syncthreads();
+      if ((threadIdx.x & 31) == 0) redd[threadIdx.x >> 5] = a;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        double e = 0.0;
+        for (int b = 0; b < LIST_BLK; ++b) e += lepart[((long long)row * LIST_BLK + b) * MAXC + j];
+        for (int w = 0; w < TPB / 32; ++w) e += redd[w];
+        s->extraE[j] = e;
+      }
+    }
+    if (threadIdx.x == 0) {
+      if (PASS == 1) {
+        s->b1[j] = res[0];
+        s->above1[j] = before + res[1];
+      } else if (PASS == 2) {
+        s->p2[j] = (s->b1[j] << 11) | res[0];
+        s->above2[j] = before + res[1];
+      } else {
+        s->T[j] = (s->p2[j] << 9) | res[0];
+        s->above[j] = before + res[1];
+        s->ntie[j] = h[res[0]];
+        s->q[j] = K - (before + res[1]);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// --------------------------------------------------------------------------
 // host side
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -737,9 +1122,17 @@ static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; 
 
 struct Layout {
   size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
+  size_t rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart;
+  long long list_row;
 };
 
-static Layout layout_of(int rows, long long d) {
+static long long list_row_of(long long d) {
+  long long a = d / 8, b = d < 65536 ? d : 65536;
+  long long r = a > b ? a : b;
+  return (r + 31) / 32 * 32;
+}
+
+static Layout layout_of(int rows, long long d, bool single_pass) {
   Layout L;
   size_t o = 0;
   L.hist1 = o; o = align_up(o + (size_t)rows * BINS1 * 4, 256);
@@ -754,14 +1147,27 @@ static Layout layout_of(int rows, long long d) {
   L.partial = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * NSLOT * 8, 256);
   L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
   L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
+  L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.list_row = 0;
+  L.shist = L.lhist1 = L.list = L.lcount = L.cntpart = L.lepart = o;
+  if (single_pass) {
+    L.list_row = list_row_of(d);
+    L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
+    L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
+    L.list = o; o = align_up(o + (size_t)rows * (size_t)L.list_row * 8, 256);
+    L.lcount = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * 4, 256);
+    L.cntpart = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * MAXC * 4, 256);
+    L.lepart = o; o = align_up(o + (size_t)rows * LIST_BLK * MAXC * 8, 256);
+  }
   L.total = o;
   return L;
 }
 
-size_t scratch_bytes(int rows, long long d) { return layout_of(rows, d).total; }
+size_t scratch_bytes(int rows, long long d, bool single_pass) { return layout_of(rows, d, single_pass).total; }
 
-void carve_scratch(Scratch* s, void* base, int rows, long long d) {
-  const Layout L = layout_of(rows, d);
+void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pass) {
+  const Layout L = layout_of(rows, d, single_pass);
   char* b = (char*)base;
   s->hist1 = (u32*)(b + L.hist1);
   s->hist2 = (u32*)(b + L.hist2);
@@ -776,6 +1182,20 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d) {
   s->partial = (double*)(b + L.partial);
   s->energy = (double*)(b + L.energy);
   s->tiecnt = (u32*)(b + L.tiecnt);
+  s->rowflag = (u32*)(b + L.rowflag);
+  s->diffflag = (u32*)(b + L.diffflag);
+  s->shist = s->lhist1 = s->lcount = s->cntpart = nullptr;
+  s->list = nullptr;
+  s->lepart = nullptr;
+  s->list_row = L.list_row;
+  if (single_pass) {
+    s->shist = (u32*)(b + L.shist);
+    s->lhist1 = (u32*)(b + L.lhist1);
+    s->list = (u64*)(b + L.list);
+    s->lcount = (u32*)(b + L.lcount);
+    s->cntpart = (u32*)(b + L.cntpart);
+    s->lepart = (double*)(b + L.lepart);
+  }
   s->rows_cap = rows;
   s->d_cap = d;
   s->nchunk_cap = nchunk_of(d);
@@ -825,6 +1245,10 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   if (!attr_done) {  // tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory
     cudaFuncSetAttribute(k_hist<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
     cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+    cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
+    cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+    cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
+    cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     attr_done = true;
   }
   const bool al = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y) &&
@@ -852,6 +1276,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   // clear the per-call accumulators
+  const bool single = (s.list != nullptr) && cs.nsel > 0;
   prof_begin(pf, KID_MEMSET, stream);
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
   cudaMemsetAsync(s.hist1, 0, (size_t)rows * BINS1 * 4, stream);
@@ -861,6 +1286,12 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   }
   cudaMemsetAsync(s.maxkey, 0, (size_t)rows * 4, stream);
   cudaMemsetAsync(s.limbs, 0, (size_t)rows * NSLOT * NLIMB * 8, stream);
+  cudaMemsetAsync(s.rowflag, 0, (size_t)rows * 4, stream);
+  cudaMemsetAsync(s.diffflag, 0, (size_t)rows * 4, stream);
+  if (single) {
+    cudaMemsetAsync(s.shist, 0, (size_t)rows * SBINS * 4, stream);
+    cudaMemsetAsync(s.lhist1, 0, (size_t)rows * MAXC * BINS1 * 4, stream);
+  }
   prof_end(pf, stream);
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
@@ -870,29 +1301,71 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   if (want < 1) want = 1;
   const int nblk = (int)want;
   const dim3 sgrid(nblk, rows);
+  const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
+  double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
 
-#define TIMED_HIST(id, PASS, shm, hist)                                                                              \
-  TIMED(id, if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr); \
-            else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, nullptr))
+#define TIMED_HIST(id, PASS, shm, hist)                                                                           \
+  TIMED(id, if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only); \
+            else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only))
+#define PASS1_CASE(N)                                                                                               \
+  case N:                                                                                                           \
+    if (al) k_pass1<N, true><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
+                                                        s.lcount, s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag); \
+    else k_pass1<N, false><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,          \
+                                                      s.lcount, s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag); \
+    break;
 
-  if (cs.nsel || cs.nquant) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
-  if (cs.nsel) {
-    TIMED(KID_SCAN, (k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, nullptr)));
-    TIMED_HIST(KID_HIST2, 2, cs.nsel * BINS2 * 4, s.hist2);
-    TIMED(KID_SCAN, (k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, nullptr)));
-    TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
-    TIMED(KID_SCAN, (k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, nullptr)));
+  if (single) {
+    // 1. brackets for every Top-K threshold from a sample of the row
+    long long stride = ntile / 128;
+    if (stride < 1) stride = 1;
+    if (stride > 32) stride = 32;
+    const long long nsamp = ntile / stride;
+    const dim3 samp_grid((unsigned)((nsamp + 47) / 48), rows);
+    TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist);
+    TIMED(KID_BRACKET, (k_bracket<<<rows, TPB, 0, stream>>>(cs, d, stride == 1 ? 1 : 0, s.shist, s.sel)));
+    // 2. the one pass over X, G, Y
+    const u32 segcap = (u32)(s.list_row / nblk);
+    prof_begin(pf, KID_PASS1, stream);
+    switch (cs.nsel) {
+      PASS1_CASE(1) PASS1_CASE(2) PASS1_CASE(3) PASS1_CASE(4)
+      PASS1_CASE(5) PASS1_CASE(6) PASS1_CASE(7) PASS1_CASE(8)
+    }
+    prof_end(pf, stream);
+    ++launches;
+    // 3. exact selection among the listed keys
+    const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
+    TIMED(KID_LHIST, (k_lhist<1><<<lgrid, TPB, cs.nsel * BINS1 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.lhist1, s.lepart, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LHIST, (k_lhist<2><<<lgrid, TPB, cs.nsel * BINS2 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist2, s.lepart, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LHIST, (k_lhist<3><<<dim3(LIST_BLK, rows), TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
   }
-  TIMED_AL(KID_ENERGY, k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial);
+  // the full radix select: every row, or (single-pass mode) only rows whose bracket failed
+  if (cs.nsel || cs.nquant) {
+    if (!single) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
+    else if (cs.nsel) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
+  }
+  if (cs.nsel) {
+    TIMED(KID_SCAN, (k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, only, s.flags)));
+    TIMED_HIST(KID_HIST2, 2, cs.nsel * BINS2 * 4, s.hist2);
+    TIMED(KID_SCAN, (k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, only, s.flags)));
+    TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
+    TIMED(KID_SCAN, (k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, only, s.flags)));
+  }
+  TIMED_AL(KID_ENERGY, k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
   if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
-  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out)));
-  TIMED_AL(KID_EXACT, k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs);
-  TIMED(KID_EXACT, (k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out)));
+  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out, s.diffflag, single ? 1 : 0, tol)));
+  TIMED_AL(KID_EXACT, k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag);
+  TIMED(KID_EXACT, (k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out, s.diffflag, s.flags)));
   if (cs.nsel) {
     TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)nchunk, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
     TIMED(KID_TIE, (k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk)));
   }
   TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+#undef PASS1_CASE
 #undef TIMED_HIST
 #undef TIMED_AL
 #undef TIMED
@@ -974,7 +1447,7 @@ extern "C" adacgd_status adacgd_compress_noalloc(const float* X_dev, float* G_de
     return ADACGD_ERR_INVALID_ARG;
   }
   if (rows < 1 || rows > ADACGD_NOALLOC_MAX_ROWS || d < 1 || d > ADACGD_NOALLOC_MAX_D ||
-      scratch_bytes(rows, d) > NOALLOC_SCRATCH_BYTES) {
+      scratch_bytes(rows, d, false) > NOALLOC_SCRATCH_BYTES) {
     set_thread_error("adacgd_compress_noalloc: shape exceeds the built-in scratch "
                      "(rows <= ADACGD_NOALLOC_MAX_ROWS = 4, d <= ADACGD_NOALLOC_MAX_D = 4194304); "
                      "use adacgd_init + adacgd_compress with a caller-owned workspace");
@@ -991,7 +1464,7 @@ extern "C" adacgd_status adacgd_compress_noalloc(const float* X_dev, float* G_de
   const adacgd_status sb = noalloc_base(&base);
   if (sb != ADACGD_OK) return sb;
   Scratch s;
-  carve_scratch(&s, base, rows, d);
+  carve_scratch(&s, base, rows, d, false);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   // the array keeps whatever the previous call left: the status words start from zero here,
   // the histograms and accumulators are cleared by launch_compress itself

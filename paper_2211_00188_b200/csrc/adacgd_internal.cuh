@@ -20,12 +20,15 @@ constexpr int BINS2 = 2048;         // key bits [19:9]
 constexpr int BINS3 = 512;          // key bits [8:0]
 constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (also the tie-order chunk)
 constexpr int MAX_BLK_PER_ROW = 2048;
+constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
+constexpr int LIST_BLK = 32;        // CTAs per row of the passes over the candidate lists
+constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
 // Optional per-kernel timing with CUDA events on the launching stream.
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_COUNT
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LSCAN, KID_COUNT
 };
 struct Prof {
   int cap, used;
@@ -60,6 +63,10 @@ struct SelRow {
   u32 above[MAXC];              // #keys  > T
   u32 ntie[MAXC];               // #keys == T
   u32 q[MAXC];                  // how many of the ties are kept (lowest indices first)
+  // single-pass path: bracket [lo, hi) of key values that must contain T, from a sample
+  u32 lo[MAXC], hi[MAXC];
+  u32 above_hi[MAXC];           // #keys >= hi
+  double extraE[MAXC];          // energy of listed keys in [lo, T)
 };
 
 // Decision for one row, consumed by the update kernel.
@@ -87,12 +94,22 @@ struct Scratch {
   double* partial; // [rows][MAX_BLK_PER_ROW][NSLOT]
   double* energy;  // [rows][NSLOT]
   u32* tiecnt;     // [rows][nchunk]  (exclusive prefix after the scan)
+  // single-pass path (null when the scratch was carved without it)
+  u32* shist;      // [rows][SBINS] sample histogram
+  u32* lhist1;     // [rows][MAXC][BINS1] first digit of the listed keys, per bracket
+  u64* list;       // [rows][list_row] (key << 32 | index), one segment of segcap entries per CTA
+  u32* lcount;     // [rows][MAX_BLK_PER_ROW] entries per segment
+  u32* cntpart;    // [rows][MAX_BLK_PER_ROW][MAXC] per-CTA counts of keys >= hi
+  double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the threshold prefix
+  u32* rowflag;    // [rows] 1: the row must take the full radix select (bracket missed or list overflow)
+  u32* diffflag;   // [rows] nonzero: some |X-G| differs from |X-Y|
+  long long list_row;
   int rows_cap; long long d_cap; long long nchunk_cap;
   Prof* prof;      // host pointer, may be null
 };
 
-size_t scratch_bytes(int rows, long long d);
-void carve_scratch(Scratch* s, void* base, int rows, long long d);
+size_t scratch_bytes(int rows, long long d, bool single_pass);
+void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pass);
 
 // Validates and converts a host candidate set. Returns ADACGD_OK / error and a message.
 adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const char** msg);
