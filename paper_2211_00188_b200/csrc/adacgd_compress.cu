@@ -387,11 +387,13 @@ __device__ void finalize_row(const CsetDev& cs, int row, int level, long long d,
     for (int j = 0; j <= cs.m; ++j) out.err[(long long)row * (cs.m + 1) + j] = e[j];
 }
 
-__global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk, const double* __restrict__ partial,
+__global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_main, int nblk_full,
+                                             const u32* __restrict__ rowflag, const double* __restrict__ partial,
                                              const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
                                              RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
                                              const u32* __restrict__ diffflag, int single_pass, double tol) {
   const int row = blockIdx.x, lane = threadIdx.x;
+  const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
   double sum[NSLOT];
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) {
@@ -606,19 +608,21 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
   const int row = blockIdx.y;
   if (!dec[row].need_tie) return;
   const u32 T = dec[row].T;
-  const long long c0 = (long long)blockIdx.x * UPD_COLS + threadIdx.x * 4;
-  u32 cnt = 0;
-  if (c0 < d) {
-    float x[4], g[4];
-    load4<ALIGNED>(X + (long long)row * d, c0, d, x);
-    load4<ALIGNED>(G + (long long)row * d, c0, d, g);
+  for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
+    const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
+    u32 cnt = 0;
+    if (c0 < d) {
+      float x[4], g[4];
+      load4<ALIGNED>(X + (long long)row * d, c0, d, x);
+      load4<ALIGNED>(G + (long long)row * d, c0, d, g);
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if ((ALIGNED || c0 + k < d) && key_of(__fsub_rn(x[k], g[k])) == T) ++cnt;
+      for (int k = 0; k < 4; ++k)
+        if ((ALIGNED || c0 + k < d) && key_of(__fsub_rn(x[k], g[k])) == T) ++cnt;
+    }
+    u32 total;
+    block_excl_scan(cnt, &total);
+    if (threadIdx.x == 0) tiecnt[(long long)row * nchunk + chunk] = total;
   }
-  u32 total;
-  block_excl_scan(cnt, &total);
-  if (threadIdx.x == 0) tiecnt[(long long)row * nchunk + blockIdx.x] = total;
 }
 
 __global__ void __launch_bounds__(TPB) k_tiescan(const RowDec* __restrict__ dec, u32* __restrict__ tiecnt,
@@ -638,102 +642,140 @@ __global__ void __launch_bounds__(TPB) k_tiescan(const RowDec* __restrict__ dec,
 }
 
 // Thread owns 4 consecutive columns and walks the rows in order, so that the mean is
-// summed in worker order.  Row i: G_i <- G_i + C_level(X_i - G_i) (EF21, Eq. 7).
+// summed in worker order.  Row i: G_i <- G_i + C_level(X_i - G_i) (EF21, Eq. 7).  The next
+// row's operands are loaded before the current row is written back.
+constexpr int UPD_ROW_TILE = 32;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
                                                 CompressOut out) {
+  __shared__ RowDec shd[UPD_ROW_TILE];
   const long long c0 = (long long)blockIdx.x * UPD_COLS + threadIdx.x * 4;
   const bool live = c0 < d;
   const int lane = threadIdx.x & 31;
+  const bool want_mean = out.mean_out != nullptr;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int i = 0; i < rows; ++i) {
-    const int mode = copy_mode ? 4 : dec[i].mode;
-    float* grow = G + (long long)i * d;
-    float g[4] = {0.f, 0.f, 0.f, 0.f};
-    if (live && mode != 4) load4<ALIGNED>(grow, c0, d, g);
-    if (mode != 0) {
-      float x[4] = {0.f, 0.f, 0.f, 0.f};
-      if (live) load4<ALIGNED>(X + (long long)i * d, c0, d, x);
-      bool kept[4] = {false, false, false, false};
-      bool any = false;
-      if (mode == 4) {
+  for (int r0 = 0; r0 < rows; r0 += UPD_ROW_TILE) {
+    const int nr = (rows - r0 < UPD_ROW_TILE) ? rows - r0 : UPD_ROW_TILE;
+    __syncthreads();
+    if (threadIdx.x < nr) {
+      RowDec t;
+      if (copy_mode) { t.level = 0; t.mode = 4; t.T = 0; t.q = 0; t.need_tie = 0; t.need_exact = 0; t.qL = t.qinv = t.qstep = 0.f; t.pad = 0; }
+      else t = dec[r0 + threadIdx.x];
+      shd[threadIdx.x] = t;
+    }
+    __syncthreads();
+    float gn[4] = {0.f, 0.f, 0.f, 0.f}, xn[4] = {0.f, 0.f, 0.f, 0.f};
+    if (live) {
+      const int m0 = shd[0].mode;
+      if (m0 != 4 && (m0 != 0 || want_mean)) load4<ALIGNED>(G + (long long)r0 * d, c0, d, gn);
+      if (m0 != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, xn);
+    }
+    for (int ii = 0; ii < nr; ++ii) {
+      const int i = r0 + ii;
+      const int mode = shd[ii].mode;
+      float* grow = G + (long long)i * d;
+      float g[4], x[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) g[k] = x[k];
-        any = live;
-      } else if (mode == 1) {
-        const u32 T = dec[i].T, q = dec[i].q;
-        const int need_tie = dec[i].need_tie;
-        u32 key[4];
-        float v[4];
-        u32 nt = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const bool ok = live && (ALIGNED || c0 + k < d);
-          v[k] = __fsub_rn(x[k], g[k]);
-          key[k] = ok ? key_of(v[k]) : 0xffffffffu;  // never equal to T, handled below
-          if (ok && key[k] == T) ++nt;
-        }
-        u32 before = 0;
-        if (need_tie) before = tiepref[(long long)i * nchunk + blockIdx.x] + block_excl_scan(nt, nullptr);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const bool ok = live && (ALIGNED || c0 + k < d);
-          if (!ok) continue;
-          if (key[k] > T) kept[k] = true;
-          else if (key[k] == T) {
-            kept[k] = need_tie ? (before < q) : true;
-            ++before;
-          }
-          if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
-        }
-      } else if (mode == 2) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
-          kept[k] = live && (ALIGNED || c0 + k < d);
-        }
-        any = live;
-      } else {  // quantiser
-        const float L = dec[i].qL, inv = dec[i].qinv, step = dec[i].qstep;
+      for (int k = 0; k < 4; ++k) { g[k] = gn[k]; x[k] = xn[k]; }
+      if (ii + 1 < nr && live) {
+        const int m1 = shd[ii + 1].mode;
+        if (m1 != 4 && (m1 != 0 || want_mean)) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, gn);
+        if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, xn);
+      }
+      if (mode == 1 && !shd[ii].need_tie && !out.kept_idx) {
+        // common case: keep every key >= T (all threshold-equal keys are kept)
+        const u32 T = shd[ii].T;
+        bool any = false;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const float v = __fsub_rn(x[k], g[k]);
-          g[k] = __fadd_rn(g[k], quant_value(v, L, inv, step));
+          const bool kept = key_of(v) >= T && (ALIGNED || c0 + k < d);
+          g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+          any = any || kept;
         }
-        any = live;
-      }
-      if (any) store4<ALIGNED>(grow, c0, d, g);
-      if (out.kept_idx && (mode == 1 || mode == 2)) {
-        int mine = 0;
+        if (any && live) store4<ALIGNED>(grow, c0, d, g);
+      } else if (mode != 0) {
+        bool kept[4] = {false, false, false, false};
+        bool any = false;
+        if (mode == 4) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) mine += kept[k] ? 1 : 0;
-        int inc = mine;
+          for (int k = 0; k < 4; ++k) g[k] = x[k];
+          any = live;
+        } else if (mode == 1) {
+          const u32 T = shd[ii].T, q = shd[ii].q;
+          const int need_tie = shd[ii].need_tie;
+          u32 key[4];
+          float v[4];
+          u32 nt = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          int t = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += t;
-        }
-        const int wtotal = __shfl_sync(0xffffffffu, inc, 31);
-        long long base = 0;
-        if (lane == 31 && wtotal) base = (long long)atomicAdd((u64*)&out.kept_cnt[i], (u64)wtotal);
-        base = __shfl_sync(0xffffffffu, base, 31);
-        long long pos = base + inc - mine;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (kept[k]) {
-            if (pos < out.kept_stride) out.kept_idx[(long long)i * out.kept_stride + pos] = (int32_t)(c0 + k);
-            ++pos;
+          for (int k = 0; k < 4; ++k) {
+            const bool ok = live && (ALIGNED || c0 + k < d);
+            v[k] = __fsub_rn(x[k], g[k]);
+            key[k] = ok ? key_of(v[k]) : 0xffffffffu;
+            if (ok && key[k] == T) ++nt;
           }
-      }
-    }
-    if (out.mean_out) {
+          u32 before = 0;
+          if (need_tie) before = tiepref[(long long)i * nchunk + blockIdx.x] + block_excl_scan(nt, nullptr);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) acc[k] = (i == 0) ? g[k] : __fadd_rn(acc[k], g[k]);
+          for (int k = 0; k < 4; ++k) {
+            const bool ok = live && (ALIGNED || c0 + k < d);
+            if (!ok) continue;
+            if (key[k] > T) kept[k] = true;
+            else if (key[k] == T) {
+              kept[k] = need_tie ? (before < q) : true;
+              ++before;
+            }
+            if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
+          }
+        } else if (mode == 2) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
+            kept[k] = live && (ALIGNED || c0 + k < d);
+          }
+          any = live;
+        } else {  // quantiser
+          const float L = shd[ii].qL, inv = shd[ii].qinv, step = shd[ii].qstep;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float v = __fsub_rn(x[k], g[k]);
+            g[k] = __fadd_rn(g[k], quant_value(v, L, inv, step));
+          }
+          any = live;
+        }
+        if (any) store4<ALIGNED>(grow, c0, d, g);
+        if (out.kept_idx && (mode == 1 || mode == 2)) {
+          int mine = 0;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mine += kept[k] ? 1 : 0;
+          int inc = mine;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+          }
+          const int wtotal = __shfl_sync(0xffffffffu, inc, 31);
+          long long base = 0;
+          if (lane == 31 && wtotal) base = (long long)atomicAdd((u64*)&out.kept_cnt[i], (u64)wtotal);
+          base = __shfl_sync(0xffffffffu, base, 31);
+          long long pos = base + inc - mine;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (kept[k]) {
+              if (pos < out.kept_stride) out.kept_idx[(long long)i * out.kept_stride + pos] = (int32_t)(c0 + k);
+              ++pos;
+            }
+        }
+      }
+      if (want_mean) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[k] = (i == 0) ? g[k] : __fadd_rn(acc[k], g[k]);
+      }
     }
   }
-  if (out.mean_out && live) {
+  if (want_mean && live) {
     const float n = (float)rows;
     float r[4];
 #pragma unroll
@@ -792,15 +834,34 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
 }
 
 // Finds the bin holding the r-th largest sampled key (1-based); all TPB threads call.
-// `excl`/`sum` are this thread's exclusive prefix and count over its 256 bins (descending order).
-__device__ void sample_rank_bin(const u32* __restrict__ h, u32 excl, u32 sum, u32 r, u32* out) {
-  if (r > excl && r <= excl + sum) {
-    u32 run = excl;
-    for (int k = 0; k < SBINS / TPB; ++k) {
-      const int bin = SBINS - 1 - (threadIdx.x * (SBINS / TPB) + k);
-      const u32 c = h[bin];
-      if (r <= run + c) { *out = (u32)bin; break; }
-      run += c;
+// csum/cexcl: counts and exclusive prefixes of the 256 chunks of 256 bins, in descending bin order.
+__device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, const u32* cexcl, u32 r, u32* out) {
+  __shared__ int chunk_sh;
+  if (cexcl[threadIdx.x] < r && r <= cexcl[threadIdx.x] + csum[threadIdx.x]) chunk_sh = threadIdx.x;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    const int c = chunk_sh;
+    const int pos0 = 256 * c + 8 * lane;                       // descending position of this lane's first bin
+    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 8 - pos0));
+    const uint4 a = p[0], b = p[1];                            // ascending addresses: positions pos0+7 .. pos0
+    const u32 v[8] = {b.w, b.z, b.y, b.x, a.w, a.z, a.y, a.x}; // v[k] = bin at descending position pos0 + k
+    u32 lsum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) lsum += v[k];
+    u32 inc = lsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    u32 run = cexcl[c] + inc - lsum;
+    if (run < r && r <= run + lsum) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (r > run && r <= run + v[k]) *out = (u32)(SBINS - 1 - (pos0 + k));
+        run += v[k];
+      }
     }
   }
   __syncthreads();
@@ -810,13 +871,22 @@ __device__ void sample_rank_bin(const u32* __restrict__ h, u32 excl, u32 sum, u3
 // holds the K-th largest key with overwhelming probability (checked exactly afterwards).
 __global__ void __launch_bounds__(TPB) k_bracket(CsetDev cs, long long d, int full_sample,
                                                  const u32* __restrict__ shist, SelRow* __restrict__ sel) {
+  __shared__ u32 csum[TPB], cexcl[TPB];
   __shared__ u32 res;
   const int row = blockIdx.x;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const u32* h = shist + (long long)row * SBINS;
-  u32 sum = 0;
-  for (int k = 0; k < SBINS / TPB; ++k) sum += h[SBINS - 1 - (threadIdx.x * (SBINS / TPB) + k)];
+  for (int c = wid; c < 256; c += TPB / 32) {
+    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 256 * (c + 1))) + 2 * lane;
+    const uint4 a = p[0], b = p[1];
+    const u32 t = warp_sum_u32(a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w);
+    if (lane == 0) csum[c] = t;
+  }
+  __syncthreads();
   u32 S;
-  const u32 excl = block_excl_scan(sum, &S);
+  const u32 ex = block_excl_scan(csum[threadIdx.x], &S);
+  cexcl[threadIdx.x] = ex;
+  __syncthreads();
   for (int j = 0; j < cs.nsel; ++j) {
     const double K = (double)cs.param[cs.sel[j]];
     const double r = K * (double)S / (double)d;
@@ -824,12 +894,12 @@ __global__ void __launch_bounds__(TPB) k_bracket(CsetDev cs, long long d, int fu
     const double r_hi = floor(r - dev), r_lo = ceil(r + dev) + 1.0;
     u32 hi = 0x80000000u, lo = 0u;
     if (r_hi >= 1.0) {
-      sample_rank_bin(h, excl, sum, (u32)r_hi, &res);
+      sample_rank_bin(h, csum, cexcl, (u32)r_hi, &res);
       hi = (res + 1u) << 15;
       __syncthreads();
     }
     if (r_lo <= (double)S) {
-      sample_rank_bin(h, excl, sum, (u32)r_lo, &res);
+      sample_rank_bin(h, csum, cexcl, (u32)r_lo, &res);
       lo = res << 15;
     }
     if (threadIdx.x == 0) { sel[row].lo[j] = lo; sel[row].hi[j] = hi; }
@@ -1038,7 +1108,7 @@ __global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow*
 }
 
 template <int PASS>
-__global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, const u32* __restrict__ hist,
+__global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, int nlb, const u32* __restrict__ hist,
                                                const u32* __restrict__ cntpart, const double* __restrict__ lepart,
                                                SelRow* __restrict__ sel, u32* __restrict__ rowflag) {
   __shared__ u32 res[2];
@@ -1090,7 +1160,7 @@ __global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, const u32* 
       __syncthreads();
       if (threadIdx.x == 0) {
         double e = 0.0;
-        for (int b = 0; b < LIST_BLK; ++b) e += lepart[((long long)row * LIST_BLK + b) * MAXC + j];
+        for (int b = 0; b < nlb; ++b) e += lepart[((long long)row * LIST_BLK + b) * MAXC + j];
         for (int w = 0; w < TPB / 32; ++w) e += redd[w];
         s->extraE[j] = e;
       }
@@ -1140,21 +1210,24 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.hist3 = o; o = align_up(o + (size_t)rows * MAXC * BINS3 * 4, 256);
   L.maxkey = o; o = align_up(o + (size_t)rows * 4, 256);
   L.limbs = o; o = align_up(o + (size_t)rows * NSLOT * NLIMB * 8, 256);
-  L.flags = o; o = align_up(o + 16, 256);
+  L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.shist = L.lhist1 = o;
+  if (single_pass) {
+    L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
+    L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
+  }
   L.zero_end = o;
+  L.flags = o; o = align_up(o + 16, 256);
   L.sel = o; o = align_up(o + (size_t)rows * sizeof(SelRow), 256);
   L.dec = o; o = align_up(o + (size_t)rows * sizeof(RowDec), 256);
   L.partial = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * NSLOT * 8, 256);
   L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
   L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
-  L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
-  L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.list_row = 0;
-  L.shist = L.lhist1 = L.list = L.lcount = L.cntpart = L.lepart = o;
+  L.list = L.lcount = L.cntpart = L.lepart = o;
   if (single_pass) {
     L.list_row = list_row_of(d);
-    L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
-    L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
     L.list = o; o = align_up(o + (size_t)rows * (size_t)L.list_row * 8, 256);
     L.lcount = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * MAXC * 4, 256);
@@ -1279,19 +1352,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const bool single = (s.list != nullptr) && cs.nsel > 0;
   prof_begin(pf, KID_MEMSET, stream);
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
-  cudaMemsetAsync(s.hist1, 0, (size_t)rows * BINS1 * 4, stream);
-  if (cs.nsel) {
-    cudaMemsetAsync(s.hist2, 0, (size_t)rows * MAXC * BINS2 * 4, stream);
-    cudaMemsetAsync(s.hist3, 0, (size_t)rows * MAXC * BINS3 * 4, stream);
-  }
-  cudaMemsetAsync(s.maxkey, 0, (size_t)rows * 4, stream);
-  cudaMemsetAsync(s.limbs, 0, (size_t)rows * NSLOT * NLIMB * 8, stream);
-  cudaMemsetAsync(s.rowflag, 0, (size_t)rows * 4, stream);
-  cudaMemsetAsync(s.diffflag, 0, (size_t)rows * 4, stream);
-  if (single) {
-    cudaMemsetAsync(s.shist, 0, (size_t)rows * SBINS * 4, stream);
-    cudaMemsetAsync(s.lhist1, 0, (size_t)rows * MAXC * BINS1 * 4, stream);
-  }
+  cudaMemsetAsync(s.zero_begin, 0, s.zero_bytes, stream);  // histograms, limbs, row flags: one contiguous region
   prof_end(pf, stream);
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
@@ -1301,12 +1362,18 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   if (want < 1) want = 1;
   const int nblk = (int)want;
   const dim3 sgrid(nblk, rows);
+  // in single-pass mode the full select only serves rows whose bracket failed: a small grid keeps the
+  // usual no-op launches cheap
+  long long want_full = single ? (148 * 2 + rows - 1) / rows : nblk;
+  if (want_full > nblk) want_full = nblk;
+  const int nblk_full = (int)want_full;
+  const dim3 fgrid(nblk_full, rows);
   const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
   double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
 
 #define TIMED_HIST(id, PASS, shm, hist)                                                                           \
-  TIMED(id, if (al) k_hist<PASS, true><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only); \
-            else k_hist<PASS, false><<<sgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only))
+  TIMED(id, if (al) k_hist<PASS, true><<<fgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only); \
+            else k_hist<PASS, false><<<fgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only))
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
     if (al) k_pass1<N, true><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
@@ -1321,7 +1388,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (stride < 1) stride = 1;
     if (stride > 32) stride = 32;
     const long long nsamp = ntile / stride;
-    const dim3 samp_grid((unsigned)((nsamp + 47) / 48), rows);
+    const dim3 samp_grid((unsigned)((nsamp + 15) / 16), rows);
     TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist);
     TIMED(KID_BRACKET, (k_bracket<<<rows, TPB, 0, stream>>>(cs, d, stride == 1 ? 1 : 0, s.shist, s.sel)));
     // 2. the one pass over X, G, Y
@@ -1336,11 +1403,11 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // 3. exact selection among the listed keys
     const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
     TIMED(KID_LHIST, (k_lhist<1><<<lgrid, TPB, cs.nsel * BINS1 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.lhist1, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag)));
     TIMED(KID_LHIST, (k_lhist<2><<<lgrid, TPB, cs.nsel * BINS2 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist2, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag)));
-    TIMED(KID_LHIST, (k_lhist<3><<<dim3(LIST_BLK, rows), TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LHIST, (k_lhist<3><<<lgrid, TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag)));
+    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag)));
     tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
   }
   // the full radix select: every row, or (single-pass mode) only rows whose bracket failed
@@ -1355,13 +1422,15 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
     TIMED(KID_SCAN, (k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, only, s.flags)));
   }
-  TIMED_AL(KID_ENERGY, k_energy, sgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
+  TIMED_AL(KID_ENERGY, k_energy, fgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
   if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
-  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, s.partial, s.sel, s.maxkey, s.dec, s.flags, out, s.diffflag, single ? 1 : 0, tol)));
-  TIMED_AL(KID_EXACT, k_exact_sums, sgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag);
+  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey, s.dec, s.flags, out, s.diffflag, single ? 1 : 0, tol)));
+  TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag);
   TIMED(KID_EXACT, (k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out, s.diffflag, s.flags)));
   if (cs.nsel) {
-    TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)nchunk, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
+    long long tgx = (148 * 4 + rows - 1) / rows;
+    if (tgx > nchunk) tgx = nchunk;
+    TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
     TIMED(KID_TIE, (k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk)));
   }
   TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);

@@ -21,7 +21,7 @@ constexpr int BINS3 = 512;          // key bits [8:0]
 constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (also the tie-order chunk)
 constexpr int MAX_BLK_PER_ROW = 2048;
 constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
-constexpr int LIST_BLK = 32;        // CTAs per row of the passes over the candidate lists
+constexpr int LIST_BLK = 256;       // CTAs per row of the passes over the candidate lists
 constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
 // Optional per-kernel timing with CUDA events on the launching stream.
