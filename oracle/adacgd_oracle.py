@@ -165,12 +165,25 @@ def message_bits(cand, d: int) -> int:
 # --------------------------------------------------------------------------
 # three point compressors
 # --------------------------------------------------------------------------
+def apply_shifted(h, v, cand) -> np.ndarray:
+    """h + C(v) in binary32.  A Top-K message is sparse: the receiver adds it at the kept
+    indices and leaves every other entry of h as it is (so a -0.0 outside the kept set stays
+    -0.0); a quantised message is dense and is added everywhere."""
+    kind, param = cand
+    if kind == TOPK:
+        out = h.copy()
+        kept = topk_kept(v, param)
+        out[kept] = (h[kept] + v[kept]).astype(F32)
+        return out
+    return (h + apply_candidate(v, cand)).astype(F32)
+
+
 def ef21(h, y, x, cand) -> np.ndarray:
     """EF21 compressor (Eq. 7): h + C(x - h), every operation in binary32."""
     h = _as_f32(h)
     x = _as_f32(x)
     v = (x - h).astype(F32)
-    return (h + apply_candidate(v, cand)).astype(F32)
+    return apply_shifted(h, v, cand)
 
 
 def lag(h, y, x, zeta) -> np.ndarray:
@@ -238,7 +251,7 @@ def adacgd(h, y, x, cands, zeta):
     if level == 0:
         return dict(out=h.copy(), level=0, bits=0, err=err, D=D, kept=None)
     cand = cands[level - 1]
-    out = (h + apply_candidate(v, cand)).astype(F32)
+    out = apply_shifted(h, v, cand)
     kept = np.sort(topk_kept(v, cand[1])) if cand[0] == TOPK else None
     return dict(out=out, level=level, bits=message_bits(cand, d), err=err, D=D, kept=kept)
 

@@ -199,6 +199,8 @@ __global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict_
         s->ntie[j] = h[res[0]];
         s->q[j] = K - (before + res[1]);
         s->extraE[j] = 0.0;
+        s->tiemode[j] = (s->q[j] < s->ntie[j]) ? 2u : 0u;
+        s->cut[j] = 0xffffffffu;
       }
     }
     __syncthreads();
@@ -360,7 +362,7 @@ __device__ void finalize_row(const CsetDev& cs, int row, int level, long long d,
                              double D) {
   RowDec r;
   r.level = level; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 0;
-  r.qL = r.qinv = r.qstep = 0.f; r.pad = 0;
+  r.qL = r.qinv = r.qstep = 0.f; r.cut = 0xffffffffu;
   if (level > 0) {
     const int c = level - 1;
     if (cs.kind[c] == ADACGD_TOPK) {
@@ -370,7 +372,8 @@ __device__ void finalize_row(const CsetDev& cs, int row, int level, long long d,
         int j = 0;
         for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
         r.mode = 1; r.T = sel[row].T[j]; r.q = sel[row].q[j];
-        r.need_tie = (sel[row].q[j] < sel[row].ntie[j]) ? 1 : 0;
+        r.need_tie = (sel[row].tiemode[j] == 2u) ? 1 : 0;
+        r.cut = (sel[row].tiemode[j] == 1u) ? sel[row].cut[j] : 0xffffffffu;
       }
     } else {
       r.mode = 3;
@@ -450,7 +453,7 @@ __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_m
   if (unsure) {
     RowDec r;
     r.level = -1; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 1;
-    r.qL = r.qinv = r.qstep = 0.f; r.pad = 0;
+    r.qL = r.qinv = r.qstep = 0.f; r.cut = 0xffffffffu;
     dec[row] = r;
     atomicAdd(&flags[1], 1u);
     return;
@@ -661,7 +664,7 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
     __syncthreads();
     if (threadIdx.x < nr) {
       RowDec t;
-      if (copy_mode) { t.level = 0; t.mode = 4; t.T = 0; t.q = 0; t.need_tie = 0; t.need_exact = 0; t.qL = t.qinv = t.qstep = 0.f; t.pad = 0; }
+      if (copy_mode) { t.level = 0; t.mode = 4; t.T = 0; t.q = 0; t.need_tie = 0; t.need_exact = 0; t.qL = t.qinv = t.qstep = 0.f; t.cut = 0xffffffffu; }
       else t = dec[r0 + threadIdx.x];
       shd[threadIdx.x] = t;
     }
@@ -685,13 +688,14 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
         if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, xn);
       }
       if (mode == 1 && !shd[ii].need_tie && !out.kept_idx) {
-        // common case: keep every key >= T (all threshold-equal keys are kept)
-        const u32 T = shd[ii].T;
+        // common case: keep every key > T and the threshold-equal keys up to index `cut`
+        const u32 T = shd[ii].T, cut = shd[ii].cut;
         bool any = false;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const float v = __fsub_rn(x[k], g[k]);
-          const bool kept = key_of(v) >= T && (ALIGNED || c0 + k < d);
+          const u32 key = key_of(v);
+          const bool kept = (key > T || (key == T && (u32)(c0 + k) <= cut)) && (ALIGNED || c0 + k < d);
           g[k] = kept ? __fadd_rn(g[k], v) : g[k];
           any = any || kept;
         }
@@ -724,7 +728,7 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
             if (!ok) continue;
             if (key[k] > T) kept[k] = true;
             else if (key[k] == T) {
-              kept[k] = need_tie ? (before < q) : true;
+              kept[k] = need_tie ? (before < q) : ((u32)(c0 + k) <= shd[ii].cut);
               ++before;
             }
             if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
@@ -1050,7 +1054,8 @@ template <int PASS>
 __global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow* __restrict__ sel,
                                                const u64* __restrict__ list, const u32* __restrict__ lcount,
                                                long long list_row, u32 segcap, u32* __restrict__ hist,
-                                               double* __restrict__ lepart, const u32* __restrict__ rowflag) {
+                                               double* __restrict__ lepart, const u32* __restrict__ rowflag,
+                                               u64* __restrict__ fl, u32* __restrict__ flcnt) {
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
   if (rowflag[row]) return;
@@ -1072,14 +1077,19 @@ __global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow*
     const u32 n = lcount[(long long)row * MAX_BLK_PER_ROW + sg];
     const u64* seg = list + (long long)row * list_row + (long long)sg * segcap;
     for (u32 i = threadIdx.x; i < n; i += TPB) {
-      const u32 key = (u32)(seg[i] >> 32);
+      const u64 ent = seg[i];
+      const u32 key = (u32)(ent >> 32);
 #pragma unroll
       for (int j = 0; j < MAXC; ++j) {
         if (j < nsel && key >= lo[j] && key < hi[j]) {
           if (PASS == 1) atomicAdd(&sh[j * NB + (key >> 20)], 1u);
           if (PASS == 2 && (key >> 20) == pref[j]) atomicAdd(&sh[j * NB + ((key >> 9) & 0x7ffu)], 1u);
           if (PASS == 3) {
-            if ((key >> 9) == pref[j]) atomicAdd(&sh[j * NB + (key & 0x1ffu)], 1u);
+            if ((key >> 9) == pref[j]) {
+              atomicAdd(&sh[j * NB + (key & 0x1ffu)], 1u);
+              const u32 pos = atomicAdd(&flcnt[row * MAXC + j], 1u);
+              if (pos < FINAL_CAP) fl[((long long)row * MAXC + j) * FINAL_CAP + pos] = ent;
+            }
             else if ((key >> 9) < pref[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
           }
         }
@@ -1110,7 +1120,8 @@ __global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow*
 template <int PASS>
 __global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, int nlb, const u32* __restrict__ hist,
                                                const u32* __restrict__ cntpart, const double* __restrict__ lepart,
-                                               SelRow* __restrict__ sel, u32* __restrict__ rowflag) {
+                                               SelRow* __restrict__ sel, u32* __restrict__ rowflag,
+                                               const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
   __shared__ u32 res[2];
   __shared__ u32 bad;
   const int row = blockIdx.x;
@@ -1180,6 +1191,35 @@ __global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, int nlb, co
       }
     }
     __syncthreads();
+    if (PASS == 3) {
+      // Which threshold-equal keys are kept: the q with the lowest indices.  They are all among the
+      // collected prefix-equal entries; the q-th smallest of their indices is the cut.
+      __shared__ u32 ties[1024];
+      __shared__ u32 nties_sh;
+      const u32 T = s->T[j], q = s->q[j], ntie = s->ntie[j];
+      const u32 nfl = flcnt[row * MAXC + j];
+      if (q == ntie) {
+        if (threadIdx.x == 0) { s->tiemode[j] = 0u; s->cut[j] = 0xffffffffu; }
+      } else if (nfl > FINAL_CAP || ntie > 1024u) {
+        if (threadIdx.x == 0) { s->tiemode[j] = 2u; s->cut[j] = 0xffffffffu; }
+      } else {
+        if (threadIdx.x == 0) nties_sh = 0;
+        __syncthreads();
+        const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
+        for (u32 i = threadIdx.x; i < nfl; i += TPB) {
+          const u64 ent = f[i];
+          if ((u32)(ent >> 32) == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)ent;
+        }
+        __syncthreads();
+        for (u32 i = threadIdx.x; i < ntie; i += TPB) {
+          const u32 mine = ties[i];
+          u32 rank = 0;
+          for (u32 k = 0; k < ntie; ++k) rank += (ties[k] < mine) ? 1u : 0u;
+          if (rank == q - 1u) { s->tiemode[j] = 1u; s->cut[j] = mine; }
+        }
+      }
+      __syncthreads();
+    }
   }
 }
 
@@ -1192,7 +1232,7 @@ static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; 
 
 struct Layout {
   size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
-  size_t rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart;
+  size_t rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, fl, flcnt;
   long long list_row;
 };
 
@@ -1212,8 +1252,9 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.limbs = o; o = align_up(o + (size_t)rows * NSLOT * NLIMB * 8, 256);
   L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
-  L.shist = L.lhist1 = o;
+  L.shist = L.lhist1 = L.flcnt = o;
   if (single_pass) {
+    L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
     L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
   }
@@ -1225,9 +1266,10 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
   L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
   L.list_row = 0;
-  L.list = L.lcount = L.cntpart = L.lepart = o;
+  L.list = L.lcount = L.cntpart = L.lepart = L.fl = o;
   if (single_pass) {
     L.list_row = list_row_of(d);
+    L.fl = o; o = align_up(o + (size_t)rows * MAXC * FINAL_CAP * 8, 256);
     L.list = o; o = align_up(o + (size_t)rows * (size_t)L.list_row * 8, 256);
     L.lcount = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * MAXC * 4, 256);
@@ -1260,6 +1302,8 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->shist = s->lhist1 = s->lcount = s->cntpart = nullptr;
   s->list = nullptr;
   s->lepart = nullptr;
+  s->fl = nullptr;
+  s->flcnt = nullptr;
   s->list_row = L.list_row;
   if (single_pass) {
     s->shist = (u32*)(b + L.shist);
@@ -1268,6 +1312,8 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
     s->lcount = (u32*)(b + L.lcount);
     s->cntpart = (u32*)(b + L.cntpart);
     s->lepart = (double*)(b + L.lepart);
+    s->fl = (u64*)(b + L.fl);
+    s->flcnt = (u32*)(b + L.flcnt);
   }
   s->rows_cap = rows;
   s->d_cap = d;
@@ -1402,12 +1448,12 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     ++launches;
     // 3. exact selection among the listed keys
     const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
-    TIMED(KID_LHIST, (k_lhist<1><<<lgrid, TPB, cs.nsel * BINS1 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.lhist1, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag)));
-    TIMED(KID_LHIST, (k_lhist<2><<<lgrid, TPB, cs.nsel * BINS2 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist2, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag)));
-    TIMED(KID_LHIST, (k_lhist<3><<<lgrid, TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag)));
-    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag)));
+    TIMED(KID_LHIST, (k_lhist<1><<<lgrid, TPB, cs.nsel * BINS1 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.lhist1, s.lepart, s.rowflag, s.fl, s.flcnt)));
+    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
+    TIMED(KID_LHIST, (k_lhist<2><<<lgrid, TPB, cs.nsel * BINS2 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist2, s.lepart, s.rowflag, s.fl, s.flcnt)));
+    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
+    TIMED(KID_LHIST, (k_lhist<3><<<lgrid, TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag, s.fl, s.flcnt)));
+    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
     tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
   }
   // the full radix select: every row, or (single-pass mode) only rows whose bracket failed

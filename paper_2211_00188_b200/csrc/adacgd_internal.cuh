@@ -22,6 +22,7 @@ constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (als
 constexpr int MAX_BLK_PER_ROW = 2048;
 constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
 constexpr int LIST_BLK = 256;       // CTAs per row of the passes over the candidate lists
+constexpr int FINAL_CAP = 2048;     // entries kept per bracket for ranking threshold-equal keys by index
 constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
 // Optional per-kernel timing with CUDA events on the launching stream.
@@ -67,6 +68,9 @@ struct SelRow {
   u32 lo[MAXC], hi[MAXC];
   u32 above_hi[MAXC];           // #keys >= hi
   double extraE[MAXC];          // energy of listed keys in [lo, T)
+  // which of the keys equal to T are kept: 0 all of them, 1 those with index <= cut, 2 the q lowest
+  // indices as ranked by the chunk-prefix pass (k_tiecount / k_tiescan)
+  u32 tiemode[MAXC], cut[MAXC];
 };
 
 // Decision for one row, consumed by the update kernel.
@@ -77,7 +81,7 @@ struct RowDec {
   int need_tie;    // q < ntie: ties must be ranked by index
   int need_exact;  // the fast comparison could not be certified
   float qL, qinv, qstep;
-  int pad;
+  u32 cut;         // threshold-equal keys are kept up to this index (need_tie == 0)
 };
 
 struct Scratch {
@@ -101,6 +105,8 @@ struct Scratch {
   u32* lcount;     // [rows][MAX_BLK_PER_ROW] entries per segment
   u32* cntpart;    // [rows][MAX_BLK_PER_ROW][MAXC] per-CTA counts of keys >= hi
   double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the threshold prefix
+  u64* fl;         // [rows][MAXC][FINAL_CAP] listed keys sharing the threshold's 22-bit prefix
+  u32* flcnt;      // [rows][MAXC]
   u32* rowflag;    // [rows] 1: the row must take the full radix select (bracket missed or list overflow)
   u32* diffflag;   // [rows] nonzero: some |X-G| differs from |X-Y|
   long long list_row;

@@ -266,3 +266,15 @@ def test_large_row_many_tiles(torch):
     Xs, G0 = S.stress_vectors(2, 2_000_000, blocks=20, period=4, seed=35, device="cpu")
     check_against_oracle(torch, Xs[2].numpy(), G0.numpy(), Xs[1].numpy(),
                          [(TOPK, 2000), (TOPK, 20000), (TOPK, 200000)], 1.0)
+
+
+@pytest.mark.parametrize("d", [5000, 70001, 600000])
+def test_small_tie_groups_at_the_threshold(torch, d):
+    # values on a grid of 1/256: a handful of equal magnitudes at every threshold, of which only the
+    # lowest indices may be kept
+    X, G, Y = S.gaussian_rows(3, d, seed=40 + d % 7)
+    X, G, Y = (np.round(a * 256) / 256 for a in (X, G, Y))
+    X, G, Y = X.astype(F32), G.astype(F32), Y.astype(F32)
+    cands = [(TOPK, max(1, d // 1000)), (TOPK, d // 100), (TOPK, d // 10), (TOPK, d // 2)]
+    for zeta in (0.0, 1.0):
+        check_against_oracle(torch, X, G, Y, cands, zeta)
