@@ -87,7 +87,7 @@ __device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 kr
   u32 sum = 0;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    loc[k] = (k < per) ? hist[nb - 1 - (threadIdx.x * per + k)] : 0;
+    loc[k] = (k < per) ? __ldcg(&hist[nb - 1 - (threadIdx.x * per + k)]) : 0;
     sum += loc[k];
   }
   u32 excl = block_excl_scan(sum, nullptr);
@@ -108,19 +108,67 @@ __device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 kr
   __syncthreads();
 }
 
+// True in exactly one CTA of the row: the one that finishes last.  Every CTA calls it after its
+// global writes; the caller may then read what the other CTAs of the row wrote.  No waiting.
+__device__ __forceinline__ bool last_cta_of_row(u32* ticket, u32 n_ctas) {
+  __shared__ u32 is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == n_ctas - 1u) ? 1u : 0u;
+  __syncthreads();
+  if (is_last) __threadfence();
+  return is_last != 0;
+}
+
 // --------------------------------------------------------------------------
 // radix-select passes
 // --------------------------------------------------------------------------
+// Run by the last CTA of a row's histogram pass: locates every candidate's K-th key in the table.
+template <int PASS>
+__device__ void scan_row(const CsetDev& cs, int row, const u32* __restrict__ hist, SelRow* __restrict__ sel,
+                         bool count_fallback, u32* __restrict__ flags) {
+  __shared__ u32 res[2];
+  if (PASS == 1 && count_fallback && threadIdx.x == 0) atomicAdd(&flags[2], 1u);  // rows sent through the full select
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  SelRow* s = sel + row;
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 K = (u32)cs.param[cs.sel[j]];
+    const u32* h = hist + (long long)row * ((PASS == 1) ? NB : MAXC * NB) + ((PASS == 1) ? 0 : j * NB);
+    const u32 before = (PASS == 1) ? 0u : (PASS == 2 ? s->above1[j] : s->above2[j]);
+    block_find_kth_desc(h, NB, K - before, res);
+    if (threadIdx.x == 0) {
+      if (PASS == 1) {
+        s->b1[j] = res[0];
+        s->above1[j] = res[1];
+      } else if (PASS == 2) {
+        s->p2[j] = (s->b1[j] << 11) | res[0];
+        s->above2[j] = before + res[1];
+      } else {
+        s->T[j] = (s->p2[j] << 9) | res[0];
+        s->above[j] = before + res[1];
+        s->ntie[j] = __ldcg(&h[res[0]]);
+        s->q[j] = K - (before + res[1]);
+        s->extraE[j] = 0.0;
+        s->tiemode[j] = (s->q[j] < s->ntie[j]) ? 2u : 0u;
+        s->cut[j] = 0xffffffffu;
+      }
+    }
+    __syncthreads();
+  }
+}
+
 // PASS 1: histogram of key[30:20] (one table per row) and the row maximum.
 // PASS 2: for every selecting candidate, histogram of key[19:9] over the keys in its pass-1 bin.
 // PASS 3: histogram of key[8:0] over the keys that share its 22-bit prefix.
 template <int PASS, bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const float* __restrict__ G,
-                                              long long d, int nsel, const SelRow* __restrict__ sel,
+                                              long long d, CsetDev cs, SelRow* __restrict__ sel,
                                               u32* __restrict__ hist, u32* __restrict__ maxkey,
-                                              const u32* __restrict__ rowflag) {
+                                              const u32* __restrict__ rowflag, u32* __restrict__ tickets,
+                                              u32* __restrict__ flags) {
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
+  const int nsel = cs.nsel;
   if (rowflag && !rowflag[row]) return;  // single-pass mode: only rows whose bracket failed
   constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
   const int ntab = (PASS == 1) ? 1 : nsel;
@@ -170,41 +218,8 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
     for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if ((threadIdx.x & 31) == 0 && mx) atomicMax(&maxkey[row], mx);
   }
-}
-
-template <int PASS>
-__global__ void __launch_bounds__(TPB) k_scan(CsetDev cs, const u32* __restrict__ hist, SelRow* __restrict__ sel,
-                                              const u32* __restrict__ rowflag, u32* __restrict__ flags) {
-  __shared__ u32 res[2];
-  const int row = blockIdx.x;
-  if (rowflag && !rowflag[row]) return;
-  if (PASS == 1 && rowflag && threadIdx.x == 0) atomicAdd(&flags[2], 1u);  // rows sent through the full select
-  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
-  SelRow* s = sel + row;
-  for (int j = 0; j < cs.nsel; ++j) {
-    const u32 K = (u32)cs.param[cs.sel[j]];
-    const u32* h = hist + (long long)row * ((PASS == 1) ? NB : MAXC * NB) + ((PASS == 1) ? 0 : j * NB);
-    const u32 before = (PASS == 1) ? 0u : (PASS == 2 ? s->above1[j] : s->above2[j]);
-    block_find_kth_desc(h, NB, K - before, res);
-    if (threadIdx.x == 0) {
-      if (PASS == 1) {
-        s->b1[j] = res[0];
-        s->above1[j] = res[1];
-      } else if (PASS == 2) {
-        s->p2[j] = (s->b1[j] << 11) | res[0];
-        s->above2[j] = before + res[1];
-      } else {
-        s->T[j] = (s->p2[j] << 9) | res[0];
-        s->above[j] = before + res[1];
-        s->ntie[j] = h[res[0]];
-        s->q[j] = K - (before + res[1]);
-        s->extraE[j] = 0.0;
-        s->tiemode[j] = (s->q[j] < s->ntie[j]) ? 2u : 0u;
-        s->cut[j] = 0xffffffffu;
-      }
-    }
-    __syncthreads();
-  }
+  if (nsel && last_cta_of_row(&tickets[row * NTICKET + 3 + PASS], gridDim.x))
+    scan_row<PASS>(cs, row, hist, sel, rowflag != nullptr, flags);
 }
 
 // --------------------------------------------------------------------------
@@ -481,12 +496,77 @@ __device__ __forceinline__ void limb_add(u64* limbs, int k, const u32 (&p)[3]) {
   if (p[2]) atomicAdd(&limbs[k + 2], (u64)p[2]);
 }
 
+// Normalised radix-2^32 digits -> nearest binary64 (ties to even); value = digits * 2^-298.
+__device__ double digits_to_double(const u32* dig) {
+  int t = NLIMB - 1;
+  while (t >= 0 && dig[t] == 0) --t;
+  if (t < 0) return 0.0;
+  const u32 hi = dig[t], mid = (t >= 1) ? dig[t - 1] : 0u, lo = (t >= 2) ? dig[t - 2] : 0u;
+  bool sticky = false;
+  for (int i = 0; i < t - 2; ++i) sticky |= (dig[i] != 0);
+  const unsigned __int128 W = ((unsigned __int128)hi << 64) | ((unsigned __int128)mid << 32) | lo;
+  const int nb = 32 - __clz(hi);         // significant bits of hi
+  const int sh = nb + 11;                // keep 53 of the 64+nb bits
+  u64 mant = (u64)(W >> sh);
+  const bool rnd = (W >> (sh - 1)) & 1;
+  sticky |= (W & (((unsigned __int128)1 << (sh - 1)) - 1)) != 0;
+  if (rnd && (sticky || (mant & 1))) ++mant;
+  return ldexp((double)mant, sh + 32 * (t - 2) - 298);
+}
+
+// Run by one thread of the last CTA of the exact pass: carries, rounds and decides the row.
+__device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* __restrict__ limbs,
+                               const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                               RowDec* __restrict__ dec, const CompressOut& out,
+                               const u32* __restrict__ diffflag, u32* __restrict__ flags) {
+  double val[NSLOT];
+  if (__ldcg(&diffflag[row]) & 0x80000000u) {  // X - Y is not finite
+    for (int s = 0; s < NSLOT; ++s) val[s] = 0.0;
+    atomicOr(&flags[0], 1u);
+    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, val + 1, 0.0);
+    return;
+  }
+  for (int s = 0; s < 2 + cs.m; ++s) {
+    u32 dig[NLIMB];
+    const u64* l = limbs + ((long long)row * NSLOT + s) * NLIMB;
+    unsigned __int128 tie = 0;
+    int tk = 0;
+    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
+      int j = 0;
+      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
+      const u32 T = sel[row].T[j];
+      const u32 ex = T >> 23, fr = T & 0x7fffffu;
+      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
+      const int off = 2 * (int)(ex ? ex : 1u) - 2;
+      tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
+      tk = off >> 5;
+    }
+    u64 carry = 0;
+    for (int k = 0; k < NLIMB; ++k) {
+      u64 add = 0;
+      if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
+      const unsigned __int128 tsum = (unsigned __int128)__ldcg(&l[k]) + carry + add;
+      dig[k] = (u32)tsum;
+      carry = (u64)(tsum >> 32);
+    }
+    val[s] = digits_to_double(dig);
+    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) val[s] = 0.0;
+  }
+  const double D = val[0];
+  const double rhs = (double)cs.zeta * D;
+  int level = cs.m;
+  for (int j = 0; j <= cs.m; ++j)
+    if (val[1 + j] <= rhs) { level = j; break; }
+  finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
+}
+
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X, const float* __restrict__ G,
                                                     const float* __restrict__ Y, long long d, CsetDev cs,
                                                     const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                                                    const RowDec* __restrict__ dec, u64* __restrict__ limbs,
-                                                    u32* __restrict__ diffflag) {
+                                                    RowDec* __restrict__ dec, u64* __restrict__ limbs,
+                                                    u32* __restrict__ diffflag, long long d_full, CompressOut out,
+                                                    u32* __restrict__ tickets, u32* __restrict__ flags) {
   const int row = blockIdx.y;
   if (!dec[row].need_exact) return;
   __shared__ u64 sh[NSLOT * NLIMB];
@@ -535,70 +615,8 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
     if (vlo) atomicAdd(&gl[i], vlo);
     if (vhi && (i % NLIMB) + 1 < NLIMB) atomicAdd(&gl[i + 1], vhi);
   }
-}
-
-// Normalised radix-2^32 digits -> nearest binary64 (ties to even); value = digits * 2^-298.
-__device__ double digits_to_double(const u32* dig) {
-  int t = NLIMB - 1;
-  while (t >= 0 && dig[t] == 0) --t;
-  if (t < 0) return 0.0;
-  const u32 hi = dig[t], mid = (t >= 1) ? dig[t - 1] : 0u, lo = (t >= 2) ? dig[t - 2] : 0u;
-  bool sticky = false;
-  for (int i = 0; i < t - 2; ++i) sticky |= (dig[i] != 0);
-  const unsigned __int128 W = ((unsigned __int128)hi << 64) | ((unsigned __int128)mid << 32) | lo;
-  const int nb = 32 - __clz(hi);         // significant bits of hi
-  const int sh = nb + 11;                // keep 53 of the 64+nb bits
-  u64 mant = (u64)(W >> sh);
-  const bool rnd = (W >> (sh - 1)) & 1;
-  sticky |= (W & (((unsigned __int128)1 << (sh - 1)) - 1)) != 0;
-  if (rnd && (sticky || (mant & 1))) ++mant;
-  return ldexp((double)mant, sh + 32 * (t - 2) - 298);
-}
-
-__global__ void k_pick_exact(CsetDev cs, long long d, const u64* __restrict__ limbs, const SelRow* __restrict__ sel,
-                             const u32* __restrict__ maxkey, RowDec* __restrict__ dec, CompressOut out,
-                             const u32* __restrict__ diffflag, u32* __restrict__ flags) {
-  const int row = blockIdx.x;
-  if (threadIdx.x != 0 || !dec[row].need_exact) return;
-  double val[NSLOT];
-  if (diffflag[row] & 0x80000000u) {  // X - Y is not finite
-    for (int s = 0; s < NSLOT; ++s) val[s] = 0.0;
-    atomicOr(&flags[0], 1u);
-    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, val + 1, 0.0);
-    return;
-  }
-  for (int s = 0; s < 2 + cs.m; ++s) {
-    u32 dig[NLIMB];
-    const u64* l = limbs + ((long long)row * NSLOT + s) * NLIMB;
-    unsigned __int128 tie = 0;
-    int tk = 0;
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
-      int j = 0;
-      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
-      const u32 T = sel[row].T[j];
-      const u32 ex = T >> 23, fr = T & 0x7fffffu;
-      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
-      const int off = 2 * (int)(ex ? ex : 1u) - 2;
-      tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
-      tk = off >> 5;
-    }
-    u64 carry = 0;
-    for (int k = 0; k < NLIMB; ++k) {
-      u64 add = 0;
-      if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
-      const unsigned __int128 tsum = (unsigned __int128)l[k] + carry + add;
-      dig[k] = (u32)tsum;
-      carry = (u64)(tsum >> 32);
-    }
-    val[s] = digits_to_double(dig);
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) val[s] = 0.0;
-  }
-  const double D = val[0];
-  const double rhs = (double)cs.zeta * D;
-  int level = cs.m;
-  for (int j = 0; j <= cs.m; ++j)
-    if (val[1 + j] <= rhs) { level = j; break; }
-  finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
+  if (last_cta_of_row(&tickets[row * NTICKET + 7], gridDim.x) && threadIdx.x == 0)
+    pick_exact_row(cs, row, d_full, limbs, sel, maxkey, dec, out, diffflag, flags);
 }
 
 // --------------------------------------------------------------------------
@@ -607,7 +625,8 @@ __global__ void k_pick_exact(CsetDev cs, long long d, const u64* __restrict__ li
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, const float* __restrict__ G,
                                                   long long d, const RowDec* __restrict__ dec,
-                                                  u32* __restrict__ tiecnt, long long nchunk) {
+                                                  u32* __restrict__ tiecnt, long long nchunk,
+                                                  u32* __restrict__ tickets) {
   const int row = blockIdx.y;
   if (!dec[row].need_tie) return;
   const u32 T = dec[row].T;
@@ -626,17 +645,13 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
     block_excl_scan(cnt, &total);
     if (threadIdx.x == 0) tiecnt[(long long)row * nchunk + chunk] = total;
   }
-}
-
-__global__ void __launch_bounds__(TPB) k_tiescan(const RowDec* __restrict__ dec, u32* __restrict__ tiecnt,
-                                                 long long nchunk) {
-  const int row = blockIdx.x;
-  if (!dec[row].need_tie) return;
+  if (!last_cta_of_row(&tickets[row * NTICKET + 8], gridDim.x)) return;
+  // exclusive prefix over the row's chunks
   u32* t = tiecnt + (long long)row * nchunk;
   u32 carry = 0;
   for (long long base = 0; base < nchunk; base += TPB) {
     const long long i = base + threadIdx.x;
-    const u32 v = (i < nchunk) ? t[i] : 0u;
+    const u32 v = (i < nchunk) ? __ldcg(&t[i]) : 0u;
     u32 total;
     const u32 ex = block_excl_scan(v, &total);
     if (i < nchunk) t[i] = carry + ex;
@@ -801,13 +816,87 @@ __global__ void k_copy_report(int rows, long long d, int m, CompressOut out) {
 // --------------------------------------------------------------------------
 // single-pass path: brackets from a sample, one streaming pass, selection on short lists
 // --------------------------------------------------------------------------
+// Finds the bin holding the r-th largest sampled key (1-based); all TPB threads call.
+// csum/cexcl: counts and exclusive prefixes of the 256 chunks of 256 bins, in descending bin order.
+__device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, const u32* cexcl, u32 r, u32* out) {
+  __shared__ int chunk_sh;
+  if (cexcl[threadIdx.x] < r && r <= cexcl[threadIdx.x] + csum[threadIdx.x]) chunk_sh = threadIdx.x;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    const int c = chunk_sh;
+    const int pos0 = 256 * c + 8 * lane;                       // descending position of this lane's first bin
+    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 8 - pos0));
+    const uint4 a = __ldcg(p), b = __ldcg(p + 1);              // ascending addresses: positions pos0+7 .. pos0
+    const u32 v[8] = {b.w, b.z, b.y, b.x, a.w, a.z, a.y, a.x}; // v[k] = bin at descending position pos0 + k
+    u32 lsum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) lsum += v[k];
+    u32 inc = lsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    u32 run = cexcl[c] + inc - lsum;
+    if (run < r && r <= run + lsum) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (r > run && r <= run + v[k]) *out = (u32)(SBINS - 1 - (pos0 + k));
+        run += v[k];
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
+// holds the K-th largest key with overwhelming probability (checked exactly afterwards).
+__device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sample,
+                            const u32* __restrict__ shist, SelRow* __restrict__ sel) {
+  __shared__ u32 csum[TPB], cexcl[TPB];
+  __shared__ u32 res;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32* h = shist + (long long)row * SBINS;
+  for (int c = wid; c < 256; c += TPB / 32) {
+    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 256 * (c + 1))) + 2 * lane;
+    const uint4 a = __ldcg(p), b = __ldcg(p + 1);
+    const u32 t = warp_sum_u32(a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w);
+    if (lane == 0) csum[c] = t;
+  }
+  __syncthreads();
+  u32 S;
+  const u32 ex = block_excl_scan(csum[threadIdx.x], &S);
+  cexcl[threadIdx.x] = ex;
+  __syncthreads();
+  for (int j = 0; j < cs.nsel; ++j) {
+    const double K = (double)cs.param[cs.sel[j]];
+    const double r = K * (double)S / (double)d;
+    const double dev = full_sample ? 0.0 : 6.0 * sqrt(r * (1.0 - K / (double)d)) + 8.0;
+    const double r_hi = floor(r - dev), r_lo = ceil(r + dev) + 1.0;
+    u32 hi = 0x80000000u, lo = 0u;
+    if (r_hi >= 1.0) {
+      sample_rank_bin(h, csum, cexcl, (u32)r_hi, &res);
+      hi = (res + 1u) << 15;
+      __syncthreads();
+    }
+    if (r_lo <= (double)S) {
+      sample_rank_bin(h, csum, cexcl, (u32)r_lo, &res);
+      lo = res << 15;
+    }
+    if (threadIdx.x == 0) { sel[row].lo[j] = lo; sel[row].hi[j] = hi; }
+    __syncthreads();
+  }
+}
+
 // Every `stride`-th tile of a row is sampled; the histogram has one bin per value of
 // key[30:15].  Per-CTA counts are 16 bit (two bins per shared word), so a CTA takes at most
 // 63 tiles.
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
                                                 long long d, long long nsamp, long long stride,
-                                                u32* __restrict__ shist) {
+                                                u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
+                                                u32* __restrict__ tickets) {
   extern __shared__ u32 sh[];  // SBINS / 2 words
   const int row = blockIdx.y;
   for (int i = threadIdx.x; i < SBINS / 2; i += TPB) sh[i] = 0;
@@ -835,80 +924,8 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
     if (w & 0xffffu) atomicAdd(&gh[2 * i], w & 0xffffu);
     if (w >> 16) atomicAdd(&gh[2 * i + 1], w >> 16);
   }
-}
-
-// Finds the bin holding the r-th largest sampled key (1-based); all TPB threads call.
-// csum/cexcl: counts and exclusive prefixes of the 256 chunks of 256 bins, in descending bin order.
-__device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, const u32* cexcl, u32 r, u32* out) {
-  __shared__ int chunk_sh;
-  if (cexcl[threadIdx.x] < r && r <= cexcl[threadIdx.x] + csum[threadIdx.x]) chunk_sh = threadIdx.x;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    const int c = chunk_sh;
-    const int pos0 = 256 * c + 8 * lane;                       // descending position of this lane's first bin
-    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 8 - pos0));
-    const uint4 a = p[0], b = p[1];                            // ascending addresses: positions pos0+7 .. pos0
-    const u32 v[8] = {b.w, b.z, b.y, b.x, a.w, a.z, a.y, a.x}; // v[k] = bin at descending position pos0 + k
-    u32 lsum = 0;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) lsum += v[k];
-    u32 inc = lsum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    u32 run = cexcl[c] + inc - lsum;
-    if (run < r && r <= run + lsum) {
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (r > run && r <= run + v[k]) *out = (u32)(SBINS - 1 - (pos0 + k));
-        run += v[k];
-      }
-    }
-  }
-  __syncthreads();
-}
-
-// Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
-// holds the K-th largest key with overwhelming probability (checked exactly afterwards).
-__global__ void __launch_bounds__(TPB) k_bracket(CsetDev cs, long long d, int full_sample,
-                                                 const u32* __restrict__ shist, SelRow* __restrict__ sel) {
-  __shared__ u32 csum[TPB], cexcl[TPB];
-  __shared__ u32 res;
-  const int row = blockIdx.x;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const u32* h = shist + (long long)row * SBINS;
-  for (int c = wid; c < 256; c += TPB / 32) {
-    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 256 * (c + 1))) + 2 * lane;
-    const uint4 a = p[0], b = p[1];
-    const u32 t = warp_sum_u32(a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w);
-    if (lane == 0) csum[c] = t;
-  }
-  __syncthreads();
-  u32 S;
-  const u32 ex = block_excl_scan(csum[threadIdx.x], &S);
-  cexcl[threadIdx.x] = ex;
-  __syncthreads();
-  for (int j = 0; j < cs.nsel; ++j) {
-    const double K = (double)cs.param[cs.sel[j]];
-    const double r = K * (double)S / (double)d;
-    const double dev = full_sample ? 0.0 : 6.0 * sqrt(r * (1.0 - K / (double)d)) + 8.0;
-    const double r_hi = floor(r - dev), r_lo = ceil(r + dev) + 1.0;
-    u32 hi = 0x80000000u, lo = 0u;
-    if (r_hi >= 1.0) {
-      sample_rank_bin(h, csum, cexcl, (u32)r_hi, &res);
-      hi = (res + 1u) << 15;
-      __syncthreads();
-    }
-    if (r_lo <= (double)S) {
-      sample_rank_bin(h, csum, cexcl, (u32)r_lo, &res);
-      lo = res << 15;
-    }
-    if (threadIdx.x == 0) { sel[row].lo[j] = lo; sel[row].hi[j] = hi; }
-    __syncthreads();
-  }
+  if (last_cta_of_row(&tickets[row * NTICKET + 0], gridDim.x))
+    bracket_row(cs, row, d, stride == 1 ? 1 : 0, shist, sel);
 }
 
 // The streaming pass: D, ||v||^2, per bracket the count of keys >= hi and the energy of keys
@@ -1047,17 +1064,124 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   }
 }
 
+// Run by the last CTA of a row's list pass.
+template <int PASS>
+__device__ void lscan_row(const CsetDev& cs, int row, int nblk, int nlb, const u32* __restrict__ hist,
+                          const u32* __restrict__ cntpart, const double* __restrict__ lepart,
+                          SelRow* __restrict__ sel, u32* __restrict__ rowflag,
+                          const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
+  __shared__ u32 res[2];
+  __shared__ u32 bad;
+  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  SelRow* s = sel + row;
+  if (PASS == 1) {
+    // exact check of every bracket: the K-th largest key must be one of the listed keys
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    for (int j = 0; j < cs.nsel; ++j) {
+      u32 a = 0, tot = 0;
+      for (int b = threadIdx.x; b < nblk; b += TPB) a += cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j];
+      const u32* h = hist + ((long long)row * MAXC + j) * NB;
+      for (int b = threadIdx.x; b < NB; b += TPB) tot += __ldcg(&h[b]);
+      u32 above, total;
+      block_excl_scan(a, &above);
+      block_excl_scan(tot, &total);
+      if (threadIdx.x == 0) {
+        const long long K = cs.param[cs.sel[j]];
+        s->above_hi[j] = above;
+        if (K <= (long long)above || K > (long long)above + (long long)total) bad = 1;
+      }
+    }
+    __syncthreads();
+    if (bad) {
+      if (threadIdx.x == 0) rowflag[row] = 1;
+      return;
+    }
+  }
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 K = (u32)cs.param[cs.sel[j]];
+    const u32* h = hist + ((long long)row * MAXC + j) * NB;
+    const u32 before = (PASS == 1) ? s->above_hi[j] : (PASS == 2 ? s->above1[j] : s->above2[j]);
+    block_find_kth_desc(h, NB, K - before, res);
+    if (PASS == 3) {
+      // energy of the keys that share the 22-bit prefix and lie below the threshold: each bin is one key value
+      double a = 0.0;
+      for (int b = threadIdx.x; b < (int)res[0]; b += TPB) {
+        const double kv = (double)__uint_as_float((s->p2[j] << 9) | (u32)b);
+        a += (double)__ldcg(&h[b]) * (kv * kv);
+      }
+      __shared__ double redd[TPB / 32];
+      a = warp_sum_f64(a);
+      __syncthreads();
+      if ((threadIdx.x & 31) == 0) redd[threadIdx.x >> 5] = a;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        double e = 0.0;
+        for (int b = 0; b < nlb; ++b) e += __ldcg(&lepart[((long long)row * LIST_BLK + b) * MAXC + j]);
+        for (int w = 0; w < TPB / 32; ++w) e += redd[w];
+        s->extraE[j] = e;
+      }
+    }
+    if (threadIdx.x == 0) {
+      if (PASS == 1) {
+        s->b1[j] = res[0];
+        s->above1[j] = before + res[1];
+      } else if (PASS == 2) {
+        s->p2[j] = (s->b1[j] << 11) | res[0];
+        s->above2[j] = before + res[1];
+      } else {
+        s->T[j] = (s->p2[j] << 9) | res[0];
+        s->above[j] = before + res[1];
+        s->ntie[j] = __ldcg(&h[res[0]]);
+        s->q[j] = K - (before + res[1]);
+      }
+    }
+    __syncthreads();
+    if (PASS == 3) {
+      // Which threshold-equal keys are kept: the q with the lowest indices.  They are all among the
+      // collected prefix-equal entries; the q-th smallest of their indices is the cut.
+      __shared__ u32 ties[1024];
+      __shared__ u32 nties_sh;
+      const u32 T = s->T[j], q = s->q[j], ntie = s->ntie[j];
+      const u32 nfl = __ldcg(&flcnt[row * MAXC + j]);
+      if (q == ntie) {
+        if (threadIdx.x == 0) { s->tiemode[j] = 0u; s->cut[j] = 0xffffffffu; }
+      } else if (nfl > FINAL_CAP || ntie > 1024u) {
+        if (threadIdx.x == 0) { s->tiemode[j] = 2u; s->cut[j] = 0xffffffffu; }
+      } else {
+        if (threadIdx.x == 0) nties_sh = 0;
+        __syncthreads();
+        const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
+        for (u32 i = threadIdx.x; i < nfl; i += TPB) {
+          const u64 ent = __ldcg(&f[i]);
+          if ((u32)(ent >> 32) == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)ent;
+        }
+        __syncthreads();
+        for (u32 i = threadIdx.x; i < ntie; i += TPB) {
+          const u32 mine = ties[i];
+          u32 rank = 0;
+          for (u32 k = 0; k < ntie; ++k) rank += (ties[k] < mine) ? 1u : 0u;
+          if (rank == q - 1u) { s->tiemode[j] = 1u; s->cut[j] = mine; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
 // Passes over the listed keys.  PASS 1: per bracket, histogram of key[30:20];
 // PASS 2: key[19:9] of the keys in the bracket's first-digit bin; PASS 3: key[8:0] of the keys
 // sharing the 22-bit prefix, plus the energy of the bracket's keys below that prefix.
 template <int PASS>
-__global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow* __restrict__ sel,
+__global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __restrict__ sel,
                                                const u64* __restrict__ list, const u32* __restrict__ lcount,
                                                long long list_row, u32 segcap, u32* __restrict__ hist,
-                                               double* __restrict__ lepart, const u32* __restrict__ rowflag,
-                                               u64* __restrict__ fl, u32* __restrict__ flcnt) {
+                                               double* __restrict__ lepart, u32* __restrict__ rowflag,
+                                               u64* __restrict__ fl, u32* __restrict__ flcnt,
+                                               const u32* __restrict__ cntpart, u32* __restrict__ tickets) {
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
+  const int nsel = cs.nsel;
   if (rowflag[row]) return;
   constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
   for (int i = threadIdx.x; i < nsel * NB; i += TPB) sh[i] = 0;
@@ -1115,112 +1239,8 @@ __global__ void __launch_bounds__(TPB) k_lhist(int nsel, int nseg, const SelRow*
       lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
     }
   }
-}
-
-template <int PASS>
-__global__ void __launch_bounds__(TPB) k_lscan(CsetDev cs, int nblk, int nlb, const u32* __restrict__ hist,
-                                               const u32* __restrict__ cntpart, const double* __restrict__ lepart,
-                                               SelRow* __restrict__ sel, u32* __restrict__ rowflag,
-                                               const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
-  __shared__ u32 res[2];
-  __shared__ u32 bad;
-  const int row = blockIdx.x;
-  if (rowflag[row]) return;  // uniform: written by earlier kernels only
-  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
-  SelRow* s = sel + row;
-  if (PASS == 1) {
-    // exact check of every bracket: the K-th largest key must be one of the listed keys
-    if (threadIdx.x == 0) bad = 0;
-    __syncthreads();
-    for (int j = 0; j < cs.nsel; ++j) {
-      u32 a = 0, tot = 0;
-      for (int b = threadIdx.x; b < nblk; b += TPB) a += cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j];
-      const u32* h = hist + ((long long)row * MAXC + j) * NB;
-      for (int b = threadIdx.x; b < NB; b += TPB) tot += h[b];
-      u32 above, total;
-      block_excl_scan(a, &above);
-      block_excl_scan(tot, &total);
-      if (threadIdx.x == 0) {
-        const long long K = cs.param[cs.sel[j]];
-        s->above_hi[j] = above;
-        if (K <= (long long)above || K > (long long)above + (long long)total) bad = 1;
-      }
-    }
-    __syncthreads();
-    if (bad) {
-      if (threadIdx.x == 0) rowflag[row] = 1;
-      return;
-    }
-  }
-  for (int j = 0; j < cs.nsel; ++j) {
-    const u32 K = (u32)cs.param[cs.sel[j]];
-    const u32* h = hist + ((long long)row * MAXC + j) * NB;
-    const u32 before = (PASS == 1) ? s->above_hi[j] : (PASS == 2 ? s->above1[j] : s->above2[j]);
-    block_find_kth_desc(h, NB, K - before, res);
-    if (PASS == 3) {
-      // energy of the keys that share the 22-bit prefix and lie below the threshold: each bin is one key value
-      double a = 0.0;
-      for (int b = threadIdx.x; b < (int)res[0]; b += TPB) {
-        const double kv = (double)__uint_as_float((s->p2[j] << 9) | (u32)b);
-        a += (double)h[b] * (kv * kv);
-      }
-      __shared__ double redd[TPB / 32];
-      a = warp_sum_f64(a);
-      __syncthreads();
-      if ((threadIdx.x & 31) == 0) redd[threadIdx.x >> 5] = a;
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        double e = 0.0;
-        for (int b = 0; b < nlb; ++b) e += lepart[((long long)row * LIST_BLK + b) * MAXC + j];
-        for (int w = 0; w < TPB / 32; ++w) e += redd[w];
-        s->extraE[j] = e;
-      }
-    }
-    if (threadIdx.x == 0) {
-      if (PASS == 1) {
-        s->b1[j] = res[0];
-        s->above1[j] = before + res[1];
-      } else if (PASS == 2) {
-        s->p2[j] = (s->b1[j] << 11) | res[0];
-        s->above2[j] = before + res[1];
-      } else {
-        s->T[j] = (s->p2[j] << 9) | res[0];
-        s->above[j] = before + res[1];
-        s->ntie[j] = h[res[0]];
-        s->q[j] = K - (before + res[1]);
-      }
-    }
-    __syncthreads();
-    if (PASS == 3) {
-      // Which threshold-equal keys are kept: the q with the lowest indices.  They are all among the
-      // collected prefix-equal entries; the q-th smallest of their indices is the cut.
-      __shared__ u32 ties[1024];
-      __shared__ u32 nties_sh;
-      const u32 T = s->T[j], q = s->q[j], ntie = s->ntie[j];
-      const u32 nfl = flcnt[row * MAXC + j];
-      if (q == ntie) {
-        if (threadIdx.x == 0) { s->tiemode[j] = 0u; s->cut[j] = 0xffffffffu; }
-      } else if (nfl > FINAL_CAP || ntie > 1024u) {
-        if (threadIdx.x == 0) { s->tiemode[j] = 2u; s->cut[j] = 0xffffffffu; }
-      } else {
-        if (threadIdx.x == 0) nties_sh = 0;
-        __syncthreads();
-        const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
-        for (u32 i = threadIdx.x; i < nfl; i += TPB) {
-          const u64 ent = f[i];
-          if ((u32)(ent >> 32) == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)ent;
-        }
-        __syncthreads();
-        for (u32 i = threadIdx.x; i < ntie; i += TPB) {
-          const u32 mine = ties[i];
-          u32 rank = 0;
-          for (u32 k = 0; k < ntie; ++k) rank += (ties[k] < mine) ? 1u : 0u;
-          if (rank == q - 1u) { s->tiemode[j] = 1u; s->cut[j] = mine; }
-        }
-      }
-      __syncthreads();
-    }
-  }
+  if (last_cta_of_row(&tickets[row * NTICKET + PASS], gridDim.x))
+    lscan_row<PASS>(cs, row, nseg, (int)gridDim.x, hist, cntpart, lepart, sel, rowflag, fl, flcnt);
 }
 
 // --------------------------------------------------------------------------
@@ -1232,7 +1252,7 @@ static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; 
 
 struct Layout {
   size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
-  size_t rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, fl, flcnt;
+  size_t tickets, rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, fl, flcnt;
   long long list_row;
 };
 
@@ -1252,6 +1272,7 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.limbs = o; o = align_up(o + (size_t)rows * NSLOT * NLIMB * 8, 256);
   L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
+  L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
   L.shist = L.lhist1 = L.flcnt = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
@@ -1299,6 +1320,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->tiecnt = (u32*)(b + L.tiecnt);
   s->rowflag = (u32*)(b + L.rowflag);
   s->diffflag = (u32*)(b + L.diffflag);
+  s->tickets = (u32*)(b + L.tickets);
   s->shist = s->lhist1 = s->lcount = s->cntpart = nullptr;
   s->list = nullptr;
   s->lepart = nullptr;
@@ -1417,9 +1439,11 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
   double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
 
-#define TIMED_HIST(id, PASS, shm, hist)                                                                           \
-  TIMED(id, if (al) k_hist<PASS, true><<<fgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only); \
-            else k_hist<PASS, false><<<fgrid, TPB, shm, stream>>>(X, G, d, cs.nsel, s.sel, hist, s.maxkey, only))
+#define TIMED_HIST(id, PASS, shm, hist)                                                                        \
+  TIMED(id, if (al) k_hist<PASS, true><<<fgrid, TPB, shm, stream>>>(X, G, d, cs, s.sel, hist, s.maxkey, only,    \
+                                                                    s.tickets, s.flags);                         \
+            else k_hist<PASS, false><<<fgrid, TPB, shm, stream>>>(X, G, d, cs, s.sel, hist, s.maxkey, only,      \
+                                                                  s.tickets, s.flags))
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
     if (al) k_pass1<N, true><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
@@ -1427,16 +1451,19 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     else k_pass1<N, false><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,          \
                                                       s.lcount, s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag); \
     break;
+#define LIST_PASS(PASS, shm, hist)                                                                                \
+  TIMED(KID_LHIST, (k_lhist<PASS><<<lgrid, TPB, shm, stream>>>(cs, nblk, s.sel, s.list, s.lcount, s.list_row,     \
+                                                               segcap, hist, s.lepart, s.rowflag, s.fl, s.flcnt,  \
+                                                               s.cntpart, s.tickets)))
 
   if (single) {
-    // 1. brackets for every Top-K threshold from a sample of the row
+    // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
     long long stride = ntile / 128;
     if (stride < 1) stride = 1;
     if (stride > 32) stride = 32;
     const long long nsamp = ntile / stride;
     const dim3 samp_grid((unsigned)((nsamp + 15) / 16), rows);
-    TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist);
-    TIMED(KID_BRACKET, (k_bracket<<<rows, TPB, 0, stream>>>(cs, d, stride == 1 ? 1 : 0, s.shist, s.sel)));
+    TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist, cs, s.sel, s.tickets);
     // 2. the one pass over X, G, Y
     const u32 segcap = (u32)(s.list_row / nblk);
     prof_begin(pf, KID_PASS1, stream);
@@ -1446,40 +1473,30 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     }
     prof_end(pf, stream);
     ++launches;
-    // 3. exact selection among the listed keys
+    // 3. exact selection among the listed keys: three digit passes, each finished by its last CTA
     const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
-    TIMED(KID_LHIST, (k_lhist<1><<<lgrid, TPB, cs.nsel * BINS1 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.lhist1, s.lepart, s.rowflag, s.fl, s.flcnt)));
-    TIMED(KID_LSCAN, (k_lscan<1><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.lhist1, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
-    TIMED(KID_LHIST, (k_lhist<2><<<lgrid, TPB, cs.nsel * BINS2 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist2, s.lepart, s.rowflag, s.fl, s.flcnt)));
-    TIMED(KID_LSCAN, (k_lscan<2><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist2, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
-    TIMED(KID_LHIST, (k_lhist<3><<<lgrid, TPB, cs.nsel * BINS3 * 4, stream>>>(cs.nsel, nblk, s.sel, s.list, s.lcount, s.list_row, segcap, s.hist3, s.lepart, s.rowflag, s.fl, s.flcnt)));
-    TIMED(KID_LSCAN, (k_lscan<3><<<rows, TPB, 0, stream>>>(cs, nblk, (int)lgrid.x, s.hist3, s.cntpart, s.lepart, s.sel, s.rowflag, s.fl, s.flcnt)));
+    LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
+    LIST_PASS(2, cs.nsel * BINS2 * 4, s.hist2);
+    LIST_PASS(3, cs.nsel * BINS3 * 4, s.hist3);
     tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
   }
   // the full radix select: every row, or (single-pass mode) only rows whose bracket failed
-  if (cs.nsel || cs.nquant) {
-    if (!single) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
-    else if (cs.nsel) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
-  }
+  if (cs.nsel || cs.nquant) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
   if (cs.nsel) {
-    TIMED(KID_SCAN, (k_scan<1><<<rows, TPB, 0, stream>>>(cs, s.hist1, s.sel, only, s.flags)));
     TIMED_HIST(KID_HIST2, 2, cs.nsel * BINS2 * 4, s.hist2);
-    TIMED(KID_SCAN, (k_scan<2><<<rows, TPB, 0, stream>>>(cs, s.hist2, s.sel, only, s.flags)));
     TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
-    TIMED(KID_SCAN, (k_scan<3><<<rows, TPB, 0, stream>>>(cs, s.hist3, s.sel, only, s.flags)));
   }
   TIMED_AL(KID_ENERGY, k_energy, fgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
   if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
   TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey, s.dec, s.flags, out, s.diffflag, single ? 1 : 0, tol)));
-  TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag);
-  TIMED(KID_EXACT, (k_pick_exact<<<rows, 32, 0, stream>>>(cs, d, s.limbs, s.sel, s.maxkey, s.dec, out, s.diffflag, s.flags)));
+  TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag, d, out, s.tickets, s.flags);
   if (cs.nsel) {
     long long tgx = (148 * 4 + rows - 1) / rows;
     if (tgx > nchunk) tgx = nchunk;
-    TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk);
-    TIMED(KID_TIE, (k_tiescan<<<rows, TPB, 0, stream>>>(s.dec, s.tiecnt, nchunk)));
+    TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk, s.tickets);
   }
   TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+#undef LIST_PASS
 #undef PASS1_CASE
 #undef TIMED_HIST
 #undef TIMED_AL

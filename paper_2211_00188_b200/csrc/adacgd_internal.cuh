@@ -22,6 +22,7 @@ constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (als
 constexpr int MAX_BLK_PER_ROW = 2048;
 constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
 constexpr int LIST_BLK = 256;       // CTAs per row of the passes over the candidate lists
+constexpr int NTICKET = 12;         // per-row completion counters: 0 sample, 1-3 list passes, 4-6 full passes, 7 exact, 8 ties
 constexpr int FINAL_CAP = 2048;     // entries kept per bracket for ranking threshold-equal keys by index
 constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
@@ -107,6 +108,7 @@ struct Scratch {
   double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the threshold prefix
   u64* fl;         // [rows][MAXC][FINAL_CAP] listed keys sharing the threshold's 22-bit prefix
   u32* flcnt;      // [rows][MAXC]
+  u32* tickets;    // [rows][NTICKET]
   u32* rowflag;    // [rows] 1: the row must take the full radix select (bracket missed or list overflow)
   u32* diffflag;   // [rows] nonzero: some |X-G| differs from |X-Y|
   long long list_row;
