@@ -454,6 +454,7 @@ __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_m
     const bool e_ok = (E >= tiny && E <= 1.7e308);
     int verdict;  // 1 true, 0 false, -1 unsure
     if (by_def) verdict = 1;
+    else if (!(D <= 1.7e308)) verdict = -1;  // overflowed chain or non-finite X - Y: the exact pass tells which
     else if (j == 0 && single_pass && (diffflag[row] & 0x7fffffffu) == 0 && d_ok)
       verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
     else if (!e_ok) verdict = -1;
@@ -664,7 +665,7 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
 // row's operands are loaded before the current row is written back.
 constexpr int UPD_ROW_TILE = 32;
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
+__global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
                                                 CompressOut out) {
@@ -673,7 +674,7 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
   const bool live = c0 < d;
   const int lane = threadIdx.x & 31;
   const bool want_mean = out.mean_out != nullptr;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float acc[4] = {-0.f, -0.f, -0.f, -0.f};  // -0 + g == g bit for bit, so the first row needs no special case
   for (int r0 = 0; r0 < rows; r0 += UPD_ROW_TILE) {
     const int nr = (rows - r0 < UPD_ROW_TILE) ? rows - r0 : UPD_ROW_TILE;
     __syncthreads();
@@ -684,6 +685,48 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
       shd[threadIdx.x] = t;
     }
     __syncthreads();
+    // Common case for the whole tile of rows: every row either skips or applies a Top-K level whose
+    // threshold-equal keys are decided by the index cut, and no kept-index list is wanted.
+    bool simple = true;
+    if (threadIdx.x < nr) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
+    simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
+    if (simple) {
+      float sg[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
+      if (live) {
+        if (shd[0].mode != 0 || want_mean) load4<ALIGNED>(G + (long long)r0 * d, c0, d, sg);
+        if (shd[0].mode != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, sx);
+      }
+      for (int ii = 0; ii < nr; ++ii) {
+        const int i = r0 + ii;
+        float g[4], x[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { g[k] = sg[k]; x[k] = sx[k]; }
+        if (ii + 1 < nr && live) {
+          const int m1 = shd[ii + 1].mode;
+          if (m1 != 0 || want_mean) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, sg);
+          if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, sx);
+        }
+        if (shd[ii].mode != 0) {
+          const u32 T = shd[ii].T, cut = shd[ii].cut;
+          bool any = false;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float v = __fsub_rn(x[k], g[k]);
+            const u32 key = key_of(v);
+            const bool kept = (key > T) || (key == T && (u32)c0 + (u32)k <= cut);
+            g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+            any = any || kept;
+          }
+          // dead lanes hold zeros: they are kept only when T == 0, and never stored
+          if (any && live) store4<ALIGNED>(G + (long long)i * d, c0, d, g);
+        }
+        if (want_mean) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+        }
+      }
+      continue;
+    }
     float gn[4] = {0.f, 0.f, 0.f, 0.f}, xn[4] = {0.f, 0.f, 0.f, 0.f};
     if (live) {
       const int m0 = shd[0].mode;
@@ -790,7 +833,7 @@ __global__ void __launch_bounds__(TPB) k_update(const float* __restrict__ X, flo
       }
       if (want_mean) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) acc[k] = (i == 0) ? g[k] : __fadd_rn(acc[k], g[k]);
+        for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
       }
     }
   }
@@ -956,7 +999,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   }
   float fD = 0.f, fE = 0.f;
   double dD = 0.0, dE = 0.0;
-  u32 mx = 0, mxw = 0, df = 0;
+  u32 mx = 0, df = 0;
   __syncthreads();
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
@@ -973,17 +1016,19 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       load4<ALIGNED>(gr, c0, d, g);
       load4<ALIGNED>(yr, c0, d, y);
     }
+    u32 keys[4];
+    u32 im = 0;  // which of the four entries fall inside a bracket
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const bool ok = live && (ALIGNED || c0 + k < d);
       const float v = __fsub_rn(x[k], g[k]);
       const float w = __fsub_rn(x[k], y[k]);
       fE = fmaf(v, v, fE);
       fD = fmaf(w, w, fD);
-      const u32 key = key_of(v), keyw = key_of(w);
+      const u32 vb = __float_as_uint(v);
+      const u32 key = vb & 0x7fffffffu;
+      keys[k] = key;
       mx = max(mx, key);
-      mxw = max(mxw, keyw);
-      df |= key ^ keyw;
+      df |= vb ^ __float_as_uint(w);
       if (NSEL > 0) {
         bool inb = false;
 #pragma unroll
@@ -994,19 +1039,17 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
           fB[j] = below ? fmaf(v, v, fB[j]) : fB[j];
           inb = inb || (!ge && !below);
         }
-        inb = inb && ok;
-        const u32 mask = __ballot_sync(0xffffffffu, inb);
-        if (mask) {
-          const int leader = __ffs(mask) - 1;
-          u32 base = 0;
-          if (lane == leader) base = atomicAdd(&sh_cnt, (u32)__popc(mask));
-          base = __shfl_sync(0xffffffffu, base, leader);
-          if (inb) {
-            const u32 pos = base + (u32)__popc(mask & ((1u << lane) - 1u));
-            if (pos < segcap) seg[pos] = ((u64)key << 32) | (u64)(u32)(c0 + k);
-          }
-        }
+        if (inb && (ALIGNED || c0 + k < d)) im |= 1u << k;
       }
+    }
+    if (NSEL > 0 && live && im) {  // zero padding of dead lanes has key 0 and is never listed
+      u32 pos = atomicAdd(&sh_cnt, (u32)__popc(im));
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (im & (1u << k)) {
+          if (pos < segcap) seg[pos] = ((u64)keys[k] << 32) | (u64)(u32)(c0 + k);
+          ++pos;
+        }
     }
     if ((it & (FLUSH_TILES - 1)) == FLUSH_TILES - 1) {
       dD += (double)fD; fD = 0.f;
@@ -1033,13 +1076,11 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    mxw = max(mxw, __shfl_xor_sync(0xffffffffu, mxw, o));
     df |= __shfl_xor_sync(0xffffffffu, df, o);
   }
   if (lane == 0) {
     if (mx) atomicMax(&maxkey[row], mx);
-    df &= 0x7fffffffu;
-    if (mxw >= 0x7f800000u) df |= 0x80000000u;
+    df &= 0x7fffffffu;  // sign differences do not matter: only |X-G| against |X-Y|
     if (df) atomicOr(&diffflag[row], df);
   }
   __syncthreads();
@@ -1460,9 +1501,12 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
     long long stride = ntile / 128;
     if (stride < 1) stride = 1;
-    if (stride > 32) stride = 32;
+    if (stride > 64) stride = 64;
     const long long nsamp = ntile / stride;
-    const dim3 samp_grid((unsigned)((nsamp + 15) / 16), rows);
+    long long sgx = (148 + rows - 1) / rows;          // about one wave of CTAs over all rows
+    if (sgx < (nsamp + 62) / 63) sgx = (nsamp + 62) / 63;  // 16-bit per-CTA counters: at most 63 tiles each
+    if (sgx > nsamp) sgx = nsamp;
+    const dim3 samp_grid((unsigned)sgx, rows);
     TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist, cs, s.sel, s.tickets);
     // 2. the one pass over X, G, Y
     const u32 segcap = (u32)(s.list_row / nblk);
