@@ -369,6 +369,7 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
   if (bits_host) cudaMemcpyAsync(bits_host, ctx->bits, (size_t)rows * 8, cudaMemcpyDeviceToHost, ctx->stream);
   cudaMemcpyAsync(&flags_after, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_compress_host");
+  if (flags_after & 2u) return fail(ctx, ADACGD_ERR_CUDA, "a device-side wait for an asynchronous copy timed out");
   if ((flags_after & 1u) && !(flags_before & 1u))
     return fail(ctx, ADACGD_ERR_NONFINITE, "an input row held Inf or NaN; its estimator was left unchanged");
   return ADACGD_OK;
@@ -450,6 +451,7 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
     unsigned int fl = 0;
     cudaMemcpyAsync(&fl, c->scr.flags, 4, cudaMemcpyDeviceToHost, c->stream);
     if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
+    if (fl & 2u) return fail(c, ADACGD_ERR_CUDA, "a device-side wait for an asynchronous copy timed out");
     if (fl & 1u) return fail(c, ADACGD_ERR_NONFINITE, "a gradient or estimator held Inf or NaN");
   }
   if (cudaGetLastError() != cudaSuccess) return cuda_fail(c, "adacgd_step");

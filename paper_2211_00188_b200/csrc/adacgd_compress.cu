@@ -16,6 +16,37 @@ namespace adacgd {
 // --------------------------------------------------------------------------
 __device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
+// ---- bulk asynchronous copies (TMA, 1-D) into shared memory, completion on an mbarrier ----
+__device__ __forceinline__ u32 smem_addr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
+  u32 ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for a phase of the barrier, giving up after a bounded number of polls.
+__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
+  for (int spin = 0; spin < (1 << 22); ++spin)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// dst (shared) and src (global) 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+
 template <bool ALIGNED>
 __device__ __forceinline__ void load4(const float* __restrict__ row, long long c0, long long d, float (&o)[4]) {
   if (ALIGNED) {
@@ -975,6 +1006,11 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
 // < lo, the row maximum, and the keys inside a bracket appended to this CTA's list segment.
 // Sums run in binary32 chains of at most 4*FLUSH_TILES fused multiply-adds (relative error
 // <= (4*FLUSH_TILES + 1) 2^-24 for non-negative terms), folded into binary64.
+// With ALIGNED rows the three streams are staged through shared memory by bulk asynchronous
+// copies, P1_STAGES tiles ahead of the arithmetic; otherwise plain loads are used.
+constexpr int P1_STAGES = 4;
+constexpr int P1_TILE = TPB * 4;                                  // elements per tile and stream
+constexpr int P1_SMEM = P1_STAGES * 3 * P1_TILE * 4;              // bytes of staging per CTA
 template <int NSEL, bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
                                                const float* __restrict__ Y, long long d, CsetDev cs,
@@ -982,12 +1018,14 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
                                                u32* __restrict__ cntpart, u64* __restrict__ list,
                                                u32* __restrict__ lcount, long long list_row, u32 segcap,
                                                u32* __restrict__ maxkey, u32* __restrict__ rowflag,
-                                               u32* __restrict__ diffflag) {
+                                               u32* __restrict__ diffflag, u32* __restrict__ flags) {
   constexpr int NS = NSEL > 0 ? NSEL : 1;
   const int row = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  __shared__ u32 sh_cnt;
-  if (threadIdx.x == 0) sh_cnt = 0;
+  extern __shared__ __align__(128) float stage[];                 // [P1_STAGES][3][P1_TILE], ALIGNED only
+  __shared__ __align__(8) u64 full_bar[P1_STAGES];
+  __shared__ u32 sh_cnt, sh_abort;
+  if (threadIdx.x == 0) { sh_cnt = 0; sh_abort = 0; }
   u32 lo[NS], hi[NS], cnt[NS];
   float fB[NS];
   double dB[NS];
@@ -1006,12 +1044,47 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   const float* yr = Y + (long long)row * d;
   u64* seg = list + (long long)row * list_row + (long long)blockIdx.x * segcap;
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
+  const long long nmy = (ntile > (long long)blockIdx.x) ? (ntile - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  // producer side of the pipeline: one thread issues the three copies of a tile and arms its barrier
+  auto issue = [&](long long i) {
+    const long long t = (long long)blockIdx.x + i * gridDim.x;
+    const long long e0 = t * P1_TILE;
+    const u32 bytes = (u32)(((d - e0 < P1_TILE) ? (d - e0) : P1_TILE) * 4);
+    const int sidx = (int)(i % P1_STAGES);
+    float* buf = stage + (size_t)sidx * 3 * P1_TILE;
+    mbar_expect_tx(&full_bar[sidx], 3 * bytes);
+    bulk_load(buf, xr + e0, bytes, &full_bar[sidx]);
+    bulk_load(buf + P1_TILE, gr + e0, bytes, &full_bar[sidx]);
+    bulk_load(buf + 2 * P1_TILE, yr + e0, bytes, &full_bar[sidx]);
+  };
+  if (ALIGNED) {
+    if (threadIdx.x == 0) {
+      for (int q = 0; q < P1_STAGES; ++q) mbar_init(&full_bar[q], 1);
+      mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (long long i = 0; i < nmy && i < P1_STAGES; ++i) issue(i);
+  }
   int it = 0;
-  for (long long t = blockIdx.x; t < ntile; t += gridDim.x, ++it) {
+  for (long long i = 0; i < nmy; ++i, ++it) {
+    const long long t = (long long)blockIdx.x + i * gridDim.x;
     const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
     const bool live = c0 < d;
     float x[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f}, y[4] = {0.f, 0.f, 0.f, 0.f};
-    if (live) {
+    if (ALIGNED) {
+      const int sidx = (int)(i % P1_STAGES);
+      if (!mbar_wait_bounded(&full_bar[sidx], (u32)((i / P1_STAGES) & 1))) sh_abort = 1;
+      else if (live) {
+        const float* buf = stage + (size_t)sidx * 3 * P1_TILE + threadIdx.x * 4;
+        const float4 a = *reinterpret_cast<const float4*>(buf);
+        const float4 b = *reinterpret_cast<const float4*>(buf + P1_TILE);
+        const float4 c = *reinterpret_cast<const float4*>(buf + 2 * P1_TILE);
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+        g[0] = b.x; g[1] = b.y; g[2] = b.z; g[3] = b.w;
+        y[0] = c.x; y[1] = c.y; y[2] = c.z; y[3] = c.w;
+      }
+    } else if (live) {
       load4<ALIGNED>(xr, c0, d, x);
       load4<ALIGNED>(gr, c0, d, g);
       load4<ALIGNED>(yr, c0, d, y);
@@ -1057,7 +1130,13 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
 #pragma unroll
       for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; fB[j] = 0.f; }
     }
+    if (ALIGNED) {
+      __syncthreads();                       // every thread has read this stage
+      if (sh_abort) break;                   // a copy never arrived: give up, the host is told
+      if (threadIdx.x == 0 && i + P1_STAGES < nmy) issue(i + P1_STAGES);
+    }
   }
+  if (ALIGNED && sh_abort && threadIdx.x == 0) atomicOr(&flags[0], 2u);
   dD += (double)fD;
   dE += (double)fE;
 #pragma unroll
@@ -1487,10 +1566,15 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                                                                   s.tickets, s.flags))
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
-    if (al) k_pass1<N, true><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
-                                                        s.lcount, s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag); \
-    else k_pass1<N, false><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,          \
-                                                      s.lcount, s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag); \
+    if (al) {                                                                                                       \
+      cudaFuncSetAttribute(k_pass1<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);                 \
+      k_pass1<N, true><<<sgrid, TPB, P1_SMEM, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
+                                                        s.lcount, s.list_row, segcap, s.maxkey, s.rowflag,          \
+                                                        s.diffflag, s.flags);                                       \
+    } else {                                                                                                        \
+      k_pass1<N, false><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list, s.lcount,   \
+                                                   s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag, s.flags);   \
+    }                                                                                                               \
     break;
 #define LIST_PASS(PASS, shm, hist)                                                                                \
   TIMED(KID_LHIST, (k_lhist<PASS><<<lgrid, TPB, shm, stream>>>(cs, nblk, s.sel, s.list, s.lcount, s.list_row,     \
