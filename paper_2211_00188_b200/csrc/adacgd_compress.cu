@@ -695,49 +695,71 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
 // summed in worker order.  Row i: G_i <- G_i + C_level(X_i - G_i) (EF21, Eq. 7).  The next
 // row's operands are loaded before the current row is written back.
 constexpr int UPD_ROW_TILE = 32;
+constexpr int UP_STAGES = 4;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
-                                                CompressOut out) {
+                                                CompressOut out, u32* __restrict__ out_flags) {
   __shared__ RowDec shd[UPD_ROW_TILE];
-  const long long c0 = (long long)blockIdx.x * UPD_COLS + threadIdx.x * 4;
-  const bool live = c0 < d;
+  __shared__ __align__(128) float ustage[UP_STAGES][2][UPD_COLS];
+  __shared__ __align__(8) u64 ubar[UP_STAGES];
+  __shared__ u32 u_abort;
+  u32 used = 0;  // rows staged so far: selects the stage and the barrier phase
+  if (ALIGNED && threadIdx.x == 0) {
+    for (int q = 0; q < UP_STAGES; ++q) mbar_init(&ubar[q], 1);
+    mbar_fence_init();
+    u_abort = 0;
+  }
   const int lane = threadIdx.x & 31;
   const bool want_mean = out.mean_out != nullptr;
-  float acc[4] = {-0.f, -0.f, -0.f, -0.f};  // -0 + g == g bit for bit, so the first row needs no special case
-  for (int r0 = 0; r0 < rows; r0 += UPD_ROW_TILE) {
-    const int nr = (rows - r0 < UPD_ROW_TILE) ? rows - r0 : UPD_ROW_TILE;
+
+  // Streaming mode: all rows fit one tile of decisions, every row either skips or applies a Top-K
+  // level decided by threshold and index cut, and no kept-index list is wanted.  The CTA then walks
+  // its column chunks as one sequence of (chunk, row) items with UP_STAGES bulk copies in flight.
+  if (ALIGNED && rows <= UPD_ROW_TILE && !copy_mode && out.kept_idx == nullptr) {
+    if (threadIdx.x < rows) shd[threadIdx.x] = dec[threadIdx.x];
     __syncthreads();
-    if (threadIdx.x < nr) {
-      RowDec t;
-      if (copy_mode) { t.level = 0; t.mode = 4; t.T = 0; t.q = 0; t.need_tie = 0; t.need_exact = 0; t.qL = t.qinv = t.qstep = 0.f; t.cut = 0xffffffffu; }
-      else t = dec[r0 + threadIdx.x];
-      shd[threadIdx.x] = t;
-    }
-    __syncthreads();
-    // Common case for the whole tile of rows: every row either skips or applies a Top-K level whose
-    // threshold-equal keys are decided by the index cut, and no kept-index list is wanted.
     bool simple = true;
-    if (threadIdx.x < nr) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
-    simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
-    if (simple) {
-      float sg[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
-      if (live) {
-        if (shd[0].mode != 0 || want_mean) load4<ALIGNED>(G + (long long)r0 * d, c0, d, sg);
-        if (shd[0].mode != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, sx);
-      }
-      for (int ii = 0; ii < nr; ++ii) {
-        const int i = r0 + ii;
-        float g[4], x[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) { g[k] = sg[k]; x[k] = sx[k]; }
-        if (ii + 1 < nr && live) {
-          const int m1 = shd[ii + 1].mode;
-          if (m1 != 0 || want_mean) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, sg);
-          if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, sx);
+    if (threadIdx.x < rows) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
+    if (__syncthreads_and(simple ? 1 : 0)) {
+      const long long mychunks = (nchunk > (long long)blockIdx.x) ? (nchunk - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+      const long long items = mychunks * rows;
+      auto issue_item = [&](long long item) {
+        const long long chunk = (long long)blockIdx.x + (item / rows) * gridDim.x;
+        const int ii = (int)(item % rows);
+        const long long cb = chunk * UPD_COLS;
+        const u32 bytes = (u32)(((d - cb < UPD_COLS) ? (d - cb) : UPD_COLS) * 4);
+        const int m = shd[ii].mode;
+        const bool ng = (m != 0) || want_mean, nx = (m != 0);
+        const int sidx = (int)(item % UP_STAGES);
+        mbar_expect_tx(&ubar[sidx], bytes * ((ng ? 1u : 0u) + (nx ? 1u : 0u)));
+        if (ng) bulk_load(&ustage[sidx][0][0], G + (long long)ii * d + cb, bytes, &ubar[sidx]);
+        if (nx) bulk_load(&ustage[sidx][1][0], X + (long long)ii * d + cb, bytes, &ubar[sidx]);
+      };
+      if (threadIdx.x == 0)
+        for (long long q = 0; q < items && q < UP_STAGES; ++q) issue_item(q);
+      float acc[4] = {-0.f, -0.f, -0.f, -0.f};
+      long long chunk = blockIdx.x;
+      int ii = 0;
+      for (long long item = 0; item < items; ++item) {
+        const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
+        const bool live = c0 < d;
+        const int sidx = (int)(item % UP_STAGES);
+        const int m = shd[ii].mode;
+        float g[4] = {0.f, 0.f, 0.f, 0.f}, x[4] = {0.f, 0.f, 0.f, 0.f};
+        if (!mbar_wait_bounded(&ubar[sidx], (u32)((item / UP_STAGES) & 1))) u_abort = 1;
+        else if (live) {
+          if (m != 0 || want_mean) {
+            const float4 a = *reinterpret_cast<const float4*>(&ustage[sidx][0][threadIdx.x * 4]);
+            g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
+          }
+          if (m != 0) {
+            const float4 b = *reinterpret_cast<const float4*>(&ustage[sidx][1][threadIdx.x * 4]);
+            x[0] = b.x; x[1] = b.y; x[2] = b.z; x[3] = b.w;
+          }
         }
-        if (shd[ii].mode != 0) {
+        if (m != 0) {
           const u32 T = shd[ii].T, cut = shd[ii].cut;
           bool any = false;
 #pragma unroll
@@ -748,132 +770,265 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
             g[k] = kept ? __fadd_rn(g[k], v) : g[k];
             any = any || kept;
           }
-          // dead lanes hold zeros: they are kept only when T == 0, and never stored
-          if (any && live) store4<ALIGNED>(G + (long long)i * d, c0, d, g);
+          if (any && live) store4<ALIGNED>(G + (long long)ii * d, c0, d, g);
         }
         if (want_mean) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
-        }
-      }
-      continue;
-    }
-    float gn[4] = {0.f, 0.f, 0.f, 0.f}, xn[4] = {0.f, 0.f, 0.f, 0.f};
-    if (live) {
-      const int m0 = shd[0].mode;
-      if (m0 != 4 && (m0 != 0 || want_mean)) load4<ALIGNED>(G + (long long)r0 * d, c0, d, gn);
-      if (m0 != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, xn);
-    }
-    for (int ii = 0; ii < nr; ++ii) {
-      const int i = r0 + ii;
-      const int mode = shd[ii].mode;
-      float* grow = G + (long long)i * d;
-      float g[4], x[4];
+          if (ii == rows - 1) {
+            if (live) {
+              const float n = (float)rows;
+              float r[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) { g[k] = gn[k]; x[k] = xn[k]; }
-      if (ii + 1 < nr && live) {
-        const int m1 = shd[ii + 1].mode;
-        if (m1 != 4 && (m1 != 0 || want_mean)) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, gn);
-        if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, xn);
-      }
-      if (mode == 1 && !shd[ii].need_tie && !out.kept_idx) {
-        // common case: keep every key > T and the threshold-equal keys up to index `cut`
-        const u32 T = shd[ii].T, cut = shd[ii].cut;
-        bool any = false;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float v = __fsub_rn(x[k], g[k]);
-          const u32 key = key_of(v);
-          const bool kept = (key > T || (key == T && (u32)(c0 + k) <= cut)) && (ALIGNED || c0 + k < d);
-          g[k] = kept ? __fadd_rn(g[k], v) : g[k];
-          any = any || kept;
-        }
-        if (any && live) store4<ALIGNED>(grow, c0, d, g);
-      } else if (mode != 0) {
-        bool kept[4] = {false, false, false, false};
-        bool any = false;
-        if (mode == 4) {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) g[k] = x[k];
-          any = live;
-        } else if (mode == 1) {
-          const u32 T = shd[ii].T, q = shd[ii].q;
-          const int need_tie = shd[ii].need_tie;
-          u32 key[4];
-          float v[4];
-          u32 nt = 0;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const bool ok = live && (ALIGNED || c0 + k < d);
-            v[k] = __fsub_rn(x[k], g[k]);
-            key[k] = ok ? key_of(v[k]) : 0xffffffffu;
-            if (ok && key[k] == T) ++nt;
-          }
-          u32 before = 0;
-          if (need_tie) before = tiepref[(long long)i * nchunk + blockIdx.x] + block_excl_scan(nt, nullptr);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const bool ok = live && (ALIGNED || c0 + k < d);
-            if (!ok) continue;
-            if (key[k] > T) kept[k] = true;
-            else if (key[k] == T) {
-              kept[k] = need_tie ? (before < q) : ((u32)(c0 + k) <= shd[ii].cut);
-              ++before;
+              for (int k = 0; k < 4; ++k) r[k] = __fdiv_rn(acc[k], n);
+              store4<ALIGNED>(out.mean_out, c0, d, r);
             }
-            if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
-          }
-        } else if (mode == 2) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
-            kept[k] = live && (ALIGNED || c0 + k < d);
+            for (int k = 0; k < 4; ++k) acc[k] = -0.f;
           }
-          any = live;
-        } else {  // quantiser
-          const float L = shd[ii].qL, inv = shd[ii].qinv, step = shd[ii].qstep;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float v = __fsub_rn(x[k], g[k]);
-            g[k] = __fadd_rn(g[k], quant_value(v, L, inv, step));
-          }
-          any = live;
         }
-        if (any) store4<ALIGNED>(grow, c0, d, g);
-        if (out.kept_idx && (mode == 1 || mode == 2)) {
-          int mine = 0;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) mine += kept[k] ? 1 : 0;
-          int inc = mine;
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += t;
-          }
-          const int wtotal = __shfl_sync(0xffffffffu, inc, 31);
-          long long base = 0;
-          if (lane == 31 && wtotal) base = (long long)atomicAdd((u64*)&out.kept_cnt[i], (u64)wtotal);
-          base = __shfl_sync(0xffffffffu, base, 31);
-          long long pos = base + inc - mine;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if (kept[k]) {
-              if (pos < out.kept_stride) out.kept_idx[(long long)i * out.kept_stride + pos] = (int32_t)(c0 + k);
-              ++pos;
-            }
-        }
+        __syncthreads();                     // the stage has been read by every thread
+        if (u_abort) break;
+        if (threadIdx.x == 0 && item + UP_STAGES < items) issue_item(item + UP_STAGES);
+        if (++ii == rows) { ii = 0; chunk += gridDim.x; }
       }
-      if (want_mean) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
-      }
+      if (u_abort && threadIdx.x == 0) atomicOr(&out_flags[0], 2u);
+      return;
     }
   }
-  if (want_mean && live) {
-    const float n = (float)rows;
-    float r[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) r[k] = __fdiv_rn(acc[k], n);
-    store4<ALIGNED>(out.mean_out, c0, d, r);
+
+  for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
+    const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
+    const bool live = c0 < d;
+    float acc[4] = {-0.f, -0.f, -0.f, -0.f};  // -0 + g == g bit for bit, so the first row needs no special case
+    for (int r0 = 0; r0 < rows; r0 += UPD_ROW_TILE) {
+      const int nr = (rows - r0 < UPD_ROW_TILE) ? rows - r0 : UPD_ROW_TILE;
+      __syncthreads();
+      if (threadIdx.x < nr) {
+        RowDec t;
+        if (copy_mode) { t.level = 0; t.mode = 4; t.T = 0; t.q = 0; t.need_tie = 0; t.need_exact = 0; t.qL = t.qinv = t.qstep = 0.f; t.cut = 0xffffffffu; }
+        else t = dec[r0 + threadIdx.x];
+        shd[threadIdx.x] = t;
+      }
+      __syncthreads();
+      // Common case for the whole tile of rows: every row either skips or applies a Top-K level whose
+      // threshold-equal keys are decided by the index cut, and no kept-index list is wanted.
+      bool simple = true;
+      if (threadIdx.x < nr) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
+      simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
+      if (simple && ALIGNED) {
+        // rows are staged through shared memory by bulk asynchronous copies, UP_STAGES rows ahead
+        const long long cb = (long long)chunk * UPD_COLS;
+        const u32 bytes = (u32)(((d - cb < UPD_COLS) ? (d - cb) : UPD_COLS) * 4);
+        auto issue_row = [&](int ii, u32 slot) {
+          const int m = shd[ii].mode;
+          const bool ng = (m != 0) || want_mean, nx = (m != 0);
+          const int sidx = (int)(slot % UP_STAGES);
+          mbar_expect_tx(&ubar[sidx], bytes * ((ng ? 1u : 0u) + (nx ? 1u : 0u)));
+          if (ng) bulk_load(&ustage[sidx][0][0], G + (long long)(r0 + ii) * d + cb, bytes, &ubar[sidx]);
+          if (nx) bulk_load(&ustage[sidx][1][0], X + (long long)(r0 + ii) * d + cb, bytes, &ubar[sidx]);
+        };
+        if (threadIdx.x == 0)
+          for (int q = 0; q < nr && q < UP_STAGES; ++q) issue_row(q, used + q);
+        for (int ii = 0; ii < nr; ++ii) {
+          const int i = r0 + ii;
+          const u32 slot = used + ii;
+          const int sidx = (int)(slot % UP_STAGES);
+          const int m = shd[ii].mode;
+          float g[4] = {0.f, 0.f, 0.f, 0.f}, x[4] = {0.f, 0.f, 0.f, 0.f};
+          if (!mbar_wait_bounded(&ubar[sidx], (slot / UP_STAGES) & 1u)) u_abort = 1;
+          else if (live) {
+            if (m != 0 || want_mean) {
+              const float4 a = *reinterpret_cast<const float4*>(&ustage[sidx][0][threadIdx.x * 4]);
+              g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
+            }
+            if (m != 0) {
+              const float4 b = *reinterpret_cast<const float4*>(&ustage[sidx][1][threadIdx.x * 4]);
+              x[0] = b.x; x[1] = b.y; x[2] = b.z; x[3] = b.w;
+            }
+          }
+          if (m != 0) {
+            const u32 T = shd[ii].T, cut = shd[ii].cut;
+            bool any = false;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float v = __fsub_rn(x[k], g[k]);
+              const u32 key = key_of(v);
+              const bool kept = (key > T) || (key == T && (u32)c0 + (u32)k <= cut);
+              g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+              any = any || kept;
+            }
+            if (any && live) store4<ALIGNED>(G + (long long)i * d, c0, d, g);
+          }
+          if (want_mean) {
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+          }
+          __syncthreads();                     // the stage has been read by every thread
+          if (u_abort) break;
+          if (threadIdx.x == 0 && ii + UP_STAGES < nr) issue_row(ii + UP_STAGES, slot + UP_STAGES);
+        }
+        if (u_abort) {
+          if (threadIdx.x == 0) atomicOr(&out_flags[0], 2u);
+          return;
+        }
+        used += (u32)nr;
+        continue;
+      }
+      if (simple) {
+        float sg[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
+        if (live) {
+          if (shd[0].mode != 0 || want_mean) load4<ALIGNED>(G + (long long)r0 * d, c0, d, sg);
+          if (shd[0].mode != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, sx);
+        }
+        for (int ii = 0; ii < nr; ++ii) {
+          const int i = r0 + ii;
+          float g[4], x[4];
+  #pragma unroll
+          for (int k = 0; k < 4; ++k) { g[k] = sg[k]; x[k] = sx[k]; }
+          if (ii + 1 < nr && live) {
+            const int m1 = shd[ii + 1].mode;
+            if (m1 != 0 || want_mean) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, sg);
+            if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, sx);
+          }
+          if (shd[ii].mode != 0) {
+            const u32 T = shd[ii].T, cut = shd[ii].cut;
+            bool any = false;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float v = __fsub_rn(x[k], g[k]);
+              const u32 key = key_of(v);
+              const bool kept = (key > T) || (key == T && (u32)c0 + (u32)k <= cut);
+              g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+              any = any || kept;
+            }
+            // dead lanes hold zeros: they are kept only when T == 0, and never stored
+            if (any && live) store4<ALIGNED>(G + (long long)i * d, c0, d, g);
+          }
+          if (want_mean) {
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+          }
+        }
+        continue;
+      }
+      float gn[4] = {0.f, 0.f, 0.f, 0.f}, xn[4] = {0.f, 0.f, 0.f, 0.f};
+      if (live) {
+        const int m0 = shd[0].mode;
+        if (m0 != 4 && (m0 != 0 || want_mean)) load4<ALIGNED>(G + (long long)r0 * d, c0, d, gn);
+        if (m0 != 0) load4<ALIGNED>(X + (long long)r0 * d, c0, d, xn);
+      }
+      for (int ii = 0; ii < nr; ++ii) {
+        const int i = r0 + ii;
+        const int mode = shd[ii].mode;
+        float* grow = G + (long long)i * d;
+        float g[4], x[4];
+  #pragma unroll
+        for (int k = 0; k < 4; ++k) { g[k] = gn[k]; x[k] = xn[k]; }
+        if (ii + 1 < nr && live) {
+          const int m1 = shd[ii + 1].mode;
+          if (m1 != 4 && (m1 != 0 || want_mean)) load4<ALIGNED>(G + (long long)(i + 1) * d, c0, d, gn);
+          if (m1 != 0) load4<ALIGNED>(X + (long long)(i + 1) * d, c0, d, xn);
+        }
+        if (mode == 1 && !shd[ii].need_tie && !out.kept_idx) {
+          // common case: keep every key > T and the threshold-equal keys up to index `cut`
+          const u32 T = shd[ii].T, cut = shd[ii].cut;
+          bool any = false;
+  #pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float v = __fsub_rn(x[k], g[k]);
+            const u32 key = key_of(v);
+            const bool kept = (key > T || (key == T && (u32)(c0 + k) <= cut)) && (ALIGNED || c0 + k < d);
+            g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+            any = any || kept;
+          }
+          if (any && live) store4<ALIGNED>(grow, c0, d, g);
+        } else if (mode != 0) {
+          bool kept[4] = {false, false, false, false};
+          bool any = false;
+          if (mode == 4) {
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) g[k] = x[k];
+            any = live;
+          } else if (mode == 1) {
+            const u32 T = shd[ii].T, q = shd[ii].q;
+            const int need_tie = shd[ii].need_tie;
+            u32 key[4];
+            float v[4];
+            u32 nt = 0;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const bool ok = live && (ALIGNED || c0 + k < d);
+              v[k] = __fsub_rn(x[k], g[k]);
+              key[k] = ok ? key_of(v[k]) : 0xffffffffu;
+              if (ok && key[k] == T) ++nt;
+            }
+            u32 before = 0;
+            if (need_tie) before = tiepref[(long long)i * nchunk + chunk] + block_excl_scan(nt, nullptr);
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const bool ok = live && (ALIGNED || c0 + k < d);
+              if (!ok) continue;
+              if (key[k] > T) kept[k] = true;
+              else if (key[k] == T) {
+                kept[k] = need_tie ? (before < q) : ((u32)(c0 + k) <= shd[ii].cut);
+                ++before;
+              }
+              if (kept[k]) { g[k] = __fadd_rn(g[k], v[k]); any = true; }
+            }
+          } else if (mode == 2) {
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
+              kept[k] = live && (ALIGNED || c0 + k < d);
+            }
+            any = live;
+          } else {  // quantiser
+            const float L = shd[ii].qL, inv = shd[ii].qinv, step = shd[ii].qstep;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float v = __fsub_rn(x[k], g[k]);
+              g[k] = __fadd_rn(g[k], quant_value(v, L, inv, step));
+            }
+            any = live;
+          }
+          if (any) store4<ALIGNED>(grow, c0, d, g);
+          if (out.kept_idx && (mode == 1 || mode == 2)) {
+            int mine = 0;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k) mine += kept[k] ? 1 : 0;
+            int inc = mine;
+  #pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              int t = __shfl_up_sync(0xffffffffu, inc, o);
+              if (lane >= o) inc += t;
+            }
+            const int wtotal = __shfl_sync(0xffffffffu, inc, 31);
+            long long base = 0;
+            if (lane == 31 && wtotal) base = (long long)atomicAdd((u64*)&out.kept_cnt[i], (u64)wtotal);
+            base = __shfl_sync(0xffffffffu, base, 31);
+            long long pos = base + inc - mine;
+  #pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (kept[k]) {
+                if (pos < out.kept_stride) out.kept_idx[(long long)i * out.kept_stride + pos] = (int32_t)(c0 + k);
+                ++pos;
+              }
+          }
+        }
+        if (want_mean) {
+  #pragma unroll
+          for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+        }
+      }
+    }
+    if (want_mean && live) {
+      const float n = (float)rows;
+      float r[4];
+  #pragma unroll
+      for (int k = 0; k < 4; ++k) r[k] = __fdiv_rn(acc[k], n);
+      store4<ALIGNED>(out.mean_out, c0, d, r);
+    }
   }
 }
 
@@ -1515,7 +1670,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const bool al = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y) &&
                   (!out.mean_out || aligned16(out.mean_out));
   const long long nchunk = nchunk_of(d);
-  const dim3 ugrid((unsigned)nchunk);
+  const dim3 ugrid((unsigned)(nchunk < 148 * 4 ? nchunk : 148 * 4));  // persistent: CTAs walk the column chunks
   Prof* pf = s.prof;
 #define TIMED(id, ...)             \
   do {                             \
@@ -1533,7 +1688,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
     prof_end(pf, stream);
     TIMED(KID_PICK, (k_copy_report<<<(rows + 127) / 128, 128, 0, stream>>>(rows, d, 0, out)));
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out, s.flags);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   // clear the per-call accumulators
@@ -1623,7 +1778,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (tgx > nchunk) tgx = nchunk;
     TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk, s.tickets);
   }
-  TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+  TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, s.flags);
 #undef LIST_PASS
 #undef PASS1_CASE
 #undef TIMED_HIST
