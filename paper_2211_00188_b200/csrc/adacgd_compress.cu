@@ -1082,7 +1082,7 @@ __device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, cons
 // Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
 // holds the K-th largest key with overwhelming probability (checked exactly afterwards).
 __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sample,
-                            const u32* __restrict__ shist, SelRow* __restrict__ sel) {
+                            const u32* __restrict__ shist, SelRow* __restrict__ sel, u32* __restrict__ tickets) {
   __shared__ u32 csum[TPB], cexcl[TPB];
   __shared__ u32 res;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -1113,7 +1113,15 @@ __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sa
       sample_rank_bin(h, csum, cexcl, (u32)r_lo, &res);
       lo = res << 15;
     }
-    if (threadIdx.x == 0) { sel[row].lo[j] = lo; sel[row].hi[j] = hi; }
+    if (threadIdx.x == 0) {
+      const u32 span = hi - lo;                                  // >= 2^15
+      const u32 nbits = 32u - (u32)__clz((int)(span - 1u));
+      const u32 sh1 = nbits > 11u ? nbits - 11u : 0u;
+      const u32 sh2 = sh1 > 11u ? sh1 - 11u : 0u;
+      sel[row].lo[j] = lo; sel[row].hi[j] = hi;
+      sel[row].sh1[j] = sh1; sel[row].sh2[j] = sh2;
+      if (sh2) tickets[row * NTICKET + 10] = 1u;
+    }
     __syncthreads();
   }
 }
@@ -1154,7 +1162,7 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
     if (w >> 16) atomicAdd(&gh[2 * i + 1], w >> 16);
   }
   if (last_cta_of_row(&tickets[row * NTICKET + 0], gridDim.x))
-    bracket_row(cs, row, d, stride == 1 ? 1 : 0, shist, sel);
+    bracket_row(cs, row, d, stride == 1 ? 1 : 0, shist, sel, tickets);
 }
 
 // The streaming pass: D, ||v||^2, per bracket the count of keys >= hi and the energy of keys
@@ -1339,23 +1347,85 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   }
 }
 
-// Run by the last CTA of a row's list pass.
-template <int PASS>
-__device__ void lscan_row(const CsetDev& cs, int row, int nblk, int nlb, const u32* __restrict__ hist,
-                          const u32* __restrict__ cntpart, const double* __restrict__ lepart,
-                          SelRow* __restrict__ sel, u32* __restrict__ rowflag,
-                          const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
+// ---- exact selection among the listed keys -------------------------------------------------
+// Inside its bracket a key is identified by rel = key - lo < hi - lo, split into up to three
+// digits: d1 = rel >> sh1 (11 bits), d2 = the next sh1 - sh2 <= 11 bits, d3 = the last sh2 <= 9 bits.
+// The first digit is histogrammed by the streaming pass itself, the second by one pass over the
+// lists, the third (only for brackets wider than 2^22 key values) by another.
+__device__ __forceinline__ u32 digit2(u32 rel, u32 sh1, u32 sh2) { return (rel >> sh2) & ((1u << (sh1 - sh2)) - 1u); }
+
+// Completes bracket j of a row once its threshold key is known (run by a whole CTA).
+__device__ void finalize_band(SelRow* s, int row, int j, u32 T, u32 above, u32 ntie, u32 K, double energy,
+                              const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
+  __shared__ u32 ties[1024];
+  __shared__ u32 nties_sh;
+  const u32 q = K - above;
+  if (threadIdx.x == 0) {
+    s->T[j] = T; s->above[j] = above; s->ntie[j] = ntie; s->q[j] = q; s->extraE[j] = energy;
+  }
+  // Which threshold-equal keys are kept: the q with the lowest indices.  They are all among the
+  // entries collected at the last digit level; the q-th smallest of their indices is the cut.
+  const u32 nfl = __ldcg(&flcnt[row * MAXC + j]);
+  if (q == ntie) {
+    if (threadIdx.x == 0) { s->tiemode[j] = 0u; s->cut[j] = 0xffffffffu; }
+  } else if (nfl > FINAL_CAP || ntie > 1024u) {
+    if (threadIdx.x == 0) { s->tiemode[j] = 2u; s->cut[j] = 0xffffffffu; }
+  } else {
+    if (threadIdx.x == 0) nties_sh = 0;
+    __syncthreads();
+    const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
+    for (u32 i = threadIdx.x; i < nfl; i += TPB) {
+      const u64 ent = __ldcg(&f[i]);
+      if ((u32)(ent >> 32) == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)ent;
+    }
+    __syncthreads();
+    for (u32 i = threadIdx.x; i < ntie; i += TPB) {
+      const u32 mine = ties[i];
+      u32 rank = 0;
+      for (u32 k = 0; k < ntie; ++k) rank += (ties[k] < mine) ? 1u : 0u;
+      if (rank == q - 1u) { s->tiemode[j] = 1u; s->cut[j] = mine; }
+    }
+  }
+  __syncthreads();
+}
+
+// Sum over the bins below `bin` of count * value^2, every bin being a single key value
+// base + b; all TPB threads call, the result is valid in thread 0.
+__device__ double bins_energy_below(const u32* __restrict__ h, u32 bin, u32 base) {
+  __shared__ double redd[TPB / 32];
+  double a = 0.0;
+  for (u32 b = threadIdx.x; b < bin; b += TPB) {
+    const double kv = (double)__uint_as_float(base + b);
+    a += (double)__ldcg(&h[b]) * (kv * kv);
+  }
+  a = warp_sum_f64(a);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) redd[threadIdx.x >> 5] = a;
+  __syncthreads();
+  double e = 0.0;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < TPB / 32; ++w) e += redd[w];
+  return e;
+}
+
+// Run by the last CTA of a row after digit level LEVEL has been histogrammed.
+template <int LEVEL>
+__device__ __noinline__ void lscan_row(const CsetDev& cs, int row, int nblk, int nlb, const u32* __restrict__ hist,
+                          const u32* __restrict__ cntpart, const double* __restrict__ lepart2,
+                          const double* __restrict__ lepart3, SelRow* __restrict__ sel,
+                          u32* __restrict__ rowflag, const u64* __restrict__ fl, const u32* __restrict__ flcnt) {
   __shared__ u32 res[2];
   __shared__ u32 bad;
-  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  constexpr int NB = (LEVEL == 3) ? BINS3 : BINS1;
   SelRow* s = sel + row;
-  if (PASS == 1) {
+  if (LEVEL == 1) {
     // exact check of every bracket: the K-th largest key must be one of the listed keys
     if (threadIdx.x == 0) bad = 0;
     __syncthreads();
     for (int j = 0; j < cs.nsel; ++j) {
       u32 a = 0, tot = 0;
-      for (int b = threadIdx.x; b < nblk; b += TPB) a += cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j];
+      for (int b = threadIdx.x; b < nblk; b += TPB)
+        a += __ldcg(&cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j]);
       const u32* h = hist + ((long long)row * MAXC + j) * NB;
       for (int b = threadIdx.x; b < NB; b += TPB) tot += __ldcg(&h[b]);
       u32 above, total;
@@ -1368,107 +1438,75 @@ __device__ void lscan_row(const CsetDev& cs, int row, int nblk, int nlb, const u
       }
     }
     __syncthreads();
-    if (bad) {
+    if (bad || __ldcg(&rowflag[row])) {   // bracket missed, or a list segment overflowed
       if (threadIdx.x == 0) rowflag[row] = 1;
       return;
     }
   }
   for (int j = 0; j < cs.nsel; ++j) {
+    const u32 sh1 = s->sh1[j], sh2 = s->sh2[j];
+    if (LEVEL == 3 && sh2 == 0) continue;  // finished at level 2
     const u32 K = (u32)cs.param[cs.sel[j]];
     const u32* h = hist + ((long long)row * MAXC + j) * NB;
-    const u32 before = (PASS == 1) ? s->above_hi[j] : (PASS == 2 ? s->above1[j] : s->above2[j]);
+    const u32 before = (LEVEL == 1) ? s->above_hi[j] : (LEVEL == 2 ? s->above1[j] : s->above2[j]);
     block_find_kth_desc(h, NB, K - before, res);
-    if (PASS == 3) {
-      // energy of the keys that share the 22-bit prefix and lie below the threshold: each bin is one key value
-      double a = 0.0;
-      for (int b = threadIdx.x; b < (int)res[0]; b += TPB) {
-        const double kv = (double)__uint_as_float((s->p2[j] << 9) | (u32)b);
-        a += (double)__ldcg(&h[b]) * (kv * kv);
+    const u32 bin = res[0], above = before + res[1];
+    if (LEVEL == 1) {
+      if (threadIdx.x == 0) { s->b1[j] = bin; s->above1[j] = above; }
+    } else if (LEVEL == 2 && sh2 != 0) {
+      if (threadIdx.x == 0) { s->p2[j] = bin; s->above2[j] = above; }
+    } else {
+      // last level of this bracket: each bin is one key value
+      const u32 base = s->lo[j] + ((LEVEL == 2) ? (s->b1[j] << sh1) : ((s->b1[j] << sh1) | (s->p2[j] << sh2)));
+      double e = bins_energy_below(h, bin, base);
+      // energies the list passes found below the chosen digits, one partial per CTA (fixed order)
+      double part = 0.0;
+      for (int b = threadIdx.x; b < nlb; b += TPB) {
+        part += __ldcg(&lepart2[((long long)row * LIST_BLK + b) * MAXC + j]);
+        if (LEVEL == 3) part += __ldcg(&lepart3[((long long)row * LIST_BLK + b) * MAXC + j]);
       }
-      __shared__ double redd[TPB / 32];
-      a = warp_sum_f64(a);
-      __syncthreads();
-      if ((threadIdx.x & 31) == 0) redd[threadIdx.x >> 5] = a;
+      __shared__ double e_sh, part_sh[TPB / 32];
+      part = warp_sum_f64(part);
+      if ((threadIdx.x & 31) == 0) part_sh[threadIdx.x >> 5] = part;
       __syncthreads();
       if (threadIdx.x == 0) {
-        double e = 0.0;
-        for (int b = 0; b < nlb; ++b) e += __ldcg(&lepart[((long long)row * LIST_BLK + b) * MAXC + j]);
-        for (int w = 0; w < TPB / 32; ++w) e += redd[w];
-        s->extraE[j] = e;
-      }
-    }
-    if (threadIdx.x == 0) {
-      if (PASS == 1) {
-        s->b1[j] = res[0];
-        s->above1[j] = before + res[1];
-      } else if (PASS == 2) {
-        s->p2[j] = (s->b1[j] << 11) | res[0];
-        s->above2[j] = before + res[1];
-      } else {
-        s->T[j] = (s->p2[j] << 9) | res[0];
-        s->above[j] = before + res[1];
-        s->ntie[j] = __ldcg(&h[res[0]]);
-        s->q[j] = K - (before + res[1]);
-      }
-    }
-    __syncthreads();
-    if (PASS == 3) {
-      // Which threshold-equal keys are kept: the q with the lowest indices.  They are all among the
-      // collected prefix-equal entries; the q-th smallest of their indices is the cut.
-      __shared__ u32 ties[1024];
-      __shared__ u32 nties_sh;
-      const u32 T = s->T[j], q = s->q[j], ntie = s->ntie[j];
-      const u32 nfl = __ldcg(&flcnt[row * MAXC + j]);
-      if (q == ntie) {
-        if (threadIdx.x == 0) { s->tiemode[j] = 0u; s->cut[j] = 0xffffffffu; }
-      } else if (nfl > FINAL_CAP || ntie > 1024u) {
-        if (threadIdx.x == 0) { s->tiemode[j] = 2u; s->cut[j] = 0xffffffffu; }
-      } else {
-        if (threadIdx.x == 0) nties_sh = 0;
-        __syncthreads();
-        const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
-        for (u32 i = threadIdx.x; i < nfl; i += TPB) {
-          const u64 ent = __ldcg(&f[i]);
-          if ((u32)(ent >> 32) == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)ent;
-        }
-        __syncthreads();
-        for (u32 i = threadIdx.x; i < ntie; i += TPB) {
-          const u32 mine = ties[i];
-          u32 rank = 0;
-          for (u32 k = 0; k < ntie; ++k) rank += (ties[k] < mine) ? 1u : 0u;
-          if (rank == q - 1u) { s->tiemode[j] = 1u; s->cut[j] = mine; }
-        }
+        for (int w = 0; w < TPB / 32; ++w) e += part_sh[w];
+        e_sh = e;
+        res[0] = __ldcg(&h[bin]);
       }
       __syncthreads();
+      finalize_band(s, row, j, base + bin, above, res[0], K, e_sh, fl, flcnt);
     }
+    __syncthreads();
   }
 }
 
-// Passes over the listed keys.  PASS 1: per bracket, histogram of key[30:20];
-// PASS 2: key[19:9] of the keys in the bracket's first-digit bin; PASS 3: key[8:0] of the keys
-// sharing the 22-bit prefix, plus the energy of the bracket's keys below that prefix.
-template <int PASS>
+// Pass over the listed keys for digit level LEVEL (1, 2 or 3).
+template <int LEVEL>
 __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __restrict__ sel,
                                                const u64* __restrict__ list, const u32* __restrict__ lcount,
                                                long long list_row, u32 segcap, u32* __restrict__ hist,
-                                               double* __restrict__ lepart, u32* __restrict__ rowflag,
-                                               u64* __restrict__ fl, u32* __restrict__ flcnt,
-                                               const u32* __restrict__ cntpart, u32* __restrict__ tickets) {
+                                               double* __restrict__ lepart2, double* __restrict__ lepart3,
+                                               u32* __restrict__ rowflag, u64* __restrict__ fl,
+                                               u32* __restrict__ flcnt, const u32* __restrict__ cntpart,
+                                               u32* __restrict__ tickets) {
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
   const int nsel = cs.nsel;
   if (rowflag[row]) return;
-  constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
+  if (LEVEL == 3 && !tickets[row * NTICKET + 10]) return;  // no bracket of this row needs a third digit
+  constexpr int NB = (LEVEL == 3) ? BINS3 : BINS1;
   for (int i = threadIdx.x; i < nsel * NB; i += TPB) sh[i] = 0;
-  u32 lo[MAXC], hi[MAXC], pref[MAXC];
+  u32 lo[MAXC], hi[MAXC], sh1[MAXC], sh2[MAXC], b1[MAXC], b2[MAXC];
   double en[MAXC];
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) {
     lo[j] = (j < nsel) ? sel[row].lo[j] : 1u;
     hi[j] = (j < nsel) ? sel[row].hi[j] : 0u;
-    pref[j] = 0;
-    if (PASS == 2 && j < nsel) pref[j] = sel[row].b1[j];
-    if (PASS == 3 && j < nsel) pref[j] = sel[row].p2[j];
+    sh1[j] = (j < nsel) ? sel[row].sh1[j] : 0u;
+    sh2[j] = (j < nsel) ? sel[row].sh2[j] : 0u;
+    b1[j] = (j < nsel && LEVEL >= 2) ? sel[row].b1[j] : 0u;
+    b2[j] = (j < nsel && LEVEL == 3) ? sel[row].p2[j] : 0u;
     en[j] = 0.0;
   }
   __syncthreads();
@@ -1481,15 +1519,27 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
 #pragma unroll
       for (int j = 0; j < MAXC; ++j) {
         if (j < nsel && key >= lo[j] && key < hi[j]) {
-          if (PASS == 1) atomicAdd(&sh[j * NB + (key >> 20)], 1u);
-          if (PASS == 2 && (key >> 20) == pref[j]) atomicAdd(&sh[j * NB + ((key >> 9) & 0x7ffu)], 1u);
-          if (PASS == 3) {
-            if ((key >> 9) == pref[j]) {
-              atomicAdd(&sh[j * NB + (key & 0x1ffu)], 1u);
+          const u32 rel = key - lo[j];
+          const u32 d1 = rel >> sh1[j];
+          if (LEVEL == 1) {
+            atomicAdd(&sh[j * NB + d1], 1u);
+          } else if (LEVEL == 2) {
+            if (d1 < b1[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
+            else if (d1 == b1[j]) {
+              atomicAdd(&sh[j * NB + digit2(rel, sh1[j], sh2[j])], 1u);
+              if (sh2[j] == 0) {
+                const u32 pos = atomicAdd(&flcnt[row * MAXC + j], 1u);
+                if (pos < FINAL_CAP) fl[((long long)row * MAXC + j) * FINAL_CAP + pos] = ent;
+              }
+            }
+          } else if (sh2[j] != 0 && d1 == b1[j]) {
+            const u32 d2 = digit2(rel, sh1[j], sh2[j]);
+            if (d2 < b2[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
+            else if (d2 == b2[j]) {
+              atomicAdd(&sh[j * NB + (rel & ((1u << sh2[j]) - 1u))], 1u);
               const u32 pos = atomicAdd(&flcnt[row * MAXC + j], 1u);
               if (pos < FINAL_CAP) fl[((long long)row * MAXC + j) * FINAL_CAP + pos] = ent;
             }
-            else if ((key >> 9) < pref[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
           }
         }
       }
@@ -1499,7 +1549,7 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
   u32* gh = hist + (long long)row * MAXC * NB;
   for (int i = threadIdx.x; i < nsel * NB; i += TPB)
     if (sh[i]) atomicAdd(&gh[i], sh[i]);
-  if (PASS == 3) {
+  if (LEVEL >= 2) {
     __shared__ double red[MAXC][TPB / 32];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 #pragma unroll
@@ -1511,11 +1561,12 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
     if (threadIdx.x < MAXC) {
       double a = 0;
       for (int w = 0; w < TPB / 32; ++w) a += red[threadIdx.x][w];
-      lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
+      double* lp = (LEVEL == 2) ? lepart2 : lepart3;
+      lp[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
     }
   }
-  if (last_cta_of_row(&tickets[row * NTICKET + PASS], gridDim.x))
-    lscan_row<PASS>(cs, row, nseg, (int)gridDim.x, hist, cntpart, lepart, sel, rowflag, fl, flcnt);
+  if (last_cta_of_row(&tickets[row * NTICKET + LEVEL], gridDim.x))
+    lscan_row<LEVEL>(cs, row, nseg, (int)gridDim.x, hist, cntpart, lepart2, lepart3, sel, rowflag, fl, flcnt);
 }
 
 // --------------------------------------------------------------------------
@@ -1527,7 +1578,7 @@ static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; 
 
 struct Layout {
   size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
-  size_t tickets, rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, fl, flcnt;
+  size_t tickets, rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
 
@@ -1562,7 +1613,7 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
   L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
   L.list_row = 0;
-  L.list = L.lcount = L.cntpart = L.lepart = L.fl = o;
+  L.list = L.lcount = L.cntpart = L.lepart = L.lepart3 = L.fl = o;
   if (single_pass) {
     L.list_row = list_row_of(d);
     L.fl = o; o = align_up(o + (size_t)rows * MAXC * FINAL_CAP * 8, 256);
@@ -1570,6 +1621,7 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
     L.lcount = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * MAXC * 4, 256);
     L.lepart = o; o = align_up(o + (size_t)rows * LIST_BLK * MAXC * 8, 256);
+    L.lepart3 = o; o = align_up(o + (size_t)rows * LIST_BLK * MAXC * 8, 256);
   }
   L.total = o;
   return L;
@@ -1599,6 +1651,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->shist = s->lhist1 = s->lcount = s->cntpart = nullptr;
   s->list = nullptr;
   s->lepart = nullptr;
+  s->lepart3 = nullptr;
   s->fl = nullptr;
   s->flcnt = nullptr;
   s->list_row = L.list_row;
@@ -1609,6 +1662,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
     s->lcount = (u32*)(b + L.lcount);
     s->cntpart = (u32*)(b + L.cntpart);
     s->lepart = (double*)(b + L.lepart);
+    s->lepart3 = (double*)(b + L.lepart3);
     s->fl = (u64*)(b + L.fl);
     s->flcnt = (u32*)(b + L.flcnt);
   }
@@ -1731,10 +1785,10 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                                                    s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag, s.flags);   \
     }                                                                                                               \
     break;
-#define LIST_PASS(PASS, shm, hist)                                                                                \
-  TIMED(KID_LHIST, (k_lhist<PASS><<<lgrid, TPB, shm, stream>>>(cs, nblk, s.sel, s.list, s.lcount, s.list_row,     \
-                                                               segcap, hist, s.lepart, s.rowflag, s.fl, s.flcnt,  \
-                                                               s.cntpart, s.tickets)))
+#define LIST_PASS(LEVEL, shm, hist)                                                                               \
+  TIMED(KID_LHIST, (k_lhist<LEVEL><<<lgrid, TPB, shm, stream>>>(cs, nblk, s.sel, s.list, s.lcount, s.list_row,    \
+                                                                segcap, hist, s.lepart, s.lepart3, s.rowflag,     \
+                                                                s.fl, s.flcnt, s.cntpart, s.tickets)))
 
   if (single) {
     // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
@@ -1756,7 +1810,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     }
     prof_end(pf, stream);
     ++launches;
-    // 3. exact selection among the listed keys: three digit passes, each finished by its last CTA
+    // 3. exact selection among the listed keys by the digits of key - lo: two passes, each finished by its
+    //    last CTA; the third only does work for brackets wider than 2^22 key values
     const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
     LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
     LIST_PASS(2, cs.nsel * BINS2 * 4, s.hist2);

@@ -22,7 +22,7 @@ constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (als
 constexpr int MAX_BLK_PER_ROW = 2048;
 constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
 constexpr int LIST_BLK = 256;       // CTAs per row of the passes over the candidate lists
-constexpr int NTICKET = 12;         // per-row completion counters: 0 sample, 1-3 list passes, 4-6 full passes, 7 exact, 8 ties
+constexpr int NTICKET = 12;         // per-row words: completion counters 0 sample, 1-3 list levels, 4-6 full passes, 7 exact, 8 ties; 10 = a third list level is needed
 constexpr int FINAL_CAP = 2048;     // entries kept per bracket for ranking threshold-equal keys by index
 constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
@@ -72,6 +72,7 @@ struct SelRow {
   // which of the keys equal to T are kept: 0 all of them, 1 those with index <= cut, 2 the q lowest
   // indices as ranked by the chunk-prefix pass (k_tiecount / k_tiescan)
   u32 tiemode[MAXC], cut[MAXC];
+  u32 sh1[MAXC], sh2[MAXC];     // digit shifts of key - lo inside the bracket
 };
 
 // Decision for one row, consumed by the update kernel.
@@ -105,7 +106,8 @@ struct Scratch {
   u64* list;       // [rows][list_row] (key << 32 | index), one segment of segcap entries per CTA
   u32* lcount;     // [rows][MAX_BLK_PER_ROW] entries per segment
   u32* cntpart;    // [rows][MAX_BLK_PER_ROW][MAXC] per-CTA counts of keys >= hi
-  double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the threshold prefix
+  double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the chosen first digit
+  double* lepart3; // same, below the chosen second digit
   u64* fl;         // [rows][MAXC][FINAL_CAP] listed keys sharing the threshold's 22-bit prefix
   u32* flcnt;      // [rows][MAXC]
   u32* tickets;    // [rows][NTICKET]
