@@ -1045,38 +1045,39 @@ __global__ void k_copy_report(int rows, long long d, int m, CompressOut out) {
 // --------------------------------------------------------------------------
 // single-pass path: brackets from a sample, one streaming pass, selection on short lists
 // --------------------------------------------------------------------------
-// Finds the bin holding the r-th largest sampled key (1-based); all TPB threads call.
-// csum/cexcl: counts and exclusive prefixes of the 256 chunks of 256 bins, in descending bin order.
-__device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, const u32* cexcl, u32 r, u32* out) {
-  __shared__ int chunk_sh;
-  if (cexcl[threadIdx.x] < r && r <= cexcl[threadIdx.x] + csum[threadIdx.x]) chunk_sh = threadIdx.x;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    const int lane = threadIdx.x;
-    const int c = chunk_sh;
-    const int pos0 = 256 * c + 8 * lane;                       // descending position of this lane's first bin
-    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 8 - pos0));
-    const uint4 a = __ldcg(p), b = __ldcg(p + 1);              // ascending addresses: positions pos0+7 .. pos0
-    const u32 v[8] = {b.w, b.z, b.y, b.x, a.w, a.z, a.y, a.x}; // v[k] = bin at descending position pos0 + k
-    u32 lsum = 0;
+// Finds the bin holding the r-th largest sampled key (1-based); one warp calls, every lane gets the
+// answer.  csum/cexcl: counts and exclusive prefixes of the 256 chunks of 256 bins, descending order.
+__device__ u32 sample_rank_bin(const u32* __restrict__ h, const u32* csum, const u32* cexcl, u32 r) {
+  const int lane = threadIdx.x & 31;
+  int c = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) lsum += v[k];
-    u32 inc = lsum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    u32 run = cexcl[c] + inc - lsum;
-    if (run < r && r <= run + lsum) {
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (r > run && r <= run + v[k]) *out = (u32)(SBINS - 1 - (pos0 + k));
-        run += v[k];
-      }
-    }
+  for (int i = 0; i < 8; ++i) {
+    const int cc = lane + 32 * i;
+    const u32 hit = __ballot_sync(0xffffffffu, cexcl[cc] < r && r <= cexcl[cc] + csum[cc]);
+    if (hit) c = 32 * i + (__ffs(hit) - 1);
   }
-  __syncthreads();
+  const int pos0 = 256 * c + 8 * lane;                         // descending position of this lane's first bin
+  const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 8 - pos0));
+  const uint4 a = __ldcg(p), b = __ldcg(p + 1);                // ascending addresses: positions pos0+7 .. pos0
+  const u32 v[8] = {b.w, b.z, b.y, b.x, a.w, a.z, a.y, a.x};   // v[k] = bin at descending position pos0 + k
+  u32 lsum = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) lsum += v[k];
+  u32 inc = lsum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  u32 run = cexcl[c] + inc - lsum;
+  u32 found = 0xffffffffu;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    if (r > run && r <= run + v[k]) found = (u32)(SBINS - 1 - (pos0 + k));
+    run += v[k];
+  }
+  const u32 who = __ballot_sync(0xffffffffu, found != 0xffffffffu);
+  return __shfl_sync(0xffffffffu, found, who ? (__ffs(who) - 1) : 0);
 }
 
 // Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
@@ -1084,45 +1085,55 @@ __device__ void sample_rank_bin(const u32* __restrict__ h, const u32* csum, cons
 __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sample,
                             const u32* __restrict__ shist, SelRow* __restrict__ sel, u32* __restrict__ tickets) {
   __shared__ u32 csum[TPB], cexcl[TPB];
-  __shared__ u32 res;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const u32* h = shist + (long long)row * SBINS;
-  for (int c = wid; c < 256; c += TPB / 32) {
-    const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 256 * (c + 1))) + 2 * lane;
-    const uint4 a = __ldcg(p), b = __ldcg(p + 1);
-    const u32 t = warp_sum_u32(a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w);
-    if (lane == 0) csum[c] = t;
+  // chunk sums, four chunks (eight 16-byte loads) in flight per warp
+  for (int c0 = wid * 4; c0 < 256; c0 += (TPB / 32) * 4) {
+    uint4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint4* p = reinterpret_cast<const uint4*>(h + (SBINS - 256 * (c0 + u + 1))) + 2 * lane;
+      a[u] = __ldcg(p);
+      b[u] = __ldcg(p + 1);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const u32 t = warp_sum_u32(a[u].x + a[u].y + a[u].z + a[u].w + b[u].x + b[u].y + b[u].z + b[u].w);
+      if (lane == 0) csum[c0 + u] = t;
+    }
   }
   __syncthreads();
   u32 S;
   const u32 ex = block_excl_scan(csum[threadIdx.x], &S);
   cexcl[threadIdx.x] = ex;
   __syncthreads();
-  for (int j = 0; j < cs.nsel; ++j) {
+  // one warp per (candidate, edge)
+  for (int w = wid; w < 2 * cs.nsel; w += TPB / 32) {
+    const int j = w >> 1;
+    const bool upper = (w & 1) == 0;
     const double K = (double)cs.param[cs.sel[j]];
     const double r = K * (double)S / (double)d;
     const double dev = full_sample ? 0.0 : 6.0 * sqrt(r * (1.0 - K / (double)d)) + 8.0;
     const double r_hi = floor(r - dev), r_lo = ceil(r + dev) + 1.0;
-    u32 hi = 0x80000000u, lo = 0u;
-    if (r_hi >= 1.0) {
-      sample_rank_bin(h, csum, cexcl, (u32)r_hi, &res);
-      hi = (res + 1u) << 15;
-      __syncthreads();
+    if (upper) {
+      u32 hi = 0x80000000u;
+      if (r_hi >= 1.0) hi = (sample_rank_bin(h, csum, cexcl, (u32)r_hi) + 1u) << 15;
+      if (lane == 0) sel[row].hi[j] = hi;
+    } else {
+      u32 lo = 0u;
+      if (r_lo <= (double)S) lo = sample_rank_bin(h, csum, cexcl, (u32)r_lo) << 15;
+      if (lane == 0) sel[row].lo[j] = lo;
     }
-    if (r_lo <= (double)S) {
-      sample_rank_bin(h, csum, cexcl, (u32)r_lo, &res);
-      lo = res << 15;
-    }
-    if (threadIdx.x == 0) {
-      const u32 span = hi - lo;                                  // >= 2^15
-      const u32 nbits = 32u - (u32)__clz((int)(span - 1u));
-      const u32 sh1 = nbits > 11u ? nbits - 11u : 0u;
-      const u32 sh2 = sh1 > 11u ? sh1 - 11u : 0u;
-      sel[row].lo[j] = lo; sel[row].hi[j] = hi;
-      sel[row].sh1[j] = sh1; sel[row].sh2[j] = sh2;
-      if (sh2) tickets[row * NTICKET + 10] = 1u;
-    }
-    __syncthreads();
+  }
+  __syncthreads();
+  if (threadIdx.x < cs.nsel) {
+    const int j = threadIdx.x;
+    const u32 span = sel[row].hi[j] - sel[row].lo[j];            // >= 2^15
+    const u32 nbits = 32u - (u32)__clz((int)(span - 1u));
+    const u32 sh1 = nbits > 11u ? nbits - 11u : 0u;
+    const u32 sh2 = sh1 > 11u ? sh1 - 11u : 0u;
+    sel[row].sh1[j] = sh1; sel[row].sh2[j] = sh2;
+    if (sh2) tickets[row * NTICKET + 10] = 1u;
   }
 }
 
@@ -1140,18 +1151,31 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
   __syncthreads();
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
-  for (long long sidx = blockIdx.x; sidx < nsamp; sidx += gridDim.x) {
-    const long long t = sidx * stride + (stride >> 1);
-    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
-    if (c0 >= d) continue;
-    float x[4], g[4];
-    load4<ALIGNED>(xr, c0, d, x);
-    load4<ALIGNED>(gr, c0, d, g);
+  // four sampled tiles per round, all loads issued before the first histogram update
+  for (long long s0 = blockIdx.x; s0 < nsamp; s0 += 4ll * gridDim.x) {
+    float x[4][4], g[4][4];
+    bool on[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if (!ALIGNED && c0 + k >= d) break;
-      const u32 bin = key_of(__fsub_rn(x[k], g[k])) >> 15;
-      atomicAdd(&sh[bin >> 1], (bin & 1u) ? 0x10000u : 1u);
+    for (int u = 0; u < 4; ++u) {
+      const long long sidx = s0 + (long long)u * gridDim.x;
+      const long long c0 = (sidx * stride + (stride >> 1)) * (TPB * 4) + threadIdx.x * 4;
+      on[u] = sidx < nsamp && c0 < d;
+      if (on[u]) {
+        load4<ALIGNED>(xr, c0, d, x[u]);
+        load4<ALIGNED>(gr, c0, d, g[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (!on[u]) continue;
+      const long long sidx = s0 + (long long)u * gridDim.x;
+      const long long c0 = (sidx * stride + (stride >> 1)) * (TPB * 4) + threadIdx.x * 4;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (!ALIGNED && c0 + k >= d) break;
+        const u32 bin = key_of(__fsub_rn(x[u][k], g[u][k])) >> 15;
+        atomicAdd(&sh[bin >> 1], (bin & 1u) ? 0x10000u : 1u);
+      }
     }
   }
   __syncthreads();
