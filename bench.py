@@ -189,7 +189,8 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- GPU legs
 # algorithmic bytes per element and row that each streaming kernel of the compression must move
-KERNEL_BYTES = {"k_hist<1>": 8, "k_hist<2>": 8, "k_hist<3>": 8, "k_energy": 12, "k_quant_err": 8, "k_update": 8}
+KERNEL_BYTES = {"k_pass1": 12, "k_update": 8, "k_hist<1>": 8, "k_hist<2>": 8, "k_hist<3>": 8, "k_energy": 12,
+                "k_quant_err": 8}
 
 
 def kernel_table(prof):

@@ -22,7 +22,7 @@ struct Counters {  // device resident, cumulative
   long long step;
   unsigned long long bits_up, bits_down;
   unsigned int rechecks_seen;
-  unsigned int pad;
+  unsigned int log_pos;  // next free record of the step log; the host rewinds it before each batch
 };
 
 thread_local std::string g_err = "";
@@ -88,8 +88,9 @@ adacgd_status check_problem(const adacgd_problem* p, const char** msg) {
 __global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned long long* __restrict__ bits,
                            const int* __restrict__ mlevel, const unsigned long long* __restrict__ mbits,
                            const double* __restrict__ loss, const unsigned int* __restrict__ flags,
-                           Counters* cnt, StepLog* log, int* loglevels, int slot) {
+                           Counters* cnt, StepLog* log, int* loglevels) {
   __shared__ unsigned long long sh[32];
+  const int slot = (int)cnt->log_pos;
   unsigned long long a = 0;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     a += bits[i];
@@ -108,6 +109,7 @@ __global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned
     r.master_level = *mlevel;
     r.rechecks = (int)(flags[1] - cnt->rechecks_seen);
     cnt->rechecks_seen = flags[1];
+    cnt->log_pos = (unsigned int)slot + 1u;
     cnt->step += 1;
     cnt->bits_up += up;
     cnt->bits_down += r.bits_down;
@@ -145,6 +147,10 @@ struct adacgd_ctx {
   int* loglevels;
   float* stage;
   long long launches;
+  cudaGraphExec_t pair_exec;   // two captured iterations (the buffers ping-pong with period 2)
+  long long pair_launches;
+  bool graph_tried;
+  bool odd;                    // parity of the iterations run since the graph's reference state
   Prof* prof;
   Prof prof_store;
   std::vector<cudaEvent_t> ev_beg, ev_end;
@@ -224,6 +230,10 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   c->flags = flags;
   c->stream = (cudaStream_t)cuda_stream;
   c->launches = 0;
+  c->pair_exec = nullptr;
+  c->pair_launches = 0;
+  c->graph_tried = false;
+  c->odd = false;
   c->prof = nullptr;
   const bool has_loss = problem->loss != ADACGD_LOSS_NONE;
   if (has_loss && (!x0_dev || !(gamma > 0.f) || g0_mode < 0 || g0_mode > 2)) {
@@ -389,44 +399,108 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
   return ADACGD_OK;
 }
 
+// Enqueues one iteration a0..a5 on the context's stream.
+static adacgd_status enqueue_iteration(adacgd_ctx* c) {
+  const int n = c->p.n;
+  const long long d = c->p.d;
+  // a0: x^{t+1} = x^t - gamma g^t
+  int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream, c->prof);
+  if (r < 0) return cuda_fail(c, "x update");
+  c->launches += r;
+  // a1: X_i = grad f_i(x^{t+1})
+  r = launch_gradient(c->p, c->gs, c->x, c->grad_nxt, c->stream);
+  if (r < 0) return cuda_fail(c, "gradient");
+  c->launches += r;
+  // a2-a4 and the mean of a5: h = g~_i^t, y = grad f_i(x^t), x = grad f_i(x^{t+1})
+  CompressOut o;
+  memset(&o, 0, sizeof(o));
+  o.mean_out = c->gt_nxt;
+  o.level = c->levels;
+  o.bits = (uint64_t*)c->bits;
+  r = launch_compress(c->scr, c->wcs, c->grad_nxt, c->G, c->grad_cur, n, d, o, c->stream);
+  if (r < 0) return cuda_fail(c, "worker compression");
+  c->launches += r;
+  // a5: master step h = g^t, y = g~^t, x = g~^{t+1}
+  adacgd_status s = run_server_and_master(c);
+  if (s != ADACGD_OK) return s;
+  float* t2 = c->grad_cur;
+  c->grad_cur = c->grad_nxt;
+  c->grad_nxt = t2;
+  prof_begin(c->prof, KID_LOG, c->stream);
+  k_log_step<<<1, 256, 0, c->stream>>>(n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
+                                       c->counters, c->log, c->loglevels);
+  prof_end(c->prof, c->stream);
+  c->launches += 1;
+  return ADACGD_OK;
+}
+
+// Captures two iterations into one graph: after two steps every ping-pong pointer is back where it
+// was, so the graph can be replayed from any even step on.  A workload whose iteration is a few
+// dozen short kernels is otherwise bound by launch latency.
+static void try_capture_pair(adacgd_ctx* c) {
+  c->graph_tried = true;
+  // one plain iteration pair first: lazy per-kernel attributes are set outside the capture
+  const long long before = c->launches;
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    return;
+  }
+  adacgd_status s1 = enqueue_iteration(c);
+  adacgd_status s2 = (s1 == ADACGD_OK) ? enqueue_iteration(c) : s1;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+  c->pair_launches = c->launches - before;
+  c->launches = before;
+  if (s1 != ADACGD_OK || s2 != ADACGD_OK || e != cudaSuccess || !graph) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    return;
+  }
+  if (cudaGraphInstantiate(&c->pair_exec, graph, 0) != cudaSuccess) {
+    cudaGetLastError();
+    c->pair_exec = nullptr;
+  }
+  cudaGraphDestroy(graph);
+}
+
 adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* report_host, int32_t* levels_host) {
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (c->p.loss == ADACGD_LOSS_NONE) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective");
   if (n_steps < 0) return fail(c, ADACGD_ERR_INVALID_ARG, "n_steps must be >= 0");
   const int n = c->p.n;
-  const long long d = c->p.d;
   std::vector<StepLog> hostlog;
   for (int done = 0; done < n_steps;) {
     const int batch = (n_steps - done < LOG_CAP) ? (n_steps - done) : LOG_CAP;
-    for (int t = 0; t < batch; ++t) {
-      // a0: x^{t+1} = x^t - gamma g^t
-      int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream, c->prof);
-      if (r < 0) return cuda_fail(c, "x update");
-      c->launches += r;
-      // a1: X_i = grad f_i(x^{t+1})
-      r = launch_gradient(c->p, c->gs, c->x, c->grad_nxt, c->stream);
-      if (r < 0) return cuda_fail(c, "gradient");
-      c->launches += r;
-      // a2-a4 and the mean of a5: h = g~_i^t, y = grad f_i(x^t), x = grad f_i(x^{t+1})
-      CompressOut o;
-      memset(&o, 0, sizeof(o));
-      o.mean_out = c->gt_nxt;
-      o.level = c->levels;
-      o.bits = (uint64_t*)c->bits;
-      r = launch_compress(c->scr, c->wcs, c->grad_nxt, c->G, c->grad_cur, n, d, o, c->stream);
-      if (r < 0) return cuda_fail(c, "worker compression");
-      c->launches += r;
-      // a5: master step h = g^t, y = g~^t, x = g~^{t+1}
-      adacgd_status s = run_server_and_master(c);
+    cudaMemsetAsync(&c->counters->log_pos, 0, 4, c->stream);
+    int t = 0;
+    // graphs hold the buffer pointers of the step parity they were captured at (always even here,
+    // because pairs are replayed whole and single iterations toggle `odd`)
+    const bool use_graph = !c->prof && batch >= 4;
+    if (use_graph && c->odd) {
+      adacgd_status s = enqueue_iteration(c);
       if (s != ADACGD_OK) return s;
-      float* t2 = c->grad_cur;
-      c->grad_cur = c->grad_nxt;
-      c->grad_nxt = t2;
-      prof_begin(c->prof, KID_LOG, c->stream);
-      k_log_step<<<1, 256, 0, c->stream>>>(n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
-                                           c->counters, c->log, c->loglevels, t);
-      prof_end(c->prof, c->stream);
-      c->launches += 1;
+      c->odd = !c->odd;
+      ++t;
+    }
+    if (use_graph && !c->graph_tried) {
+      // the first pair runs uncaptured so that one-time kernel attributes are set before the capture
+      for (int k = 0; k < 2 && t < batch; ++k, ++t) {
+        adacgd_status s = enqueue_iteration(c);
+        if (s != ADACGD_OK) return s;
+        c->odd = !c->odd;
+      }
+      if (!c->odd) try_capture_pair(c);
+    }
+    if (use_graph && c->pair_exec && !c->odd) {
+      for (; t + 2 <= batch; t += 2) {
+        if (cudaGraphLaunch(c->pair_exec, c->stream) != cudaSuccess) return cuda_fail(c, "graph launch");
+        c->launches += c->pair_launches;
+      }
+    }
+    for (; t < batch; ++t) {
+      adacgd_status s = enqueue_iteration(c);
+      if (s != ADACGD_OK) return s;
+      c->odd = !c->odd;
     }
     if (report_host || levels_host) {
       hostlog.resize(batch);
@@ -436,13 +510,13 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
                         cudaMemcpyDeviceToHost, c->stream);
       if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
       if (report_host)
-        for (int t = 0; t < batch; ++t) {
-          adacgd_step_report& rr = report_host[done + t];
-          rr.loss = hostlog[t].loss;
-          rr.bits_up = hostlog[t].bits_up;
-          rr.bits_down = hostlog[t].bits_down;
-          rr.master_level = hostlog[t].master_level;
-          rr.exact_rechecks = hostlog[t].rechecks;
+        for (int q = 0; q < batch; ++q) {
+          adacgd_step_report& rr = report_host[done + q];
+          rr.loss = hostlog[q].loss;
+          rr.bits_up = hostlog[q].bits_up;
+          rr.bits_down = hostlog[q].bits_down;
+          rr.master_level = hostlog[q].master_level;
+          rr.exact_rechecks = hostlog[q].rechecks;
         }
     }
     done += batch;
@@ -515,6 +589,7 @@ void adacgd_destroy(adacgd_ctx* ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_beg) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->ev_end) cudaEventDestroy(e);
+  if (ctx->pair_exec) cudaGraphExecDestroy(ctx->pair_exec);
   delete ctx;
 }
 
