@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) T[j] = (j < cs.nsel) ? sel[row].T[j] : 0u;
   double aD = 0, aE = 0, aB[MAXC];
-  u32 mxw = 0;
+  u32 mxw = 0, dfl = 0;
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) aB[j] = 0;
   const float* xr = X + (long long)row * d;
@@ -290,6 +290,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
       const float w = __fsub_rn(x[k], y[k]);
       const double dv = (double)v, dw = (double)w;
       mxw = max(mxw, key_of(w));
+      dfl |= __float_as_uint(v) ^ __float_as_uint(w);
       const double sq = __dmul_rn(dv, dv);
       aD = __dadd_rn(aD, __dmul_rn(dw, dw));
       aE = __dadd_rn(aE, sq);
@@ -300,6 +301,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
     }
   }
   if (mxw >= 0x7f800000u) atomicOr(&diffflag[row], 0x80000000u);
+  if (dfl & 0x7fffffffu) atomicOr(&diffflag[row], dfl & 0x7fffffffu);  // some |X-G| differs from |X-Y|
   __shared__ double red[NSLOT][TPB / 32];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   double v0 = warp_sum_f64(aD), v1 = warp_sum_f64(aE);
@@ -486,7 +488,7 @@ __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_m
     int verdict;  // 1 true, 0 false, -1 unsure
     if (by_def) verdict = 1;
     else if (!(D <= 1.7e308)) verdict = -1;  // overflowed chain or non-finite X - Y: the exact pass tells which
-    else if (j == 0 && single_pass && (diffflag[row] & 0x7fffffffu) == 0 && d_ok)
+    else if (j == 0 && (diffflag[row] & 0x7fffffffu) == 0 && d_ok)
       verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
     else if (!e_ok) verdict = -1;
     else if (cs.zeta == 0.f) verdict = 0;  // E > 0 for certain, right side is 0
@@ -1770,7 +1772,9 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   // clear the per-call accumulators
-  const bool single = (s.list != nullptr) && cs.nsel > 0;
+  // Small problems live in L2 and are bound by launch latency: the plain three-pass select needs fewer
+  // kernels there than sampling + streaming pass + list passes.
+  const bool single = (s.list != nullptr) && cs.nsel > 0 && (long long)rows * d >= (1ll << 19);
   prof_begin(pf, KID_MEMSET, stream);
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
   cudaMemsetAsync(s.zero_begin, 0, s.zero_bytes, stream);  // histograms, limbs, row flags: one contiguous region
