@@ -80,8 +80,9 @@ typedef struct {
 #define ADACGD_LOSS_NONE 3          /* no data: the context only serves adacgd_compress */
 
 #define ADACGD_LAYOUT_DENSE 0 /* A: [n][m_rows][d] row-major binary32 */
-#define ADACGD_LAYOUT_CSR 1   /* per worker i: rowptr[i*(m_rows+1) ..], entries of worker i stored from
-                                 nnz_offset = sum of the previous workers' nnz; columns ascending in a row */
+#define ADACGD_LAYOUT_CSR 1   /* CSR over all n*m_rows sample rows: row l of worker i is row i*m_rows + l; column
+                                 indices in [0, d); adacgd_init builds the transposed (CSC) copy it needs for
+                                 A_i^T r in the workspace, on the host, once */
 
 typedef struct {
   int32_t loss;
@@ -92,9 +93,10 @@ typedef struct {
   int64_t m_rows;     /* samples per worker */
   const float* A;           /* dev, dense layout */
   const float* target;      /* dev, [n][m_rows]: labels in {-1,+1} or least-squares targets */
-  const int64_t* csr_rowptr;/* dev, [n][m_rows+1], offsets into csr_col/csr_val, global (not per worker) */
-  const int32_t* csr_col;   /* dev */
-  const float* csr_val;     /* dev */
+  const int64_t* csr_rowptr;/* dev, [n*m_rows + 1], offsets into csr_col / csr_val */
+  const int32_t* csr_col;   /* dev, [csr_nnz] */
+  const float* csr_val;     /* dev, [csr_nnz] */
+  int64_t csr_nnz;          /* stored entries over all workers (CSR layout only) */
 } adacgd_problem; /* device arrays are BORROWED for the lifetime of the context */
 
 #define ADACGD_FLAG_HOST_STAGING 1 /* reserve device staging so that adacgd_compress_host can be used */

@@ -42,7 +42,7 @@ class _Cset(C.Structure):
 class _Problem(C.Structure):
     _fields_ = [("loss", C.c_int32), ("lambda_", C.c_float), ("n", C.c_int32), ("layout", C.c_int32),
                 ("d", C.c_int64), ("m_rows", C.c_int64), ("A", C.c_void_p), ("target", C.c_void_p),
-                ("csr_rowptr", C.c_void_p), ("csr_col", C.c_void_p), ("csr_val", C.c_void_p)]
+                ("csr_rowptr", C.c_void_p), ("csr_col", C.c_void_p), ("csr_val", C.c_void_p), ("csr_nnz", C.c_int64)]
 
 
 class StepReport(C.Structure):
@@ -116,7 +116,7 @@ class AdaCGD:
 
     def __init__(self, n: int, d: int, worker: Sequence[Cand] = (), worker_zeta: float = 0.0,
                  master: Sequence[Cand] = (), master_zeta: float = 0.0, *, loss: int = LOSS_NONE,
-                 lam: float = 0.0, A=None, target=None, x0=None, gamma: float = 1.0, g0_mode: int = 1,
+                 lam: float = 0.0, A=None, target=None, csr=None, x0=None, gamma: float = 1.0, g0_mode: int = 1,
                  host_staging: bool = False, device="cuda:0", stream=None):
         import torch
 
@@ -128,15 +128,25 @@ class AdaCGD:
         self.n, self.d = int(n), int(d)
         self.worker, self.worker_zeta = list(worker), float(worker_zeta)
         self.master, self.master_zeta = list(master), float(master_zeta)
-        self._keep = [A, target, x0]
+        self._keep = [A, target, x0, csr]
         m_rows = 0
+        layout, rowptr, col, val, nnz = LAYOUT_DENSE, None, None, None, 0
         if loss != LOSS_NONE:
-            assert A.dtype == torch.float32 and A.is_contiguous() and A.is_cuda
             assert target.dtype == torch.float32 and target.is_contiguous() and target.is_cuda
-            m_rows = A.shape[1]
-            assert tuple(A.shape) == (n, m_rows, d) and tuple(target.shape) == (n, m_rows)
-        self.problem = _Problem(loss, float(lam), self.n, LAYOUT_DENSE, self.d, m_rows, _ptr(A) if A is not None else None,
-                                _ptr(target) if target is not None else None, None, None, None)
+            m_rows = target.shape[1]
+            assert tuple(target.shape) == (n, m_rows)
+            if csr is not None:   # (rowptr int64 [n*m+1], col int32 [nnz], val float32 [nnz]) on the device
+                layout = LAYOUT_CSR
+                rowptr, col, val = csr
+                assert rowptr.dtype == torch.int64 and col.dtype == torch.int32 and val.dtype == torch.float32
+                assert rowptr.numel() == n * m_rows + 1 and col.numel() == val.numel()
+                assert rowptr.is_cuda and col.is_cuda and val.is_cuda
+                nnz = col.numel()
+            else:
+                assert A.dtype == torch.float32 and A.is_contiguous() and A.is_cuda
+                assert tuple(A.shape) == (n, m_rows, d)
+        self.problem = _Problem(loss, float(lam), self.n, layout, self.d, m_rows, _ptr(A) if A is not None else None,
+                                _ptr(target) if target is not None else None, _ptr(rowptr), _ptr(col), _ptr(val), nnz)
         self.flags = FLAG_HOST_STAGING if host_staging else 0
         wcs, k1 = _cset(self.worker, worker_zeta)
         mcs, k2 = _cset(self.master, master_zeta)

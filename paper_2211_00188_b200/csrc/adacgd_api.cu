@@ -74,8 +74,10 @@ adacgd_status check_problem(const adacgd_problem* p, const char** msg) {
     if (p->layout == ADACGD_LAYOUT_DENSE) {
       if (!p->A || !p->target) { *msg = "dense layout needs A and target"; return ADACGD_ERR_INVALID_ARG; }
     } else if (p->layout == ADACGD_LAYOUT_CSR) {
-      *msg = "CSR layout is not implemented in this build";
-      return ADACGD_ERR_UNSUPPORTED;
+      if (!p->csr_rowptr || !p->csr_col || !p->csr_val || !p->target || p->csr_nnz < 0) {
+        *msg = "CSR layout needs csr_rowptr, csr_col, csr_val, target and csr_nnz >= 0";
+        return ADACGD_ERR_INVALID_ARG;
+      }
     } else {
       *msg = "unknown layout";
       return ADACGD_ERR_INVALID_ARG;
@@ -273,6 +275,13 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   }
   if (has_loss) {
     carve_grad_scratch(&c->gs, b + L.grad, *problem);
+    if (problem->layout == ADACGD_LAYOUT_CSR) {
+      const char* why = build_csc(*problem, c->gs, c->stream);
+      if (why) {
+        delete c;
+        return fail(nullptr, ADACGD_ERR_INVALID_ARG, why);
+      }
+    }
     c->x = (float*)(b + L.x);
     c->G = (float*)(b + L.G);
     c->grad_cur = (float*)(b + L.gradA);

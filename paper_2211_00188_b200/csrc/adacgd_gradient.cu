@@ -2,6 +2,8 @@
 // objective (Eq. 1) for the three objectives of the workloads:
 //   logistic loss + non-convex regulariser (Section 6), logistic + l2, least squares.
 // A memory-bound GEMV pair per worker: z = A_i x (forward), X_i = A_i^T r(z) (backward).
+#include <vector>
+
 #include "adacgd_internal.cuh"
 
 namespace adacgd {
@@ -170,6 +172,53 @@ __global__ void k_grad_reduce(const float* __restrict__ part, const float* __res
   grads[(long long)worker * d + c] = v + reg_grad(loss, lambda, x[c]);
 }
 
+// CSR forward: one warp per sample row.
+__global__ void __launch_bounds__(TPB) k_csr_fwd(const long long* __restrict__ rowptr, const int* __restrict__ col,
+                                                 const float* __restrict__ val, const float* __restrict__ target,
+                                                 const float* __restrict__ x, long long m_rows, int loss,
+                                                 float* __restrict__ r, double* __restrict__ losspart) {
+  const int worker = blockIdx.y;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const long long row = (long long)blockIdx.x * LOSS_BLOCK_ROWS + wid;
+  const bool live = row < m_rows;
+  float acc = 0.f;
+  if (live) {
+    const long long g = (long long)worker * m_rows + row;
+    const long long e0 = rowptr[g], e1 = rowptr[g + 1];
+    for (long long e = e0 + lane; e < e1; e += 32) acc = fmaf(val[e], x[col[e]], acc);
+  }
+  const float z = warp_sum_f32(acc);
+  __shared__ double ls[TPB / 32];
+  double l = 0.0;
+  if (live && lane == 0) {
+    float rr;
+    residual(loss, z, target[(long long)worker * m_rows + row], 1.f / (float)m_rows, &rr, &l);
+    r[(long long)worker * m_rows + row] = rr;
+  }
+  if (lane == 0) ls[wid] = l;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < TPB / 32; ++w) s += ls[w];
+    losspart[(long long)worker * gridDim.x + blockIdx.x] = s;
+  }
+}
+
+// CSR backward on the transposed copy: one thread per column, entries in ascending sample row.
+__global__ void __launch_bounds__(TPB) k_csc_bwd(const long long* __restrict__ cptr, const int* __restrict__ crow,
+                                                 const float* __restrict__ cval, const float* __restrict__ r,
+                                                 const float* __restrict__ x, long long d, long long m_rows, int loss,
+                                                 float lambda, float* __restrict__ grads) {
+  const int worker = blockIdx.y;
+  const long long c = (long long)blockIdx.x * TPB + threadIdx.x;
+  if (c >= d) return;
+  const long long e0 = cptr[(long long)worker * d + c], e1 = cptr[(long long)worker * d + c + 1];
+  const float* rw = r + (long long)worker * m_rows;
+  float acc = 0.f;
+  for (long long e = e0; e < e1; ++e) acc = fmaf(cval[e], rw[crow[e]], acc);
+  grads[(long long)worker * d + c] = acc + reg_grad(loss, lambda, x[c]);
+}
+
 // f(x) = (1/n) sum_i [ (1/m) sum_l loss_l + reg(x) ]  in binary64, fixed summation order.
 __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__ losspart, int n, int blocks,
                                                       long long m_rows, const float* __restrict__ x, long long d,
@@ -202,6 +251,7 @@ __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 static int choose_split(const adacgd_problem& p) {
+  if (p.layout == ADACGD_LAYOUT_CSR) return 1;
   const long long ctas = (long long)p.n * ((p.d + TPB * 4 - 1) / (TPB * 4));
   long long split = (148 * 4 + ctas - 1) / ctas;
   if (split < 1) split = 1;
@@ -210,7 +260,7 @@ static int choose_split(const adacgd_problem& p) {
   return (int)split;
 }
 
-static bool cta_row_mode(const adacgd_problem& p) { return p.d >= 32768; }
+static bool cta_row_mode(const adacgd_problem& p) { return p.layout == ADACGD_LAYOUT_DENSE && p.d >= 32768; }
 
 static int loss_blocks_of(const adacgd_problem& p) {
   return cta_row_mode(p) ? (int)p.m_rows : (int)((p.m_rows + LOSS_BLOCK_ROWS - 1) / LOSS_BLOCK_ROWS);
@@ -224,6 +274,11 @@ size_t grad_scratch_bytes(const adacgd_problem& p) {
   if (split > 1) o = align_up(o + (size_t)split * p.n * p.d * 4, 256);
   o = align_up(o + (size_t)p.n * loss_blocks_of(p) * 8, 256);
   o = align_up(o + 8, 256);
+  if (p.layout == ADACGD_LAYOUT_CSR) {
+    o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
+    o = align_up(o + (size_t)p.csr_nnz * 4, 256);
+    o = align_up(o + (size_t)p.csr_nnz * 4, 256);
+  }
   return o;
 }
 
@@ -236,13 +291,36 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p) {
   g->part = nullptr;
   if (g->split > 1) { g->part = (float*)(b + o); o = align_up(o + (size_t)g->split * p.n * p.d * 4, 256); }
   g->losspart = (double*)(b + o); o = align_up(o + (size_t)p.n * g->loss_blocks * 8, 256);
-  g->loss = (double*)(b + o);
+  g->loss = (double*)(b + o); o = align_up(o + 8, 256);
+  g->csc_ptr = nullptr; g->csc_row = nullptr; g->csc_val = nullptr;
+  if (p.layout == ADACGD_LAYOUT_CSR) {
+    g->csc_ptr = (long long*)(b + o); o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
+    g->csc_row = (int*)(b + o); o = align_up(o + (size_t)p.csr_nnz * 4, 256);
+    g->csc_val = (float*)(b + o);
+  }
   g->prof = nullptr;
 }
 
 int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
                     cudaStream_t stream) {
-  if (p.layout != ADACGD_LAYOUT_DENSE) return -2;
+  if (p.layout == ADACGD_LAYOUT_CSR) {
+    int launches = 0;
+    prof_begin(g.prof, KID_GRAD_FWD, stream);
+    k_csr_fwd<<<dim3((unsigned)g.loss_blocks, p.n), TPB, 0, stream>>>((const long long*)p.csr_rowptr, p.csr_col, p.csr_val,
+                                                                      p.target, x, p.m_rows, p.loss, g.r, g.losspart);
+    prof_end(g.prof, stream);
+    ++launches;
+    prof_begin(g.prof, KID_GRAD_BWD, stream);
+    k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
+                                                                                p.d, p.m_rows, p.loss, p.lambda, grads);
+    prof_end(g.prof, stream);
+    ++launches;
+    prof_begin(g.prof, KID_LOSS, stream);
+    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, g.loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+    prof_end(g.prof, stream);
+    ++launches;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+  }
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
   prof_begin(g.prof, KID_GRAD_FWD, stream);
@@ -274,6 +352,50 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
   prof_end(g.prof, stream);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+}  // namespace adacgd
+
+namespace adacgd {
+
+// Builds the transposed copy of a CSR problem (host side, once per context): stable counting sort by
+// (worker, column), so that the entries of a column keep ascending sample-row order and the
+// backward sums have a fixed order.  Returns a message on failure, nullptr on success.
+const char* build_csc(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream) {
+  const long long rows = (long long)p.n * p.m_rows, nnz = p.csr_nnz, cols = (long long)p.n * p.d;
+  std::vector<long long> rowptr((size_t)rows + 1), cptr((size_t)cols + 1, 0);
+  std::vector<int> col((size_t)nnz), crow((size_t)nnz);
+  std::vector<float> val((size_t)nnz), cval((size_t)nnz);
+  if (cudaMemcpyAsync(rowptr.data(), p.csr_rowptr, (rows + 1) * 8, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(col.data(), p.csr_col, nnz * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(val.data(), p.csr_val, nnz * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return "copying the CSR arrays to the host failed";
+  if (rowptr[0] != 0 || rowptr[(size_t)rows] != nnz) return "csr_rowptr must start at 0 and end at csr_nnz";
+  for (long long r = 0; r < rows; ++r) {
+    if (rowptr[(size_t)r + 1] < rowptr[(size_t)r]) return "csr_rowptr must be non-decreasing";
+    const long long w = r / p.m_rows;
+    for (long long e = rowptr[(size_t)r]; e < rowptr[(size_t)r + 1]; ++e) {
+      if (col[(size_t)e] < 0 || col[(size_t)e] >= p.d) return "csr_col out of range";
+      ++cptr[(size_t)(w * p.d + col[(size_t)e]) + 1];
+    }
+  }
+  for (long long c = 0; c < cols; ++c) cptr[(size_t)c + 1] += cptr[(size_t)c];
+  std::vector<long long> fill(cptr.begin(), cptr.end() - 1);
+  for (long long r = 0; r < rows; ++r) {
+    const long long w = r / p.m_rows;
+    for (long long e = rowptr[(size_t)r]; e < rowptr[(size_t)r + 1]; ++e) {
+      const long long at = fill[(size_t)(w * p.d + col[(size_t)e])]++;
+      crow[(size_t)at] = (int)(r - w * p.m_rows);
+      cval[(size_t)at] = val[(size_t)e];
+    }
+  }
+  if (cudaMemcpyAsync(g.csc_ptr, cptr.data(), (cols + 1) * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(g.csc_row, crow.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(g.csc_val, cval.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return "copying the transposed arrays to the device failed";
+  return nullptr;
 }
 
 }  // namespace adacgd

@@ -140,12 +140,18 @@ struct GradScratch {
   double* losspart; // [n][loss_blocks]
   double* loss;     // [1]
   int split; int loss_blocks;
+  // CSR layout: transposed copy built at init (column-major over all workers: column c of worker i
+  // is "row" i*d + c)
+  long long* csc_ptr;   // [n*d + 1]
+  int* csc_row;         // [nnz] sample row inside the worker
+  float* csc_val;       // [nnz]
   Prof* prof;
 };
 size_t grad_scratch_bytes(const adacgd_problem& p);
 void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p);
 int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
                     cudaStream_t stream);
+const char* build_csc(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream);
 
 // x <- x - gamma * g  (two binary32 roundings: the product, then the difference)
 int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof);

@@ -186,3 +186,15 @@ def smoothness_estimate(A, loss: int, lam: float, iters: int = 30, seed: int = 0
     if loss == 2:
         return lam_max
     return 0.25 * lam_max + (2.0 * lam if loss == 0 else lam)
+
+
+def csr_global(rowptr, col, val):
+    """Concatenates per-worker CSR triplets (as returned by `sparse_logistic_problem`) into one CSR
+    over all n*m sample rows: (rowptr int64 [n*m+1], col int32 [nnz], val float32 [nnz])."""
+    n, m1 = rowptr.shape
+    out = [np.zeros(1, dtype=np.int64)]
+    base = 0
+    for i in range(n):
+        out.append(rowptr[i, 1:] + base)
+        base += int(rowptr[i, -1])
+    return np.concatenate(out), np.ascontiguousarray(col.reshape(-1)), np.ascontiguousarray(val.reshape(-1))

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def problem(n=4, d=100, loss=B.LOSS_NONE):
-    return B._Problem(loss, 0.0, n, 0, d, 0, None, None, None, None, None)
+    return B._Problem(loss, 0.0, n, 0, d, 0, None, None, None, None, None, 0)
 
 
 def ws_bytes(lib, prob, worker, master=(), zeta=1.0):
@@ -76,7 +76,7 @@ def test_workspace_bytes_and_descriptor_validation(lib):
     st, _, msg = ws_bytes(lib, problem(), [(B.TOPK, i + 1) for i in range(9)])
     assert st == 1
     # a dense objective without data pointers
-    st, _, msg = ws_bytes(lib, B._Problem(0, 0.1, 4, 0, 100, 10, None, None, None, None, None), [(B.TOPK, 5)])
+    st, _, msg = ws_bytes(lib, B._Problem(0, 0.1, 4, 0, 100, 10, None, None, None, None, None, 0), [(B.TOPK, 5)])
     assert st == 1 and "A" in msg
     # two identity-or-wider Top-K candidates cannot both be last
     st, _, msg = ws_bytes(lib, problem(d=100), [(B.TOPK, 100), (B.TOPK, 200)])

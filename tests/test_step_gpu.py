@@ -188,3 +188,54 @@ def test_state_roundtrip_and_errors(torch):
     with pytest.raises(pkg.AdacgdError):
         pkg.AdaCGD(2, 100, [(TOPK, 5)], 1.0, loss=0, lam=0.1, A=torch.zeros(2, 10, 100, device="cuda"),
                    target=torch.zeros(2, 10, device="cuda"), x0=torch.zeros(100, device="cuda"), gamma=-1.0)
+
+
+# ---------------------------------------------------------------- sparse features (workload c3 shape)
+def make_sparse(torch, n, d, m, density, seed, wc, wz, mc=(), mz=0.0, lam=1e-3, gamma=1.0, g0_mode=1):
+    import scipy.sparse as sp
+    import paper_2211_00188_b200 as pkg
+    rowptr, col, val, y = S.sparse_logistic_problem(n, d, m, density=density, seed=seed)
+    grp, gcol, gval = S.csr_global(rowptr, col, val)
+    dev = torch.device("cuda:0")
+    csr = tuple(torch.from_numpy(a).to(dev) for a in (grp, gcol, gval))
+    x0 = np.zeros(d, F32)
+    eng = pkg.AdaCGD(n, d, wc, wz, mc, mz, loss=1, lam=lam, csr=csr, target=torch.from_numpy(y).to(dev),
+                     x0=torch.from_numpy(x0).to(dev), gamma=gamma, g0_mode=g0_mode)
+    A = [sp.csr_matrix((val[i], col[i], rowptr[i]), shape=(m, d)) for i in range(n)]
+    prob = dict(A=A, target=[y[i] for i in range(n)], loss=1, lam=lam)
+    return eng, prob, x0
+
+
+def test_sparse_gradient_and_loss(torch):
+    n, d, m = 5, 3000, 40
+    eng, prob, x0 = make_sparse(torch, n, d, m, 0.01, 7, [(TOPK, 1)], 0.0)
+    x = (0.5 * np.random.Generator(np.random.PCG64(2)).standard_normal(d)).astype(F32)
+    out = torch.zeros(n, d, device="cuda:0")
+    f = eng.gradient(torch.from_numpy(x).cuda(), out, want_loss=True)
+    want = O.all_gradients(prob, x)
+    got = out.cpu().numpy()
+    for i in range(n):
+        assert relerr(got[i], want[i]) <= 1e-5
+    assert abs(f - O.global_loss(prob, x)) <= 1e-6 * abs(O.global_loss(prob, x))
+
+
+def test_sparse_lockstep_mixed_candidates(torch):
+    # the candidate mix of workload c3 (Top-K and 2/4/8-bit quantisers in the user's order), scaled down
+    n, d, m = 6, 4000, 50
+    wc = [(TOPK, 4), (TOPK, 40), (QUANT, 2), (QUANT, 4), (TOPK, 400), (QUANT, 8)]
+    eng, prob, x0 = make_sparse(torch, n, d, m, 0.01, 8, wc, 1.0, gamma=2.0)
+    st = O.init_state(prob, x0, wc)
+    seen = set()
+    for it in range(12):
+        push_state(eng, torch, st)
+        before = {k: np.copy(v) for k, v in st.items() if isinstance(v, np.ndarray)}
+        recs, levels = eng.step(1, report=True)
+        O.step(st, prob, 2.0, wc, 1.0)
+        ggrad = eng.get_state("grad").cpu().numpy()
+        assert relerr(ggrad, st["X"]) <= 1e-5
+        G_ref, res = O.compress_rows(ggrad, before["G"], before["X"], wc, 1.0)
+        assert levels[0] == [r["level"] for r in res], it
+        assert np.array_equal(eng.get_state("G").cpu().numpy().view(np.uint32), G_ref.view(np.uint32)), it
+        assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), O.server_mean(G_ref).view(np.uint32))
+        seen.update(levels[0])
+    assert len(seen) >= 2
