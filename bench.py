@@ -314,6 +314,7 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     dev = torch.device("cuda", local)
     steps = steps or args.steps
     warmup = warmup or args.warmup
+    csr = None
     if name == "c4":  # 16.4 GB of features: drawn on the device with the same law
         gen = torch.Generator(device=dev)
         gen.manual_seed(rank)
@@ -324,6 +325,11 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
         tgt = torch.einsum("nmd,d->nm", A, xs) + 0.1 * torch.randn(n, m, generator=gen, device=dev)
         # Gaussian features: lambda_max of the stacked (n m) x d matrix is about (1 + sqrt(n m / d))^2
         gamma = 0.5 / ((1.0 + (n * m / d) ** 0.5) ** 2 / (n * m))
+    elif W["layout"] == "csr":
+        rowptr, col, val, th = S.sparse_logistic_problem(n, d, m, density=W["density"], seed=rank)
+        csr = tuple(torch.from_numpy(a).to(dev) for a in S.csr_global(rowptr, col, val))
+        A, tgt = None, torch.from_numpy(th).to(dev)
+        gamma = 0.5 / (0.25 + W["lam"])   # unit-norm rows: lambda_max(A^T A)/m <= 1
     else:
         if W["loss"] == 2:
             Ah, th, _ = S.least_squares_problem(n, d, m, seed=rank)
@@ -333,7 +339,7 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
         A, tgt = torch.from_numpy(Ah).to(dev), torch.from_numpy(th).to(dev)
     x0 = torch.zeros(d, device=dev)
     eng = pkg.AdaCGD(n, d, W["worker"], 1.0, W["master"], 1.0, loss=W["loss"], lam=W["lam"], A=A, target=tgt,
-                     x0=x0, gamma=gamma, device=dev)
+                     csr=csr, x0=x0, gamma=gamma, device=dev)
     eng.step(warmup)
     barrier_sync(world)
     launches0 = eng.launch_count()
@@ -354,7 +360,8 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     elems_per_step = n * d + (d if W["master"] else 0)
     value = world * elems_per_step * steps / (ms * 1e-3)
     peak, peak_src = measured_peaks()
-    a_bytes = 4 * n * m * d
+    # one pass over the features: dense 4 B per entry; CSR value + column index per stored entry
+    a_bytes = 4 * n * m * d if csr is None else 8 * int(csr[1].numel())
     top = max(("k_dense_fwd", "k_dense_bwd"), key=lambda k: prof[k][0])
     achieved = a_bytes * prof[top][1] / (prof[top][0] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -379,7 +386,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5", choices=["c5", "c4", "c2", "c1"])
+    ap.add_argument("--workload", default="c5", choices=["c5", "c4", "c3", "c2", "c1"])
     ap.add_argument("--zeta", type=float, default=1.0)
     ap.add_argument("--scale", type=float, default=1.0, help="shrink d of workload c5 (profiling captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
