@@ -622,7 +622,10 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
       if (!ALIGNED && c0 + k >= d) break;
       const float v = __fsub_rn(x[k], g[k]);
       int kk; u32 p[3];
-      if (key_of(__fsub_rn(x[k], y[k])) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
+      if (key_of(__fsub_rn(x[k], y[k])) >= 0x7f800000u || key_of(v) >= 0x7f800000u) {
+        atomicOr(&diffflag[row], 0x80000000u);   // Inf/NaN in X - Y or X - G: the row is reported, not summed
+        continue;
+      }
       sq_pieces(__fsub_rn(x[k], y[k]), &kk, p);
       limb_add(sh + 0 * NLIMB, kk, p);
       sq_pieces(v, &kk, p);
@@ -762,17 +765,25 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
           }
         }
         if (m != 0) {
-          const u32 T = shd[ii].T, cut = shd[ii].cut;
-          bool any = false;
+          // kept <=> |v| >= T for indices up to the cut, |v| > T (>= the next key value) beyond it;
+          // finite non-negative binary32 values order like their bit patterns
+          const u32 T = shd[ii].T, cut = shd[ii].cut, c0u = (u32)c0;
+          const float Tf = __uint_as_float(T), Tn = __uint_as_float(T + 1u);
+          float th[4];
+          if (cut >= c0u + 3u) { th[0] = th[1] = th[2] = th[3] = Tf; }
+          else if (cut < c0u) { th[0] = th[1] = th[2] = th[3] = Tn; }
+          else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) th[k] = (c0u + (u32)k <= cut) ? Tf : Tn;
+          }
+          bool kept[4];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const float v = __fsub_rn(x[k], g[k]);
-            const u32 key = key_of(v);
-            const bool kept = (key > T) || (key == T && (u32)c0 + (u32)k <= cut);
-            g[k] = kept ? __fadd_rn(g[k], v) : g[k];
-            any = any || kept;
+            kept[k] = fabsf(v) >= th[k];
+            g[k] = kept[k] ? __fadd_rn(g[k], v) : g[k];
           }
-          if (any && live) store4<ALIGNED>(G + (long long)ii * d, c0, d, g);
+          if ((kept[0] || kept[1] || kept[2] || kept[3]) && live) store4<ALIGNED>(G + (long long)ii * d, c0, d, g);
         }
         if (want_mean) {
 #pragma unroll
@@ -1200,7 +1211,7 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
 constexpr int P1_STAGES = 4;
 constexpr int P1_TILE = TPB * 4;                                  // elements per tile and stream
 constexpr int P1_SMEM = P1_STAGES * 3 * P1_TILE * 4;              // bytes of staging per CTA
-template <int NSEL, bool ALIGNED>
+template <int NSEL, bool ALIGNED, bool QMAX>
 __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
                                                const float* __restrict__ Y, long long d, CsetDev cs,
                                                const SelRow* __restrict__ sel, double* __restrict__ partial,
@@ -1215,14 +1226,16 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   __shared__ __align__(8) u64 full_bar[P1_STAGES];
   __shared__ u32 sh_cnt, sh_abort;
   if (threadIdx.x == 0) { sh_cnt = 0; sh_abort = 0; }
-  u32 lo[NS], hi[NS], cnt[NS];
-  float fB[NS];
+  u32 cnt[NS];
+  float lof[NS], hif[NS], fB[NS], fcnt[NS];
   double dB[NS];
 #pragma unroll
   for (int j = 0; j < NS; ++j) {
-    lo[j] = (j < NSEL) ? sel[row].lo[j] : 0u;
-    hi[j] = (j < NSEL) ? sel[row].hi[j] : 0u;
-    cnt[j] = 0; fB[j] = 0.f; dB[j] = 0.0;
+    const u32 lo = (j < NSEL) ? sel[row].lo[j] : 0u;
+    const u32 hi = (j < NSEL) ? sel[row].hi[j] : 0u;
+    lof[j] = __uint_as_float(lo);
+    hif[j] = __uint_as_float(hi >= 0x7f800000u ? 0x7f800000u : hi);  // "no upper edge" compares as +inf
+    cnt[j] = 0; fB[j] = 0.f; fcnt[j] = 0.f; dB[j] = 0.0;
   }
   float fD = 0.f, fE = 0.f;
   double dD = 0.0, dE = 0.0;
@@ -1278,7 +1291,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       load4<ALIGNED>(gr, c0, d, g);
       load4<ALIGNED>(yr, c0, d, y);
     }
-    u32 keys[4];
+    float av[4];
     u32 im = 0;  // which of the four entries fall inside a bracket
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -1286,30 +1299,29 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       const float w = __fsub_rn(x[k], y[k]);
       fE = fmaf(v, v, fE);
       fD = fmaf(w, w, fD);
-      const u32 vb = __float_as_uint(v);
-      const u32 key = vb & 0x7fffffffu;
-      keys[k] = key;
-      mx = max(mx, key);
-      df |= vb ^ __float_as_uint(w);
+      av[k] = fabsf(v);
+      if (QMAX) mx = max(mx, __float_as_uint(av[k]));
+      df |= __float_as_uint(v) ^ __float_as_uint(w);
       if (NSEL > 0) {
+        // finite non-negative binary32 values order like their bit patterns: compare as floats
         bool inb = false;
 #pragma unroll
         for (int j = 0; j < NS; ++j) {
-          const bool ge = key >= hi[j];
-          const bool below = key < lo[j];
-          cnt[j] += ge ? 1u : 0u;
+          const bool ge = av[k] >= hif[j];
+          const bool below = av[k] < lof[j];
+          fcnt[j] = ge ? fcnt[j] + 1.f : fcnt[j];           // exact: far fewer than 2^24 per flush
           fB[j] = below ? fmaf(v, v, fB[j]) : fB[j];
           inb = inb || (!ge && !below);
         }
         if (inb && (ALIGNED || c0 + k < d)) im |= 1u << k;
       }
     }
-    if (NSEL > 0 && live && im) {  // zero padding of dead lanes has key 0 and is never listed
+    if (NSEL > 0 && live && im) {  // zero padding of dead lanes is never listed
       u32 pos = atomicAdd(&sh_cnt, (u32)__popc(im));
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (im & (1u << k)) {
-          if (pos < segcap) seg[pos] = ((u64)keys[k] << 32) | (u64)(u32)(c0 + k);
+          if (pos < segcap) seg[pos] = ((u64)__float_as_uint(av[k]) << 32) | (u64)(u32)(c0 + k);
           ++pos;
         }
     }
@@ -1317,7 +1329,10 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       dD += (double)fD; fD = 0.f;
       dE += (double)fE; fE = 0.f;
 #pragma unroll
-      for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; fB[j] = 0.f; }
+      for (int j = 0; j < NS; ++j) {
+        dB[j] += (double)fB[j]; fB[j] = 0.f;
+        cnt[j] += (u32)fcnt[j]; fcnt[j] = 0.f;
+      }
     }
     if (ALIGNED) {
       __syncthreads();                       // every thread has read this stage
@@ -1329,7 +1344,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   dD += (double)fD;
   dE += (double)fE;
 #pragma unroll
-  for (int j = 0; j < NS; ++j) dB[j] += (double)fB[j];
+  for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; cnt[j] += (u32)fcnt[j]; }
 
   __shared__ double red[2 + NS][TPB / 32];
   __shared__ u32 redc[NS][TPB / 32];
@@ -1801,16 +1816,21 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                                                                     s.tickets, s.flags);                         \
             else k_hist<PASS, false><<<fgrid, TPB, shm, stream>>>(X, G, d, cs, s.sel, hist, s.maxkey, only,      \
                                                                   s.tickets, s.flags))
+#define P1_ARGS                                                                                               \
+  X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list, s.lcount, s.list_row, segcap, s.maxkey, s.rowflag,     \
+      s.diffflag, s.flags
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
     if (al) {                                                                                                       \
-      cudaFuncSetAttribute(k_pass1<N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);                 \
-      k_pass1<N, true><<<sgrid, TPB, P1_SMEM, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list,        \
-                                                        s.lcount, s.list_row, segcap, s.maxkey, s.rowflag,          \
-                                                        s.diffflag, s.flags);                                       \
+      if (cs.nquant) {                                                                                              \
+        cudaFuncSetAttribute(k_pass1<N, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);         \
+        k_pass1<N, true, true><<<sgrid, TPB, P1_SMEM, stream>>>(P1_ARGS);                                           \
+      } else {                                                                                                      \
+        cudaFuncSetAttribute(k_pass1<N, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);        \
+        k_pass1<N, true, false><<<sgrid, TPB, P1_SMEM, stream>>>(P1_ARGS);                                          \
+      }                                                                                                             \
     } else {                                                                                                        \
-      k_pass1<N, false><<<sgrid, TPB, 0, stream>>>(X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list, s.lcount,   \
-                                                   s.list_row, segcap, s.maxkey, s.rowflag, s.diffflag, s.flags);   \
+      k_pass1<N, false, true><<<sgrid, TPB, 0, stream>>>(P1_ARGS);                                                  \
     }                                                                                                               \
     break;
 #define LIST_PASS(LEVEL, shm, hist)                                                                               \
@@ -1864,6 +1884,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, s.flags);
 #undef LIST_PASS
 #undef PASS1_CASE
+#undef P1_ARGS
 #undef TIMED_HIST
 #undef TIMED_AL
 #undef TIMED

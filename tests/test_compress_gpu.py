@@ -278,3 +278,17 @@ def test_small_tie_groups_at_the_threshold(torch, d):
     cands = [(TOPK, max(1, d // 1000)), (TOPK, d // 100), (TOPK, d // 10), (TOPK, d // 2)]
     for zeta in (0.0, 1.0):
         check_against_oracle(torch, X, G, Y, cands, zeta)
+
+
+def test_nonfinite_rows_on_the_single_pass_path(torch):
+    # large enough for the sampled single-pass pipeline: Inf in X - G (row 0), NaN only in X - Y (row 2)
+    X, G, Y = S.gaussian_rows(3, 300_000, seed=41)
+    X[0, 1234] = -np.inf
+    Y[2, 99] = np.nan
+    got = gpu_compress(torch, X, G, Y, [(TOPK, 300), (TOPK, 30000)], 1.0)
+    assert got["flags"] & 1
+    assert got["level"][0] == 0 and got["level"][2] == 0
+    assert_bitwise(got["G"][[0, 2]], G[[0, 2]], "flagged rows")
+    G_ref, res = O.compress_rows(X[[1]], G[[1]], Y[[1]], [(TOPK, 300), (TOPK, 30000)], 1.0)
+    assert_bitwise(got["G"][[1]], G_ref, "clean row")
+    assert got["level"][1] == res[0]["level"]
