@@ -1208,7 +1208,8 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
 // <= (4*FLUSH_TILES + 1) 2^-24 for non-negative terms), folded into binary64.
 // With ALIGNED rows the three streams are staged through shared memory by bulk asynchronous
 // copies, P1_STAGES tiles ahead of the arithmetic; otherwise plain loads are used.
-constexpr int P1_STAGES = 4;
+constexpr int P1_STAGES = 3;
+constexpr int P1_QCAP = 160;                                      // 31 left over + 128 new entries per warp
 constexpr int P1_TILE = TPB * 4;                                  // elements per tile and stream
 constexpr int P1_SMEM = P1_STAGES * 3 * P1_TILE * 4;              // bytes of staging per CTA
 template <int NSEL, bool ALIGNED, bool QMAX>
@@ -1225,10 +1226,15 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   extern __shared__ __align__(128) float stage[];                 // [P1_STAGES][3][P1_TILE], ALIGNED only
   __shared__ __align__(8) u64 full_bar[P1_STAGES];
   __shared__ u32 sh_cnt, sh_abort;
+  __shared__ u32 qcnt[TPB / 32];
+  __shared__ __align__(8) u64 qbuf[TPB / 32][P1_QCAP];
   if (threadIdx.x == 0) { sh_cnt = 0; sh_abort = 0; }
+  if (threadIdx.x < TPB / 32) qcnt[threadIdx.x] = 0;
   u32 cnt[NS];
   float lof[NS], hif[NS], fB[NS], fcnt[NS];
   double dB[NS];
+  float lomin = __uint_as_float(0x7f800000u), fBall = 0.f;
+  double dBall = 0.0;
 #pragma unroll
   for (int j = 0; j < NS; ++j) {
     const u32 lo = (j < NSEL) ? sel[row].lo[j] : 0u;
@@ -1236,6 +1242,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
     lof[j] = __uint_as_float(lo);
     hif[j] = __uint_as_float(hi >= 0x7f800000u ? 0x7f800000u : hi);  // "no upper edge" compares as +inf
     cnt[j] = 0; fB[j] = 0.f; fcnt[j] = 0.f; dB[j] = 0.0;
+    if (j < NSEL) lomin = fminf(lomin, lof[j]);
   }
   float fD = 0.f, fE = 0.f;
   double dD = 0.0, dE = 0.0;
@@ -1268,6 +1275,30 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
     if (threadIdx.x == 0)
       for (long long i = 0; i < nmy && i < P1_STAGES; ++i) issue(i);
   }
+  // A queued entry meets every bracket: count it if it lies above, add its square if it lies
+  // below (fB[j] holds only what fBall does not: keys in [lomin, lo_j)), list it if inside one.
+  auto drain = [&](u32 slot, bool act) {
+    const u64 e = act ? qbuf[wid][slot] : 0ull;
+    const float a = __uint_as_float((u32)(e >> 32));
+    bool inb = false;
+#pragma unroll
+    for (int j = 0; j < NS; ++j) {
+      const bool ge = a >= hif[j];
+      const bool below = a < lof[j];
+      fcnt[j] = (act && ge) ? fcnt[j] + 1.f : fcnt[j];       // exact: far fewer than 2^24 per flush
+      fB[j] = (act && below) ? fmaf(a, a, fB[j]) : fB[j];
+      inb = inb || (!ge && !below);
+    }
+    inb = inb && act;
+    const u32 m = __ballot_sync(0xffffffffu, inb);
+    if (m) {
+      u32 base = 0;
+      if (lane == 0) base = atomicAdd(&sh_cnt, (u32)__popc(m));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      const u32 pos = base + (u32)__popc(m & ((1u << lane) - 1u));
+      if (inb && pos < segcap) seg[pos] = e;
+    }
+  };
   int it = 0;
   for (long long i = 0; i < nmy; ++i, ++it) {
     const long long t = (long long)blockIdx.x + i * gridDim.x;
@@ -1292,7 +1323,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       load4<ALIGNED>(yr, c0, d, y);
     }
     float av[4];
-    u32 im = 0;  // which of the four entries fall inside a bracket
+    u32 rm = 0;  // which of the four entries reach the lowest bracket edge
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float v = __fsub_rn(x[k], g[k]);
@@ -1304,30 +1335,31 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       df |= __float_as_uint(v) ^ __float_as_uint(w);
       if (NSEL > 0) {
         // finite non-negative binary32 values order like their bit patterns: compare as floats
-        bool inb = false;
-#pragma unroll
-        for (int j = 0; j < NS; ++j) {
-          const bool ge = av[k] >= hif[j];
-          const bool below = av[k] < lof[j];
-          fcnt[j] = ge ? fcnt[j] + 1.f : fcnt[j];           // exact: far fewer than 2^24 per flush
-          fB[j] = below ? fmaf(v, v, fB[j]) : fB[j];
-          inb = inb || (!ge && !below);
-        }
-        if (inb && (ALIGNED || c0 + k < d)) im |= 1u << k;
+        const bool small = av[k] < lomin;
+        fBall = small ? fmaf(v, v, fBall) : fBall;
+        if (!small && (ALIGNED || c0 + k < d)) rm |= 1u << k;
       }
     }
-    if (NSEL > 0 && live && im) {  // zero padding of dead lanes is never listed
-      u32 pos = atomicAdd(&sh_cnt, (u32)__popc(im));
+    if (NSEL > 0) {
+      if (live && rm) {  // zero padding of dead lanes is never queued
+        u32 pos = atomicAdd(&qcnt[wid], (u32)__popc(rm));
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (im & (1u << k)) {
-          if (pos < segcap) seg[pos] = ((u64)__float_as_uint(av[k]) << 32) | (u64)(u32)(c0 + k);
-          ++pos;
-        }
+        for (int k = 0; k < 4; ++k)
+          if (rm & (1u << k)) qbuf[wid][pos++] = ((u64)__float_as_uint(av[k]) << 32) | (u64)(u32)(c0 + k);
+      }
+      __syncwarp();
+      u32 qc = *reinterpret_cast<volatile u32*>(&qcnt[wid]);
+      if (qc >= 32) {
+        do { qc -= 32; drain(qc + lane, true); } while (qc >= 32);
+        __syncwarp();
+        if (lane == 0) qcnt[wid] = qc;
+        __syncwarp();
+      }
     }
     if ((it & (FLUSH_TILES - 1)) == FLUSH_TILES - 1) {
       dD += (double)fD; fD = 0.f;
       dE += (double)fE; fE = 0.f;
+      dBall += (double)fBall; fBall = 0.f;
 #pragma unroll
       for (int j = 0; j < NS; ++j) {
         dB[j] += (double)fB[j]; fB[j] = 0.f;
@@ -1341,10 +1373,16 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
     }
   }
   if (ALIGNED && sh_abort && threadIdx.x == 0) atomicOr(&flags[0], 2u);
+  if (NSEL > 0) {  // what is left in the queue: fewer than 32 entries
+    __syncwarp();
+    const u32 qc = *reinterpret_cast<volatile u32*>(&qcnt[wid]);
+    if (qc) drain((u32)lane, (u32)lane < qc);
+  }
   dD += (double)fD;
   dE += (double)fE;
+  dBall += (double)fBall;
 #pragma unroll
-  for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; cnt[j] += (u32)fcnt[j]; }
+  for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j] + dBall; cnt[j] += (u32)fcnt[j]; }
 
   __shared__ double red[2 + NS][TPB / 32];
   __shared__ u32 redc[NS][TPB / 32];
