@@ -298,7 +298,7 @@ def bench_c5(args, rank, world, local):
                "ms_per_step": ems / args.e2e_steps}
     return dict(value=value, ms=ms, launches=launches, roofline=roofline, step_roofline=step_roofline,
                 kernels=kernel_table(prof), clocks=clk.summary(), e2e=e2e,
-                iters_per_s=world * args.steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"),
+                iters_per_s=world * args.steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"), side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
                 config={"workload": "c5", "n": n, "d": d, "topk": [p for _, p in W["worker"]],
                         "master_topk": [p for _, p in W["master"]], "zeta": zeta,
                         "l2": "inputs (3 x %.0f MB per pass) exceed the 126 MB L2; no flush needed" % (n * d * 4 / 1e6),
@@ -372,7 +372,7 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     step_roofline = {"algorithmic_bytes_per_step": floor, "achieved_gbs": step_gbs, "frac": step_gbs / peak}
     return dict(value=value, ms=ms, steps=steps, launches=launches, roofline=roofline, step_roofline=step_roofline,
                 kernels=kernel_table(prof), clocks=clk.summary(), e2e=None,
-                iters_per_s=world * steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"),
+                iters_per_s=world * steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"), side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
                 config={"workload": name, "n": n, "d": d, "m": m, "loss": W["loss"], "gamma": gamma,
                         "topk": [p for _, p in W["worker"]], "bidirectional": bool(W["master"]),
                         "loss_after": recs[0]["loss"], "levels_last_step": levels[0],
@@ -432,7 +432,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": res["config"],
             "iters_per_s": res["iters_per_s"], "roofline": res["roofline"], "step_roofline": res["step_roofline"],
             "kernels": res["kernels"], "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
-            "exact_rechecks": res["rechecks"], "cpu_baseline": cpu,
+            "exact_rechecks": res["rechecks"], "side_paths": res["side_paths"], "cpu_baseline": cpu,
         }
         if extra:
             line["full_iteration"] = extra

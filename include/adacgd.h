@@ -217,6 +217,9 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
 #define ADACGD_STATE_RECHECKS 10/* uint32: trigger comparisons redone in exact arithmetic since init (get only) */
 #define ADACGD_STATE_FALLBACKS 11/* uint32: rows whose sampled threshold bracket failed and that took the full
                                    three-pass radix select instead, since init (get only) */
+#define ADACGD_STATE_LIST_LEVELS 12/* uint32: rows whose threshold shared the first digit of its bracket with more keys
+                                   than the collection buffer holds (many equal or nearly equal magnitudes) and
+                                   that went through the three-level passes over the key lists, since init (get only) */
 adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,
                                int32_t dst_is_device);
 adacgd_status adacgd_set_state(adacgd_ctx* ctx, int32_t which, const void* src, size_t bytes,

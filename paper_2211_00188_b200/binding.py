@@ -12,7 +12,7 @@ TOPK, QUANT = 0, 1
 LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE = 0, 1, 2, 3
 LAYOUT_DENSE, LAYOUT_CSR = 0, 1
 FLAG_HOST_STAGING = 1
-STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11)
+STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11, list_levels=12)
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "BAD_ORDER", 3: "NONFINITE", 4: "WORKSPACE", 5: "CUDA", 6: "UNSUPPORTED"}
 
 EXPORTED_SYMBOLS = [
@@ -228,7 +228,7 @@ class AdaCGD:
             self._check(self.lib.adacgd_get_state(self.ctx, STATE[which], _ptr(out), out.numel() * out.element_size(), 1),
                         self.ctx)
             return out
-        buf = C.c_uint64(0) if which not in ("flags", "rechecks", "fallbacks") else C.c_uint32(0)
+        buf = C.c_uint64(0) if which not in ("flags", "rechecks", "fallbacks", "list_levels") else C.c_uint32(0)
         self._check(self.lib.adacgd_get_state(self.ctx, STATE[which], C.byref(buf), C.sizeof(buf), 0), self.ctx)
         return int(buf.value)
 

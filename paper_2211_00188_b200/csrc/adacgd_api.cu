@@ -557,6 +557,7 @@ static adacgd_status state_ptr(adacgd_ctx* c, int32_t which, void** p, size_t* b
     case ADACGD_STATE_FLAGS: *p = c->scr.flags; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_RECHECKS: *p = c->scr.flags + 1; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_FALLBACKS: *p = c->scr.flags + 2; *bytes = 4; return ADACGD_OK;
+    case ADACGD_STATE_LIST_LEVELS: *p = c->scr.flags + 3; *bytes = 4; return ADACGD_OK;
     default: return fail(c, ADACGD_ERR_INVALID_ARG, "unknown state item");
   }
   if (!has) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective, hence no iterate state");
@@ -580,7 +581,7 @@ adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, si
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (!src) return fail(c, ADACGD_ERR_INVALID_ARG, "src is NULL");
   if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS ||
-      which == ADACGD_STATE_FALLBACKS)
+      which == ADACGD_STATE_FALLBACKS || which == ADACGD_STATE_LIST_LEVELS)
     return fail(c, ADACGD_ERR_INVALID_ARG, "this item is read-only");
   void* p;
   size_t want;
@@ -605,7 +606,7 @@ void adacgd_destroy(adacgd_ctx* ctx) {
 static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
-    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lscan"};
+    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
 

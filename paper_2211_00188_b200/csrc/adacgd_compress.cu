@@ -14,6 +14,14 @@ namespace adacgd {
 // --------------------------------------------------------------------------
 // small helpers
 // --------------------------------------------------------------------------
+// Programmatic dependent launch: lets the next kernel of the stream be scheduled while this one
+// runs, then waits until every kernel before this one has completed and its writes are visible.
+// Called first thing by every kernel, before any access to global memory.
+__device__ __forceinline__ void pdl_begin() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
 // ---- bulk asynchronous copies (TMA, 1-D) into shared memory, completion on an mbarrier ----
@@ -197,6 +205,7 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
                                               u32* __restrict__ hist, u32* __restrict__ maxkey,
                                               const u32* __restrict__ rowflag, u32* __restrict__ tickets,
                                               u32* __restrict__ flags) {
+  pdl_begin();
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
   const int nsel = cs.nsel;
@@ -263,6 +272,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
                                                 const float* __restrict__ Y, long long d, CsetDev cs,
                                                 const SelRow* __restrict__ sel, double* __restrict__ partial,
                                                 const u32* __restrict__ rowflag, u32* __restrict__ diffflag) {
+  pdl_begin();
   const int row = blockIdx.y;
   if (rowflag && !rowflag[row]) return;
   u32 T[MAXC];
@@ -336,6 +346,7 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_quant_err(const float* __restrict__ X, const float* __restrict__ G,
                                                    long long d, CsetDev cs, const u32* __restrict__ maxkey,
                                                    double* __restrict__ partial) {
+  pdl_begin();
   const int row = blockIdx.y;
   const float s = __uint_as_float(maxkey[row]);
   float L[MAXC], inv[MAXC], step[MAXC];
@@ -438,20 +449,26 @@ __device__ void finalize_row(const CsetDev& cs, int row, int level, long long d,
     for (int j = 0; j <= cs.m; ++j) out.err[(long long)row * (cs.m + 1) + j] = e[j];
 }
 
-__global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_main, int nblk_full,
-                                             const u32* __restrict__ rowflag, const double* __restrict__ partial,
-                                             const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                                             RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
-                                             const u32* __restrict__ diffflag, int single_pass, double tol) {
-  const int row = blockIdx.x, lane = threadIdx.x;
-  const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
+// Chooses the level of one row from its sums (Eq. 10 and 11); run by one full warp.
+__device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, const double* __restrict__ partial,
+                         const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                         RowDec* __restrict__ dec, u32* __restrict__ flags, const CompressOut& out,
+                         const u32* __restrict__ diffflag, double tol) {
+  const int lane = threadIdx.x & 31;
   double sum[NSLOT];
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) {
-    double a = 0;
-    if (s < 2 + cs.m)
-      for (int b = lane; b < nblk; b += 32) a += partial[((long long)row * MAX_BLK_PER_ROW + b) * NSLOT + s];
-    sum[s] = warp_sum_f64(a);
+    double a0 = 0, a1 = 0, a2 = 0, a3 = 0;  // four independent chains: the loads overlap
+    if (s < 2 + cs.m) {
+      const double* p = partial + (long long)row * MAX_BLK_PER_ROW * NSLOT + s;
+      for (int b = lane; b < nblk; b += 128) {
+        a0 += p[(long long)b * NSLOT];
+        if (b + 32 < nblk) a1 += p[(long long)(b + 32) * NSLOT];
+        if (b + 64 < nblk) a2 += p[(long long)(b + 64) * NSLOT];
+        if (b + 96 < nblk) a3 += p[(long long)(b + 96) * NSLOT];
+      }
+    }
+    sum[s] = warp_sum_f64((a0 + a1) + (a2 + a3));
   }
   if (lane != 0) return;
   const double D = sum[0];
@@ -508,6 +525,20 @@ __global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_m
     return;
   }
   finalize_row(cs, row, level, d, sel, maxkey, dec, out, e, D);
+}
+
+// `picked` (may be null): per-row ticket words; a row whose word 9 is set was already decided.
+__global__ void __launch_bounds__(32) k_pick(CsetDev cs, long long d, int nblk_main, int nblk_full,
+                                             const u32* __restrict__ rowflag, const double* __restrict__ partial,
+                                             const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                                             RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
+                                             const u32* __restrict__ diffflag, const u32* __restrict__ picked,
+                                             double tol) {
+  pdl_begin();
+  const int row = blockIdx.x;
+  if (picked && picked[row * NTICKET + 9]) return;
+  const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
+  pick_row(cs, d, row, nblk, partial, sel, maxkey, dec, flags, out, diffflag, tol);
 }
 
 // --------------------------------------------------------------------------
@@ -601,6 +632,7 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
                                                     RowDec* __restrict__ dec, u64* __restrict__ limbs,
                                                     u32* __restrict__ diffflag, long long d_full, CompressOut out,
                                                     u32* __restrict__ tickets, u32* __restrict__ flags) {
+  pdl_begin();
   const int row = blockIdx.y;
   if (!dec[row].need_exact) return;
   __shared__ u64 sh[NSLOT * NLIMB];
@@ -664,6 +696,7 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
                                                   long long d, const RowDec* __restrict__ dec,
                                                   u32* __restrict__ tiecnt, long long nchunk,
                                                   u32* __restrict__ tickets) {
+  pdl_begin();
   const int row = blockIdx.y;
   if (!dec[row].need_tie) return;
   const u32 T = dec[row].T;
@@ -706,6 +739,7 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
                                                 CompressOut out, u32* __restrict__ out_flags) {
+  pdl_begin();
   __shared__ RowDec shd[UPD_ROW_TILE];
   __shared__ __align__(128) float ustage[UP_STAGES][2][UPD_COLS];
   __shared__ __align__(8) u64 ubar[UP_STAGES];
@@ -1046,6 +1080,7 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
 }
 
 __global__ void k_copy_report(int rows, long long d, int m, CompressOut out) {
+  pdl_begin();
   // identity compressor: level 0, bits 32 d, no error values
   const int row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= rows) return;
@@ -1158,6 +1193,7 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
                                                 long long d, long long nsamp, long long stride,
                                                 u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
                                                 u32* __restrict__ tickets) {
+  pdl_begin();
   extern __shared__ u32 sh[];  // SBINS / 2 words
   const int row = blockIdx.y;
   for (int i = threadIdx.x; i < SBINS / 2; i += TPB) sh[i] = 0;
@@ -1202,6 +1238,55 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
     bracket_row(cs, row, d, stride == 1 ? 1 : 0, shist, sel, tickets);
 }
 
+// Shift that leaves the first LB1-valued digit of key - lo for a bracket [lo, hi).
+static_assert(LB1 == TPB, "first_digit_scan reads one bin per thread");
+__device__ __forceinline__ u32 first_digit_shift(u32 lo, u32 hi) {
+  const u32 span = hi - lo;
+  const u32 nbits = span > 1u ? 32u - (u32)__clz((int)(span - 1u)) : 0u;
+  return nbits > 8u ? nbits - 8u : 0u;
+}
+
+// Run by the last CTA of a row's streaming pass.  Checks every bracket exactly (the K-th largest key
+// must be one of the listed keys; otherwise the row is flagged for the full select) and locates the
+// first-digit bin of each threshold.  A bin with more than FINAL_CAP keys sends the row through the
+// three-level list passes.
+__device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, int nblk, const u32* __restrict__ fhist,
+                                              const u32* __restrict__ cntpart, SelRow* __restrict__ sel,
+                                              u32* __restrict__ rowflag, u32* __restrict__ tickets,
+                                              u32* __restrict__ flags) {
+  __shared__ u32 res[2];
+  __shared__ u32 bad;
+  SelRow* s = sel + row;
+  if (threadIdx.x == 0) bad = 0;
+  __syncthreads();
+  for (int j = 0; j < cs.nsel; ++j) {
+    u32 a = 0;
+    for (int b = threadIdx.x; b < nblk; b += TPB)
+      a += __ldcg(&cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j]);
+    const u32* h = fhist + ((long long)row * MAXC + j) * LB1;
+    const u32 mine = (threadIdx.x < LB1) ? __ldcg(&h[threadIdx.x]) : 0u;
+    u32 above, total;
+    block_excl_scan(a, &above);
+    block_excl_scan(mine, &total);
+    const long long K = cs.param[cs.sel[j]];
+    if (K <= (long long)above || K > (long long)above + (long long)total) {
+      if (threadIdx.x == 0) bad = 1;
+    } else {
+      block_find_kth_desc(h, LB1, (u32)K - above, res);
+      if (threadIdx.x == 0) {
+        const u32 c1 = __ldcg(&h[res[0]]);
+        s->above_hi[j] = above; s->fb1[j] = res[0]; s->fabove1[j] = above + res[1]; s->fc1[j] = c1;
+        if (c1 > (u32)FINAL_CAP) tickets[row * NTICKET + 13] = 1u;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    if (bad || __ldcg(&rowflag[row])) rowflag[row] = 1;   // bracket missed, or a segment overflowed
+    else if (tickets[row * NTICKET + 13]) atomicAdd(&flags[3], 1u);
+  }
+}
+
 // The streaming pass: D, ||v||^2, per bracket the count of keys >= hi and the energy of keys
 // < lo, the row maximum, and the keys inside a bracket appended to this CTA's list segment.
 // Sums run in binary32 chains of at most 4*FLUSH_TILES fused multiply-adds (relative error
@@ -1215,11 +1300,13 @@ constexpr int P1_SMEM = P1_STAGES * 3 * P1_TILE * 4;              // bytes of st
 template <int NSEL, bool ALIGNED, bool QMAX>
 __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
                                                const float* __restrict__ Y, long long d, CsetDev cs,
-                                               const SelRow* __restrict__ sel, double* __restrict__ partial,
+                                               SelRow* __restrict__ sel, double* __restrict__ partial,
                                                u32* __restrict__ cntpart, u64* __restrict__ list,
                                                u32* __restrict__ lcount, long long list_row, u32 segcap,
                                                u32* __restrict__ maxkey, u32* __restrict__ rowflag,
-                                               u32* __restrict__ diffflag, u32* __restrict__ flags) {
+                                               u32* __restrict__ diffflag, u32* __restrict__ flags,
+                                               u32* __restrict__ fhist, u32* __restrict__ tickets) {
+  pdl_begin();
   constexpr int NS = NSEL > 0 ? NSEL : 1;
   const int row = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -1228,10 +1315,12 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   __shared__ u32 sh_cnt, sh_abort;
   __shared__ u32 qcnt[TPB / 32];
   __shared__ __align__(8) u64 qbuf[TPB / 32][P1_QCAP];
+  __shared__ u32 lh[NS * LB1];                                   // first digit of key - lo, per bracket
   if (threadIdx.x == 0) { sh_cnt = 0; sh_abort = 0; }
   if (threadIdx.x < TPB / 32) qcnt[threadIdx.x] = 0;
-  u32 cnt[NS];
-  float lof[NS], hif[NS], fB[NS], fcnt[NS];
+  for (int i = threadIdx.x; i < NS * LB1; i += TPB) lh[i] = 0;
+  u32 cnt[NS], lou[NS], hiu[NS], shq[NS];
+  float fB[NS], fcnt[NS];
   double dB[NS];
   float lomin = __uint_as_float(0x7f800000u), fBall = 0.f;
   double dBall = 0.0;
@@ -1239,10 +1328,9 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   for (int j = 0; j < NS; ++j) {
     const u32 lo = (j < NSEL) ? sel[row].lo[j] : 0u;
     const u32 hi = (j < NSEL) ? sel[row].hi[j] : 0u;
-    lof[j] = __uint_as_float(lo);
-    hif[j] = __uint_as_float(hi >= 0x7f800000u ? 0x7f800000u : hi);  // "no upper edge" compares as +inf
+    lou[j] = lo; hiu[j] = hi; shq[j] = first_digit_shift(lo, hi);
     cnt[j] = 0; fB[j] = 0.f; fcnt[j] = 0.f; dB[j] = 0.0;
-    if (j < NSEL) lomin = fminf(lomin, lof[j]);
+    if (j < NSEL) lomin = fminf(lomin, __uint_as_float(lo));       // lo < 2^31 - 2^15: finite or +inf
   }
   float fD = 0.f, fE = 0.f;
   double dD = 0.0, dE = 0.0;
@@ -1279,17 +1367,19 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   // below (fB[j] holds only what fBall does not: keys in [lomin, lo_j)), list it if inside one.
   auto drain = [&](u32 slot, bool act) {
     const u64 e = act ? qbuf[wid][slot] : 0ull;
-    const float a = __uint_as_float((u32)(e >> 32));
+    const u32 ka = (u32)(e >> 32);
+    const float a = __uint_as_float(ka);
     bool inb = false;
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
-      const bool ge = a >= hif[j];
-      const bool below = a < lof[j];
+      const bool ge = ka >= hiu[j];
+      const bool below = ka < lou[j];
       fcnt[j] = (act && ge) ? fcnt[j] + 1.f : fcnt[j];       // exact: far fewer than 2^24 per flush
       fB[j] = (act && below) ? fmaf(a, a, fB[j]) : fB[j];
-      inb = inb || (!ge && !below);
+      const bool in = act && !ge && !below && j < NSEL;
+      if (in) atomicAdd(&lh[j * LB1 + ((ka - lou[j]) >> shq[j])], 1u);
+      inb = inb || in;
     }
-    inb = inb && act;
     const u32 m = __ballot_sync(0xffffffffu, inb);
     if (m) {
       u32 base = 0;
@@ -1423,6 +1513,15 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
     const u32 n = sh_cnt;
     lcount[pbase] = n < segcap ? n : segcap;
     if (n > segcap) atomicOr(&rowflag[row], 1u);
+  }
+  if (NSEL > 0) {
+    u32* gh = fhist + (long long)row * MAXC * LB1;
+    for (int i = threadIdx.x; i < NSEL * LB1; i += TPB) {
+      const u32 c = lh[i];
+      if (c) atomicAdd(&gh[i], c);
+    }
+    if (last_cta_of_row(&tickets[row * NTICKET + 11], gridDim.x))
+      first_digit_scan(cs, row, (int)gridDim.x, fhist, cntpart, sel, rowflag, tickets, flags);
   }
 }
 
@@ -1569,10 +1668,11 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
                                                u32* __restrict__ rowflag, u64* __restrict__ fl,
                                                u32* __restrict__ flcnt, const u32* __restrict__ cntpart,
                                                u32* __restrict__ tickets) {
+  pdl_begin();
   extern __shared__ u32 sh[];
   const int row = blockIdx.y;
   const int nsel = cs.nsel;
-  if (rowflag[row]) return;
+  if (rowflag[row] || !tickets[row * NTICKET + 13]) return;  // only rows whose first-digit bin is too full
   if (LEVEL == 3 && !tickets[row * NTICKET + 10]) return;  // no bracket of this row needs a third digit
   constexpr int NB = (LEVEL == 3) ? BINS3 : BINS1;
   for (int i = threadIdx.x; i < nsel * NB; i += TPB) sh[i] = 0;
@@ -1648,6 +1748,155 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
     lscan_row<LEVEL>(cs, row, nseg, (int)gridDim.x, hist, cntpart, lepart2, lepart3, sel, rowflag, fl, flcnt);
 }
 
+// ---- the usual case: the threshold's first-digit bin holds at most FINAL_CAP keys ----------------
+// Completes every bracket of a row from the keys collected out of the threshold's bin: a radix
+// select over the remaining low bits of key - lo (8 bits per round, one bin per thread) gives the
+// threshold, the counts above and equal, and how many threshold-equal keys are kept; those are the
+// ones with the lowest indices, found by ranking the equal keys' indices.
+__device__ __noinline__ void collected_finish_row(const CsetDev& cs, int row, int nlb, SelRow* __restrict__ sel,
+                                                  const u64* __restrict__ fl, const double* __restrict__ lepart) {
+  __shared__ u32 ek[FINAL_CAP];
+  __shared__ u32 hist[TPB];
+  __shared__ u32 res[3];
+  __shared__ u32 ties[1024];
+  __shared__ u32 nties_sh;
+  __shared__ double wsum_d[TPB / 32];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  SelRow* s = sel + row;
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 c1 = s->fc1[j];
+    const u32 K = (u32)cs.param[cs.sel[j]];
+    const u32 need = K - s->fabove1[j];               // 1 <= need <= c1 <= FINAL_CAP
+    const u32 shq = first_digit_shift(s->lo[j], s->hi[j]);
+    const u32 base = s->lo[j] + (s->fb1[j] << shq);   // every collected key lies in [base, base + 2^shq)
+    const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
+    for (u32 i = threadIdx.x; i < c1; i += TPB) ek[i] = (u32)(__ldcg(&f[i]) >> 32);
+    if (threadIdx.x == 0) { res[0] = 0; res[1] = 0; res[2] = c1; nties_sh = 0; }
+    __syncthreads();
+    u32 prefix = 0, pmask = 0, krem = need, neq = c1;
+    for (u32 bits = shq; bits > 0;) {
+      const u32 nb = bits < 8u ? bits : 8u, shift = bits - nb;
+      hist[threadIdx.x] = 0;
+      __syncthreads();
+      for (u32 i = threadIdx.x; i < c1; i += TPB) {
+        const u32 rel = ek[i] - base;
+        if ((rel & pmask) == prefix) atomicAdd(&hist[(rel >> shift) & ((1u << nb) - 1u)], 1u);
+      }
+      __syncthreads();
+      const u32 v = hist[TPB - 1 - threadIdx.x];      // bins in descending order
+      const u32 excl = block_excl_scan(v, nullptr);
+      if (krem > excl && krem <= excl + v) { res[0] = TPB - 1 - threadIdx.x; res[1] = excl; res[2] = v; }
+      __syncthreads();
+      prefix |= res[0] << shift;
+      pmask |= ((1u << nb) - 1u) << shift;
+      krem -= res[1];
+      neq = res[2];
+      bits = shift;
+      __syncthreads();
+    }
+    const u32 T = base + prefix, q = krem;            // q of the neq keys equal to T are kept
+    // energy of the listed keys in [lo, T): collected keys below T, then the per-CTA sums over lower bins
+    double e = 0.0;
+    for (u32 i = threadIdx.x; i < c1; i += TPB)
+      if (ek[i] < T) { const double kv = (double)__uint_as_float(ek[i]); e += kv * kv; }
+    for (int b = threadIdx.x; b < nlb; b += TPB) e += __ldcg(&lepart[((long long)row * LIST_BLK + b) * MAXC + j]);
+    e = warp_sum_f64(e);
+    if (lane == 0) wsum_d[wid] = e;
+    u32 mode = 0u;
+    if (q < neq) {
+      mode = 2u;
+      if (neq <= 1024u) {
+        mode = 1u;
+        for (u32 i = threadIdx.x; i < c1; i += TPB)
+          if (ek[i] == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)__ldcg(&f[i]);
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+      for (int w = 0; w < TPB / 32; ++w) tot += wsum_d[w];
+      s->T[j] = T; s->above[j] = K - q; s->ntie[j] = neq; s->q[j] = q; s->extraE[j] = tot;
+      s->tiemode[j] = mode;
+      if (mode != 1u) s->cut[j] = 0xffffffffu;   // mode 1: written below by the thread holding the q-th index
+    }
+    if (mode == 1u) {
+      for (u32 i = threadIdx.x; i < neq; i += TPB) {
+        const u32 mine = ties[i];
+        u32 rank = 0;
+        for (u32 k = 0; k < neq; ++k) rank += (ties[k] < mine) ? 1u : 0u;
+        if (rank == q - 1u) s->cut[j] = mine;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// One pass over the listed keys: energies below the threshold's first-digit bin, and the keys of
+// that bin collected for collected_finish_row; the last CTA of a row finishes it and, when no other
+// kernel has to contribute sums first (pick_here), chooses the row's level at once.
+__global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* __restrict__ sel,
+                                                  const u64* __restrict__ list, const u32* __restrict__ lcount,
+                                                  long long list_row, u32 segcap, double* __restrict__ lepart,
+                                                  const u32* __restrict__ rowflag, u64* __restrict__ fl,
+                                                  u32* __restrict__ flcnt, u32* __restrict__ tickets,
+                                                  int pick_here, long long d, int nblk_main,
+                                                  const double* __restrict__ partial, const u32* __restrict__ maxkey,
+                                                  RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
+                                                  const u32* __restrict__ diffflag, double tol) {
+  pdl_begin();
+  const int row = blockIdx.y;
+  const int nsel = cs.nsel;
+  if (rowflag[row] || tickets[row * NTICKET + 13]) return;
+  u32 lo[MAXC], hi[MAXC], shq[MAXC], b1[MAXC];
+  double en[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    lo[j] = (j < nsel) ? sel[row].lo[j] : 1u;
+    hi[j] = (j < nsel) ? sel[row].hi[j] : 0u;
+    shq[j] = first_digit_shift(lo[j], hi[j]);
+    b1[j] = (j < nsel) ? sel[row].fb1[j] : 0u;
+    en[j] = 0.0;
+  }
+  for (int sg = blockIdx.x; sg < nseg; sg += gridDim.x) {
+    const u32 n = lcount[(long long)row * MAX_BLK_PER_ROW + sg];
+    const u64* seg = list + (long long)row * list_row + (long long)sg * segcap;
+    for (u32 i = threadIdx.x; i < n; i += TPB) {
+      const u64 ent = seg[i];
+      const u32 key = (u32)(ent >> 32);
+#pragma unroll
+      for (int j = 0; j < MAXC; ++j) {
+        if (j < nsel && key >= lo[j] && key < hi[j]) {
+          const u32 d1 = (key - lo[j]) >> shq[j];
+          if (d1 < b1[j]) { const double kv = (double)__uint_as_float(key); en[j] += kv * kv; }
+          else if (d1 == b1[j]) {
+            const u32 pos = atomicAdd(&flcnt[row * MAXC + j], 1u);
+            if (pos < FINAL_CAP) fl[((long long)row * MAXC + j) * FINAL_CAP + pos] = ent;
+          }
+        }
+      }
+    }
+  }
+  __shared__ double red[MAXC][TPB / 32];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    const double vb = warp_sum_f64(en[j]);
+    if (lane == 0) red[j][wid] = vb;
+  }
+  __syncthreads();
+  if (threadIdx.x < MAXC) {
+    double a = 0;
+    for (int w = 0; w < TPB / 32; ++w) a += red[threadIdx.x][w];
+    lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
+  }
+  if (!last_cta_of_row(&tickets[row * NTICKET + 12], gridDim.x)) return;
+  collected_finish_row(cs, row, (int)gridDim.x, sel, fl, lepart);
+  if (pick_here) {
+    if (threadIdx.x < 32) pick_row(cs, d, row, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+    if (threadIdx.x == 0) tickets[row * NTICKET + 9] = 1u;
+  }
+}
+
 // --------------------------------------------------------------------------
 // host side
 // --------------------------------------------------------------------------
@@ -1657,7 +1906,7 @@ static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; 
 
 struct Layout {
   size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
-  size_t tickets, rowflag, diffflag, shist, lhist1, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
+  size_t tickets, rowflag, diffflag, shist, lhist1, fhist, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
 
@@ -1678,11 +1927,12 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
-  L.shist = L.lhist1 = L.flcnt = o;
+  L.shist = L.lhist1 = L.fhist = L.flcnt = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
     L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
+    L.fhist = o; o = align_up(o + (size_t)rows * MAXC * LB1 * 4, 256);
   }
   L.zero_end = o;
   L.flags = o; o = align_up(o + 16, 256);
@@ -1727,7 +1977,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->rowflag = (u32*)(b + L.rowflag);
   s->diffflag = (u32*)(b + L.diffflag);
   s->tickets = (u32*)(b + L.tickets);
-  s->shist = s->lhist1 = s->lcount = s->cntpart = nullptr;
+  s->shist = s->lhist1 = s->fhist = s->lcount = s->cntpart = nullptr;
   s->list = nullptr;
   s->lepart = nullptr;
   s->lepart3 = nullptr;
@@ -1737,6 +1987,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   if (single_pass) {
     s->shist = (u32*)(b + L.shist);
     s->lhist1 = (u32*)(b + L.lhist1);
+    s->fhist = (u32*)(b + L.fhist);
     s->list = (u64*)(b + L.list);
     s->lcount = (u32*)(b + L.lcount);
     s->cntpart = (u32*)(b + L.cntpart);
@@ -1787,6 +2038,20 @@ adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const 
 
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+// Launches a kernel, optionally as a programmatic dependent of the kernel before it on the stream:
+// its CTAs may be scheduled before that kernel has finished and wait in pdl_begin().
+template <typename... KArgs, typename... Args>
+static void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t shm, cudaStream_t stream, bool pdl,
+                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = shm; cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
                     long long d, const CompressOut& out, cudaStream_t stream) {
   int launches = 0;
@@ -1812,15 +2077,16 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     prof_end(pf, stream);          \
     ++launches;                    \
   } while (0)
-#define TIMED_AL(id, kern, grid, shm, ...)                                  \
-  TIMED(id, if (al) kern<true><<<grid, TPB, shm, stream>>>(__VA_ARGS__);    \
-            else kern<false><<<grid, TPB, shm, stream>>>(__VA_ARGS__))
+#define TIMED_AL(id, kern, grid, shm, ...)                                               \
+  TIMED(id, if (al) launch_k(kern<true>, grid, dim3(TPB), shm, stream, pdl, __VA_ARGS__);   \
+            else launch_k(kern<false>, grid, dim3(TPB), shm, stream, pdl, __VA_ARGS__))
+  const bool pdl = pf == nullptr;   // event records between kernels would break the pairing anyway
 
   if (cs.m == 0) {
     prof_begin(pf, KID_MEMSET, stream);
     if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
     prof_end(pf, stream);
-    TIMED(KID_PICK, (k_copy_report<<<(rows + 127) / 128, 128, 0, stream>>>(rows, d, 0, out)));
+    TIMED(KID_PICK, launch_k(k_copy_report, dim3((rows + 127) / 128), dim3(128), 0, stream, false, rows, d, 0, out));
     TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out, s.flags);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
@@ -1849,32 +2115,32 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
   double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
 
-#define TIMED_HIST(id, PASS, shm, hist)                                                                        \
-  TIMED(id, if (al) k_hist<PASS, true><<<fgrid, TPB, shm, stream>>>(X, G, d, cs, s.sel, hist, s.maxkey, only,    \
-                                                                    s.tickets, s.flags);                         \
-            else k_hist<PASS, false><<<fgrid, TPB, shm, stream>>>(X, G, d, cs, s.sel, hist, s.maxkey, only,      \
-                                                                  s.tickets, s.flags))
+#define TIMED_HIST(id, PASS, shm, hist)                                                                          \
+  TIMED(id, if (al) launch_k(k_hist<PASS, true>, fgrid, dim3(TPB), shm, stream, pdl, X, G, d, cs, s.sel, hist,    \
+                             s.maxkey, only, s.tickets, s.flags);                                                  \
+            else launch_k(k_hist<PASS, false>, fgrid, dim3(TPB), shm, stream, pdl, X, G, d, cs, s.sel, hist,      \
+                          s.maxkey, only, s.tickets, s.flags))
 #define P1_ARGS                                                                                               \
   X, G, Y, d, cs, s.sel, s.partial, s.cntpart, s.list, s.lcount, s.list_row, segcap, s.maxkey, s.rowflag,     \
-      s.diffflag, s.flags
+      s.diffflag, s.flags, s.fhist, s.tickets
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
     if (al) {                                                                                                       \
       if (cs.nquant) {                                                                                              \
         cudaFuncSetAttribute(k_pass1<N, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);         \
-        k_pass1<N, true, true><<<sgrid, TPB, P1_SMEM, stream>>>(P1_ARGS);                                           \
+        launch_k(k_pass1<N, true, true>, sgrid, dim3(TPB), P1_SMEM, stream, pdl, P1_ARGS);                          \
       } else {                                                                                                      \
         cudaFuncSetAttribute(k_pass1<N, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);        \
-        k_pass1<N, true, false><<<sgrid, TPB, P1_SMEM, stream>>>(P1_ARGS);                                          \
+        launch_k(k_pass1<N, true, false>, sgrid, dim3(TPB), P1_SMEM, stream, pdl, P1_ARGS);                         \
       }                                                                                                             \
     } else {                                                                                                        \
-      k_pass1<N, false, true><<<sgrid, TPB, 0, stream>>>(P1_ARGS);                                                  \
+      launch_k(k_pass1<N, false, true>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                 \
     }                                                                                                               \
     break;
-#define LIST_PASS(LEVEL, shm, hist)                                                                               \
-  TIMED(KID_LHIST, (k_lhist<LEVEL><<<lgrid, TPB, shm, stream>>>(cs, nblk, s.sel, s.list, s.lcount, s.list_row,    \
-                                                                segcap, hist, s.lepart, s.lepart3, s.rowflag,     \
-                                                                s.fl, s.flcnt, s.cntpart, s.tickets)))
+#define LIST_PASS(LEVEL, shm, hist)                                                                              \
+  TIMED(KID_LHIST, launch_k(k_lhist<LEVEL>, lgrid, dim3(TPB), shm, stream, pdl, cs, nblk, s.sel, s.list,         \
+                            s.lcount, s.list_row, segcap, hist, s.lepart, s.lepart3, s.rowflag, s.fl, s.flcnt,   \
+                            s.cntpart, s.tickets))
 
   if (single) {
     // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
@@ -1898,11 +2164,16 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     ++launches;
     // 3. exact selection among the listed keys by the digits of key - lo: two passes, each finished by its
     //    last CTA; the third only does work for brackets wider than 2^22 key values
+    tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
     const dim3 lgrid(nblk < LIST_BLK ? nblk : LIST_BLK, rows);
+    TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), 0, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
+                                 s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
+                                 cs.nquant == 0 ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
+                                 s.diffflag, tol));
+    // rows whose first-digit bin holds too many keys: three digit levels of 11, 11 and 9 bits (usually no row)
     LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
     LIST_PASS(2, cs.nsel * BINS2 * 4, s.hist2);
     LIST_PASS(3, cs.nsel * BINS3 * 4, s.hist3);
-    tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
   }
   // the full radix select: every row, or (single-pass mode) only rows whose bracket failed
   if (cs.nsel || cs.nquant) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
@@ -1912,7 +2183,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   }
   TIMED_AL(KID_ENERGY, k_energy, fgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
   if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
-  TIMED(KID_PICK, (k_pick<<<rows, 32, 0, stream>>>(cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey, s.dec, s.flags, out, s.diffflag, single ? 1 : 0, tol)));
+  TIMED(KID_PICK, launch_k(k_pick, dim3(rows), dim3(32), 0, stream, pdl, cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey,
+                           s.dec, s.flags, out, s.diffflag, single ? s.tickets : nullptr, tol));
   TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag, d, out, s.tickets, s.flags);
   if (cs.nsel) {
     long long tgx = (148 * 4 + rows - 1) / rows;
@@ -1933,6 +2205,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
 // small vector kernels of the loop
 // --------------------------------------------------------------------------
 __global__ void k_axpy(float* __restrict__ x, const float* __restrict__ g, float gamma, long long d) {
+  pdl_begin();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));
 }
@@ -1944,6 +2217,7 @@ int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t
 }
 
 __global__ void k_mean_rows(const float* __restrict__ G, int rows, long long d, float* __restrict__ out) {
+  pdl_begin();
   const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= d) return;
   float acc = G[c];

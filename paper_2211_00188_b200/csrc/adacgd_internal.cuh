@@ -22,7 +22,10 @@ constexpr int UPD_COLS = TPB * 4;   // columns per CTA of the update kernel (als
 constexpr int MAX_BLK_PER_ROW = 2048;
 constexpr int SBINS = 65536;        // sample histogram: key bits [30:15]
 constexpr int LIST_BLK = 256;       // CTAs per row of the passes over the candidate lists
-constexpr int NTICKET = 12;         // per-row words: completion counters 0 sample, 1-3 list levels, 4-6 full passes, 7 exact, 8 ties; 10 = a third list level is needed
+constexpr int NTICKET = 16;         // per-row words: completion counters 0 sample, 1-3 list levels, 4-6 full passes, 7 exact, 8 ties,
+                                    // 11 streaming pass, 12 collection pass; flags 9 = level already picked, 10 = a third list
+                                    // level is needed, 13 = the row takes the three-level list passes
+constexpr int LB1 = 256;            // bins of the first digit of key - lo histogrammed by the streaming pass
 constexpr int FINAL_CAP = 2048;     // entries kept per bracket for ranking threshold-equal keys by index
 constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 every 16 tiles (64 terms)
 
@@ -30,7 +33,7 @@ constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LSCAN, KID_COUNT
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_COUNT
 };
 struct Prof {
   int cap, used;
@@ -73,6 +76,9 @@ struct SelRow {
   // indices as ranked by the chunk-prefix pass (k_tiecount / k_tiescan)
   u32 tiemode[MAXC], cut[MAXC];
   u32 sh1[MAXC], sh2[MAXC];     // digit shifts of key - lo inside the bracket
+  // first digit (8 bits) of key - lo as histogrammed by the streaming pass: bin holding the K-th
+  // largest key, #keys above that bin, #keys inside it
+  u32 fb1[MAXC], fabove1[MAXC], fc1[MAXC];
 };
 
 // Decision for one row, consumed by the update kernel.
@@ -102,7 +108,8 @@ struct Scratch {
   u32* tiecnt;     // [rows][nchunk]  (exclusive prefix after the scan)
   // single-pass path (null when the scratch was carved without it)
   u32* shist;      // [rows][SBINS] sample histogram
-  u32* lhist1;     // [rows][MAXC][BINS1] first digit of the listed keys, per bracket
+  u32* lhist1;     // [rows][MAXC][BINS1] first digit of the listed keys, per bracket (three-level passes)
+  u32* fhist;      // [rows][MAXC][LB1] first digit as histogrammed by the streaming pass
   u64* list;       // [rows][list_row] (key << 32 | index), one segment of segcap entries per CTA
   u32* lcount;     // [rows][MAX_BLK_PER_ROW] entries per segment
   u32* cntpart;    // [rows][MAX_BLK_PER_ROW][MAXC] per-CTA counts of keys >= hi
