@@ -1130,13 +1130,15 @@ __device__ u32 sample_rank_bin(const u32* __restrict__ h, const u32* csum, const
 
 // Per row and Top-K candidate: a bracket [lo, hi) of key values, aligned to sample bins, that
 // holds the K-th largest key with overwhelming probability (checked exactly afterwards).
+// Called by a whole CTA of any size that is a multiple of 32 threads.
 __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sample,
                             const u32* __restrict__ shist, SelRow* __restrict__ sel, u32* __restrict__ tickets) {
-  __shared__ u32 csum[TPB], cexcl[TPB];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  __shared__ u32 csum[256], cexcl[256];
+  __shared__ u32 s_total;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const u32* h = shist + (long long)row * SBINS;
   // chunk sums, four chunks (eight 16-byte loads) in flight per warp
-  for (int c0 = wid * 4; c0 < 256; c0 += (TPB / 32) * 4) {
+  for (int c0 = wid * 4; c0 < 256; c0 += nwarp * 4) {
     uint4 a[4], b[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -1151,12 +1153,25 @@ __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sa
     }
   }
   __syncthreads();
-  u32 S;
-  const u32 ex = block_excl_scan(csum[threadIdx.x], &S);
-  cexcl[threadIdx.x] = ex;
+  if (wid == 0) {  // exclusive prefix over the 256 chunk sums: eight per lane
+    u32 loc[8], sum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { loc[k] = csum[lane * 8 + k]; sum += loc[k]; }
+    u32 inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    u32 run = inc - sum;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { cexcl[lane * 8 + k] = run; run += loc[k]; }
+    if (lane == 31) s_total = inc;
+  }
   __syncthreads();
+  const u32 S = s_total;
   // one warp per (candidate, edge)
-  for (int w = wid; w < 2 * cs.nsel; w += TPB / 32) {
+  for (int w = wid; w < 2 * cs.nsel; w += nwarp) {
     const int j = w >> 1;
     const bool upper = (w & 1) == 0;
     const double K = (double)cs.param[cs.sel[j]];
@@ -1185,43 +1200,57 @@ __device__ void bracket_row(const CsetDev& cs, int row, long long d, int full_sa
   }
 }
 
-// Every `stride`-th tile of a row is sampled; the histogram has one bin per value of
-// key[30:15].  Per-CTA counts are 16 bit (two bins per shared word), so a CTA takes at most
-// 63 tiles.
+// The sample of a row: its d elements are cut into granules of SAMP_G consecutive elements (64
+// bytes), the granules into windows of `win`, and one granule of every window is taken, at an
+// offset that changes from window to window (a hash of the window index), so that neither a period
+// nor a block structure of the data lines up with the sample.  The histogram has one bin per value
+// of key[30:15].  Per-CTA counts are 16 bit (two bins per shared word): a CTA takes fewer than
+// 65536 elements.  Four threads share a granule; SAMP_NL granules are in flight per thread.
+constexpr int SAMP_TPB = 1024;
+constexpr int SAMP_G = 16;
+constexpr int SAMP_NL = 4;
+__device__ __forceinline__ long long sample_granule(long long w, long long win, long long ngran) {
+  const long long first = w * win;
+  const long long span = (ngran - first < win) ? (ngran - first) : win;
+  u32 h = (u32)w * 2654435761u;
+  h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+  return first + (long long)(h % (u32)span);
+}
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
-                                                long long d, long long nsamp, long long stride,
-                                                u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
-                                                u32* __restrict__ tickets) {
+__global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
+                                                     long long d, long long nwin, long long win,
+                                                     u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
+                                                     u32* __restrict__ tickets) {
   pdl_begin();
-  extern __shared__ u32 sh[];  // SBINS / 2 words
+  extern __shared__ __align__(16) u32 sh[];  // SBINS / 2 words
   const int row = blockIdx.y;
-  for (int i = threadIdx.x; i < SBINS / 2; i += TPB) sh[i] = 0;
+  for (int i = threadIdx.x; i < SBINS / 8; i += SAMP_TPB) reinterpret_cast<uint4*>(sh)[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
-  // four sampled tiles per round, all loads issued before the first histogram update
-  for (long long s0 = blockIdx.x; s0 < nsamp; s0 += 4ll * gridDim.x) {
-    float x[4][4], g[4][4];
-    bool on[4];
+  const long long ngran = (d + SAMP_G - 1) / SAMP_G;
+  const long long nquad = (long long)gridDim.x * (SAMP_TPB / 4);
+  const int ql = threadIdx.x & 3;
+  for (long long w0 = (long long)blockIdx.x * (SAMP_TPB / 4) + (threadIdx.x >> 2); w0 < nwin; w0 += nquad * SAMP_NL) {
+    float x[SAMP_NL][4], g[SAMP_NL][4];
+    long long c0[SAMP_NL];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const long long sidx = s0 + (long long)u * gridDim.x;
-      const long long c0 = (sidx * stride + (stride >> 1)) * (TPB * 4) + threadIdx.x * 4;
-      on[u] = sidx < nsamp && c0 < d;
-      if (on[u]) {
-        load4<ALIGNED>(xr, c0, d, x[u]);
-        load4<ALIGNED>(gr, c0, d, g[u]);
+    for (int u = 0; u < SAMP_NL; ++u) {
+      const long long w = w0 + (long long)u * nquad;
+      c0[u] = d;
+      if (w < nwin) {
+        c0[u] = sample_granule(w, win, ngran) * SAMP_G + ql * 4;
+        if (c0[u] < d) {
+          load4<ALIGNED>(xr, c0[u], d, x[u]);
+          load4<ALIGNED>(gr, c0[u], d, g[u]);
+        }
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (!on[u]) continue;
-      const long long sidx = s0 + (long long)u * gridDim.x;
-      const long long c0 = (sidx * stride + (stride >> 1)) * (TPB * 4) + threadIdx.x * 4;
+    for (int u = 0; u < SAMP_NL; ++u) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        if (!ALIGNED && c0 + k >= d) break;
+        if (c0[u] + k >= d) break;
         const u32 bin = key_of(__fsub_rn(x[u][k], g[u][k])) >> 15;
         atomicAdd(&sh[bin >> 1], (bin & 1u) ? 0x10000u : 1u);
       }
@@ -1229,13 +1258,13 @@ __global__ void __launch_bounds__(TPB) k_sample(const float* __restrict__ X, con
   }
   __syncthreads();
   u32* gh = shist + (long long)row * SBINS;
-  for (int i = threadIdx.x; i < SBINS / 2; i += TPB) {
+  for (int i = threadIdx.x; i < SBINS / 2; i += SAMP_TPB) {
     const u32 w = sh[i];
     if (w & 0xffffu) atomicAdd(&gh[2 * i], w & 0xffffu);
     if (w >> 16) atomicAdd(&gh[2 * i + 1], w >> 16);
   }
   if (last_cta_of_row(&tickets[row * NTICKET + 0], gridDim.x))
-    bracket_row(cs, row, d, stride == 1 ? 1 : 0, shist, sel, tickets);
+    bracket_row(cs, row, d, win == 1 ? 1 : 0, shist, sel, tickets);
 }
 
 // Shift that leaves the first LB1-valued digit of key - lo for a bracket [lo, hi).
@@ -1291,36 +1320,39 @@ __device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, int nb
 // < lo, the row maximum, and the keys inside a bracket appended to this CTA's list segment.
 // Sums run in binary32 chains of at most 4*FLUSH_TILES fused multiply-adds (relative error
 // <= (4*FLUSH_TILES + 1) 2^-24 for non-negative terms), folded into binary64.
-// With ALIGNED rows the three streams are staged through shared memory by bulk asynchronous
-// copies, P1_STAGES tiles ahead of the arithmetic; otherwise plain loads are used.
-constexpr int P1_STAGES = 3;
+// Every warp runs on its own: P1_UNR tiles of plain 128-bit loads are in flight per thread, and
+// the keys that reach the lowest bracket edge (about K_max/d of them) go through a per-warp queue
+// compacted with warp votes, drained 32 entries at a time; there is no CTA-wide barrier in the loop.
+constexpr int P1_UNR = 3;                                         // tiles in flight per CTA iteration
 constexpr int P1_QCAP = 160;                                      // 31 left over + 128 new entries per warp
-constexpr int P1_TILE = TPB * 4;                                  // elements per tile and stream
-constexpr int P1_SMEM = P1_STAGES * 3 * P1_TILE * 4;              // bytes of staging per CTA
+constexpr int P1_FLUSH_IT = FLUSH_TILES / P1_UNR;                 // iterations between folds into binary64
+#ifndef P1_MINB3
+#define P1_MINB3 4
+#endif
+// resident CTAs per SM the register budget is set for: more brackets need more state per thread
+constexpr int p1_min_ctas(int nsel) { return nsel <= 3 ? P1_MINB3 : (nsel <= 5 ? 3 : 2); }
 template <int NSEL, bool ALIGNED, bool QMAX>
-__global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
-                                               const float* __restrict__ Y, long long d, CsetDev cs,
-                                               SelRow* __restrict__ sel, double* __restrict__ partial,
-                                               u32* __restrict__ cntpart, u64* __restrict__ list,
-                                               u32* __restrict__ lcount, long long list_row, u32 segcap,
-                                               u32* __restrict__ maxkey, u32* __restrict__ rowflag,
-                                               u32* __restrict__ diffflag, u32* __restrict__ flags,
-                                               u32* __restrict__ fhist, u32* __restrict__ tickets) {
+__global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
+                                                  const float* __restrict__ Y, long long d, CsetDev cs,
+                                                  SelRow* __restrict__ sel, double* __restrict__ partial,
+                                                  u32* __restrict__ cntpart, u64* __restrict__ list,
+                                                  u32* __restrict__ lcount, long long list_row, u32 segcap,
+                                                  u32* __restrict__ maxkey, u32* __restrict__ rowflag,
+                                                  u32* __restrict__ diffflag, u32* __restrict__ flags,
+                                                  u32* __restrict__ fhist, u32* __restrict__ tickets) {
   pdl_begin();
   constexpr int NS = NSEL > 0 ? NSEL : 1;
   const int row = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  extern __shared__ __align__(128) float stage[];                 // [P1_STAGES][3][P1_TILE], ALIGNED only
-  __shared__ __align__(8) u64 full_bar[P1_STAGES];
-  __shared__ u32 sh_cnt, sh_abort;
-  __shared__ u32 qcnt[TPB / 32];
+  __shared__ u32 sh_cnt;
   __shared__ __align__(8) u64 qbuf[TPB / 32][P1_QCAP];
   __shared__ u32 lh[NS * LB1];                                   // first digit of key - lo, per bracket
-  if (threadIdx.x == 0) { sh_cnt = 0; sh_abort = 0; }
-  if (threadIdx.x < TPB / 32) qcnt[threadIdx.x] = 0;
+  if (threadIdx.x == 0) sh_cnt = 0;
   for (int i = threadIdx.x; i < NS * LB1; i += TPB) lh[i] = 0;
-  u32 cnt[NS], lou[NS], hiu[NS], shq[NS];
-  float fB[NS], fcnt[NS];
+  // bracket edges and digit shifts are only read when a queue is drained: kept in shared memory
+  __shared__ u32 s_lo[NS], s_hi[NS], s_shq[NS];
+  u32 cnt[NS];
+  float fB[NS];
   double dB[NS];
   float lomin = __uint_as_float(0x7f800000u), fBall = 0.f;
   double dBall = 0.0;
@@ -1328,8 +1360,8 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   for (int j = 0; j < NS; ++j) {
     const u32 lo = (j < NSEL) ? sel[row].lo[j] : 0u;
     const u32 hi = (j < NSEL) ? sel[row].hi[j] : 0u;
-    lou[j] = lo; hiu[j] = hi; shq[j] = first_digit_shift(lo, hi);
-    cnt[j] = 0; fB[j] = 0.f; fcnt[j] = 0.f; dB[j] = 0.0;
+    if (threadIdx.x == 0) { s_lo[j] = lo; s_hi[j] = hi; s_shq[j] = first_digit_shift(lo, hi); }
+    cnt[j] = 0; fB[j] = 0.f; dB[j] = 0.0;
     if (j < NSEL) lomin = fminf(lomin, __uint_as_float(lo));       // lo < 2^31 - 2^15: finite or +inf
   }
   float fD = 0.f, fE = 0.f;
@@ -1341,28 +1373,7 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
   const float* yr = Y + (long long)row * d;
   u64* seg = list + (long long)row * list_row + (long long)blockIdx.x * segcap;
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  const long long nmy = (ntile > (long long)blockIdx.x) ? (ntile - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  // producer side of the pipeline: one thread issues the three copies of a tile and arms its barrier
-  auto issue = [&](long long i) {
-    const long long t = (long long)blockIdx.x + i * gridDim.x;
-    const long long e0 = t * P1_TILE;
-    const u32 bytes = (u32)(((d - e0 < P1_TILE) ? (d - e0) : P1_TILE) * 4);
-    const int sidx = (int)(i % P1_STAGES);
-    float* buf = stage + (size_t)sidx * 3 * P1_TILE;
-    mbar_expect_tx(&full_bar[sidx], 3 * bytes);
-    bulk_load(buf, xr + e0, bytes, &full_bar[sidx]);
-    bulk_load(buf + P1_TILE, gr + e0, bytes, &full_bar[sidx]);
-    bulk_load(buf + 2 * P1_TILE, yr + e0, bytes, &full_bar[sidx]);
-  };
-  if (ALIGNED) {
-    if (threadIdx.x == 0) {
-      for (int q = 0; q < P1_STAGES; ++q) mbar_init(&full_bar[q], 1);
-      mbar_fence_init();
-    }
-    __syncthreads();
-    if (threadIdx.x == 0)
-      for (long long i = 0; i < nmy && i < P1_STAGES; ++i) issue(i);
-  }
+  const u32 ltmask = (1u << lane) - 1u;
   // A queued entry meets every bracket: count it if it lies above, add its square if it lies
   // below (fB[j] holds only what fBall does not: keys in [lomin, lo_j)), list it if inside one.
   auto drain = [&](u32 slot, bool act) {
@@ -1372,12 +1383,13 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
     bool inb = false;
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
-      const bool ge = ka >= hiu[j];
-      const bool below = ka < lou[j];
-      fcnt[j] = (act && ge) ? fcnt[j] + 1.f : fcnt[j];       // exact: far fewer than 2^24 per flush
+      const u32 lo = s_lo[j];
+      const bool ge = ka >= s_hi[j];
+      const bool below = ka < lo;
+      cnt[j] += (act && ge) ? 1u : 0u;
       fB[j] = (act && below) ? fmaf(a, a, fB[j]) : fB[j];
       const bool in = act && !ge && !below && j < NSEL;
-      if (in) atomicAdd(&lh[j * LB1 + ((ka - lou[j]) >> shq[j])], 1u);
+      if (in) atomicAdd(&lh[j * LB1 + ((ka - lo) >> s_shq[j])], 1u);
       inb = inb || in;
     }
     const u32 m = __ballot_sync(0xffffffffu, inb);
@@ -1385,94 +1397,88 @@ __global__ void __launch_bounds__(TPB) k_pass1(const float* __restrict__ X, cons
       u32 base = 0;
       if (lane == 0) base = atomicAdd(&sh_cnt, (u32)__popc(m));
       base = __shfl_sync(0xffffffffu, base, 0);
-      const u32 pos = base + (u32)__popc(m & ((1u << lane) - 1u));
+      const u32 pos = base + (u32)__popc(m & ltmask);
       if (inb && pos < segcap) seg[pos] = e;
     }
   };
+  u32 qc = 0;  // entries waiting in this warp's queue: the same value in every lane
   int it = 0;
-  for (long long i = 0; i < nmy; ++i, ++it) {
-    const long long t = (long long)blockIdx.x + i * gridDim.x;
-    const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
-    const bool live = c0 < d;
-    float x[4] = {0.f, 0.f, 0.f, 0.f}, g[4] = {0.f, 0.f, 0.f, 0.f}, y[4] = {0.f, 0.f, 0.f, 0.f};
-    if (ALIGNED) {
-      const int sidx = (int)(i % P1_STAGES);
-      if (!mbar_wait_bounded(&full_bar[sidx], (u32)((i / P1_STAGES) & 1))) sh_abort = 1;
-      else if (live) {
-        const float* buf = stage + (size_t)sidx * 3 * P1_TILE + threadIdx.x * 4;
-        const float4 a = *reinterpret_cast<const float4*>(buf);
-        const float4 b = *reinterpret_cast<const float4*>(buf + P1_TILE);
-        const float4 c = *reinterpret_cast<const float4*>(buf + 2 * P1_TILE);
-        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-        g[0] = b.x; g[1] = b.y; g[2] = b.z; g[3] = b.w;
-        y[0] = c.x; y[1] = c.y; y[2] = c.z; y[3] = c.w;
-      }
-    } else if (live) {
-      load4<ALIGNED>(xr, c0, d, x);
-      load4<ALIGNED>(gr, c0, d, g);
-      load4<ALIGNED>(yr, c0, d, y);
-    }
-    float av[4];
-    u32 rm = 0;  // which of the four entries reach the lowest bracket edge
+  for (long long t0 = blockIdx.x; t0 < ntile; t0 += (long long)gridDim.x * P1_UNR, ++it) {
+    float x[P1_UNR][4], g[P1_UNR][4], y[P1_UNR][4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float v = __fsub_rn(x[k], g[k]);
-      const float w = __fsub_rn(x[k], y[k]);
-      fE = fmaf(v, v, fE);
-      fD = fmaf(w, w, fD);
-      av[k] = fabsf(v);
-      if (QMAX) mx = max(mx, __float_as_uint(av[k]));
-      df |= __float_as_uint(v) ^ __float_as_uint(w);
-      if (NSEL > 0) {
-        // finite non-negative binary32 values order like their bit patterns: compare as floats
-        const bool small = av[k] < lomin;
-        fBall = small ? fmaf(v, v, fBall) : fBall;
-        if (!small && (ALIGNED || c0 + k < d)) rm |= 1u << k;
-      }
-    }
-    if (NSEL > 0) {
-      if (live && rm) {  // zero padding of dead lanes is never queued
-        u32 pos = atomicAdd(&qcnt[wid], (u32)__popc(rm));
+    for (int u = 0; u < P1_UNR; ++u) {
+      const long long c0 = (t0 + (long long)u * gridDim.x) * (TPB * 4) + threadIdx.x * 4;
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (rm & (1u << k)) qbuf[wid][pos++] = ((u64)__float_as_uint(av[k]) << 32) | (u64)(u32)(c0 + k);
-      }
-      __syncwarp();
-      u32 qc = *reinterpret_cast<volatile u32*>(&qcnt[wid]);
-      if (qc >= 32) {
-        do { qc -= 32; drain(qc + lane, true); } while (qc >= 32);
-        __syncwarp();
-        if (lane == 0) qcnt[wid] = qc;
-        __syncwarp();
+      for (int k = 0; k < 4; ++k) { x[u][k] = 0.f; g[u][k] = 0.f; y[u][k] = 0.f; }
+      if (c0 < d) {
+        if (ALIGNED) {  // streamed once: evict-first loads
+          const float4 a = __ldcs(reinterpret_cast<const float4*>(xr + c0));
+          const float4 b = __ldcs(reinterpret_cast<const float4*>(gr + c0));
+          const float4 c = __ldcs(reinterpret_cast<const float4*>(yr + c0));
+          x[u][0] = a.x; x[u][1] = a.y; x[u][2] = a.z; x[u][3] = a.w;
+          g[u][0] = b.x; g[u][1] = b.y; g[u][2] = b.z; g[u][3] = b.w;
+          y[u][0] = c.x; y[u][1] = c.y; y[u][2] = c.z; y[u][3] = c.w;
+        } else {
+          load4<false>(xr, c0, d, x[u]);
+          load4<false>(gr, c0, d, g[u]);
+          load4<false>(yr, c0, d, y[u]);
+        }
       }
     }
-    if ((it & (FLUSH_TILES - 1)) == FLUSH_TILES - 1) {
+#pragma unroll
+    for (int u = 0; u < P1_UNR; ++u) {
+      const long long c0 = (t0 + (long long)u * gridDim.x) * (TPB * 4) + threadIdx.x * 4;
+      float av[4];
+      u32 rm = 0;  // which of the four entries reach the lowest bracket edge
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float v = __fsub_rn(x[u][k], g[u][k]);
+        const float w = __fsub_rn(x[u][k], y[u][k]);
+        fE = fmaf(v, v, fE);
+        fD = fmaf(w, w, fD);
+        av[k] = fabsf(v);
+        if (QMAX) mx = max(mx, __float_as_uint(av[k]));
+        df |= __float_as_uint(v) ^ __float_as_uint(w);
+        if (NSEL > 0) {
+          // finite non-negative binary32 values order like their bit patterns: compare as floats
+          const bool small = av[k] < lomin;
+          fBall = small ? fmaf(v, v, fBall) : fBall;
+          if (!small && (ALIGNED || c0 + k < d)) rm |= 1u << k;
+        }
+      }
+      if (ALIGNED && c0 >= d) rm = 0u;                             // zero padding past the row end is never queued
+      if (NSEL > 0 && __any_sync(0xffffffffu, rm != 0u)) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const bool p = (rm >> k) & 1u;
+          const u32 m = __ballot_sync(0xffffffffu, p);
+          if (p) qbuf[wid][qc + (u32)__popc(m & ltmask)] = ((u64)__float_as_uint(av[k]) << 32) | (u64)(u32)(c0 + k);
+          qc += (u32)__popc(m);
+        }
+        if (qc >= 32) {
+          __syncwarp();
+          do { qc -= 32; drain(qc + lane, true); } while (qc >= 32);
+          __syncwarp();
+        }
+      }
+    }
+    if (it % P1_FLUSH_IT == P1_FLUSH_IT - 1) {
       dD += (double)fD; fD = 0.f;
       dE += (double)fE; fE = 0.f;
       dBall += (double)fBall; fBall = 0.f;
 #pragma unroll
-      for (int j = 0; j < NS; ++j) {
-        dB[j] += (double)fB[j]; fB[j] = 0.f;
-        cnt[j] += (u32)fcnt[j]; fcnt[j] = 0.f;
-      }
-    }
-    if (ALIGNED) {
-      __syncthreads();                       // every thread has read this stage
-      if (sh_abort) break;                   // a copy never arrived: give up, the host is told
-      if (threadIdx.x == 0 && i + P1_STAGES < nmy) issue(i + P1_STAGES);
+      for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; fB[j] = 0.f; }
     }
   }
-  if (ALIGNED && sh_abort && threadIdx.x == 0) atomicOr(&flags[0], 2u);
   if (NSEL > 0) {  // what is left in the queue: fewer than 32 entries
     __syncwarp();
-    const u32 qc = *reinterpret_cast<volatile u32*>(&qcnt[wid]);
-    if (qc) drain((u32)lane, (u32)lane < qc);
+    if (qc) drain((u32)lane < qc ? (u32)lane : 0u, (u32)lane < qc);
   }
   dD += (double)fD;
   dE += (double)fE;
   dBall += (double)fBall;
 #pragma unroll
-  for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j] + dBall; cnt[j] += (u32)fcnt[j]; }
+  for (int j = 0; j < NS; ++j) dB[j] += (double)fB[j] + dBall;
 
   __shared__ double red[2 + NS][TPB / 32];
   __shared__ u32 redc[NS][TPB / 32];
@@ -2101,6 +2107,9 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
   long long want = (148 * 8 + rows - 1) / rows;
+  // a CTA takes at least eight tiles (spread over the row by the grid stride) where the row has them, so
+  // that its share of the key list is sized for an average over the row rather than for one tile
+  if (single && want > (ntile + 7) / 8) want = (ntile + 7) / 8;
   if (want > ntile) want = ntile;
   if (want > MAX_BLK_PER_ROW) want = MAX_BLK_PER_ROW;
   if (want < 1) want = 1;
@@ -2126,13 +2135,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
     if (al) {                                                                                                       \
-      if (cs.nquant) {                                                                                              \
-        cudaFuncSetAttribute(k_pass1<N, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);         \
-        launch_k(k_pass1<N, true, true>, sgrid, dim3(TPB), P1_SMEM, stream, pdl, P1_ARGS);                          \
-      } else {                                                                                                      \
-        cudaFuncSetAttribute(k_pass1<N, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM);        \
-        launch_k(k_pass1<N, true, false>, sgrid, dim3(TPB), P1_SMEM, stream, pdl, P1_ARGS);                         \
-      }                                                                                                             \
+      if (cs.nquant) launch_k(k_pass1<N, true, true>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                   \
+      else launch_k(k_pass1<N, true, false>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                            \
     } else {                                                                                                        \
       launch_k(k_pass1<N, false, true>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                 \
     }                                                                                                               \
@@ -2144,15 +2148,24 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
 
   if (single) {
     // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
-    long long stride = ntile / 128;
-    if (stride < 1) stride = 1;
-    if (stride > 64) stride = 64;
-    const long long nsamp = ntile / stride;
-    long long sgx = (148 + rows - 1) / rows;          // about one wave of CTAs over all rows
-    if (sgx < (nsamp + 62) / 63) sgx = (nsamp + 62) / 63;  // 16-bit per-CTA counters: at most 63 tiles each
-    if (sgx > nsamp) sgx = nsamp;
+    // windows of `win` granules, one granule sampled per window: at least 8192 granules (131072
+    // elements) where the row has that many, at most every 64th granule
+    const long long ngran = (d + SAMP_G - 1) / SAMP_G;
+    long long win = ngran / 8192;
+    if (win < 1) win = 1;
+    if (win > 64) win = 64;
+    const long long nwin = (ngran + win - 1) / win;
+    long long sgx = (148 + rows - 1) / rows;          // about one CTA per SM over all rows
+    const long long per_cta = 49152 / SAMP_G;         // 16-bit per-CTA counters: fewer than 65536 elements each
+    if (sgx < (nwin + per_cta - 1) / per_cta) sgx = (nwin + per_cta - 1) / per_cta;
+    const long long quads = SAMP_TPB / 4;
+    if (sgx > (nwin + quads - 1) / quads) sgx = (nwin + quads - 1) / quads;
     const dim3 samp_grid((unsigned)sgx, rows);
-    TIMED_AL(KID_SAMPLE, k_sample, samp_grid, SBINS * 2, X, G, d, nsamp, stride, s.shist, cs, s.sel, s.tickets);
+    prof_begin(pf, KID_SAMPLE, stream);
+    if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets);
+    else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets);
+    prof_end(pf, stream);
+    ++launches;
     // 2. the one pass over X, G, Y
     const u32 segcap = (u32)(s.list_row / nblk);
     prof_begin(pf, KID_PASS1, stream);

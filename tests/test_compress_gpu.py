@@ -237,18 +237,44 @@ def test_host_entry_point(torch):
     assert level.tolist() == [r["level"] for r in res] and bits.tolist() == [r["bits"] for r in res]
 
 
+def sampled_granules(d):
+    """The granules (16 consecutive entries) of a row of d entries that the sampling kernel reads:
+    one per window of `win` granules, at an offset hashed from the window index."""
+    ngran = (d + 15) // 16
+    win = min(max(ngran // 8192, 1), 64)
+    w = np.arange((ngran + win - 1) // win, dtype=np.uint64)
+    h = (w * np.uint64(2654435761)) & np.uint64(0xFFFFFFFF)
+    h ^= h >> np.uint64(15)
+    h = (h * np.uint64(2246822519)) & np.uint64(0xFFFFFFFF)
+    h ^= h >> np.uint64(13)
+    span = np.minimum(np.uint64(ngran) - w * np.uint64(win), np.uint64(win))
+    return (w * np.uint64(win) + h % span).astype(np.int64)
+
+
 def test_single_pass_falls_back_when_the_sample_misleads(torch):
-    # d = 1e6: every 7th tile of 1024 entries is sampled (tiles 3, 10, 17, ...).  Large entries
-    # are placed only in tiles the sample never sees, so every bracket misses the true
-    # threshold and the row must take the full radix select; the result may not change.
+    # d = 1e6: one granule of 16 entries out of every 7 is sampled.  Large entries are placed
+    # only in granules the sample never sees, so every bracket misses the true threshold and
+    # the row must take the full radix select; the result may not change.
     d = 1_000_000
     X, G, Y = S.gaussian_rows(2, d, seed=31, drift=0.01, move=0.02)
-    tiles = np.arange(d) // 1024
-    hidden = (tiles % 7) != 3
+    hidden = np.ones(d, dtype=bool)
+    seen = sampled_granules(d)
+    assert len(seen) == 8929 and len(np.unique(seen)) == len(seen) and seen.max() < 62500
+    for k in range(16):
+        hidden[np.minimum(seen * 16 + k, d - 1)] = False
     rng = np.random.Generator(np.random.PCG64(32))
     X[0, hidden] += (5.0 * rng.standard_normal(int(hidden.sum()))).astype(F32)
     got, _ = check_against_oracle(torch, X, G, Y, [(TOPK, 1000), (TOPK, 10000), (TOPK, 100000)], 0.5)
     assert got["fallbacks"] == 1          # row 0 only; row 1 is homogeneous
+
+
+def test_block_scaled_rows_keep_the_single_pass(torch):
+    # contiguous blocks of very different scale (the structure of the c5 workload) at a size where
+    # each block is only a few dozen tiles long: the sample must still bracket every threshold
+    Xs, G0 = S.stress_vectors(2, 4_000_000, blocks=100, period=4, seed=36, device="cpu")
+    got, _ = check_against_oracle(torch, Xs[1].numpy(), G0.numpy(), Xs[0].numpy(),
+                                  [(TOPK, 4000), (TOPK, 40000), (TOPK, 400000)], 1.0)
+    assert got["fallbacks"] == 0
 
 
 def test_single_pass_list_overflow_falls_back(torch):
