@@ -35,6 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-fmad=false",  # every binary32 operation of the bit-exact path is a single rounding
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    cmd[1:1] = os.environ.get("ADACGD_NVCC_FLAGS", "").split()  # extra compiler flags, e.g. -D switches
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
