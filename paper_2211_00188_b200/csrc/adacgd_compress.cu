@@ -457,8 +457,17 @@ __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, cons
                          RowDec* __restrict__ dec, u32* __restrict__ flags, const CompressOut& out,
                          const u32* __restrict__ diffflag, double tol) {
   __shared__ double ps[NSLOT][TPB / 32];
+  __shared__ double p_extra[MAXC];
+  __shared__ u32 p_T[MAXC], p_ntie[MAXC], p_q[MAXC], p_max, p_diff;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int nslot = 2 + cs.m;
+  // what the deciding thread needs from the selection records is fetched by several threads at once
+  if (threadIdx.x < cs.nsel) {
+    const int j = threadIdx.x;
+    p_T[j] = __ldcg(&sel[row].T[j]); p_ntie[j] = __ldcg(&sel[row].ntie[j]);
+    p_q[j] = __ldcg(&sel[row].q[j]); p_extra[j] = __ldcg(&sel[row].extraE[j]);
+  }
+  if (threadIdx.x == 32) { p_max = __ldcg(&maxkey[row]); p_diff = __ldcg(&diffflag[row]); }
   double a[NSLOT];
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) a[s] = 0.0;
@@ -490,13 +499,14 @@ __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, cons
       if (cs.param[c] >= d) { e[c + 1] = 0.0; continue; }
       int j = 0;
       for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
-      const double tv = (double)__uint_as_float(sel[row].T[j]);
-      e[c + 1] = (sum[2 + c] + sel[row].extraE[j]) + (double)(sel[row].ntie[j] - sel[row].q[j]) * (tv * tv);
+      const double tv = (double)__uint_as_float(p_T[j]);
+      e[c + 1] = (sum[2 + c] + p_extra[j]) + (double)(p_ntie[j] - p_q[j]) * (tv * tv);
     } else {
       e[c + 1] = sum[2 + c];
     }
   }
-  if (maxkey[row] >= 0x7f800000u || (diffflag[row] & 0x80000000u)) {  // Inf/NaN in X - G or X - Y: estimator kept
+  const u32 diff = p_diff;
+  if (p_max >= 0x7f800000u || (diff & 0x80000000u)) {  // Inf/NaN in X - G or X - Y: estimator kept
     atomicOr(&flags[0], 1u);
     finalize_row(cs, row, 0, d, sel, maxkey, dec, out, e, D);
     return;
@@ -516,7 +526,7 @@ __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, cons
     int verdict;  // 1 true, 0 false, -1 unsure
     if (by_def) verdict = 1;
     else if (!(D <= 1.7e308)) verdict = -1;  // overflowed chain or non-finite X - Y: the exact pass tells which
-    else if (j == 0 && (diffflag[row] & 0x7fffffffu) == 0 && d_ok)
+    else if (j == 0 && (diff & 0x7fffffffu) == 0 && d_ok)
       verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
     else if (!e_ok) verdict = -1;
     else if (cs.zeta == 0.f) verdict = 0;  // E > 0 for certain, right side is 0
@@ -1269,44 +1279,57 @@ __device__ __forceinline__ u32 first_digit_shift(u32 lo, u32 hi) {
   return nbits > 8u ? nbits - 8u : 0u;
 }
 
-// Run by the last CTA of a row's streaming pass.  Checks every bracket exactly (the K-th largest key
-// must be one of the listed keys; otherwise the row is flagged for the full select) and locates the
-// first-digit bin of each threshold.  A bin with more than FINAL_CAP keys sends the row through the
-// three-level list passes.
-__device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, int nblk, const u32* __restrict__ fhist,
-                                              const u32* __restrict__ cntpart, SelRow* __restrict__ sel,
+// Run by the last CTA of a row's streaming pass, one warp per bracket.  Checks the bracket exactly
+// (the K-th largest key must be one of the listed keys; otherwise the row is flagged for the full
+// select) and locates the first-digit bin of its threshold.  A bin with more than FINAL_CAP keys
+// sends the row through the three-level list passes.
+__device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, const u32* __restrict__ fhist,
+                                              const u32* __restrict__ cnttot, SelRow* __restrict__ sel,
                                               u32* __restrict__ rowflag, u32* __restrict__ tickets,
                                               u32* __restrict__ flags) {
-  __shared__ u32 res[2];
-  __shared__ u32 bad;
+  static_assert(MAXC <= TPB / 32 && LB1 == 256, "one warp per bracket, eight bins per lane");
+  __shared__ u32 bad, toofull;
+  const int lane = threadIdx.x & 31, j = threadIdx.x >> 5;
   SelRow* s = sel + row;
-  if (threadIdx.x == 0) bad = 0;
+  if (threadIdx.x == 0) { bad = 0; toofull = 0; }
   __syncthreads();
-  for (int j = 0; j < cs.nsel; ++j) {
-    u32 a = 0;
-    for (int b = threadIdx.x; b < nblk; b += TPB)
-      a += __ldcg(&cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j]);
+  if (j < cs.nsel) {
+    const u32 above = __ldcg(&cnttot[row * MAXC + j]);            // keys >= hi
     const u32* h = fhist + ((long long)row * MAXC + j) * LB1;
-    const u32 mine = (threadIdx.x < LB1) ? __ldcg(&h[threadIdx.x]) : 0u;
-    u32 above, total;
-    block_excl_scan(a, &above);
-    block_excl_scan(mine, &total);
+    // bins in descending order: this lane holds positions 8*lane .. 8*lane + 7
+    const uint4 q0 = __ldcg(reinterpret_cast<const uint4*>(h + (LB1 - 8 - 8 * lane)));
+    const uint4 q1 = __ldcg(reinterpret_cast<const uint4*>(h + (LB1 - 4 - 8 * lane)));
+    const u32 v[8] = {q1.w, q1.z, q1.y, q1.x, q0.w, q0.z, q0.y, q0.x};
+    u32 lsum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) lsum += v[k];
+    u32 inc = lsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    const u32 total = __shfl_sync(0xffffffffu, inc, 31);
     const long long K = cs.param[cs.sel[j]];
     if (K <= (long long)above || K > (long long)above + (long long)total) {
-      if (threadIdx.x == 0) bad = 1;
+      if (lane == 0) bad = 1;
     } else {
-      block_find_kth_desc(h, LB1, (u32)K - above, res);
-      if (threadIdx.x == 0) {
-        const u32 c1 = __ldcg(&h[res[0]]);
-        s->above_hi[j] = above; s->fb1[j] = res[0]; s->fabove1[j] = above + res[1]; s->fc1[j] = c1;
-        if (c1 > (u32)FINAL_CAP) tickets[row * NTICKET + 13] = 1u;
+      const u32 krem = (u32)K - above;
+      u32 run = inc - lsum;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (krem > run && krem <= run + v[k]) {                  // true in exactly one lane, for one k
+          s->above_hi[j] = above; s->fb1[j] = (u32)(LB1 - 1 - (8 * lane + k)); s->fabove1[j] = above + run; s->fc1[j] = v[k];
+          if (v[k] > (u32)FINAL_CAP) toofull = 1;
+        }
+        run += v[k];
       }
     }
-    __syncthreads();
   }
+  __syncthreads();
   if (threadIdx.x == 0) {
     if (bad || __ldcg(&rowflag[row])) rowflag[row] = 1;   // bracket missed, or a segment overflowed
-    else if (tickets[row * NTICKET + 13]) atomicAdd(&flags[3], 1u);
+    else if (toofull) { tickets[row * NTICKET + 13] = 1u; atomicAdd(&flags[3], 1u); }
   }
 }
 
@@ -1507,7 +1530,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
     const int j = threadIdx.x - 32;
     u32 acc = 0;
     for (int w = 0; w < TPB / 32; ++w) acc += redc[j][w];
-    cntpart[pbase * MAXC + j] = acc;
+    if (acc) atomicAdd(&cntpart[row * MAXC + j], acc);
   }
   if (threadIdx.x == 0 && NSEL > 0) {
     const u32 n = sh_cnt;
@@ -1521,7 +1544,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
       if (c) atomicAdd(&gh[i], c);
     }
     if (last_cta_of_row(&tickets[row * NTICKET + 11], gridDim.x))
-      first_digit_scan(cs, row, (int)gridDim.x, fhist, cntpart, sel, rowflag, tickets, flags);
+      first_digit_scan(cs, row, fhist, cntpart, sel, rowflag, tickets, flags);
   }
 }
 
@@ -1602,8 +1625,7 @@ __device__ __noinline__ void lscan_row(const CsetDev& cs, int row, int nblk, int
     __syncthreads();
     for (int j = 0; j < cs.nsel; ++j) {
       u32 a = 0, tot = 0;
-      for (int b = threadIdx.x; b < nblk; b += TPB)
-        a += __ldcg(&cntpart[((long long)row * MAX_BLK_PER_ROW + b) * MAXC + j]);
+      if (threadIdx.x == 0) a = __ldcg(&cntpart[row * MAXC + j]);
       const u32* h = hist + ((long long)row * MAXC + j) * NB;
       for (int b = threadIdx.x; b < NB; b += TPB) tot += __ldcg(&h[b]);
       u32 above, total;
@@ -1749,85 +1771,107 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
 }
 
 // ---- the usual case: the threshold's first-digit bin holds at most FINAL_CAP keys ----------------
-// Completes every bracket of a row from the keys collected out of the threshold's bin: a radix
-// select over the remaining low bits of key - lo (8 bits per round, one bin per thread) gives the
-// threshold, the counts above and equal, and how many threshold-equal keys are kept; those are the
-// ones with the lowest indices, found by ranking the equal keys' indices.
+// Completes the brackets of a row from the keys collected out of each threshold's bin.  One warp
+// per bracket, all brackets at once: a radix select over the remaining low bits of key - lo (8 bits
+// per round, 256 bins scanned by the warp) gives the threshold, the counts above and equal, and how
+// many threshold-equal keys are kept; those are the ones with the lowest indices, found by ranking
+// the equal keys' indices.  `wbuf` is dynamic shared memory, FINISH_WORDS words per bracket.
+constexpr int TIE_CAP = 1024;                        // threshold-equal keys ranked here; more go to the chunk-prefix pass
+constexpr int FINISH_WORDS = FINAL_CAP + TIE_CAP;
 __device__ __noinline__ void collected_finish_row(const CsetDev& cs, int row, int nlb, SelRow* __restrict__ sel,
-                                                  const u64* __restrict__ fl, const double* __restrict__ lepart) {
-  __shared__ u32 ek[FINAL_CAP];
-  __shared__ u32 hist[TPB];
-  __shared__ u32 res[3];
-  __shared__ u32 ties[1024];
-  __shared__ u32 nties_sh;
-  __shared__ double wsum_d[TPB / 32];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+                                                  const u64* __restrict__ fl, const double* __restrict__ lepart,
+                                                  u32* __restrict__ wbuf) {
+  static_assert(MAXC <= TPB / 32, "one warp per bracket");
+  __shared__ u32 whist[TPB / 32][256];
+  const int lane = threadIdx.x & 31, j = threadIdx.x >> 5;
+  if (j >= cs.nsel) return;
   SelRow* s = sel + row;
-  for (int j = 0; j < cs.nsel; ++j) {
-    const u32 c1 = s->fc1[j];
-    const u32 K = (u32)cs.param[cs.sel[j]];
-    const u32 need = K - s->fabove1[j];               // 1 <= need <= c1 <= FINAL_CAP
-    const u32 shq = first_digit_shift(s->lo[j], s->hi[j]);
-    const u32 base = s->lo[j] + (s->fb1[j] << shq);   // every collected key lies in [base, base + 2^shq)
-    const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
-    for (u32 i = threadIdx.x; i < c1; i += TPB) ek[i] = (u32)(__ldcg(&f[i]) >> 32);
-    if (threadIdx.x == 0) { res[0] = 0; res[1] = 0; res[2] = c1; nties_sh = 0; }
-    __syncthreads();
-    u32 prefix = 0, pmask = 0, krem = need, neq = c1;
-    for (u32 bits = shq; bits > 0;) {
-      const u32 nb = bits < 8u ? bits : 8u, shift = bits - nb;
-      hist[threadIdx.x] = 0;
-      __syncthreads();
-      for (u32 i = threadIdx.x; i < c1; i += TPB) {
-        const u32 rel = ek[i] - base;
-        if ((rel & pmask) == prefix) atomicAdd(&hist[(rel >> shift) & ((1u << nb) - 1u)], 1u);
+  u32* ek = wbuf + (size_t)j * FINISH_WORDS;
+  u32* ties = ek + FINAL_CAP;
+  u32* hist = whist[j];
+  const u32 c1 = __ldcg(&s->fc1[j]);
+  const u32 K = (u32)cs.param[cs.sel[j]];
+  const u32 need = K - __ldcg(&s->fabove1[j]);        // 1 <= need <= c1 <= FINAL_CAP
+  const u32 lo = __ldcg(&s->lo[j]);
+  const u32 shq = first_digit_shift(lo, __ldcg(&s->hi[j]));
+  const u32 base = lo + (__ldcg(&s->fb1[j]) << shq);  // every collected key lies in [base, base + 2^shq)
+  const u64* f = fl + ((long long)row * MAXC + j) * FINAL_CAP;
+  for (u32 i = lane; i < c1; i += 32) ek[i] = (u32)(__ldcg(&f[i]) >> 32);
+  __syncwarp();
+  u32 prefix = 0, pmask = 0, krem = need, neq = c1;
+  for (u32 bits = shq; bits > 0;) {
+    const u32 nb = bits < 8u ? bits : 8u, shift = bits - nb;
+    for (int b = lane; b < 256; b += 32) hist[b] = 0;
+    __syncwarp();
+    for (u32 i = lane; i < c1; i += 32) {
+      const u32 rel = ek[i] - base;
+      if ((rel & pmask) == prefix) atomicAdd(&hist[(rel >> shift) & ((1u << nb) - 1u)], 1u);
+    }
+    __syncwarp();
+    // bins in descending order: this lane holds positions 8*lane .. 8*lane + 7
+    u32 v[8], lsum = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { v[k] = hist[255 - (8 * lane + k)]; lsum += v[k]; }
+    u32 inc = lsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    u32 run = inc - lsum, fbin = 0, fabove = 0, fcnt = 0;
+    bool found = false;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (!found && krem > run && krem <= run + v[k]) { found = true; fbin = 255u - (u32)(8 * lane + k); fabove = run; fcnt = v[k]; }
+      run += v[k];
+    }
+    const u32 who = __ballot_sync(0xffffffffu, found);
+    const int src = who ? (__ffs(who) - 1) : 0;       // exactly one lane finds it: 1 <= krem <= matching keys
+    fbin = __shfl_sync(0xffffffffu, fbin, src);
+    fabove = __shfl_sync(0xffffffffu, fabove, src);
+    fcnt = __shfl_sync(0xffffffffu, fcnt, src);
+    prefix |= fbin << shift;
+    pmask |= ((1u << nb) - 1u) << shift;
+    krem -= fabove;
+    neq = fcnt;
+    bits = shift;
+    __syncwarp();
+  }
+  const u32 T = base + prefix, q = krem;              // q of the neq keys equal to T are kept
+  // energy of the listed keys in [lo, T): collected keys below T, then the per-CTA sums over lower bins
+  double e = 0.0;
+  for (u32 i = lane; i < c1; i += 32)
+    if (ek[i] < T) { const double kv = (double)__uint_as_float(ek[i]); e += kv * kv; }
+  for (int b = lane; b < nlb; b += 32) e += __ldcg(&lepart[((long long)row * LIST_BLK + b) * MAXC + j]);
+  e = warp_sum_f64(e);
+  u32 mode = 0u, cut = 0xffffffffu;
+  if (q < neq) {
+    mode = 2u;
+    if (neq <= (u32)TIE_CAP) {
+      mode = 1u;
+      // indices of the threshold-equal keys, compacted in any order; the q-th smallest is the cut
+      u32 nt = 0;
+      for (u32 i0 = 0; i0 < c1; i0 += 32) {
+        const u32 i = i0 + lane;
+        const bool eq = i < c1 && ek[i] == T;
+        const u32 m = __ballot_sync(0xffffffffu, eq);
+        if (eq) ties[nt + (u32)__popc(m & ((1u << lane) - 1u))] = (u32)__ldcg(&f[i]);
+        nt += (u32)__popc(m);
       }
-      __syncthreads();
-      const u32 v = hist[TPB - 1 - threadIdx.x];      // bins in descending order
-      const u32 excl = block_excl_scan(v, nullptr);
-      if (krem > excl && krem <= excl + v) { res[0] = TPB - 1 - threadIdx.x; res[1] = excl; res[2] = v; }
-      __syncthreads();
-      prefix |= res[0] << shift;
-      pmask |= ((1u << nb) - 1u) << shift;
-      krem -= res[1];
-      neq = res[2];
-      bits = shift;
-      __syncthreads();
-    }
-    const u32 T = base + prefix, q = krem;            // q of the neq keys equal to T are kept
-    // energy of the listed keys in [lo, T): collected keys below T, then the per-CTA sums over lower bins
-    double e = 0.0;
-    for (u32 i = threadIdx.x; i < c1; i += TPB)
-      if (ek[i] < T) { const double kv = (double)__uint_as_float(ek[i]); e += kv * kv; }
-    for (int b = threadIdx.x; b < nlb; b += TPB) e += __ldcg(&lepart[((long long)row * LIST_BLK + b) * MAXC + j]);
-    e = warp_sum_f64(e);
-    if (lane == 0) wsum_d[wid] = e;
-    u32 mode = 0u;
-    if (q < neq) {
-      mode = 2u;
-      if (neq <= 1024u) {
-        mode = 1u;
-        for (u32 i = threadIdx.x; i < c1; i += TPB)
-          if (ek[i] == T) ties[atomicAdd(&nties_sh, 1u)] = (u32)__ldcg(&f[i]);
-      }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      double tot = 0.0;
-      for (int w = 0; w < TPB / 32; ++w) tot += wsum_d[w];
-      s->T[j] = T; s->above[j] = K - q; s->ntie[j] = neq; s->q[j] = q; s->extraE[j] = tot;
-      s->tiemode[j] = mode;
-      if (mode != 1u) s->cut[j] = 0xffffffffu;   // mode 1: written below by the thread holding the q-th index
-    }
-    if (mode == 1u) {
-      for (u32 i = threadIdx.x; i < neq; i += TPB) {
+      __syncwarp();
+      for (u32 i = lane; i < neq; i += 32) {
         const u32 mine = ties[i];
         u32 rank = 0;
         for (u32 k = 0; k < neq; ++k) rank += (ties[k] < mine) ? 1u : 0u;
-        if (rank == q - 1u) s->cut[j] = mine;
+        if (rank == q - 1u) cut = mine;
       }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) cut = min(cut, __shfl_xor_sync(0xffffffffu, cut, o));
     }
-    __syncthreads();
+  }
+  if (lane == 0) {
+    s->T[j] = T; s->above[j] = K - q; s->ntie[j] = neq; s->q[j] = q; s->extraE[j] = e;
+    s->tiemode[j] = mode; s->cut[j] = cut;
   }
 }
 
@@ -1844,22 +1888,26 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
                                                   RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
                                                   const u32* __restrict__ diffflag, double tol) {
   pdl_begin();
+  extern __shared__ __align__(16) u32 wbuf[];          // cs.nsel * FINISH_WORDS words, used by the row's last CTA
   const int row = blockIdx.y;
   const int nsel = cs.nsel;
-  if (rowflag[row] || tickets[row * NTICKET + 13]) return;
+  // everything the pass needs is requested before the first value is looked at
+  const u32 skip_a = __ldcg(&rowflag[row]), skip_b = __ldcg(&tickets[row * NTICKET + 13]);
+  int sg = blockIdx.x;
+  u32 n_next = (sg < nseg) ? __ldcg(&lcount[(long long)row * MAX_BLK_PER_ROW + sg]) : 0u;
   u32 lo[MAXC], hi[MAXC], shq[MAXC], b1[MAXC];
   double en[MAXC];
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) {
-    lo[j] = (j < nsel) ? sel[row].lo[j] : 1u;
-    hi[j] = (j < nsel) ? sel[row].hi[j] : 0u;
-    shq[j] = first_digit_shift(lo[j], hi[j]);
-    b1[j] = (j < nsel) ? sel[row].fb1[j] : 0u;
+    lo[j] = (j < nsel) ? __ldcg(&sel[row].lo[j]) : 1u;
+    hi[j] = (j < nsel) ? __ldcg(&sel[row].hi[j]) : 0u;
+    b1[j] = (j < nsel) ? __ldcg(&sel[row].fb1[j]) : 0u;
     en[j] = 0.0;
   }
+  if (skip_a || skip_b) return;
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) shq[j] = first_digit_shift(lo[j], hi[j]);
   // the segment lengths are fetched one segment ahead, the entries four per thread at a time
-  int sg = blockIdx.x;
-  u32 n_next = (sg < nseg) ? __ldcg(&lcount[(long long)row * MAX_BLK_PER_ROW + sg]) : 0u;
   for (; sg < nseg; sg += gridDim.x) {
     const u32 n = n_next;
     const int sgn = sg + (int)gridDim.x;
@@ -1902,7 +1950,8 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
     lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
   }
   if (!last_cta_of_row(&tickets[row * NTICKET + 12], gridDim.x)) return;
-  collected_finish_row(cs, row, (int)gridDim.x, sel, fl, lepart);
+  collected_finish_row(cs, row, (int)gridDim.x, sel, fl, lepart, wbuf);
+  __syncthreads();   // the brackets' results, written by one warp each, are read by the level choice
   if (pick_here) {
     pick_row(cs, d, row, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
     if (threadIdx.x == 0) tickets[row * NTICKET + 9] = 1u;
@@ -1939,9 +1988,10 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
-  L.shist = L.lhist1 = L.fhist = L.flcnt = o;
+  L.shist = L.lhist1 = L.fhist = L.flcnt = L.cntpart = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
+    L.cntpart = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
     L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
     L.fhist = o; o = align_up(o + (size_t)rows * MAXC * LB1 * 4, 256);
@@ -1954,13 +2004,12 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.energy = o; o = align_up(o + (size_t)rows * NSLOT * 8, 256);
   L.tiecnt = o; o = align_up(o + (size_t)rows * (size_t)nchunk_of(d) * 4, 256);
   L.list_row = 0;
-  L.list = L.lcount = L.cntpart = L.lepart = L.lepart3 = L.fl = o;
+  L.list = L.lcount = L.lepart = L.lepart3 = L.fl = o;
   if (single_pass) {
     L.list_row = list_row_of(d);
     L.fl = o; o = align_up(o + (size_t)rows * MAXC * FINAL_CAP * 8, 256);
     L.list = o; o = align_up(o + (size_t)rows * (size_t)L.list_row * 8, 256);
     L.lcount = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * 4, 256);
-    L.cntpart = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * MAXC * 4, 256);
     L.lepart = o; o = align_up(o + (size_t)rows * LIST_BLK * MAXC * 8, 256);
     L.lepart3 = o; o = align_up(o + (size_t)rows * LIST_BLK * MAXC * 8, 256);
   }
@@ -2073,6 +2122,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
     cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
     cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+    cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
     cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     attr_done = true;
@@ -2188,7 +2238,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (lgx > LIST_BLK) lgx = LIST_BLK;
     if (lgx > nblk) lgx = nblk;
     const dim3 lgrid((unsigned)lgx, rows);
-    TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), 0, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
+    TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), (size_t)cs.nsel * FINISH_WORDS * 4, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
                                  s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
                                  cs.nquant == 0 ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
                                  s.diffflag, tol));

@@ -112,7 +112,7 @@ struct Scratch {
   u32* fhist;      // [rows][MAXC][LB1] first digit as histogrammed by the streaming pass
   u64* list;       // [rows][list_row] (key << 32 | index), one segment of segcap entries per CTA
   u32* lcount;     // [rows][MAX_BLK_PER_ROW] entries per segment
-  u32* cntpart;    // [rows][MAX_BLK_PER_ROW][MAXC] per-CTA counts of keys >= hi
+  u32* cntpart;    // [rows][MAXC] keys >= hi of each bracket, added up by the CTAs of the streaming pass
   double* lepart;  // [rows][LIST_BLK][MAXC] per-CTA energies of listed keys below the chosen first digit
   double* lepart3; // same, below the chosen second digit
   u64* fl;         // [rows][MAXC][FINAL_CAP] listed keys sharing the threshold's 22-bit prefix
