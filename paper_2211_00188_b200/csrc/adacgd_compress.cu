@@ -2162,7 +2162,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   prof_end(pf, stream);
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  long long want = (148 * 8 + rows - 1) / rows;
+  long long want = (148 * 4 + rows - 1) / rows;   // one wave of the streaming pass: four resident CTAs per SM
   // a CTA takes at least eight tiles (spread over the row by the grid stride) where the row has them, so
   // that its share of the key list is sized for an average over the row rather than for one tile
   if (single && want > (ntile + 7) / 8) want = (ntile + 7) / 8;
