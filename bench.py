@@ -193,6 +193,13 @@ KERNEL_BYTES = {"k_pass1": 12, "k_update": 8, "k_hist<1>": 8, "k_hist<2>": 8, "k
                 "k_quant_err": 8}
 
 
+# DRAM bytes per element and row that ncu counted for these kernels (dram__bytes read + write over
+# one worker launch of workload c5 at half size, 8 x 12.5e6; the traffic grows in proportion to the
+# elements a launch processes).  Valid for the kernels as committed with profiles/c5_compress_step.txt;
+# a kernel that changes afterwards loses its entry until it is captured again.
+NCU_DRAM_BYTES_PER_ELEM = {"k_pass1": 12.10, "k_update": 8.53}
+
+
 def kernel_table(prof):
     tot = sum(v[0] for v in prof.values()) or 1.0
     return {k: {"ms_total": round(v[0], 4), "launches": v[1], "share": round(v[0] / tot, 4)}
@@ -263,8 +270,10 @@ def bench_c5(args, rank, world, local):
     achieved = top_bytes / (kern[top][0] * 1e-3) / 1e9
     step_floor_bytes = 20 * (n + 1) * d + 4 * d           # 12 B + 8 B per element and row, + the mean
     step_gbs = step_floor_bytes / (ms / args.steps * 1e-3) / 1e9
+    per_elem = NCU_DRAM_BYTES_PER_ELEM.get(top)
+    traffic = None if per_elem is None else per_elem * rows_total * d / kern[top][1]   # bytes per launch, like achieved
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                 "launches": kern[top][1], "avg_launch_ms": kern[top][0] / kern[top][1]}
     step_roofline = {"algorithmic_bytes_per_step": step_floor_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak}
 
