@@ -8,3 +8,4 @@ from .binding import (  # noqa: F401
     AdaCGD, Cand, TOPK, QUANT, LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE,
     AdacgdError, load_library, EXPORTED_SYMBOLS, compress_noalloc, NOALLOC_MAX_ROWS, NOALLOC_MAX_D,
 )
+from . import protocol  # noqa: F401,E402

@@ -185,7 +185,24 @@ __global__ void __launch_bounds__(TPB) k_csr_fwd(const long long* __restrict__ r
   if (live) {
     const long long g = (long long)worker * m_rows + row;
     const long long e0 = rowptr[g], e1 = rowptr[g + 1];
-    for (long long e = e0 + lane; e < e1; e += 32) acc = fmaf(val[e], x[col[e]], acc);
+    // eight entries per lane in flight: their values and column indices first, then the eight gathers;
+    // a lane still adds its products in ascending entry order
+    for (long long e = e0 + lane; e < e1; e += 32 * 8) {
+      int c[8];
+      float v[8], xv[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const long long ee = e + 32 * k;
+        const bool ok = ee < e1;
+        c[k] = ok ? __ldcs(&col[ee]) : 0;
+        v[k] = ok ? __ldcs(&val[ee]) : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) xv[k] = __ldg(&x[c[k]]);
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (e + 32 * k < e1) acc = fmaf(v[k], xv[k], acc);
+    }
   }
   const float z = warp_sum_f32(acc);
   __shared__ double ls[TPB / 32];
