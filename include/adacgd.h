@@ -212,8 +212,8 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
 #define ADACGD_STATE_BITS_UP 6  /* cumulative     uint64 */
 #define ADACGD_STATE_BITS_DOWN 7/* cumulative     uint64 */
 #define ADACGD_STATE_LEVELS 8   /* last step      int32 [n] */
-#define ADACGD_STATE_FLAGS 9    /* uint32: bit 0 = a non-finite input was seen since init; bit 1 = a bounded
-                                   device-side wait for an asynchronous copy gave up (get only) */
+#define ADACGD_STATE_FLAGS 9    /* uint32: bit 0 = a non-finite input was seen since init; bit 1 is reserved for a
+                                   device-side wait that gave up (no kernel of this version waits) (get only) */
 #define ADACGD_STATE_RECHECKS 10/* uint32: trigger comparisons redone in exact arithmetic since init (get only) */
 #define ADACGD_STATE_FALLBACKS 11/* uint32: rows whose sampled threshold bracket failed and that took the full
                                    three-pass radix select instead, since init (get only) */

@@ -24,37 +24,6 @@ __device__ __forceinline__ void pdl_begin() {
 
 __device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
-// ---- bulk asynchronous copies (TMA, 1-D) into shared memory, completion on an mbarrier ----
-__device__ __forceinline__ u32 smem_addr(const void* p) { return (u32)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
-  u32 ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_addr(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Waits for a phase of the barrier, giving up after a bounded number of polls.
-__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity) {
-  for (int spin = 0; spin < (1 << 22); ++spin)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-// dst (shared) and src (global) 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
-               "l"(src), "r"(bytes), "r"(smem_addr(bar))
-               : "memory");
-}
-
 template <bool ALIGNED>
 __device__ __forceinline__ void load4(const float* __restrict__ row, long long c0, long long d, float (&o)[4]) {
   if (ALIGNED) {
@@ -754,26 +723,74 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
 // summed in worker order.  Row i: G_i <- G_i + C_level(X_i - G_i) (EF21, Eq. 7).  The next
 // row's operands are loaded before the current row is written back.
 constexpr int UPD_ROW_TILE = 32;
-constexpr int UP_STAGES = 4;
 #ifndef UPD_RB
 #define UPD_RB 2    // rows whose operands a thread of the update kernel keeps in flight
 #endif
+// g <- g + C(x - g) on four columns for a Top-K level given by threshold key T and index cut:
+// kept <=> |v| >= T for indices up to the cut, |v| > T (>= the next key value) beyond it; finite
+// non-negative binary32 values order like their bit patterns.  Returns whether anything was kept.
+__device__ __forceinline__ bool apply_topk4(float (&g)[4], const float (&x)[4], u32 T, u32 cut, u32 c0u) {
+  const float Tf = __uint_as_float(T), Tn = __uint_as_float(T + 1u);
+  float th[4];
+  if (cut >= c0u + 3u) { th[0] = th[1] = th[2] = th[3] = Tf; }
+  else if (cut < c0u) { th[0] = th[1] = th[2] = th[3] = Tn; }
+  else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) th[k] = (c0u + (u32)k <= cut) ? Tf : Tn;
+  }
+  bool any = false;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float v = __fsub_rn(x[k], g[k]);
+    const bool kept = fabsf(v) >= th[k];
+    g[k] = kept ? __fadd_rn(g[k], v) : g[k];
+    any = any || kept;
+  }
+  return any;
+}
+// Rows r0 .. r0 + nr - 1 of one chunk for a thread's four columns, every row either skipped or a Top-K
+// level with an index cut (modes 0 and 1 of `rd`): UPD_RB rows in flight as plain 128-bit loads, applied
+// in row order so that `acc` sums the mean in worker order.
+__device__ __forceinline__ void update_rows_simple(const float* __restrict__ X, float* __restrict__ G, long long d,
+                                                   long long c0, int r0, int nr, const RowDec* rd, bool want_mean,
+                                                   float (&acc)[4]) {
+  const u32 c0u = (u32)c0;
+  for (int q0 = 0; q0 < nr; q0 += UPD_RB) {
+    float4 gq[UPD_RB], xq[UPD_RB];
+#pragma unroll
+    for (int u = 0; u < UPD_RB; ++u) {
+      gq[u] = make_float4(0.f, 0.f, 0.f, 0.f); xq[u] = gq[u];
+      const int ii = q0 + u;
+      if (ii < nr) {
+        const int m = rd[ii].mode;
+        if (m != 0 || want_mean) gq[u] = *reinterpret_cast<const float4*>(G + (long long)(r0 + ii) * d + c0);
+        if (m != 0) xq[u] = __ldcs(reinterpret_cast<const float4*>(X + (long long)(r0 + ii) * d + c0));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UPD_RB; ++u) {
+      const int ii = q0 + u;
+      if (ii >= nr) break;
+      float g[4] = {gq[u].x, gq[u].y, gq[u].z, gq[u].w};
+      if (rd[ii].mode != 0) {
+        const float x[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
+        if (apply_topk4(g, x, rd[ii].T, rd[ii].cut, c0u))
+          *reinterpret_cast<float4*>(G + (long long)(r0 + ii) * d + c0) = make_float4(g[0], g[1], g[2], g[3]);
+      }
+      if (want_mean) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
+      }
+    }
+  }
+}
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
-                                                CompressOut out, u32* __restrict__ out_flags) {
+                                                CompressOut out) {
   pdl_begin();
   __shared__ RowDec shd[UPD_ROW_TILE];
-  __shared__ __align__(128) float ustage[UP_STAGES][2][UPD_COLS];
-  __shared__ __align__(8) u64 ubar[UP_STAGES];
-  __shared__ u32 u_abort;
-  u32 used = 0;  // rows staged so far: selects the stage and the barrier phase
-  if (ALIGNED && threadIdx.x == 0) {
-    for (int q = 0; q < UP_STAGES; ++q) mbar_init(&ubar[q], 1);
-    mbar_fence_init();
-    u_abort = 0;
-  }
   const int lane = threadIdx.x & 31;
   const bool want_mean = out.mean_out != nullptr;
 
@@ -790,54 +807,8 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
       for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
         const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
         if (c0 >= d) continue;
-        const u32 c0u = (u32)c0;
         float acc[4] = {-0.f, -0.f, -0.f, -0.f};  // -0 + g == g bit for bit, so the first row needs no special case
-        for (int r0 = 0; r0 < rows; r0 += UPD_RB) {
-          float4 gq[UPD_RB], xq[UPD_RB];
-#pragma unroll
-          for (int u = 0; u < UPD_RB; ++u) {
-            gq[u] = make_float4(0.f, 0.f, 0.f, 0.f); xq[u] = gq[u];
-            const int i = r0 + u;
-            if (i < rows) {
-              const int m = shd[i].mode;
-              if (m != 0 || want_mean) gq[u] = *reinterpret_cast<const float4*>(G + (long long)i * d + c0);
-              if (m != 0) xq[u] = __ldcs(reinterpret_cast<const float4*>(X + (long long)i * d + c0));
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < UPD_RB; ++u) {
-            const int i = r0 + u;
-            if (i >= rows) break;
-            float g[4] = {gq[u].x, gq[u].y, gq[u].z, gq[u].w};
-            if (shd[i].mode != 0) {
-              const float x[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
-              // kept <=> |v| >= T for indices up to the cut, |v| > T (>= the next key value) beyond it;
-              // finite non-negative binary32 values order like their bit patterns
-              const u32 T = shd[i].T, cut = shd[i].cut;
-              const float Tf = __uint_as_float(T), Tn = __uint_as_float(T + 1u);
-              float th[4];
-              if (cut >= c0u + 3u) { th[0] = th[1] = th[2] = th[3] = Tf; }
-              else if (cut < c0u) { th[0] = th[1] = th[2] = th[3] = Tn; }
-              else {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) th[k] = (c0u + (u32)k <= cut) ? Tf : Tn;
-              }
-              bool any = false;
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float v = __fsub_rn(x[k], g[k]);
-                const bool kept = fabsf(v) >= th[k];
-                g[k] = kept ? __fadd_rn(g[k], v) : g[k];
-                any = any || kept;
-              }
-              if (any) *reinterpret_cast<float4*>(G + (long long)i * d + c0) = make_float4(g[0], g[1], g[2], g[3]);
-            }
-            if (want_mean) {
-#pragma unroll
-              for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
-            }
-          }
-        }
+        update_rows_simple(X, G, d, c0, 0, rows, shd, want_mean, acc);
         if (want_mean) {
           const float n = (float)rows;
           *reinterpret_cast<float4*>(out.mean_out + c0) =
@@ -868,62 +839,7 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
       if (threadIdx.x < nr) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
       simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
       if (simple && ALIGNED) {
-        // rows are staged through shared memory by bulk asynchronous copies, UP_STAGES rows ahead
-        const long long cb = (long long)chunk * UPD_COLS;
-        const u32 bytes = (u32)(((d - cb < UPD_COLS) ? (d - cb) : UPD_COLS) * 4);
-        auto issue_row = [&](int ii, u32 slot) {
-          const int m = shd[ii].mode;
-          const bool ng = (m != 0) || want_mean, nx = (m != 0);
-          const int sidx = (int)(slot % UP_STAGES);
-          mbar_expect_tx(&ubar[sidx], bytes * ((ng ? 1u : 0u) + (nx ? 1u : 0u)));
-          if (ng) bulk_load(&ustage[sidx][0][0], G + (long long)(r0 + ii) * d + cb, bytes, &ubar[sidx]);
-          if (nx) bulk_load(&ustage[sidx][1][0], X + (long long)(r0 + ii) * d + cb, bytes, &ubar[sidx]);
-        };
-        if (threadIdx.x == 0)
-          for (int q = 0; q < nr && q < UP_STAGES; ++q) issue_row(q, used + q);
-        for (int ii = 0; ii < nr; ++ii) {
-          const int i = r0 + ii;
-          const u32 slot = used + ii;
-          const int sidx = (int)(slot % UP_STAGES);
-          const int m = shd[ii].mode;
-          float g[4] = {0.f, 0.f, 0.f, 0.f}, x[4] = {0.f, 0.f, 0.f, 0.f};
-          if (!mbar_wait_bounded(&ubar[sidx], (slot / UP_STAGES) & 1u)) u_abort = 1;
-          else if (live) {
-            if (m != 0 || want_mean) {
-              const float4 a = *reinterpret_cast<const float4*>(&ustage[sidx][0][threadIdx.x * 4]);
-              g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
-            }
-            if (m != 0) {
-              const float4 b = *reinterpret_cast<const float4*>(&ustage[sidx][1][threadIdx.x * 4]);
-              x[0] = b.x; x[1] = b.y; x[2] = b.z; x[3] = b.w;
-            }
-          }
-          if (m != 0) {
-            const u32 T = shd[ii].T, cut = shd[ii].cut;
-            bool any = false;
-  #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const float v = __fsub_rn(x[k], g[k]);
-              const u32 key = key_of(v);
-              const bool kept = (key > T) || (key == T && (u32)c0 + (u32)k <= cut);
-              g[k] = kept ? __fadd_rn(g[k], v) : g[k];
-              any = any || kept;
-            }
-            if (any && live) store4<ALIGNED>(G + (long long)i * d, c0, d, g);
-          }
-          if (want_mean) {
-  #pragma unroll
-            for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[k]);
-          }
-          __syncthreads();                     // the stage has been read by every thread
-          if (u_abort) break;
-          if (threadIdx.x == 0 && ii + UP_STAGES < nr) issue_row(ii + UP_STAGES, slot + UP_STAGES);
-        }
-        if (u_abort) {
-          if (threadIdx.x == 0) atomicOr(&out_flags[0], 2u);
-          return;
-        }
-        used += (u32)nr;
+        if (live) update_rows_simple(X, G, d, c0, r0, nr, shd, want_mean, acc);
         continue;
       }
       if (simple) {
@@ -2149,7 +2065,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
     prof_end(pf, stream);
     TIMED(KID_PICK, launch_k(k_copy_report, dim3((rows + 127) / 128), dim3(128), 0, stream, false, rows, d, 0, out));
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out, s.flags);
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   // clear the per-call accumulators
@@ -2268,7 +2184,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // still hold part of the SMs end up unevenly spread, and the fullest SM then sets the pace (measured:
     // 400 us instead of 270 us on 8 x 25e6).
     const bool pdl = false;
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, s.flags);
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
   }
 #undef LIST_PASS
 #undef PASS1_CASE
