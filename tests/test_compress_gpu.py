@@ -18,7 +18,7 @@ def torch():
     return t
 
 
-def gpu_compress(torch, X, G, Y, cands, zeta, want_mean=True, engine=None):
+def gpu_compress(torch, X, G, Y, cands, zeta, want_mean=True, engine=None, want_kept=True):
     import paper_2211_00188_b200 as pkg
     rows, d = X.shape
     dev = torch.device("cuda:0")
@@ -30,16 +30,20 @@ def gpu_compress(torch, X, G, Y, cands, zeta, want_mean=True, engine=None):
     err = torch.zeros(rows, m + 1, dtype=torch.float64, device=dev)
     D = torch.zeros(rows, dtype=torch.float64, device=dev)
     stride = d
-    kept_idx = torch.full((rows, stride), -1, dtype=torch.int32, device=dev)
-    kept_cnt = torch.zeros(rows, dtype=torch.int64, device=dev)
+    # without the kept-index outputs the update kernel takes its streaming path
+    kept_idx = torch.full((rows, stride), -1, dtype=torch.int32, device=dev) if want_kept else None
+    kept_cnt = torch.zeros(rows, dtype=torch.int64, device=dev) if want_kept else None
     mean = torch.zeros(d, dtype=torch.float32, device=dev) if want_mean else None
     eng.compress(Xd, Gd, Yd, cands, zeta, mean_out=mean, level=level, bits=bits, err=err, D=D,
                  kept_idx=kept_idx, kept_cnt=kept_cnt)
     torch.cuda.synchronize()
-    cnt = kept_cnt.cpu().numpy()
-    idx = kept_idx.cpu().numpy()
+    kept = None
+    if want_kept:
+        cnt = kept_cnt.cpu().numpy()
+        idx = kept_idx.cpu().numpy()
+        kept = [np.sort(idx[i, :cnt[i]]) for i in range(rows)]
     return dict(G=Gd.cpu().numpy(), level=level.cpu().numpy(), bits=bits.cpu().numpy(), err=err.cpu().numpy(),
-                D=D.cpu().numpy(), kept=[np.sort(idx[i, :cnt[i]]) for i in range(rows)],
+                D=D.cpu().numpy(), kept=kept, list_levels=eng.get_state("list_levels"),
                 mean=mean.cpu().numpy() if want_mean else None, rechecks=eng.get_state("rechecks"), fallbacks=eng.get_state("fallbacks"),
                 flags=eng.get_state("flags"), engine=eng)
 
@@ -50,9 +54,14 @@ def assert_bitwise(a, b, what):
     assert bad[0].size == 0, f"{what}: {bad[0].size} mismatches, first at {tuple(x[0] for x in bad)}"
 
 
-def check_against_oracle(torch, X, G, Y, cands, zeta):
+def check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=False):
     got = gpu_compress(torch, X, G, Y, cands, zeta)
     G_ref, res = O.compress_rows(X, G, Y, cands, zeta)
+    if both_update_paths:
+        again = gpu_compress(torch, X, G, Y, cands, zeta, want_kept=False)
+        assert_bitwise(again["G"], G_ref, "G (streaming update)")
+        assert_bitwise(again["mean"], O.server_mean(G_ref), "mean (streaming update)")
+        assert again["level"].tolist() == [r["level"] for r in res] and again["bits"].tolist() == [r["bits"] for r in res]
     rows, d = X.shape
     for i, r in enumerate(res):
         assert got["level"][i] == r["level"], (i, got["level"][i], r["level"], r["err"], r["D"])
@@ -318,3 +327,44 @@ def test_nonfinite_rows_on_the_single_pass_path(torch):
     G_ref, res = O.compress_rows(X[[1]], G[[1]], Y[[1]], [(TOPK, 300), (TOPK, 30000)], 1.0)
     assert_bitwise(got["G"][[1]], G_ref, "clean row")
     assert got["level"][1] == res[0]["level"]
+
+
+@pytest.mark.parametrize("d", [700_000, 700_001])
+def test_single_pass_eight_candidates(torch, d):
+    # the most brackets a set can have, on rows with and without 16-byte alignment; both update paths
+    X, G, Y = S.gaussian_rows(2, d, seed=50)
+    cands = [(TOPK, k) for k in (70, 700, 2000, 7000, 20000, 70000, 200000, 350000)]
+    got, _ = check_against_oracle(torch, X, G, Y, cands, 1.0, both_update_paths=True)
+    assert got["fallbacks"] == 0
+
+
+def test_single_pass_many_short_rows(torch):
+    # more rows than one tile of decisions holds, each only twenty tiles long (every element is sampled)
+    X, G, Y = S.gaussian_rows(40, 20_000, seed=51)
+    got, res = check_against_oracle(torch, X, G, Y, [(TOPK, 20), (TOPK, 200), (TOPK, 2000)], 0.5, both_update_paths=True)
+    assert got["fallbacks"] == 0 and len({r["level"] for r in res}) >= 1
+
+
+def test_single_pass_with_quantisers(torch):
+    # quantisers need the row maximum first, so the level is picked by its own kernel after the list pass
+    X, G, Y = S.gaussian_rows(2, 600_000, seed=52)
+    cands = [(TOPK, 600), (QUANT, 2), (TOPK, 60000), (QUANT, 8)]
+    for zeta in (0.05, 1.0):
+        check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+
+
+def test_single_pass_crowded_threshold_bin(torch):
+    # 30 000 magnitudes within a few units in the last place around the 1 % threshold: the first-digit bin of
+    # that bracket holds far more keys than the collection buffer, so the row takes the three-level list passes
+    d = 1_000_000
+    X, G, Y = S.gaussian_rows(2, d, seed=53, drift=0.3, move=0.3)
+    v = (X[0] - G[0]).astype(F32)
+    t = np.sort(np.abs(v))[-10_000]                     # the 1 % threshold of row 0
+    rng = np.random.Generator(np.random.PCG64(54))
+    where = rng.choice(d, 30_000, replace=False)
+    near = (F32(t) * (1.0 + 1e-7 * rng.integers(-3, 4, 30_000))).astype(F32) * rng.choice([-1.0, 1.0], 30_000).astype(F32)
+    G[0, where] = 0.0
+    X[0, where] = near                                   # v = X - 0 exactly
+    got, _ = check_against_oracle(torch, X, G, Y, [(TOPK, 1000), (TOPK, 10_000), (TOPK, 100_000)], 1.0,
+                                  both_update_paths=True)
+    assert got["fallbacks"] == 0 and got["list_levels"] >= 1
