@@ -89,13 +89,15 @@ __device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
 
 // Finds, in a histogram of nb bins ordered by key, the bin that holds the krem-th
 // largest key: out[0] = bin, out[1] = number of keys in higher bins.  All TPB threads call.
+template <bool SHARED_TABLE = false>
 __device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 krem, u32* out) {
   const int per = nb / TPB;  // 8 or 2
   u32 loc[8];
   u32 sum = 0;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    loc[k] = (k < per) ? __ldcg(&hist[nb - 1 - (threadIdx.x * per + k)]) : 0;
+    const u32* src = &hist[nb - 1 - (threadIdx.x * per + k)];
+    loc[k] = (k < per) ? (SHARED_TABLE ? *src : __ldcg(src)) : 0;
     sum += loc[k];
   }
   u32 excl = block_excl_scan(sum, nullptr);
@@ -570,7 +572,9 @@ __device__ double digits_to_double(const u32* dig) {
 }
 
 // Run by one thread of the last CTA of the exact pass: carries, rounds and decides the row.
-__device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* __restrict__ limbs,
+// `row_limbs`: the row's NSLOT x NLIMB accumulators, in global memory or (SHARED_LIMBS) in shared memory.
+template <bool SHARED_LIMBS = false>
+__device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* row_limbs,
                                const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
                                RowDec* __restrict__ dec, const CompressOut& out,
                                const u32* __restrict__ diffflag, u32* __restrict__ flags) {
@@ -583,7 +587,7 @@ __device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u6
   }
   for (int s = 0; s < 2 + cs.m; ++s) {
     u32 dig[NLIMB];
-    const u64* l = limbs + ((long long)row * NSLOT + s) * NLIMB;
+    const u64* l = row_limbs + s * NLIMB;
     unsigned __int128 tie = 0;
     int tk = 0;
     if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
@@ -600,7 +604,7 @@ __device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u6
     for (int k = 0; k < NLIMB; ++k) {
       u64 add = 0;
       if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
-      const unsigned __int128 tsum = (unsigned __int128)__ldcg(&l[k]) + carry + add;
+      const unsigned __int128 tsum = (unsigned __int128)(SHARED_LIMBS ? l[k] : __ldcg(&l[k])) + carry + add;
       dig[k] = (u32)tsum;
       carry = (u64)(tsum >> 32);
     }
@@ -675,7 +679,7 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
     if (vhi && (i % NLIMB) + 1 < NLIMB) atomicAdd(&gl[i + 1], vhi);
   }
   if (last_cta_of_row(&tickets[row * NTICKET + 7], gridDim.x) && threadIdx.x == 0)
-    pick_exact_row(cs, row, d_full, limbs, sel, maxkey, dec, out, diffflag, flags);
+    pick_exact_row(cs, row, d_full, limbs + (long long)row * NSLOT * NLIMB, sel, maxkey, dec, out, diffflag, flags);
 }
 
 // --------------------------------------------------------------------------
@@ -1875,6 +1879,366 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
 }
 
 // --------------------------------------------------------------------------
+// short rows: stages a2-a4 and the mean in one launch
+// --------------------------------------------------------------------------
+// One CTA per row, the row's difference vector v = X - G kept in shared memory: three radix passes
+// (11 + 11 + 9 bits, all Top-K candidates at once), tail energies and quantiser errors in binary64,
+// the index cut of threshold-equal keys, the level choice (pick_row, with the exact integer sums
+// when a comparison cannot be certified), the update of the row, and - by the CTA that finishes
+// last - the mean over the rows.  Serves problems too small to keep the multi-kernel path busy.
+constexpr int SMALL_DMAX = 32768;
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
+                                                    int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
+                                                    double* partial, u32* maxkey, u32* diffflag, u64* limbs,
+                                                    u32* flags, u32* tickets, CompressOut out, double tol) {
+  pdl_begin();
+  extern __shared__ __align__(16) unsigned char small_smem[];
+  const int dn = (int)d;
+  float* vs = reinterpret_cast<float*>(small_smem);                       // [d rounded up to 4]
+  u32* tab = reinterpret_cast<u32*>(small_smem) + ((dn + 3) / 4) * 4;     // max(BINS1, nsel * BINS2) words
+  __shared__ double redd[NSLOT][TPB / 32];
+  __shared__ u32 redu[3][TPB / 32];
+  __shared__ u32 res[2];
+  __shared__ u32 s_b1[MAXC], s_ab1[MAXC], s_p2[MAXC], s_ab2[MAXC], s_T[MAXC], s_above[MAXC], s_ntie[MAXC], s_q[MAXC], s_cut[MAXC];
+  __shared__ u64 lsh[NSLOT * NLIMB];
+  const int row = blockIdx.x;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int nsel = cs.nsel;
+  const float* xr = X + (long long)row * d;
+  float* gr = G + (long long)row * d;
+  const float* yr = Y + (long long)row * d;
+
+  // ---- v into shared memory; D, ||v||^2, row maximum, |X-G| against |X-Y|
+  double aD = 0.0, aE = 0.0;
+  u32 mx = 0, mxw = 0, dfl = 0;
+  constexpr int SB = 4;   // tiles of TPB * 4 columns requested at once: the row is short, its latency is what counts
+  for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
+    float x[SB][4], g[SB][4], y[SB][4];
+#pragma unroll
+    for (int u = 0; u < SB; ++u) {
+      const int c0 = base + u * TPB * 4;
+      if (c0 < dn) {
+        load4<ALIGNED>(xr, c0, d, x[u]);
+        load4<ALIGNED>(gr, c0, d, g[u]);
+        load4<ALIGNED>(yr, c0, d, y[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < SB; ++u) {
+      const int c0 = base + u * TPB * 4;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (c0 + k >= dn) break;
+        const float v = __fsub_rn(x[u][k], g[u][k]);
+        const float w = __fsub_rn(x[u][k], y[u][k]);
+        vs[c0 + k] = v;
+        const double dv = (double)v, dw = (double)w;
+        aD = __dadd_rn(aD, __dmul_rn(dw, dw));
+        aE = __dadd_rn(aE, __dmul_rn(dv, dv));
+        mx = max(mx, key_of(v));
+        mxw = max(mxw, key_of(w));
+        dfl |= __float_as_uint(v) ^ __float_as_uint(w);
+      }
+    }
+  }
+  aD = warp_sum_f64(aD); aE = warp_sum_f64(aE);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mxw = max(mxw, __shfl_xor_sync(0xffffffffu, mxw, o));
+    dfl |= __shfl_xor_sync(0xffffffffu, dfl, o);
+  }
+  if (lane == 0) { redd[0][wid] = aD; redd[1][wid] = aE; redu[0][wid] = mx; redu[1][wid] = mxw; redu[2][wid] = dfl; }
+  __syncthreads();
+  mx = 0; mxw = 0; dfl = 0;
+  for (int w = 0; w < TPB / 32; ++w) { mx = max(mx, redu[0][w]); mxw = max(mxw, redu[1][w]); dfl |= redu[2][w]; }
+  const float smax = __uint_as_float(mx);
+
+  // ---- radix select, all candidates at once
+  if (nsel) {
+    for (int i = threadIdx.x; i < BINS1; i += TPB) tab[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < dn; i += TPB) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
+    __syncthreads();
+    for (int j = 0; j < nsel; ++j) {
+      block_find_kth_desc<true>(tab, BINS1, (u32)cs.param[cs.sel[j]], res);
+      if (threadIdx.x == 0) { s_b1[j] = res[0]; s_ab1[j] = res[1]; }
+      __syncthreads();
+    }
+    for (int i = threadIdx.x; i < nsel * BINS2; i += TPB) tab[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < dn; i += TPB) {
+      const u32 key = key_of(vs[i]);
+      for (int j = 0; j < nsel; ++j)
+        if ((key >> 20) == s_b1[j]) atomicAdd(&tab[j * BINS2 + ((key >> 9) & 0x7ffu)], 1u);
+    }
+    __syncthreads();
+    for (int j = 0; j < nsel; ++j) {
+      block_find_kth_desc<true>(tab + j * BINS2, BINS2, (u32)cs.param[cs.sel[j]] - s_ab1[j], res);
+      if (threadIdx.x == 0) { s_p2[j] = (s_b1[j] << 11) | res[0]; s_ab2[j] = s_ab1[j] + res[1]; }
+      __syncthreads();
+    }
+    for (int i = threadIdx.x; i < nsel * BINS3; i += TPB) tab[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < dn; i += TPB) {
+      const u32 key = key_of(vs[i]);
+      for (int j = 0; j < nsel; ++j)
+        if ((key >> 9) == s_p2[j]) atomicAdd(&tab[j * BINS3 + (key & 0x1ffu)], 1u);
+    }
+    __syncthreads();
+    for (int j = 0; j < nsel; ++j) {
+      const u32 K = (u32)cs.param[cs.sel[j]];
+      block_find_kth_desc<true>(tab + j * BINS3, BINS3, K - s_ab2[j], res);
+      if (threadIdx.x == 0) {
+        s_T[j] = (s_p2[j] << 9) | res[0];
+        s_above[j] = s_ab2[j] + res[1];
+        s_ntie[j] = tab[j * BINS3 + res[0]];
+        s_q[j] = K - s_above[j];
+        s_cut[j] = 0xffffffffu;
+      }
+      __syncthreads();
+    }
+    // of the keys equal to a threshold the q with the lowest indices are kept: index of the q-th
+    for (int j = 0; j < nsel; ++j) {
+      if (s_q[j] >= s_ntie[j]) continue;
+      const u32 T = s_T[j], q = s_q[j];
+      const int per = (dn + TPB - 1) / TPB;
+      const int i0 = threadIdx.x * per, i1 = (i0 + per < dn) ? i0 + per : dn;
+      u32 cnt = 0;
+      for (int i = i0; i < i1; ++i) cnt += (key_of(vs[i]) == T) ? 1u : 0u;
+      const u32 ex = block_excl_scan(cnt, nullptr);
+      if (ex < q && q <= ex + cnt) {
+        u32 seen = ex;
+        for (int i = i0; i < i1; ++i)
+          if (key_of(vs[i]) == T && ++seen == q) { s_cut[j] = (u32)i; break; }
+      }
+      __syncthreads();
+    }
+  }
+
+  // ---- tail energies of the Top-K candidates, errors of the quantisers (binary64, exact terms)
+  double aB[MAXC], aQ[MAXC];
+  float qL[MAXC], qinv[MAXC], qstep[MAXC];
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    aB[j] = 0.0; aQ[j] = 0.0; qL[j] = qinv[j] = qstep[j] = 0.f;
+    if (j < cs.nquant) {
+      qL[j] = (float)((1 << ((int)cs.param[cs.qsel[j]] - 1)) - 1);
+      if (smax > 0.f) { qinv[j] = __fdiv_rn(qL[j], smax); qstep[j] = __fdiv_rn(smax, qL[j]); }
+    }
+  }
+  for (int i = threadIdx.x; i < dn; i += TPB) {
+    const float v = vs[i];
+    const u32 key = key_of(v);
+    const double dv = (double)v;
+    const double sq = __dmul_rn(dv, dv);
+#pragma unroll
+    for (int j = 0; j < MAXC; ++j) {
+      if (j < nsel && key < s_T[j]) aB[j] = __dadd_rn(aB[j], sq);
+      if (j < cs.nquant) {
+        const double r = (double)__fsub_rn(v, quant_value(v, qL[j], qinv[j], qstep[j]));
+        aQ[j] = __dadd_rn(aQ[j], __dmul_rn(r, r));
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < MAXC; ++j) {
+    if (j < nsel) { const double t = warp_sum_f64(aB[j]); if (lane == 0) redd[2 + cs.sel[j]][wid] = t; }
+    if (j < cs.nquant) { const double t = warp_sum_f64(aQ[j]); if (lane == 0) redd[2 + cs.qsel[j]][wid] = t; }
+  }
+  __syncthreads();
+  // ---- the row's records, in the form the level choice reads them
+  if (threadIdx.x < NSLOT) {
+    const int sl = threadIdx.x;
+    bool used = (sl < 2);
+    for (int j = 0; j < nsel; ++j) used |= (sl == 2 + cs.sel[j]);
+    for (int j = 0; j < cs.nquant; ++j) used |= (sl == 2 + cs.qsel[j]);
+    double acc = 0.0;
+    if (used)
+      for (int w = 0; w < TPB / 32; ++w) acc += redd[sl][w];
+    partial[(long long)row * MAX_BLK_PER_ROW * NSLOT + sl] = acc;
+  }
+  if (threadIdx.x >= 32 && threadIdx.x < 32 + nsel) {
+    const int j = threadIdx.x - 32;
+    SelRow* sr = sel + row;
+    sr->T[j] = s_T[j]; sr->above[j] = s_above[j]; sr->ntie[j] = s_ntie[j]; sr->q[j] = s_q[j];
+    sr->extraE[j] = 0.0; sr->tiemode[j] = (s_q[j] < s_ntie[j]) ? 1u : 0u; sr->cut[j] = s_cut[j];
+  }
+  if (threadIdx.x == 64) {
+    maxkey[row] = mx;
+    diffflag[row] = ((mxw >= 0x7f800000u) ? 0x80000000u : 0u) | (dfl & 0x7fffffffu);
+  }
+  __syncthreads();
+  pick_row(cs, d, row, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+  __syncthreads();
+  if (__ldcg(&dec[row].need_exact)) {
+    // the comparison could not be certified: exact integer sums of the row, then the decision from them
+    for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) lsh[i] = 0;
+    __syncthreads();
+    // A square is mant^2 * 2^off units of 2^-298.  Squares whose offset lies within 64 bits below the
+    // largest one of the row are added in per-thread 128-bit integers anchored at bit `wb` (at most 128
+    // terms of at most 113 bits each); the few that lie lower go straight to the shared limbs.
+    const u32 kmax = max(mx, mxw);
+    const int off_max = 2 * (int)((kmax >> 23) ? (kmax >> 23) : 1u) - 2;
+    const int wb = off_max > 64 ? off_max - 64 : 0;
+    unsigned __int128 accD = 0, accE = 0, accC[MAXC];
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) accC[c] = 0;
+    // square of a finite value as a 128-bit integer anchored at bit wb; false if it lies below the window
+    auto sq_term = [&](float val, unsigned __int128* term) -> bool {
+      const u32 bkey = key_of(val);
+      const u32 ex = bkey >> 23, fr = bkey & 0x7fffffu;
+      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
+      const int off = 2 * (int)(ex ? ex : 1u) - 2;
+      *term = (off >= wb) ? (unsigned __int128)(m * m) << (off - wb) : (unsigned __int128)0;
+      return off >= wb || m == 0;
+    };
+    auto slow_add = [&](int slot, float val) {   // rare: more than 2^32 times smaller than the row's largest entry
+      int kk; u32 p[3];
+      sq_pieces(val, &kk, p);
+      limb_add(lsh + slot * NLIMB, kk, p);
+    };
+    for (int i = threadIdx.x; i < dn; i += TPB) {
+      const float v = vs[i];
+      const float w = __fsub_rn(xr[i], yr[i]);
+      if (key_of(w) >= 0x7f800000u || key_of(v) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
+      unsigned __int128 tw, tv;
+      if (sq_term(w, &tw)) accD += tw; else slow_add(0, w);
+      const bool v_in = sq_term(v, &tv);
+      if (v_in) accE += tv; else slow_add(1, v);
+      const u32 key = key_of(v);
+#pragma unroll
+      for (int j = 0; j < MAXC; ++j)
+        if (j < nsel && key < s_T[j] && v_in) accC[j] += tv;
+      if (!v_in)
+        for (int j = 0; j < nsel; ++j)
+          if (key < s_T[j]) slow_add(2 + cs.sel[j], v);
+      for (int j = 0; j < cs.nquant; ++j) {
+        const float r = __fsub_rn(v, quant_value(v, qL[j], qinv[j], qstep[j]));
+        unsigned __int128 tr;
+        if (sq_term(r, &tr)) {
+#pragma unroll
+          for (int c = 0; c < MAXC; ++c)
+            if (c == MAXC - 1 - j) accC[c] += tr;
+        } else slow_add(2 + cs.qsel[j], r);
+      }
+    }
+    // The per-thread integers are added up as four 32-bit pieces each: over the warp with shuffles, over the
+    // warps through `wacc` (64-bit shared atomics are compare-and-swap loops: with every thread of the CTA on
+    // the same few words they would take hundreds of microseconds), and only the totals go into the limbs.
+    __shared__ u64 wacc[TPB / 32][NSLOT][4];
+    auto stash = [&](unsigned __int128 acc, int slot) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        u64 piece = (u64)(u32)(acc >> (32 * i));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) piece += __shfl_xor_sync(0xffffffffu, piece, o);
+        if (lane == 0) wacc[wid][slot][i] = piece;
+      }
+    };
+    for (int i = threadIdx.x; i < (TPB / 32) * NSLOT * 4; i += TPB) (&wacc[0][0][0])[i] = 0;
+    __syncthreads();
+    stash(accD, 0);
+    stash(accE, 1);
+#pragma unroll
+    for (int j = 0; j < MAXC; ++j) {
+      if (j < nsel) stash(accC[j], 2 + cs.sel[j]);
+      if (j < cs.nquant) stash(accC[MAXC - 1 - j], 2 + cs.qsel[j]);
+    }
+    __syncthreads();
+    if (threadIdx.x < NSLOT * 4) {
+      const int slot = threadIdx.x >> 2, i = threadIdx.x & 3;
+      u64 tot = 0;                                     // < 2^32 * 256 threads = 2^40
+      for (int w = 0; w < TPB / 32; ++w) tot += wacc[w][slot][i];
+      const int k0 = (wb >> 5) + i, sh = wb & 31;
+      const u64 lo = (tot & 0xffffffffull) << sh, hi = (tot >> 32) << sh;      // weights 2^(32 k0) and 2^(32 (k0 + 1))
+      if (lo & 0xffffffffull) atomicAdd(&lsh[slot * NLIMB + k0], lo & 0xffffffffull);
+      if ((lo >> 32) + (hi & 0xffffffffull)) atomicAdd(&lsh[slot * NLIMB + k0 + 1], (lo >> 32) + (hi & 0xffffffffull));
+      if (hi >> 32) atomicAdd(&lsh[slot * NLIMB + k0 + 2], hi >> 32);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) pick_exact_row<true>(cs, row, d, lsh, sel, maxkey, dec, out, diffflag, flags);
+    __syncthreads();
+  }
+
+  // ---- the update of the row (Eq. 7 at the chosen level)
+  const int mode = __ldcg(&dec[row].mode);
+  if (mode != 0) {
+    const u32 T = __ldcg(&dec[row].T), cut = __ldcg(&dec[row].cut);
+    const float L = __ldcg(&dec[row].qL), inv = __ldcg(&dec[row].qinv), step = __ldcg(&dec[row].qstep);
+    for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
+      float gq[SB][4];
+#pragma unroll
+      for (int u = 0; u < SB; ++u)
+        if (base + u * TPB * 4 < dn) load4<ALIGNED>(gr, base + u * TPB * 4, d, gq[u]);
+#pragma unroll
+      for (int u = 0; u < SB; ++u) {
+        const int c0 = base + u * TPB * 4;
+        if (c0 >= dn) break;
+        bool any = false;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (c0 + k >= dn) break;
+          const float v = vs[c0 + k];
+          const u32 key = key_of(v);
+          bool kept = true;
+          float add = v;
+          if (mode == 1) kept = (key > T) || (key == T && (u32)(c0 + k) <= cut);
+          else if (mode == 3) add = quant_value(v, L, inv, step);
+          if (kept) {
+            gq[u][k] = __fadd_rn(gq[u][k], add);
+            any = true;
+            if (out.kept_idx && mode != 3) {
+              const long long pos = (long long)atomicAdd((u64*)&out.kept_cnt[row], 1ull);
+              if (pos < out.kept_stride) out.kept_idx[(long long)row * out.kept_stride + pos] = c0 + k;
+            }
+          }
+        }
+        if (any) store4<ALIGNED>(gr, c0, d, gq[u]);
+      }
+    }
+  }
+
+  // ---- the mean over the rows, by the CTA that finishes last (rows summed in order, one division)
+  if (out.mean_out == nullptr) return;
+  if (!last_cta_of_row(&tickets[15], (u32)rows)) return;
+  const float nf = (float)rows;
+  for (int c0 = threadIdx.x * 4; c0 < dn; c0 += TPB * 4) {
+    float acc[4] = {-0.f, -0.f, -0.f, -0.f};
+    for (int i0 = 0; i0 < rows; i0 += 8) {   // eight rows requested at once, added in row order
+      float g[8][4];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) g[u][k] = 0.f;
+        if (i < rows) {
+          const float* src = G + (long long)i * d + c0;
+          if (ALIGNED) {
+            const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
+            g[u][0] = t.x; g[u][1] = t.y; g[u][2] = t.z; g[u][3] = t.w;
+          } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (c0 + k < dn) g[u][k] = __ldcg(src + k);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (i0 + u >= rows) break;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[u][k]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (c0 + k < dn) out.mean_out[c0 + k] = __fdiv_rn(acc[k], nf);
+  }
+}
+
+// --------------------------------------------------------------------------
 // host side
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -2039,6 +2403,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
     cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
     cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
+    cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
+    cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
     cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     attr_done = true;
@@ -2076,6 +2442,21 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
   cudaMemsetAsync(s.zero_begin, 0, s.zero_bytes, stream);  // histograms, limbs, row flags: one contiguous region
   prof_end(pf, stream);
+
+  if (!single && d <= SMALL_DMAX) {
+    // short rows: everything in one launch, one CTA per row
+    const size_t shm = 4 * ((size_t)((d + 3) / 4) * 4 + (size_t)(cs.nsel > 1 ? cs.nsel : 1) * BINS2);
+    const double tol64 = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
+    const bool al4 = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y);
+    prof_begin(pf, KID_SMALL, stream);
+    if (al4) launch_k(k_small_rows<true>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
+                      s.maxkey, s.diffflag, s.limbs, s.flags, s.tickets, out, tol64);
+    else launch_k(k_small_rows<false>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
+                  s.maxkey, s.diffflag, s.limbs, s.flags, s.tickets, out, tol64);
+    prof_end(pf, stream);
+    ++launches;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+  }
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
   long long want = (148 * 4 + rows - 1) / rows;   // one wave of the streaming pass: four resident CTAs per SM
