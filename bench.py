@@ -197,7 +197,7 @@ KERNEL_BYTES = {"k_pass1": 12, "k_update": 8, "k_hist<1>": 8, "k_hist<2>": 8, "k
 # one worker launch of workload c5 at half size, 8 x 12.5e6; the traffic grows in proportion to the
 # elements a launch processes).  Valid for the kernels as committed with profiles/c5_compress_step.txt;
 # a kernel that changes afterwards loses its entry until it is captured again.
-NCU_DRAM_BYTES_PER_ELEM = {"k_pass1": 12.10, "k_update": 8.53}
+NCU_DRAM_BYTES_PER_ELEM = {"k_pass1": 12.10, "k_update": 8.50}
 
 
 def kernel_table(prof):

@@ -1884,14 +1884,44 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
 // One CTA per row, the row's difference vector v = X - G kept in shared memory: three radix passes
 // (11 + 11 + 9 bits, all Top-K candidates at once), tail energies and quantiser errors in binary64,
 // the index cut of threshold-equal keys, the level choice (pick_row, with the exact integer sums
-// when a comparison cannot be certified), the update of the row, and - by the CTA that finishes
-// last - the mean over the rows.  Serves problems too small to keep the multi-kernel path busy.
+// when a comparison cannot be certified) and the update of the row; the mean over the rows follows in
+// k_small_mean.  Serves problems too small to keep the multi-kernel path busy.
+// Finds, in a shared-memory histogram of nb bins (a multiple of 32) ordered by key, the bin that holds
+// the krem-th largest key; one warp calls, every lane gets (bin, number of keys in higher bins).
+__device__ __forceinline__ void warp_find_kth_desc(const u32* hist, int nb, u32 krem, u32* bin, u32* above) {
+  const int lane = threadIdx.x & 31;
+  const int per = nb / 32;                              // this lane: descending positions per*lane .. per*lane + per - 1
+  u32 sum = 0;
+  for (int k = 0; k < per; ++k) sum += hist[nb - 1 - (per * lane + k)];
+  u32 inc = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  const u32 excl = inc - sum;
+  const bool mine = krem > excl && krem <= excl + sum;   // true in exactly one lane when 1 <= krem <= total
+  u32 fb = 0, fa = 0;
+  if (mine) {
+    u32 run = excl;
+    for (int k = 0; k < per; ++k) {
+      const u32 v = hist[nb - 1 - (per * lane + k)];
+      if (krem <= run + v) { fb = (u32)(nb - 1 - (per * lane + k)); fa = run; break; }
+      run += v;
+    }
+  }
+  const u32 who = __ballot_sync(0xffffffffu, mine);
+  const int src = who ? (__ffs(who) - 1) : 0;
+  *bin = __shfl_sync(0xffffffffu, fb, src);
+  *above = __shfl_sync(0xffffffffu, fa, src);
+}
+
 constexpr int SMALL_DMAX = 32768;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
                                                     int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
-                                                    double* partial, u32* maxkey, u32* diffflag, u64* limbs,
-                                                    u32* flags, u32* tickets, CompressOut out, double tol) {
+                                                    double* partial, u32* maxkey, u32* diffflag, u32* flags,
+                                                    CompressOut out, double tol) {
   pdl_begin();
   extern __shared__ __align__(16) unsigned char small_smem[];
   const int dn = (int)d;
@@ -1899,7 +1929,6 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   u32* tab = reinterpret_cast<u32*>(small_smem) + ((dn + 3) / 4) * 4;     // max(BINS1, nsel * BINS2) words
   __shared__ double redd[NSLOT][TPB / 32];
   __shared__ u32 redu[3][TPB / 32];
-  __shared__ u32 res[2];
   __shared__ u32 s_b1[MAXC], s_ab1[MAXC], s_p2[MAXC], s_ab2[MAXC], s_T[MAXC], s_above[MAXC], s_ntie[MAXC], s_q[MAXC], s_cut[MAXC];
   __shared__ u64 lsh[NSLOT * NLIMB];
   const int row = blockIdx.x;
@@ -1961,11 +1990,12 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     __syncthreads();
     for (int i = threadIdx.x; i < dn; i += TPB) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
     __syncthreads();
-    for (int j = 0; j < nsel; ++j) {
-      block_find_kth_desc<true>(tab, BINS1, (u32)cs.param[cs.sel[j]], res);
-      if (threadIdx.x == 0) { s_b1[j] = res[0]; s_ab1[j] = res[1]; }
-      __syncthreads();
+    if (wid < nsel) {   // one warp per candidate
+      u32 bin, above;
+      warp_find_kth_desc(tab, BINS1, (u32)cs.param[cs.sel[wid]], &bin, &above);
+      if (lane == 0) { s_b1[wid] = bin; s_ab1[wid] = above; }
     }
+    __syncthreads();
     for (int i = threadIdx.x; i < nsel * BINS2; i += TPB) tab[i] = 0;
     __syncthreads();
     for (int i = threadIdx.x; i < dn; i += TPB) {
@@ -1974,11 +2004,12 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
         if ((key >> 20) == s_b1[j]) atomicAdd(&tab[j * BINS2 + ((key >> 9) & 0x7ffu)], 1u);
     }
     __syncthreads();
-    for (int j = 0; j < nsel; ++j) {
-      block_find_kth_desc<true>(tab + j * BINS2, BINS2, (u32)cs.param[cs.sel[j]] - s_ab1[j], res);
-      if (threadIdx.x == 0) { s_p2[j] = (s_b1[j] << 11) | res[0]; s_ab2[j] = s_ab1[j] + res[1]; }
-      __syncthreads();
+    if (wid < nsel) {
+      u32 bin, above;
+      warp_find_kth_desc(tab + wid * BINS2, BINS2, (u32)cs.param[cs.sel[wid]] - s_ab1[wid], &bin, &above);
+      if (lane == 0) { s_p2[wid] = (s_b1[wid] << 11) | bin; s_ab2[wid] = s_ab1[wid] + above; }
     }
+    __syncthreads();
     for (int i = threadIdx.x; i < nsel * BINS3; i += TPB) tab[i] = 0;
     __syncthreads();
     for (int i = threadIdx.x; i < dn; i += TPB) {
@@ -1987,18 +2018,20 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
         if ((key >> 9) == s_p2[j]) atomicAdd(&tab[j * BINS3 + (key & 0x1ffu)], 1u);
     }
     __syncthreads();
-    for (int j = 0; j < nsel; ++j) {
+    if (wid < nsel) {
+      const int j = wid;
       const u32 K = (u32)cs.param[cs.sel[j]];
-      block_find_kth_desc<true>(tab + j * BINS3, BINS3, K - s_ab2[j], res);
-      if (threadIdx.x == 0) {
-        s_T[j] = (s_p2[j] << 9) | res[0];
-        s_above[j] = s_ab2[j] + res[1];
-        s_ntie[j] = tab[j * BINS3 + res[0]];
+      u32 bin, above;
+      warp_find_kth_desc(tab + j * BINS3, BINS3, K - s_ab2[j], &bin, &above);
+      if (lane == 0) {
+        s_T[j] = (s_p2[j] << 9) | bin;
+        s_above[j] = s_ab2[j] + above;
+        s_ntie[j] = tab[j * BINS3 + bin];
         s_q[j] = K - s_above[j];
         s_cut[j] = 0xffffffffu;
       }
-      __syncthreads();
     }
+    __syncthreads();
     // of the keys equal to a threshold the q with the lowest indices are kept: index of the q-th
     for (int j = 0; j < nsel; ++j) {
       if (s_q[j] >= s_ntie[j]) continue;
@@ -2200,42 +2233,47 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     }
   }
 
-  // ---- the mean over the rows, by the CTA that finishes last (rows summed in order, one division)
-  if (out.mean_out == nullptr) return;
-  if (!last_cta_of_row(&tickets[15], (u32)rows)) return;
+}
+
+// The mean over short rows (summed in row order, one division): a thread owns four columns and
+// requests eight rows at once.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_small_mean(const float* G, int rows, long long d, float* __restrict__ mean_out) {
+  pdl_begin();
+  const int dn = (int)d;
+  const int c0 = (blockIdx.x * TPB + threadIdx.x) * 4;
+  if (c0 >= dn) return;
   const float nf = (float)rows;
-  for (int c0 = threadIdx.x * 4; c0 < dn; c0 += TPB * 4) {
-    float acc[4] = {-0.f, -0.f, -0.f, -0.f};
-    for (int i0 = 0; i0 < rows; i0 += 8) {   // eight rows requested at once, added in row order
-      float g[8][4];
+  float acc[4] = {-0.f, -0.f, -0.f, -0.f};
+  for (int i0 = 0; i0 < rows; i0 += 8) {
+    float g[8][4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = i0 + u;
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) g[u][k] = 0.f;
-        if (i < rows) {
-          const float* src = G + (long long)i * d + c0;
-          if (ALIGNED) {
-            const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
-            g[u][0] = t.x; g[u][1] = t.y; g[u][2] = t.z; g[u][3] = t.w;
-          } else {
+      for (int k = 0; k < 4; ++k) g[u][k] = 0.f;
+      if (i < rows) {
+        const float* src = G + (long long)i * d + c0;
+        if (ALIGNED) {
+          const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
+          g[u][0] = t.x; g[u][1] = t.y; g[u][2] = t.z; g[u][3] = t.w;
+        } else {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              if (c0 + k < dn) g[u][k] = __ldcg(src + k);
-          }
+          for (int k = 0; k < 4; ++k)
+            if (c0 + k < dn) g[u][k] = __ldcg(src + k);
         }
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (i0 + u >= rows) break;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[u][k]);
       }
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (c0 + k < dn) out.mean_out[c0 + k] = __fdiv_rn(acc[k], nf);
+    for (int u = 0; u < 8; ++u) {
+      if (i0 + u >= rows) break;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[u][k]);
+    }
   }
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (c0 + k < dn) mean_out[c0 + k] = __fdiv_rn(acc[k], nf);
 }
 
 // --------------------------------------------------------------------------
@@ -2450,11 +2488,19 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     const bool al4 = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y);
     prof_begin(pf, KID_SMALL, stream);
     if (al4) launch_k(k_small_rows<true>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                      s.maxkey, s.diffflag, s.limbs, s.flags, s.tickets, out, tol64);
+                      s.maxkey, s.diffflag, s.flags, out, tol64);
     else launch_k(k_small_rows<false>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                  s.maxkey, s.diffflag, s.limbs, s.flags, s.tickets, out, tol64);
+                  s.maxkey, s.diffflag, s.flags, out, tol64);
     prof_end(pf, stream);
     ++launches;
+    if (out.mean_out) {
+      const dim3 mgrid((unsigned)((d + TPB * 4 - 1) / (TPB * 4)));
+      prof_begin(pf, KID_SMALL, stream);
+      if (al4 && aligned16(out.mean_out)) launch_k(k_small_mean<true>, mgrid, dim3(TPB), 0, stream, pdl, (const float*)G, rows, d, out.mean_out);
+      else launch_k(k_small_mean<false>, mgrid, dim3(TPB), 0, stream, pdl, (const float*)G, rows, d, out.mean_out);
+      prof_end(pf, stream);
+      ++launches;
+    }
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
 
