@@ -752,17 +752,18 @@ __device__ __forceinline__ bool apply_topk4(float (&g)[4], const float (&x)[4], 
   }
   return any;
 }
-// Rows r0 .. r0 + nr - 1 of one chunk for a thread's four columns, every row either skipped or a Top-K
-// level with an index cut (modes 0 and 1 of `rd`): UPD_RB rows in flight as plain 128-bit loads, applied
-// in row order so that `acc` sums the mean in worker order.
+// Rows r0 .. r0 + nr - 1 of one chunk for a thread's four columns, every row skipped (mode 0), a Top-K
+// level with an index cut (1), the identity (2) or a quantiser (3): RB rows in flight as plain 128-bit
+// loads, applied in row order so that `acc` sums the mean in worker order.
+template <int RB>
 __device__ __forceinline__ void update_rows_simple(const float* __restrict__ X, float* __restrict__ G, long long d,
                                                    long long c0, int r0, int nr, const RowDec* rd, bool want_mean,
                                                    float (&acc)[4]) {
   const u32 c0u = (u32)c0;
-  for (int q0 = 0; q0 < nr; q0 += UPD_RB) {
-    float4 gq[UPD_RB], xq[UPD_RB];
+  for (int q0 = 0; q0 < nr; q0 += RB) {
+    float4 gq[RB], xq[RB];
 #pragma unroll
-    for (int u = 0; u < UPD_RB; ++u) {
+    for (int u = 0; u < RB; ++u) {
       gq[u] = make_float4(0.f, 0.f, 0.f, 0.f); xq[u] = gq[u];
       const int ii = q0 + u;
       if (ii < nr) {
@@ -772,14 +773,24 @@ __device__ __forceinline__ void update_rows_simple(const float* __restrict__ X, 
       }
     }
 #pragma unroll
-    for (int u = 0; u < UPD_RB; ++u) {
+    for (int u = 0; u < RB; ++u) {
       const int ii = q0 + u;
       if (ii >= nr) break;
       float g[4] = {gq[u].x, gq[u].y, gq[u].z, gq[u].w};
-      if (rd[ii].mode != 0) {
+      const int m = rd[ii].mode;
+      if (m != 0) {
         const float x[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
-        if (apply_topk4(g, x, rd[ii].T, rd[ii].cut, c0u))
-          *reinterpret_cast<float4*>(G + (long long)(r0 + ii) * d + c0) = make_float4(g[0], g[1], g[2], g[3]);
+        bool any = true;
+        if (m == 1) any = apply_topk4(g, x, rd[ii].T, rd[ii].cut, c0u);
+        else if (m == 2) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) g[k] = __fadd_rn(g[k], __fsub_rn(x[k], g[k]));
+        } else {
+          const float L = rd[ii].qL, inv = rd[ii].qinv, step = rd[ii].qstep;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) g[k] = __fadd_rn(g[k], quant_value(__fsub_rn(x[k], g[k]), L, inv, step));
+        }
+        if (any) *reinterpret_cast<float4*>(G + (long long)(r0 + ii) * d + c0) = make_float4(g[0], g[1], g[2], g[3]);
       }
       if (want_mean) {
 #pragma unroll
@@ -806,13 +817,13 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
     if (threadIdx.x < rows) shd[threadIdx.x] = dec[threadIdx.x];
     __syncthreads();
     bool simple = true;
-    if (threadIdx.x < rows) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
+    if (threadIdx.x < rows) simple = shd[threadIdx.x].mode != 4 && !(shd[threadIdx.x].mode == 1 && shd[threadIdx.x].need_tie);
     if (__syncthreads_and(simple ? 1 : 0)) {
       for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
         const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
         if (c0 >= d) continue;
         float acc[4] = {-0.f, -0.f, -0.f, -0.f};  // -0 + g == g bit for bit, so the first row needs no special case
-        update_rows_simple(X, G, d, c0, 0, rows, shd, want_mean, acc);
+        update_rows_simple<UPD_RB>(X, G, d, c0, 0, rows, shd, want_mean, acc);
         if (want_mean) {
           const float n = (float)rows;
           *reinterpret_cast<float4*>(out.mean_out + c0) =
@@ -840,10 +851,13 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
       // Common case for the whole tile of rows: every row either skips or applies a Top-K level whose
       // threshold-equal keys are decided by the index cut, and no kept-index list is wanted.
       bool simple = true;
-      if (threadIdx.x < nr) simple = (shd[threadIdx.x].mode == 0) || (shd[threadIdx.x].mode == 1 && !shd[threadIdx.x].need_tie);
+      if (threadIdx.x < nr) simple = shd[threadIdx.x].mode != 4 && !(shd[threadIdx.x].mode == 1 && shd[threadIdx.x].need_tie);
       simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
       if (simple && ALIGNED) {
-        if (live) update_rows_simple(X, G, d, c0, r0, nr, shd, want_mean, acc);
+        if (live) {   // few chunks (short rows): more rows in flight per thread, the SMs are not full
+          if (gridDim.x < 148 * 2) update_rows_simple<4>(X, G, d, c0, r0, nr, shd, want_mean, acc);
+          else update_rows_simple<UPD_RB>(X, G, d, c0, r0, nr, shd, want_mean, acc);
+        }
         continue;
       }
       if (simple) {
