@@ -96,35 +96,49 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def dist_setup():
-    import torch
+def dist_setup(backend: str = "nccl"):
+    """One process per GPU (replicas only: the ranks exchange nothing but the timing).  With backend
+    "gloo" no GPU is touched: the CPU tests run the same rendezvous, barrier and reduction."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
+    if backend == "nccl":
+        import torch
+        torch.cuda.set_device(local)
     if world > 1:
+        import torch
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     return rank, world, local
 
 
-def barrier_sync(world):
+def barrier_sync(world, device: str = "cuda"):
     import torch
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if device == "cuda":
+        torch.cuda.synchronize()
 
 
-def max_over_ranks(value: float, world) -> float:
+def max_over_ranks(value: float, world, device: str = "cuda") -> float:
+    """The slowest rank sets the time of the job."""
     import torch
     if world == 1:
         return value
     import torch.distributed as dist
-    t = torch.tensor([value], dtype=torch.float64, device="cuda")
+    t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def job_throughput(units_per_rank_step: float, steps: int, ms_max: float, world: int) -> float:
+    """Whole-job units per second: every rank processed the same units in the time of the slowest."""
+    return world * units_per_rank_step * steps / (ms_max * 1e-3)
 
 
 # ----------------------------------------------------------------------------- oracle legs
@@ -259,7 +273,7 @@ def bench_c5(args, rank, world, local):
     levels_seen = level.cpu().tolist() + mlevel.cpu().tolist()
     ms = max_over_ranks(ms, world)
     elems_per_step = n * d + d
-    value = world * elems_per_step * args.steps / (ms * 1e-3)
+    value = job_throughput(elems_per_step, args.steps, ms, world)
 
     # roofline of the dominant kernel: algorithmic bytes of its launches / its device time
     peak, peak_src = measured_peaks()
@@ -367,7 +381,7 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     eng.profile_enable(0)
     recs, levels = eng.step(1, report=True)
     elems_per_step = n * d + (d if W["master"] else 0)
-    value = world * elems_per_step * steps / (ms * 1e-3)
+    value = job_throughput(elems_per_step, steps, ms, world)
     peak, peak_src = measured_peaks()
     # one pass over the features: dense 4 B per entry; CSR value + column index per stored entry
     a_bytes = 4 * n * m * d if csr is None else 8 * int(csr[1].numel())
