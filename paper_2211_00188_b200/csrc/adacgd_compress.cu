@@ -3,10 +3,16 @@
 //   (both sides of the trigger, Eq. 10), the adaptive level choice and the
 //   estimator update (Eq. 11), and g~ = (1/n) sum_i g_i (Algorithm 1).
 //
-// Selection is an exact three-pass radix select on the bit pattern of |v|
-// (11 + 11 + 9 bits), shared by all Top-K candidates of a row.  Energies are
-// summed in binary64 from non-negative exact terms; a comparison whose margin is
-// below the worst-case summation error is redone in exact integer arithmetic.
+// Three routes to the same results, chosen by size in launch_compress():
+//   - large problems: thresholds are bracketed from a sample (k_sample), one streaming pass over
+//     X, G, Y (k_pass1) gathers the sums and lists the few keys inside a bracket, the exact
+//     selection runs on those lists (k_lcollect, k_lhist), k_update applies the chosen level;
+//   - the three-pass radix select on the bit pattern of |v| (11 + 11 + 9 bits: k_hist, k_energy),
+//     shared by all Top-K candidates of a row: mid-size problems, and the per-row fallback of
+//     the first route;
+//   - short rows: everything in one CTA per row (k_small_rows).
+// Energies are sums of non-negative exact terms; a comparison whose margin is below the
+// worst-case summation error is redone in exact integer arithmetic.
 #include "adacgd_internal.cuh"
 
 namespace adacgd {
@@ -2621,9 +2627,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk, s.tickets);
   }
   {
-    // Not a programmatic dependent: CTAs of this persistent grid that become resident while earlier kernels
-    // still hold part of the SMs end up unevenly spread, and the fullest SM then sets the pace (measured:
-    // 400 us instead of 270 us on 8 x 25e6).
+    // Not a programmatic dependent: launched as one, this persistent grid ran 400 us instead of 270 us on
+    // 8 x 25e6 (its CTAs become resident while earlier kernels still hold part of the SMs).
     const bool pdl = false;
     TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
   }
