@@ -159,8 +159,11 @@ adacgd_status adacgd_compress(adacgd_ctx* ctx, const float* X_dev, float* G_dev,
 
 /* The same operation on HOST arrays: copies X, G, Y to the context's staging area
  * (requires ADACGD_FLAG_HOST_STAGING), runs adacgd_compress, copies G (and the mean,
- * levels, bits if requested) back, and synchronises.  Pinned host memory makes the
- * copies asynchronous but is not required. */
+ * levels, bits if requested) back, and synchronises.  The rows are taken in up to four
+ * groups so that a group's results go back (on a second stream the context creates at
+ * the first call) while the next group is still coming in; the results are those of one
+ * adacgd_compress call on all rows.  Pinned host memory makes the copies asynchronous
+ * but is not required. */
 adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* G_host,
                                    const float* Y_host, int32_t rows, int64_t d,
                                    const adacgd_cset* cset, float* mean_out_host,

@@ -148,6 +148,8 @@ struct adacgd_ctx {
   StepLog* log;
   int* loglevels;
   float* stage;
+  cudaStream_t copy_stream;    // second stream of adacgd_compress_host (created at its first call): results go back
+  cudaEvent_t copy_ev[5];      // to the host while the next group of rows is still coming in
   long long launches;
   cudaGraphExec_t pair_exec;   // two captured iterations (the buffers ping-pong with period 2)
   long long pair_launches;
@@ -265,6 +267,8 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   c->log = (StepLog*)(b + L.log);
   c->loglevels = (int*)(b + L.loglevels);
   c->stage = (flags & ADACGD_FLAG_HOST_STAGING) ? (float*)(b + L.stage) : nullptr;
+  c->copy_stream = nullptr;
+  for (cudaEvent_t& e : c->copy_ev) e = nullptr;
   c->x = c->G = c->grad_cur = c->grad_nxt = c->gt_cur = c->gt_nxt = c->gm = c->gm_buf = nullptr;
 
   if (cudaMemsetAsync(c->scr.flags, 0, 16, c->stream) != cudaSuccess ||
@@ -367,7 +371,6 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
   if (!X_host || !G_host || !Y_host) return fail(ctx, ADACGD_ERR_INVALID_ARG, "X, G, Y must be non-NULL");
   if (rows < 1 || rows > ctx->p.n || d < 1 || d > ctx->p.d)
     return fail(ctx, ADACGD_ERR_INVALID_ARG, "rows/d exceed the shape given at init");
-  const size_t nd = (size_t)rows * (size_t)d * 4;
   const size_t cap = (size_t)ctx->p.n * (size_t)ctx->p.d;
   float* Xs = ctx->stage;
   float* Gs = Xs + cap;
@@ -375,17 +378,38 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
   float* Ms = Ys + cap;
   unsigned int flags_before = 0, flags_after = 0;
   cudaMemcpyAsync(&flags_before, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
-  cudaMemcpyAsync(Xs, X_host, nd, cudaMemcpyHostToDevice, ctx->stream);
-  cudaMemcpyAsync(Gs, G_host, nd, cudaMemcpyHostToDevice, ctx->stream);
-  cudaMemcpyAsync(Ys, Y_host, nd, cudaMemcpyHostToDevice, ctx->stream);
-  adacgd_status s = adacgd_compress(ctx, Xs, Gs, Ys, rows, d, cset, mean_out_host ? Ms : nullptr,
-                                    level_host ? ctx->levels : nullptr, bits_host ? (uint64_t*)ctx->bits : nullptr,
-                                    nullptr, nullptr, nullptr, 0, nullptr);
-  if (s != ADACGD_OK) return s;
-  cudaMemcpyAsync(G_host, Gs, nd, cudaMemcpyDeviceToHost, ctx->stream);
-  if (mean_out_host) cudaMemcpyAsync(mean_out_host, Ms, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  // The rows are taken in up to four groups: while a group's estimators travel back to the host on a second
+  // stream, the next group's operands are still coming in (the link carries both directions at once).  The
+  // mean needs every row and follows in a kernel of its own, summed in row order like the fused one.
+  if (!ctx->copy_stream) {
+    if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return cuda_fail(ctx, "stream for host copies");
+    for (cudaEvent_t& e : ctx->copy_ev)
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return cuda_fail(ctx, "event for host copies");
+  }
+  const int ngroups = rows < 4 ? rows : 4;
+  for (int g = 0; g < ngroups; ++g) {
+    const int r0 = (int)((long long)rows * g / ngroups), r1 = (int)((long long)rows * (g + 1) / ngroups);
+    const size_t off = (size_t)r0 * (size_t)d, bytes = (size_t)(r1 - r0) * (size_t)d * 4;
+    cudaMemcpyAsync(Xs + off, X_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
+    cudaMemcpyAsync(Gs + off, G_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
+    cudaMemcpyAsync(Ys + off, Y_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
+    adacgd_status s = adacgd_compress(ctx, Xs + off, Gs + off, Ys + off, r1 - r0, d, cset, nullptr,
+                                      level_host ? ctx->levels + r0 : nullptr,
+                                      bits_host ? (uint64_t*)ctx->bits + r0 : nullptr, nullptr, nullptr, nullptr, 0, nullptr);
+    if (s != ADACGD_OK) { cudaStreamSynchronize(ctx->copy_stream); return s; }
+    cudaEventRecord(ctx->copy_ev[g], ctx->stream);
+    cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_ev[g], 0);
+    cudaMemcpyAsync(G_host + off, Gs + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_stream);
+  }
+  if (mean_out_host) {
+    if (launch_mean_rows(Gs, rows, d, Ms, ctx->stream) < 0) return cuda_fail(ctx, "mean over rows");
+    ctx->launches += 1;
+    cudaMemcpyAsync(mean_out_host, Ms, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->stream);
+  }
   if (level_host) cudaMemcpyAsync(level_host, ctx->levels, (size_t)rows * 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (bits_host) cudaMemcpyAsync(bits_host, ctx->bits, (size_t)rows * 8, cudaMemcpyDeviceToHost, ctx->stream);
+  cudaEventRecord(ctx->copy_ev[4], ctx->copy_stream);
+  cudaStreamWaitEvent(ctx->stream, ctx->copy_ev[4], 0);
   cudaMemcpyAsync(&flags_after, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_compress_host");
   if (flags_after & 2u) return fail(ctx, ADACGD_ERR_CUDA, "a device-side wait for an asynchronous copy timed out");
@@ -600,6 +624,8 @@ void adacgd_destroy(adacgd_ctx* ctx) {
   for (cudaEvent_t e : ctx->ev_beg) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->ev_end) cudaEventDestroy(e);
   if (ctx->pair_exec) cudaGraphExecDestroy(ctx->pair_exec);
+  for (cudaEvent_t e : ctx->copy_ev) if (e) cudaEventDestroy(e);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   delete ctx;
 }
 

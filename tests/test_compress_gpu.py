@@ -230,9 +230,11 @@ def test_argument_errors(torch):
         eng.step(1)
 
 
-def test_host_entry_point(torch):
+@pytest.mark.parametrize("n", [1, 3, 6])
+def test_host_entry_point(torch, n):
+    # the rows travel in up to four groups, results going back while the next group comes in
     import paper_2211_00188_b200 as pkg
-    n, d = 3, 10000
+    d = 10000
     X, G, Y = S.gaussian_rows(n, d, seed=10)
     eng = pkg.AdaCGD(n, d, CANDS3, 1.0, host_staging=True)
     Xh, Gh, Yh = (torch.from_numpy(a.copy()).pin_memory() for a in (X, G, Y))
