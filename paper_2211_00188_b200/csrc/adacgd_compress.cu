@@ -825,6 +825,31 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
     bool simple = true;
     if (threadIdx.x < rows) simple = shd[threadIdx.x].mode != 4 && !(shd[threadIdx.x].mode == 1 && shd[threadIdx.x].need_tie);
     if (__syncthreads_and(simple ? 1 : 0)) {
+      if (rows == 1 && !want_mean && shd[0].mode == 1) {
+        // a single row (the master step): nothing to keep in flight across rows, so four chunks at a time
+        const u32 T = shd[0].T, cut = shd[0].cut;
+        for (long long chunk = blockIdx.x; chunk < nchunk; chunk += 4ll * gridDim.x) {
+          float4 gq[4], xq[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const long long c0 = (chunk + (long long)u * gridDim.x) * UPD_COLS + threadIdx.x * 4;
+            gq[u] = make_float4(0.f, 0.f, 0.f, 0.f); xq[u] = gq[u];
+            if (c0 < d) {
+              gq[u] = *reinterpret_cast<const float4*>(G + c0);
+              xq[u] = __ldcs(reinterpret_cast<const float4*>(X + c0));
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const long long c0 = (chunk + (long long)u * gridDim.x) * UPD_COLS + threadIdx.x * 4;
+            if (c0 >= d) break;
+            float g[4] = {gq[u].x, gq[u].y, gq[u].z, gq[u].w};
+            const float x[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
+            if (apply_topk4(g, x, T, cut, (u32)c0)) *reinterpret_cast<float4*>(G + c0) = make_float4(g[0], g[1], g[2], g[3]);
+          }
+        }
+        return;
+      }
       for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
         const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
         if (c0 >= d) continue;
