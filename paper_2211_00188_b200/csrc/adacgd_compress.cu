@@ -2586,7 +2586,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     }                                                                                                               \
     break;
 #define LIST_PASS(LEVEL, shm, hist)                                                                              \
-  TIMED(KID_LHIST, launch_k(k_lhist<LEVEL>, lgrid, dim3(TPB), shm, stream, pdl, cs, nblk, s.sel, s.list,         \
+  TIMED(KID_LHIST, launch_k(k_lhist<LEVEL>, lhgrid, dim3(TPB), shm, stream, pdl, cs, nblk, s.sel, s.list,         \
                             s.lcount, s.list_row, segcap, hist, s.lepart, s.lepart3, s.rowflag, s.fl, s.flcnt,   \
                             s.cntpart, s.tickets))
 
@@ -2626,6 +2626,9 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (lgx > LIST_BLK) lgx = LIST_BLK;
     if (lgx > nblk) lgx = nblk;
     const dim3 lgrid((unsigned)lgx, rows);
+    // the three-level list passes serve rows with a crowded threshold bin only; their work is the key lists
+    // (about 1 % of a row), so a few CTAs per row do, and the usual launch that finds nothing to do stays short
+    const dim3 lhgrid((unsigned)(lgx < 16 ? lgx : 16), rows);
     TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), (size_t)cs.nsel * FINISH_WORDS * 4, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
                                  s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
                                  cs.nquant == 0 ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
