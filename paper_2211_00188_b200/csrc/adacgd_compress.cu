@@ -95,15 +95,13 @@ __device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
 
 // Finds, in a histogram of nb bins ordered by key, the bin that holds the krem-th
 // largest key: out[0] = bin, out[1] = number of keys in higher bins.  All TPB threads call.
-template <bool SHARED_TABLE = false>
 __device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 krem, u32* out) {
   const int per = nb / TPB;  // 8 or 2
   u32 loc[8];
   u32 sum = 0;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    const u32* src = &hist[nb - 1 - (threadIdx.x * per + k)];
-    loc[k] = (k < per) ? (SHARED_TABLE ? *src : __ldcg(src)) : 0;
+    loc[k] = (k < per) ? __ldcg(&hist[nb - 1 - (threadIdx.x * per + k)]) : 0;
     sum += loc[k];
   }
   u32 excl = block_excl_scan(sum, nullptr);
