@@ -1,6 +1,7 @@
-"""Parity at the benchmark's full size (workload c5: 8 rows of 25e6 entries, the launch
-configuration bench.py times): one sampled worker row and the master row are checked against
-the oracle bit for bit; every other row through properties that hold at any size."""
+"""Parity at the benchmark's full sizes, in the launch configurations bench.py times.  Workload c5
+(8 rows of 25e6 entries): one sampled worker row and the master row are checked against the oracle bit
+for bit, every other row through properties that hold at any size.  Workloads c2, c3, c4: gradients
+of sampled workers against the oracle (rel 1e-5) and the selections of an iteration on sampled rows."""
 import numpy as np
 import pytest
 
@@ -64,3 +65,98 @@ def test_c5_full_size_step():
     mref = O.adacgd(gm_before[0].cpu().numpy(), gt_old.cpu().numpy(), gt_new.cpu().numpy(), W["master"], 1.0)
     assert int(mlevel.item()) == mref["level"]
     assert np.array_equal(gm[0].cpu().numpy().view(np.uint32), mref["out"].view(np.uint32))
+
+
+def relerr(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def check_rows_after_one_step(eng, rows, G_before, Y_before, cands, zeta, recs, levels):
+    """The rows `rows` of a step the engine has just run, against the oracle's compressor fed with the
+    engine's own gradients: level, bits and the updated estimator row, bit for bit."""
+    X = eng.get_state("grad").cpu().numpy()
+    G_after = eng.get_state("G").cpu().numpy()
+    for i in rows:
+        ref = O.adacgd(G_before[i], Y_before[i], X[i], cands, zeta)
+        assert levels[0][i] == ref["level"], (i, levels[0][i], ref["level"])
+        assert np.array_equal(G_after[i].view(np.uint32), ref["out"].view(np.uint32)), i
+    return X, G_after
+
+
+def test_c2_full_size_lockstep():
+    # workload c2 as benchmarked (20 x 8 000, 2 000 samples per worker, bidirectional): two lock-step iterations
+    from test_step_gpu import lockstep
+    import torch
+    W = S.WORKLOADS["c2"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"], iters=8)
+    lockstep(torch, A, t, W["loss"], W["lam"], gamma, W["worker"], 1.0, W["master"], 1.0, T=2)
+
+
+def test_c3_full_size_gradient_and_step():
+    # workload c3 as benchmarked (100 x 100 000, CSR 1 %, 500 samples per worker, Top-K and quantisers mixed)
+    import scipy.sparse as sp
+    import torch
+    import paper_2211_00188_b200 as pkg
+    W = S.WORKLOADS["c3"]
+    n, d, m = W["n"], W["d"], W["m"]
+    rowptr, col, val, y = S.sparse_logistic_problem(n, d, m, density=W["density"], seed=0)
+    dev = torch.device("cuda:0")
+    csr = tuple(torch.from_numpy(a).to(dev) for a in S.csr_global(rowptr, col, val))
+    eng = pkg.AdaCGD(n, d, W["worker"], 1.0, W["master"], 1.0, loss=W["loss"], lam=W["lam"], csr=csr,
+                     target=torch.from_numpy(y).to(dev), x0=torch.zeros(d, device=dev), gamma=0.5 / (0.25 + W["lam"]))
+    sample = [0, 57, 99]
+    prob = dict(A=[sp.csr_matrix((val[i], col[i], rowptr[i]), shape=(m, d)) for i in sample],
+                target=[y[i] for i in sample], loss=W["loss"], lam=W["lam"])
+    x = (0.3 * np.random.Generator(np.random.PCG64(3)).standard_normal(d)).astype(F32)
+    out = torch.zeros(n, d, device=dev)
+    eng.gradient(torch.from_numpy(x).to(dev), out)
+    want = O.all_gradients(prob, x)
+    got = out.cpu().numpy()
+    for k, i in enumerate(sample):
+        assert relerr(got[i], want[k]) <= 1e-5, (i, relerr(got[i], want[k]))
+    # one iteration from the initial state: sampled rows against the oracle's compressor
+    eng.step(3)
+    G_before = eng.get_state("G").cpu().numpy()
+    Y_before = eng.get_state("grad").cpu().numpy()
+    recs, levels = eng.step(1, report=True)
+    check_rows_after_one_step(eng, sample, G_before, Y_before, W["worker"], 1.0, recs, levels)
+    assert eng.get_state("flags") == 0
+
+
+def test_c4_full_size_gradient_and_step():
+    # workload c4 as benchmarked (16 x 1 000 000, 256 samples per worker, 16.4 GB of features drawn on the device)
+    import torch
+    import paper_2211_00188_b200 as pkg
+    W = S.WORKLOADS["c4"]
+    n, d, m = W["n"], W["d"], W["m"]
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    A = torch.empty(n, m, d, device=dev)
+    for i in range(n):
+        A[i] = torch.randn(m, d, generator=gen, device=dev) / d ** 0.5
+    xs = torch.randn(d, generator=gen, device=dev)
+    tgt = torch.einsum("nmd,d->nm", A, xs) + 0.1 * torch.randn(n, m, generator=gen, device=dev)
+    gamma = 0.5 / ((1.0 + (n * m / d) ** 0.5) ** 2 / (n * m))
+    eng = pkg.AdaCGD(n, d, W["worker"], 1.0, W["master"], 1.0, loss=W["loss"], lam=W["lam"], A=A, target=tgt,
+                     x0=torch.zeros(d, device=dev), gamma=gamma)
+    sample = [0, 11]
+    x = (0.5 * np.random.Generator(np.random.PCG64(4)).standard_normal(d)).astype(F32)
+    out = torch.zeros(n, d, device=dev)
+    eng.gradient(torch.from_numpy(x).to(dev), out)
+    for i in sample:
+        want = O.local_gradient(A[i].cpu().numpy(), tgt[i].cpu().numpy(), x, W["loss"], W["lam"])
+        got = out[i].cpu().numpy()
+        assert relerr(got, want) <= 1e-5, (i, relerr(got, want))
+        assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max()
+    del out
+    eng.step(2)
+    G_before = eng.get_state("G").cpu().numpy()
+    Y_before = eng.get_state("grad").cpu().numpy()
+    recs, levels = eng.step(1, report=True)
+    _, G_after = check_rows_after_one_step(eng, sample, G_before, Y_before, W["worker"], 1.0, recs, levels)
+    # the server mean of the full 16 x 1e6 state, bit for bit
+    assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), O.server_mean(G_after).view(np.uint32))
+    assert eng.get_state("flags") == 0
