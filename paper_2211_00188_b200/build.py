@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libadacgd.so")
-SOURCES = ["adacgd_api.cu", "adacgd_compress.cu", "adacgd_gradient.cu"]
+SOURCES = ["adacgd_api.cu", "adacgd_compress.cu", "adacgd_small.cu", "adacgd_noalloc.cu", "adacgd_gradient.cu"]
 
 
 def nvcc_path() -> str:

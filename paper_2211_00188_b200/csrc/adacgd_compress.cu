@@ -13,126 +13,9 @@
 //   - short rows: everything in one CTA per row (k_small_rows).
 // Energies are sums of non-negative exact terms; a comparison whose margin is below the
 // worst-case summation error is redone in exact integer arithmetic.
-#include "adacgd_internal.cuh"
+#include "adacgd_device.cuh"
 
 namespace adacgd {
-
-// --------------------------------------------------------------------------
-// small helpers
-// --------------------------------------------------------------------------
-// Programmatic dependent launch: lets the next kernel of the stream be scheduled while this one
-// runs, then waits until every kernel before this one has completed and its writes are visible.
-// Called first thing by every kernel, before any access to global memory.
-__device__ __forceinline__ void pdl_begin() {
-  asm volatile("griddepcontrol.launch_dependents;");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
-__device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
-
-template <bool ALIGNED>
-__device__ __forceinline__ void load4(const float* __restrict__ row, long long c0, long long d, float (&o)[4]) {
-  if (ALIGNED) {
-    float4 t = *reinterpret_cast<const float4*>(row + c0);
-    o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
-  } else {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) o[k] = (c0 + k < d) ? row[c0 + k] : 0.f;
-  }
-}
-
-template <bool ALIGNED>
-__device__ __forceinline__ void store4(float* __restrict__ row, long long c0, long long d, const float (&o)[4]) {
-  if (ALIGNED) {
-    *reinterpret_cast<float4*>(row + c0) = make_float4(o[0], o[1], o[2], o[3]);
-  } else {
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (c0 + k < d) row[c0 + k] = o[k];
-  }
-}
-
-__device__ __forceinline__ u32 warp_sum_u32(u32 v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-__device__ __forceinline__ double warp_sum_f64(double v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Exclusive prefix sum of one u32 per thread over the CTA (TPB threads); also returns the total.
-__device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
-  __shared__ u32 wsum[TPB / 32];
-  __shared__ u32 wtot;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  u32 inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    u32 t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  __syncthreads();  // protects wsum against the previous call
-  if (lane == 31) wsum[wid] = inc;
-  __syncthreads();
-  if (wid == 0) {
-    u32 w = (lane < TPB / 32) ? wsum[lane] : 0;
-    u32 winc = w;
-#pragma unroll
-    for (int o = 1; o < TPB / 32; o <<= 1) {
-      u32 t = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += t;
-    }
-    if (lane < TPB / 32) wsum[lane] = winc - w;
-    if (lane == TPB / 32 - 1) wtot = winc;
-  }
-  __syncthreads();
-  if (total) *total = wtot;
-  return wsum[wid] + inc - v;
-}
-
-// Finds, in a histogram of nb bins ordered by key, the bin that holds the krem-th
-// largest key: out[0] = bin, out[1] = number of keys in higher bins.  All TPB threads call.
-__device__ void block_find_kth_desc(const u32* __restrict__ hist, int nb, u32 krem, u32* out) {
-  const int per = nb / TPB;  // 8 or 2
-  u32 loc[8];
-  u32 sum = 0;
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    loc[k] = (k < per) ? __ldcg(&hist[nb - 1 - (threadIdx.x * per + k)]) : 0;
-    sum += loc[k];
-  }
-  u32 excl = block_excl_scan(sum, nullptr);
-  if (krem > excl && krem <= excl + sum) {
-    u32 run = excl;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      if (k < per) {
-        if (krem <= run + loc[k]) {
-          out[0] = nb - 1 - (threadIdx.x * per + k);
-          out[1] = run;
-          break;
-        }
-        run += loc[k];
-      }
-    }
-  }
-  __syncthreads();
-}
-
-// True in exactly one CTA of the row: the one that finishes last.  Every CTA calls it after its
-// global writes; the caller may then read what the other CTAs of the row wrote.  No waiting.
-__device__ __forceinline__ bool last_cta_of_row(u32* ticket, u32 n_ctas) {
-  __shared__ u32 is_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == n_ctas - 1u) ? 1u : 0u;
-  __syncthreads();
-  if (is_last) __threadfence();
-  return is_last != 0;
-}
 
 // --------------------------------------------------------------------------
 // radix-select passes
@@ -311,10 +194,6 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
   }
 }
 
-__device__ __forceinline__ float quant_value(float v, float L, float inv, float step) {
-  const float code = fminf(L, rintf(__fmul_rn(fabsf(v), inv)));
-  return copysignf(__fmul_rn(code, step), v);
-}
 
 // slot 2+c for quantiser candidate c: sum (v - Q_c(v))^2 with the row scale s = max|v|.
 template <bool ALIGNED>
@@ -374,155 +253,6 @@ __global__ void __launch_bounds__(TPB) k_quant_err(const float* __restrict__ X, 
   }
 }
 
-// --------------------------------------------------------------------------
-// level choice (Eq. 11)
-// --------------------------------------------------------------------------
-__device__ uint64_t level_bits(const CsetDev& cs, int level, long long d) {
-  if (level == 0) return 0;
-  const int c = level - 1;
-  if (cs.kind[c] == ADACGD_TOPK) {
-    if (cs.param[c] >= d) return 32ull * (uint64_t)d;
-    int idx_bits = 64 - __clzll((unsigned long long)(d - 1));
-    if (d == 1) idx_bits = 1;
-    if (idx_bits < 1) idx_bits = 1;
-    return (uint64_t)cs.param[c] * (uint64_t)(32 + idx_bits);
-  }
-  return 32ull + (uint64_t)cs.param[c] * (uint64_t)d;
-}
-
-// Fills the decision record of a row once its level is known.
-__device__ void finalize_row(const CsetDev& cs, int row, int level, long long d, const SelRow* sel,
-                             const u32* maxkey, RowDec* dec, const CompressOut& out, const double* e,
-                             double D) {
-  RowDec r;
-  r.level = level; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 0;
-  r.qL = r.qinv = r.qstep = 0.f; r.cut = 0xffffffffu;
-  if (level > 0) {
-    const int c = level - 1;
-    if (cs.kind[c] == ADACGD_TOPK) {
-      if (cs.param[c] >= d) {
-        r.mode = 2;
-      } else {
-        int j = 0;
-        for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
-        r.mode = 1; r.T = sel[row].T[j]; r.q = sel[row].q[j];
-        r.need_tie = (sel[row].tiemode[j] == 2u) ? 1 : 0;
-        r.cut = (sel[row].tiemode[j] == 1u) ? sel[row].cut[j] : 0xffffffffu;
-      }
-    } else {
-      r.mode = 3;
-      const float s = __uint_as_float(maxkey[row]);
-      r.qL = (float)((1 << ((int)cs.param[c] - 1)) - 1);
-      if (s > 0.f) { r.qinv = __fdiv_rn(r.qL, s); r.qstep = __fdiv_rn(s, r.qL); }
-    }
-  }
-  dec[row] = r;
-  if (out.level) out.level[row] = level;
-  if (out.bits) out.bits[row] = level_bits(cs, level, d);
-  if (out.D) out.D[row] = D;
-  if (out.err)
-    for (int j = 0; j <= cs.m; ++j) out.err[(long long)row * (cs.m + 1) + j] = e[j];
-}
-
-// Chooses the level of one row from its sums (Eq. 10 and 11); run by a whole CTA of TPB threads.
-// The per-CTA partial sums of the streaming pass are added in a fixed order: thread t takes
-// blocks t, t + TPB, ..., then lanes, then warps.
-__device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, const double* __restrict__ partial,
-                         const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                         RowDec* __restrict__ dec, u32* __restrict__ flags, const CompressOut& out,
-                         const u32* __restrict__ diffflag, double tol) {
-  __shared__ double ps[NSLOT][TPB / 32];
-  __shared__ double p_extra[MAXC];
-  __shared__ u32 p_T[MAXC], p_ntie[MAXC], p_q[MAXC], p_max, p_diff;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int nslot = 2 + cs.m;
-  // what the deciding thread needs from the selection records is fetched by several threads at once
-  if (threadIdx.x < cs.nsel) {
-    const int j = threadIdx.x;
-    p_T[j] = __ldcg(&sel[row].T[j]); p_ntie[j] = __ldcg(&sel[row].ntie[j]);
-    p_q[j] = __ldcg(&sel[row].q[j]); p_extra[j] = __ldcg(&sel[row].extraE[j]);
-  }
-  if (threadIdx.x == 32) { p_max = __ldcg(&maxkey[row]); p_diff = __ldcg(&diffflag[row]); }
-  double a[NSLOT];
-#pragma unroll
-  for (int s = 0; s < NSLOT; ++s) a[s] = 0.0;
-  const double* p = partial + (long long)row * MAX_BLK_PER_ROW * NSLOT;
-  for (int b = threadIdx.x; b < nblk; b += TPB) {
-#pragma unroll
-    for (int s = 0; s < NSLOT; ++s)
-      if (s < nslot) a[s] += __ldcg(&p[(long long)b * NSLOT + s]);
-  }
-#pragma unroll
-  for (int s = 0; s < NSLOT; ++s) {
-    const double v = warp_sum_f64(a[s]);
-    if (lane == 0) ps[s][wid] = v;
-  }
-  __syncthreads();
-  if (threadIdx.x != 0) return;
-  double sum[NSLOT];
-#pragma unroll
-  for (int s = 0; s < NSLOT; ++s) {
-    double t = 0.0;
-    for (int w = 0; w < TPB / 32; ++w) t += ps[s][w];
-    sum[s] = t;
-  }
-  const double D = sum[0];
-  double e[MAXC + 1];
-  e[0] = sum[1];
-  for (int c = 0; c < cs.m; ++c) {
-    if (cs.kind[c] == ADACGD_TOPK) {
-      if (cs.param[c] >= d) { e[c + 1] = 0.0; continue; }
-      int j = 0;
-      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == c) j = t;
-      const double tv = (double)__uint_as_float(p_T[j]);
-      e[c + 1] = (sum[2 + c] + p_extra[j]) + (double)(p_ntie[j] - p_q[j]) * (tv * tv);
-    } else {
-      e[c + 1] = sum[2 + c];
-    }
-  }
-  const u32 diff = p_diff;
-  if (p_max >= 0x7f800000u || (diff & 0x80000000u)) {  // Inf/NaN in X - G or X - Y: estimator kept
-    atomicOr(&flags[0], 1u);
-    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, e, D);
-    return;
-  }
-  // `tol` bounds the relative error of every sum above (non-negative terms).  A sum is only
-  // trusted inside [2^-90, inf): below, binary32 squares may have underflowed; above, a chain
-  // overflowed (or X - Y is not finite, which the exact pass reports).
-  const double tiny = 8.0e-28;
-  const double rhs = (double)cs.zeta * D;
-  const bool d_ok = (D >= tiny && D <= 1.7e308);
-  int level = cs.m;
-  bool unsure = false;
-  for (int j = 0; j <= cs.m; ++j) {
-    const double E = e[j];
-    const bool by_def = (j > 0 && cs.kind[j - 1] == ADACGD_TOPK && cs.param[j - 1] >= d);  // identity: error 0
-    const bool e_ok = (E >= tiny && E <= 1.7e308);
-    int verdict;  // 1 true, 0 false, -1 unsure
-    if (by_def) verdict = 1;
-    else if (!(D <= 1.7e308)) verdict = -1;  // overflowed chain or non-finite X - Y: the exact pass tells which
-    else if (j == 0 && (diff & 0x7fffffffu) == 0 && d_ok)
-      verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
-    else if (!e_ok) verdict = -1;
-    else if (cs.zeta == 0.f) verdict = 0;  // E > 0 for certain, right side is 0
-    else if (!d_ok) verdict = -1;
-    else if (E * (1.0 + tol) < rhs * (1.0 - tol)) verdict = 1;
-    else if (E * (1.0 - tol) > rhs * (1.0 + tol)) verdict = 0;
-    else verdict = -1;
-    if (verdict == 1) { level = j; break; }
-    if (verdict < 0) { unsure = true; break; }
-  }
-  if (unsure) {
-    RowDec r;
-    r.level = -1; r.mode = 0; r.T = 0; r.q = 0; r.need_tie = 0; r.need_exact = 1;
-    r.qL = r.qinv = r.qstep = 0.f; r.cut = 0xffffffffu;
-    dec[row] = r;
-    atomicAdd(&flags[1], 1u);
-    return;
-  }
-  finalize_row(cs, row, level, d, sel, maxkey, dec, out, e, D);
-}
-
 // `picked` (may be null): per-row ticket words; a row whose word 9 is set was already decided.
 __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs, long long d, int nblk_main, int nblk_full,
                                              const u32* __restrict__ rowflag, const double* __restrict__ partial,
@@ -535,92 +265,6 @@ __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs, long long d, int nblk_
   if (picked && picked[row * NTICKET + 9]) return;
   const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
   pick_row(cs, d, row, nblk, partial, sel, maxkey, dec, flags, out, diffflag, tol);
-}
-
-// --------------------------------------------------------------------------
-// exact re-evaluation of a row whose comparison could not be certified
-// --------------------------------------------------------------------------
-// A square of a binary32 value is mant^2 * 2^(2*eff-2) units of 2^-298; it is added as
-// three 32-bit pieces into 64-bit limbs (radix 2^32, carries resolved at the end).
-__device__ __forceinline__ void sq_pieces(float w, int* k, u32 (&p)[3]) {
-  const u32 b = key_of(w);
-  const u32 ex = b >> 23, fr = b & 0x7fffffu;
-  const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
-  const int off = 2 * (int)(ex ? ex : 1u) - 2;
-  const unsigned __int128 t = (unsigned __int128)(m * m) << (off & 31);
-  *k = off >> 5;
-  p[0] = (u32)t; p[1] = (u32)(t >> 32); p[2] = (u32)(t >> 64);
-}
-__device__ __forceinline__ void limb_add(u64* limbs, int k, const u32 (&p)[3]) {
-  if (p[0]) atomicAdd(&limbs[k], (u64)p[0]);
-  if (p[1]) atomicAdd(&limbs[k + 1], (u64)p[1]);
-  if (p[2]) atomicAdd(&limbs[k + 2], (u64)p[2]);
-}
-
-// Normalised radix-2^32 digits -> nearest binary64 (ties to even); value = digits * 2^-298.
-__device__ double digits_to_double(const u32* dig) {
-  int t = NLIMB - 1;
-  while (t >= 0 && dig[t] == 0) --t;
-  if (t < 0) return 0.0;
-  const u32 hi = dig[t], mid = (t >= 1) ? dig[t - 1] : 0u, lo = (t >= 2) ? dig[t - 2] : 0u;
-  bool sticky = false;
-  for (int i = 0; i < t - 2; ++i) sticky |= (dig[i] != 0);
-  const unsigned __int128 W = ((unsigned __int128)hi << 64) | ((unsigned __int128)mid << 32) | lo;
-  const int nb = 32 - __clz(hi);         // significant bits of hi
-  const int sh = nb + 11;                // keep 53 of the 64+nb bits
-  u64 mant = (u64)(W >> sh);
-  const bool rnd = (W >> (sh - 1)) & 1;
-  sticky |= (W & (((unsigned __int128)1 << (sh - 1)) - 1)) != 0;
-  if (rnd && (sticky || (mant & 1))) ++mant;
-  return ldexp((double)mant, sh + 32 * (t - 2) - 298);
-}
-
-// Run by one thread of the last CTA of the exact pass: carries, rounds and decides the row.
-// `row_limbs`: the row's NSLOT x NLIMB accumulators, in global memory or (SHARED_LIMBS) in shared memory.
-template <bool SHARED_LIMBS = false>
-__device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* row_limbs,
-                               const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                               RowDec* __restrict__ dec, const CompressOut& out,
-                               const u32* __restrict__ diffflag, u32* __restrict__ flags) {
-  double val[NSLOT];
-  if (__ldcg(&diffflag[row]) & 0x80000000u) {  // X - Y is not finite
-    for (int s = 0; s < NSLOT; ++s) val[s] = 0.0;
-    atomicOr(&flags[0], 1u);
-    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, val + 1, 0.0);
-    return;
-  }
-  for (int s = 0; s < 2 + cs.m; ++s) {
-    u32 dig[NLIMB];
-    const u64* l = row_limbs + s * NLIMB;
-    unsigned __int128 tie = 0;
-    int tk = 0;
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
-      int j = 0;
-      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
-      const u32 T = sel[row].T[j];
-      const u32 ex = T >> 23, fr = T & 0x7fffffu;
-      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
-      const int off = 2 * (int)(ex ? ex : 1u) - 2;
-      tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
-      tk = off >> 5;
-    }
-    u64 carry = 0;
-    for (int k = 0; k < NLIMB; ++k) {
-      u64 add = 0;
-      if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
-      const unsigned __int128 tsum = (unsigned __int128)(SHARED_LIMBS ? l[k] : __ldcg(&l[k])) + carry + add;
-      dig[k] = (u32)tsum;
-      carry = (u64)(tsum >> 32);
-    }
-    val[s] = digits_to_double(dig);
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) val[s] = 0.0;
-  }
-  const double D = val[0];
-  const double rhs = (double)cs.zeta * D;
-  int level = cs.m;
-  for (int j = 0; j <= cs.m; ++j)
-    if (val[1 + j] <= rhs) { level = j; break; }
-  finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
 }
 
 template <bool ALIGNED>
@@ -1922,404 +1566,6 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
 }
 
 // --------------------------------------------------------------------------
-// short rows: stages a2-a4 and the mean in one launch
-// --------------------------------------------------------------------------
-// One CTA per row, the row's difference vector v = X - G kept in shared memory: three radix passes
-// (11 + 11 + 9 bits, all Top-K candidates at once), tail energies and quantiser errors in binary64,
-// the index cut of threshold-equal keys, the level choice (pick_row, with the exact integer sums
-// when a comparison cannot be certified) and the update of the row; the mean over the rows follows in
-// k_small_mean.  Serves problems too small to keep the multi-kernel path busy.
-// Finds, in a shared-memory histogram of nb bins (a multiple of 32) ordered by key, the bin that holds
-// the krem-th largest key; one warp calls, every lane gets (bin, number of keys in higher bins).
-__device__ __forceinline__ void warp_find_kth_desc(const u32* hist, int nb, u32 krem, u32* bin, u32* above) {
-  const int lane = threadIdx.x & 31;
-  const int per = nb / 32;                              // this lane: descending positions per*lane .. per*lane + per - 1
-  u32 sum = 0;
-  for (int k = 0; k < per; ++k) sum += hist[nb - 1 - (per * lane + k)];
-  u32 inc = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  const u32 excl = inc - sum;
-  const bool mine = krem > excl && krem <= excl + sum;   // true in exactly one lane when 1 <= krem <= total
-  u32 fb = 0, fa = 0;
-  if (mine) {
-    u32 run = excl;
-    for (int k = 0; k < per; ++k) {
-      const u32 v = hist[nb - 1 - (per * lane + k)];
-      if (krem <= run + v) { fb = (u32)(nb - 1 - (per * lane + k)); fa = run; break; }
-      run += v;
-    }
-  }
-  const u32 who = __ballot_sync(0xffffffffu, mine);
-  const int src = who ? (__ffs(who) - 1) : 0;
-  *bin = __shfl_sync(0xffffffffu, fb, src);
-  *above = __shfl_sync(0xffffffffu, fa, src);
-}
-
-constexpr int SMALL_DMAX = 32768;
-template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
-                                                    int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
-                                                    double* partial, u32* maxkey, u32* diffflag, u32* flags,
-                                                    CompressOut out, double tol) {
-  pdl_begin();
-  extern __shared__ __align__(16) unsigned char small_smem[];
-  const int dn = (int)d;
-  float* vs = reinterpret_cast<float*>(small_smem);                       // [d rounded up to 4]
-  u32* tab = reinterpret_cast<u32*>(small_smem) + ((dn + 3) / 4) * 4;     // max(BINS1, nsel * BINS2) words
-  __shared__ double redd[NSLOT][TPB / 32];
-  __shared__ u32 redu[3][TPB / 32];
-  __shared__ u32 s_b1[MAXC], s_ab1[MAXC], s_p2[MAXC], s_ab2[MAXC], s_T[MAXC], s_above[MAXC], s_ntie[MAXC], s_q[MAXC], s_cut[MAXC];
-  __shared__ u64 lsh[NSLOT * NLIMB];
-  const int row = blockIdx.x;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int nsel = cs.nsel;
-  const float* xr = X + (long long)row * d;
-  float* gr = G + (long long)row * d;
-  const float* yr = Y + (long long)row * d;
-
-  // ---- v into shared memory; D, ||v||^2, row maximum, |X-G| against |X-Y|
-  double aD = 0.0, aE = 0.0;
-  u32 mx = 0, mxw = 0, dfl = 0;
-  constexpr int SB = 4;   // tiles of TPB * 4 columns requested at once: the row is short, its latency is what counts
-  for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
-    float x[SB][4], g[SB][4], y[SB][4];
-#pragma unroll
-    for (int u = 0; u < SB; ++u) {
-      const int c0 = base + u * TPB * 4;
-      if (c0 < dn) {
-        load4<ALIGNED>(xr, c0, d, x[u]);
-        load4<ALIGNED>(gr, c0, d, g[u]);
-        load4<ALIGNED>(yr, c0, d, y[u]);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < SB; ++u) {
-      const int c0 = base + u * TPB * 4;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (c0 + k >= dn) break;
-        const float v = __fsub_rn(x[u][k], g[u][k]);
-        const float w = __fsub_rn(x[u][k], y[u][k]);
-        vs[c0 + k] = v;
-        const double dv = (double)v, dw = (double)w;
-        aD = __dadd_rn(aD, __dmul_rn(dw, dw));
-        aE = __dadd_rn(aE, __dmul_rn(dv, dv));
-        mx = max(mx, key_of(v));
-        mxw = max(mxw, key_of(w));
-        dfl |= __float_as_uint(v) ^ __float_as_uint(w);
-      }
-    }
-  }
-  aD = warp_sum_f64(aD); aE = warp_sum_f64(aE);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    mxw = max(mxw, __shfl_xor_sync(0xffffffffu, mxw, o));
-    dfl |= __shfl_xor_sync(0xffffffffu, dfl, o);
-  }
-  if (lane == 0) { redd[0][wid] = aD; redd[1][wid] = aE; redu[0][wid] = mx; redu[1][wid] = mxw; redu[2][wid] = dfl; }
-  __syncthreads();
-  mx = 0; mxw = 0; dfl = 0;
-  for (int w = 0; w < TPB / 32; ++w) { mx = max(mx, redu[0][w]); mxw = max(mxw, redu[1][w]); dfl |= redu[2][w]; }
-  const float smax = __uint_as_float(mx);
-
-  // ---- radix select, all candidates at once
-  if (nsel) {
-    for (int i = threadIdx.x; i < BINS1; i += TPB) tab[i] = 0;
-    __syncthreads();
-    for (int i = threadIdx.x; i < dn; i += TPB) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
-    __syncthreads();
-    if (wid < nsel) {   // one warp per candidate
-      u32 bin, above;
-      warp_find_kth_desc(tab, BINS1, (u32)cs.param[cs.sel[wid]], &bin, &above);
-      if (lane == 0) { s_b1[wid] = bin; s_ab1[wid] = above; }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < nsel * BINS2; i += TPB) tab[i] = 0;
-    __syncthreads();
-    for (int i = threadIdx.x; i < dn; i += TPB) {
-      const u32 key = key_of(vs[i]);
-      for (int j = 0; j < nsel; ++j)
-        if ((key >> 20) == s_b1[j]) atomicAdd(&tab[j * BINS2 + ((key >> 9) & 0x7ffu)], 1u);
-    }
-    __syncthreads();
-    if (wid < nsel) {
-      u32 bin, above;
-      warp_find_kth_desc(tab + wid * BINS2, BINS2, (u32)cs.param[cs.sel[wid]] - s_ab1[wid], &bin, &above);
-      if (lane == 0) { s_p2[wid] = (s_b1[wid] << 11) | bin; s_ab2[wid] = s_ab1[wid] + above; }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < nsel * BINS3; i += TPB) tab[i] = 0;
-    __syncthreads();
-    for (int i = threadIdx.x; i < dn; i += TPB) {
-      const u32 key = key_of(vs[i]);
-      for (int j = 0; j < nsel; ++j)
-        if ((key >> 9) == s_p2[j]) atomicAdd(&tab[j * BINS3 + (key & 0x1ffu)], 1u);
-    }
-    __syncthreads();
-    if (wid < nsel) {
-      const int j = wid;
-      const u32 K = (u32)cs.param[cs.sel[j]];
-      u32 bin, above;
-      warp_find_kth_desc(tab + j * BINS3, BINS3, K - s_ab2[j], &bin, &above);
-      if (lane == 0) {
-        s_T[j] = (s_p2[j] << 9) | bin;
-        s_above[j] = s_ab2[j] + above;
-        s_ntie[j] = tab[j * BINS3 + bin];
-        s_q[j] = K - s_above[j];
-        s_cut[j] = 0xffffffffu;
-      }
-    }
-    __syncthreads();
-    // of the keys equal to a threshold the q with the lowest indices are kept: index of the q-th
-    for (int j = 0; j < nsel; ++j) {
-      if (s_q[j] >= s_ntie[j]) continue;
-      const u32 T = s_T[j], q = s_q[j];
-      const int per = (dn + TPB - 1) / TPB;
-      const int i0 = threadIdx.x * per, i1 = (i0 + per < dn) ? i0 + per : dn;
-      u32 cnt = 0;
-      for (int i = i0; i < i1; ++i) cnt += (key_of(vs[i]) == T) ? 1u : 0u;
-      const u32 ex = block_excl_scan(cnt, nullptr);
-      if (ex < q && q <= ex + cnt) {
-        u32 seen = ex;
-        for (int i = i0; i < i1; ++i)
-          if (key_of(vs[i]) == T && ++seen == q) { s_cut[j] = (u32)i; break; }
-      }
-      __syncthreads();
-    }
-  }
-
-  // ---- tail energies of the Top-K candidates, errors of the quantisers (binary64, exact terms)
-  double aB[MAXC], aQ[MAXC];
-  float qL[MAXC], qinv[MAXC], qstep[MAXC];
-#pragma unroll
-  for (int j = 0; j < MAXC; ++j) {
-    aB[j] = 0.0; aQ[j] = 0.0; qL[j] = qinv[j] = qstep[j] = 0.f;
-    if (j < cs.nquant) {
-      qL[j] = (float)((1 << ((int)cs.param[cs.qsel[j]] - 1)) - 1);
-      if (smax > 0.f) { qinv[j] = __fdiv_rn(qL[j], smax); qstep[j] = __fdiv_rn(smax, qL[j]); }
-    }
-  }
-  for (int i = threadIdx.x; i < dn; i += TPB) {
-    const float v = vs[i];
-    const u32 key = key_of(v);
-    const double dv = (double)v;
-    const double sq = __dmul_rn(dv, dv);
-#pragma unroll
-    for (int j = 0; j < MAXC; ++j) {
-      if (j < nsel && key < s_T[j]) aB[j] = __dadd_rn(aB[j], sq);
-      if (j < cs.nquant) {
-        const double r = (double)__fsub_rn(v, quant_value(v, qL[j], qinv[j], qstep[j]));
-        aQ[j] = __dadd_rn(aQ[j], __dmul_rn(r, r));
-      }
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < MAXC; ++j) {
-    if (j < nsel) { const double t = warp_sum_f64(aB[j]); if (lane == 0) redd[2 + cs.sel[j]][wid] = t; }
-    if (j < cs.nquant) { const double t = warp_sum_f64(aQ[j]); if (lane == 0) redd[2 + cs.qsel[j]][wid] = t; }
-  }
-  __syncthreads();
-  // ---- the row's records, in the form the level choice reads them
-  if (threadIdx.x < NSLOT) {
-    const int sl = threadIdx.x;
-    bool used = (sl < 2);
-    for (int j = 0; j < nsel; ++j) used |= (sl == 2 + cs.sel[j]);
-    for (int j = 0; j < cs.nquant; ++j) used |= (sl == 2 + cs.qsel[j]);
-    double acc = 0.0;
-    if (used)
-      for (int w = 0; w < TPB / 32; ++w) acc += redd[sl][w];
-    partial[(long long)row * MAX_BLK_PER_ROW * NSLOT + sl] = acc;
-  }
-  if (threadIdx.x >= 32 && threadIdx.x < 32 + nsel) {
-    const int j = threadIdx.x - 32;
-    SelRow* sr = sel + row;
-    sr->T[j] = s_T[j]; sr->above[j] = s_above[j]; sr->ntie[j] = s_ntie[j]; sr->q[j] = s_q[j];
-    sr->extraE[j] = 0.0; sr->tiemode[j] = (s_q[j] < s_ntie[j]) ? 1u : 0u; sr->cut[j] = s_cut[j];
-  }
-  if (threadIdx.x == 64) {
-    maxkey[row] = mx;
-    diffflag[row] = ((mxw >= 0x7f800000u) ? 0x80000000u : 0u) | (dfl & 0x7fffffffu);
-  }
-  __syncthreads();
-  pick_row(cs, d, row, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
-  __syncthreads();
-  if (__ldcg(&dec[row].need_exact)) {
-    // the comparison could not be certified: exact integer sums of the row, then the decision from them
-    for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) lsh[i] = 0;
-    __syncthreads();
-    // A square is mant^2 * 2^off units of 2^-298.  Squares whose offset lies within 64 bits below the
-    // largest one of the row are added in per-thread 128-bit integers anchored at bit `wb` (at most 128
-    // terms of at most 113 bits each); the few that lie lower go straight to the shared limbs.
-    const u32 kmax = max(mx, mxw);
-    const int off_max = 2 * (int)((kmax >> 23) ? (kmax >> 23) : 1u) - 2;
-    const int wb = off_max > 64 ? off_max - 64 : 0;
-    unsigned __int128 accD = 0, accE = 0, accC[MAXC];
-#pragma unroll
-    for (int c = 0; c < MAXC; ++c) accC[c] = 0;
-    // square of a finite value as a 128-bit integer anchored at bit wb; false if it lies below the window
-    auto sq_term = [&](float val, unsigned __int128* term) -> bool {
-      const u32 bkey = key_of(val);
-      const u32 ex = bkey >> 23, fr = bkey & 0x7fffffu;
-      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
-      const int off = 2 * (int)(ex ? ex : 1u) - 2;
-      *term = (off >= wb) ? (unsigned __int128)(m * m) << (off - wb) : (unsigned __int128)0;
-      return off >= wb || m == 0;
-    };
-    auto slow_add = [&](int slot, float val) {   // rare: more than 2^32 times smaller than the row's largest entry
-      int kk; u32 p[3];
-      sq_pieces(val, &kk, p);
-      limb_add(lsh + slot * NLIMB, kk, p);
-    };
-    for (int i = threadIdx.x; i < dn; i += TPB) {
-      const float v = vs[i];
-      const float w = __fsub_rn(xr[i], yr[i]);
-      if (key_of(w) >= 0x7f800000u || key_of(v) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
-      unsigned __int128 tw, tv;
-      if (sq_term(w, &tw)) accD += tw; else slow_add(0, w);
-      const bool v_in = sq_term(v, &tv);
-      if (v_in) accE += tv; else slow_add(1, v);
-      const u32 key = key_of(v);
-#pragma unroll
-      for (int j = 0; j < MAXC; ++j)
-        if (j < nsel && key < s_T[j] && v_in) accC[j] += tv;
-      if (!v_in)
-        for (int j = 0; j < nsel; ++j)
-          if (key < s_T[j]) slow_add(2 + cs.sel[j], v);
-      for (int j = 0; j < cs.nquant; ++j) {
-        const float r = __fsub_rn(v, quant_value(v, qL[j], qinv[j], qstep[j]));
-        unsigned __int128 tr;
-        if (sq_term(r, &tr)) {
-#pragma unroll
-          for (int c = 0; c < MAXC; ++c)
-            if (c == MAXC - 1 - j) accC[c] += tr;
-        } else slow_add(2 + cs.qsel[j], r);
-      }
-    }
-    // The per-thread integers are added up as four 32-bit pieces each: over the warp with shuffles, over the
-    // warps through `wacc` (64-bit shared atomics are compare-and-swap loops: with every thread of the CTA on
-    // the same few words they would take hundreds of microseconds), and only the totals go into the limbs.
-    __shared__ u64 wacc[TPB / 32][NSLOT][4];
-    auto stash = [&](unsigned __int128 acc, int slot) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        u64 piece = (u64)(u32)(acc >> (32 * i));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) piece += __shfl_xor_sync(0xffffffffu, piece, o);
-        if (lane == 0) wacc[wid][slot][i] = piece;
-      }
-    };
-    for (int i = threadIdx.x; i < (TPB / 32) * NSLOT * 4; i += TPB) (&wacc[0][0][0])[i] = 0;
-    __syncthreads();
-    stash(accD, 0);
-    stash(accE, 1);
-#pragma unroll
-    for (int j = 0; j < MAXC; ++j) {
-      if (j < nsel) stash(accC[j], 2 + cs.sel[j]);
-      if (j < cs.nquant) stash(accC[MAXC - 1 - j], 2 + cs.qsel[j]);
-    }
-    __syncthreads();
-    if (threadIdx.x < NSLOT * 4) {
-      const int slot = threadIdx.x >> 2, i = threadIdx.x & 3;
-      u64 tot = 0;                                     // < 2^32 * 256 threads = 2^40
-      for (int w = 0; w < TPB / 32; ++w) tot += wacc[w][slot][i];
-      const int k0 = (wb >> 5) + i, sh = wb & 31;
-      const u64 lo = (tot & 0xffffffffull) << sh, hi = (tot >> 32) << sh;      // weights 2^(32 k0) and 2^(32 (k0 + 1))
-      if (lo & 0xffffffffull) atomicAdd(&lsh[slot * NLIMB + k0], lo & 0xffffffffull);
-      if ((lo >> 32) + (hi & 0xffffffffull)) atomicAdd(&lsh[slot * NLIMB + k0 + 1], (lo >> 32) + (hi & 0xffffffffull));
-      if (hi >> 32) atomicAdd(&lsh[slot * NLIMB + k0 + 2], hi >> 32);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) pick_exact_row<true>(cs, row, d, lsh, sel, maxkey, dec, out, diffflag, flags);
-    __syncthreads();
-  }
-
-  // ---- the update of the row (Eq. 7 at the chosen level)
-  const int mode = __ldcg(&dec[row].mode);
-  if (mode != 0) {
-    const u32 T = __ldcg(&dec[row].T), cut = __ldcg(&dec[row].cut);
-    const float L = __ldcg(&dec[row].qL), inv = __ldcg(&dec[row].qinv), step = __ldcg(&dec[row].qstep);
-    for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
-      float gq[SB][4];
-#pragma unroll
-      for (int u = 0; u < SB; ++u)
-        if (base + u * TPB * 4 < dn) load4<ALIGNED>(gr, base + u * TPB * 4, d, gq[u]);
-#pragma unroll
-      for (int u = 0; u < SB; ++u) {
-        const int c0 = base + u * TPB * 4;
-        if (c0 >= dn) break;
-        bool any = false;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (c0 + k >= dn) break;
-          const float v = vs[c0 + k];
-          const u32 key = key_of(v);
-          bool kept = true;
-          float add = v;
-          if (mode == 1) kept = (key > T) || (key == T && (u32)(c0 + k) <= cut);
-          else if (mode == 3) add = quant_value(v, L, inv, step);
-          if (kept) {
-            gq[u][k] = __fadd_rn(gq[u][k], add);
-            any = true;
-            if (out.kept_idx && mode != 3) {
-              const long long pos = (long long)atomicAdd((u64*)&out.kept_cnt[row], 1ull);
-              if (pos < out.kept_stride) out.kept_idx[(long long)row * out.kept_stride + pos] = c0 + k;
-            }
-          }
-        }
-        if (any) store4<ALIGNED>(gr, c0, d, gq[u]);
-      }
-    }
-  }
-
-}
-
-// The mean over short rows (summed in row order, one division): a thread owns four columns and
-// requests eight rows at once.
-template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_small_mean(const float* G, int rows, long long d, float* __restrict__ mean_out) {
-  pdl_begin();
-  const int dn = (int)d;
-  const int c0 = (blockIdx.x * TPB + threadIdx.x) * 4;
-  if (c0 >= dn) return;
-  const float nf = (float)rows;
-  float acc[4] = {-0.f, -0.f, -0.f, -0.f};
-  for (int i0 = 0; i0 < rows; i0 += 8) {
-    float g[8][4];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int i = i0 + u;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) g[u][k] = 0.f;
-      if (i < rows) {
-        const float* src = G + (long long)i * d + c0;
-        if (ALIGNED) {
-          const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
-          g[u][0] = t.x; g[u][1] = t.y; g[u][2] = t.z; g[u][3] = t.w;
-        } else {
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if (c0 + k < dn) g[u][k] = __ldcg(src + k);
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      if (i0 + u >= rows) break;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) acc[k] = __fadd_rn(acc[k], g[u][k]);
-    }
-  }
-#pragma unroll
-  for (int k = 0; k < 4; ++k)
-    if (c0 + k < dn) mean_out[c0 + k] = __fdiv_rn(acc[k], nf);
-}
-
-// --------------------------------------------------------------------------
 // host side
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -2458,22 +1704,6 @@ adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const 
   return ADACGD_OK;
 }
 
-static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
-
-// Launches a kernel, optionally as a programmatic dependent of the kernel before it on the stream:
-// its CTAs may be scheduled before that kernel has finished and wait in pdl_begin().
-template <typename... KArgs, typename... Args>
-static void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t shm, cudaStream_t stream, bool pdl,
-                     Args&&... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = shm; cfg.stream = stream;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = pdl ? 1 : 0;
-  cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
-}
-
 int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
                     long long d, const CompressOut& out, cudaStream_t stream) {
   int launches = 0;
@@ -2484,8 +1714,6 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
     cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
     cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
-    cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
-    cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
     cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
     attr_done = true;
@@ -2525,26 +1753,9 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   prof_end(pf, stream);
 
   if (!single && d <= SMALL_DMAX) {
-    // short rows: everything in one launch, one CTA per row
-    const size_t shm = 4 * ((size_t)((d + 3) / 4) * 4 + (size_t)(cs.nsel > 1 ? cs.nsel : 1) * BINS2);
-    const double tol64 = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
-    const bool al4 = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y);
-    prof_begin(pf, KID_SMALL, stream);
-    if (al4) launch_k(k_small_rows<true>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                      s.maxkey, s.diffflag, s.flags, out, tol64);
-    else launch_k(k_small_rows<false>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                  s.maxkey, s.diffflag, s.flags, out, tol64);
-    prof_end(pf, stream);
-    ++launches;
-    if (out.mean_out) {
-      const dim3 mgrid((unsigned)((d + TPB * 4 - 1) / (TPB * 4)));
-      prof_begin(pf, KID_SMALL, stream);
-      if (al4 && aligned16(out.mean_out)) launch_k(k_small_mean<true>, mgrid, dim3(TPB), 0, stream, pdl, (const float*)G, rows, d, out.mean_out);
-      else launch_k(k_small_mean<false>, mgrid, dim3(TPB), 0, stream, pdl, (const float*)G, rows, d, out.mean_out);
-      prof_end(pf, stream);
-      ++launches;
-    }
-    return cudaGetLastError() == cudaSuccess ? launches : -1;
+    // short rows: everything in one launch, one CTA per row, then the mean
+    const int n = launch_small_rows(s, cs, X, G, Y, rows, d, out, stream, pdl);
+    return n < 0 ? -1 : launches + n;
   }
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
@@ -2696,87 +1907,3 @@ int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStre
 }
 
 }  // namespace adacgd
-
-// --------------------------------------------------------------------------
-// compression without any device allocation
-// --------------------------------------------------------------------------
-namespace adacgd {
-
-// Scratch of adacgd_compress_noalloc.  It is part of the library image: every GPU that
-// loads libadacgd holds these 2 MiB until the process exits, whether or not the entry
-// point is ever called.
-constexpr size_t NOALLOC_SCRATCH_BYTES = 2u << 20;
-static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
-
-constexpr int NOALLOC_MAX_DEVICES = 64;
-static void* g_noalloc_base[NOALLOC_MAX_DEVICES] = {nullptr};
-
-// In host code `g_noalloc_scratch` is only a handle; the address a kernel may use has to be
-// asked for, per device, with that device current.
-static adacgd_status noalloc_base(void** base) {
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) {
-    set_thread_error("adacgd_compress_noalloc: no current CUDA device (or device ordinal above 63)");
-    return ADACGD_ERR_CUDA;
-  }
-  if (!g_noalloc_base[dev]) {
-    void* p = nullptr;
-    const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-    if (e != cudaSuccess || !p) {
-      set_thread_error("adacgd_compress_noalloc: cudaGetSymbolAddress failed for the built-in scratch");
-      return ADACGD_ERR_CUDA;
-    }
-    g_noalloc_base[dev] = p;
-  }
-  *base = g_noalloc_base[dev];
-  return ADACGD_OK;
-}
-
-}  // namespace adacgd
-
-extern "C" adacgd_status adacgd_compress_noalloc(const float* X_dev, float* G_dev, const float* Y_dev,
-                                                 int32_t rows, int64_t d, const adacgd_cset* cset,
-                                                 float* mean_out_dev, int32_t* level_dev, uint64_t* bits_dev,
-                                                 void* cuda_stream) {
-  using namespace adacgd;
-  if (!X_dev || !G_dev || !Y_dev) {
-    set_thread_error("adacgd_compress_noalloc: X, G, Y must be non-NULL");
-    return ADACGD_ERR_INVALID_ARG;
-  }
-  if (rows < 1 || rows > ADACGD_NOALLOC_MAX_ROWS || d < 1 || d > ADACGD_NOALLOC_MAX_D ||
-      scratch_bytes(rows, d, false) > NOALLOC_SCRATCH_BYTES) {
-    set_thread_error("adacgd_compress_noalloc: shape exceeds the built-in scratch "
-                     "(rows <= ADACGD_NOALLOC_MAX_ROWS = 4, d <= ADACGD_NOALLOC_MAX_D = 4194304); "
-                     "use adacgd_init + adacgd_compress with a caller-owned workspace");
-    return ADACGD_ERR_INVALID_ARG;
-  }
-  const char* msg = "";
-  CsetDev cs;
-  const adacgd_status st = make_cset(cset, d, &cs, &msg);
-  if (st != ADACGD_OK) {
-    set_thread_error(msg);
-    return st;
-  }
-  void* base = nullptr;
-  const adacgd_status sb = noalloc_base(&base);
-  if (sb != ADACGD_OK) return sb;
-  Scratch s;
-  carve_scratch(&s, base, rows, d, false);
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
-  // the array keeps whatever the previous call left: the status words start from zero here,
-  // the histograms and accumulators are cleared by launch_compress itself
-  if (cudaMemsetAsync(s.flags, 0, 16, stream) != cudaSuccess) {
-    set_thread_error("adacgd_compress_noalloc: cudaMemsetAsync failed");
-    return ADACGD_ERR_CUDA;
-  }
-  CompressOut o;
-  memset(&o, 0, sizeof(o));
-  o.mean_out = mean_out_dev;
-  o.level = level_dev;
-  o.bits = bits_dev;
-  if (launch_compress(s, cs, X_dev, G_dev, Y_dev, rows, d, o, stream) < 0) {
-    set_thread_error("adacgd_compress_noalloc: kernel launch failed");
-    return ADACGD_ERR_CUDA;
-  }
-  return ADACGD_OK;
-}

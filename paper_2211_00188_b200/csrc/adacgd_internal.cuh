@@ -140,6 +140,11 @@ struct CompressOut {
 int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y,
                     int rows, long long d, const CompressOut& out, cudaStream_t stream);
 
+// Short rows (d <= SMALL_DMAX): stages a2-a4 in one launch, one CTA per row, then the mean.
+constexpr int SMALL_DMAX = 32768;
+int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
+                      long long d, const CompressOut& out, cudaStream_t stream, bool pdl);
+
 // ---- gradient stage (a1) ----
 struct GradScratch {
   float* r;         // [n][m_rows] residuals scaled by 1/m
