@@ -41,6 +41,7 @@ __device__ __forceinline__ void warp_find_kth_desc(const u32* hist, int nb, u32 
   *above = __shfl_sync(0xffffffffu, fa, src);
 }
 
+constexpr int SMALL_LIST = 4096;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
                                                     int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
@@ -51,10 +52,12 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   const int dn = (int)d;
   float* vs = reinterpret_cast<float*>(small_smem);                       // [d rounded up to 4]
   u32* tab = reinterpret_cast<u32*>(small_smem) + ((dn + 3) / 4) * 4;     // max(BINS1, nsel * BINS2) words
+  u32* cl = tab + (cs.nsel > 1 ? cs.nsel : 1) * BINS2;                           // SMALL_LIST keys sharing a first digit with a threshold
   __shared__ double redd[NSLOT][TPB / 32];
   __shared__ u32 redu[3][TPB / 32];
   __shared__ u32 s_b1[MAXC], s_ab1[MAXC], s_p2[MAXC], s_ab2[MAXC], s_T[MAXC], s_above[MAXC], s_ntie[MAXC], s_q[MAXC], s_cut[MAXC];
   __shared__ u64 lsh[NSLOT * NLIMB];
+  __shared__ u32 s_ncl;
   const int row = blockIdx.x;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int nsel = cs.nsel;
@@ -112,6 +115,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   if (nsel) {
     for (int i = threadIdx.x; i < BINS1; i += TPB) tab[i] = 0;
     __syncthreads();
+#pragma unroll 4
     for (int i = threadIdx.x; i < dn; i += TPB) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
     __syncthreads();
     if (wid < nsel) {   // one warp per candidate
@@ -120,10 +124,32 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       if (lane == 0) { s_b1[wid] = bin; s_ab1[wid] = above; }
     }
     __syncthreads();
+    // The keys that share a first digit with some threshold (usually a few per cent of the row) are
+    // compacted once, with warp votes; the second and third digit are then histogrammed from that list.
+    // A list that does not fit sends the two passes over the whole row instead.
     for (int i = threadIdx.x; i < nsel * BINS2; i += TPB) tab[i] = 0;
+    if (threadIdx.x == 0) s_ncl = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < dn; i += TPB) {
-      const u32 key = key_of(vs[i]);
+    for (int i0 = 0; i0 < dn; i0 += TPB) {
+      const int i = i0 + threadIdx.x;
+      const u32 key = (i < dn) ? key_of(vs[i]) : 0xffffffffu;
+      bool hit = false;
+      for (int j = 0; j < nsel; ++j) hit = hit || ((key >> 20) == s_b1[j]);
+      const u32 m = __ballot_sync(0xffffffffu, hit);
+      if (m) {
+        u32 base = 0;
+        if (lane == 0) base = atomicAdd(&s_ncl, (u32)__popc(m));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        const u32 pos = base + (u32)__popc(m & ((1u << lane) - 1u));
+        if (hit && pos < (u32)SMALL_LIST) cl[pos] = key;
+      }
+    }
+    __syncthreads();
+    const u32 ncl = s_ncl;
+    const bool listed = ncl <= (u32)SMALL_LIST;
+    const int nscan = listed ? (int)ncl : dn;
+    for (int i = threadIdx.x; i < nscan; i += TPB) {
+      const u32 key = listed ? cl[i] : key_of(vs[i]);
       for (int j = 0; j < nsel; ++j)
         if ((key >> 20) == s_b1[j]) atomicAdd(&tab[j * BINS2 + ((key >> 9) & 0x7ffu)], 1u);
     }
@@ -136,8 +162,8 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     __syncthreads();
     for (int i = threadIdx.x; i < nsel * BINS3; i += TPB) tab[i] = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < dn; i += TPB) {
-      const u32 key = key_of(vs[i]);
+    for (int i = threadIdx.x; i < nscan; i += TPB) {
+      const u32 key = listed ? cl[i] : key_of(vs[i]);
       for (int j = 0; j < nsel; ++j)
         if ((key >> 9) == s_p2[j]) atomicAdd(&tab[j * BINS3 + (key & 0x1ffu)], 1u);
     }
@@ -185,6 +211,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       if (smax > 0.f) { qinv[j] = __fdiv_rn(qL[j], smax); qstep[j] = __fdiv_rn(smax, qL[j]); }
     }
   }
+#pragma unroll 2
   for (int i = threadIdx.x; i < dn; i += TPB) {
     const float v = vs[i];
     const u32 key = key_of(v);
@@ -406,13 +433,13 @@ int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float
                       long long d, const CompressOut& out, cudaStream_t stream, bool pdl) {
   static bool attr_done = false;
   if (!attr_done) {  // the row and the tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory
-    cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
-    cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2));
+    cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
+    cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
     attr_done = true;
   }
   Prof* pf = s.prof;
   int launches = 0;
-  const size_t shm = 4 * ((size_t)((d + 3) / 4) * 4 + (size_t)(cs.nsel > 1 ? cs.nsel : 1) * BINS2);
+  const size_t shm = 4 * ((size_t)((d + 3) / 4) * 4 + (size_t)(cs.nsel > 1 ? cs.nsel : 1) * BINS2 + SMALL_LIST);
   const double tol64 = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
   const bool al4 = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y);
   prof_begin(pf, KID_SMALL, stream);

@@ -114,7 +114,7 @@ def test_levels_differ_across_rows(torch):
     assert len(set(got["level"].tolist())) >= 3
 
 
-@pytest.mark.parametrize("d", [7, 1000, 4099, 50000])
+@pytest.mark.parametrize("d", [7, 1000, 4099, 20000, 50000])   # 20000: a short row whose first-digit lists overflow
 def test_ties_and_equalities_use_the_exact_path(torch, d):
     # small integers: many equal magnitudes (lowest index wins), signed zeros, and
     # trigger comparisons that hold with equality, which only exact sums decide
