@@ -318,45 +318,48 @@ inline __device__ double digits_to_double(const u32* dig) {
   return ldexp((double)mant, sh + 32 * (t - 2) - 298);
 }
 
-// Run by one thread of the last CTA of the exact pass: carries, rounds and decides the row.
-// `row_limbs`: the row's NSLOT x NLIMB accumulators, in global memory or (SHARED_LIMBS) in shared memory.
+// The exact value of energy slot s of a row (0: D, 1: ||v||^2, 2 + c: candidate c): carries resolved, the
+// dropped threshold-equal keys of a Top-K candidate added, rounded once to binary64.
 template <bool SHARED_LIMBS = false>
-inline __device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* row_limbs,
-                               const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                               RowDec* __restrict__ dec, const CompressOut& out,
-                               const u32* __restrict__ diffflag, u32* __restrict__ flags) {
-  double val[NSLOT];
-  if (__ldcg(&diffflag[row]) & 0x80000000u) {  // X - Y is not finite
-    for (int s = 0; s < NSLOT; ++s) val[s] = 0.0;
-    atomicOr(&flags[0], 1u);
-    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, val + 1, 0.0);
-    return;
+inline __device__ double exact_slot_value(const CsetDev& cs, int row, long long d, const u64* row_limbs,
+                                          const SelRow* __restrict__ sel, int s) {
+  if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) return 0.0;   // identity: no error
+  u32 dig[NLIMB];
+  const u64* l = row_limbs + s * NLIMB;
+  unsigned __int128 tie = 0;
+  int tk = 0;
+  if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK) {
+    int j = 0;
+    for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
+    const u32 T = sel[row].T[j];
+    const u32 ex = T >> 23, fr = T & 0x7fffffu;
+    const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
+    const int off = 2 * (int)(ex ? ex : 1u) - 2;
+    tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
+    tk = off >> 5;
   }
-  for (int s = 0; s < 2 + cs.m; ++s) {
-    u32 dig[NLIMB];
-    const u64* l = row_limbs + s * NLIMB;
-    unsigned __int128 tie = 0;
-    int tk = 0;
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] < d) {
-      int j = 0;
-      for (int t = 0; t < cs.nsel; ++t) if (cs.sel[t] == s - 2) j = t;
-      const u32 T = sel[row].T[j];
-      const u32 ex = T >> 23, fr = T & 0x7fffffu;
-      const u64 m = ex ? (u64)(fr | 0x800000u) : (u64)fr;
-      const int off = 2 * (int)(ex ? ex : 1u) - 2;
-      tie = ((unsigned __int128)(m * m) * (u64)(sel[row].ntie[j] - sel[row].q[j])) << (off & 31);
-      tk = off >> 5;
-    }
-    u64 carry = 0;
-    for (int k = 0; k < NLIMB; ++k) {
-      u64 add = 0;
-      if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
-      const unsigned __int128 tsum = (unsigned __int128)(SHARED_LIMBS ? l[k] : __ldcg(&l[k])) + carry + add;
-      dig[k] = (u32)tsum;
-      carry = (u64)(tsum >> 32);
-    }
-    val[s] = digits_to_double(dig);
-    if (s >= 2 && cs.kind[s - 2] == ADACGD_TOPK && cs.param[s - 2] >= d) val[s] = 0.0;
+  u64 carry = 0;
+  for (int k = 0; k < NLIMB; ++k) {
+    u64 add = 0;
+    if (k >= tk && k < tk + 4) add = (u64)(u32)(tie >> (32 * (k - tk)));
+    const unsigned __int128 tsum = (unsigned __int128)(SHARED_LIMBS ? l[k] : __ldcg(&l[k])) + carry + add;
+    dig[k] = (u32)tsum;
+    carry = (u64)(tsum >> 32);
+  }
+  return digits_to_double(dig);
+}
+
+// The decision of a row from its exact sums val[0 .. 1 + m] (Eq. 10 and 11 with no rounding left to doubt).
+inline __device__ void decide_exact_row(const CsetDev& cs, int row, long long d, const double* val,
+                                        const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                                        RowDec* __restrict__ dec, const CompressOut& out,
+                                        const u32* __restrict__ diffflag, u32* __restrict__ flags) {
+  if (__ldcg(&diffflag[row]) & 0x80000000u) {  // X - Y is not finite
+    double zero[NSLOT];
+    for (int s = 0; s < NSLOT; ++s) zero[s] = 0.0;
+    atomicOr(&flags[0], 1u);
+    finalize_row(cs, row, 0, d, sel, maxkey, dec, out, zero + 1, 0.0);
+    return;
   }
   const double D = val[0];
   const double rhs = (double)cs.zeta * D;
@@ -364,6 +367,17 @@ inline __device__ void pick_exact_row(const CsetDev& cs, int row, long long d, c
   for (int j = 0; j <= cs.m; ++j)
     if (val[1 + j] <= rhs) { level = j; break; }
   finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
+}
+
+// Run by one thread of the last CTA of the exact pass: carries, rounds and decides the row.
+// `row_limbs`: the row's NSLOT x NLIMB accumulators in global memory.
+inline __device__ void pick_exact_row(const CsetDev& cs, int row, long long d, const u64* row_limbs,
+                               const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                               RowDec* __restrict__ dec, const CompressOut& out,
+                               const u32* __restrict__ diffflag, u32* __restrict__ flags) {
+  double val[NSLOT];
+  for (int s = 0; s < NSLOT; ++s) val[s] = (s < 2 + cs.m) ? exact_slot_value<false>(cs, row, d, row_limbs, sel, s) : 0.0;
+  decide_exact_row(cs, row, d, val, sel, maxkey, dec, out, diffflag, flags);
 }
 
 // --------------------------------------------------------------------------

@@ -283,12 +283,28 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       sq_pieces(val, &kk, p);
       limb_add(lsh + slot * NLIMB, kk, p);
     };
+    // D needs X - Y again: four loads of each in flight per thread
+    for (int base = threadIdx.x; base < dn; base += 4 * TPB) {
+      float xw[4], yw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = base + u * TPB;
+        xw[u] = (i < dn) ? xr[i] : 0.f;
+        yw[u] = (i < dn) ? yr[i] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (base + u * TPB >= dn) break;
+        const float w = __fsub_rn(xw[u], yw[u]);
+        if (key_of(w) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
+        unsigned __int128 tw;
+        if (sq_term(w, &tw)) accD += tw; else slow_add(0, w);
+      }
+    }
     for (int i = threadIdx.x; i < dn; i += TPB) {
       const float v = vs[i];
-      const float w = __fsub_rn(xr[i], yr[i]);
-      if (key_of(w) >= 0x7f800000u || key_of(v) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
-      unsigned __int128 tw, tv;
-      if (sq_term(w, &tw)) accD += tw; else slow_add(0, w);
+      if (key_of(v) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
+      unsigned __int128 tv;
       const bool v_in = sq_term(v, &tv);
       if (v_in) accE += tv; else slow_add(1, v);
       const u32 key = key_of(v);
@@ -342,7 +358,12 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       if (hi >> 32) atomicAdd(&lsh[slot * NLIMB + k0 + 2], hi >> 32);
     }
     __syncthreads();
-    if (threadIdx.x == 0) pick_exact_row<true>(cs, row, d, lsh, sel, maxkey, dec, out, diffflag, flags);
+    // one thread per energy slot resolves its carries and rounds; one thread decides
+    __shared__ double xval[NSLOT];
+    if (threadIdx.x < NSLOT)
+      xval[threadIdx.x] = (threadIdx.x < 2 + cs.m) ? exact_slot_value<true>(cs, row, d, lsh, sel, threadIdx.x) : 0.0;
+    __syncthreads();
+    if (threadIdx.x == 0) decide_exact_row(cs, row, d, xval, sel, maxkey, dec, out, diffflag, flags);
     __syncthreads();
   }
 
