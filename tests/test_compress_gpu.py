@@ -370,3 +370,34 @@ def test_single_pass_crowded_threshold_bin(torch):
     got, _ = check_against_oracle(torch, X, G, Y, [(TOPK, 1000), (TOPK, 10_000), (TOPK, 100_000)], 1.0,
                                   both_update_paths=True)
     assert got["fallbacks"] == 0 and got["list_levels"] >= 1
+
+
+def test_short_rows_random_sweep(torch):
+    # seeded sweep over the short-row kernel: random shapes, candidate lists (Top-K up to and beyond d, quantisers,
+    # in any admissible order), triggers, and a mix of continuous and tie-heavy rows
+    rng = np.random.Generator(np.random.PCG64(77))
+    for case in range(48):
+        rows = int(rng.integers(1, 6))
+        d = int(rng.choice([1, 2, 3, 4, 5, 31, 32, 33, 255, 256, 257, 1000, 1023, 1025, 2999]))
+        if case % 3 == 0:
+            X, G, Y = S.tie_vectors(rows, d, seed=1000 + case, levels=int(rng.integers(1, 6)))
+        else:
+            X, G, Y = S.gaussian_rows(rows, d, seed=1000 + case, drift=float(rng.choice([0.0, 0.01, 0.3])),
+                                      move=float(rng.choice([0.0, 0.1])))
+        if case % 5 == 0:
+            Y = G.copy()                      # |X - G| == |X - Y| everywhere: the equality shortcut of the skip test
+        ks = sorted(set(int(k) for k in rng.integers(1, max(2, 2 * d), size=int(rng.integers(0, 5)))))
+        ks = [k for i, k in enumerate(ks) if i == 0 or ks[i - 1] < d]          # only the last Top-K may reach d
+        qs = sorted(set(int(b) for b in rng.integers(2, 17, size=int(rng.integers(0, 3)))))
+        cands, ki, qi = [], 0, 0
+        while ki < len(ks) or qi < len(qs):    # interleave, each kind in increasing order
+            take_k = ki < len(ks) and (qi >= len(qs) or rng.random() < 0.5)
+            if take_k:
+                cands.append((TOPK, ks[ki])); ki += 1
+            else:
+                cands.append((QUANT, qs[qi])); qi += 1
+        cands = cands[:8]
+        if not cands:
+            cands = [(TOPK, 1)]
+        zeta = float(rng.choice([0.0, 0.1, 1.0, 3.0, 1e30]))
+        check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
