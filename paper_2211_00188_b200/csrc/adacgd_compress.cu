@@ -524,7 +524,12 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
       // Common case for the whole tile of rows: every row either skips or applies a Top-K level whose
       // threshold-equal keys are decided by the index cut, and no kept-index list is wanted.
       bool simple = true;
-      if (threadIdx.x < nr) simple = shd[threadIdx.x].mode != 4 && !(shd[threadIdx.x].mode == 1 && shd[threadIdx.x].need_tie);
+      // rows that need no per-key tie ranking; without 16-byte alignment the batched loop below only takes
+      // skipped rows and Top-K rows, identity and quantiser rows go through the general loop
+      if (threadIdx.x < nr) {
+        const int m = shd[threadIdx.x].mode;
+        simple = ALIGNED ? (m != 4 && !(m == 1 && shd[threadIdx.x].need_tie)) : (m == 0 || (m == 1 && !shd[threadIdx.x].need_tie));
+      }
       simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
       if (simple && ALIGNED) {
         if (live) {   // few chunks (short rows): more rows in flight per thread, the SMs are not full

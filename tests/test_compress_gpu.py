@@ -401,3 +401,33 @@ def test_short_rows_random_sweep(torch):
             cands = [(TOPK, 1)]
         zeta = float(rng.choice([0.0, 0.1, 1.0, 3.0, 1e30]))
         check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+
+
+def test_single_pass_random_sweep(torch):
+    # seeded sweep over the sampled single-pass pipeline: odd and even row lengths, heavy ties, rows equal to their
+    # previous gradient, blocks of very different scale, quantisers mixed in, several triggers
+    rng = np.random.Generator(np.random.PCG64(88))
+    for case in range(8):
+        rows = int(rng.integers(1, 4))
+        d = int(rng.choice([524_288, 600_001, 750_000, 1_000_003])) // (1 if rows == 1 else 1)
+        kind = case % 4
+        if kind == 0:
+            X, G, Y = S.gaussian_rows(rows, d, seed=2000 + case)
+        elif kind == 1:   # values on a coarse grid: tie groups at every threshold
+            X, G, Y = S.gaussian_rows(rows, d, seed=2000 + case)
+            X, G, Y = ((np.round(a * 64) / 64).astype(F32) for a in (X, G, Y))
+        elif kind == 2:   # contiguous blocks of very different scale
+            X, G, Y = S.gaussian_rows(rows, d, seed=2000 + case)
+            scale = np.repeat(np.exp(2.0 * rng.standard_normal(50)), -(-d // 50))[:d].astype(F32)
+            X, G, Y = (a * scale for a in (X, G, Y))
+        else:             # most of the row unchanged since the last round
+            X, G, Y = S.gaussian_rows(rows, d, seed=2000 + case)
+            same = rng.random(d) < 0.9
+            G[:, same] = X[:, same]
+        ks = sorted(set(int(k) for k in (d * np.array([1e-4, 1e-3, 1e-2, 0.1, 0.5]) * rng.uniform(0.5, 1.5, 5))))
+        ks = [k for k in ks if 0 < k < d][:int(rng.integers(1, 6))]
+        cands = [(TOPK, k) for k in ks]
+        if case % 2 == 1:
+            cands.insert(int(rng.integers(0, len(cands) + 1)), (QUANT, int(rng.integers(2, 9))))
+        zeta = float(rng.choice([0.0, 0.3, 1.0, 4.0]))
+        check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
