@@ -431,3 +431,23 @@ def test_single_pass_random_sweep(torch):
             cands.insert(int(rng.integers(0, len(cands) + 1)), (QUANT, int(rng.integers(2, 9))))
         zeta = float(rng.choice([0.0, 0.3, 1.0, 4.0]))
         check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+
+
+def test_three_pass_random_sweep(torch):
+    # seeded sweep over the mid-size route (rows too long for the short-row kernel, problem too small for the
+    # sampled pipeline): aligned and unaligned rows, ties, quantisers, identity as the last candidate
+    rng = np.random.Generator(np.random.PCG64(99))
+    for case in range(8):
+        d = int(rng.choice([32_769, 40_000, 65_537, 100_000, 131_071]))
+        rows = int(rng.integers(1, max(2, min(5, (1 << 19) // d))))
+        if case % 3 == 1:
+            X, G, Y = S.tie_vectors(rows, d, seed=3000 + case, levels=3)
+        else:
+            X, G, Y = S.gaussian_rows(rows, d, seed=3000 + case, drift=float(rng.choice([0.01, 0.3])))
+        ks = sorted(set(int(k) for k in (d * np.array([1e-4, 1e-2, 0.2, 1.0]) * rng.uniform(0.6, 1.4, 4))))
+        ks = [k for i, k in enumerate(ks) if k > 0 and (i == 0 or ks[i - 1] < d)]
+        cands = [(TOPK, k) for k in ks]
+        if case % 2 == 0:
+            cands.insert(int(rng.integers(0, len(cands) + 1)), (QUANT, int(rng.integers(2, 17))))
+        zeta = float(rng.choice([0.0, 0.5, 1.0, 1e30]))
+        check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
