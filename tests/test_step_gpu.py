@@ -239,3 +239,33 @@ def test_sparse_lockstep_mixed_candidates(torch):
         assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), O.server_mean(G_ref).view(np.uint32))
         seen.update(levels[0])
     assert len(seen) >= 2
+
+
+def test_lockstep_random_sweep(torch):
+    # seeded sweep over whole iterations: the three objectives, worker and master lists with Top-K and quantisers,
+    # the three initialisations, several triggers and shapes (short rows and the mid-size route)
+    rng = np.random.Generator(np.random.PCG64(123))
+    for case in range(6):
+        n = int(rng.integers(2, 6))
+        d = int(rng.choice([257, 1000, 4096, 40_000]))
+        m = int(rng.choice([16, 40]))
+        loss = case % 3
+        if loss == 2:
+            A, t, _ = S.least_squares_problem(n, d, m, seed=200 + case)
+        else:
+            A, t = S.logistic_problem(n, d, m, seed=200 + case)
+        lam = 0.0 if loss == 2 else (0.1 if loss == 0 else 1e-3)
+        gamma = 0.5 / S.smoothness_estimate(A, loss, lam)
+
+        def cands():
+            ks = sorted(set(int(k) for k in (d * np.array([1e-3, 1e-2, 0.1, 1.0]) * rng.uniform(0.5, 1.2, 4))))
+            ks = [k for i, k in enumerate(ks) if k > 0 and (i == 0 or ks[i - 1] < d)][:int(rng.integers(1, 5))]
+            c = [(TOPK, k) for k in ks]
+            if rng.random() < 0.5:
+                c.insert(int(rng.integers(0, len(c) + 1)), (QUANT, int(rng.integers(2, 9))))
+            return c
+
+        wc = cands()
+        mc = cands() if case % 2 == 0 else []
+        lockstep(torch, A, t, loss, lam, gamma, wc, float(rng.choice([0.0, 0.5, 1.0, 2.0])), mc,
+                 float(rng.choice([0.25, 1.0])), T=int(rng.integers(4, 9)), g0_mode=case % 3)
