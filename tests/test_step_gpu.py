@@ -269,3 +269,37 @@ def test_lockstep_random_sweep(torch):
         mc = cands() if case % 2 == 0 else []
         lockstep(torch, A, t, loss, lam, gamma, wc, float(rng.choice([0.0, 0.5, 1.0, 2.0])), mc,
                  float(rng.choice([0.25, 1.0])), T=int(rng.integers(4, 9)), g0_mode=case % 3)
+
+
+def test_sparse_lockstep_random_sweep(torch):
+    # seeded sweep over CSR problems: densities, row lengths on both sides of the short-row limit, empty columns,
+    # master compression on and off
+    rng = np.random.Generator(np.random.PCG64(321))
+    for case in range(5):
+        n = int(rng.integers(2, 6))
+        d = int(rng.choice([999, 5000, 40_000]))
+        m = int(rng.choice([7, 33]))
+        density = float(rng.choice([0.002, 0.01, 0.05]))
+        ks = sorted(set(int(k) for k in (d * np.array([1e-3, 1e-2, 0.2]) * rng.uniform(0.5, 1.5, 3))))
+        wc = [(TOPK, k) for k in ks if 0 < k < d]
+        if case % 2 == 0:
+            wc.insert(int(rng.integers(0, len(wc) + 1)), (QUANT, int(rng.integers(2, 9))))
+        mc = [(TOPK, max(1, d // 50)), (TOPK, d)] if case % 2 == 1 else []
+        wz, mz = float(rng.choice([0.0, 1.0, 3.0])), 0.5
+        gamma = float(rng.choice([0.5, 2.0]))
+        eng, prob, x0 = make_sparse(torch, n, d, m, density, 300 + case, wc, wz, mc, mz, gamma=gamma)
+        st = O.init_state(prob, x0, wc)
+        for it in range(5):
+            push_state(eng, torch, st)
+            before = {k: np.copy(v) for k, v in st.items() if isinstance(v, np.ndarray)}
+            recs, levels = eng.step(1, report=True)
+            O.step(st, prob, gamma, wc, wz, mc, mz)
+            ggrad = eng.get_state("grad").cpu().numpy()
+            assert relerr(ggrad, st["X"]) <= 1e-5, (case, it)
+            G_ref, res = O.compress_rows(ggrad, before["G"], before["X"], wc, wz)
+            assert levels[0] == [r["level"] for r in res], (case, it)
+            assert np.array_equal(eng.get_state("G").cpu().numpy().view(np.uint32), G_ref.view(np.uint32)), (case, it)
+            gt_ref = O.server_mean(G_ref)
+            assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), gt_ref.view(np.uint32))
+            mres = O.adacgd(before["gm"], before["gt"], gt_ref, list(mc), mz)
+            assert np.array_equal(eng.get_state("gm").cpu().numpy().view(np.uint32), mres["out"].view(np.uint32)), (case, it)
