@@ -451,3 +451,22 @@ def test_three_pass_random_sweep(torch):
             cands.insert(int(rng.integers(0, len(cands) + 1)), (QUANT, int(rng.integers(2, 17))))
         zeta = float(rng.choice([0.0, 0.5, 1.0, 1e30]))
         check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+
+
+@pytest.mark.parametrize("cands", [[], [(TOPK, 7), (QUANT, 4), (TOPK, 9999)]])
+def test_host_entry_point_unaligned_and_identity(torch, cands):
+    import paper_2211_00188_b200 as pkg
+    n, d = 5, 9999
+    X, G, Y = S.gaussian_rows(n, d, seed=12)
+    eng = pkg.AdaCGD(n, d, cands, 0.7, host_staging=True)
+    Xh, Gh, Yh = (torch.from_numpy(a.copy()).pin_memory() for a in (X, G, Y))
+    mean = torch.zeros(d).pin_memory()
+    level = torch.full((n,), -3, dtype=torch.int32).pin_memory()
+    eng.compress_host(Xh, Gh, Yh, mean_out=mean, level=level)
+    if cands:
+        G_ref, res = O.compress_rows(X, G, Y, cands, 0.7)
+        assert level.tolist() == [r["level"] for r in res]
+    else:
+        G_ref = X.copy()                      # the identity compressor sends the gradient itself
+    assert_bitwise(Gh.numpy(), G_ref, "G")
+    assert_bitwise(mean.numpy(), O.server_mean(G_ref), "mean")
