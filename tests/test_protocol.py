@@ -177,3 +177,27 @@ def test_run_to_budget_on_the_engine():
     assert rec["bits_up"][-1] >= budget and (len(rec["bits_up"]) == 1 or rec["bits_up"][-2] < budget)
     assert eng.get_state("bits_up") == rec["bits_up"][-1] and eng.get_state("step") == len(rec["loss"])
     assert rec["loss"][-1] < rec["loss"][0]
+
+
+@pytest.mark.gpu
+def test_gamma_sweep_on_the_engine():
+    import torch
+    import paper_2211_00188_b200 as pkg
+
+    n, d, m = 3, 300, 30
+    A, t, _ = S.least_squares_problem(n, d, m, seed=9)
+    base = 0.125 / S.smoothness_estimate(A, 2, 0.0)
+    cands, z = P.method_set("clag", d, K=5, zeta=1.0)
+    dev = torch.device("cuda:0")
+    Ad, td = torch.from_numpy(A).to(dev), torch.from_numpy(t).to(dev)
+
+    def make(gamma):
+        return pkg.AdaCGD(n, d, cands, z, loss=2, lam=0.0, A=Ad, target=td, x0=torch.zeros(d, device=dev), gamma=gamma)
+
+    budget = 60 * P.max_bits_per_round(n, d, cands)
+    res = P.gamma_sweep(make, base, budget, exponents=range(0, 7), max_rounds=400)
+    finals = {e: r["loss"][-1] for e, r in res["runs"].items()}
+    finite = {e: v for e, v in finals.items() if np.isfinite(v)}
+    assert res["best"] == min(finite, key=finite.get)
+    assert finite and finals[res["best"]] <= min(finite.values())
+    assert all(r["bits_up"][-1] >= budget or len(r["loss"]) == 400 for r in res["runs"].values())
