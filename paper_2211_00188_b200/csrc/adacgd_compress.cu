@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs, long long d, int nblk_
   const int row = blockIdx.x;
   if (picked && picked[row * NTICKET + 9]) return;
   const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
-  pick_row(cs, d, row, nblk, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+  pick_row(cs, d, row, nblk, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);  // k_quant_err: main grid
 }
 
 template <bool ALIGNED>
@@ -1565,7 +1565,7 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
   collected_finish_row(cs, row, (int)gridDim.x, sel, fl, lepart, wbuf);
   __syncthreads();   // the brackets' results, written by one warp each, are read by the level choice
   if (pick_here) {
-    pick_row(cs, d, row, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+    pick_row(cs, d, row, nblk_main, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
     if (threadIdx.x == 0) tickets[row * NTICKET + 9] = 1u;
   }
 }

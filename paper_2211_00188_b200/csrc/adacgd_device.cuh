@@ -182,8 +182,9 @@ inline __device__ void finalize_row(const CsetDev& cs, int row, int level, long 
 
 // Chooses the level of one row from its sums (Eq. 10 and 11); run by a whole CTA of TPB threads.
 // The per-CTA partial sums of the streaming pass are added in a fixed order: thread t takes
-// blocks t, t + TPB, ..., then lanes, then warps.
-inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, const double* __restrict__ partial,
+// blocks t, t + TPB, ..., then lanes, then warps.  D, ||v||^2 and the Top-K slots hold nblk partial
+// sums per row, the quantiser slots nblk_q (their pass may run on another grid).
+inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, int nblk_q, const double* __restrict__ partial,
                          const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
                          RowDec* __restrict__ dec, u32* __restrict__ flags, const CompressOut& out,
                          const u32* __restrict__ diffflag, double tol) {
@@ -203,10 +204,13 @@ inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nbl
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) a[s] = 0.0;
   const double* p = partial + (long long)row * MAX_BLK_PER_ROW * NSLOT;
-  for (int b = threadIdx.x; b < nblk; b += TPB) {
+  u32 qmask = 0;   // slots written by the quantiser pass
+  for (int j = 0; j < cs.nquant; ++j) qmask |= 1u << (2 + cs.qsel[j]);
+  const int nblk_max = nblk > nblk_q ? nblk : nblk_q;
+  for (int b = threadIdx.x; b < nblk_max; b += TPB) {
 #pragma unroll
     for (int s = 0; s < NSLOT; ++s)
-      if (s < nslot) a[s] += __ldcg(&p[(long long)b * NSLOT + s]);
+      if (s < nslot && b < (((qmask >> s) & 1u) ? nblk_q : nblk)) a[s] += __ldcg(&p[(long long)b * NSLOT + s]);
   }
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) {

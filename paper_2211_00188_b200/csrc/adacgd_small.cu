@@ -254,7 +254,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     diffflag[row] = ((mxw >= 0x7f800000u) ? 0x80000000u : 0u) | (dfl & 0x7fffffffu);
   }
   __syncthreads();
-  pick_row(cs, d, row, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+  pick_row(cs, d, row, 1, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
   __syncthreads();
   if (__ldcg(&dec[row].need_exact)) {
     // the comparison could not be certified: exact integer sums of the row, then the decision from them

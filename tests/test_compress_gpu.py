@@ -296,6 +296,23 @@ def test_single_pass_list_overflow_falls_back(torch):
     assert got["fallbacks"] == 2
 
 
+def test_single_pass_fallback_rows_with_quantisers(torch):
+    # Top-K and quantiser candidates mixed, on rows that all fall back to the full select (their lists overflow) in a
+    # shape where the fallback kernels run on fewer CTAs per row than the streaming pass: every error sum of a row
+    # must be taken over the CTAs of the pass that wrote it.  zeta sits between one half and the whole of the 2-bit
+    # quantiser's error, so that an error summed over too few CTAs would pass the trigger.
+    X, G, Y = S.tie_vectors(40, 200_000, seed=37, levels=1)
+    cands = [(TOPK, 100), (QUANT, 2), (TOPK, 50_000), (QUANT, 8)]
+    got, res = check_against_oracle(torch, X, G, Y, cands, 0.25, both_update_paths=True)
+    assert got["fallbacks"] == 40
+    assert {r["level"] for r in res} == {4}
+    # one long row: 367 CTAs in the streaming pass, 296 in the fallback kernels
+    X, G, Y = S.tie_vectors(1, 3_000_000, seed=38, levels=1)
+    cands = [(TOPK, 1000), (QUANT, 2), (TOPK, 750_000), (QUANT, 8)]
+    got, res = check_against_oracle(torch, X, G, Y, cands, 0.25)
+    assert got["fallbacks"] == 1 and res[0]["level"] == 4
+
+
 def test_large_row_many_tiles(torch):
     X, G, Y = S.gaussian_rows(2, 3_000_001, seed=34)
     got, _ = check_against_oracle(torch, X, G, Y, [(TOPK, 3000), (TOPK, 30000), (TOPK, 300000)], 1.0)

@@ -174,6 +174,23 @@ def test_golden_adacgd_hand_examples():
             assert (res["kept"].tolist() if res["kept"] is not None else None) == z["kept"]
 
 
+def test_golden_message_bit_patterns():
+    # Eq. 7 bit for bit, signs of zero included: a Top-K message touches the kept entries only, a quantised one
+    # every entry.  Compared as uint32 patterns (== and array_equal do not see the sign of a zero).
+    for case in json.load(open(GOLDEN))["message_bit_patterns"]:
+        h = np.array([int(b, 16) for b in case["h_bits"]], dtype=np.uint32).view(F32)
+        x = np.array([int(b, 16) for b in case["x_bits"]], dtype=np.uint32).view(F32)
+        want = np.array([int(b, 16) for b in case["out_bits"]], dtype=np.uint32)
+        cand = tuple(case["cand"])
+        y = np.zeros_like(x)
+        assert O.ef21(h, y, x, cand).view(np.uint32).tolist() == want.tolist(), case["cite"]
+        # zeta = 0 with one candidate applies that candidate (x != h): the same update through Eq. 11
+        res = O.adacgd(h, y, x, [cand], 0.0)
+        assert res["level"] == 1 and res["out"].view(np.uint32).tolist() == want.tolist(), case["cite"]
+        # the inputs are untouched
+        assert h.view(np.uint32).tolist() == [int(b, 16) for b in case["h_bits"]]
+
+
 def test_zeta_zero_is_ef21():
     # Section 4.3: zeta = 0 reduces AdaCGD to EF21 (with the last candidate)
     r = rng(6)
