@@ -20,6 +20,10 @@
  *   - All device work is enqueued on the stream given to adacgd_init.  A call
  *     that returns results to the host synchronises that stream; the others
  *     return as soon as the work is enqueued.
+ *   - A context is bound to the CUDA device that is current when adacgd_init is
+ *     called (its workspace and stream must belong to it).  Every later call on the
+ *     context must be made with that device current and returns
+ *     ADACGD_ERR_INVALID_ARG otherwise.
  *   - Every entry point returns an adacgd_status and never aborts; a message for
  *     the last failure is available from adacgd_last_error.
  *   - Arithmetic: every elementwise operation is one IEEE binary32 operation
@@ -223,6 +227,8 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
 #define ADACGD_STATE_LIST_LEVELS 12/* uint32: rows whose threshold shared the first digit of its bracket with more keys
                                    than the collection buffer holds (many equal or nearly equal magnitudes) and
                                    that went through the three-level passes over the key lists, since init (get only) */
+#define ADACGD_STATE_DEVICE 13  /* int32: ordinal of the CUDA device the context is bound to (the device that was
+                                   current at adacgd_init); host destination only (get only) */
 adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,
                                int32_t dst_is_device);
 adacgd_status adacgd_set_state(adacgd_ctx* ctx, int32_t which, const void* src, size_t bytes,
@@ -234,6 +240,15 @@ const char* adacgd_last_error(const adacgd_ctx* ctx);
 
 /* Releases host bookkeeping.  Device memory belongs to the caller. */
 void adacgd_destroy(adacgd_ctx* ctx);
+
+/* Bits of the message one worker sends when it applies candidate `cand` to a vector of d entries.  The paper
+ * measures communication cost (Appendix C stops every method at a bit budget) but prints no formula; this is
+ * the library's reading and its only definition: Top-K with K < d sends K values of 32 bits, each with an
+ * index of ceil(log2 d) bits; Top-K with K >= d sends the d values; a b-bit quantiser sends its 32-bit scale
+ * and b bits per entry; skipping sends nothing.  The bit counts that adacgd_compress and adacgd_step report
+ * are this function of the chosen level.  Host only, needs no device.  Returns 0 for an invalid candidate
+ * (NULL, unknown kind, K < 1, width outside [2,16]) or d outside [1, 2^31). */
+uint64_t adacgd_message_bits(const adacgd_cand* cand, int64_t d);
 
 /* Number of kernels this library has launched on behalf of ctx since init. */
 int64_t adacgd_launch_count(const adacgd_ctx* ctx);

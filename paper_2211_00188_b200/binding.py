@@ -12,14 +12,14 @@ TOPK, QUANT = 0, 1
 LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE = 0, 1, 2, 3
 LAYOUT_DENSE, LAYOUT_CSR = 0, 1
 FLAG_HOST_STAGING = 1
-STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11, list_levels=12)
+STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11, list_levels=12, device=13)
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "BAD_ORDER", 3: "NONFINITE", 4: "WORKSPACE", 5: "CUDA", 6: "UNSUPPORTED"}
 
 EXPORTED_SYMBOLS = [
     "adacgd_workspace_bytes", "adacgd_init", "adacgd_step", "adacgd_compress", "adacgd_compress_host",
     "adacgd_gradient", "adacgd_get_state", "adacgd_set_state", "adacgd_last_error", "adacgd_destroy",
     "adacgd_launch_count", "adacgd_profile_kernel_count", "adacgd_profile_kernel_name", "adacgd_profile_enable",
-    "adacgd_profile_read", "adacgd_compress_noalloc",
+    "adacgd_profile_read", "adacgd_compress_noalloc", "adacgd_message_bits",
 ]
 
 Cand = Tuple[int, int]
@@ -84,6 +84,8 @@ def load_library():
     lib.adacgd_launch_count.argtypes = [vp]
     lib.adacgd_launch_count.restype = i64
     lib.adacgd_compress_noalloc.argtypes = [vp, vp, vp, i32, i64, C.POINTER(_Cset), vp, vp, vp, vp]
+    lib.adacgd_message_bits.argtypes = [C.POINTER(_Cand), i64]
+    lib.adacgd_message_bits.restype = C.c_uint64
     lib.adacgd_profile_kernel_count.argtypes = []
     lib.adacgd_profile_kernel_name.argtypes = [i32]
     lib.adacgd_profile_kernel_name.restype = C.c_char_p
@@ -91,7 +93,7 @@ def load_library():
     lib.adacgd_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     for name in EXPORTED_SYMBOLS:
         if name not in ("adacgd_last_error", "adacgd_destroy", "adacgd_launch_count",
-                        "adacgd_profile_kernel_name"):
+                        "adacgd_profile_kernel_name", "adacgd_message_bits"):
             getattr(lib, name).restype = i32
     _LIB = lib
     return lib
@@ -105,6 +107,12 @@ def _cset(cands: Optional[Sequence[Cand]], zeta: float):
         arr[i].kind, arr[i].reserved, arr[i].param = int(kind), 0, int(param)
     cs = _Cset(C.cast(arr, C.POINTER(_Cand)), len(cands), float(zeta))
     return cs, arr
+
+
+def message_bits(cand: Cand, d: int) -> int:
+    """adacgd_message_bits: bits of the message a worker sends with candidate `cand` at dimension d."""
+    c = _Cand(int(cand[0]), 0, int(cand[1]))
+    return int(load_library().adacgd_message_bits(C.byref(c), int(d)))
 
 
 def _ptr(t):
@@ -228,7 +236,7 @@ class AdaCGD:
             self._check(self.lib.adacgd_get_state(self.ctx, STATE[which], _ptr(out), out.numel() * out.element_size(), 1),
                         self.ctx)
             return out
-        buf = C.c_uint64(0) if which not in ("flags", "rechecks", "fallbacks", "list_levels") else C.c_uint32(0)
+        buf = C.c_uint64(0) if which not in ("flags", "rechecks", "fallbacks", "list_levels", "device") else C.c_uint32(0)
         self._check(self.lib.adacgd_get_state(self.ctx, STATE[which], C.byref(buf), C.sizeof(buf), 0), self.ctx)
         return int(buf.value)
 

@@ -4,7 +4,7 @@
 #include <string>
 #include <vector>
 
-#include "adacgd_internal.cuh"
+#include "adacgd_device.cuh"
 
 using namespace adacgd;
 
@@ -137,6 +137,7 @@ struct adacgd_ctx {
   float gamma;
   int flags;
   cudaStream_t stream;
+  int device;                  // ordinal of the device that was current at adacgd_init; every later call must find it current
   Scratch scr;
   GradScratch gs;
   float *x, *G, *grad_cur, *grad_nxt, *gt_cur, *gt_nxt, *gm, *gm_buf;
@@ -173,6 +174,30 @@ adacgd_status fail(adacgd_ctx* c, adacgd_status s, const std::string& m) {
 adacgd_status cuda_fail(adacgd_ctx* c, const char* what) {
   cudaError_t e = cudaGetLastError();
   return fail(c, ADACGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+adacgd_status cuda_fail(adacgd_ctx* c, const char* what, cudaError_t e) {
+  cudaGetLastError();  // the sticky copy of the same error
+  return fail(c, ADACGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+// Runs a CUDA runtime call and leaves the entry point with a message that names it when it fails.
+#define CK(c, call, what)                                          \
+  do {                                                             \
+    const cudaError_t ck_e_ = (call);                              \
+    if (ck_e_ != cudaSuccess) return cuda_fail((c), (what), ck_e_); \
+  } while (0)
+
+// A context is bound to the device that was current when it was created: its workspace, its stream and
+// the per-device kernel attributes belong to that device.
+adacgd_status check_device(adacgd_ctx* c, const char* entry) {
+  int dev = -1;
+  const cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(c, (std::string(entry) + " (cudaGetDevice)").c_str(), e);
+  if (dev != c->device)
+    return fail(c, ADACGD_ERR_INVALID_ARG, std::string(entry) + ": the current CUDA device is " + std::to_string(dev) +
+                                               " but the context was created on device " + std::to_string(c->device));
+  return ADACGD_OK;
 }
 
 // Worker side + mean, then master side, on the context's own state.
@@ -213,22 +238,17 @@ adacgd_status adacgd_workspace_bytes(const adacgd_problem* problem, const adacgd
   return ADACGD_OK;
 }
 
-adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, const adacgd_cset* worker,
-                          const adacgd_cset* master, const float* x0_dev, float gamma, int32_t g0_mode,
-                          int32_t flags, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+// Everything of adacgd_init that can fail after the context object exists; messages go to the thread's
+// slot because the caller gets no context back on failure.
+static adacgd_status init_body(adacgd_ctx* c, const adacgd_problem* problem, const adacgd_cset* worker,
+                               const adacgd_cset* master, const float* x0_dev, float gamma, int32_t g0_mode,
+                               int32_t flags, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
   const char* msg = "";
-  if (!ctx_out) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx_out is NULL");
-  *ctx_out = nullptr;
-  adacgd_status s = check_problem(problem, &msg);
-  if (s != ADACGD_OK) return fail(nullptr, s, msg);
-  adacgd_ctx* c = new (std::nothrow) adacgd_ctx();
-  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "out of host memory");
+  adacgd_status s;
   c->p = *problem;
   if ((s = make_cset(worker, problem->d, &c->wcs, &msg)) != ADACGD_OK ||
-      (s = make_cset(master, problem->d, &c->mcs, &msg)) != ADACGD_OK) {
-    delete c;
+      (s = make_cset(master, problem->d, &c->mcs, &msg)) != ADACGD_OK)
     return fail(nullptr, s, msg);
-  }
   c->master_compresses = master && master->m > 0;
   c->gamma = gamma;
   c->flags = flags;
@@ -239,24 +259,21 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   c->graph_tried = false;
   c->odd = false;
   c->prof = nullptr;
+  c->copy_stream = nullptr;
+  for (cudaEvent_t& e : c->copy_ev) e = nullptr;
+  c->x = c->G = c->grad_cur = c->grad_nxt = c->gt_cur = c->gt_nxt = c->gm = c->gm_buf = nullptr;
   const bool has_loss = problem->loss != ADACGD_LOSS_NONE;
-  if (has_loss && (!x0_dev || !(gamma > 0.f) || g0_mode < 0 || g0_mode > 2)) {
-    delete c;
+  if (has_loss && (!x0_dev || !(gamma > 0.f) || g0_mode < 0 || g0_mode > 2))
     return fail(nullptr, ADACGD_ERR_INVALID_ARG, "x0_dev must be non-NULL, gamma > 0, g0_mode in {0,1,2}");
-  }
-  if (has_loss && g0_mode == 2 && c->wcs.m == 0) {
-    delete c;
+  if (has_loss && g0_mode == 2 && c->wcs.m == 0)
     return fail(nullptr, ADACGD_ERR_INVALID_ARG, "g0_mode 2 needs a worker candidate");
-  }
   const WsLayout L = ws_layout(*problem, c->master_compresses, flags);
-  if (!workspace_dev || ((uintptr_t)workspace_dev & 255)) {
-    delete c;
+  if (!workspace_dev || ((uintptr_t)workspace_dev & 255))
     return fail(nullptr, ADACGD_ERR_INVALID_ARG, "workspace_dev must be non-NULL and 256-byte aligned");
-  }
-  if (workspace_bytes < L.total) {
-    delete c;
+  if (workspace_bytes < L.total)
     return fail(nullptr, ADACGD_ERR_WORKSPACE, "workspace smaller than adacgd_workspace_bytes reports");
-  }
+  CK(nullptr, cudaGetDevice(&c->device), "adacgd_init (cudaGetDevice)");
+  if (!current_device()) return cuda_fail(nullptr, "adacgd_init (device attributes)");
   char* b = (char*)workspace_dev;
   carve_scratch(&c->scr, b + L.scratch, problem->n, problem->d, true);
   c->levels = (int*)(b + L.levels);
@@ -267,24 +284,14 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
   c->log = (StepLog*)(b + L.log);
   c->loglevels = (int*)(b + L.loglevels);
   c->stage = (flags & ADACGD_FLAG_HOST_STAGING) ? (float*)(b + L.stage) : nullptr;
-  c->copy_stream = nullptr;
-  for (cudaEvent_t& e : c->copy_ev) e = nullptr;
-  c->x = c->G = c->grad_cur = c->grad_nxt = c->gt_cur = c->gt_nxt = c->gm = c->gm_buf = nullptr;
 
-  if (cudaMemsetAsync(c->scr.flags, 0, 16, c->stream) != cudaSuccess ||
-      cudaMemsetAsync(c->counters, 0, sizeof(Counters), c->stream) != cudaSuccess) {
-    adacgd_status st = cuda_fail(nullptr, "adacgd_init (memset)");
-    delete c;
-    return st;
-  }
+  CK(nullptr, cudaMemsetAsync(c->scr.flags, 0, 16, c->stream), "adacgd_init (clearing the status words)");
+  CK(nullptr, cudaMemsetAsync(c->counters, 0, sizeof(Counters), c->stream), "adacgd_init (clearing the counters)");
   if (has_loss) {
     carve_grad_scratch(&c->gs, b + L.grad, *problem);
     if (problem->layout == ADACGD_LAYOUT_CSR) {
       const char* why = build_csc(*problem, c->gs, c->stream);
-      if (why) {
-        delete c;
-        return fail(nullptr, ADACGD_ERR_INVALID_ARG, why);
-      }
+      if (why) return fail(nullptr, ADACGD_ERR_INVALID_ARG, why);
     }
     c->x = (float*)(b + L.x);
     c->G = (float*)(b + L.G);
@@ -294,21 +301,16 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
     c->gt_nxt = (float*)(b + L.gtB);
     c->gm_buf = c->master_compresses ? (float*)(b + L.gm) : nullptr;
     const size_t nd = (size_t)problem->n * problem->d * 4, dd = (size_t)problem->d * 4;
-    cudaMemcpyAsync(c->x, x0_dev, dd, cudaMemcpyDeviceToDevice, c->stream);
+    CK(nullptr, cudaMemcpyAsync(c->x, x0_dev, dd, cudaMemcpyDeviceToDevice, c->stream), "adacgd_init (copy of x0)");
     int r = launch_gradient(c->p, c->gs, c->x, c->grad_cur, c->stream);
-    if (r < 0) {
-      adacgd_status st = (r == -2) ? fail(nullptr, ADACGD_ERR_UNSUPPORTED, "layout not implemented")
-                                   : cuda_fail(nullptr, "adacgd_init (gradient)");
-      delete c;
-      return st;
-    }
+    if (r < 0) return cuda_fail(nullptr, "adacgd_init (gradient)");
     c->launches += r;
     if (g0_mode == 0) {
-      cudaMemsetAsync(c->G, 0, nd, c->stream);
+      CK(nullptr, cudaMemsetAsync(c->G, 0, nd, c->stream), "adacgd_init (zero estimators)");
     } else if (g0_mode == 1) {
-      cudaMemcpyAsync(c->G, c->grad_cur, nd, cudaMemcpyDeviceToDevice, c->stream);
+      CK(nullptr, cudaMemcpyAsync(c->G, c->grad_cur, nd, cudaMemcpyDeviceToDevice, c->stream), "adacgd_init (estimators = gradients)");
     } else {
-      cudaMemsetAsync(c->G, 0, nd, c->stream);
+      CK(nullptr, cudaMemsetAsync(c->G, 0, nd, c->stream), "adacgd_init (zero estimators)");
       adacgd_cand first = worker->cands[0];
       adacgd_cset one = {&first, 1, 0.f};
       CsetDev cs1;
@@ -316,14 +318,14 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
       CompressOut o;
       memset(&o, 0, sizeof(o));
       r = launch_compress(c->scr, cs1, c->grad_cur, c->G, c->grad_cur, problem->n, problem->d, o, c->stream);
-      if (r < 0) { adacgd_status st = cuda_fail(nullptr, "adacgd_init (g0)"); delete c; return st; }
+      if (r < 0) return cuda_fail(nullptr, "adacgd_init (g0)");
       c->launches += r;
     }
     r = launch_mean_rows(c->G, problem->n, problem->d, c->gt_cur, c->stream);
-    if (r < 0) { adacgd_status st = cuda_fail(nullptr, "adacgd_init (mean)"); delete c; return st; }
+    if (r < 0) return cuda_fail(nullptr, "adacgd_init (mean)");
     c->launches += r;
     if (c->master_compresses) {
-      cudaMemcpyAsync(c->gm_buf, c->gt_cur, dd, cudaMemcpyDeviceToDevice, c->stream);
+      CK(nullptr, cudaMemcpyAsync(c->gm_buf, c->gt_cur, dd, cudaMemcpyDeviceToDevice, c->stream), "adacgd_init (copy of the mean)");
       c->gm = c->gm_buf;
     } else {
       c->gm = c->gt_cur;
@@ -331,10 +333,25 @@ adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, c
       c->launches += 1;
     }
   }
-  if (cudaStreamSynchronize(c->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
-    adacgd_status st = cuda_fail(nullptr, "adacgd_init");
+  CK(nullptr, cudaStreamSynchronize(c->stream), "adacgd_init (synchronising the stream)");
+  CK(nullptr, cudaGetLastError(), "adacgd_init");
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_init(adacgd_ctx** ctx_out, const adacgd_problem* problem, const adacgd_cset* worker,
+                          const adacgd_cset* master, const float* x0_dev, float gamma, int32_t g0_mode,
+                          int32_t flags, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+  const char* msg = "";
+  if (!ctx_out) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx_out is NULL");
+  *ctx_out = nullptr;
+  adacgd_status s = check_problem(problem, &msg);
+  if (s != ADACGD_OK) return fail(nullptr, s, msg);
+  adacgd_ctx* c = new (std::nothrow) adacgd_ctx();
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "out of host memory");
+  s = init_body(c, problem, worker, master, x0_dev, gamma, g0_mode, flags, workspace_dev, workspace_bytes, cuda_stream);
+  if (s != ADACGD_OK) {
     delete c;
-    return st;
+    return s;
   }
   *ctx_out = c;
   return ADACGD_OK;
@@ -354,6 +371,7 @@ adacgd_status adacgd_compress(adacgd_ctx* ctx, const float* X_dev, float* G_dev,
   CsetDev cs;
   adacgd_status s = make_cset(cset, d, &cs, &msg);
   if (s != ADACGD_OK) return fail(ctx, s, msg);
+  if ((s = check_device(ctx, "adacgd_compress")) != ADACGD_OK) return s;
   CompressOut o;
   o.mean_out = mean_out_dev; o.level = level_dev; o.bits = bits_dev; o.err = err_dev; o.D = D_dev;
   o.kept_idx = kept_idx_dev; o.kept_stride = kept_stride; o.kept_cnt = (long long*)kept_cnt_dev;
@@ -377,7 +395,11 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
   float* Ys = Gs + cap;
   float* Ms = Ys + cap;
   unsigned int flags_before = 0, flags_after = 0;
-  cudaMemcpyAsync(&flags_before, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
+  {
+    const adacgd_status sd = check_device(ctx, "adacgd_compress_host");
+    if (sd != ADACGD_OK) return sd;
+  }
+  CK(ctx, cudaMemcpyAsync(&flags_before, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_compress_host (status words to the host)");
   // The rows are taken in up to four groups: while a group's estimators travel back to the host on a second
   // stream, the next group's operands are still coming in (the link carries both directions at once).  The
   // mean needs every row and follows in a kernel of its own, summed in row order like the fused one.
@@ -390,28 +412,28 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
   for (int g = 0; g < ngroups; ++g) {
     const int r0 = (int)((long long)rows * g / ngroups), r1 = (int)((long long)rows * (g + 1) / ngroups);
     const size_t off = (size_t)r0 * (size_t)d, bytes = (size_t)(r1 - r0) * (size_t)d * 4;
-    cudaMemcpyAsync(Xs + off, X_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
-    cudaMemcpyAsync(Gs + off, G_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
-    cudaMemcpyAsync(Ys + off, Y_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream);
+    CK(ctx, cudaMemcpyAsync(Xs + off, X_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream), "adacgd_compress_host (copy of X to the device)");
+    CK(ctx, cudaMemcpyAsync(Gs + off, G_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream), "adacgd_compress_host (copy of G to the device)");
+    CK(ctx, cudaMemcpyAsync(Ys + off, Y_host + off, bytes, cudaMemcpyHostToDevice, ctx->stream), "adacgd_compress_host (copy of Y to the device)");
     adacgd_status s = adacgd_compress(ctx, Xs + off, Gs + off, Ys + off, r1 - r0, d, cset, nullptr,
                                       level_host ? ctx->levels + r0 : nullptr,
                                       bits_host ? (uint64_t*)ctx->bits + r0 : nullptr, nullptr, nullptr, nullptr, 0, nullptr);
-    if (s != ADACGD_OK) { cudaStreamSynchronize(ctx->copy_stream); return s; }
-    cudaEventRecord(ctx->copy_ev[g], ctx->stream);
-    cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_ev[g], 0);
-    cudaMemcpyAsync(G_host + off, Gs + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_stream);
+    if (s != ADACGD_OK) { cudaStreamSynchronize(ctx->copy_stream); return s; }   // earlier groups may still be on their way back
+    CK(ctx, cudaEventRecord(ctx->copy_ev[g], ctx->stream), "adacgd_compress_host (event after a group of rows)");
+    CK(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_ev[g], 0), "adacgd_compress_host (copy stream waiting for a group)");
+    CK(ctx, cudaMemcpyAsync(G_host + off, Gs + off, bytes, cudaMemcpyDeviceToHost, ctx->copy_stream), "adacgd_compress_host (copy of G to the host)");
   }
   if (mean_out_host) {
     if (launch_mean_rows(Gs, rows, d, Ms, ctx->stream) < 0) return cuda_fail(ctx, "mean over rows");
     ctx->launches += 1;
-    cudaMemcpyAsync(mean_out_host, Ms, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->stream);
+    CK(ctx, cudaMemcpyAsync(mean_out_host, Ms, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_compress_host (copy of the mean to the host)");
   }
-  if (level_host) cudaMemcpyAsync(level_host, ctx->levels, (size_t)rows * 4, cudaMemcpyDeviceToHost, ctx->stream);
-  if (bits_host) cudaMemcpyAsync(bits_host, ctx->bits, (size_t)rows * 8, cudaMemcpyDeviceToHost, ctx->stream);
-  cudaEventRecord(ctx->copy_ev[4], ctx->copy_stream);
-  cudaStreamWaitEvent(ctx->stream, ctx->copy_ev[4], 0);
-  cudaMemcpyAsync(&flags_after, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream);
-  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_compress_host");
+  if (level_host) CK(ctx, cudaMemcpyAsync(level_host, ctx->levels, (size_t)rows * 4, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_compress_host (copy of the levels to the host)");
+  if (bits_host) CK(ctx, cudaMemcpyAsync(bits_host, ctx->bits, (size_t)rows * 8, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_compress_host (copy of the bit counts to the host)");
+  CK(ctx, cudaEventRecord(ctx->copy_ev[4], ctx->copy_stream), "adacgd_compress_host (event after the last copy)");
+  CK(ctx, cudaStreamWaitEvent(ctx->stream, ctx->copy_ev[4], 0), "adacgd_compress_host (waiting for the copy stream)");
+  CK(ctx, cudaMemcpyAsync(&flags_after, ctx->scr.flags, 4, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_compress_host (status words to the host)");
+  CK(ctx, cudaStreamSynchronize(ctx->stream), "adacgd_compress_host (synchronising the stream)");
   if (flags_after & 2u) return fail(ctx, ADACGD_ERR_CUDA, "a device-side wait for an asynchronous copy timed out");
   if ((flags_after & 1u) && !(flags_before & 1u))
     return fail(ctx, ADACGD_ERR_NONFINITE, "an input row held Inf or NaN; its estimator was left unchanged");
@@ -422,12 +444,16 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
   if (!ctx) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (ctx->p.loss == ADACGD_LOSS_NONE) return fail(ctx, ADACGD_ERR_INVALID_ARG, "context has no objective");
   if (!x_dev || !grads_out_dev) return fail(ctx, ADACGD_ERR_INVALID_ARG, "x_dev and grads_out_dev must be non-NULL");
+  {
+    const adacgd_status sd = check_device(ctx, "adacgd_gradient");
+    if (sd != ADACGD_OK) return sd;
+  }
   int r = launch_gradient(ctx->p, ctx->gs, x_dev, grads_out_dev, ctx->stream);
   if (r < 0) return cuda_fail(ctx, "adacgd_gradient");
   ctx->launches += r;
   if (loss_out_host) {
-    cudaMemcpyAsync(loss_out_host, ctx->gs.loss, 8, cudaMemcpyDeviceToHost, ctx->stream);
-    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return cuda_fail(ctx, "adacgd_gradient");
+    CK(ctx, cudaMemcpyAsync(loss_out_host, ctx->gs.loss, 8, cudaMemcpyDeviceToHost, ctx->stream), "adacgd_gradient (copy of the loss to the host)");
+    CK(ctx, cudaStreamSynchronize(ctx->stream), "adacgd_gradient (synchronising the stream)");
   }
   return ADACGD_OK;
 }
@@ -500,11 +526,15 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (c->p.loss == ADACGD_LOSS_NONE) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective");
   if (n_steps < 0) return fail(c, ADACGD_ERR_INVALID_ARG, "n_steps must be >= 0");
+  {
+    const adacgd_status sd = check_device(c, "adacgd_step");
+    if (sd != ADACGD_OK) return sd;
+  }
   const int n = c->p.n;
   std::vector<StepLog> hostlog;
   for (int done = 0; done < n_steps;) {
     const int batch = (n_steps - done < LOG_CAP) ? (n_steps - done) : LOG_CAP;
-    cudaMemsetAsync(&c->counters->log_pos, 0, 4, c->stream);
+    CK(c, cudaMemsetAsync(&c->counters->log_pos, 0, 4, c->stream), "adacgd_step (rewinding the step log)");
     int t = 0;
     // graphs hold the buffer pointers of the step parity they were captured at (always even here,
     // because pairs are replayed whole and single iterations toggle `odd`)
@@ -537,11 +567,11 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
     }
     if (report_host || levels_host) {
       hostlog.resize(batch);
-      cudaMemcpyAsync(hostlog.data(), c->log, sizeof(StepLog) * batch, cudaMemcpyDeviceToHost, c->stream);
+      CK(c, cudaMemcpyAsync(hostlog.data(), c->log, sizeof(StepLog) * batch, cudaMemcpyDeviceToHost, c->stream), "adacgd_step (copy of the step log to the host)");
       if (levels_host)
-        cudaMemcpyAsync(levels_host + (size_t)done * n, c->loglevels, (size_t)batch * n * 4,
-                        cudaMemcpyDeviceToHost, c->stream);
-      if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
+        CK(c, cudaMemcpyAsync(levels_host + (size_t)done * n, c->loglevels, (size_t)batch * n * 4, cudaMemcpyDeviceToHost, c->stream),
+           "adacgd_step (copy of the levels to the host)");
+      CK(c, cudaStreamSynchronize(c->stream), "adacgd_step (synchronising the stream)");
       if (report_host)
         for (int q = 0; q < batch; ++q) {
           adacgd_step_report& rr = report_host[done + q];
@@ -556,8 +586,8 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
   }
   if (report_host || levels_host) {
     unsigned int fl = 0;
-    cudaMemcpyAsync(&fl, c->scr.flags, 4, cudaMemcpyDeviceToHost, c->stream);
-    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_step");
+    CK(c, cudaMemcpyAsync(&fl, c->scr.flags, 4, cudaMemcpyDeviceToHost, c->stream), "adacgd_step (status words to the host)");
+    CK(c, cudaStreamSynchronize(c->stream), "adacgd_step (synchronising the stream)");
     if (fl & 2u) return fail(c, ADACGD_ERR_CUDA, "a device-side wait for an asynchronous copy timed out");
     if (fl & 1u) return fail(c, ADACGD_ERR_NONFINITE, "a gradient or estimator held Inf or NaN");
   }
@@ -582,6 +612,7 @@ static adacgd_status state_ptr(adacgd_ctx* c, int32_t which, void** p, size_t* b
     case ADACGD_STATE_RECHECKS: *p = c->scr.flags + 1; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_FALLBACKS: *p = c->scr.flags + 2; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_LIST_LEVELS: *p = c->scr.flags + 3; *bytes = 4; return ADACGD_OK;
+    case ADACGD_STATE_DEVICE: *p = nullptr; *bytes = 4; return ADACGD_OK;   // host-side value, handled by the caller
     default: return fail(c, ADACGD_ERR_INVALID_ARG, "unknown state item");
   }
   if (!has) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective, hence no iterate state");
@@ -596,8 +627,14 @@ adacgd_status adacgd_get_state(adacgd_ctx* c, int32_t which, void* dst, size_t b
   adacgd_status s = state_ptr(c, which, &p, &want);
   if (s != ADACGD_OK) return s;
   if (bytes != want) return fail(c, ADACGD_ERR_INVALID_ARG, "bytes does not match the item's size");
-  cudaMemcpyAsync(dst, p, bytes, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream);
-  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_get_state");
+  if (which == ADACGD_STATE_DEVICE) {   // needs no device work, so it also answers when another device is current
+    if (dst_is_device) return fail(c, ADACGD_ERR_INVALID_ARG, "ADACGD_STATE_DEVICE is returned to host memory");
+    *(int32_t*)dst = c->device;
+    return ADACGD_OK;
+  }
+  if ((s = check_device(c, "adacgd_get_state")) != ADACGD_OK) return s;
+  CK(c, cudaMemcpyAsync(dst, p, bytes, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream), "adacgd_get_state (copy)");
+  CK(c, cudaStreamSynchronize(c->stream), "adacgd_get_state (synchronising the stream)");
   return ADACGD_OK;
 }
 
@@ -605,15 +642,16 @@ adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, si
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (!src) return fail(c, ADACGD_ERR_INVALID_ARG, "src is NULL");
   if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS ||
-      which == ADACGD_STATE_FALLBACKS || which == ADACGD_STATE_LIST_LEVELS)
+      which == ADACGD_STATE_FALLBACKS || which == ADACGD_STATE_LIST_LEVELS || which == ADACGD_STATE_DEVICE)
     return fail(c, ADACGD_ERR_INVALID_ARG, "this item is read-only");
   void* p;
   size_t want;
   adacgd_status s = state_ptr(c, which, &p, &want);
   if (s != ADACGD_OK) return s;
   if (bytes != want) return fail(c, ADACGD_ERR_INVALID_ARG, "bytes does not match the item's size");
-  cudaMemcpyAsync(p, src, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream);
-  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return cuda_fail(c, "adacgd_set_state");
+  if ((s = check_device(c, "adacgd_set_state")) != ADACGD_OK) return s;
+  CK(c, cudaMemcpyAsync(p, src, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream), "adacgd_set_state (copy)");
+  CK(c, cudaStreamSynchronize(c->stream), "adacgd_set_state (synchronising the stream)");
   return ADACGD_OK;
 }
 
@@ -632,7 +670,8 @@ void adacgd_destroy(adacgd_ctx* ctx) {
 static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
-    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows"};
+    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows",
+    "k_csr_fwd", "k_csc_bwd"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
 
@@ -683,5 +722,16 @@ adacgd_status adacgd_profile_read(adacgd_ctx* c, double* ms_out, int64_t* record
 }
 
 int64_t adacgd_launch_count(const adacgd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+uint64_t adacgd_message_bits(const adacgd_cand* cand, int64_t d) {
+  if (!cand || d < 1 || d >= (1ll << 31)) return 0;
+  if (cand->kind == ADACGD_TOPK ? cand->param < 1 : (cand->kind != ADACGD_QUANT || cand->param < 2 || cand->param > 16)) return 0;
+  CsetDev cs;
+  memset(&cs, 0, sizeof(cs));
+  cs.m = 1;
+  cs.kind[0] = cand->kind;
+  cs.param[0] = cand->param;
+  return level_bits(cs, 1, d);
+}
 
 }  // extern "C"

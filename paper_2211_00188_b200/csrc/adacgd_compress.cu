@@ -13,6 +13,8 @@
 //   - short rows: everything in one CTA per row (k_small_rows).
 // Energies are sums of non-negative exact terms; a comparison whose margin is below the
 // worst-case summation error is redone in exact integer arithmetic.
+#include <mutex>
+
 #include "adacgd_device.cuh"
 
 namespace adacgd {
@@ -533,7 +535,7 @@ __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, 
       simple = __syncthreads_and(simple ? 1 : 0) != 0 && out.kept_idx == nullptr;
       if (simple && ALIGNED) {
         if (live) {   // few chunks (short rows): more rows in flight per thread, the SMs are not full
-          if (gridDim.x < 148 * 2) update_rows_simple<4>(X, G, d, c0, r0, nr, shd, want_mean, acc);
+          if (gridDim.x < 2 * sm_count()) update_rows_simple<4>(X, G, d, c0, r0, nr, shd, want_mean, acc);
           else update_rows_simple<UPD_RB>(X, G, d, c0, r0, nr, shd, want_mean, acc);
         }
         continue;
@@ -1709,24 +1711,49 @@ adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const 
   return ADACGD_OK;
 }
 
+// Tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory.
+void set_compress_kernel_attributes() {
+  cudaFuncSetAttribute(k_hist<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+  cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+  cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
+  cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+  cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
+  cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
+  cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
+}
+
+// One record per device ordinal, filled at the first use of that device by this process.
+const DevProps* current_device() {
+  constexpr int MAX_DEVICES = 64;
+  static DevProps table[MAX_DEVICES];
+  static bool known[MAX_DEVICES] = {false};
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!known[dev]) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return nullptr;
+    set_compress_kernel_attributes();
+    set_small_kernel_attributes();
+    if (cudaGetLastError() != cudaSuccess) return nullptr;
+    table[dev].ordinal = dev;
+    table[dev].sms = sms;
+    known[dev] = true;
+  }
+  return &table[dev];
+}
+
 int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
                     long long d, const CompressOut& out, cudaStream_t stream) {
   int launches = 0;
-  static bool attr_done = false;
-  if (!attr_done) {  // tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory
-    cudaFuncSetAttribute(k_hist<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
-    cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
-    cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
-    cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
-    cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
-    cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
-    cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
-    attr_done = true;
-  }
+  const DevProps* dp = current_device();
+  if (!dp) return -1;
+  const int SMS = dp->sms;
   const bool al = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y) &&
                   (!out.mean_out || aligned16(out.mean_out));
   const long long nchunk = nchunk_of(d);
-  const dim3 ugrid((unsigned)(nchunk < 148 * 4 ? nchunk : 148 * 4));  // persistent: CTAs walk the column chunks
+  const dim3 ugrid((unsigned)(nchunk < SMS * 4 ? nchunk : SMS * 4));  // persistent: CTAs walk the column chunks
   Prof* pf = s.prof;
 #define TIMED(id, ...)             \
   do {                             \
@@ -1764,7 +1791,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   }
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  long long want = (148 * 4 + rows - 1) / rows;   // one wave of the streaming pass: four resident CTAs per SM
+  long long want = (SMS * 4 + rows - 1) / rows;   // one wave of the streaming pass: four resident CTAs per SM
   // a CTA takes at least eight tiles (spread over the row by the grid stride) where the row has them, so
   // that its share of the key list is sized for an average over the row rather than for one tile
   if (single && want > (ntile + 7) / 8) want = (ntile + 7) / 8;
@@ -1775,7 +1802,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const dim3 sgrid(nblk, rows);
   // in single-pass mode the full select only serves rows whose bracket failed: a small grid keeps the
   // usual no-op launches cheap
-  long long want_full = single ? (148 * 2 + rows - 1) / rows : nblk;
+  long long want_full = single ? (SMS * 2 + rows - 1) / rows : nblk;
   if (want_full > nblk) want_full = nblk;
   const int nblk_full = (int)want_full;
   const dim3 fgrid(nblk_full, rows);
@@ -1813,7 +1840,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (win < 1) win = 1;
     if (win > 64) win = 64;
     const long long nwin = (ngran + win - 1) / win;
-    long long sgx = (148 + rows - 1) / rows;          // about one CTA per SM over all rows
+    long long sgx = (SMS + rows - 1) / rows;          // about one CTA per SM over all rows
     const long long per_cta = 49152 / SAMP_G;         // 16-bit per-CTA counters: fewer than 65536 elements each
     if (sgx < (nwin + per_cta - 1) / per_cta) sgx = (nwin + per_cta - 1) / per_cta;
     const long long quads = SAMP_TPB / 4;
@@ -1836,7 +1863,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // 3. exact selection among the listed keys by the digits of key - lo: two passes, each finished by its
     //    last CTA; the third only does work for brackets wider than 2^22 key values
     tol = 1.3 * (4.0 * FLUSH_TILES + 2.0) * 5.9604644775390625e-08;  // binary32 chains of 4*FLUSH_TILES terms
-    long long lgx = (148 * 4 + rows - 1) / rows;       // one wave of CTAs over all rows, each walking its share of the segments
+    long long lgx = (SMS * 4 + rows - 1) / rows;       // one wave of CTAs over all rows, each walking its share of the segments
     if (lgx > LIST_BLK) lgx = LIST_BLK;
     if (lgx > nblk) lgx = nblk;
     const dim3 lgrid((unsigned)lgx, rows);
@@ -1864,7 +1891,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                            s.dec, s.flags, out, s.diffflag, single ? s.tickets : nullptr, tol));
   TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag, d, out, s.tickets, s.flags);
   if (cs.nsel) {
-    long long tgx = (148 * 4 + rows - 1) / rows;
+    long long tgx = (SMS * 4 + rows - 1) / rows;
     if (tgx > nchunk) tgx = nchunk;
     TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk, s.tickets);
   }

@@ -18,6 +18,13 @@ __device__ __forceinline__ void pdl_begin() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// Number of SMs of the device the kernel runs on.
+__device__ __forceinline__ int sm_count() {
+  u32 n;
+  asm("mov.u32 %0, %%nsmid;" : "=r"(n));
+  return (int)n;
+}
+
 __device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
 template <bool ALIGNED>
@@ -133,13 +140,16 @@ __device__ __forceinline__ float quant_value(float v, float L, float inv, float 
 // --------------------------------------------------------------------------
 // level choice (Eq. 11)
 // --------------------------------------------------------------------------
-inline __device__ uint64_t level_bits(const CsetDev& cs, int level, long long d) {
+// Bits of the message of a level (the paper counts communication but prints no formula; this is the
+// library's reading): skip 0; Top-K with K < d: K values of 32 bits with an index of ceil(log2 d) bits
+// each; K >= d: d values; a b-bit quantiser: the 32-bit scale and b bits per entry.  Host and device.
+inline __host__ __device__ uint64_t level_bits(const CsetDev& cs, int level, long long d) {
   if (level == 0) return 0;
   const int c = level - 1;
   if (cs.kind[c] == ADACGD_TOPK) {
     if (cs.param[c] >= d) return 32ull * (uint64_t)d;
-    int idx_bits = 64 - __clzll((unsigned long long)(d - 1));
-    if (d == 1) idx_bits = 1;
+    int idx_bits = 0;
+    while (idx_bits < 63 && (1ll << idx_bits) < d) ++idx_bits;   // ceil(log2 d)
     if (idx_bits < 1) idx_bits = 1;
     return (uint64_t)cs.param[c] * (uint64_t)(32 + idx_bits);
   }

@@ -267,10 +267,13 @@ __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// The split decides the size of the partial-sum buffer, so it is part of the workspace layout and must not
+// depend on the device a context later runs on: it is taken for a nominal 148 SMs.
 static int choose_split(const adacgd_problem& p) {
   if (p.layout == ADACGD_LAYOUT_CSR) return 1;
+  constexpr int NOMINAL_SMS = 148;
   const long long ctas = (long long)p.n * ((p.d + TPB * 4 - 1) / (TPB * 4));
-  long long split = (148 * 4 + ctas - 1) / ctas;
+  long long split = (NOMINAL_SMS * 4 + ctas - 1) / ctas;
   if (split < 1) split = 1;
   if (split > 16) split = 16;
   if (split > p.m_rows) split = p.m_rows;
@@ -322,12 +325,12 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
                     cudaStream_t stream) {
   if (p.layout == ADACGD_LAYOUT_CSR) {
     int launches = 0;
-    prof_begin(g.prof, KID_GRAD_FWD, stream);
+    prof_begin(g.prof, KID_CSR_FWD, stream);
     k_csr_fwd<<<dim3((unsigned)g.loss_blocks, p.n), TPB, 0, stream>>>((const long long*)p.csr_rowptr, p.csr_col, p.csr_val,
                                                                       p.target, x, p.m_rows, p.loss, g.r, g.losspart);
     prof_end(g.prof, stream);
     ++launches;
-    prof_begin(g.prof, KID_GRAD_BWD, stream);
+    prof_begin(g.prof, KID_CSC_BWD, stream);
     k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
                                                                                 p.d, p.m_rows, p.loss, p.lambda, grads);
     prof_end(g.prof, stream);

@@ -33,7 +33,8 @@ constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_COUNT
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD,
+  KID_COUNT
 };
 struct Prof {
   int cap, used;
@@ -47,6 +48,17 @@ inline void prof_begin(Prof* p, int id, cudaStream_t s) {
 inline void prof_end(Prof* p, cudaStream_t s) {
   if (p && p->used < p->cap) { cudaEventRecord(p->end[p->used], s); ++p->used; }
 }
+
+// What the launch code needs to know about the current device.  The first call on a device also raises
+// the dynamic shared memory limit of the kernels that need more than the default (the limit is a
+// per-device attribute).  Returns nullptr when there is no usable current device.
+struct DevProps {
+  int ordinal;
+  int sms;       // streaming multiprocessors: grids are sized in multiples of it
+};
+const DevProps* current_device();
+void set_compress_kernel_attributes();   // adacgd_compress.cu
+void set_small_kernel_attributes();      // adacgd_small.cu
 
 // Candidate set as the kernels see it (passed by value).
 struct CsetDev {

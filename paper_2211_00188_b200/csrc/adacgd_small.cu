@@ -449,15 +449,16 @@ __global__ void __launch_bounds__(TPB) k_small_mean(const float* G, int rows, lo
 }
 
 
+// The row and the tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory.
+void set_small_kernel_attributes() {
+  cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
+  cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
+}
+
 // Enqueues k_small_rows and, if a mean is wanted, k_small_mean; returns the number of launches (< 0: CUDA error).
 int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float* G, const float* Y, int rows,
                       long long d, const CompressOut& out, cudaStream_t stream, bool pdl) {
-  static bool attr_done = false;
-  if (!attr_done) {  // the row and the tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory
-    cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
-    cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
-    attr_done = true;
-  }
+  if (!current_device()) return -1;   // also sets the shared-memory limits at the first use of a device
   Prof* pf = s.prof;
   int launches = 0;
   const size_t shm = 4 * ((size_t)((d + 3) / 4) * 4 + (size_t)(cs.nsel > 1 ? cs.nsel : 1) * BINS2 + SMALL_LIST);

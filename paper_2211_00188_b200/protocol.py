@@ -14,7 +14,7 @@ from __future__ import annotations
 
 from typing import Callable, Dict, Iterable, List, Optional, Sequence, Tuple
 
-from .binding import TOPK
+from .binding import TOPK, message_bits
 
 Cand = Tuple[int, int]
 METHODS = ("gd", "ef21", "lag", "clag", "adacgd")
@@ -49,16 +49,9 @@ def method_set(method: str, d: int, *, K: int = 1, zeta: float = 1.0,
 
 
 def max_bits_per_round(n: int, d: int, cands: Sequence[Cand]) -> int:
-    """Upper bound of the bits n workers send in one round: the weakest compressor of the list."""
-    best = 0
-    for kind, p in cands:
-        if kind == TOPK:
-            idx_bits = max(1, (d - 1).bit_length())
-            b = 32 * d if p >= d else p * (32 + idx_bits)
-        else:
-            b = 32 + p * d
-        best = max(best, b)
-    return n * best
+    """Upper bound of the bits n workers send in one round: the largest message of the list, as the
+    library counts it (adacgd_message_bits)."""
+    return n * max((message_bits(c, d) for c in cands), default=0)
 
 
 def run_to_budget(engine, bit_budget: int, *, max_rounds: int = 1_000_000, batch: int = 64) -> Dict[str, list]:

@@ -228,6 +228,8 @@ def test_argument_errors(torch):
     assert e.value.status == 2
     with pytest.raises(pkg.AdacgdError):
         eng.step(1)
+    # the context reports the device it is bound to (the one that was current at adacgd_init)
+    assert eng.get_state("device") == torch.cuda.current_device() == 0
 
 
 @pytest.mark.parametrize("n", [1, 3, 6])

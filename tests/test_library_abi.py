@@ -111,3 +111,29 @@ def test_binding_fails_loudly_without_gpu():
         pytest.skip("device present")
     with pytest.raises(RuntimeError):
         pkg.AdaCGD(2, 10, [(pkg.TOPK, 1)], 1.0)
+
+
+def test_message_bits_is_exported_and_matches_the_oracle_formula(lib):
+    from oracle import adacgd_oracle as O
+    for d in (1, 2, 3, 8, 9, 1000, 1024, 1025, 25_000_000, 2 ** 31 - 1):
+        for cand in [(B.TOPK, 1), (B.TOPK, 7), (B.TOPK, d), (B.TOPK, d + 5), (B.QUANT, 2), (B.QUANT, 8), (B.QUANT, 16)]:
+            assert B.message_bits(cand, d) == O.message_bits(cand, d), (cand, d)
+    # invalid descriptors give 0, not a crash
+    assert B.message_bits((B.TOPK, 0), 10) == 0 and B.message_bits((B.QUANT, 1), 10) == 0
+    assert B.message_bits((9, 3), 10) == 0 and B.message_bits((B.TOPK, 3), 0) == 0
+    assert lib.adacgd_message_bits(None, 10) == 0
+
+
+def test_init_without_a_device_names_the_failing_call(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("device present")
+    prob = problem()
+    w, k = B._cset([(B.TOPK, 5)], 1.0)
+    nbytes = C.c_size_t(0)
+    assert lib.adacgd_workspace_bytes(C.byref(prob), C.byref(w), None, 0, C.byref(nbytes)) == 0
+    ctx = C.c_void_p()
+    st = lib.adacgd_init(C.byref(ctx), C.byref(prob), C.byref(w), None, None, 1.0, 1, 0, C.c_void_p(4096), nbytes.value, None)
+    assert st == 5 and not ctx.value                       # ADACGD_ERR_CUDA, no context handed out
+    msg = lib.adacgd_last_error(None).decode()
+    assert msg.startswith("adacgd_init (") and ":" in msg, msg   # which call failed, then the runtime's reason
