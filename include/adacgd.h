@@ -186,7 +186,14 @@ adacgd_status adacgd_compress_host(adacgd_ctx* ctx, const float* X_host, float* 
  *   Limits: rows <= ADACGD_NOALLOC_MAX_ROWS, d <= ADACGD_NOALLOC_MAX_D; larger shapes
  *   return ADACGD_ERR_INVALID_ARG (message via adacgd_last_error(NULL)).
  *   X_dev, G_dev, Y_dev, cset, mean_out_dev, level_dev, bits_dev: as in adacgd_compress
- *   (the last three may be NULL); results are identical to adacgd_compress.
+ *   (the last three may be NULL); results are identical to adacgd_compress.  With no
+ *   context there is no status word to read back: a row that holds Inf or NaN is
+ *   reported only through level_dev (level 0) and its untouched row of G, and the call
+ *   still returns ADACGD_OK.
+ *   Cost: the built-in scratch has no room for the key lists of the sampled single-pass
+ *   pipeline, so rows longer than 32 768 entries take the three-pass radix select (about
+ *   44 bytes of traffic per entry and row, against about 21 for adacgd_compress with a
+ *   workspace).
  *   cuda_stream: the cudaStream_t the work is enqueued on (NULL = default stream); the
  *   call does not synchronise.
  *   The first call on each device looks up the array's device address, with the current

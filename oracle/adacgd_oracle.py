@@ -267,13 +267,13 @@ LEAST_SQUARES = 2   # ||A x - b||^2 / (2 m)
 def _matvec64(A, x64):
     if hasattr(A, "tocsr"):
         return np.asarray(A.astype(np.float64) @ x64).ravel()
-    return A.astype(np.float64) @ x64
+    return np.asarray(A, dtype=np.float64) @ x64   # features already held in binary64 are used as they are
 
 
 def _rmatvec64(A, r64):
     if hasattr(A, "tocsr"):
         return np.asarray(A.astype(np.float64).T @ r64).ravel()
-    return A.astype(np.float64).T @ r64
+    return np.asarray(A, dtype=np.float64).T @ r64
 
 
 def local_loss(A, target, x, loss: int, lam: float) -> float:

@@ -1,7 +1,10 @@
 """Parity at the benchmark's full sizes, in the launch configurations bench.py times.  Workload c5
-(8 rows of 25e6 entries): one sampled worker row and the master row are checked against the oracle bit
-for bit, every other row through properties that hold at any size.  Workloads c2, c3, c4: gradients
+(8 rows of 25e6 entries): every worker row and the master row are checked against the oracle bit for bit
+(the oracle rows run in a pool of spawned processes), and through properties that hold at any size.  Workloads c2, c3, c4: gradients
 of sampled workers against the oracle (rel 1e-5) and the selections of an iteration on sampled rows."""
+import multiprocessing as mp
+import os
+
 import numpy as np
 import pytest
 
@@ -57,12 +60,20 @@ def test_c5_full_size_step():
     Gh = G.cpu().numpy()
     assert np.array_equal(gt_new.cpu().numpy().view(np.uint32), O.server_mean(Gh).view(np.uint32))
 
-    # one worker row and the master row against the oracle
-    i = 3
-    ref = O.adacgd(G_before[i].cpu().numpy(), Y[i].cpu().numpy(), X[i].cpu().numpy(), W["worker"], 1.0)
-    assert levels[i] == ref["level"] and int(bits[i]) == ref["bits"]
-    assert np.array_equal(Gh[i].view(np.uint32), ref["out"].view(np.uint32))
-    mref = O.adacgd(gm_before[0].cpu().numpy(), gt_old.cpu().numpy(), gt_new.cpu().numpy(), W["master"], 1.0)
+    # every worker row and the master row against the oracle: level, bits, number of entries written, and the
+    # estimator bit for bit.  The nine oracle calls run side by side in spawned processes (a process forked
+    # after the first CUDA call would not be safe).
+    jobs = [(G_before[i].cpu().numpy(), Y[i].cpu().numpy(), X[i].cpu().numpy(), W["worker"], 1.0) for i in range(n)]
+    jobs.append((gm_before[0].cpu().numpy(), gt_old.cpu().numpy(), gt_new.cpu().numpy(), W["master"], 1.0))
+    with mp.get_context("spawn").Pool(min(len(jobs), max(1, (os.cpu_count() or 2) // 2))) as pool:
+        refs = pool.starmap(O.adacgd, jobs)
+    for i in range(n):
+        ref = refs[i]
+        assert levels[i] == ref["level"] and int(bits[i]) == ref["bits"], (i, levels[i], ref["level"])
+        assert np.array_equal(Gh[i].view(np.uint32), ref["out"].view(np.uint32)), i
+        if ref["kept"] is not None:
+            assert len(ref["kept"]) == W["worker"][ref["level"] - 1][1]
+    mref = refs[n]
     assert int(mlevel.item()) == mref["level"]
     assert np.array_equal(gm[0].cpu().numpy().view(np.uint32), mref["out"].view(np.uint32))
 

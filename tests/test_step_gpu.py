@@ -126,10 +126,12 @@ def test_lockstep_least_squares_and_quantisers(torch):
     lockstep(torch, A, t, 2, 0.0, gamma, [(TOPK, 30), (TOPK, 300)], 2.0, [], 0.0, T=10, g0_mode=2)
 
 
-def free_run(torch, A, t, loss, lam, gamma, wc, wz, mc, mz, T):
+def free_run(torch, A, t, loss, lam, gamma, wc, wz, mc, mz, T, wide=False):
     n, m, d = A.shape
     x0 = np.zeros(d, F32)
     prob = oracle_problem(A, t, loss, lam)
+    if wide:   # long runs: the oracle's binary64 copy of the features is made once instead of at every product
+        prob["A"] = [a.astype(np.float64) for a in prob["A"]]
     st = O.init_state(prob, x0, wc)
     eng = make_engine(torch, A, t, loss, lam, x0, gamma, wc, wz, mc, mz)
     recs, levels = eng.step(T, report=True)
@@ -150,6 +152,37 @@ def test_free_running_c1_loss_trajectory(torch):
     assert eng.get_state("bits_up") == sum(r["bits_up"] for r in recs)
     assert eng.get_state("bits_down") == sum(r["bits_down"] for r in recs)
     assert relerr(eng.get_state("x").cpu().numpy(), st["x"]) <= 1e-2
+
+
+def test_free_running_c2_bidirectional(torch):
+    # workload c2 as benchmarked (20 x 8 000, 2 000 samples per worker, worker and master Top-K {8, 80, 800, 8000}),
+    # both sides left to run on their own for as many of its 1 000 iterations as the oracle does in about two minutes
+    W = S.WORKLOADS["c2"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"], iters=8)
+    T = 400
+    recs, levels, f_ref, f0, st, eng = free_run(torch, A, t, W["loss"], W["lam"], gamma, W["worker"], 1.0, W["master"], 1.0,
+                                                T, wide=True)
+    assert abs(recs[-1]["loss"] - f_ref) <= 1e-3 * abs(f_ref)
+    assert f_ref < 0.9 * f0
+    assert eng.get_state("step") == T
+    assert len({l for lv in levels for l in lv}) >= 2 and len({r["master_level"] for r in recs}) >= 2
+
+
+def test_free_running_c4_shape_scaled(torch):
+    # the shape of workload c4 (least squares, A ~ N(0, 1/d), Top-K {0.1 %, 1 %, 10 %}) at 8 x 100 000 with 64 samples
+    # per worker: large enough for the sampled single-pass pipeline
+    n, d, m = 8, 100_000, 64
+    A, t, _ = S.least_squares_problem(n, d, m, seed=5)
+    gamma = 0.5 / S.smoothness_estimate(A, 2, 0.0, iters=8)
+    wc = [(TOPK, 100), (TOPK, 1000), (TOPK, 10_000)]
+    # n m < d: the minimum of the objective is zero and the loss falls by a factor of about 0.7 per iteration, so
+    # the run is compared where the loss is still far above the resolution of binary32 gradients
+    T = 12
+    recs, levels, f_ref, f0, st, eng = free_run(torch, A, t, 2, 0.0, gamma, wc, 1.0, [], 0.0, T, wide=True)
+    assert abs(recs[-1]["loss"] - f_ref) <= 1e-3 * abs(f_ref)
+    assert f_ref < 0.1 * f0
+    assert eng.get_state("fallbacks") == 0
 
 
 def test_free_running_gd_special_case_matches_closed_form(torch):
@@ -239,6 +272,24 @@ def test_sparse_lockstep_mixed_candidates(torch):
         assert np.array_equal(eng.get_state("gt").cpu().numpy().view(np.uint32), O.server_mean(G_ref).view(np.uint32))
         seen.update(levels[0])
     assert len(seen) >= 2
+
+
+def test_free_running_c3_shape_scaled(torch):
+    # the shape of workload c3 (CSR 1 %, logistic + l2, Top-K and 2/4/8-bit quantisers mixed) at 10 x 20 000 with 100
+    # samples per worker, both sides left to run on their own
+    n, d, m = 10, 20_000, 100
+    wc = [(TOPK, 20), (TOPK, 200), (QUANT, 2), (QUANT, 4), (TOPK, 2000), (QUANT, 8)]
+    gamma = 0.5 / (0.25 + 1e-3)
+    eng, prob, x0 = make_sparse(torch, n, d, m, 0.01, 11, wc, 1.0, gamma=gamma)
+    st = O.init_state(prob, x0, wc)
+    T = 100
+    recs, levels = eng.step(T, report=True)
+    for it in range(T):
+        O.step(st, prob, gamma, wc, 1.0)
+    f_ref, f0 = O.global_loss(prob, st["x"]), O.global_loss(prob, x0)
+    assert abs(recs[-1]["loss"] - f_ref) <= 1e-3 * abs(f_ref)
+    assert f_ref < 0.96 * f0
+    assert len({l for lv in levels for l in lv}) >= 2
 
 
 def test_lockstep_random_sweep(torch):

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 
 import synthetic_inputs as S
+from oracle import adacgd_oracle as O
 
 pytestmark = pytest.mark.gpu
 TOPK, QUANT = 0, 1
@@ -51,6 +52,62 @@ def test_noalloc_matches_workspace_entry_point_on_consecutive_calls():
         assert not np.array_equal(G1, G) or set(l1) == {0}
         levels_seen.update(l1)
     assert len(levels_seen) >= 2
+
+
+def noalloc_against_oracle(torch, pkg, X, G, Y, cands, zeta):
+    dev = torch.device("cuda:0")
+    rows, d = X.shape
+    Xd, Gd, Yd = (torch.from_numpy(a.copy()).to(dev) for a in (X, G, Y))
+    mean = torch.zeros(d, device=dev)
+    level = torch.full((rows,), -1, dtype=torch.int32, device=dev)
+    bits = torch.zeros(rows, dtype=torch.int64, device=dev)
+    pkg.compress_noalloc(Xd, Gd, Yd, cands, zeta, mean_out=mean, level=level, bits=bits)
+    torch.cuda.synchronize()
+    G_ref, res = O.compress_rows(X, G, Y, cands, zeta)
+    assert level.cpu().tolist() == [r["level"] for r in res]
+    assert bits.cpu().tolist() == [r["bits"] for r in res]
+    assert np.array_equal(Gd.cpu().numpy().view(np.uint32), G_ref.view(np.uint32))
+    assert np.array_equal(mean.cpu().numpy().view(np.uint32), O.server_mean(G_ref).view(np.uint32))
+    return [r["level"] for r in res]
+
+
+def test_noalloc_matches_the_oracle_at_the_maximum_shape_and_unaligned():
+    # the largest shape the built-in scratch takes, on heavy-tailed block-scaled rows, then (the scratch now
+    # full of that call's tables) rows whose length is not a multiple of four, with ties and quantisers
+    import torch
+    import paper_2211_00188_b200 as pkg
+
+    n, d = pkg.NOALLOC_MAX_ROWS, pkg.NOALLOC_MAX_D
+    Xs, G0 = S.stress_vectors(n, d, blocks=64, period=4, seed=24, device="cpu")
+    lv = noalloc_against_oracle(torch, pkg, Xs[1].numpy(), G0.numpy(), Xs[0].numpy(),
+                                [(TOPK, d // 1000), (TOPK, d // 100), (TOPK, d // 10)], 1.0)
+    assert any(l > 0 for l in lv)
+    X, G, Y = S.gaussian_rows(3, 100_003, seed=25)
+    X, G, Y = (np.round(a * 64) / 64 for a in (X, G, Y))          # a few equal magnitudes at every threshold
+    lv = noalloc_against_oracle(torch, pkg, X.astype(np.float32), G.astype(np.float32), Y.astype(np.float32),
+                                [(TOPK, 100), (QUANT, 3), (TOPK, 10_000), (QUANT, 8)], 0.3)
+    assert any(l > 0 for l in lv)
+
+
+def test_noalloc_leaves_a_nonfinite_row_unchanged_at_level_zero():
+    # there is no context to hold a status word: a row with Inf or NaN is reported through its level (0)
+    # and an untouched estimator, the other rows are compressed as usual
+    import torch
+    import paper_2211_00188_b200 as pkg
+
+    X, G, Y = S.gaussian_rows(3, 40_000, seed=26)
+    X[1, 77] = np.inf
+    cands = [(TOPK, 40), (TOPK, 4000)]
+    dev = torch.device("cuda:0")
+    Xd, Gd, Yd = (torch.from_numpy(a.copy()).to(dev) for a in (X, G, Y))
+    level = torch.full((3,), -1, dtype=torch.int32, device=dev)
+    pkg.compress_noalloc(Xd, Gd, Yd, cands, 0.0, level=level)
+    torch.cuda.synchronize()
+    got = Gd.cpu().numpy()
+    assert level.cpu().tolist()[1] == 0 and np.array_equal(got[1].view(np.uint32), G[1].view(np.uint32))
+    G_ref, res = O.compress_rows(X[[0, 2]], G[[0, 2]], Y[[0, 2]], cands, 0.0)
+    assert [level.cpu().tolist()[i] for i in (0, 2)] == [r["level"] for r in res] == [2, 2]
+    assert np.array_equal(got[[0, 2]].view(np.uint32), G_ref.view(np.uint32))
 
 
 def test_noalloc_rejects_shapes_beyond_the_builtin_scratch():
