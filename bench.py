@@ -1,19 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the AdaCGD hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5|c4|c2|c1] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--repeats R] [--workload c5|c4|c3|c2|c1] [--impl reference]
 
 One JSON line on stdout (rank 0).  The default workload is the compression-only
 stress c5 (n = 8 rows, d = 25e6): one step = worker-side diff + select + error +
 pick + update + mean over the 8 rows, followed by the master-side compression of
-the d-vector.  The dense workloads (c1, c2, c4) time full iterations a0-a5 of
-Algorithm 1 through adacgd_step.  With --gpus N > 1 (launched by torchrun) every
-rank runs an independent replica of the workload on its own GPU: the path has no
-exchange step on one node, so there is no data-path collective.
+the d-vector.  The timed region of K steps is repeated R times (each repeat bracketed
+by a barrier and a synchronize); `value` is the median repeat, the others are listed.
+The default line also carries `worst_case` (the same workload with the trigger at
+zeta = 0, which forces every row to its weakest compressor, 10 % of the entries) and
+`full_iteration`: workloads c1-c4 timed as whole iterations a0-a5 of Algorithm 1
+through adacgd_step.  With --gpus N > 1 (launched by torchrun) every rank runs an
+independent replica of the workload on its own GPU: the path has no exchange step on
+one node, so there is no data-path collective.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -205,19 +210,59 @@ def run_reference(args):
 # algorithmic bytes per element and row that each streaming kernel of the compression must move
 KERNEL_BYTES = {"k_pass1": 12, "k_update": 8, "k_hist<1>": 8, "k_hist<2>": 8, "k_hist<3>": 8, "k_energy": 12,
                 "k_quant_err": 8}
+NOMINAL_HBM_GBS = 7700.0   # HGX B200 data-sheet figure, for context beside the measured copy bandwidth
 
 
-# DRAM bytes per element and row that ncu counted for these kernels (dram__bytes read + write over
-# one worker launch of workload c5 at half size, 8 x 12.5e6; the traffic grows in proportion to the
-# elements a launch processes).  Valid for the kernels as committed with profiles/c5_compress_step.txt;
-# a kernel that changes afterwards loses its entry until it is captured again.
-NCU_DRAM_BYTES_PER_ELEM = {"k_pass1": 12.10, "k_update": 8.50}
+def counted_traffic(kernel: str):
+    """DRAM bytes per element and row that ncu counted for `kernel` (dram__bytes_read.sum +
+    dram__bytes_write.sum over one launch), from profiles/dram_bytes_per_element.txt.  Each line of that
+    table names the source files the kernel lives in and their hash at the time of the capture: once one of
+    them has changed the figure is stale and None is returned."""
+    path = os.path.join(ROOT, "profiles", "dram_bytes_per_element.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        parts = line.split()
+        if len(parts) < 4 or parts[0] != kernel:
+            continue
+        h = hashlib.sha256()
+        for f in parts[2].split(","):
+            src = os.path.join(ROOT, "paper_2211_00188_b200", "csrc", f)
+            if not os.path.exists(src):
+                return None
+            h.update(open(src, "rb").read())
+        return float(parts[1]) if h.hexdigest()[:16] == parts[3] else None
+    return None
 
 
-def kernel_table(prof):
+def kernel_table(prof, steps):
     tot = sum(v[0] for v in prof.values()) or 1.0
-    return {k: {"ms_total": round(v[0], 4), "launches": v[1], "share": round(v[0] / tot, 4)}
+    return {k: {"ms_total": round(v[0], 4), "launches": v[1], "us_per_step": round(1e3 * v[0] / steps, 2),
+                "share": round(v[0] / tot, 4)}
             for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])}
+
+
+def timed_repeats(run_steps, steps, repeats, world, local):
+    """`repeats` timed regions of exactly `steps` steps, each bracketed by a barrier and a synchronize and
+    timed with CUDA events on the launching stream; the slowest rank sets each repeat's time."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    with ClockSampler(local) as clk:
+        for _ in range(repeats):
+            barrier_sync(world)
+            e0.record()
+            run_steps(steps)
+            e1.record()
+            barrier_sync(world)
+            times.append(max_over_ranks(e0.elapsed_time(e1), world))
+    return times, clk.summary()
+
+
+def repeat_stats(times, steps):
+    per = sorted(t / steps for t in times)
+    return {"n": len(per), "ms_per_step": [round(t, 5) for t in per], "median": float(np.median(per)),
+            "min": per[0], "max": per[-1]}
 
 
 def bench_c5(args, rank, world, local):
@@ -231,69 +276,86 @@ def bench_c5(args, rank, world, local):
         W["master"] = [(k, max(1, int(p * args.scale))) for k, p in W["master"]]
     n, d = W["n"], W["d"]
     dev = torch.device("cuda", local)
-    zeta = args.zeta
-    Xs, G = S.stress_vectors(n, d, W["blocks"], W["period"], seed=rank, device=dev)
-    eng = pkg.AdaCGD(n, d, W["worker"], zeta, W["master"], zeta, host_staging=args.e2e_steps > 0, device=dev)
-    gt = [G.mean(0), torch.empty(d, device=dev)]
-    gm = gt[0].clone().view(1, d)
+    Xs, G0 = S.stress_vectors(n, d, W["blocks"], W["period"], seed=rank, device=dev)
+    eng = pkg.AdaCGD(n, d, W["worker"], args.zeta, W["master"], args.zeta, host_staging=args.e2e_steps > 0, device=dev)
     level = torch.zeros(n, dtype=torch.int32, device=dev)
     bits = torch.zeros(n, dtype=torch.int64, device=dev)
     mlevel = torch.zeros(1, dtype=torch.int32, device=dev)
     P = W["period"]
-
-    def step(t):
-        X, Y = Xs[t % P], Xs[(t - 1) % P]
-        cur, nxt = gt[t % 2], gt[(t + 1) % 2]
-        eng.compress(X, G, Y, mean_out=nxt, level=level, bits=bits)
-        eng.compress(nxt.view(1, d), gm, cur.view(1, d), W["master"], zeta, level=mlevel)
-
-    t = 1
-    for _ in range(args.warmup):
-        step(t)
-        t += 1
-    barrier_sync(world)
-    launches0 = eng.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clk:
-        e0.record()
-        for _ in range(args.steps):
-            step(t)
-            t += 1
-        e1.record()
-        barrier_sync(world)
-    ms = e0.elapsed_time(e1)
-    launches = eng.launch_count() - launches0
-    # the same K steps once more with the library's per-kernel CUDA-event timers switched on
-    eng.profile_enable(64 * args.steps + 64)
-    for _ in range(args.steps):
-        step(t)
-        t += 1
-    prof = eng.profile_read()
-    eng.profile_enable(0)
-    levels_seen = level.cpu().tolist() + mlevel.cpu().tolist()
-    ms = max_over_ranks(ms, world)
+    peak, peak_src = measured_peaks()
     elems_per_step = n * d + d
+    step_floor_bytes = 20 * (n + 1) * d + 4 * d           # 12 B + 8 B per element and row, + the mean
+
+    def run_case(zeta, steps, warmup, repeats):
+        """The step loop at trigger `zeta` from a fresh copy of the start state."""
+        G = G0.clone()
+        gt = [G.mean(0), torch.empty(d, device=dev)]
+        gm = gt[0].clone().view(1, d)
+        state = {"t": 1}
+
+        def run_steps(k):
+            for _ in range(k):
+                t = state["t"]
+                X, Y = Xs[t % P], Xs[(t - 1) % P]
+                cur, nxt = gt[t % 2], gt[(t + 1) % 2]
+                eng.compress(X, G, Y, W["worker"], zeta, mean_out=nxt, level=level, bits=bits)
+                eng.compress(nxt.view(1, d), gm, cur.view(1, d), W["master"], zeta, level=mlevel)
+                state["t"] = t + 1
+
+        run_steps(warmup)
+        launches0 = eng.launch_count()
+        times, clocks = timed_repeats(run_steps, steps, repeats, world, local)
+        launches = (eng.launch_count() - launches0) // repeats
+        # the same K steps once more with the library's per-kernel CUDA-event timers switched on
+        eng.profile_enable(64 * steps + 64)
+        hist = {}
+        for _ in range(steps):
+            run_steps(1)
+            for l in level.cpu().tolist():
+                hist[l] = hist.get(l, 0) + 1
+        prof = eng.profile_read()
+        eng.profile_enable(0)
+        st = repeat_stats(times, steps)
+        step_gbs = step_floor_bytes / (st["median"] * 1e-3) / 1e9
+        return dict(stats=st, clocks=clocks, launches=launches, prof=prof, level_histogram={str(k): v for k, v in sorted(hist.items())},
+                    levels_last_step=level.cpu().tolist() + mlevel.cpu().tolist(),
+                    step_roofline={"algorithmic_bytes_per_step": step_floor_bytes, "achieved_gbs": step_gbs,
+                                   "frac": step_gbs / peak, "frac_of_nominal_7700": step_gbs / NOMINAL_HBM_GBS},
+                    state=(G, gt, gm, state))
+
+    main = run_case(args.zeta, args.steps, args.warmup, args.repeats)
+    ms = main["stats"]["median"] * args.steps
     value = job_throughput(elems_per_step, args.steps, ms, world)
+    prof = main["prof"]
 
     # roofline of the dominant kernel: algorithmic bytes of its launches / its device time
-    peak, peak_src = measured_peaks()
     kern = {k: v for k, v in prof.items() if k in KERNEL_BYTES}
     top = max(kern, key=lambda k: kern[k][0])
     rows_total = (n + 1) * args.steps          # worker launch (n rows) + master launch (1 row) per step
     top_bytes = KERNEL_BYTES[top] * rows_total * d + (4 * d * args.steps if top == "k_update" else 0)
     achieved = top_bytes / (kern[top][0] * 1e-3) / 1e9
-    step_floor_bytes = 20 * (n + 1) * d + 4 * d           # 12 B + 8 B per element and row, + the mean
-    step_gbs = step_floor_bytes / (ms / args.steps * 1e-3) / 1e9
-    per_elem = NCU_DRAM_BYTES_PER_ELEM.get(top)
+    per_elem = counted_traffic(top)
     traffic = None if per_elem is None else per_elem * rows_total * d / kern[top][1]   # bytes per launch, like achieved
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                "launches": kern[top][1], "avg_launch_ms": kern[top][0] / kern[top][1]}
-    step_roofline = {"algorithmic_bytes_per_step": step_floor_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak}
+                "launches": kern[top][1], "avg_launch_ms": kern[top][0] / kern[top][1],
+                "whole_step_frac": main["step_roofline"]["frac"]}
+
+    worst = None
+    if not args.no_extra and args.zeta != 0.0:
+        w = run_case(0.0, args.steps, args.warmup, 3)
+        worst = {"what": "same workload with zeta = 0: no row may skip, every row applies its weakest compressor (10 % of the entries)",
+                 "zeta": 0.0, "ms_per_step": w["stats"]["median"], "repeats": w["stats"],
+                 "compressed_elems_per_s": job_throughput(elems_per_step, 1, w["stats"]["median"], world),
+                 "level_histogram": w["level_histogram"], "levels_last_step": w["levels_last_step"],
+                 "step_roofline": w["step_roofline"], "kernels": kernel_table(w["prof"], args.steps)}
+        del w
 
     # end to end through the host entry point: pinned host buffers, copies inside the timed region
     e2e = None
     if args.e2e_steps > 0:
+        G, gt, gm, state = main["state"]
+        t = state["t"]
         hX = [x.cpu().pin_memory() for x in Xs]
         hG = G.cpu().pin_memory()
         hgt = [gt[0].cpu().pin_memory(), gt[1].cpu().pin_memory()]
@@ -304,8 +366,9 @@ def bench_c5(args, rank, world, local):
         def host_step(tt):
             cur, nxt = hgt[tt % 2], hgt[(tt + 1) % 2]
             eng.compress_host(hX[tt % P], hG, hX[(tt - 1) % P], mean_out=nxt, level=hlevel, bits=hbits)
-            eng.compress_host(nxt.view(1, d), hgm, cur.view(1, d), W["master"], zeta)
+            eng.compress_host(nxt.view(1, d), hgm, cur.view(1, d), W["master"], args.zeta)
 
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         host_step(t)
         barrier_sync(world)
         e0.record()
@@ -319,24 +382,27 @@ def bench_c5(args, rank, world, local):
         e2e = {"value": world * elems_per_step * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "ms_per_step": ems / args.e2e_steps}
-    return dict(value=value, ms=ms, launches=launches, roofline=roofline, step_roofline=step_roofline,
-                kernels=kernel_table(prof), clocks=clk.summary(), e2e=e2e,
-                iters_per_s=world * args.steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"), side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
+    return dict(value=value, ms=ms, launches=main["launches"], roofline=roofline, step_roofline=main["step_roofline"],
+                kernels=kernel_table(prof, args.steps), clocks=main["clocks"], e2e=e2e, repeats=main["stats"], worst_case=worst,
+                iters_per_s=world * args.steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"),
+                side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
                 config={"workload": "c5", "n": n, "d": d, "topk": [p for _, p in W["worker"]],
-                        "master_topk": [p for _, p in W["master"]], "zeta": zeta,
+                        "master_topk": [p for _, p in W["master"]], "zeta": args.zeta,
+                        "levels_last_step": main["levels_last_step"], "level_histogram": main["level_histogram"],
                         "l2": "inputs (3 x %.0f MB per pass) exceed the 126 MB L2; no flush needed" % (n * d * 4 / 1e6),
-                        "levels_last_step": levels_seen, "replicas": world})
+                        "replicas": world})
 
 
-def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
+def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats=None):
     import torch
     import paper_2211_00188_b200 as pkg
 
     W = S.WORKLOADS[name]
-    n, d, m = W["n"], W["d"], W["m"]
+    n, d, m = (args.workers or W["n"]), W["d"], W["m"]
     dev = torch.device("cuda", local)
     steps = steps or args.steps
     warmup = warmup or args.warmup
+    repeats = repeats or args.repeats
     csr = None
     if name == "c4":  # 16.4 GB of features: drawn on the device with the same law
         gen = torch.Generator(device=dev)
@@ -364,16 +430,11 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     eng = pkg.AdaCGD(n, d, W["worker"], 1.0, W["master"], 1.0, loss=W["loss"], lam=W["lam"], A=A, target=tgt,
                      csr=csr, x0=x0, gamma=gamma, device=dev)
     eng.step(warmup)
-    barrier_sync(world)
     launches0 = eng.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clk:
-        e0.record()
-        eng.step(steps)
-        e1.record()
-        barrier_sync(world)
-    ms = max_over_ranks(e0.elapsed_time(e1), world)
-    launches = eng.launch_count() - launches0
+    times, clocks = timed_repeats(lambda k: eng.step(k), steps, repeats, world, local)
+    launches = (eng.launch_count() - launches0) // repeats
+    st = repeat_stats(times, steps)
+    ms = st["median"] * steps
     # the same number of steps once more with the library's per-kernel CUDA-event timers switched on
     eng.profile_enable(80 * steps + 64)
     eng.step(steps)
@@ -385,22 +446,30 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None):
     peak, peak_src = measured_peaks()
     # one pass over the features: dense 4 B per entry; CSR value + column index per stored entry
     a_bytes = 4 * n * m * d if csr is None else 8 * int(csr[1].numel())
-    top = max(("k_dense_fwd", "k_dense_bwd"), key=lambda k: prof[k][0])
+    top = max((k for k in ("k_dense_fwd", "k_dense_bwd", "k_csr_fwd", "k_csc_bwd") if k in prof), key=lambda k: prof[k][0])
     achieved = a_bytes * prof[top][1] / (prof[top][0] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": peak_src, "launches": prof[top][1],
+                "frac": achieved / peak, "traffic": counted_traffic(top), "peak_source": peak_src, "launches": prof[top][1],
                 "avg_launch_ms": prof[top][0] / prof[top][1]}
     floor = 2 * a_bytes + 20 * n * d + (24 * d if W["master"] else 0)
     step_gbs = floor / (ms / steps * 1e-3) / 1e9
-    step_roofline = {"algorithmic_bytes_per_step": floor, "achieved_gbs": step_gbs, "frac": step_gbs / peak}
+    step_roofline = {"algorithmic_bytes_per_step": floor, "achieved_gbs": step_gbs, "frac": step_gbs / peak,
+                     "frac_of_nominal_7700": step_gbs / NOMINAL_HBM_GBS}
+    hist = {}
+    for l in levels[0]:
+        hist[str(l)] = hist.get(str(l), 0) + 1
     return dict(value=value, ms=ms, steps=steps, launches=launches, roofline=roofline, step_roofline=step_roofline,
-                kernels=kernel_table(prof), clocks=clk.summary(), e2e=None,
-                iters_per_s=world * steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"), side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
+                kernels=kernel_table(prof, steps), clocks=clocks, e2e=None, repeats=st, worst_case=None,
+                iters_per_s=world * steps / (ms * 1e-3), rechecks=eng.get_state("rechecks"),
+                side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
                 config={"workload": name, "n": n, "d": d, "m": m, "loss": W["loss"], "gamma": gamma,
-                        "topk": [p for _, p in W["worker"]], "bidirectional": bool(W["master"]),
-                        "loss_after": recs[0]["loss"], "levels_last_step": levels[0],
+                        "cands": [list(c) for c in W["worker"]], "bidirectional": bool(W["master"]),
+                        "loss_after": recs[0]["loss"], "level_histogram_last_step": hist,
                         "l2": ("features (%.2f GB) exceed the 126 MB L2" % (a_bytes / 1e9)) if a_bytes > 2e8
                         else "working set fits in L2 (launch-latency bound workload)", "replicas": world})
+
+
+FULL_ITERATION_RUNS = {"c1": (400, 20), "c2": (200, 20), "c3": (100, 10), "c4": (30, 5)}   # workload: (steps, warm-up)
 
 
 def main():
@@ -408,19 +477,22 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps steps; value is their median")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", choices=["c5", "c4", "c3", "c2", "c1"])
     ap.add_argument("--zeta", type=float, default=1.0)
     ap.add_argument("--scale", type=float, default=1.0, help="shrink d of workload c5 (profiling captures)")
+    ap.add_argument("--workers", type=int, default=0, help="fewer workers for workloads c1-c4 (profiling captures)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extra", action="store_true", help="skip the secondary full-iteration measurement")
+    ap.add_argument("--no-extra", action="store_true", help="skip the worst-case and the full-iteration measurements")
     args = ap.parse_args()
 
     if args.impl == "reference":
         run_reference(args)
         return
     args.warmup = max(args.warmup, 3)
+    args.repeats = max(args.repeats, 1)
 
     import torch
     if not torch.cuda.is_available():
@@ -435,12 +507,17 @@ def main():
 
     extra = None
     if args.workload == "c5" and not args.no_extra and args.scale == 1.0:
-        torch.cuda.empty_cache()
-        r2 = bench_dense(args, "c2", rank, world, local, steps=200, warmup=20)
-        extra = {"workload": "c2", "what": "full iterations a0-a5 through adacgd_step", "iters_per_s": r2["iters_per_s"],
-                 "ms_per_step": r2["ms"] / r2["steps"], "compressed_elems_per_s": r2["value"],
-                 "roofline": r2["roofline"], "step_roofline": r2["step_roofline"], "kernels": r2["kernels"],
-                 "config": r2["config"], "gpu_launches": r2["launches"], "exact_rechecks": r2["rechecks"]}
+        extra = []
+        for name, (steps, warm) in FULL_ITERATION_RUNS.items():
+            torch.cuda.empty_cache()
+            r2 = bench_dense(args, name, rank, world, local, steps=steps, warmup=warm, repeats=3)
+            extra.append({"workload": name, "what": "full iterations a0-a5 through adacgd_step", "steps": steps,
+                          "iters_per_s": r2["iters_per_s"], "ms_per_step": r2["ms"] / r2["steps"], "repeats": r2["repeats"],
+                          "compressed_elems_per_s": r2["value"], "roofline": r2["roofline"],
+                          "step_roofline": r2["step_roofline"], "kernels": r2["kernels"], "config": r2["config"],
+                          "gpu_launches": r2["launches"], "exact_rechecks": r2["rechecks"], "side_paths": r2["side_paths"],
+                          "clocks": r2["clocks"]})
+            del r2
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -452,11 +529,14 @@ def main():
         line = {
             "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": res["config"],
-            "iters_per_s": res["iters_per_s"], "roofline": res["roofline"], "step_roofline": res["step_roofline"],
-            "kernels": res["kernels"], "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"],
-            "exact_rechecks": res["rechecks"], "side_paths": res["side_paths"], "cpu_baseline": cpu,
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "gpu_launches": res["launches"],
+            "config": res["config"], "side_paths": res["side_paths"], "exact_rechecks": res["rechecks"],
+            "repeats": res["repeats"], "iters_per_s": res["iters_per_s"], "roofline": res["roofline"],
+            "step_roofline": res["step_roofline"], "clocks": res["clocks"], "e2e": res["e2e"], "cpu_baseline": cpu,
+            "kernels": res["kernels"],
         }
+        if res["worst_case"]:
+            line["worst_case"] = res["worst_case"]
         if extra:
             line["full_iteration"] = extra
         print(json.dumps(line))

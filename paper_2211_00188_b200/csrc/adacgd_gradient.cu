@@ -236,6 +236,188 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd(const long long* __restrict__ c
   grads[(long long)worker * d + c] = acc + reg_grad(loss, lambda, x[c]);
 }
 
+
+// ---- CSR, column-blocked forward ------------------------------------------------------------------
+// A gathered word of x costs a whole L1 wavefront when it comes from global memory but only a bank
+// access when it comes from shared memory, and the forward pass gathers one word per stored entry.  So the
+// columns are cut into nb blocks of `blk` columns that fit in shared memory; a CTA keeps one block of x
+// there and walks the sample rows of ALL workers (they share x), one warp per row, over the entries of
+// that block only.  Column indices ascend inside a row, so those entries are the contiguous span
+// [split[b][row], split[b+1][row]) found once at init.  zpart[b][row] receives the block's share of
+// a_row . x; k_csr_residual adds the shares in block order.
+constexpr int CSR_BLK_MAX = 49152;   // columns of x per block: 192 KB of shared memory
+constexpr int CSR_FWD_TPB = 1024;
+constexpr int CSR_NB_MAX = 8;        // wider problems take the plain warp-per-row kernel
+constexpr int CSR_FWD_UNR = 6;       // entries a lane requests at once
+
+__global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long* __restrict__ split, const int* __restrict__ col,
+                                                                 const float* __restrict__ val, const float* __restrict__ x,
+                                                                 long long rows, long long d, int blk,
+                                                                 float* __restrict__ zpart) {
+  extern __shared__ __align__(16) float xs[];
+  const int b = blockIdx.y;
+  const long long cbase = (long long)b * blk;
+  const int ncol = (int)((d - cbase < blk) ? (d - cbase) : blk);
+  for (int i = threadIdx.x; i < ncol; i += CSR_FWD_TPB) xs[i] = x[cbase + i];
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const long long* s0 = split + (long long)b * rows;
+  const long long* s1 = split + (long long)(b + 1) * rows;
+  const int cb = (int)cbase;
+  const long long stride = (long long)gridDim.x * (CSR_FWD_TPB / 32);
+  long long row = (long long)blockIdx.x * (CSR_FWD_TPB / 32) + wid;
+  // the span of the next row is requested while the current one is summed
+  long long e0 = 0, e1 = 0;
+  if (row < rows) { e0 = s0[row]; e1 = s1[row]; }
+  for (; row < rows; row += stride) {
+    const long long nrow = row + stride;
+    long long n0 = 0, n1 = 0;
+    if (nrow < rows) { n0 = s0[nrow]; n1 = s1[nrow]; }
+    float acc = 0.f;
+    // CSR_FWD_UNR entries per lane in flight; a lane adds its products in ascending entry order.  Offsets
+    // are 32-bit and relative to the lane's first entry, so that a load is one instruction and its guard.
+    const int* cp = col + e0 + lane;
+    const float* vp = val + e0 + lane;
+    const int cnt = (int)(e1 - e0) - lane;               // this lane owns entries 32 k with 32 k < cnt
+    for (int o = 0; o < cnt; o += 32 * CSR_FWD_UNR) {
+      int c[CSR_FWD_UNR];
+      float v[CSR_FWD_UNR];
+#pragma unroll
+      for (int k = 0; k < CSR_FWD_UNR; ++k) {
+        const bool ok = o + 32 * k < cnt;
+        c[k] = ok ? __ldcs(cp + o + 32 * k) : cb;
+        v[k] = ok ? __ldcs(vp + o + 32 * k) : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < CSR_FWD_UNR; ++k) acc = fmaf(v[k], xs[c[k] - cb], acc);   // absent entries add 0 * xs[0]
+    }
+    acc = warp_sum_f32(acc);
+    if (lane == 0) zpart[(long long)b * rows + row] = acc;
+    e0 = n0; e1 = n1;
+  }
+}
+
+// z = sum over the column blocks (in block order), residual and loss of every sample row.
+__global__ void __launch_bounds__(TPB) k_csr_residual(const float* __restrict__ zpart, int nb, long long rows,
+                                                      const float* __restrict__ target, long long m_rows, int loss,
+                                                      float* __restrict__ r, double* __restrict__ losspart) {
+  const int worker = blockIdx.y;
+  const long long l = (long long)blockIdx.x * TPB + threadIdx.x;
+  double ls = 0.0;
+  if (l < m_rows) {
+    const long long g = (long long)worker * m_rows + l;
+    float z = zpart[g];
+    for (int b = 1; b < nb; ++b) z += zpart[(long long)b * rows + g];
+    float rr;
+    residual(loss, z, target[g], 1.f / (float)m_rows, &rr, &ls);
+    r[g] = rr;
+  }
+  __shared__ double red[TPB / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < TPB / 32; ++w) t += red[w];
+    losspart[(long long)worker * gridDim.x + blockIdx.x] = t;
+  }
+}
+
+// ---- CSR backward on the transposed copy, one contiguous span per warp --------------------------------
+// A warp owns CSC_WCOLS consecutive columns of one worker at a time (two per lane).  Their entries are one contiguous
+// span of the transposed arrays: it is read with coalesced loads, every entry is multiplied by its
+// sample's residual (the worker's residuals sit in shared memory) and the products are parked in the
+// warp's part of shared memory; then each lane adds the products of its columns in ascending sample
+// order, so the sums have a fixed order.  A span that does not fit (the columns hold more than CSC_WPCAP
+// entries) is walked column by column instead.  The warps of a CTA work on their own: the only CTA-wide
+// barrier follows the load of the residuals.
+constexpr int CSC_WCOLS = 64;      // columns a warp takes at a time (two per lane)
+constexpr int CSC_WPCAP = 768;     // products parked per warp
+constexpr int CSC_UNR = 6;         // entries a lane requests at once
+constexpr int CSC_RCAP = 8192;     // residuals of a worker kept in shared memory
+__global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restrict__ wbase, const u32* __restrict__ ptr32,
+                                                      const int* __restrict__ crow, const float* __restrict__ cval,
+                                                      const float* __restrict__ r, const float* __restrict__ x,
+                                                      long long d, long long m_rows, int loss, float lambda,
+                                                      float* __restrict__ grads) {
+  extern __shared__ __align__(16) float bsm[];   // [m_rows] residuals, then [TPB / 32][CSC_WPCAP] products
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  float* rs = bsm;
+  float* prod = bsm + m_rows + (size_t)wid * CSC_WPCAP;
+  const int worker = blockIdx.y;
+  const u32* ptr = ptr32 + (long long)worker * (d + 1);
+  const long long base = wbase[worker];
+  const float* rw = r + (long long)worker * m_rows;
+  for (int i = threadIdx.x; i < (int)m_rows; i += TPB) rs[i] = rw[i];
+  __syncthreads();
+  const long long ngroups = (d + CSC_WCOLS - 1) / CSC_WCOLS;
+  const long long gstride = (long long)gridDim.x * (TPB / 32);
+  // Column pointers and x of a group: this lane's columns c0 + lane and c0 + lane + 32, and the ends of the
+  // warp's span.  The next group's are requested before the current group's entries.
+  struct Grp { u32 pa[2], pb[2], e0, e1; float xv[2]; };
+  auto fetch = [&](long long grp, Grp& q) {
+    const long long c0 = grp * CSC_WCOLS;
+    const long long c1 = (c0 + CSC_WCOLS < d) ? c0 + CSC_WCOLS : d;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const long long c = c0 + lane + 32 * k;
+      const bool ok = c < c1;
+      q.pa[k] = ok ? ptr[c] : 0u;
+      q.pb[k] = ok ? ptr[c + 1] : 0u;
+      q.xv[k] = ok ? x[c] : 0.f;
+    }
+    q.e0 = ptr[c0];
+    q.e1 = ptr[c1];
+  };
+  long long grp = (long long)blockIdx.x * (TPB / 32) + wid;
+  Grp cur, nxt;
+  if (grp < ngroups) fetch(grp, cur);
+  for (; grp < ngroups; grp += gstride) {
+    if (grp + gstride < ngroups) fetch(grp + gstride, nxt);
+    const long long c0 = grp * CSC_WCOLS;
+    const long long c1 = (c0 + CSC_WCOLS < d) ? c0 + CSC_WCOLS : d;
+    const u32 e0 = cur.e0, span = cur.e1 - cur.e0;
+    const int* er = crow + base + e0;
+    const float* ev = cval + base + e0;
+    float acc[2] = {0.f, 0.f};
+    if (span <= (u32)CSC_WPCAP) {
+      const int* erl = er + lane;
+      const float* evl = ev + lane;
+      float* pl = prod + lane;
+      const int cnt = (int)span - lane;                  // this lane owns entries 32 k with 32 k < cnt
+      for (int o = 0; o < cnt; o += 32 * CSC_UNR) {
+        int rr[CSC_UNR];
+        float vv[CSC_UNR];
+#pragma unroll
+        for (int k = 0; k < CSC_UNR; ++k) {
+          const bool ok = o + 32 * k < cnt;
+          rr[k] = ok ? __ldcs(erl + o + 32 * k) : 0;
+          vv[k] = ok ? __ldcs(evl + o + 32 * k) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < CSC_UNR; ++k)
+          if (o + 32 * k < cnt) pl[o + 32 * k] = vv[k] * rs[rr[k]];
+      }
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < 2; ++k)
+        for (u32 j = cur.pa[k] - e0; j < cur.pb[k] - e0; ++j) acc[k] += prod[j];   // empty for columns past the end
+      __syncwarp();
+    } else {
+#pragma unroll
+      for (int k = 0; k < 2; ++k)
+        for (u32 j = cur.pa[k] - e0; j < cur.pb[k] - e0; ++j) acc[k] += ev[j] * rs[er[j]];
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const long long c = c0 + lane + 32 * k;
+      if (c < c1) grads[(long long)worker * d + c] = acc[k] + reg_grad(loss, lambda, cur.xv[k]);
+    }
+    cur = nxt;
+  }
+}
+
 // f(x) = (1/n) sum_i [ (1/m) sum_l loss_l + reg(x) ]  in binary64, fixed summation order.
 __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__ losspart, int n, int blocks,
                                                       long long m_rows, const float* __restrict__ x, long long d,
@@ -286,6 +468,24 @@ static int loss_blocks_of(const adacgd_problem& p) {
   return cta_row_mode(p) ? (int)p.m_rows : (int)((p.m_rows + LOSS_BLOCK_ROWS - 1) / LOSS_BLOCK_ROWS);
 }
 
+// Column blocks of the CSR forward pass (0: the plain kernel) and the route of the backward pass, from
+// the shape alone so that sizing and carving agree.
+static int csr_blocks_of(const adacgd_problem& p) {
+  const long long nb = (p.d + CSR_BLK_MAX - 1) / CSR_BLK_MAX;
+  return nb <= CSR_NB_MAX ? (int)nb : 0;
+}
+static int csr_block_cols(const adacgd_problem& p, int nb) {
+  if (nb == 0) return 0;
+  const long long blk = (p.d + nb - 1) / nb;
+  return (int)((blk + 3) / 4 * 4);
+}
+// Whether the backward pass walks spans (1) or takes one thread per column (0).
+static int csc_cols_per_cta(const adacgd_problem& p) {
+  if (p.m_rows > CSC_RCAP) return 0;
+  const double avg = (double)p.csr_nnz / ((double)p.n * (double)p.d);   // stored entries per column of a worker
+  return avg * CSC_WCOLS <= 0.75 * CSC_WPCAP ? 1 : 0;                    // a warp's span fits its buffer on average
+}
+
 size_t grad_scratch_bytes(const adacgd_problem& p) {
   if (p.loss == ADACGD_LOSS_NONE) return 0;
   size_t o = 0;
@@ -298,6 +498,14 @@ size_t grad_scratch_bytes(const adacgd_problem& p) {
     o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
     o = align_up(o + (size_t)p.csr_nnz * 4, 256);
     o = align_up(o + (size_t)p.csr_nnz * 4, 256);
+    const int nb = csr_blocks_of(p);
+    const size_t rows = (size_t)p.n * p.m_rows;
+    if (nb) {
+      o = align_up(o + (size_t)(nb + 1) * rows * 8, 256);
+      o = align_up(o + (size_t)nb * rows * 4, 256);
+    }
+    o = align_up(o + ((size_t)p.n + 1) * 8, 256);
+    o = align_up(o + (size_t)p.n * ((size_t)p.d + 1) * 4, 256);
   }
   return o;
 }
@@ -313,10 +521,21 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p) {
   g->losspart = (double*)(b + o); o = align_up(o + (size_t)p.n * g->loss_blocks * 8, 256);
   g->loss = (double*)(b + o); o = align_up(o + 8, 256);
   g->csc_ptr = nullptr; g->csc_row = nullptr; g->csc_val = nullptr;
+  g->nb = 0; g->blk = 0; g->csr_split = nullptr; g->zpart = nullptr; g->ccols = 0; g->wbase = nullptr; g->ptr32 = nullptr;
   if (p.layout == ADACGD_LAYOUT_CSR) {
     g->csc_ptr = (long long*)(b + o); o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
     g->csc_row = (int*)(b + o); o = align_up(o + (size_t)p.csr_nnz * 4, 256);
-    g->csc_val = (float*)(b + o);
+    g->csc_val = (float*)(b + o); o = align_up(o + (size_t)p.csr_nnz * 4, 256);
+    g->nb = csr_blocks_of(p);
+    g->blk = csr_block_cols(p, g->nb);
+    const size_t rows = (size_t)p.n * p.m_rows;
+    if (g->nb) {
+      g->csr_split = (long long*)(b + o); o = align_up(o + (size_t)(g->nb + 1) * rows * 8, 256);
+      g->zpart = (float*)(b + o); o = align_up(o + (size_t)g->nb * rows * 4, 256);
+    }
+    g->ccols = csc_cols_per_cta(p);
+    g->wbase = (long long*)(b + o); o = align_up(o + ((size_t)p.n + 1) * 8, 256);
+    g->ptr32 = (u32*)(b + o);
   }
   g->prof = nullptr;
 }
@@ -325,18 +544,49 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
                     cudaStream_t stream) {
   if (p.layout == ADACGD_LAYOUT_CSR) {
     int launches = 0;
-    prof_begin(g.prof, KID_CSR_FWD, stream);
-    k_csr_fwd<<<dim3((unsigned)g.loss_blocks, p.n), TPB, 0, stream>>>((const long long*)p.csr_rowptr, p.csr_col, p.csr_val,
-                                                                      p.target, x, p.m_rows, p.loss, g.r, g.losspart);
-    prof_end(g.prof, stream);
-    ++launches;
+    const DevProps* dp = current_device();
+    if (!dp) return -1;
+    int loss_blocks = g.loss_blocks;
+    if (g.nb) {
+      const long long rows = (long long)p.n * p.m_rows;
+      long long gx = dp->sms / g.nb;            // one 1024-thread CTA per SM over all column blocks
+      if (gx < 1) gx = 1;
+      if (gx > (rows + 31) / 32) gx = (rows + 31) / 32;
+      prof_begin(g.prof, KID_CSR_FWD, stream);
+      k_csr_fwd_blocked<<<dim3((unsigned)gx, g.nb), CSR_FWD_TPB, (size_t)g.blk * 4, stream>>>(
+          g.csr_split, p.csr_col, p.csr_val, x, rows, p.d, g.blk, g.zpart);
+      prof_end(g.prof, stream);
+      ++launches;
+      loss_blocks = (int)((p.m_rows + TPB - 1) / TPB);
+      prof_begin(g.prof, KID_CSR_RES, stream);
+      k_csr_residual<<<dim3((unsigned)loss_blocks, p.n), TPB, 0, stream>>>(g.zpart, g.nb, rows, p.target, p.m_rows, p.loss,
+                                                                           g.r, g.losspart);
+      prof_end(g.prof, stream);
+      ++launches;
+    } else {
+      prof_begin(g.prof, KID_CSR_FWD, stream);
+      k_csr_fwd<<<dim3((unsigned)g.loss_blocks, p.n), TPB, 0, stream>>>((const long long*)p.csr_rowptr, p.csr_col, p.csr_val,
+                                                                        p.target, x, p.m_rows, p.loss, g.r, g.losspart);
+      prof_end(g.prof, stream);
+      ++launches;
+    }
     prof_begin(g.prof, KID_CSC_BWD, stream);
-    k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
-                                                                                p.d, p.m_rows, p.loss, p.lambda, grads);
+    if (g.ccols) {
+      // about eight CTAs per SM over all workers, each walking groups of columns of its worker
+      const long long ngroups = (p.d + CSC_WCOLS - 1) / CSC_WCOLS;
+      long long gx = (8ll * dp->sms + p.n - 1) / p.n;
+      if (gx > (ngroups + TPB / 32 - 1) / (TPB / 32)) gx = (ngroups + TPB / 32 - 1) / (TPB / 32);
+      if (gx < 1) gx = 1;
+      k_csc_bwd_span<<<dim3((unsigned)gx, p.n), TPB, ((size_t)p.m_rows + (size_t)(TPB / 32) * CSC_WPCAP) * 4, stream>>>(
+          g.wbase, g.ptr32, g.csc_row, g.csc_val, g.r, x, p.d, p.m_rows, p.loss, p.lambda, grads);
+    }
+    else
+      k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
+                                                                                  p.d, p.m_rows, p.loss, p.lambda, grads);
     prof_end(g.prof, stream);
     ++launches;
     prof_begin(g.prof, KID_LOSS, stream);
-    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, g.loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
     prof_end(g.prof, stream);
     ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -381,7 +631,8 @@ namespace adacgd {
 // Builds the transposed copy of a CSR problem (host side, once per context): stable counting sort by
 // (worker, column), so that the entries of a column keep ascending sample-row order and the
 // backward sums have a fixed order.  Returns a message on failure, nullptr on success.
-const char* build_csc(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream) {
+const char* build_csc(const adacgd_problem& p, GradScratch* gp, cudaStream_t stream) {
+  GradScratch& g = *gp;
   const long long rows = (long long)p.n * p.m_rows, nnz = p.csr_nnz, cols = (long long)p.n * p.d;
   std::vector<long long> rowptr((size_t)rows + 1), cptr((size_t)cols + 1, 0);
   std::vector<int> col((size_t)nnz), crow((size_t)nnz);
@@ -410,11 +661,42 @@ const char* build_csc(const adacgd_problem& p, const GradScratch& g, cudaStream_
       cval[(size_t)at] = val[(size_t)e];
     }
   }
+  // column pointers relative to each worker's first entry (32 bits: half the pointer traffic of the backward pass)
+  std::vector<long long> wbase((size_t)p.n + 1);
+  std::vector<u32> ptr32((size_t)p.n * ((size_t)p.d + 1));
+  for (long long w = 0; w <= p.n; ++w) wbase[(size_t)w] = cptr[(size_t)(w * p.d)];
+  for (long long w = 0; w < p.n; ++w) {
+    if (wbase[(size_t)w + 1] - wbase[(size_t)w] >= (1ll << 32)) g.ccols = 0;   // would not fit: one thread per column instead
+    for (long long c = 0; c <= p.d; ++c)
+      ptr32[(size_t)(w * (p.d + 1) + c)] = (u32)(cptr[(size_t)(w * p.d + c)] - wbase[(size_t)w]);
+  }
+  // first entry of every column block inside every sample row (needs ascending columns inside a row)
+  std::vector<long long> split;
+  if (g.nb) {
+    split.resize((size_t)(g.nb + 1) * (size_t)rows);
+    for (long long r = 0; r < rows && g.nb; ++r) {
+      long long e = rowptr[(size_t)r];
+      const long long e1 = rowptr[(size_t)r + 1];
+      for (long long q = e + 1; q < e1; ++q)
+        if (col[(size_t)q] < col[(size_t)q - 1]) { g.nb = 0; break; }   // unsorted row: the plain forward kernel
+      if (!g.nb) break;
+      for (int b = 0; b <= g.nb; ++b) {
+        const long long first_col = (long long)b * g.blk;
+        while (e < e1 && col[(size_t)e] < first_col) ++e;
+        split[(size_t)b * (size_t)rows + (size_t)r] = (b == g.nb) ? e1 : e;
+      }
+    }
+  }
   if (cudaMemcpyAsync(g.csc_ptr, cptr.data(), (cols + 1) * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.csc_row, crow.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.csc_val, cval.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(g.wbase, wbase.data(), wbase.size() * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(g.ptr32, ptr32.data(), ptr32.size() * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      (g.nb && cudaMemcpyAsync(g.csr_split, split.data(), split.size() * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
       cudaStreamSynchronize(stream) != cudaSuccess)
     return "copying the transposed arrays to the device failed";
+  if (g.nb) cudaFuncSetAttribute(k_csr_fwd_blocked, cudaFuncAttributeMaxDynamicSharedMemorySize, CSR_BLK_MAX * 4);
+  if (g.ccols) cudaFuncSetAttribute(k_csc_bwd_span, cudaFuncAttributeMaxDynamicSharedMemorySize, (CSC_RCAP + (TPB / 32) * CSC_WPCAP) * 4);
   return nullptr;
 }
 

@@ -33,7 +33,7 @@ constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD,
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD, KID_CSR_RES,
   KID_COUNT
 };
 struct Prof {
@@ -169,13 +169,22 @@ struct GradScratch {
   long long* csc_ptr;   // [n*d + 1]
   int* csc_row;         // [nnz] sample row inside the worker
   float* csc_val;       // [nnz]
+  // column-blocked forward: the entries of sample row g whose column lies in block b are
+  // [csr_split[b*rows + g], csr_split[(b+1)*rows + g]); zpart[b*rows + g] is that block's share of a_g . x
+  int nb, blk;          // column blocks and columns per block (nb = 0: plain warp-per-row kernel)
+  long long* csr_split; // [(nb+1)][n*m_rows]
+  float* zpart;         // [nb][n*m_rows]
+  // span backward: column pointers relative to the worker's first entry
+  int ccols;            // 1: contiguous spans per warp; 0: one thread per column on csc_ptr
+  long long* wbase;     // [n+1] first transposed entry of every worker
+  u32* ptr32;           // [n][d+1]
   Prof* prof;
 };
 size_t grad_scratch_bytes(const adacgd_problem& p);
 void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p);
 int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
                     cudaStream_t stream);
-const char* build_csc(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream);
+const char* build_csc(const adacgd_problem& p, GradScratch* g, cudaStream_t stream);
 
 // x <- x - gamma * g  (two binary32 roundings: the product, then the difference)
 int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof);

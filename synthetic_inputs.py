@@ -100,6 +100,25 @@ def sparse_logistic_problem(n, d, m, density=0.01, seed=0, flip=0.05):
     return rowptr, col, val, y
 
 
+def sparse_problem_with_dense_columns(n, d, m, dense_cols=64, extra=16, seed=0):
+    """CSR classification data whose first `dense_cols` columns are stored in every sample row while
+    every row has only `extra` more columns, drawn uniformly from the rest: a few very long columns
+    next to many short ones.  Values ~ U(0,1), labels +-1 uniformly.  Same return layout as
+    `sparse_logistic_problem`."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    k = dense_cols + extra
+    rowptr = np.tile(np.arange(0, (m + 1) * k, k, dtype=np.int64), (n, 1))
+    col = np.empty((n, m * k), dtype=np.int32)
+    val = rng.random((n, m * k)).astype(F32)
+    y = np.where(rng.random((n, m)) < 0.5, -1.0, 1.0).astype(F32)
+    head = np.arange(dense_cols, dtype=np.int32)
+    for i in range(n):
+        for r in range(m):
+            tail = np.sort(rng.choice(d - dense_cols, size=extra, replace=False)).astype(np.int32) + dense_cols
+            col[i, r * k:(r + 1) * k] = np.concatenate([head, tail])
+    return rowptr, col, val, y
+
+
 def stress_vectors(n, d, blocks=100, period=4, seed=0, device="cpu"):
     """Gradient-like rows for the compression-only workload.
 

@@ -252,6 +252,54 @@ def test_sparse_gradient_and_loss(torch):
     assert abs(f - O.global_loss(prob, x)) <= 1e-6 * abs(O.global_loss(prob, x))
 
 
+def sparse_engine_and_oracle(torch, rowptr, col, val, y, d, lam=1e-3):
+    import scipy.sparse as sp
+    import paper_2211_00188_b200 as pkg
+    n, m = y.shape
+    dev = torch.device("cuda:0")
+    csr = tuple(torch.from_numpy(a).to(dev) for a in S.csr_global(rowptr, col, val))
+    eng = pkg.AdaCGD(n, d, [(TOPK, 1)], 0.0, loss=1, lam=lam, csr=csr, target=torch.from_numpy(y).to(dev),
+                     x0=torch.zeros(d, device=dev), gamma=1.0)
+    A = [sp.csr_matrix((val[i], col[i], rowptr[i]), shape=(m, d)) for i in range(n)]
+    return eng, dict(A=A, target=[y[i] for i in range(n)], loss=1, lam=lam)
+
+
+@pytest.mark.parametrize("shape", ["two_column_blocks", "three_column_blocks_ragged", "long_columns", "many_samples", "dense", "very_wide"])
+def test_sparse_gradient_kernel_routes(torch, shape):
+    # the routes of the sparse gradient pair: forward with x cut into several shared-memory blocks (d above 49 152),
+    # backward spans that do not fit a CTA's buffer (a few columns stored in every row), more samples per worker than
+    # the backward kernel keeps residuals for (plain kernels), and columns too long on average for spans at all
+    if shape == "two_column_blocks":
+        n, d, m = 2, 60_000, 24
+        data = S.sparse_logistic_problem(n, d, m, density=0.01, seed=61)
+    elif shape == "three_column_blocks_ragged":
+        n, d, m = 3, 100_003, 9
+        data = S.sparse_logistic_problem(n, d, m, density=0.002, seed=62)
+    elif shape == "long_columns":
+        n, d, m = 2, 50_000, 300
+        data = S.sparse_problem_with_dense_columns(n, d, m, dense_cols=64, extra=16, seed=63)
+    elif shape == "many_samples":
+        n, d, m = 2, 2_000, 9_000
+        data = S.sparse_logistic_problem(n, d, m, density=0.005, seed=64)
+    elif shape == "very_wide":
+        n, d, m = 2, 400_000, 6      # more column blocks than the blocked forward kernel takes: one warp per row
+        data = S.sparse_logistic_problem(n, d, m, density=1e-4, seed=67)
+    else:
+        n, d, m = 2, 300, 400
+        data = S.sparse_logistic_problem(n, d, m, density=0.3, seed=65)
+    rowptr, col, val, y = data
+    eng, prob = sparse_engine_and_oracle(torch, rowptr, col, val, y, d)
+    x = (0.5 * np.random.Generator(np.random.PCG64(66)).standard_normal(d)).astype(F32)
+    out = torch.zeros(n, d, device="cuda:0")
+    f = eng.gradient(torch.from_numpy(x).cuda(), out, want_loss=True)
+    want = O.all_gradients(prob, x)
+    got = out.cpu().numpy()
+    for i in range(n):
+        assert relerr(got[i], want[i]) <= 1e-5, (i, relerr(got[i], want[i]))
+        assert np.abs(got[i] - want[i]).max() <= 1e-5 * np.abs(want[i]).max()
+    assert abs(f - O.global_loss(prob, x)) <= 1e-6 * abs(O.global_loss(prob, x))
+
+
 def test_sparse_lockstep_mixed_candidates(torch):
     # the candidate mix of workload c3 (Top-K and 2/4/8-bit quantisers in the user's order), scaled down
     n, d, m = 6, 4000, 50
