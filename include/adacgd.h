@@ -104,6 +104,8 @@ typedef struct {
 } adacgd_problem; /* device arrays are BORROWED for the lifetime of the context */
 
 #define ADACGD_FLAG_HOST_STAGING 1 /* reserve device staging so that adacgd_compress_host can be used */
+#define ADACGD_FLAG_INCREMENTAL_FORWARD 2 /* dense layout only: reserve a column-major copy of A (as large as A) and
+                                             keep z_i = A_i x between iterations; see adacgd_set_refresh_period */
 
 /* Bytes of device workspace adacgd_init needs for this problem and these sets.
  * adacgd_compress later accepts any shape with rows <= n and d <= problem->d.
@@ -139,6 +141,17 @@ typedef struct {
  * Synchronises the stream iff a host pointer is given. */
 adacgd_status adacgd_step(adacgd_ctx* ctx, int32_t n_steps, adacgd_step_report* report_host,
                           int32_t* levels_host);
+
+/* Incremental forward pass (contexts created with ADACGD_FLAG_INCREMENTAL_FORWARD).  Algorithm 1 moves the
+ * iterate by x^{t+1} = x^t - gamma g^t, so z_i = A_i x moves by -gamma A_i g^t, and g^t differs from g^{t-1}
+ * only in the entries some worker's message touched (identity master: g is the mean of the estimators) or the
+ * master's message touched (Algorithm 2).  adacgd_step then keeps z_i and u_i = A_i g and advances them by the
+ * changed entries alone, u_i += sum_c A_i[:, c] (g^t[c] - g^{t-1}[c]) and z_i <- fl(z_i - fl(gamma u_i)), instead
+ * of reading A for z_i = A_i x; the backward product A_i^T r is unchanged.  Rounding makes the kept z_i drift from
+ * A_i x, so every `period` iterations (and after any adacgd_set_state) both products are recomputed in full.
+ * period >= 1; 1 recomputes every iteration; the default is 16, which keeps the gradients within the 1e-5
+ * relative agreement the library is tested to.  Returns ADACGD_ERR_INVALID_ARG for a context without the flag. */
+adacgd_status adacgd_set_refresh_period(adacgd_ctx* ctx, int32_t period);
 
 /* Stages a2-a4 (and the mean of a5) on caller arrays: for every row i
  *     G_i <- AdaCGD_{h=G_i, y=Y_i}(X_i)      (Eq. 11 with EF21 candidates, Eq. 7)
@@ -236,6 +249,10 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
                                    that went through the three-level passes over the key lists, since init (get only) */
 #define ADACGD_STATE_DEVICE 13  /* int32: ordinal of the CUDA device the context is bound to (the device that was
                                    current at adacgd_init); host destination only (get only) */
+#define ADACGD_STATE_INC_COLUMNS 14 /* uint64: columns of A the incremental forward passes have gathered since init,
+                                      summed over iterations (each counts once per worker) (get only) */
+#define ADACGD_STATE_REFRESHES 15  /* uint64: iterations since init whose forward products were recomputed in full;
+                                      host destination only (get only) */
 adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,
                                int32_t dst_is_device);
 adacgd_status adacgd_set_state(adacgd_ctx* ctx, int32_t which, const void* src, size_t bytes,

@@ -12,14 +12,15 @@ TOPK, QUANT = 0, 1
 LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE = 0, 1, 2, 3
 LAYOUT_DENSE, LAYOUT_CSR = 0, 1
 FLAG_HOST_STAGING = 1
-STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11, list_levels=12, device=13)
+FLAG_INCREMENTAL_FORWARD = 2
+STATE = dict(x=0, G=1, grad=2, gt=3, gm=4, step=5, bits_up=6, bits_down=7, levels=8, flags=9, rechecks=10, fallbacks=11, list_levels=12, device=13, inc_columns=14, refreshes=15)
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "BAD_ORDER", 3: "NONFINITE", 4: "WORKSPACE", 5: "CUDA", 6: "UNSUPPORTED"}
 
 EXPORTED_SYMBOLS = [
     "adacgd_workspace_bytes", "adacgd_init", "adacgd_step", "adacgd_compress", "adacgd_compress_host",
     "adacgd_gradient", "adacgd_get_state", "adacgd_set_state", "adacgd_last_error", "adacgd_destroy",
     "adacgd_launch_count", "adacgd_profile_kernel_count", "adacgd_profile_kernel_name", "adacgd_profile_enable",
-    "adacgd_profile_read", "adacgd_compress_noalloc", "adacgd_message_bits",
+    "adacgd_profile_read", "adacgd_compress_noalloc", "adacgd_message_bits", "adacgd_set_refresh_period",
 ]
 
 Cand = Tuple[int, int]
@@ -84,6 +85,7 @@ def load_library():
     lib.adacgd_launch_count.argtypes = [vp]
     lib.adacgd_launch_count.restype = i64
     lib.adacgd_compress_noalloc.argtypes = [vp, vp, vp, i32, i64, C.POINTER(_Cset), vp, vp, vp, vp]
+    lib.adacgd_set_refresh_period.argtypes = [vp, i32]
     lib.adacgd_message_bits.argtypes = [C.POINTER(_Cand), i64]
     lib.adacgd_message_bits.restype = C.c_uint64
     lib.adacgd_profile_kernel_count.argtypes = []
@@ -125,7 +127,7 @@ class AdaCGD:
     def __init__(self, n: int, d: int, worker: Sequence[Cand] = (), worker_zeta: float = 0.0,
                  master: Sequence[Cand] = (), master_zeta: float = 0.0, *, loss: int = LOSS_NONE,
                  lam: float = 0.0, A=None, target=None, csr=None, x0=None, gamma: float = 1.0, g0_mode: int = 1,
-                 host_staging: bool = False, device="cuda:0", stream=None):
+                 host_staging: bool = False, incremental_forward: bool = False, device="cuda:0", stream=None):
         import torch
 
         self.torch = torch
@@ -155,7 +157,7 @@ class AdaCGD:
                 assert tuple(A.shape) == (n, m_rows, d)
         self.problem = _Problem(loss, float(lam), self.n, layout, self.d, m_rows, _ptr(A) if A is not None else None,
                                 _ptr(target) if target is not None else None, _ptr(rowptr), _ptr(col), _ptr(val), nnz)
-        self.flags = FLAG_HOST_STAGING if host_staging else 0
+        self.flags = (FLAG_HOST_STAGING if host_staging else 0) | (FLAG_INCREMENTAL_FORWARD if incremental_forward else 0)
         wcs, k1 = _cset(self.worker, worker_zeta)
         mcs, k2 = _cset(self.master, master_zeta)
         nbytes = C.c_size_t(0)
@@ -248,6 +250,10 @@ class AdaCGD:
         else:
             buf = C.c_uint64(int(value))
             self._check(self.lib.adacgd_set_state(self.ctx, STATE[which], C.byref(buf), 8, 0), self.ctx)
+
+    def set_refresh_period(self, period: int):
+        """adacgd_set_refresh_period: iterations between full recomputations of the kept forward products."""
+        self._check(self.lib.adacgd_set_refresh_period(self.ctx, int(period)), self.ctx)
 
     def profile_enable(self, max_records: int):
         self._check(self.lib.adacgd_profile_enable(self.ctx, int(max_records)), self.ctx)

@@ -39,7 +39,7 @@ WsLayout ws_layout(const adacgd_problem& p, bool master_compresses, int flags) {
   size_t o = 0;
   const size_t nd = (size_t)p.n * (size_t)p.d * 4, dd = (size_t)p.d * 4;
   L.scratch = o; o = align_up(o + scratch_bytes(p.n, p.d, true), 256);
-  L.grad = o; o = align_up(o + grad_scratch_bytes(p), 256);
+  L.grad = o; o = align_up(o + grad_scratch_bytes(p, flags), 256);
   L.levels = o; o = align_up(o + (size_t)p.n * 4, 256);
   L.bits = o; o = align_up(o + (size_t)p.n * 8, 256);
   L.mlevel = o; o = align_up(o + 4, 256);
@@ -156,6 +156,11 @@ struct adacgd_ctx {
   long long pair_launches;
   bool graph_tried;
   bool odd;                    // parity of the iterations run since the graph's reference state
+  // incremental forward pass: z_i = A_i x and u_i = A_i g live in the workspace
+  int refresh_period;          // iterations between full recomputations
+  int since_refresh;           // iterations run since the last one
+  bool inc_dirty;              // the kept products do not belong to the current x and g (fresh context, set_state)
+  unsigned long long refreshes;
   Prof* prof;
   Prof prof_store;
   std::vector<cudaEvent_t> ev_beg, ev_end;
@@ -258,6 +263,10 @@ static adacgd_status init_body(adacgd_ctx* c, const adacgd_problem* problem, con
   c->pair_launches = 0;
   c->graph_tried = false;
   c->odd = false;
+  c->refresh_period = 16;
+  c->since_refresh = 0;
+  c->inc_dirty = true;
+  c->refreshes = 0;
   c->prof = nullptr;
   c->copy_stream = nullptr;
   for (cudaEvent_t& e : c->copy_ev) e = nullptr;
@@ -288,7 +297,9 @@ static adacgd_status init_body(adacgd_ctx* c, const adacgd_problem* problem, con
   CK(nullptr, cudaMemsetAsync(c->scr.flags, 0, 16, c->stream), "adacgd_init (clearing the status words)");
   CK(nullptr, cudaMemsetAsync(c->counters, 0, sizeof(Counters), c->stream), "adacgd_init (clearing the counters)");
   if (has_loss) {
-    carve_grad_scratch(&c->gs, b + L.grad, *problem);
+    carve_grad_scratch(&c->gs, b + L.grad, *problem, flags);
+    if (c->gs.inc && build_transposed_features(*problem, c->gs, c->stream) < 0)
+      return cuda_fail(nullptr, "adacgd_init (column-major copy of the features)");
     if (problem->layout == ADACGD_LAYOUT_CSR) {
       const char* why = build_csc(*problem, &c->gs, c->stream);
       if (why) return fail(nullptr, ADACGD_ERR_INVALID_ARG, why);
@@ -458,8 +469,9 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
   return ADACGD_OK;
 }
 
-// Enqueues one iteration a0..a5 on the context's stream.
-static adacgd_status enqueue_iteration(adacgd_ctx* c) {
+// Enqueues one iteration a0..a5 on the context's stream.  `capturing`: the iteration is being recorded into the
+// graph of incremental iterations, so it takes the incremental forward pass and leaves the refresh counters alone.
+static adacgd_status enqueue_iteration(adacgd_ctx* c, bool capturing = false) {
   const int n = c->p.n;
   const long long d = c->p.d;
   // a0: x^{t+1} = x^t - gamma g^t
@@ -467,7 +479,16 @@ static adacgd_status enqueue_iteration(adacgd_ctx* c) {
   if (r < 0) return cuda_fail(c, "x update");
   c->launches += r;
   // a1: X_i = grad f_i(x^{t+1})
-  r = launch_gradient(c->p, c->gs, c->x, c->grad_nxt, c->stream);
+  if (c->gs.inc) {
+    const bool refresh = !capturing && (c->inc_dirty || c->since_refresh + 1 >= c->refresh_period);
+    r = launch_gradient_incremental(c->p, c->gs, c->x, c->gm, c->gamma, refresh, c->grad_nxt, c->stream);
+    if (!capturing) {
+      if (refresh) { c->since_refresh = 0; c->inc_dirty = false; c->refreshes += 1; }
+      else c->since_refresh += 1;
+    }
+  } else {
+    r = launch_gradient(c->p, c->gs, c->x, c->grad_nxt, c->stream);
+  }
   if (r < 0) return cuda_fail(c, "gradient");
   c->launches += r;
   // a2-a4 and the mean of a5: h = g~_i^t, y = grad f_i(x^t), x = grad f_i(x^{t+1})
@@ -505,8 +526,8 @@ static void try_capture_pair(adacgd_ctx* c) {
     cudaGetLastError();
     return;
   }
-  adacgd_status s1 = enqueue_iteration(c);
-  adacgd_status s2 = (s1 == ADACGD_OK) ? enqueue_iteration(c) : s1;
+  adacgd_status s1 = enqueue_iteration(c, true);
+  adacgd_status s2 = (s1 == ADACGD_OK) ? enqueue_iteration(c, true) : s1;
   const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
   c->pair_launches = c->launches - before;
   c->launches = before;
@@ -554,16 +575,21 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
       }
       if (!c->odd) try_capture_pair(c);
     }
-    if (use_graph && c->pair_exec && !c->odd) {
-      for (; t + 2 <= batch; t += 2) {
+    while (t < batch) {
+      // a recorded pair holds two incremental iterations: it is replayed while no refresh falls inside it
+      const bool pair_ok = use_graph && c->pair_exec && !c->odd && t + 2 <= batch &&
+                           (!c->gs.inc || (!c->inc_dirty && c->since_refresh + 2 < c->refresh_period));
+      if (pair_ok) {
         if (cudaGraphLaunch(c->pair_exec, c->stream) != cudaSuccess) return cuda_fail(c, "graph launch");
         c->launches += c->pair_launches;
+        if (c->gs.inc) c->since_refresh += 2;
+        t += 2;
+      } else {
+        adacgd_status s = enqueue_iteration(c);
+        if (s != ADACGD_OK) return s;
+        c->odd = !c->odd;
+        ++t;
       }
-    }
-    for (; t < batch; ++t) {
-      adacgd_status s = enqueue_iteration(c);
-      if (s != ADACGD_OK) return s;
-      c->odd = !c->odd;
     }
     if (report_host || levels_host) {
       hostlog.resize(batch);
@@ -613,6 +639,10 @@ static adacgd_status state_ptr(adacgd_ctx* c, int32_t which, void** p, size_t* b
     case ADACGD_STATE_FALLBACKS: *p = c->scr.flags + 2; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_LIST_LEVELS: *p = c->scr.flags + 3; *bytes = 4; return ADACGD_OK;
     case ADACGD_STATE_DEVICE: *p = nullptr; *bytes = 4; return ADACGD_OK;   // host-side value, handled by the caller
+    case ADACGD_STATE_REFRESHES: *p = nullptr; *bytes = 8; return ADACGD_OK;   // host-side value
+    case ADACGD_STATE_INC_COLUMNS:
+      if (!c->gs.inc) return fail(c, ADACGD_ERR_INVALID_ARG, "context was created without ADACGD_FLAG_INCREMENTAL_FORWARD");
+      *p = c->gs.inc_cols; *bytes = 8; return ADACGD_OK;
     default: return fail(c, ADACGD_ERR_INVALID_ARG, "unknown state item");
   }
   if (!has) return fail(c, ADACGD_ERR_INVALID_ARG, "context has no objective, hence no iterate state");
@@ -632,6 +662,11 @@ adacgd_status adacgd_get_state(adacgd_ctx* c, int32_t which, void* dst, size_t b
     *(int32_t*)dst = c->device;
     return ADACGD_OK;
   }
+  if (which == ADACGD_STATE_REFRESHES) {
+    if (dst_is_device) return fail(c, ADACGD_ERR_INVALID_ARG, "ADACGD_STATE_REFRESHES is returned to host memory");
+    *(uint64_t*)dst = c->refreshes;
+    return ADACGD_OK;
+  }
   if ((s = check_device(c, "adacgd_get_state")) != ADACGD_OK) return s;
   CK(c, cudaMemcpyAsync(dst, p, bytes, dst_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->stream), "adacgd_get_state (copy)");
   CK(c, cudaStreamSynchronize(c->stream), "adacgd_get_state (synchronising the stream)");
@@ -642,7 +677,8 @@ adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, si
   if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
   if (!src) return fail(c, ADACGD_ERR_INVALID_ARG, "src is NULL");
   if (which == ADACGD_STATE_FLAGS || which == ADACGD_STATE_LEVELS || which == ADACGD_STATE_RECHECKS ||
-      which == ADACGD_STATE_FALLBACKS || which == ADACGD_STATE_LIST_LEVELS || which == ADACGD_STATE_DEVICE)
+      which == ADACGD_STATE_FALLBACKS || which == ADACGD_STATE_LIST_LEVELS || which == ADACGD_STATE_DEVICE ||
+      which == ADACGD_STATE_INC_COLUMNS || which == ADACGD_STATE_REFRESHES)
     return fail(c, ADACGD_ERR_INVALID_ARG, "this item is read-only");
   void* p;
   size_t want;
@@ -650,8 +686,17 @@ adacgd_status adacgd_set_state(adacgd_ctx* c, int32_t which, const void* src, si
   if (s != ADACGD_OK) return s;
   if (bytes != want) return fail(c, ADACGD_ERR_INVALID_ARG, "bytes does not match the item's size");
   if ((s = check_device(c, "adacgd_set_state")) != ADACGD_OK) return s;
+  c->inc_dirty = true;   // the kept forward products no longer belong to the state
   CK(c, cudaMemcpyAsync(p, src, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream), "adacgd_set_state (copy)");
   CK(c, cudaStreamSynchronize(c->stream), "adacgd_set_state (synchronising the stream)");
+  return ADACGD_OK;
+}
+
+adacgd_status adacgd_set_refresh_period(adacgd_ctx* c, int32_t period) {
+  if (!c) return fail(nullptr, ADACGD_ERR_INVALID_ARG, "ctx is NULL");
+  if (!c->gs.inc) return fail(c, ADACGD_ERR_INVALID_ARG, "context was created without ADACGD_FLAG_INCREMENTAL_FORWARD (dense layout)");
+  if (period < 1) return fail(c, ADACGD_ERR_INVALID_ARG, "period must be >= 1");
+  c->refresh_period = period;
   return ADACGD_OK;
 }
 
@@ -671,7 +716,7 @@ static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
     "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows",
-    "k_csr_fwd", "k_csc_bwd", "k_csr_residual"};
+    "k_csr_fwd", "k_csc_bwd", "k_csr_residual", "k_delta_scan", "k_dense_inc", "k_inc_finish"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
 

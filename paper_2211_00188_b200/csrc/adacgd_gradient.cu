@@ -36,7 +36,9 @@ __device__ __forceinline__ void residual(int loss, float z, float t, float inv_m
 template <bool CTA_ROW, bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, const float* __restrict__ target,
                                                    const float* __restrict__ x, long long d, long long m_rows,
-                                                   int loss, float* __restrict__ r, double* __restrict__ losspart) {
+                                                   int loss, float* __restrict__ r, double* __restrict__ losspart,
+                                                   float* __restrict__ zout) {
+  // r == nullptr: only the products z = A x are wanted (zout)
   const int worker = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const long long row = CTA_ROW ? (long long)blockIdx.x : (long long)blockIdx.x * LOSS_BLOCK_ROWS + wid;
@@ -80,10 +82,14 @@ __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, 
   }
   double l = 0.0;
   if (live && lane == 0 && (!CTA_ROW || wid == 0)) {
-    float rr;
-    residual(loss, z, target[(long long)worker * m_rows + row], 1.f / (float)m_rows, &rr, &l);
-    r[(long long)worker * m_rows + row] = rr;
+    if (zout) zout[(long long)worker * m_rows + row] = z;
+    if (r) {
+      float rr;
+      residual(loss, z, target[(long long)worker * m_rows + row], 1.f / (float)m_rows, &rr, &l);
+      r[(long long)worker * m_rows + row] = rr;
+    }
   }
+  if (r == nullptr) return;
   if (CTA_ROW) {
     if (threadIdx.x == 0) losspart[(long long)worker * gridDim.x + blockIdx.x] = l;
   } else {
@@ -446,8 +452,151 @@ __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__
   }
 }
 
+
+// ---- incremental forward: z_i = A_i x kept up to date from the entries of g that changed -----------------
+// x moves by -gamma g every iteration (Algorithm 1), so z_i = A_i x moves by -gamma u_i with u_i = A_i g, and g
+// itself changes only where a worker (identity master) or the master sent something.  u_i is therefore
+// kept between iterations and corrected by the changed entries alone: u_i += sum_c A_i[:, c] (g[c] - g_prev[c]),
+// columns read from a column-major copy of the features.  Sums run in ascending column order inside a chunk
+// of INC_CHUNK columns and the chunks are added in chunk order, so the result does not depend on scheduling.
+
+// AT[w][c][l] = A[w][l][c]
+__global__ void k_transpose_features(const float* __restrict__ A, float* __restrict__ AT, long long m_rows, long long d) {
+  __shared__ float tile[32][33];
+  const int w = blockIdx.z;
+  const long long c0 = (long long)blockIdx.x * 32, l0 = (long long)blockIdx.y * 32;
+  const float* a = A + (long long)w * m_rows * d;
+  float* at = AT + (long long)w * m_rows * d;
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const long long l = l0 + j, c = c0 + threadIdx.x;
+    tile[j][threadIdx.x] = (l < m_rows && c < d) ? a[l * d + c] : 0.f;
+  }
+  __syncthreads();
+  for (int j = threadIdx.y; j < 32; j += 8) {
+    const long long c = c0 + j, l = l0 + threadIdx.x;
+    if (c < d && l < m_rows) at[c * m_rows + l] = tile[threadIdx.x][j];
+  }
+}
+
+// One CTA per chunk of INC_CHUNK columns: the entries where g differs from g_prev, compacted in ascending
+// column order with their differences; g_prev takes the new values.
+__global__ void __launch_bounds__(TPB) k_delta_scan(const float* __restrict__ g, float* __restrict__ g_prev, long long d,
+                                                    u32* __restrict__ count, int* __restrict__ idx, float* __restrict__ val,
+                                                    u64* __restrict__ inc_cols) {
+  static_assert(INC_CHUNK == 2 * TPB, "two columns per thread");
+  __shared__ u32 wsum[TPB / 32];
+  const int chunk = blockIdx.x;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const long long c0 = (long long)chunk * INC_CHUNK + 2 * threadIdx.x;
+  float dv[2] = {0.f, 0.f};
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    if (c0 + k < d) {
+      const float a = g[c0 + k], b = g_prev[c0 + k];
+      dv[k] = __fsub_rn(a, b);
+      if (dv[k] != 0.f) g_prev[c0 + k] = a;
+    }
+  }
+  const u32 mine = (dv[0] != 0.f ? 1u : 0u) + (dv[1] != 0.f ? 1u : 0u);
+  u32 inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[wid] = inc;
+  __syncthreads();
+  u32 before = 0, total = 0;
+  for (int w = 0; w < TPB / 32; ++w) {
+    if (w < wid) before += wsum[w];
+    total += wsum[w];
+  }
+  u32 pos = before + inc - mine;
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    if (dv[k] != 0.f) {
+      idx[(long long)chunk * INC_CHUNK + pos] = (int)(c0 + k);
+      val[(long long)chunk * INC_CHUNK + pos] = dv[k];
+      ++pos;
+    }
+  }
+  if (threadIdx.x == 0) {
+    count[chunk] = total;
+    if (total) atomicAdd(inc_cols, (u64)total);
+  }
+}
+
+// Contribution of one chunk's changed columns to u of one worker: ipart[w][chunk][l] = sum_c AT[w][c][l] dv[c],
+// columns in ascending order, a thread per sample row (coalesced along l), four columns in flight.
+__global__ void __launch_bounds__(TPB) k_dense_inc(const float* __restrict__ AT, const u32* __restrict__ count,
+                                                   const int* __restrict__ idx, const float* __restrict__ val, long long d,
+                                                   long long m_rows, float* __restrict__ ipart) {
+  const int chunk = blockIdx.x, w = blockIdx.y;
+  const u32 cnt = count[chunk];
+  if (cnt == 0) return;
+  __shared__ int s_idx[INC_CHUNK];
+  __shared__ float s_val[INC_CHUNK];
+  for (u32 i = threadIdx.x; i < cnt; i += TPB) {
+    s_idx[i] = idx[(long long)chunk * INC_CHUNK + i];
+    s_val[i] = val[(long long)chunk * INC_CHUNK + i];
+  }
+  __syncthreads();
+  const float* at = AT + (long long)w * d * m_rows;
+  float* out = ipart + ((long long)w * gridDim.x + chunk) * m_rows;
+  for (long long l = threadIdx.x; l < m_rows; l += TPB) {
+    float acc = 0.f;
+    u32 e = 0;
+    for (; e + 4 <= cnt; e += 4) {
+      float a[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) a[k] = __ldcs(at + (long long)s_idx[e + k] * m_rows + l);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc = fmaf(a[k], s_val[e + k], acc);
+    }
+    for (; e < cnt; ++e) acc = fmaf(__ldcs(at + (long long)s_idx[e] * m_rows + l), s_val[e], acc);
+    out[l] = acc;
+  }
+}
+
+// u += the chunks' contributions (chunk order), z <- z - gamma u (two roundings, like the update of x), then
+// the residual and the loss of every sample row from the new z.
+__global__ void __launch_bounds__(TPB) k_inc_finish(const float* __restrict__ ipart, const u32* __restrict__ count, int nchunk,
+                                                    long long m_rows, float gamma, const float* __restrict__ target, int loss,
+                                                    float* __restrict__ u, float* __restrict__ z, float* __restrict__ r,
+                                                    double* __restrict__ losspart) {
+  const int w = blockIdx.y;
+  const long long l = (long long)blockIdx.x * TPB + threadIdx.x;
+  double ls = 0.0;
+  if (l < m_rows) {
+    const long long gi = (long long)w * m_rows + l;
+    float s = u[gi];
+    for (int c = 0; c < nchunk; ++c)
+      if (__ldg(&count[c])) s += ipart[((long long)w * nchunk + c) * m_rows + l];
+    u[gi] = s;
+    const float zn = __fsub_rn(z[gi], __fmul_rn(gamma, s));
+    z[gi] = zn;
+    float rr;
+    residual(loss, zn, target[gi], 1.f / (float)m_rows, &rr, &ls);
+    r[gi] = rr;
+  }
+  __shared__ double red[TPB / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int k = 0; k < TPB / 32; ++k) t += red[k];
+    losspart[(long long)w * gridDim.x + blockIdx.x] = t;
+  }
+}
+
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout, cudaStream_t stream);
+int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks, bool al,
+                              cudaStream_t stream);
 
 // The split decides the size of the partial-sum buffer, so it is part of the workspace layout and must not
 // depend on the device a context later runs on: it is taken for a nominal 148 SMs.
@@ -486,9 +635,25 @@ static int csc_cols_per_cta(const adacgd_problem& p) {
   return avg * CSC_WCOLS <= 0.75 * CSC_WPCAP ? 1 : 0;                    // a warp's span fits its buffer on average
 }
 
-size_t grad_scratch_bytes(const adacgd_problem& p) {
+static bool incremental_wanted(const adacgd_problem& p, int flags) {
+  return (flags & ADACGD_FLAG_INCREMENTAL_FORWARD) && p.loss != ADACGD_LOSS_NONE && p.layout == ADACGD_LAYOUT_DENSE;
+}
+
+size_t grad_scratch_bytes(const adacgd_problem& p, int flags) {
   if (p.loss == ADACGD_LOSS_NONE) return 0;
   size_t o = 0;
+  if (incremental_wanted(p, flags)) {
+    const size_t nm = (size_t)p.n * p.m_rows, chunks = ((size_t)p.d + INC_CHUNK - 1) / INC_CHUNK;
+    o = align_up(o + nm * (size_t)p.d * 4, 256);         // AT
+    o = align_up(o + nm * 4, 256);                        // z
+    o = align_up(o + nm * 4, 256);                        // u
+    o = align_up(o + (size_t)p.d * 4, 256);               // g_prev
+    o = align_up(o + chunks * 4, 256);                    // dl_count
+    o = align_up(o + chunks * INC_CHUNK * 4, 256);        // dl_idx
+    o = align_up(o + chunks * INC_CHUNK * 4, 256);        // dl_val
+    o = align_up(o + nm * chunks * 4, 256);               // ipart
+    o = align_up(o + 8, 256);                             // inc_cols
+  }
   o = align_up(o + (size_t)p.n * p.m_rows * 4, 256);
   const int split = choose_split(p);
   if (split > 1) o = align_up(o + (size_t)split * p.n * p.d * 4, 256);
@@ -510,9 +675,25 @@ size_t grad_scratch_bytes(const adacgd_problem& p) {
   return o;
 }
 
-void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p) {
+void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int flags) {
   char* b = (char*)base;
   size_t o = 0;
+  g->inc = incremental_wanted(p, flags) ? 1 : 0;
+  g->AT = g->z = g->u = g->g_prev = g->dl_val = g->ipart = nullptr;
+  g->dl_count = nullptr; g->dl_idx = nullptr; g->inc_cols = nullptr; g->inc_chunks = 0;
+  if (g->inc) {
+    const size_t nm = (size_t)p.n * p.m_rows, chunks = ((size_t)p.d + INC_CHUNK - 1) / INC_CHUNK;
+    g->inc_chunks = (int)chunks;
+    g->AT = (float*)(b + o); o = align_up(o + nm * (size_t)p.d * 4, 256);
+    g->z = (float*)(b + o); o = align_up(o + nm * 4, 256);
+    g->u = (float*)(b + o); o = align_up(o + nm * 4, 256);
+    g->g_prev = (float*)(b + o); o = align_up(o + (size_t)p.d * 4, 256);
+    g->dl_count = (u32*)(b + o); o = align_up(o + chunks * 4, 256);
+    g->dl_idx = (int*)(b + o); o = align_up(o + chunks * INC_CHUNK * 4, 256);
+    g->dl_val = (float*)(b + o); o = align_up(o + chunks * INC_CHUNK * 4, 256);
+    g->ipart = (float*)(b + o); o = align_up(o + nm * chunks * 4, 256);
+    g->inc_cols = (u64*)(b + o); o = align_up(o + 8, 256);
+  }
   g->split = choose_split(p);
   g->loss_blocks = loss_blocks_of(p);
   g->r = (float*)(b + o); o = align_up(o + (size_t)p.n * p.m_rows * 4, 256);
@@ -593,18 +774,32 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
   }
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
+  launch_dense_fwd(p, g, x, g.r, nullptr, stream);
+  ++launches;
+  return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream);
+}
+
+// The forward kernel in the shape the problem calls for: z = A v for a d-vector v, residuals if r != nullptr.
+void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout,
+                      cudaStream_t stream) {
+  const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)v) & 15) == 0;
   prof_begin(g.prof, KID_GRAD_FWD, stream);
   if (cta_row_mode(p)) {
     const dim3 grid((unsigned)p.m_rows, p.n);
-    if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
-    else k_dense_fwd<true, false><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
+    if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
+    else k_dense_fwd<true, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
   } else {
     const dim3 grid((unsigned)g.loss_blocks, p.n);
-    if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
-    else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, x, p.d, p.m_rows, p.loss, g.r, g.losspart);
+    if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
+    else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
   }
   prof_end(g.prof, stream);
-  ++launches;
+}
+
+// X_i = A_i^T r + reg'(x) and the loss from `loss_blocks` partial sums per worker; returns the launches.
+int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks,
+                              bool al, cudaStream_t stream) {
+  int launches = 0;
   const dim3 bgrid((unsigned)((p.d + TPB * 4 - 1) / (TPB * 4)), p.n * g.split);
   prof_begin(g.prof, KID_GRAD_BWD, stream);
   if (al) k_dense_bwd<true><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n);
@@ -618,10 +813,45 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
     ++launches;
   }
   prof_begin(g.prof, KID_LOSS, stream);
-  k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, g.loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+  k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
   prof_end(g.prof, stream);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, const float* x, const float* gvec,
+                                float gamma, bool refresh, float* grads, cudaStream_t stream) {
+  const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
+  int launches = 0;
+  if (refresh) {
+    // z = A x (with the residuals), u = A g, and g is remembered as the vector u belongs to
+    launch_dense_fwd(p, g, x, g.r, g.z, stream);
+    launch_dense_fwd(p, g, gvec, nullptr, g.u, stream);
+    launches += 2;
+    if (cudaMemcpyAsync(g.g_prev, gvec, (size_t)p.d * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return -1;
+    return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream);
+  }
+  prof_begin(g.prof, KID_DELTA, stream);
+  k_delta_scan<<<g.inc_chunks, TPB, 0, stream>>>(gvec, g.g_prev, p.d, g.dl_count, g.dl_idx, g.dl_val, g.inc_cols);
+  prof_end(g.prof, stream);
+  prof_begin(g.prof, KID_INC, stream);
+  k_dense_inc<<<dim3((unsigned)g.inc_chunks, p.n), TPB, 0, stream>>>(g.AT, g.dl_count, g.dl_idx, g.dl_val, p.d, p.m_rows, g.ipart);
+  prof_end(g.prof, stream);
+  const int fin_blocks = (int)((p.m_rows + TPB - 1) / TPB);
+  prof_begin(g.prof, KID_INC_FINISH, stream);
+  k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), TPB, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
+                                                                    g.u, g.z, g.r, g.losspart);
+  prof_end(g.prof, stream);
+  launches += 3;
+  return launches + launch_dense_bwd_and_loss(p, g, x, grads, fin_blocks, al, stream);
+}
+
+// Column-major copy of the dense features, once per context.
+int build_transposed_features(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream) {
+  const dim3 grid((unsigned)((p.d + 31) / 32), (unsigned)((p.m_rows + 31) / 32), p.n);
+  k_transpose_features<<<grid, dim3(32, 8), 0, stream>>>(p.A, g.AT, p.m_rows, p.d);
+  if (cudaMemsetAsync(g.inc_cols, 0, 8, stream) != cudaSuccess) return -1;
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace adacgd

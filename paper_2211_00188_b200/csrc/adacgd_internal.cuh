@@ -33,7 +33,7 @@ constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD, KID_CSR_RES,
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD, KID_CSR_RES, KID_DELTA, KID_INC, KID_INC_FINISH,
   KID_COUNT
 };
 struct Prof {
@@ -178,12 +178,31 @@ struct GradScratch {
   int ccols;            // 1: contiguous spans per warp; 0: one thread per column on csc_ptr
   long long* wbase;     // [n+1] first transposed entry of every worker
   u32* ptr32;           // [n][d+1]
+  // incremental forward (dense layout, ADACGD_FLAG_INCREMENTAL_FORWARD): z_i = A_i x and u_i = A_i g are kept
+  // between iterations and moved along by the entries of g that changed
+  int inc;              // 1: the buffers below exist
+  float* AT;            // [n][d][m_rows] column-major copy of the features
+  float* z;             // [n][m_rows]  A_i x
+  float* u;             // [n][m_rows]  A_i g_prev
+  float* g_prev;        // [d] the g that u belongs to
+  u32* dl_count;        // [inc_chunks] changed entries of g per chunk of INC_CHUNK columns
+  int* dl_idx;          // [inc_chunks][INC_CHUNK] their columns, ascending
+  float* dl_val;        // [inc_chunks][INC_CHUNK] g - g_prev there
+  float* ipart;         // [n][inc_chunks][m_rows] a chunk's contribution to u_i
+  u64* inc_cols;        // [1] columns gathered by incremental passes since init
+  int inc_chunks;
   Prof* prof;
 };
-size_t grad_scratch_bytes(const adacgd_problem& p);
-void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p);
+constexpr int INC_CHUNK = 512;
+size_t grad_scratch_bytes(const adacgd_problem& p, int flags);
+void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int flags);
 int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads,
                     cudaStream_t stream);
+// Incremental variant of stage a1 (the caller has already moved x): u += A (g - g_prev), z -= gamma u, then the
+// residuals from z and the backward pass.  `refresh`: z = A x and u = A g are recomputed in full instead.
+int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, const float* x, const float* gvec,
+                                float gamma, bool refresh, float* grads, cudaStream_t stream);
+int build_transposed_features(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream);
 const char* build_csc(const adacgd_problem& p, GradScratch* g, cudaStream_t stream);
 
 // x <- x - gamma * g  (two binary32 roundings: the product, then the difference)

@@ -1,0 +1,125 @@
+"""The incremental forward pass: z_i = A_i x is advanced by the entries of g that changed (x moves by -gamma g in
+Algorithm 1, and g changes only where a message touched it) instead of being recomputed from A, with a full
+recomputation every `period` iterations.  The gradients it leads to must stay within the same 1e-5 of the oracle's
+gradient at the engine's own iterate, right after a recomputation and after period - 1 incremental iterations; the
+selections taken from those gradients must be the oracle's, and a free run must reach the oracle's loss."""
+import numpy as np
+import pytest
+
+import synthetic_inputs as S
+from oracle import adacgd_oracle as O
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+TOPK, QUANT = 0, 1
+
+
+def relerr(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def engine(A, t, loss, lam, gamma, wc, wz, mc=(), mz=0.0, incremental=True):
+    import torch
+    import paper_2211_00188_b200 as pkg
+    dev = torch.device("cuda:0")
+    n, m, d = A.shape
+    return pkg.AdaCGD(n, d, wc, wz, mc, mz, loss=loss, lam=lam, A=torch.from_numpy(A).to(dev),
+                      target=torch.from_numpy(t).to(dev), x0=torch.zeros(d, device=dev), gamma=gamma,
+                      incremental_forward=incremental)
+
+
+def problem(A, t, loss, lam):
+    n = A.shape[0]
+    return dict(A=[A[i] for i in range(n)], target=[t[i] for i in range(n)], loss=loss, lam=lam)
+
+
+def check_last_iteration(eng, prob, G_before, Y_before, wc, wz, levels):
+    """The iteration the engine has just run: its gradients against the oracle's at the engine's iterate, and its
+    selections against the oracle's compressor fed with the engine's gradients."""
+    x = eng.get_state("x").cpu().numpy()
+    grad = eng.get_state("grad").cpu().numpy()
+    want = O.all_gradients(prob, x)
+    for i in range(grad.shape[0]):
+        assert relerr(grad[i], want[i]) <= 1e-5, (i, relerr(grad[i], want[i]))
+    assert np.abs(grad - want).max() <= 1e-5 * np.abs(want).max()
+    G_ref, res = O.compress_rows(grad, G_before, Y_before, wc, wz)
+    assert levels == [r["level"] for r in res]
+    assert np.array_equal(eng.get_state("G").cpu().numpy().view(np.uint32), G_ref.view(np.uint32))
+
+
+@pytest.mark.parametrize("case", ["identity_master_c1", "bidirectional", "ragged_least_squares", "quantised_master"])
+def test_gradients_after_refresh_and_after_incremental_iterations(case):
+    period = 8
+    if case == "identity_master_c1":
+        W = S.WORKLOADS["c1"]
+        A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+        loss, lam, wc, wz, mc, mz = W["loss"], W["lam"], W["worker"], 1.0, [], 0.0
+    elif case == "bidirectional":
+        A, t = S.logistic_problem(5, 800, 200, seed=1)
+        loss, lam, wc, wz = 0, 0.1, [(TOPK, 1), (TOPK, 8), (TOPK, 80), (TOPK, 800)], 1.0
+        mc, mz = wc, 1.0
+    elif case == "ragged_least_squares":
+        A, t, _ = S.least_squares_problem(3, 1333, 41, seed=2)     # neither d nor m a multiple of anything
+        loss, lam, wc, wz, mc, mz = 2, 0.0, [(TOPK, 13), (TOPK, 133)], 0.5, [], 0.0
+    else:
+        A, t = S.logistic_problem(3, 600, 50, seed=3)
+        loss, lam, wc, wz, mc, mz = 1, 1e-3, [(TOPK, 6), (TOPK, 60)], 1.0, [(QUANT, 4)], 0.0   # every entry of g moves
+    gamma = 0.5 / S.smoothness_estimate(A, loss, lam)
+    prob = problem(A, t, loss, lam)
+    eng = engine(A, t, loss, lam, gamma, wc, wz, mc, mz)
+    eng.set_refresh_period(period)
+    # iteration 1 recomputes (fresh context), 2 .. period are incremental, period + 1 recomputes again
+    done = 0
+    for upto in (1, period - 1, period, period + 1, 2 * period + 3):
+        eng.step(upto - 1 - done)
+        G_before = eng.get_state("G").cpu().numpy()
+        Y_before = eng.get_state("grad").cpu().numpy()
+        recs, levels = eng.step(1, report=True)
+        done = upto
+        check_last_iteration(eng, prob, G_before, Y_before, wc, wz, levels[0])
+    assert eng.get_state("refreshes") == 3 and eng.get_state("step") == done
+    assert eng.get_state("inc_columns") > 0
+    # pushing state invalidates the kept products: the next iteration recomputes them
+    eng.set_state("x", eng.get_state("x"))
+    eng.step(1)
+    assert eng.get_state("refreshes") == 4
+
+
+def test_incremental_and_full_forward_runs_agree_and_match_the_oracle():
+    # workload c1 for its 100 iterations, once with the incremental forward pass and once without, against the
+    # oracle left to run on its own: same loss to 1e-3, and the incremental run gathers far fewer columns than
+    # the n d it would read in full
+    W = S.WORKLOADS["c1"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"])
+    prob = problem(A, t, W["loss"], W["lam"])
+    st = O.init_state(prob, np.zeros(W["d"], F32), W["worker"])
+    for _ in range(W["iters"]):
+        O.step(st, prob, gamma, W["worker"], 1.0)
+    f_ref = O.global_loss(prob, st["x"])
+    finals = []
+    for inc in (True, False):
+        eng = engine(A, t, W["loss"], W["lam"], gamma, W["worker"], 1.0, incremental=inc)
+        recs, levels = eng.step(W["iters"], report=True)
+        assert abs(recs[-1]["loss"] - f_ref) <= 1e-3 * abs(f_ref)
+        finals.append(recs[-1]["loss"])
+        if inc:
+            assert eng.get_state("refreshes") == 7            # iterations 1, 17, 33, ... of 100 with the default period 16
+            assert 0 < eng.get_state("inc_columns") < 0.5 * W["iters"] * W["d"]
+    assert abs(finals[0] - finals[1]) <= 1e-4 * abs(finals[1])
+
+
+def test_refresh_period_needs_the_flag_and_a_positive_value():
+    import paper_2211_00188_b200 as pkg
+    A, t = S.logistic_problem(2, 100, 10, seed=4)
+    plain = engine(A, t, 0, 0.1, 0.1, [(TOPK, 5)], 1.0, incremental=False)
+    with pytest.raises(pkg.AdacgdError) as e:
+        plain.set_refresh_period(4)
+    assert e.value.status == 1
+    inc = engine(A, t, 0, 0.1, 0.1, [(TOPK, 5)], 1.0)
+    with pytest.raises(pkg.AdacgdError):
+        inc.set_refresh_period(0)
+    inc.set_refresh_period(1)                                  # every iteration recomputes
+    inc.step(5)
+    assert inc.get_state("refreshes") == 5 and inc.get_state("inc_columns") == 0
