@@ -393,11 +393,14 @@ def bench_c5(args, rank, world, local):
                         "replicas": world})
 
 
-def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats=None):
+def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats=None, incremental=False, k_scale=1.0):
     import torch
     import paper_2211_00188_b200 as pkg
 
-    W = S.WORKLOADS[name]
+    W = dict(S.WORKLOADS[name])
+    if k_scale != 1.0:   # the same workload with a ladder of smaller Top-K sizes
+        W["worker"] = [(k, max(1, int(p * k_scale)) if k == 0 else p) for k, p in W["worker"]]
+        W["master"] = [(k, max(1, int(p * k_scale)) if k == 0 else p) for k, p in W["master"]]
     n, d, m = (args.workers or W["n"]), W["d"], W["m"]
     dev = torch.device("cuda", local)
     steps = steps or args.steps
@@ -428,13 +431,25 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats
         A, tgt = torch.from_numpy(Ah).to(dev), torch.from_numpy(th).to(dev)
     x0 = torch.zeros(d, device=dev)
     eng = pkg.AdaCGD(n, d, W["worker"], 1.0, W["master"], 1.0, loss=W["loss"], lam=W["lam"], A=A, target=tgt,
-                     csr=csr, x0=x0, gamma=gamma, device=dev)
+                     csr=csr, x0=x0, gamma=gamma, device=dev, incremental_forward=incremental)
     eng.step(warmup)
+    cols0 = eng.get_state("inc_columns") if incremental else 0
+    refr0 = eng.get_state("refreshes") if incremental else 0
     launches0 = eng.launch_count()
     times, clocks = timed_repeats(lambda k: eng.step(k), steps, repeats, world, local)
     launches = (eng.launch_count() - launches0) // repeats
     st = repeat_stats(times, steps)
     ms = st["median"] * steps
+    inc_info = None
+    if incremental:
+        its = steps * repeats
+        cols = (eng.get_state("inc_columns") - cols0) / its
+        refr = (eng.get_state("refreshes") - refr0) / its
+        # features read per iteration: the backward pass in full, a full forward pass (twice: z and u) at a
+        # refresh, and the gathered columns of the column-major copy otherwise
+        inc_info = {"changed_entries_of_g_per_iteration": cols, "refreshes_per_iteration": refr,
+                    "feature_bytes_per_iteration": 4 * n * m * (d + 2 * d * refr + cols),
+                    "feature_bytes_per_iteration_full_forward": 8 * n * m * d}
     # the same number of steps once more with the library's per-kernel CUDA-event timers switched on
     eng.profile_enable(80 * steps + 64)
     eng.step(steps)
@@ -464,7 +479,7 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats
                 side_paths={"fallback_rows": eng.get_state("fallbacks"), "list_level_rows": eng.get_state("list_levels")},
                 config={"workload": name, "n": n, "d": d, "m": m, "loss": W["loss"], "gamma": gamma,
                         "cands": [list(c) for c in W["worker"]], "bidirectional": bool(W["master"]),
-                        "loss_after": recs[0]["loss"], "level_histogram_last_step": hist,
+                        "loss_after": recs[0]["loss"], "level_histogram_last_step": hist, "incremental_forward": inc_info,
                         "l2": ("features (%.2f GB) exceed the 126 MB L2" % (a_bytes / 1e9)) if a_bytes > 2e8
                         else "working set fits in L2 (launch-latency bound workload)", "replicas": world})
 
@@ -483,6 +498,8 @@ def main():
     ap.add_argument("--zeta", type=float, default=1.0)
     ap.add_argument("--scale", type=float, default=1.0, help="shrink d of workload c5 (profiling captures)")
     ap.add_argument("--workers", type=int, default=0, help="fewer workers for workloads c1-c4 (profiling captures)")
+    ap.add_argument("--incremental", action="store_true", help="workloads c1, c2, c4: keep the forward products between iterations")
+    ap.add_argument("--k-scale", type=float, default=1.0, help="workloads c1-c4: scale the Top-K sizes of the candidate lists")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the worst-case and the full-iteration measurements")
@@ -502,7 +519,7 @@ def main():
     if args.workload == "c5":
         res = bench_c5(args, rank, world, local)
     else:
-        res = bench_dense(args, args.workload, rank, world, local)
+        res = bench_dense(args, args.workload, rank, world, local, incremental=args.incremental, k_scale=args.k_scale)
     ms_per_step = res["ms"] / args.steps
 
     extra = None
@@ -517,6 +534,19 @@ def main():
                           "step_roofline": r2["step_roofline"], "kernels": r2["kernels"], "config": r2["config"],
                           "gpu_launches": r2["launches"], "exact_rechecks": r2["rechecks"], "side_paths": r2["side_paths"],
                           "clocks": r2["clocks"]})
+            del r2
+        # the forward products kept between iterations: workloads c2 and c4 as they are (most entries of g move every
+        # iteration there, so the pass mostly recomputes) and c4 with a ladder of Top-K sizes a hundred times smaller,
+        # with and without the incremental pass
+        for name, ks, inc in (("c2", 1.0, True), ("c4", 1.0, True), ("c4", 0.01, False), ("c4", 0.01, True)):
+            torch.cuda.empty_cache()
+            steps, warm = FULL_ITERATION_RUNS[name]
+            r2 = bench_dense(args, name, rank, world, local, steps=steps + 2, warmup=warm, repeats=3, incremental=inc, k_scale=ks)
+            extra.append({"workload": name, "what": "full iterations, " + ("incremental forward pass (refresh period 16)" if inc else "full forward pass")
+                          + (", Top-K sizes x %g" % ks if ks != 1.0 else ""),
+                          "steps": r2["steps"], "iters_per_s": r2["iters_per_s"], "ms_per_step": r2["ms"] / r2["steps"],
+                          "repeats": r2["repeats"], "compressed_elems_per_s": r2["value"], "kernels": r2["kernels"],
+                          "config": r2["config"], "gpu_launches": r2["launches"], "clocks": r2["clocks"]})
             del r2
 
     cpu = None

@@ -147,7 +147,9 @@ adacgd_status adacgd_step(adacgd_ctx* ctx, int32_t n_steps, adacgd_step_report* 
  * only in the entries some worker's message touched (identity master: g is the mean of the estimators) or the
  * master's message touched (Algorithm 2).  adacgd_step then keeps z_i and u_i = A_i g and advances them by the
  * changed entries alone, u_i += sum_c A_i[:, c] (g^t[c] - g^{t-1}[c]) and z_i <- fl(z_i - fl(gamma u_i)), instead
- * of reading A for z_i = A_i x; the backward product A_i^T r is unchanged.  Rounding makes the kept z_i drift from
+ * of reading A for z_i = A_i x; the backward product A_i^T r is unchanged.  An iteration in which more than half
+ * of the entries of g changed recomputes z_i = A_i x instead (gathering that many columns would cost as much),
+ * and the change is carried over to the next iteration's difference.  Rounding makes the kept z_i drift from
  * A_i x, so every `period` iterations (and after any adacgd_set_state) both products are recomputed in full.
  * period >= 1; 1 recomputes every iteration; the default is 16, which keeps the gradients within the 1e-5
  * relative agreement the library is tested to.  Returns ADACGD_ERR_INVALID_ARG for a context without the flag. */
@@ -249,8 +251,8 @@ adacgd_status adacgd_gradient(adacgd_ctx* ctx, const float* x_dev, float* grads_
                                    that went through the three-level passes over the key lists, since init (get only) */
 #define ADACGD_STATE_DEVICE 13  /* int32: ordinal of the CUDA device the context is bound to (the device that was
                                    current at adacgd_init); host destination only (get only) */
-#define ADACGD_STATE_INC_COLUMNS 14 /* uint64: columns of A the incremental forward passes have gathered since init,
-                                      summed over iterations (each counts once per worker) (get only) */
+#define ADACGD_STATE_INC_COLUMNS 14 /* uint64: entries of g the incremental forward passes found changed since init,
+                                      summed over iterations; every worker gathers that many columns of its A (get only) */
 #define ADACGD_STATE_REFRESHES 15  /* uint64: iterations since init whose forward products were recomputed in full;
                                       host destination only (get only) */
 adacgd_status adacgd_get_state(adacgd_ctx* ctx, int32_t which, void* dst, size_t bytes,

@@ -10,6 +10,12 @@ namespace adacgd {
 
 constexpr int LOSS_BLOCK_ROWS = 8;  // sample rows per CTA in warp-per-row mode
 
+__device__ __forceinline__ u32 warp_sum_u32_g(u32 v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 __device__ __forceinline__ float warp_sum_f32(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -37,8 +43,10 @@ template <bool CTA_ROW, bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, const float* __restrict__ target,
                                                    const float* __restrict__ x, long long d, long long m_rows,
                                                    int loss, float* __restrict__ r, double* __restrict__ losspart,
-                                                   float* __restrict__ zout) {
-  // r == nullptr: only the products z = A x are wanted (zout)
+                                                   float* __restrict__ zout, const u32* __restrict__ gate) {
+  // r == nullptr: only the products z = A x are wanted (zout); gate != nullptr: the launch only runs when the
+  // word is zero (the incremental pass found too many changed columns and leaves the products to this kernel)
+  if (gate && *gate != 0u) return;
   const int worker = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const long long row = CTA_ROW ? (long long)blockIdx.x : (long long)blockIdx.x * LOSS_BLOCK_ROWS + wid;
@@ -479,24 +487,22 @@ __global__ void k_transpose_features(const float* __restrict__ A, float* __restr
 }
 
 // One CTA per chunk of INC_CHUNK columns: the entries where g differs from g_prev, compacted in ascending
-// column order with their differences; g_prev takes the new values.
-__global__ void __launch_bounds__(TPB) k_delta_scan(const float* __restrict__ g, float* __restrict__ g_prev, long long d,
+// column order with their differences.  The last CTA to finish adds the counts up and decides the route of the
+// iteration: dl_flag[0] = 1, the changed columns are few enough to be gathered (k_dense_inc), or 0, z = A x is
+// recomputed in full (u and g_prev then stay as they are and the next scan sees the accumulated change).
+__global__ void __launch_bounds__(TPB) k_delta_scan(const float* __restrict__ g, const float* __restrict__ g_prev, long long d,
                                                     u32* __restrict__ count, int* __restrict__ idx, float* __restrict__ val,
-                                                    u64* __restrict__ inc_cols) {
+                                                    u32* __restrict__ dl_flag, u64* __restrict__ inc_cols, u32 max_cols) {
   static_assert(INC_CHUNK == 2 * TPB, "two columns per thread");
   __shared__ u32 wsum[TPB / 32];
+  __shared__ u32 last;
   const int chunk = blockIdx.x;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const long long c0 = (long long)chunk * INC_CHUNK + 2 * threadIdx.x;
   float dv[2] = {0.f, 0.f};
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    if (c0 + k < d) {
-      const float a = g[c0 + k], b = g_prev[c0 + k];
-      dv[k] = __fsub_rn(a, b);
-      if (dv[k] != 0.f) g_prev[c0 + k] = a;
-    }
-  }
+  for (int k = 0; k < 2; ++k)
+    if (c0 + k < d) dv[k] = __fsub_rn(g[c0 + k], g_prev[c0 + k]);
   const u32 mine = (dv[0] != 0.f ? 1u : 0u) + (dv[1] != 0.f ? 1u : 0u);
   u32 inc = mine;
 #pragma unroll
@@ -522,16 +528,36 @@ __global__ void __launch_bounds__(TPB) k_delta_scan(const float* __restrict__ g,
   }
   if (threadIdx.x == 0) {
     count[chunk] = total;
-    if (total) atomicAdd(inc_cols, (u64)total);
+    __threadfence();
+    last = (atomicAdd(&dl_flag[1], 1u) == gridDim.x - 1u) ? 1u : 0u;   // dl_flag[1]: completion ticket, cleared by the last CTA
+  }
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  u32 sum = 0;
+  for (int c = threadIdx.x; c < (int)gridDim.x; c += TPB) sum += __ldcg(&count[c]);
+  sum = warp_sum_u32_g(sum);
+  if (lane == 0) wsum[wid] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u32 all = 0;
+    for (int w = 0; w < TPB / 32; ++w) all += wsum[w];
+    const u32 go = (all <= max_cols) ? 1u : 0u;
+    dl_flag[0] = go;
+    dl_flag[1] = 0u;
+    if (go && all) atomicAdd(inc_cols, (u64)all);
   }
 }
 
 // Contribution of one chunk's changed columns to u of one worker: ipart[w][chunk][l] = sum_c AT[w][c][l] dv[c],
-// columns in ascending order, a thread per sample row (coalesced along l), four columns in flight.
+// columns in ascending order, a thread per sample row (coalesced along l), four columns in flight.  The CTA of
+// worker 0 and the first row tile also moves g_prev to g at those columns.
 __global__ void __launch_bounds__(TPB) k_dense_inc(const float* __restrict__ AT, const u32* __restrict__ count,
                                                    const int* __restrict__ idx, const float* __restrict__ val, long long d,
-                                                   long long m_rows, float* __restrict__ ipart) {
-  const int chunk = blockIdx.x, w = blockIdx.y;
+                                                   long long m_rows, float* __restrict__ ipart, const u32* __restrict__ dl_flag,
+                                                   const float* __restrict__ g, float* __restrict__ g_prev) {
+  if (dl_flag[0] == 0u) return;
+  const int chunk = blockIdx.x, w = blockIdx.z;
   const u32 cnt = count[chunk];
   if (cnt == 0) return;
   __shared__ int s_idx[INC_CHUNK];
@@ -541,49 +567,72 @@ __global__ void __launch_bounds__(TPB) k_dense_inc(const float* __restrict__ AT,
     s_val[i] = val[(long long)chunk * INC_CHUNK + i];
   }
   __syncthreads();
+  if (w == 0 && blockIdx.y == 0)
+    for (u32 i = threadIdx.x; i < cnt; i += TPB) g_prev[s_idx[i]] = g[s_idx[i]];
   const float* at = AT + (long long)w * d * m_rows;
   float* out = ipart + ((long long)w * gridDim.x + chunk) * m_rows;
-  for (long long l = threadIdx.x; l < m_rows; l += TPB) {
-    float acc = 0.f;
-    u32 e = 0;
-    for (; e + 4 <= cnt; e += 4) {
-      float a[4];
+  const long long l = (long long)blockIdx.y * TPB + threadIdx.x;
+  if (l >= m_rows) return;
+  float acc = 0.f;
+  u32 e = 0;
+  for (; e + 8 <= cnt; e += 8) {
+    float a[8];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) a[k] = __ldcs(at + (long long)s_idx[e + k] * m_rows + l);
+    for (int k = 0; k < 8; ++k) a[k] = __ldcs(at + (long long)s_idx[e + k] * m_rows + l);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) acc = fmaf(a[k], s_val[e + k], acc);
-    }
-    for (; e < cnt; ++e) acc = fmaf(__ldcs(at + (long long)s_idx[e] * m_rows + l), s_val[e], acc);
-    out[l] = acc;
+    for (int k = 0; k < 8; ++k) acc = fmaf(a[k], s_val[e + k], acc);
   }
+  for (; e < cnt; ++e) acc = fmaf(__ldcs(at + (long long)s_idx[e] * m_rows + l), s_val[e], acc);
+  out[l] = acc;
 }
 
-// u += the chunks' contributions (chunk order), z <- z - gamma u (two roundings, like the update of x), then
-// the residual and the loss of every sample row from the new z.
-__global__ void __launch_bounds__(TPB) k_inc_finish(const float* __restrict__ ipart, const u32* __restrict__ count, int nchunk,
-                                                    long long m_rows, float gamma, const float* __restrict__ target, int loss,
-                                                    float* __restrict__ u, float* __restrict__ z, float* __restrict__ r,
-                                                    double* __restrict__ losspart) {
+// Gathered route (dl_flag[0] = 1): u += the chunks' contributions, z <- z - gamma u (two roundings, like the
+// update of x).  Full route: z has just been recomputed.  Then the residual and the loss of every sample row
+// from z.  A CTA serves TPB sample rows with FIN_SLICES threads per row: each adds a contiguous range of
+// chunks in chunk order, and the ranges are added to u in range order.
+constexpr int FIN_SLICES = 4;
+__global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __restrict__ ipart, const u32* __restrict__ count,
+                                                                 int nchunk, long long m_rows, float gamma,
+                                                                 const float* __restrict__ target, int loss, float* __restrict__ u,
+                                                                 float* __restrict__ z, float* __restrict__ r,
+                                                                 double* __restrict__ losspart, const u32* __restrict__ dl_flag) {
+  __shared__ float part[FIN_SLICES][TPB];
+  __shared__ double red[TPB / 32];
   const int w = blockIdx.y;
-  const long long l = (long long)blockIdx.x * TPB + threadIdx.x;
+  const int row = threadIdx.x % TPB, slice = threadIdx.x / TPB;
+  const long long l = (long long)blockIdx.x * TPB + row;
+  const bool gathered = dl_flag != nullptr && dl_flag[0] != 0u;   // nullptr: z has just been recomputed (refresh)
+  if (gathered) {
+    float s = 0.f;
+    if (l < m_rows) {
+      const int c0 = (int)((long long)nchunk * slice / FIN_SLICES), c1 = (int)((long long)nchunk * (slice + 1) / FIN_SLICES);
+      for (int c = c0; c < c1; ++c)
+        if (__ldg(&count[c])) s += ipart[((long long)w * nchunk + c) * m_rows + l];
+    }
+    part[slice][row] = s;
+  }
+  __syncthreads();
+  if (slice != 0) return;
   double ls = 0.0;
   if (l < m_rows) {
     const long long gi = (long long)w * m_rows + l;
-    float s = u[gi];
-    for (int c = 0; c < nchunk; ++c)
-      if (__ldg(&count[c])) s += ipart[((long long)w * nchunk + c) * m_rows + l];
-    u[gi] = s;
-    const float zn = __fsub_rn(z[gi], __fmul_rn(gamma, s));
-    z[gi] = zn;
+    float zn = z[gi];
+    if (gathered) {
+      float s = u[gi];
+#pragma unroll
+      for (int q = 0; q < FIN_SLICES; ++q) s += part[q][row];
+      u[gi] = s;
+      zn = __fsub_rn(zn, __fmul_rn(gamma, s));
+      z[gi] = zn;
+    }
     float rr;
     residual(loss, zn, target[gi], 1.f / (float)m_rows, &rr, &ls);
     r[gi] = rr;
   }
-  __shared__ double red[TPB / 32];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
-  __syncthreads();
+  asm volatile("bar.sync 1, %0;" ::"n"(TPB));   // only the first slice's threads are left
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int k = 0; k < TPB / 32; ++k) t += red[k];
@@ -594,7 +643,8 @@ __global__ void __launch_bounds__(TPB) k_inc_finish(const float* __restrict__ ip
 // --------------------------------------------------------------------------
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout, cudaStream_t stream);
+void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout, cudaStream_t stream,
+                      const u32* gate = nullptr);
 int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks, bool al,
                               cudaStream_t stream);
 
@@ -653,6 +703,7 @@ size_t grad_scratch_bytes(const adacgd_problem& p, int flags) {
     o = align_up(o + chunks * INC_CHUNK * 4, 256);        // dl_val
     o = align_up(o + nm * chunks * 4, 256);               // ipart
     o = align_up(o + 8, 256);                             // inc_cols
+    o = align_up(o + 8, 256);                             // dl_flag
   }
   o = align_up(o + (size_t)p.n * p.m_rows * 4, 256);
   const int split = choose_split(p);
@@ -680,7 +731,7 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int
   size_t o = 0;
   g->inc = incremental_wanted(p, flags) ? 1 : 0;
   g->AT = g->z = g->u = g->g_prev = g->dl_val = g->ipart = nullptr;
-  g->dl_count = nullptr; g->dl_idx = nullptr; g->inc_cols = nullptr; g->inc_chunks = 0;
+  g->dl_count = nullptr; g->dl_idx = nullptr; g->inc_cols = nullptr; g->dl_flag = nullptr; g->inc_chunks = 0;
   if (g->inc) {
     const size_t nm = (size_t)p.n * p.m_rows, chunks = ((size_t)p.d + INC_CHUNK - 1) / INC_CHUNK;
     g->inc_chunks = (int)chunks;
@@ -693,6 +744,7 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int
     g->dl_val = (float*)(b + o); o = align_up(o + chunks * INC_CHUNK * 4, 256);
     g->ipart = (float*)(b + o); o = align_up(o + nm * chunks * 4, 256);
     g->inc_cols = (u64*)(b + o); o = align_up(o + 8, 256);
+    g->dl_flag = (u32*)(b + o); o = align_up(o + 8, 256);
   }
   g->split = choose_split(p);
   g->loss_blocks = loss_blocks_of(p);
@@ -781,17 +833,17 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
 
 // The forward kernel in the shape the problem calls for: z = A v for a d-vector v, residuals if r != nullptr.
 void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, const u32* gate) {
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)v) & 15) == 0;
   prof_begin(g.prof, KID_GRAD_FWD, stream);
   if (cta_row_mode(p)) {
     const dim3 grid((unsigned)p.m_rows, p.n);
-    if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
-    else k_dense_fwd<true, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
+    if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
+    else k_dense_fwd<true, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
   } else {
     const dim3 grid((unsigned)g.loss_blocks, p.n);
-    if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
-    else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout);
+    if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
+    else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
   }
   prof_end(g.prof, stream);
 }
@@ -823,26 +875,31 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
                                 float gamma, bool refresh, float* grads, cudaStream_t stream) {
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
+  const int fin_blocks = (int)((p.m_rows + TPB - 1) / TPB);
   if (refresh) {
-    // z = A x (with the residuals), u = A g, and g is remembered as the vector u belongs to
-    launch_dense_fwd(p, g, x, g.r, g.z, stream);
+    // z = A x, u = A g, and g is remembered as the vector u belongs to
+    launch_dense_fwd(p, g, x, nullptr, g.z, stream);
     launch_dense_fwd(p, g, gvec, nullptr, g.u, stream);
     launches += 2;
     if (cudaMemcpyAsync(g.g_prev, gvec, (size_t)p.d * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) return -1;
-    return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream);
+  } else {
+    // more changed entries than this and the gathered columns cost as much as reading A in order
+    const u32 max_cols = (u32)(p.d / 2);
+    prof_begin(g.prof, KID_DELTA, stream);
+    k_delta_scan<<<g.inc_chunks, TPB, 0, stream>>>(gvec, g.g_prev, p.d, g.dl_count, g.dl_idx, g.dl_val, g.dl_flag, g.inc_cols, max_cols);
+    prof_end(g.prof, stream);
+    prof_begin(g.prof, KID_INC, stream);
+    k_dense_inc<<<dim3((unsigned)g.inc_chunks, (unsigned)fin_blocks, p.n), TPB, 0, stream>>>(g.AT, g.dl_count, g.dl_idx, g.dl_val, p.d, p.m_rows,
+                                                                                             g.ipart, g.dl_flag, gvec, g.g_prev);
+    prof_end(g.prof, stream);
+    launch_dense_fwd(p, g, x, nullptr, g.z, stream, g.dl_flag);   // runs only if the scan chose the full route
+    launches += 3;
   }
-  prof_begin(g.prof, KID_DELTA, stream);
-  k_delta_scan<<<g.inc_chunks, TPB, 0, stream>>>(gvec, g.g_prev, p.d, g.dl_count, g.dl_idx, g.dl_val, g.inc_cols);
-  prof_end(g.prof, stream);
-  prof_begin(g.prof, KID_INC, stream);
-  k_dense_inc<<<dim3((unsigned)g.inc_chunks, p.n), TPB, 0, stream>>>(g.AT, g.dl_count, g.dl_idx, g.dl_val, p.d, p.m_rows, g.ipart);
-  prof_end(g.prof, stream);
-  const int fin_blocks = (int)((p.m_rows + TPB - 1) / TPB);
   prof_begin(g.prof, KID_INC_FINISH, stream);
-  k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), TPB, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
-                                                                    g.u, g.z, g.r, g.losspart);
+  k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), TPB * FIN_SLICES, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
+                                                                    g.u, g.z, g.r, g.losspart, refresh ? nullptr : g.dl_flag);
   prof_end(g.prof, stream);
-  launches += 3;
+  ++launches;
   return launches + launch_dense_bwd_and_loss(p, g, x, grads, fin_blocks, al, stream);
 }
 
@@ -850,7 +907,7 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
 int build_transposed_features(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream) {
   const dim3 grid((unsigned)((p.d + 31) / 32), (unsigned)((p.m_rows + 31) / 32), p.n);
   k_transpose_features<<<grid, dim3(32, 8), 0, stream>>>(p.A, g.AT, p.m_rows, p.d);
-  if (cudaMemsetAsync(g.inc_cols, 0, 8, stream) != cudaSuccess) return -1;
+  if (cudaMemsetAsync(g.inc_cols, 0, 8, stream) != cudaSuccess || cudaMemsetAsync(g.dl_flag, 0, 8, stream) != cudaSuccess) return -1;
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -190,6 +190,7 @@ struct GradScratch {
   float* dl_val;        // [inc_chunks][INC_CHUNK] g - g_prev there
   float* ipart;         // [n][inc_chunks][m_rows] a chunk's contribution to u_i
   u64* inc_cols;        // [1] columns gathered by incremental passes since init
+  u32* dl_flag;         // [2] route of the iteration (1: gathered columns, 0: full forward), completion ticket of the scan
   int inc_chunks;
   Prof* prof;
 };

@@ -79,7 +79,10 @@ def test_gradients_after_refresh_and_after_incremental_iterations(case):
         done = upto
         check_last_iteration(eng, prob, G_before, Y_before, wc, wz, levels[0])
     assert eng.get_state("refreshes") == 3 and eng.get_state("step") == done
-    assert eng.get_state("inc_columns") > 0
+    # an iteration in which more than half of g moved recomputes z in full and gathers nothing (nearly always on
+    # workload c1: Top-500 of 1 000 on four workers); the small Top-K sizes of the least-squares case always gather
+    if case == "ragged_least_squares":
+        assert eng.get_state("inc_columns") > 0
     # pushing state invalidates the kept products: the next iteration recomputes them
     eng.set_state("x", eng.get_state("x"))
     eng.step(1)
@@ -106,7 +109,7 @@ def test_incremental_and_full_forward_runs_agree_and_match_the_oracle():
         finals.append(recs[-1]["loss"])
         if inc:
             assert eng.get_state("refreshes") == 7            # iterations 1, 17, 33, ... of 100 with the default period 16
-            assert 0 < eng.get_state("inc_columns") < (W["iters"] - 7) * W["d"]
+            assert eng.get_state("inc_columns") <= (W["iters"] - 7) * (W["d"] // 2)   # gathered only when at most half of g moved
     assert abs(finals[0] - finals[1]) <= 1e-4 * abs(finals[1])
 
 
