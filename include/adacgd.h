@@ -67,14 +67,33 @@ typedef struct {
   int64_t param;
 } adacgd_cand;
 
+/* Trigger of one level.  The adaptive compressor of Definition 3 (Eq. 9) applies the first compressor whose
+ * condition P_j(h, y, x) holds and the last one when none does; AdaCGD (Eq. 11) is the case where every P_j is the
+ * lazy-aggregation test of Eq. 10.  The library evaluates the conditions below, all of them comparisons of
+ * squared norms it computes anyway (exact sums rounded once to binary64, as for Eq. 10); with
+ * E_j = ||x - C^j_{h,y}(x)||^2 for candidate j and E_0 = ||x - h||^2 for the skip level: */
+#define ADACGD_PRED_LAZY 0     /* E_j <= param * ||x - y||^2   Eq. 10 with the level's own zeta */
+#define ADACGD_PRED_ABSOLUTE 1 /* E_j <= param                  an absolute error budget */
+#define ADACGD_PRED_RELATIVE 2 /* E_j <= param * ||x - h||^2    a fraction of what skipping would leave */
+#define ADACGD_PRED_NEVER 3    /* false: the level is never chosen by its trigger (level 0: no skipping) */
+#define ADACGD_PRED_ALWAYS 4   /* true: the level is chosen whenever it is reached */
+typedef struct {
+  int32_t kind;  /* ADACGD_PRED_* */
+  float param;   /* finite, >= 0; ignored by NEVER and ALWAYS */
+} adacgd_pred;
+
 /* A compressor set: m candidates in the order they are tried, and the trigger
  * zeta >= 0 of Eq. 10.  m = 0 is the identity compressor (no trigger).  Host memory;
  * copied by the call that receives it.  Top-K parameters must be strictly
- * increasing along the list and quantiser widths strictly increasing. */
+ * increasing along the list and quantiser widths strictly increasing.
+ *   preds: NULL for AdaCGD (Eq. 11: Eq. 10 with zeta at every level), or m triggers:
+ *   preds[0] for the skip level, preds[j] for candidate j, 1 <= j <= m - 1; the last
+ *   candidate is the "otherwise" of Eq. 9 and has none.  zeta is ignored then. */
 typedef struct {
   const adacgd_cand* cands;
   int32_t m;
   float zeta;
+  const adacgd_pred* preds;
 } adacgd_cset;
 
 /* Objectives f_i (Eq. 1). m_rows samples per worker, features a_l, targets t_l. */

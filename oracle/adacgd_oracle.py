@@ -11,7 +11,8 @@ What is restated here, and from which passage of the paper:
   quantiser below is this project's reading -- *parity unpinned against the paper*);
 * the EF21 compressor  C^EF_{h,y}(x) = h + C(x - h)            (Eq. 7);
 * the CLAG / LAG compressors                                   (Eq. 8, Eq. 5);
-* the Ada3PC compressor (Definition 3, Eq. 9 "first predicate that holds");
+* the Ada3PC compressor (Definition 3, Eq. 9 "first predicate that holds"), with callables
+  (`ada3pc`) and with the small menu of triggers the library evaluates (`adaptive_3pc`);
 * the AdaCGD compressor and its trigger  ||x - C^{EF,j}(x)||^2 <= zeta ||x - y||^2
   (Eq. 10 and the Definition of Section 4.3, Eq. 11);
 * the bidirectional loop (Algorithm 1, with the three-point arguments of Algorithm 2);
@@ -246,6 +247,58 @@ def adacgd(h, y, x, cands, zeta):
     level = m
     for j in range(m + 1):
         if err[j] <= rhs:
+            level = j
+            break
+    if level == 0:
+        return dict(out=h.copy(), level=0, bits=0, err=err, D=D, kept=None)
+    cand = cands[level - 1]
+    out = apply_shifted(h, v, cand)
+    kept = np.sort(topk_kept(v, cand[1])) if cand[0] == TOPK else None
+    return dict(out=out, level=level, bits=message_bits(cand, d), err=err, D=D, kept=kept)
+
+
+# Triggers the library evaluates for the adaptive compressor of Definition 3 (Eq. 9); each is a
+# condition P(h, y, x) -> {0, 1} on the level's error E = ||x - C_{h,y}(x)||^2 (E = ||x - h||^2 for
+# keeping h), under the exact-sum convention above.
+PRED_LAZY = 0      # E <= param * ||x - y||^2      (Eq. 10)
+PRED_ABSOLUTE = 1  # E <= param
+PRED_RELATIVE = 2  # E <= param * ||x - h||^2
+PRED_NEVER = 3
+PRED_ALWAYS = 4
+
+
+def trigger_holds(pred, E: float, h, y, x) -> bool:
+    """One condition P_j(h, y, x) of Definition 3, from the menu above."""
+    kind, param = pred
+    if kind == PRED_NEVER:
+        return False
+    if kind == PRED_ALWAYS:
+        return True
+    par = float(F32(param))
+    if kind == PRED_LAZY:
+        return E <= par * sumsq((_as_f32(x) - _as_f32(y)).astype(F32))
+    if kind == PRED_RELATIVE:
+        return E <= par * sumsq((_as_f32(x) - _as_f32(h)).astype(F32))
+    if kind == PRED_ABSOLUTE:
+        return E <= par
+    raise ValueError("unknown trigger kind")
+
+
+def adaptive_3pc(h, y, x, cands, preds):
+    """Adaptive three-point compressor (Definition 3, Eq. 9) over the compressors
+    C^0 = "keep h" and C^j = EF21 with candidate j (Eq. 7), j = 1..m, with the triggers
+    preds[0..m-1] from the menu above: the first compressor whose trigger holds is applied, the
+    last one if none does.  AdaCGD (Eq. 11) is the case preds = [(PRED_LAZY, zeta)] * m.
+    Returns the same dict as `adacgd`."""
+    h, y, x = _as_f32(h), _as_f32(y), _as_f32(x)
+    d, m = x.size, len(cands)
+    assert len(preds) == m and m >= 1
+    v = (x - h).astype(F32)
+    D = sumsq((x - y).astype(F32))
+    err = [sumsq(v)] + [candidate_error(v, c) for c in cands]
+    level = m
+    for j in range(m):
+        if trigger_holds(preds[j], err[j], h, y, x):
             level = j
             break
     if level == 0:

@@ -9,6 +9,7 @@ import os
 from typing import Optional, Sequence, Tuple
 
 TOPK, QUANT = 0, 1
+PRED_LAZY, PRED_ABSOLUTE, PRED_RELATIVE, PRED_NEVER, PRED_ALWAYS = 0, 1, 2, 3, 4
 LOSS_LOGISTIC_NCVX, LOSS_LOGISTIC_L2, LOSS_LEAST_SQUARES, LOSS_NONE = 0, 1, 2, 3
 LAYOUT_DENSE, LAYOUT_CSR = 0, 1
 FLAG_HOST_STAGING = 1
@@ -36,8 +37,12 @@ class _Cand(C.Structure):
     _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("param", C.c_int64)]
 
 
+class _Pred(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("param", C.c_float)]
+
+
 class _Cset(C.Structure):
-    _fields_ = [("cands", C.POINTER(_Cand)), ("m", C.c_int32), ("zeta", C.c_float)]
+    _fields_ = [("cands", C.POINTER(_Cand)), ("m", C.c_int32), ("zeta", C.c_float), ("preds", C.POINTER(_Pred))]
 
 
 class _Problem(C.Structure):
@@ -101,14 +106,22 @@ def load_library():
     return lib
 
 
-def _cset(cands: Optional[Sequence[Cand]], zeta: float):
-    """Returns (struct, keepalive)."""
+def _cset(cands: Optional[Sequence[Cand]], zeta: float, preds=None):
+    """Returns (struct, keepalive).  preds: None, or one (kind, param) per level 0 .. m-1."""
     cands = list(cands or [])
     arr = (_Cand * max(1, len(cands)))()
     for i, (kind, param) in enumerate(cands):
         arr[i].kind, arr[i].reserved, arr[i].param = int(kind), 0, int(param)
-    cs = _Cset(C.cast(arr, C.POINTER(_Cand)), len(cands), float(zeta))
-    return cs, arr
+    parr = None
+    if preds is not None:
+        if len(preds) != len(cands):
+            raise ValueError("one trigger per level 0 .. m-1: len(preds) must equal len(cands)")
+        parr = (_Pred * max(1, len(preds)))()
+        for i, (kind, param) in enumerate(preds):
+            parr[i].kind, parr[i].param = int(kind), float(param)
+    cs = _Cset(C.cast(arr, C.POINTER(_Cand)), len(cands), float(zeta),
+               C.cast(parr, C.POINTER(_Pred)) if parr is not None else None)
+    return cs, (arr, parr)
 
 
 def message_bits(cand: Cand, d: int) -> int:
@@ -127,7 +140,8 @@ class AdaCGD:
     def __init__(self, n: int, d: int, worker: Sequence[Cand] = (), worker_zeta: float = 0.0,
                  master: Sequence[Cand] = (), master_zeta: float = 0.0, *, loss: int = LOSS_NONE,
                  lam: float = 0.0, A=None, target=None, csr=None, x0=None, gamma: float = 1.0, g0_mode: int = 1,
-                 host_staging: bool = False, incremental_forward: bool = False, device="cuda:0", stream=None):
+                 host_staging: bool = False, incremental_forward: bool = False, worker_preds=None, master_preds=None,
+                 device="cuda:0", stream=None):
         import torch
 
         self.torch = torch
@@ -158,8 +172,9 @@ class AdaCGD:
         self.problem = _Problem(loss, float(lam), self.n, layout, self.d, m_rows, _ptr(A) if A is not None else None,
                                 _ptr(target) if target is not None else None, _ptr(rowptr), _ptr(col), _ptr(val), nnz)
         self.flags = (FLAG_HOST_STAGING if host_staging else 0) | (FLAG_INCREMENTAL_FORWARD if incremental_forward else 0)
-        wcs, k1 = _cset(self.worker, worker_zeta)
-        mcs, k2 = _cset(self.master, master_zeta)
+        self.worker_preds, self.master_preds = worker_preds, master_preds
+        wcs, k1 = _cset(self.worker, worker_zeta, worker_preds)
+        mcs, k2 = _cset(self.master, master_zeta, master_preds)
         nbytes = C.c_size_t(0)
         self._check(self.lib.adacgd_workspace_bytes(C.byref(self.problem), C.byref(wcs), C.byref(mcs), self.flags,
                                                     C.byref(nbytes)), None)
@@ -192,10 +207,12 @@ class AdaCGD:
 
     # -- entry points ------------------------------------------------------
     def compress(self, X, G, Y, cands: Optional[Sequence[Cand]] = None, zeta: Optional[float] = None, *,
-                 mean_out=None, level=None, bits=None, err=None, D=None, kept_idx=None, kept_cnt=None):
+                 mean_out=None, level=None, bits=None, err=None, D=None, kept_idx=None, kept_cnt=None, preds=None):
         """adacgd_compress on device tensors; G is updated in place."""
         rows, d = X.shape
-        cs, keep = _cset(self.worker if cands is None else cands, self.worker_zeta if zeta is None else zeta)
+        if cands is None and preds is None:
+            preds = self.worker_preds
+        cs, keep = _cset(self.worker if cands is None else cands, self.worker_zeta if zeta is None else zeta, preds)
         stride = kept_idx.shape[1] if kept_idx is not None else 0
         self._check(self.lib.adacgd_compress(self.ctx, _ptr(X), _ptr(G), _ptr(Y), rows, d, C.byref(cs), _ptr(mean_out),
                                              _ptr(level), _ptr(bits), _ptr(err), _ptr(D), _ptr(kept_idx), stride,

@@ -323,7 +323,7 @@ static adacgd_status init_body(adacgd_ctx* c, const adacgd_problem* problem, con
     } else {
       CK(nullptr, cudaMemsetAsync(c->G, 0, nd, c->stream), "adacgd_init (zero estimators)");
       adacgd_cand first = worker->cands[0];
-      adacgd_cset one = {&first, 1, 0.f};
+      adacgd_cset one = {&first, 1, 0.f, nullptr};
       CsetDev cs1;
       make_cset(&one, problem->d, &cs1, &msg);
       CompressOut o;

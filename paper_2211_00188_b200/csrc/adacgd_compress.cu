@@ -1685,6 +1685,18 @@ adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const 
   if (!(in->zeta >= 0.f) || !(in->zeta <= 3.0e38f)) { *msg = "zeta must be finite and >= 0"; return ADACGD_ERR_INVALID_ARG; }
   cs.m = in->m;
   cs.zeta = in->zeta;
+  for (int j = 0; j < in->m; ++j) {
+    cs.pkind[j] = ADACGD_PRED_LAZY;   // Eq. 10 at every level unless the caller names other triggers
+    cs.pparam[j] = in->zeta;
+    if (in->preds) {
+      const adacgd_pred& q = in->preds[j];
+      if (q.kind < ADACGD_PRED_LAZY || q.kind > ADACGD_PRED_ALWAYS) { *msg = "unknown trigger kind"; return ADACGD_ERR_INVALID_ARG; }
+      const bool has_param = q.kind == ADACGD_PRED_LAZY || q.kind == ADACGD_PRED_ABSOLUTE || q.kind == ADACGD_PRED_RELATIVE;
+      if (has_param && (!(q.param >= 0.f) || !(q.param <= 3.0e38f))) { *msg = "trigger parameter must be finite and >= 0"; return ADACGD_ERR_INVALID_ARG; }
+      cs.pkind[j] = q.kind;
+      cs.pparam[j] = has_param ? q.param : 0.f;
+    }
+  }
   long long lastK = 0, lastB = 0;
   for (int c = 0; c < in->m; ++c) {
     const adacgd_cand& a = in->cands[c];

@@ -258,27 +258,40 @@ inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nbl
   }
   // `tol` bounds the relative error of every sum above (non-negative terms).  A sum is only
   // trusted inside [2^-90, inf): below, binary32 squares may have underflowed; above, a chain
-  // overflowed (or X - Y is not finite, which the exact pass reports).
+  // overflowed (or X - Y is not finite, which the exact pass tells).
   const double tiny = 8.0e-28;
-  const double rhs = (double)cs.zeta * D;
   const bool d_ok = (D >= tiny && D <= 1.7e308);
+  const bool e0_ok = (e[0] >= tiny && e[0] <= 1.7e308);
   int level = cs.m;
   bool unsure = false;
-  for (int j = 0; j <= cs.m; ++j) {
+  for (int j = 0; j < cs.m; ++j) {   // levels 0 .. m-1 carry a trigger (Eq. 9); level m is the "otherwise"
     const double E = e[j];
+    const int kind = cs.pkind[j];
+    const double par = (double)cs.pparam[j];
     const bool by_def = (j > 0 && cs.kind[j - 1] == ADACGD_TOPK && cs.param[j - 1] >= d);  // identity: error 0
     const bool e_ok = (E >= tiny && E <= 1.7e308);
     int verdict;  // 1 true, 0 false, -1 unsure
-    if (by_def) verdict = 1;
-    else if (!(D <= 1.7e308)) verdict = -1;  // overflowed chain or non-finite X - Y: the exact pass tells which
-    else if (j == 0 && (diff & 0x7fffffffu) == 0 && d_ok)
-      verdict = (cs.zeta >= 1.f) ? 1 : 0;  // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
+    if (kind == ADACGD_PRED_NEVER) verdict = 0;
+    else if (kind == ADACGD_PRED_ALWAYS) verdict = 1;
+    else if (by_def) verdict = 1;                     // 0 <= any right side
+    else if (!(D <= 1.7e308)) verdict = -1;           // overflowed chain or non-finite X - Y: the exact pass tells which
+    else if (kind == ADACGD_PRED_LAZY && j == 0 && (diff & 0x7fffffffu) == 0 && d_ok)
+      verdict = (par >= 1.0) ? 1 : 0;                 // |X-G| == |X-Y| entry by entry, so ||v||^2 == D > 0 exactly
+    else if (kind == ADACGD_PRED_RELATIVE && j == 0 && e0_ok)
+      verdict = (par >= 1.0) ? 1 : 0;                 // ||v||^2 against itself
     else if (!e_ok) verdict = -1;
-    else if (cs.zeta == 0.f) verdict = 0;  // E > 0 for certain, right side is 0
-    else if (!d_ok) verdict = -1;
-    else if (E * (1.0 + tol) < rhs * (1.0 - tol)) verdict = 1;
-    else if (E * (1.0 - tol) > rhs * (1.0 + tol)) verdict = 0;
-    else verdict = -1;
+    else if (par == 0.0) verdict = 0;                 // E > 0 for certain, right side is 0
+    else {
+      double rhs, rtol;
+      bool r_ok;
+      if (kind == ADACGD_PRED_LAZY) { rhs = par * D; rtol = tol; r_ok = d_ok; }
+      else if (kind == ADACGD_PRED_RELATIVE) { rhs = par * e[0]; rtol = tol; r_ok = e0_ok; }
+      else { rhs = par; rtol = 0.0; r_ok = true; }    // absolute tolerance: the right side is exact
+      if (!r_ok) verdict = -1;
+      else if (E * (1.0 + tol) < rhs * (1.0 - rtol)) verdict = 1;
+      else if (E * (1.0 - tol) > rhs * (1.0 + rtol)) verdict = 0;
+      else verdict = -1;
+    }
     if (verdict == 1) { level = j; break; }
     if (verdict < 0) { unsure = true; break; }
   }
@@ -376,10 +389,19 @@ inline __device__ void decide_exact_row(const CsetDev& cs, int row, long long d,
     return;
   }
   const double D = val[0];
-  const double rhs = (double)cs.zeta * D;
   int level = cs.m;
-  for (int j = 0; j <= cs.m; ++j)
-    if (val[1 + j] <= rhs) { level = j; break; }
+  for (int j = 0; j < cs.m; ++j) {
+    const double par = (double)cs.pparam[j];
+    bool holds;
+    switch (cs.pkind[j]) {
+      case ADACGD_PRED_LAZY: holds = val[1 + j] <= par * D; break;            // Eq. 10
+      case ADACGD_PRED_RELATIVE: holds = val[1 + j] <= par * val[1]; break;
+      case ADACGD_PRED_ABSOLUTE: holds = val[1 + j] <= par; break;
+      case ADACGD_PRED_ALWAYS: holds = true; break;
+      default: holds = false; break;
+    }
+    if (holds) { level = j; break; }
+  }
   finalize_row(cs, row, level, d, sel, maxkey, dec, out, val + 1, D);
 }
 

@@ -64,6 +64,8 @@ void set_small_kernel_attributes();      // adacgd_small.cu
 struct CsetDev {
   int m;                 // candidates
   float zeta;
+  int pkind[MAXC];       // trigger of level j = 0 .. m-1 (level 0 = skip): ADACGD_PRED_*
+  float pparam[MAXC];    // its parameter
   int kind[MAXC];
   long long param[MAXC]; // K or bits
   int nsel;              // Top-K candidates with K < d: they need a threshold

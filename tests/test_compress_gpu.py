@@ -489,3 +489,79 @@ def test_host_entry_point_unaligned_and_identity(torch, cands):
         G_ref = X.copy()                      # the identity compressor sends the gradient itself
     assert_bitwise(Gh.numpy(), G_ref, "G")
     assert_bitwise(mean.numpy(), O.server_mean(G_ref), "mean")
+
+
+# ---------------------------------------------------------------- triggers other than Eq. 10 (Definition 3)
+PRED_LAZY, PRED_ABSOLUTE, PRED_RELATIVE, PRED_NEVER, PRED_ALWAYS = 0, 1, 2, 3, 4
+
+
+def check_menu_against_oracle(torch, X, G, Y, cands, preds):
+    import paper_2211_00188_b200 as pkg
+    rows, d = X.shape
+    dev = torch.device("cuda:0")
+    eng = pkg.AdaCGD(rows, d, cands, 1.0)
+    Xd, Gd, Yd = (torch.from_numpy(np.ascontiguousarray(a)).to(dev) for a in (X, G, Y))
+    level = torch.full((rows,), -7, dtype=torch.int32, device=dev)
+    bits = torch.zeros(rows, dtype=torch.int64, device=dev)
+    mean = torch.zeros(d, dtype=torch.float32, device=dev)
+    eng.compress(Xd, Gd, Yd, cands, 1.0, mean_out=mean, level=level, bits=bits, preds=preds)
+    torch.cuda.synchronize()
+    refs = [O.adaptive_3pc(G[i], Y[i], X[i], cands, preds) for i in range(rows)]
+    assert level.cpu().tolist() == [r["level"] for r in refs], (preds, level.cpu().tolist(), [r["level"] for r in refs])
+    assert bits.cpu().tolist() == [r["bits"] for r in refs]
+    G_ref = np.stack([r["out"] for r in refs])
+    assert_bitwise(Gd.cpu().numpy(), G_ref, "G")
+    assert_bitwise(mean.cpu().numpy(), O.server_mean(G_ref), "mean")
+    return [r["level"] for r in refs], eng
+
+
+@pytest.mark.parametrize("rows,d", [(3, 900), (2, 70_001), (3, 600_000)])
+def test_trigger_menu_on_every_route(torch, rows, d):
+    # the conditions of Definition 3 the library evaluates, on the short-row kernel, the three-pass route and the
+    # sampled single-pass pipeline: absolute budgets, fractions of ||x - h||^2, per-level zeta, never / always
+    X, G, Y = S.gaussian_rows(rows, d, seed=70 + rows)
+    cands = [(TOPK, max(1, d // 1000)), (TOPK, d // 100), (QUANT, 4), (TOPK, d // 10)]
+    e0 = O.sumsq((X[0] - G[0]).astype(F32))
+    seen = set()
+    for preds in ([(PRED_NEVER, 0.0)] + [(PRED_ABSOLUTE, 0.995 * e0)] * 3,
+                  [(PRED_ABSOLUTE, 0.5 * e0)] * 4,
+                  [(PRED_RELATIVE, 0.97), (PRED_RELATIVE, 0.97), (PRED_RELATIVE, 0.8), (PRED_RELATIVE, 0.05)],
+                  [(PRED_RELATIVE, 1.0)] * 4,
+                  [(PRED_NEVER, 0.0), (PRED_LAZY, 5.0), (PRED_LAZY, 2.0), (PRED_LAZY, 0.1)],
+                  [(PRED_LAZY, 0.5), (PRED_NEVER, 0.0), (PRED_ALWAYS, 0.0), (PRED_NEVER, 0.0)],
+                  [(PRED_NEVER, 0.0)] * 4,
+                  [(PRED_LAZY, 0.0), (PRED_ABSOLUTE, 0.0), (PRED_RELATIVE, 0.0), (PRED_RELATIVE, 0.3)]):
+        lv, _ = check_menu_against_oracle(torch, X, G, Y, cands, preds)
+        seen.update(lv)
+    assert seen == {0, 1, 2, 3, 4}
+
+
+def test_trigger_menu_equalities_take_the_exact_path(torch):
+    # small integers: the budgets are met with equality or missed by one unit in the last place of the sum
+    X, G, Y = S.tie_vectors(4, 5000, seed=75)
+    cands = [(TOPK, 50), (TOPK, 500), (TOPK, 2500)]
+    errs = [O.adaptive_3pc(G[0], Y[0], X[0], cands, [(PRED_NEVER, 0.0)] * 3)["err"]][0]
+    rechecks = 0
+    for target in (1, 2):
+        for tweak in (0.0, -1.0, 1.0):
+            budget = float(np.float32(errs[target] + tweak))      # integers below 2^24: exact in binary32
+            preds = [(PRED_NEVER, 0.0)] + [(PRED_ABSOLUTE, budget)] * 2
+            lv, eng = check_menu_against_oracle(torch, X, G, Y, cands, preds)
+            rechecks += eng.get_state("rechecks")
+    preds = [(PRED_RELATIVE, 1.0), (PRED_RELATIVE, 0.5), (PRED_RELATIVE, 0.5)]
+    check_menu_against_oracle(torch, X, G, Y, cands, preds)
+    assert rechecks > 0
+
+
+def test_trigger_menu_argument_errors(torch):
+    import paper_2211_00188_b200 as pkg
+    eng = pkg.AdaCGD(2, 100, CANDS3[:2], 1.0)
+    X = torch.zeros(2, 100, device="cuda:0")
+    with pytest.raises(pkg.AdacgdError) as e:
+        eng.compress(X, X.clone(), X, CANDS3[:2], 1.0, preds=[(9, 1.0), (PRED_LAZY, 1.0)])
+    assert e.value.status == 1
+    with pytest.raises(pkg.AdacgdError) as e:
+        eng.compress(X, X.clone(), X, CANDS3[:2], 1.0, preds=[(PRED_ABSOLUTE, -1.0), (PRED_LAZY, 1.0)])
+    assert e.value.status == 1
+    with pytest.raises(ValueError):
+        eng.compress(X, X.clone(), X, CANDS3[:2], 1.0, preds=[(PRED_LAZY, 1.0)])

@@ -243,6 +243,60 @@ def test_lemma_adacgd_is_ada3pc():
     assert len(levels) >= 4
 
 
+def test_golden_adaptive_3pc_menu():
+    for case in json.load(open(GOLDEN))["adaptive_3pc"]:
+        h, y, x = (np.array(case[k], dtype=F32) for k in ("h", "y", "x"))
+        cands = [tuple(c) for c in case["cands"]]
+        for z in case["cases"]:
+            res = O.adaptive_3pc(h, y, x, cands, [tuple(q) for q in z["preds"]])
+            assert res["level"] == z["level"], z
+            assert res["out"].tolist() == [float(t) for t in z["out"]], z
+
+
+def test_adaptive_3pc_menu_is_definition_3_and_contains_adacgd():
+    # (a) the menu version against Definition 3 written with callables (`ada3pc`), the compressors being "keep h" and
+    # separately composed EF21 steps; (b) Eq. 10 at every level is AdaCGD (Eq. 11); (c) no skipping and one candidate
+    # is EF21 (Eq. 7); (d) a trigger that always holds at level j stops there
+    r = rng(21)
+    for trial in range(30):
+        d = int(r.integers(3, 40))
+        h, y, x = random_triplet(r, d, integer=(trial % 3 == 0))
+        ks = sorted(set(int(k) for k in r.integers(1, d + 1, size=3)))
+        cands = [(O.TOPK, k) for k in ks]
+        if trial % 2:
+            cands.insert(int(r.integers(0, len(cands) + 1)), (O.QUANT, int(r.integers(2, 6))))
+        m = len(cands)
+        scale = O.sumsq((x - h).astype(F32))
+        preds = []
+        for j in range(m):
+            kind = int(r.integers(0, 5))
+            param = float(r.choice([0.0, 0.1, 0.5, 1.0, 2.0])) * (scale if kind == O.PRED_ABSOLUTE else 1.0)
+            preds.append((kind, param))
+        res = O.adaptive_3pc(h, y, x, cands, preds)
+        # (a)
+        comps = [lambda h_, y_, x_: h_.copy()] + [(lambda c: (lambda h_, y_, x_: O.ef21(h_, y_, x_, c)))(c) for c in cands]
+
+        def make_pred(j):
+            def P(h_, y_, x_):   # the level's error on the difference vector: x - (h + C(x - h)) = v - C(v)
+                v_ = (x_ - h_).astype(F32)
+                return O.trigger_holds(preds[j], O.sumsq(v_) if j == 0 else O.candidate_error(v_, cands[j - 1]), h_, y_, x_)
+            return P
+        want = O.ada3pc(h, y, x, comps, [make_pred(j) for j in range(m)])
+        assert np.array_equal(res["out"].view(np.uint32), want.view(np.uint32)), (trial, preds)
+        # (b)
+        for zeta in (0.0, 0.5, 2.0):
+            a = O.adacgd(h, y, x, cands, zeta)
+            b = O.adaptive_3pc(h, y, x, cands, [(O.PRED_LAZY, zeta)] * m)
+            assert a["level"] == b["level"] and np.array_equal(a["out"].view(np.uint32), b["out"].view(np.uint32))
+        # (c)
+        e = O.adaptive_3pc(h, y, x, cands[:1], [(O.PRED_NEVER, 0.0)])
+        assert e["level"] == 1 and np.array_equal(e["out"].view(np.uint32), O.ef21(h, y, x, cands[0]).view(np.uint32))
+        # (d)
+        j = int(r.integers(0, m))
+        stop = O.adaptive_3pc(h, y, x, cands, [(O.PRED_NEVER, 0.0)] * j + [(O.PRED_ALWAYS, 0.0)] * (m - j))
+        assert stop["level"] == j
+
+
 def test_trigger_postcondition_and_monotone_in_zeta():
     r = rng(9)
     cands = [(O.TOPK, 1), (O.TOPK, 8), (O.QUANT, 4), (O.TOPK, 100)]
