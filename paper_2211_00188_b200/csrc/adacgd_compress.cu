@@ -838,7 +838,9 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
                                                      long long d, long long nwin, long long win,
                                                      u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
-                                                     u32* __restrict__ tickets) {
+                                                     u32* __restrict__ tickets, u32* __restrict__ maxkey) {
+  // maxkey != nullptr: every element is sampled (win == 1) and the row maximum is wanted already here, so that the
+  // streaming pass can evaluate the quantisers
   pdl_begin();
   extern __shared__ __align__(16) u32 sh[];  // SBINS / 2 words
   const int row = blockIdx.y;
@@ -849,6 +851,7 @@ __global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X
   const long long ngran = (d + SAMP_G - 1) / SAMP_G;
   const long long nquad = (long long)gridDim.x * (SAMP_TPB / 4);
   const int ql = threadIdx.x & 3;
+  u32 mxs = 0;
   for (long long w0 = (long long)blockIdx.x * (SAMP_TPB / 4) + (threadIdx.x >> 2); w0 < nwin; w0 += nquad * SAMP_NL) {
     float x[SAMP_NL][4], g[SAMP_NL][4];
     long long c0[SAMP_NL];
@@ -869,10 +872,17 @@ __global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         if (c0[u] + k >= d) break;
-        const u32 bin = key_of(__fsub_rn(x[u][k], g[u][k])) >> 15;
+        const u32 key = key_of(__fsub_rn(x[u][k], g[u][k]));
+        mxs = max(mxs, key);
+        const u32 bin = key >> 15;
         atomicAdd(&sh[bin >> 1], (bin & 1u) ? 0x10000u : 1u);
       }
     }
+  }
+  if (maxkey) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mxs = max(mxs, __shfl_xor_sync(0xffffffffu, mxs, o));
+    if ((threadIdx.x & 31) == 0 && mxs) atomicMax(&maxkey[row], mxs);
   }
   __syncthreads();
   u32* gh = shist + (long long)row * SBINS;
@@ -962,7 +972,8 @@ constexpr int P1_FLUSH_IT = FLUSH_TILES / P1_UNR;                 // iterations 
 #endif
 // resident CTAs per SM the register budget is set for: more brackets need more state per thread
 constexpr int p1_min_ctas(int nsel) { return nsel <= 3 ? P1_MINB3 : (nsel <= 5 ? 3 : 2); }
-template <int NSEL, bool ALIGNED, bool QMAX>
+constexpr int P1_NQ = 3;   // quantisers the streaming pass evaluates itself when the row maximum is known beforehand
+template <int NSEL, bool ALIGNED, int QM>
 __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* __restrict__ X, const float* __restrict__ G,
                                                   const float* __restrict__ Y, long long d, CsetDev cs,
                                                   SelRow* __restrict__ sel, double* __restrict__ partial,
@@ -998,6 +1009,19 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
   float fD = 0.f, fE = 0.f;
   double dD = 0.0, dE = 0.0;
   u32 mx = 0, df = 0;
+  // QM == 2: scale, reciprocal and step of the row's quantisers (the maximum comes from the sampling kernel)
+  constexpr int NQR = (QM == 2) ? P1_NQ : 1;
+  float qL[NQR], qinv[NQR], qstep[NQR], fQ[NQR];
+  double dQ[NQR];
+#pragma unroll
+  for (int q = 0; q < NQR; ++q) {
+    qL[q] = qinv[q] = qstep[q] = fQ[q] = 0.f; dQ[q] = 0.0;
+    if (QM == 2 && q < cs.nquant) {
+      const float smax = __uint_as_float(__ldcg(&maxkey[row]));
+      qL[q] = (float)((1 << ((int)cs.param[cs.qsel[q]] - 1)) - 1);
+      if (smax > 0.f) { qinv[q] = __fdiv_rn(qL[q], smax); qstep[q] = __fdiv_rn(smax, qL[q]); }
+    }
+  }
   __syncthreads();
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
@@ -1068,7 +1092,14 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
         fE = fmaf(v, v, fE);
         fD = fmaf(w, w, fD);
         av[k] = fabsf(v);
-        if (QMAX) mx = max(mx, __float_as_uint(av[k]));
+        if (QM == 1) mx = max(mx, __float_as_uint(av[k]));
+        if (QM == 2) {
+#pragma unroll
+          for (int q = 0; q < P1_NQ; ++q) {
+            const float rq = __fsub_rn(v, quant_value(v, qL[q], qinv[q], qstep[q]));
+            fQ[q] = fmaf(rq, rq, fQ[q]);   // a quantiser that is not in the list has L = 0: its slot is never read
+          }
+        }
         df |= __float_as_uint(v) ^ __float_as_uint(w);
         if (NSEL > 0) {
           // finite non-negative binary32 values order like their bit patterns: compare as floats
@@ -1099,6 +1130,10 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
       dBall += (double)fBall; fBall = 0.f;
 #pragma unroll
       for (int j = 0; j < NS; ++j) { dB[j] += (double)fB[j]; fB[j] = 0.f; }
+      if (QM == 2) {
+#pragma unroll
+        for (int q = 0; q < NQR; ++q) { dQ[q] += (double)fQ[q]; fQ[q] = 0.f; }
+      }
     }
   }
   if (NSEL > 0) {  // what is left in the queue: fewer than 32 entries
@@ -1113,6 +1148,14 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
 
   __shared__ double red[2 + NS][TPB / 32];
   __shared__ u32 redc[NS][TPB / 32];
+  __shared__ double redq[NQR][TPB / 32];
+  if (QM == 2) {
+#pragma unroll
+    for (int q = 0; q < NQR; ++q) {
+      const double vq = warp_sum_f64(dQ[q] + (double)fQ[q]);
+      if (lane == 0) redq[q][wid] = vq;
+    }
+  }
   double v0 = warp_sum_f64(dD), v1 = warp_sum_f64(dE);
   if (lane == 0) { red[0][wid] = v0; red[1][wid] = v1; }
 #pragma unroll
@@ -1139,6 +1182,12 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
     for (int w = 0; w < TPB / 32; ++w) acc += red[s][w];
     const int slot = (s < 2) ? s : 2 + cs.sel[s - 2];
     partial[pbase * NSLOT + slot] = acc;
+  }
+  if (QM == 2 && threadIdx.x >= 64 && threadIdx.x < 64 + cs.nquant) {
+    const int q = threadIdx.x - 64;
+    double acc = 0;
+    for (int w = 0; w < TPB / 32; ++w) acc += redq[q][w];
+    partial[pbase * NSLOT + 2 + cs.qsel[q]] = acc;
   }
   if (threadIdx.x >= 32 && threadIdx.x < 32 + NSEL) {
     const int j = threadIdx.x - 32;
@@ -1819,6 +1868,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const int nblk_full = (int)want_full;
   const dim3 fgrid(nblk_full, rows);
   const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
+  bool qinline = false;                            // the streaming pass evaluates the quantisers itself
   double tol = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
 
 #define TIMED_HIST(id, PASS, shm, hist)                                                                          \
@@ -1831,11 +1881,14 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
       s.diffflag, s.flags, s.fhist, s.tickets
 #define PASS1_CASE(N)                                                                                               \
   case N:                                                                                                           \
-    if (al) {                                                                                                       \
-      if (cs.nquant) launch_k(k_pass1<N, true, true>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                   \
-      else launch_k(k_pass1<N, true, false>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                            \
+    if (qinline) {                                                                                                  \
+      if (al) launch_k(k_pass1<N, true, 2>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                             \
+      else launch_k(k_pass1<N, false, 2>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                               \
+    } else if (al) {                                                                                                \
+      if (cs.nquant) launch_k(k_pass1<N, true, 1>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                      \
+      else launch_k(k_pass1<N, true, 0>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                \
     } else {                                                                                                        \
-      launch_k(k_pass1<N, false, true>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                 \
+      launch_k(k_pass1<N, false, 1>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                    \
     }                                                                                                               \
     break;
 #define LIST_PASS(LEVEL, shm, hist)                                                                              \
@@ -1858,9 +1911,13 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     const long long quads = SAMP_TPB / 4;
     if (sgx > (nwin + quads - 1) / quads) sgx = (nwin + quads - 1) / quads;
     const dim3 samp_grid((unsigned)sgx, rows);
+    // every element sampled and few quantisers: the sample yields the row maximum and the streaming pass the
+    // quantisers' errors, so that no further pass over X and G is needed for them
+    qinline = cs.nquant > 0 && cs.nquant <= P1_NQ && win == 1;
+    u32* samp_max = qinline ? s.maxkey : nullptr;
     prof_begin(pf, KID_SAMPLE, stream);
-    if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets);
-    else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets);
+    if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
+    else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
     prof_end(pf, stream);
     ++launches;
     // 2. the one pass over X, G, Y
@@ -1884,7 +1941,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     const dim3 lhgrid((unsigned)(lgx < 16 ? lgx : 16), rows);
     TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), (size_t)cs.nsel * FINISH_WORDS * 4, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
                                  s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
-                                 cs.nquant == 0 ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
+                                 (cs.nquant == 0 || qinline) ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
                                  s.diffflag, tol));
     // rows whose first-digit bin holds too many keys: three digit levels of 11, 11 and 9 bits (usually no row)
     LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
@@ -1898,7 +1955,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
   }
   TIMED_AL(KID_ENERGY, k_energy, fgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
-  if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
+  if (cs.nquant && !qinline) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
   TIMED(KID_PICK, launch_k(k_pick, dim3(rows), dim3(TPB), 0, stream, pdl, cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey,
                            s.dec, s.flags, out, s.diffflag, single ? s.tickets : nullptr, tol));
   TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag, d, out, s.tickets, s.flags);

@@ -375,6 +375,22 @@ def test_single_pass_with_quantisers(torch):
         check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
 
 
+@pytest.mark.parametrize("d", [60_000, 60_001])
+def test_single_pass_quantiser_errors_inside_the_streaming_pass(torch, d):
+    # rows short enough that the sampling kernel reads every element: it then also yields the row maximum, and the
+    # streaming pass evaluates up to three quantisers itself (no separate pass, level picked with the collection)
+    X, G, Y = S.gaussian_rows(12, d, seed=55)
+    X[3] *= 1e-3; G[3] *= 1e-3; Y[3] *= 1e-3                     # rows of different scale
+    X[7, 11] = 40.0                                                # one dominant entry: coarse quantisers lose the rest
+    cands = [(TOPK, 60), (QUANT, 2), (TOPK, 600), (QUANT, 4), (TOPK, 6000), (QUANT, 8)]
+    seen = set()
+    for zeta in (0.02, 0.3, 5.0, 8.5):
+        got, res = check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+        seen.update(r["level"] for r in res)
+        assert got["fallbacks"] == 0
+    assert seen >= {0, 2, 4, 6}                                    # skip, a Top-K level, two quantiser levels
+
+
 def test_single_pass_crowded_threshold_bin(torch):
     # 30 000 magnitudes within a few units in the last place around the 1 % threshold: the first-digit bin of
     # that bracket holds far more keys than the collection buffer, so the row takes the three-level list passes
