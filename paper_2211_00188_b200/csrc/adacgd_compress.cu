@@ -895,6 +895,95 @@ __global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X
     bracket_row(cs, row, d, win == 1 ? 1 : 0, shist, sel, tickets);
 }
 
+// The same brackets for rows short enough to be read in full by one CTA (d < 2^18) when there are many
+// rows: the histogram, on key[30:16], stays in shared memory with 32-bit counts, the bracket of a candidate is
+// the bin that holds its K-th largest key (exact, since every element is counted), and nothing goes through
+// global memory but the brackets themselves.  Also yields the row maximum.
+constexpr int RS_BINS = 32768;
+constexpr int RS_SHIFT = 16;
+template <bool ALIGNED>
+__global__ void __launch_bounds__(SAMP_TPB) k_sample_row(const float* __restrict__ X, const float* __restrict__ G, long long d,
+                                                         CsetDev cs, SelRow* __restrict__ sel, u32* __restrict__ tickets,
+                                                         u32* __restrict__ maxkey) {
+  pdl_begin();
+  extern __shared__ __align__(16) u32 sh[];   // RS_BINS counts
+  __shared__ u32 wsum[SAMP_TPB / 32];
+  const int row = blockIdx.x;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < RS_BINS / 4; i += SAMP_TPB) reinterpret_cast<uint4*>(sh)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  const float* xr = X + (long long)row * d;
+  const float* gr = G + (long long)row * d;
+  u32 mx = 0;
+  for (long long base = (long long)threadIdx.x * 4; base < d; base += (long long)SAMP_TPB * 4 * SAMP_NL) {
+    float x[SAMP_NL][4], g[SAMP_NL][4];
+#pragma unroll
+    for (int u = 0; u < SAMP_NL; ++u) {
+      const long long c0 = base + (long long)u * SAMP_TPB * 4;
+      if (c0 < d) {
+        load4<ALIGNED>(xr, c0, d, x[u]);
+        load4<ALIGNED>(gr, c0, d, g[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < SAMP_NL; ++u) {
+      const long long c0 = base + (long long)u * SAMP_TPB * 4;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (c0 + k >= d) break;
+        const u32 key = key_of(__fsub_rn(x[u][k], g[u][k]));
+        mx = max(mx, key);
+        atomicAdd(&sh[key >> RS_SHIFT], 1u);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) wsum[wid] = mx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u32 m = 0;
+    for (int w = 0; w < SAMP_TPB / 32; ++w) m = max(m, wsum[w]);
+    maxkey[row] = m;
+  }
+  __syncthreads();
+  // thread t owns the RS_BINS / SAMP_TPB = 32 bins at descending positions 32 t .. 32 t + 31
+  constexpr int PER = RS_BINS / SAMP_TPB;
+  u32 mine = 0;
+#pragma unroll 8
+  for (int k = 0; k < PER; ++k) mine += sh[RS_BINS - 1 - (threadIdx.x * PER + k)];
+  u32 inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u32 t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[wid] = inc;
+  __syncthreads();
+  u32 before = 0;
+  for (int w = 0; w < wid; ++w) before += wsum[w];
+  const u32 excl = before + inc - mine;                 // keys in bins above this thread's
+  for (int j = 0; j < cs.nsel; ++j) {
+    const u32 K = (u32)cs.param[cs.sel[j]];             // K < d: the K-th largest key exists
+    if (K > excl && K <= excl + mine) {
+      u32 run = excl;
+      for (int k = 0; k < PER; ++k) {
+        const u32 bin = (u32)(RS_BINS - 1 - (threadIdx.x * PER + k));
+        const u32 c = sh[bin];
+        if (K <= run + c) {
+          SelRow* sr = sel + row;
+          sr->lo[j] = bin << RS_SHIFT;
+          sr->hi[j] = (bin + 1u) << RS_SHIFT;
+          sr->sh1[j] = RS_SHIFT - 11;                    // digits of key - lo inside a bracket of 2^16 key values
+          sr->sh2[j] = 0u;
+          break;
+        }
+        run += c;
+      }
+    }
+  }
+}
+
 // Shift that leaves the first LB1-valued digit of key - lo for a bracket [lo, hi).
 static_assert(LB1 == TPB, "first_digit_scan reads one bin per thread");
 __device__ __forceinline__ u32 first_digit_shift(u32 lo, u32 hi) {
@@ -1629,7 +1718,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; }
 
 struct Layout {
-  size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, sel, dec, partial, energy, tiecnt, total;
+  size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, zero_noshist, sel, dec, partial, energy, tiecnt, total;
   size_t tickets, rowflag, diffflag, shist, lhist1, fhist, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
@@ -1652,12 +1741,14 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
   L.shist = L.lhist1 = L.fhist = L.flcnt = L.cntpart = o;
+  L.zero_noshist = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
-    L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
     L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
     L.fhist = o; o = align_up(o + (size_t)rows * MAXC * LB1 * 4, 256);
+    L.zero_noshist = o;   // the sample histogram comes last: calls that sample per row in shared memory do not clear it
+    L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
   }
   L.zero_end = o;
   L.flags = o; o = align_up(o + 16, 256);
@@ -1693,6 +1784,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->flags = (u32*)(b + L.flags);
   s->zero_begin = b;
   s->zero_bytes = L.zero_end;
+  s->zero_bytes_noshist = L.zero_noshist;
   s->sel = (SelRow*)(b + L.sel);
   s->dec = (RowDec*)(b + L.dec);
   s->partial = (double*)(b + L.partial);
@@ -1781,6 +1873,8 @@ void set_compress_kernel_attributes() {
   cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
   cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
   cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
+  cudaFuncSetAttribute(k_sample_row<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, RS_BINS * 4);
+  cudaFuncSetAttribute(k_sample_row<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, RS_BINS * 4);
 }
 
 // One record per device ordinal, filled at the first use of that device by this process.
@@ -1842,7 +1936,10 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const bool single = (s.list != nullptr) && cs.nsel > 0 && (long long)rows * d >= (1ll << 19);
   prof_begin(pf, KID_MEMSET, stream);
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
-  cudaMemsetAsync(s.zero_begin, 0, s.zero_bytes, stream);  // histograms, limbs, row flags: one contiguous region
+  // every element sampled and many rows: one CTA per row samples into shared memory (no global sample histogram)
+  const long long ngran_all = (d + SAMP_G - 1) / SAMP_G;
+  const bool row_sampler = single && ngran_all / 8192 < 2 && rows >= 32;
+  cudaMemsetAsync(s.zero_begin, 0, row_sampler ? s.zero_bytes_noshist : s.zero_bytes, stream);  // histograms, limbs, row flags
   prof_end(pf, stream);
 
   if (!single && d <= SMALL_DMAX) {
@@ -1916,7 +2013,10 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     qinline = cs.nquant > 0 && cs.nquant <= P1_NQ && win == 1;
     u32* samp_max = qinline ? s.maxkey : nullptr;
     prof_begin(pf, KID_SAMPLE, stream);
-    if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
+    if (row_sampler) {
+      if (al) launch_k(k_sample_row<true>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey);
+      else launch_k(k_sample_row<false>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey);
+    } else if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
     else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
     prof_end(pf, stream);
     ++launches;

@@ -115,6 +115,7 @@ struct Scratch {
   u64* limbs;      // [rows][NSLOT][NLIMB] exact accumulators
   u32* flags;      // [4]: 0 nonfinite seen, 1 #exact rechecks
   void* zero_begin; size_t zero_bytes;  // region cleared at the start of every call
+  size_t zero_bytes_noshist;            // the same without the sample histogram (its last part)
   SelRow* sel;     // [rows]
   RowDec* dec;     // [rows]
   double* partial; // [rows][MAX_BLK_PER_ROW][NSLOT]
