@@ -294,10 +294,11 @@ static adacgd_status init_body(adacgd_ctx* c, const adacgd_problem* problem, con
   c->loglevels = (int*)(b + L.loglevels);
   c->stage = (flags & ADACGD_FLAG_HOST_STAGING) ? (float*)(b + L.stage) : nullptr;
 
-  CK(nullptr, cudaMemsetAsync(c->scr.flags, 0, 16, c->stream), "adacgd_init (clearing the status words)");
+  CK(nullptr, cudaMemsetAsync(c->scr.flags, 0, 64, c->stream), "adacgd_init (clearing the status words)");
   CK(nullptr, cudaMemsetAsync(c->counters, 0, sizeof(Counters), c->stream), "adacgd_init (clearing the counters)");
   if (has_loss) {
     carve_grad_scratch(&c->gs, b + L.grad, *problem, flags);
+    CK(nullptr, cudaMemsetAsync(c->gs.loss_ticket, 0, c->gs.ticket_bytes, c->stream), "adacgd_init (clearing the gradient tickets)");
     if (c->gs.inc && build_transposed_features(*problem, c->gs, c->stream) < 0)
       return cuda_fail(nullptr, "adacgd_init (column-major copy of the features)");
     if (problem->layout == ADACGD_LAYOUT_CSR) {

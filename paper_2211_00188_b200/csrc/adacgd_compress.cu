@@ -1751,7 +1751,7 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
   }
   L.zero_end = o;
-  L.flags = o; o = align_up(o + 16, 256);
+  L.flags = o; o = align_up(o + 64, 256);   // status words 0-3, word 8: completion count of the short-row kernel
   L.sel = o; o = align_up(o + (size_t)rows * sizeof(SelRow), 256);
   L.dec = o; o = align_up(o + (size_t)rows * sizeof(RowDec), 256);
   L.partial = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * NSLOT * 8, 256);
@@ -1934,6 +1934,17 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   // Small problems live in L2 and are bound by launch latency: the plain three-pass select needs fewer
   // kernels there than sampling + streaming pass + list passes.
   const bool single = (s.list != nullptr) && cs.nsel > 0 && (long long)rows * d >= (1ll << 19);
+  if (!single && d <= SMALL_DMAX) {
+    // short rows: everything in one launch, one CTA per row, then the mean; the kernel keeps its tables in shared
+    // memory and writes every record it reads, so nothing of the scratch has to be cleared
+    if (out.kept_cnt) {
+      prof_begin(pf, KID_MEMSET, stream);
+      cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
+      prof_end(pf, stream);
+    }
+    const int n = launch_small_rows(s, cs, X, G, Y, rows, d, out, stream, pdl);
+    return n < 0 ? -1 : launches + n;
+  }
   prof_begin(pf, KID_MEMSET, stream);
   if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
   // every element sampled and many rows: one CTA per row samples into shared memory (no global sample histogram)
@@ -1941,12 +1952,6 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   const bool row_sampler = single && ngran_all / 8192 < 2 && rows >= 32;
   cudaMemsetAsync(s.zero_begin, 0, row_sampler ? s.zero_bytes_noshist : s.zero_bytes, stream);  // histograms, limbs, row flags
   prof_end(pf, stream);
-
-  if (!single && d <= SMALL_DMAX) {
-    // short rows: everything in one launch, one CTA per row, then the mean
-    const int n = launch_small_rows(s, cs, X, G, Y, rows, d, out, stream, pdl);
-    return n < 0 ? -1 : launches + n;
-  }
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
   long long want = (SMS * 4 + rows - 1) / rows;   // one wave of the streaming pass: four resident CTAs per SM

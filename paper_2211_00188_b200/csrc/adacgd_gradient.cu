@@ -38,11 +38,92 @@ __device__ __forceinline__ void residual(int loss, float z, float t, float inv_m
   }
 }
 
+// f(x) = (1/n) sum_i [ (1/m) sum_l loss_l + reg(x) ] in binary64, finished by whichever CTA of the forward kernel
+// comes last.  Every CTA leaves the loss of its sample rows and the regulariser of its share of x; the last one
+// (a ticket that it resets for the next launch) adds both lists up, thread t taking entries t, t + blockDim, ...
+// and then lanes and warps, so the sum depends on the launch shape only.
+struct LossTail {
+  double* losspart;   // [CTAs of the launch]
+  double* regpart;    // [CTAs of the launch]
+  u32* ticket;
+  const float* x;
+  long long d, m_rows;
+  int loss, n;
+  float lambda;
+  double* out;
+  int fused;          // 0: the CTAs only leave their losses; k_loss_reduce adds them up (grids of thousands of short CTAs,
+                      // where a completion count at the end of every CTA costs more than one more launch)
+};
+__device__ __forceinline__ double block_sum_f64(double v, double* red32) {   // result valid in thread 0
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if (lane == 0) red32[wid] = v;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0)
+    for (int w = 0; w < nw; ++w) t += red32[w];
+  return t;
+}
+// Called by every thread of every CTA (a 2-D grid); `cta_loss` is read from thread 0.  The regulariser is left to
+// the first ceil(d / REG_SLICE) CTAs (the others have nothing to add), and the completion count has two levels, one
+// word per grid row and one for the rows, so that thousands of short CTAs do not queue up on a single address.
+constexpr int REG_SLICE = 4096;
+__device__ void loss_tail(const LossTail& t, double cta_loss) {
+  __shared__ double lt_red[32];
+  __shared__ u32 lt_last;
+  const long long ncta = (long long)gridDim.x * gridDim.y;
+  const long long cta = (long long)blockIdx.y * gridDim.x + blockIdx.x;
+  if (!t.fused) {
+    if (threadIdx.x == 0) t.losspart[cta] = cta_loss;
+    return;
+  }
+  const bool has_reg = t.loss == ADACGD_LOSS_LOGISTIC_NCVX || t.loss == ADACGD_LOSS_LOGISTIC_L2;
+  long long per = REG_SLICE;
+  while ((t.d + per - 1) / per > ncta) per *= 2;
+  const long long nreg = has_reg ? (t.d + per - 1) / per : 0;
+  if (cta < nreg) {
+    double rg = 0.0;
+    const long long c0 = cta * per, c1 = (c0 + per < t.d) ? c0 + per : t.d;
+    for (long long c = c0 + threadIdx.x; c < c1; c += blockDim.x) {
+      const double xv = (double)t.x[c];
+      rg += (t.loss == ADACGD_LOSS_LOGISTIC_NCVX) ? xv * xv / (1.0 + xv * xv) : 0.5 * xv * xv;
+    }
+    rg = block_sum_f64(rg, lt_red);
+    if (threadIdx.x == 0) t.regpart[cta] = rg;
+  }
+  if (threadIdx.x == 0) {
+    t.losspart[cta] = cta_loss;
+    __threadfence();
+    u32 last = 0u;
+    if (atomicAdd(&t.ticket[1 + blockIdx.y], 1u) == gridDim.x - 1u) {        // last CTA of this grid row
+      t.ticket[1 + blockIdx.y] = 0u;
+      __threadfence();
+      last = (atomicAdd(&t.ticket[0], 1u) == gridDim.y - 1u) ? 1u : 0u;       // last grid row
+    }
+    lt_last = last;
+  }
+  __syncthreads();
+  if (!lt_last) return;
+  __threadfence();
+  double a = 0.0, b = 0.0;
+  for (long long i = threadIdx.x; i < ncta; i += blockDim.x) a += __ldcg(&t.losspart[i]);
+  for (long long i = threadIdx.x; i < nreg; i += blockDim.x) b += __ldcg(&t.regpart[i]);
+  a = block_sum_f64(a, lt_red);
+  b = block_sum_f64(b, lt_red);
+  if (threadIdx.x == 0) {
+    *t.out = a / ((double)t.m_rows * (double)t.n) + (double)t.lambda * b;
+    t.ticket[0] = 0u;
+  }
+}
+
 // One warp (CTA_ROW = false) or one CTA (CTA_ROW = true) per sample row.
-template <bool CTA_ROW, bool ALIGNED>
+// FUSED: the last CTA adds up the loss (loss_tail); otherwise every CTA only leaves its share for k_loss_reduce.
+template <bool CTA_ROW, bool ALIGNED, bool FUSED>
 __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, const float* __restrict__ target,
                                                    const float* __restrict__ x, long long d, long long m_rows,
-                                                   int loss, float* __restrict__ r, double* __restrict__ losspart,
+                                                   int loss, float* __restrict__ r, LossTail lt,
                                                    float* __restrict__ zout, const u32* __restrict__ gate) {
   // r == nullptr: only the products z = A x are wanted (zout); gate != nullptr: the launch only runs when the
   // word is zero (the incremental pass found too many changed columns and leaves the products to this kernel)
@@ -98,17 +179,16 @@ __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, 
     }
   }
   if (r == nullptr) return;
-  if (CTA_ROW) {
-    if (threadIdx.x == 0) losspart[(long long)worker * gridDim.x + blockIdx.x] = l;
-  } else {
+  if (!CTA_ROW) {
     if (lane == 0) ls[wid] = l;
     __syncthreads();
     if (threadIdx.x == 0) {
-      double s = 0.0;
-      for (int w = 0; w < TPB / 32; ++w) s += ls[w];
-      losspart[(long long)worker * gridDim.x + blockIdx.x] = s;
+      l = 0.0;
+      for (int w = 0; w < TPB / 32; ++w) l += ls[w];
     }
   }
+  if (FUSED) loss_tail(lt, l);
+  else if (threadIdx.x == 0) lt.losspart[(long long)worker * gridDim.x + blockIdx.x] = l;
 }
 
 __device__ __forceinline__ float reg_grad(int loss, float lambda, float x) {
@@ -125,7 +205,7 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_dense_bwd(const float* __restrict__ A, const float* __restrict__ r,
                                                    const float* __restrict__ x, long long d, long long m_rows,
                                                    int split, int loss, float lambda, float* __restrict__ grads,
-                                                   float* __restrict__ part, int n) {
+                                                   float* __restrict__ part, int n, u32* __restrict__ tickets) {
   const int worker = blockIdx.y / split, s = blockIdx.y % split;
   const long long per = (m_rows + split - 1) / split;
   const long long l0 = s * per, l1 = (l0 + per < m_rows) ? l0 + per : m_rows;
@@ -166,7 +246,6 @@ __global__ void __launch_bounds__(TPB) k_dense_bwd(const float* __restrict__ A, 
       }
     }
   }
-  if (c0 >= d) return;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     if (c0 + k >= d) break;
@@ -174,23 +253,33 @@ __global__ void __launch_bounds__(TPB) k_dense_bwd(const float* __restrict__ A, 
     if (split == 1) grads[(long long)worker * d + c0 + k] = v + reg_grad(loss, lambda, x[c0 + k]);
     else part[((long long)s * n + worker) * d + c0 + k] = v;
   }
-}
-
-__global__ void k_grad_reduce(const float* __restrict__ part, const float* __restrict__ x, long long d, int n,
-                              int split, int loss, float lambda, float* __restrict__ grads) {
-  const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int worker = blockIdx.y;
-  if (c >= d) return;
-  float v = 0.f;
-  for (int s = 0; s < split; ++s) v += part[((long long)s * n + worker) * d + c];
-  grads[(long long)worker * d + c] = v + reg_grad(loss, lambda, x[c]);
+  if (split == 1) return;
+  // the slice of a column tile that finishes last adds the slices up, in slice order
+  __shared__ u32 is_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u32* t = &tickets[(long long)worker * gridDim.x + blockIdx.x];
+    is_last = (atomicAdd(t, 1u) == (u32)(split - 1)) ? 1u : 0u;
+    if (is_last) *t = 0u;   // ready for the next launch
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (c0 + k >= d) break;
+    float v = 0.f;
+    for (int q = 0; q < split; ++q) v += __ldcg(&part[((long long)q * n + worker) * d + c0 + k]);
+    grads[(long long)worker * d + c0 + k] = v + reg_grad(loss, lambda, x[c0 + k]);
+  }
 }
 
 // CSR forward: one warp per sample row.
 __global__ void __launch_bounds__(TPB) k_csr_fwd(const long long* __restrict__ rowptr, const int* __restrict__ col,
                                                  const float* __restrict__ val, const float* __restrict__ target,
                                                  const float* __restrict__ x, long long m_rows, int loss,
-                                                 float* __restrict__ r, double* __restrict__ losspart) {
+                                                 float* __restrict__ r, LossTail lt) {
   const int worker = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const long long row = (long long)blockIdx.x * LOSS_BLOCK_ROWS + wid;
@@ -229,10 +318,10 @@ __global__ void __launch_bounds__(TPB) k_csr_fwd(const long long* __restrict__ r
   if (lane == 0) ls[wid] = l;
   __syncthreads();
   if (threadIdx.x == 0) {
-    double s = 0.0;
-    for (int w = 0; w < TPB / 32; ++w) s += ls[w];
-    losspart[(long long)worker * gridDim.x + blockIdx.x] = s;
+    l = 0.0;
+    for (int w = 0; w < TPB / 32; ++w) l += ls[w];
   }
+  loss_tail(lt, l);
 }
 
 // CSR backward on the transposed copy: one thread per column, entries in ascending sample row.
@@ -314,7 +403,7 @@ __global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long
 // z = sum over the column blocks (in block order), residual and loss of every sample row.
 __global__ void __launch_bounds__(TPB) k_csr_residual(const float* __restrict__ zpart, int nb, long long rows,
                                                       const float* __restrict__ target, long long m_rows, int loss,
-                                                      float* __restrict__ r, double* __restrict__ losspart) {
+                                                      float* __restrict__ r, LossTail lt) {
   const int worker = blockIdx.y;
   const long long l = (long long)blockIdx.x * TPB + threadIdx.x;
   double ls = 0.0;
@@ -331,11 +420,10 @@ __global__ void __launch_bounds__(TPB) k_csr_residual(const float* __restrict__ 
   for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    double t = 0.0;
+  double t = 0.0;
+  if (threadIdx.x == 0)
     for (int w = 0; w < TPB / 32; ++w) t += red[w];
-    losspart[(long long)worker * gridDim.x + blockIdx.x] = t;
-  }
+  loss_tail(lt, t);
 }
 
 // ---- CSR backward on the transposed copy, one contiguous span per warp --------------------------------
@@ -432,13 +520,13 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
   }
 }
 
-// f(x) = (1/n) sum_i [ (1/m) sum_l loss_l + reg(x) ]  in binary64, fixed summation order.
-__global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__ losspart, int n, int blocks,
+// The same sum by a kernel of its own, for forward launches whose CTAs do not count themselves.
+__global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__ losspart, long long nparts, int n,
                                                       long long m_rows, const float* __restrict__ x, long long d,
                                                       int loss, float lambda, double* __restrict__ out) {
   __shared__ double red[32];
   double a = 0.0;
-  for (long long i = threadIdx.x; i < (long long)n * blocks; i += blockDim.x) a += losspart[i];
+  for (long long i = threadIdx.x; i < nparts; i += blockDim.x) a += losspart[i];
   a /= ((double)m_rows * (double)n);
   double rg = 0.0;
   if (loss == ADACGD_LOSS_LOGISTIC_NCVX || loss == ADACGD_LOSS_LOGISTIC_L2) {
@@ -448,18 +536,9 @@ __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__
     }
     rg *= (double)lambda;
   }
-  a += rg;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double s = 0.0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w];
-    *out = s;
-  }
+  a = block_sum_f64(a + rg, red);
+  if (threadIdx.x == 0) *out = a;
 }
-
 
 // ---- incremental forward: z_i = A_i x kept up to date from the entries of g that changed -----------------
 // x moves by -gamma g every iteration (Algorithm 1), so z_i = A_i x moves by -gamma u_i with u_i = A_i g, and g
@@ -595,7 +674,7 @@ __global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __
                                                                  int nchunk, long long m_rows, float gamma,
                                                                  const float* __restrict__ target, int loss, float* __restrict__ u,
                                                                  float* __restrict__ z, float* __restrict__ r,
-                                                                 double* __restrict__ losspart, const u32* __restrict__ dl_flag) {
+                                                                 LossTail lt, const u32* __restrict__ dl_flag) {
   __shared__ float part[FIN_SLICES][TPB];
   __shared__ double red[TPB / 32];
   const int w = blockIdx.y;
@@ -612,9 +691,8 @@ __global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __
     part[slice][row] = s;
   }
   __syncthreads();
-  if (slice != 0) return;
   double ls = 0.0;
-  if (l < m_rows) {
+  if (slice == 0 && l < m_rows) {
     const long long gi = (long long)w * m_rows + l;
     float zn = z[gi];
     if (gathered) {
@@ -631,13 +709,12 @@ __global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
-  asm volatile("bar.sync 1, %0;" ::"n"(TPB));   // only the first slice's threads are left
-  if (threadIdx.x == 0) {
-    double t = 0.0;
+  if (slice == 0 && (threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ls;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0)
     for (int k = 0; k < TPB / 32; ++k) t += red[k];
-    losspart[(long long)w * gridDim.x + blockIdx.x] = t;
-  }
+  loss_tail(lt, t);
 }
 
 // --------------------------------------------------------------------------
@@ -645,6 +722,17 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout, cudaStream_t stream,
                       const u32* gate = nullptr);
+// Above this many short CTAs (a few sample rows each) in a forward launch the loss is added up by k_loss_reduce
+// instead of the last CTA; a CTA that walks a whole long row does not notice the count at its end.
+constexpr long long FUSED_LOSS_MAX_CTAS = 1024;
+static long long dense_fwd_short_ctas(const adacgd_problem& p, const GradScratch& g);
+static LossTail make_tail(const adacgd_problem& p, const GradScratch& g, const float* x, long long ctas = 0) {
+  LossTail t;
+  t.fused = ctas <= FUSED_LOSS_MAX_CTAS ? 1 : 0;
+  t.losspart = g.losspart; t.regpart = g.regpart; t.ticket = g.loss_ticket; t.x = x; t.d = p.d; t.m_rows = p.m_rows;
+  t.loss = p.loss; t.n = p.n; t.lambda = p.lambda; t.out = g.loss;
+  return t;
+}
 int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks, bool al,
                               cudaStream_t stream);
 
@@ -709,7 +797,9 @@ size_t grad_scratch_bytes(const adacgd_problem& p, int flags) {
   const int split = choose_split(p);
   if (split > 1) o = align_up(o + (size_t)split * p.n * p.d * 4, 256);
   o = align_up(o + (size_t)p.n * loss_blocks_of(p) * 8, 256);
+  o = align_up(o + (size_t)p.n * loss_blocks_of(p) * 8, 256);   // regpart
   o = align_up(o + 8, 256);
+  o = align_up(o + 4 * (1 + (size_t)p.n) + (size_t)p.n * ((p.d + TPB * 4 - 1) / (TPB * 4)) * 4, 256);   // loss tickets, backward tickets
   if (p.layout == ADACGD_LAYOUT_CSR) {
     o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
     o = align_up(o + (size_t)p.csr_nnz * 4, 256);
@@ -752,7 +842,12 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int
   g->part = nullptr;
   if (g->split > 1) { g->part = (float*)(b + o); o = align_up(o + (size_t)g->split * p.n * p.d * 4, 256); }
   g->losspart = (double*)(b + o); o = align_up(o + (size_t)p.n * g->loss_blocks * 8, 256);
+  g->regpart = (double*)(b + o); o = align_up(o + (size_t)p.n * g->loss_blocks * 8, 256);
   g->loss = (double*)(b + o); o = align_up(o + 8, 256);
+  g->loss_ticket = (u32*)(b + o);
+  g->bwd_tickets = g->loss_ticket + 1 + p.n;
+  g->ticket_bytes = 4 * (1 + (size_t)p.n) + (size_t)p.n * ((p.d + TPB * 4 - 1) / (TPB * 4)) * 4;
+  o = align_up(o + g->ticket_bytes, 256);
   g->csc_ptr = nullptr; g->csc_row = nullptr; g->csc_val = nullptr;
   g->nb = 0; g->blk = 0; g->csr_split = nullptr; g->zpart = nullptr; g->ccols = 0; g->wbase = nullptr; g->ptr32 = nullptr;
   if (p.layout == ADACGD_LAYOUT_CSR) {
@@ -793,13 +888,13 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
       loss_blocks = (int)((p.m_rows + TPB - 1) / TPB);
       prof_begin(g.prof, KID_CSR_RES, stream);
       k_csr_residual<<<dim3((unsigned)loss_blocks, p.n), TPB, 0, stream>>>(g.zpart, g.nb, rows, p.target, p.m_rows, p.loss,
-                                                                           g.r, g.losspart);
+                                                                           g.r, make_tail(p, g, x));
       prof_end(g.prof, stream);
       ++launches;
     } else {
       prof_begin(g.prof, KID_CSR_FWD, stream);
       k_csr_fwd<<<dim3((unsigned)g.loss_blocks, p.n), TPB, 0, stream>>>((const long long*)p.csr_rowptr, p.csr_col, p.csr_val,
-                                                                        p.target, x, p.m_rows, p.loss, g.r, g.losspart);
+                                                                        p.target, x, p.m_rows, p.loss, g.r, make_tail(p, g, x));
       prof_end(g.prof, stream);
       ++launches;
     }
@@ -818,17 +913,23 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
                                                                                   p.d, p.m_rows, p.loss, p.lambda, grads);
     prof_end(g.prof, stream);
     ++launches;
-    prof_begin(g.prof, KID_LOSS, stream);
-    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
-    prof_end(g.prof, stream);
-    ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
   launch_dense_fwd(p, g, x, g.r, nullptr, stream);
   ++launches;
+  if (dense_fwd_short_ctas(p, g) > FUSED_LOSS_MAX_CTAS) {
+    prof_begin(g.prof, KID_LOSS, stream);
+    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, (long long)p.n * g.loss_blocks, p.n, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+    prof_end(g.prof, stream);
+    ++launches;
+  }
   return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream);
+}
+
+static long long dense_fwd_short_ctas(const adacgd_problem& p, const GradScratch& g) {
+  return cta_row_mode(p) ? 0 : (long long)p.n * g.loss_blocks;
 }
 
 // The forward kernel in the shape the problem calls for: z = A v for a d-vector v, residuals if r != nullptr.
@@ -836,15 +937,15 @@ void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float
                       cudaStream_t stream, const u32* gate) {
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)v) & 15) == 0;
   prof_begin(g.prof, KID_GRAD_FWD, stream);
-  if (cta_row_mode(p)) {
-    const dim3 grid((unsigned)p.m_rows, p.n);
-    if (al) k_dense_fwd<true, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
-    else k_dense_fwd<true, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
-  } else {
-    const dim3 grid((unsigned)g.loss_blocks, p.n);
-    if (al) k_dense_fwd<false, true><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
-    else k_dense_fwd<false, false><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, g.losspart, zout, gate);
-  }
+  const long long fwd_ctas = dense_fwd_short_ctas(p, g);
+  const LossTail lt = make_tail(p, g, v, fwd_ctas);
+  const bool cta_row = cta_row_mode(p);
+  const dim3 grid((unsigned)(cta_row ? p.m_rows : g.loss_blocks), p.n);
+#define FWD(CR, AL, FU) k_dense_fwd<CR, AL, FU><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, lt, zout, gate)
+  if (cta_row) { if (al) FWD(true, true, true); else FWD(true, false, true); }      // long CTAs always count themselves
+  else if (lt.fused) { if (al) FWD(false, true, true); else FWD(false, false, true); }
+  else { if (al) FWD(false, true, false); else FWD(false, false, false); }
+#undef FWD
   prof_end(g.prof, stream);
 }
 
@@ -854,18 +955,8 @@ int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, con
   int launches = 0;
   const dim3 bgrid((unsigned)((p.d + TPB * 4 - 1) / (TPB * 4)), p.n * g.split);
   prof_begin(g.prof, KID_GRAD_BWD, stream);
-  if (al) k_dense_bwd<true><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n);
-  else k_dense_bwd<false><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n);
-  prof_end(g.prof, stream);
-  ++launches;
-  if (g.split > 1) {
-    prof_begin(g.prof, KID_GRAD_REDUCE, stream);
-    k_grad_reduce<<<dim3((unsigned)((p.d + 255) / 256), p.n), 256, 0, stream>>>(g.part, x, p.d, p.n, g.split, p.loss, p.lambda, grads);
-    prof_end(g.prof, stream);
-    ++launches;
-  }
-  prof_begin(g.prof, KID_LOSS, stream);
-  k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, p.n, loss_blocks, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+  if (al) k_dense_bwd<true><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n, g.bwd_tickets);
+  else k_dense_bwd<false><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n, g.bwd_tickets);
   prof_end(g.prof, stream);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
@@ -897,7 +988,7 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
   }
   prof_begin(g.prof, KID_INC_FINISH, stream);
   k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), TPB * FIN_SLICES, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
-                                                                    g.u, g.z, g.r, g.losspart, refresh ? nullptr : g.dl_flag);
+                                                                    g.u, g.z, g.r, make_tail(p, g, x), refresh ? nullptr : g.dl_flag);
   prof_end(g.prof, stream);
   ++launches;
   return launches + launch_dense_bwd_and_loss(p, g, x, grads, fin_blocks, al, stream);

@@ -164,8 +164,12 @@ int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float
 struct GradScratch {
   float* r;         // [n][m_rows] residuals scaled by 1/m
   float* part;      // [split][n][d] partial column sums (split > 1 only)
-  double* losspart; // [n][loss_blocks]
+  double* losspart; // [n][loss_blocks] loss of the sample rows of every CTA of the forward kernel
+  double* regpart;  // [n][loss_blocks] regulariser of every CTA's share of x
   double* loss;     // [1]
+  u32* loss_ticket; // [1 + n] completion counts of the forward kernel: grid rows done, then CTAs done per grid row (reset by the last)
+  u32* bwd_tickets; // [n][column tiles] completion counts of the backward kernel's row slices
+  size_t ticket_bytes;
   int split; int loss_blocks;
   // CSR layout: transposed copy built at init (column-major over all workers: column c of worker i
   // is "row" i*d + c)

@@ -69,7 +69,7 @@ extern "C" adacgd_status adacgd_compress_noalloc(const float* X_dev, float* G_de
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   // the array keeps whatever the previous call left: the status words start from zero here,
   // the histograms and accumulators are cleared by launch_compress itself
-  if (cudaMemsetAsync(s.flags, 0, 16, stream) != cudaSuccess) {
+  if (cudaMemsetAsync(s.flags, 0, 64, stream) != cudaSuccess) {
     set_thread_error("adacgd_compress_noalloc: cudaMemsetAsync failed");
     return ADACGD_ERR_CUDA;
   }

@@ -46,7 +46,9 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
                                                     int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
                                                     double* partial, u32* maxkey, u32* diffflag, u32* flags,
-                                                    CompressOut out, double tol) {
+                                                    CompressOut out, double tol, u32* mean_ticket) {
+  // mean_ticket != nullptr: the rows are so short that the CTA that finishes last also takes the mean over them
+  // (summed in row order, one division), instead of a kernel of its own
   pdl_begin();
   extern __shared__ __align__(16) unsigned char small_smem[];
   const int dn = (int)d;
@@ -404,7 +406,23 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       }
     }
   }
-
+  if (mean_ticket == nullptr) return;
+  __shared__ u32 mean_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mean_last = (atomicAdd(mean_ticket, 1u) == gridDim.x - 1u) ? 1u : 0u;
+    if (mean_last) *mean_ticket = 0u;   // ready for the next call
+  }
+  __syncthreads();
+  if (!mean_last) return;
+  __threadfence();
+  const float nf = (float)rows;
+  for (int c = threadIdx.x; c < dn; c += TPB) {
+    float acc = -0.f;                    // -0 + g == g bit for bit
+    for (int i = 0; i < rows; ++i) acc = __fadd_rn(acc, __ldcg(G + (long long)i * d + c));
+    out.mean_out[c] = __fdiv_rn(acc, nf);
+  }
 }
 
 // The mean over short rows (summed in row order, one division): a thread owns four columns and
@@ -465,13 +483,17 @@ int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float
   const double tol64 = 4.0 * ((double)d + 16.0) * 1.1102230246251565e-16;  // binary64 sums of <= d exact terms
   const bool al4 = (d % 4 == 0) && aligned16(X) && aligned16(G) && aligned16(Y);
   prof_begin(pf, KID_SMALL, stream);
+  // a few thousand entries in all: the last CTA takes the mean as well (the ticket lives in the status words'
+  // block, word 8, zero between calls)
+  const bool tiny_mean = out.mean_out != nullptr && (long long)rows * d <= 16384;
+  u32* mean_ticket = tiny_mean ? s.flags + 8 : nullptr;
   if (al4) launch_k(k_small_rows<true>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                    s.maxkey, s.diffflag, s.flags, out, tol64);
+                    s.maxkey, s.diffflag, s.flags, out, tol64, mean_ticket);
   else launch_k(k_small_rows<false>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                s.maxkey, s.diffflag, s.flags, out, tol64);
+                s.maxkey, s.diffflag, s.flags, out, tol64, mean_ticket);
   prof_end(pf, stream);
   ++launches;
-  if (out.mean_out) {
+  if (out.mean_out && !tiny_mean) {
     const dim3 mgrid((unsigned)((d + TPB * 4 - 1) / (TPB * 4)));
     prof_begin(pf, KID_SMALL, stream);
     if (al4 && aligned16(out.mean_out)) launch_k(k_small_mean<true>, mgrid, dim3(TPB), 0, stream, pdl, (const float*)G, rows, d, out.mean_out);
