@@ -449,12 +449,80 @@ __device__ __forceinline__ void update_rows_simple(const float* __restrict__ X, 
     }
   }
 }
+// The same update for many short rows, one column per thread: a thread of k_update owns four columns of every
+// row, which leaves a 100 x 100 000 problem with 98 CTAs; here it is 391.  Only calls whose rows all take the
+// simple path (skip, Top-K by threshold and index cut, identity, quantiser) are served: the kernel checks that
+// first, and if it does the work it sets `done`, on which the general kernel that follows returns at once.
+constexpr int UPDN_RB = 8;   // rows whose operands a thread keeps in flight
+__global__ void __launch_bounds__(TPB) k_update_narrow(const float* __restrict__ X, float* __restrict__ G, int rows, long long d,
+                                                       const RowDec* __restrict__ dec, CompressOut out, u32* __restrict__ done) {
+  pdl_begin();
+  __shared__ RowDec shd[UPD_ROW_TILE];
+  bool simple = true;
+  for (int i = threadIdx.x; i < rows; i += TPB) {
+    const int m = dec[i].mode;
+    simple = simple && m != 4 && !(m == 1 && dec[i].need_tie);
+  }
+  if (!__syncthreads_and(simple ? 1 : 0)) return;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *done = 1u;
+  const bool want_mean = out.mean_out != nullptr;
+  const long long c = (long long)blockIdx.x * TPB + threadIdx.x;
+  const bool live = c < d;
+  const u32 cu = (u32)c;
+  float acc = -0.f;   // -0 + g == g bit for bit
+  for (int r0 = 0; r0 < rows; r0 += UPD_ROW_TILE) {
+    const int nr = (rows - r0 < UPD_ROW_TILE) ? rows - r0 : UPD_ROW_TILE;
+    __syncthreads();
+    if (threadIdx.x < nr) shd[threadIdx.x] = dec[r0 + threadIdx.x];
+    __syncthreads();
+    if (!live) continue;
+    for (int q0 = 0; q0 < nr; q0 += UPDN_RB) {
+      float gq[UPDN_RB], xq[UPDN_RB];
+#pragma unroll
+      for (int u = 0; u < UPDN_RB; ++u) {
+        gq[u] = 0.f; xq[u] = 0.f;
+        const int ii = q0 + u;
+        if (ii < nr) {
+          const int m = shd[ii].mode;
+          if (m != 0 || want_mean) gq[u] = G[(long long)(r0 + ii) * d + c];
+          if (m != 0) xq[u] = __ldcs(X + (long long)(r0 + ii) * d + c);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < UPDN_RB; ++u) {
+        const int ii = q0 + u;
+        if (ii >= nr) break;
+        float g = gq[u];
+        const int m = shd[ii].mode;
+        if (m != 0) {
+          const float v = __fsub_rn(xq[u], g);
+          bool kept = true;
+          float add = v;
+          if (m == 1) {
+            const u32 T = shd[ii].T;
+            kept = fabsf(v) >= __uint_as_float(cu <= shd[ii].cut ? T : T + 1u);
+          } else if (m == 3) {
+            add = quant_value(v, shd[ii].qL, shd[ii].qinv, shd[ii].qstep);
+          }
+          if (kept) {
+            g = __fadd_rn(g, add);
+            G[(long long)(r0 + ii) * d + c] = g;
+          }
+        }
+        if (want_mean) acc = __fadd_rn(acc, g);
+      }
+    }
+  }
+  if (want_mean && live) out.mean_out[c] = __fdiv_rn(acc, (float)rows);
+}
+
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
-                                                CompressOut out) {
+                                                CompressOut out, const u32* __restrict__ skip_flag) {
   pdl_begin();
+  if (skip_flag && __ldcg(skip_flag)) return;   // the one-column-per-thread kernel has done the work
   __shared__ RowDec shd[UPD_ROW_TILE];
   const int lane = threadIdx.x & 31;
   const bool want_mean = out.mean_out != nullptr;
@@ -1927,7 +1995,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     if (out.kept_cnt) cudaMemsetAsync(out.kept_cnt, 0, (size_t)rows * 8, stream);
     prof_end(pf, stream);
     TIMED(KID_PICK, launch_k(k_copy_report, dim3((rows + 127) / 128), dim3(128), 0, stream, false, rows, d, 0, out));
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out);
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 1, out, (const u32*)nullptr);
     return cudaGetLastError() == cudaSuccess ? launches : -1;
   }
   // clear the per-call accumulators
@@ -2073,7 +2141,16 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // Not a programmatic dependent: launched as one, this persistent grid ran 400 us instead of 270 us on
     // 8 x 25e6 (its CTAs become resident while earlier kernels still hold part of the SMs).
     const bool pdl = false;
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out);
+    // many rows of few chunks: first the kernel with one column per thread, which does the work unless a row needs
+    // the general path (word 14 of the first row's ticket block, cleared with the rest, says whether it did)
+    const u32* skip = nullptr;
+    if (rows >= 16 && nchunk < 2 * SMS && out.kept_idx == nullptr) {
+      u32* done = s.tickets + 14;
+      TIMED(KID_UPDATE, launch_k(k_update_narrow, dim3((unsigned)((d + TPB - 1) / TPB)), dim3(TPB), 0, stream, false, X, G, rows, d,
+                                 (const RowDec*)s.dec, out, done));
+      skip = done;
+    }
+    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, skip);
   }
 #undef LIST_PASS
 #undef PASS1_CASE
