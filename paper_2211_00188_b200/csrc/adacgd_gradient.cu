@@ -667,19 +667,21 @@ __global__ void __launch_bounds__(TPB) k_dense_inc(const float* __restrict__ AT,
 
 // Gathered route (dl_flag[0] = 1): u += the chunks' contributions, z <- z - gamma u (two roundings, like the
 // update of x).  Full route: z has just been recomputed.  Then the residual and the loss of every sample row
-// from z.  A CTA serves TPB sample rows with FIN_SLICES threads per row: each adds a contiguous range of
-// chunks in chunk order, and the ranges are added to u in range order.
-constexpr int FIN_SLICES = 4;
-__global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __restrict__ ipart, const u32* __restrict__ count,
-                                                                 int nchunk, long long m_rows, float gamma,
-                                                                 const float* __restrict__ target, int loss, float* __restrict__ u,
-                                                                 float* __restrict__ z, float* __restrict__ r,
-                                                                 LossTail lt, const u32* __restrict__ dl_flag) {
-  __shared__ float part[FIN_SLICES][TPB];
-  __shared__ double red[TPB / 32];
+// from z.  A CTA serves FIN_ROWS sample rows with FIN_SLICES threads per row: each adds a contiguous range of
+// chunks in chunk order (the ranges are latency chains of dependent loads, so there are many of them), and the
+// ranges are added to u in range order.
+constexpr int FIN_ROWS = 64;
+constexpr int FIN_SLICES = 16;
+__global__ void __launch_bounds__(FIN_ROWS * FIN_SLICES) k_inc_finish(const float* __restrict__ ipart, const u32* __restrict__ count,
+                                                                      int nchunk, long long m_rows, float gamma,
+                                                                      const float* __restrict__ target, int loss, float* __restrict__ u,
+                                                                      float* __restrict__ z, float* __restrict__ r,
+                                                                      LossTail lt, const u32* __restrict__ dl_flag) {
+  __shared__ float part[FIN_SLICES][FIN_ROWS];
+  __shared__ double red[FIN_ROWS / 32];
   const int w = blockIdx.y;
-  const int row = threadIdx.x % TPB, slice = threadIdx.x / TPB;
-  const long long l = (long long)blockIdx.x * TPB + row;
+  const int row = threadIdx.x % FIN_ROWS, slice = threadIdx.x / FIN_ROWS;
+  const long long l = (long long)blockIdx.x * FIN_ROWS + row;
   const bool gathered = dl_flag != nullptr && dl_flag[0] != 0u;   // nullptr: z has just been recomputed (refresh)
   if (gathered) {
     float s = 0.f;
@@ -713,7 +715,7 @@ __global__ void __launch_bounds__(TPB * FIN_SLICES) k_inc_finish(const float* __
   __syncthreads();
   double t = 0.0;
   if (threadIdx.x == 0)
-    for (int k = 0; k < TPB / 32; ++k) t += red[k];
+    for (int k = 0; k < FIN_ROWS / 32; ++k) t += red[k];
   loss_tail(lt, t);
 }
 
@@ -966,7 +968,8 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
                                 float gamma, bool refresh, float* grads, cudaStream_t stream) {
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
-  const int fin_blocks = (int)((p.m_rows + TPB - 1) / TPB);
+  const int fin_blocks = (int)((p.m_rows + FIN_ROWS - 1) / FIN_ROWS);
+  const int inc_tiles = (int)((p.m_rows + TPB - 1) / TPB);
   if (refresh) {
     // z = A x, u = A g, and g is remembered as the vector u belongs to
     launch_dense_fwd(p, g, x, nullptr, g.z, stream);
@@ -980,14 +983,14 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
     k_delta_scan<<<g.inc_chunks, TPB, 0, stream>>>(gvec, g.g_prev, p.d, g.dl_count, g.dl_idx, g.dl_val, g.dl_flag, g.inc_cols, max_cols);
     prof_end(g.prof, stream);
     prof_begin(g.prof, KID_INC, stream);
-    k_dense_inc<<<dim3((unsigned)g.inc_chunks, (unsigned)fin_blocks, p.n), TPB, 0, stream>>>(g.AT, g.dl_count, g.dl_idx, g.dl_val, p.d, p.m_rows,
+    k_dense_inc<<<dim3((unsigned)g.inc_chunks, (unsigned)inc_tiles, p.n), TPB, 0, stream>>>(g.AT, g.dl_count, g.dl_idx, g.dl_val, p.d, p.m_rows,
                                                                                              g.ipart, g.dl_flag, gvec, g.g_prev);
     prof_end(g.prof, stream);
     launch_dense_fwd(p, g, x, nullptr, g.z, stream, g.dl_flag);   // runs only if the scan chose the full route
     launches += 3;
   }
   prof_begin(g.prof, KID_INC_FINISH, stream);
-  k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), TPB * FIN_SLICES, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
+  k_inc_finish<<<dim3((unsigned)fin_blocks, p.n), FIN_ROWS * FIN_SLICES, 0, stream>>>(g.ipart, g.dl_count, g.inc_chunks, p.m_rows, gamma, p.target, p.loss,
                                                                     g.u, g.z, g.r, make_tail(p, g, x), refresh ? nullptr : g.dl_flag);
   prof_end(g.prof, stream);
   ++launches;
