@@ -463,8 +463,10 @@ def bench_dense(args, name, rank, world, local, steps=None, warmup=None, repeats
     a_bytes = 4 * n * m * d if csr is None else 8 * int(csr[1].numel())
     top = max((k for k in ("k_dense_fwd", "k_dense_bwd", "k_csr_fwd", "k_csc_bwd") if k in prof), key=lambda k: prof[k][0])
     achieved = a_bytes * prof[top][1] / (prof[top][0] * 1e-3) / 1e9
+    per_entry = counted_traffic(top)   # counted DRAM bytes per feature entry (dense) or stored entry (CSR)
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": counted_traffic(top), "peak_source": peak_src, "launches": prof[top][1],
+                "frac": achieved / peak, "traffic": None if per_entry is None else per_entry * a_bytes / (4 if csr is None else 8),
+                "peak_source": peak_src, "launches": prof[top][1],
                 "avg_launch_ms": prof[top][0] / prof[top][1]}
     floor = 2 * a_bytes + 20 * n * d + (24 * d if W["master"] else 0)
     step_gbs = floor / (ms / steps * 1e-3) / 1e9
