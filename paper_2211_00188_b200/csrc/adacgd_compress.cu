@@ -906,10 +906,12 @@ template <bool ALIGNED>
 __global__ void __launch_bounds__(SAMP_TPB) k_sample(const float* __restrict__ X, const float* __restrict__ G,
                                                      long long d, long long nwin, long long win,
                                                      u32* __restrict__ shist, CsetDev cs, SelRow* __restrict__ sel,
-                                                     u32* __restrict__ tickets, u32* __restrict__ maxkey) {
+                                                     u32* __restrict__ tickets, u32* __restrict__ maxkey,
+                                                     CsetDev* __restrict__ cs_global) {
   // maxkey != nullptr: every element is sampled (win == 1) and the row maximum is wanted already here, so that the
   // streaming pass can evaluate the quantisers
   pdl_begin();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *cs_global = cs;   // for the last CTAs of the collection pass
   extern __shared__ __align__(16) u32 sh[];  // SBINS / 2 words
   const int row = blockIdx.y;
   for (int i = threadIdx.x; i < SBINS / 8; i += SAMP_TPB) reinterpret_cast<uint4*>(sh)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -972,8 +974,9 @@ constexpr int RS_SHIFT = 16;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(SAMP_TPB) k_sample_row(const float* __restrict__ X, const float* __restrict__ G, long long d,
                                                          CsetDev cs, SelRow* __restrict__ sel, u32* __restrict__ tickets,
-                                                         u32* __restrict__ maxkey) {
+                                                         u32* __restrict__ maxkey, CsetDev* __restrict__ cs_global) {
   pdl_begin();
+  if (blockIdx.x == 0 && threadIdx.x == 0) *cs_global = cs;   // for the last CTAs of the collection pass
   extern __shared__ __align__(16) u32 sh[];   // RS_BINS counts
   __shared__ u32 wsum[SAMP_TPB / 32];
   const int row = blockIdx.x;
@@ -1052,6 +1055,28 @@ __global__ void __launch_bounds__(SAMP_TPB) k_sample_row(const float* __restrict
   }
 }
 
+// Entries of the candidate set by a run-time index, written as compile-time indexed selects: indexing the kernel
+// parameter with a run-time value (or handing its address to a function) makes every thread copy the whole
+// structure to local memory first.
+__device__ __forceinline__ long long cs_param_at(const CsetDev& cs, int c) {
+  long long v = 0;
+#pragma unroll
+  for (int k = 0; k < MAXC; ++k) v = (k == c) ? cs.param[k] : v;
+  return v;
+}
+__device__ __forceinline__ int cs_sel_at(const CsetDev& cs, int j) {
+  int v = 0;
+#pragma unroll
+  for (int k = 0; k < MAXC; ++k) v = (k == j) ? cs.sel[k] : v;
+  return v;
+}
+__device__ __forceinline__ int cs_qsel_at(const CsetDev& cs, int j) {
+  int v = 0;
+#pragma unroll
+  for (int k = 0; k < MAXC; ++k) v = (k == j) ? cs.qsel[k] : v;
+  return v;
+}
+
 // Shift that leaves the first LB1-valued digit of key - lo for a bracket [lo, hi).
 static_assert(LB1 == TPB, "first_digit_scan reads one bin per thread");
 __device__ __forceinline__ u32 first_digit_shift(u32 lo, u32 hi) {
@@ -1064,7 +1089,7 @@ __device__ __forceinline__ u32 first_digit_shift(u32 lo, u32 hi) {
 // (the K-th largest key must be one of the listed keys; otherwise the row is flagged for the full
 // select) and locates the first-digit bin of its threshold.  A bin with more than FINAL_CAP keys
 // sends the row through the three-level list passes.
-__device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, const u32* __restrict__ fhist,
+__device__ __noinline__ void first_digit_scan(int nsel, const long long* s_K, int row, const u32* __restrict__ fhist,
                                               const u32* __restrict__ cnttot, SelRow* __restrict__ sel,
                                               u32* __restrict__ rowflag, u32* __restrict__ tickets,
                                               u32* __restrict__ flags) {
@@ -1074,7 +1099,7 @@ __device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, const 
   SelRow* s = sel + row;
   if (threadIdx.x == 0) { bad = 0; toofull = 0; }
   __syncthreads();
-  if (j < cs.nsel) {
+  if (j < nsel) {
     const u32 above = __ldcg(&cnttot[row * MAXC + j]);            // keys >= hi
     const u32* h = fhist + ((long long)row * MAXC + j) * LB1;
     // bins in descending order: this lane holds positions 8*lane .. 8*lane + 7
@@ -1091,7 +1116,7 @@ __device__ __noinline__ void first_digit_scan(const CsetDev& cs, int row, const 
       if (lane >= o) inc += t;
     }
     const u32 total = __shfl_sync(0xffffffffu, inc, 31);
-    const long long K = cs.param[cs.sel[j]];
+    const long long K = s_K[j];
     if (K <= (long long)above || K > (long long)above + (long long)total) {
       if (lane == 0) bad = 1;
     } else {
@@ -1150,6 +1175,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
   for (int i = threadIdx.x; i < NS * LB1; i += TPB) lh[i] = 0;
   // bracket edges and digit shifts are only read when a queue is drained: kept in shared memory
   __shared__ u32 s_lo[NS], s_hi[NS], s_shq[NS];
+  __shared__ long long s_K[NS];
   u32 cnt[NS];
   float fB[NS];
   double dB[NS];
@@ -1159,7 +1185,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
   for (int j = 0; j < NS; ++j) {
     const u32 lo = (j < NSEL) ? sel[row].lo[j] : 0u;
     const u32 hi = (j < NSEL) ? sel[row].hi[j] : 0u;
-    if (threadIdx.x == 0) { s_lo[j] = lo; s_hi[j] = hi; s_shq[j] = first_digit_shift(lo, hi); }
+    if (threadIdx.x == 0) { s_lo[j] = lo; s_hi[j] = hi; s_shq[j] = first_digit_shift(lo, hi); s_K[j] = cs_param_at(cs, cs_sel_at(cs, j)); }
     cnt[j] = 0; fB[j] = 0.f; dB[j] = 0.0;
     if (j < NSEL) lomin = fminf(lomin, __uint_as_float(lo));       // lo < 2^31 - 2^15: finite or +inf
   }
@@ -1175,7 +1201,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
     qL[q] = qinv[q] = qstep[q] = fQ[q] = 0.f; dQ[q] = 0.0;
     if (QM == 2 && q < cs.nquant) {
       const float smax = __uint_as_float(__ldcg(&maxkey[row]));
-      qL[q] = (float)((1 << ((int)cs.param[cs.qsel[q]] - 1)) - 1);
+      qL[q] = (float)((1 << ((int)cs_param_at(cs, cs_qsel_at(cs, q)) - 1)) - 1);
       if (smax > 0.f) { qinv[q] = __fdiv_rn(qL[q], smax); qstep[q] = __fdiv_rn(smax, qL[q]); }
     }
   }
@@ -1337,14 +1363,14 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
     const int s = threadIdx.x;
     double acc = 0;
     for (int w = 0; w < TPB / 32; ++w) acc += red[s][w];
-    const int slot = (s < 2) ? s : 2 + cs.sel[s - 2];
+    const int slot = (s < 2) ? s : 2 + cs_sel_at(cs, s - 2);
     partial[pbase * NSLOT + slot] = acc;
   }
   if (QM == 2 && threadIdx.x >= 64 && threadIdx.x < 64 + cs.nquant) {
     const int q = threadIdx.x - 64;
     double acc = 0;
     for (int w = 0; w < TPB / 32; ++w) acc += redq[q][w];
-    partial[pbase * NSLOT + 2 + cs.qsel[q]] = acc;
+    partial[pbase * NSLOT + 2 + cs_qsel_at(cs, q)] = acc;
   }
   if (threadIdx.x >= 32 && threadIdx.x < 32 + NSEL) {
     const int j = threadIdx.x - 32;
@@ -1364,7 +1390,7 @@ __global__ void __launch_bounds__(TPB, p1_min_ctas(NSEL)) k_pass1(const float* _
       if (c) atomicAdd(&gh[i], c);
     }
     if (last_cta_of_row(&tickets[row * NTICKET + 11], gridDim.x))
-      first_digit_scan(cs, row, fhist, cntpart, sel, rowflag, tickets, flags);
+      first_digit_scan(NSEL, s_K, row, fhist, cntpart, sel, rowflag, tickets, flags);
   }
 }
 
@@ -1706,7 +1732,11 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
                                                   int pick_here, long long d, int nblk_main,
                                                   const double* __restrict__ partial, const u32* __restrict__ maxkey,
                                                   RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
-                                                  const u32* __restrict__ diffflag, double tol) {
+                                                  const u32* __restrict__ diffflag, double tol,
+                                                  const CsetDev* __restrict__ cs_global) {
+  // cs_global: the same candidate set in global memory (written by the sampling kernel).  The row's last CTA hands
+  // the set to functions that index it with run-time values; doing that with the kernel parameter would make every
+  // thread of every CTA copy it to local memory first.
   pdl_begin();
   extern __shared__ __align__(16) u32 wbuf[];          // cs.nsel * FINISH_WORDS words, used by the row's last CTA
   const int row = blockIdx.y;
@@ -1770,10 +1800,10 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
     lepart[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
   }
   if (!last_cta_of_row(&tickets[row * NTICKET + 12], gridDim.x)) return;
-  collected_finish_row(cs, row, (int)gridDim.x, sel, fl, lepart, wbuf);
+  collected_finish_row(*cs_global, row, (int)gridDim.x, sel, fl, lepart, wbuf);
   __syncthreads();   // the brackets' results, written by one warp each, are read by the level choice
   if (pick_here) {
-    pick_row(cs, d, row, nblk_main, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+    pick_row(*cs_global, d, row, nblk_main, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);
     if (threadIdx.x == 0) tickets[row * NTICKET + 9] = 1u;
   }
 }
@@ -1786,7 +1816,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; }
 
 struct Layout {
-  size_t hist1, hist2, hist3, maxkey, limbs, flags, zero_end, zero_noshist, sel, dec, partial, energy, tiecnt, total;
+  size_t hist1, hist2, hist3, maxkey, limbs, flags, csdev, zero_end, zero_noshist, sel, dec, partial, energy, tiecnt, total;
   size_t tickets, rowflag, diffflag, shist, lhist1, fhist, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
@@ -1820,6 +1850,7 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   }
   L.zero_end = o;
   L.flags = o; o = align_up(o + 64, 256);   // status words 0-3, word 8: completion count of the short-row kernel
+  L.csdev = o; o = align_up(o + sizeof(CsetDev), 256);
   L.sel = o; o = align_up(o + (size_t)rows * sizeof(SelRow), 256);
   L.dec = o; o = align_up(o + (size_t)rows * sizeof(RowDec), 256);
   L.partial = o; o = align_up(o + (size_t)rows * MAX_BLK_PER_ROW * NSLOT * 8, 256);
@@ -1850,6 +1881,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->maxkey = (u32*)(b + L.maxkey);
   s->limbs = (u64*)(b + L.limbs);
   s->flags = (u32*)(b + L.flags);
+  s->csdev = (CsetDev*)(b + L.csdev);
   s->zero_begin = b;
   s->zero_bytes = L.zero_end;
   s->zero_bytes_noshist = L.zero_noshist;
@@ -2087,10 +2119,10 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     u32* samp_max = qinline ? s.maxkey : nullptr;
     prof_begin(pf, KID_SAMPLE, stream);
     if (row_sampler) {
-      if (al) launch_k(k_sample_row<true>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey);
-      else launch_k(k_sample_row<false>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey);
-    } else if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
-    else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max);
+      if (al) launch_k(k_sample_row<true>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev);
+      else launch_k(k_sample_row<false>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev);
+    } else if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max, s.csdev);
+    else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max, s.csdev);
     prof_end(pf, stream);
     ++launches;
     // 2. the one pass over X, G, Y
@@ -2115,7 +2147,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     TIMED(KID_LCOLLECT, launch_k(k_lcollect, lgrid, dim3(TPB), (size_t)cs.nsel * FINISH_WORDS * 4, stream, pdl, cs, nblk, s.sel, s.list, s.lcount,
                                  s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
                                  (cs.nquant == 0 || qinline) ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
-                                 s.diffflag, tol));
+                                 s.diffflag, tol, (const CsetDev*)s.csdev));
     // rows whose first-digit bin holds too many keys: three digit levels of 11, 11 and 9 bits (usually no row)
     LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
     LIST_PASS(2, cs.nsel * BINS2 * 4, s.hist2);

@@ -114,6 +114,7 @@ struct Scratch {
   u32* maxkey;     // [rows]
   u64* limbs;      // [rows][NSLOT][NLIMB] exact accumulators
   u32* flags;      // [4]: 0 nonfinite seen, 1 #exact rechecks
+  CsetDev* csdev;  // the call's candidate set, for code that indexes it with run-time values
   void* zero_begin; size_t zero_bytes;  // region cleared at the start of every call
   size_t zero_bytes_noshist;            // the same without the sample histogram (its last part)
   SelRow* sel;     // [rows]
