@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(TPB) k_quant_err(const float* __restrict__ X, 
 }
 
 // `picked` (may be null): per-row ticket words; a row whose word 9 is set was already decided.
-__global__ void __launch_bounds__(TPB) k_pick(CsetDev cs, long long d, int nblk_main, int nblk_full,
+__global__ void __launch_bounds__(TPB) k_pick(CsetDev cs_param, long long d, int nblk_main, int nblk_full,
                                              const u32* __restrict__ rowflag, const double* __restrict__ partial,
                                              const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
                                              RowDec* __restrict__ dec, u32* __restrict__ flags, CompressOut out,
@@ -265,6 +265,9 @@ __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs, long long d, int nblk_
   pdl_begin();
   const int row = blockIdx.x;
   if (picked && picked[row * NTICKET + 9]) return;
+  __shared__ CsetDev cs;   // indexed with run-time values below: a shared copy instead of a local one per thread
+  if (threadIdx.x == 0) cs_copy_static(cs, cs_param);
+  __syncthreads();
   const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
   pick_row(cs, d, row, nblk, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);  // k_quant_err: main grid
 }
@@ -516,8 +519,11 @@ __global__ void __launch_bounds__(TPB) k_update_narrow(const float* __restrict__
   if (want_mean && live) out.mean_out[c] = __fdiv_rn(acc, (float)rows);
 }
 
+#ifndef UPD_MINB
+#define UPD_MINB 4   // resident CTAs per SM the register budget of the update kernel is set for
+#endif
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB, 4) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
+__global__ void __launch_bounds__(TPB, UPD_MINB) k_update(const float* __restrict__ X, float* __restrict__ G, int rows,
                                                 long long d, const RowDec* __restrict__ dec,
                                                 const u32* __restrict__ tiepref, long long nchunk, int copy_mode,
                                                 CompressOut out, const u32* __restrict__ skip_flag) {

@@ -25,6 +25,19 @@ __device__ __forceinline__ int sm_count() {
   return (int)n;
 }
 
+// Copies a candidate set member by member with compile-time indices.  A kernel that indexes its by-value
+// CsetDev parameter with run-time values (or hands its address to a function) makes every thread copy the whole
+// structure to local memory; kernels that need such indexing let one thread copy the parameter to shared memory
+// with this function and work on that copy.
+__device__ __forceinline__ void cs_copy_static(CsetDev& dst, const CsetDev& src) {
+  dst.m = src.m; dst.zeta = src.zeta; dst.nsel = src.nsel; dst.nquant = src.nquant;
+#pragma unroll
+  for (int k = 0; k < MAXC; ++k) {
+    dst.kind[k] = src.kind[k]; dst.param[k] = src.param[k]; dst.sel[k] = src.sel[k]; dst.qsel[k] = src.qsel[k];
+    dst.pkind[k] = src.pkind[k]; dst.pparam[k] = src.pparam[k];
+  }
+}
+
 __device__ __forceinline__ u32 key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
 template <bool ALIGNED>

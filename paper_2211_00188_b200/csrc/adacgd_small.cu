@@ -44,12 +44,15 @@ __device__ __forceinline__ void warp_find_kth_desc(const u32* hist, int nb, u32 
 constexpr int SMALL_LIST = 4096;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
-                                                    int rows, long long d, CsetDev cs, SelRow* sel, RowDec* dec,
+                                                    int rows, long long d, CsetDev cs_param, SelRow* sel, RowDec* dec,
                                                     double* partial, u32* maxkey, u32* diffflag, u32* flags,
                                                     CompressOut out, double tol, u32* mean_ticket) {
   // mean_ticket != nullptr: the rows are so short that the CTA that finishes last also takes the mean over them
   // (summed in row order, one division), instead of a kernel of its own
   pdl_begin();
+  __shared__ CsetDev cs;   // the kernel indexes the set with run-time values: a shared copy instead of a local one per thread
+  if (threadIdx.x == 0) cs_copy_static(cs, cs_param);
+  __syncthreads();
   extern __shared__ __align__(16) unsigned char small_smem[];
   const int dn = (int)d;
   float* vs = reinterpret_cast<float*>(small_smem);                       // [d rounded up to 4]
