@@ -717,7 +717,7 @@ static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
     "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows",
-    "k_csr_fwd", "k_csc_bwd", "k_csr_residual", "k_delta_scan", "k_dense_inc", "k_inc_finish"};
+    "k_csr_fwd", "k_csc_bwd", "k_csr_residual", "k_delta_scan", "k_dense_inc", "k_inc_finish", "k_side"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }
 

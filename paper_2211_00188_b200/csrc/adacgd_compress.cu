@@ -15,6 +15,7 @@
 // worst-case summation error is redone in exact integer arithmetic.
 #include <mutex>
 
+#include <cooperative_groups.h>
 #include "adacgd_device.cuh"
 
 namespace adacgd {
@@ -59,17 +60,16 @@ __device__ void scan_row(const CsetDev& cs, int row, const u32* __restrict__ his
 // PASS 1: histogram of key[30:20] (one table per row) and the row maximum.
 // PASS 2: for every selecting candidate, histogram of key[19:9] over the keys in its pass-1 bin.
 // PASS 3: histogram of key[8:0] over the keys that share its 22-bit prefix.
+// Body of one CTA (bx of gx CTAs of row by) of the histogram passes: shared by the kernel of that name and by k_side.
 template <int PASS, bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const float* __restrict__ G,
-                                              long long d, CsetDev cs, SelRow* __restrict__ sel,
-                                              u32* __restrict__ hist, u32* __restrict__ maxkey,
-                                              const u32* __restrict__ rowflag, u32* __restrict__ tickets,
-                                              u32* __restrict__ flags) {
-  pdl_begin();
-  extern __shared__ u32 sh[];
-  const int row = blockIdx.y;
+__device__ __forceinline__ void d_hist(int bx, int by, int gx, u32* sh, const float* __restrict__ X, const float* __restrict__ G,
+                                              long long d, const CsetDev& cs, SelRow* sel,
+                                              u32* hist, u32* maxkey,
+                                              const u32* rowflag, u32* tickets,
+                                              u32* flags) {
+  const int row = by;
   const int nsel = cs.nsel;
-  if (rowflag && !rowflag[row]) return;  // single-pass mode: only rows whose bracket failed
+  if (rowflag && !__ldcg(&rowflag[row])) return;  // single-pass mode: only rows whose bracket failed
   constexpr int NB = (PASS == 3) ? BINS3 : BINS1;
   const int ntab = (PASS == 1) ? 1 : nsel;
   for (int i = threadIdx.x; i < ntab * NB; i += TPB) sh[i] = 0;
@@ -77,15 +77,15 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
 #pragma unroll
   for (int j = 0; j < MAXC; ++j) {
     pref[j] = 0xffffffffu;
-    if (PASS == 2 && j < nsel) pref[j] = sel[row].b1[j];
-    if (PASS == 3 && j < nsel) pref[j] = sel[row].p2[j];
+    if (PASS == 2 && j < nsel) pref[j] = __ldcg(&sel[row].b1[j]);
+    if (PASS == 3 && j < nsel) pref[j] = __ldcg(&sel[row].p2[j]);
   }
   __syncthreads();
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
   u32 mx = 0;
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+  for (long long t = bx; t < ntile; t += gx) {
     const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
     if (c0 >= d) continue;
     float x[4], g[4];
@@ -118,8 +118,19 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
     for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if ((threadIdx.x & 31) == 0 && mx) atomicMax(&maxkey[row], mx);
   }
-  if (nsel && last_cta_of_row(&tickets[row * NTICKET + 3 + PASS], gridDim.x))
+  if (nsel && last_cta_of_row(&tickets[row * NTICKET + 3 + PASS], gx))
     scan_row<PASS>(cs, row, hist, sel, rowflag != nullptr, flags);
+}
+
+template <int PASS, bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const float* __restrict__ G,
+                                              long long d, CsetDev cs, SelRow* __restrict__ sel,
+                                              u32* __restrict__ hist, u32* __restrict__ maxkey,
+                                              const u32* __restrict__ rowflag, u32* __restrict__ tickets,
+                                              u32* __restrict__ flags) {
+  pdl_begin();
+  extern __shared__ u32 sh[];
+  d_hist<PASS, ALIGNED>(blockIdx.x, blockIdx.y, gridDim.x, sh, X, G, d, cs, sel, hist, maxkey, rowflag, tickets, flags);
 }
 
 // --------------------------------------------------------------------------
@@ -128,16 +139,15 @@ __global__ void __launch_bounds__(TPB) k_hist(const float* __restrict__ X, const
 // slot 0: D = sum (x-y)^2; slot 1: sum v^2; slot 2+c (Top-K candidate c with a
 // threshold): sum of v^2 over keys strictly below its threshold.
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, const float* __restrict__ G,
-                                                const float* __restrict__ Y, long long d, CsetDev cs,
-                                                const SelRow* __restrict__ sel, double* __restrict__ partial,
-                                                const u32* __restrict__ rowflag, u32* __restrict__ diffflag) {
-  pdl_begin();
-  const int row = blockIdx.y;
-  if (rowflag && !rowflag[row]) return;
+__device__ __forceinline__ void d_energy(int bx, int by, int gx, const float* __restrict__ X, const float* __restrict__ G,
+                                                const float* __restrict__ Y, long long d, const CsetDev& cs,
+                                                const SelRow* sel, double* partial,
+                                                const u32* rowflag, u32* diffflag) {
+  const int row = by;
+  if (rowflag && !__ldcg(&rowflag[row])) return;
   u32 T[MAXC];
 #pragma unroll
-  for (int j = 0; j < MAXC; ++j) T[j] = (j < cs.nsel) ? sel[row].T[j] : 0u;
+  for (int j = 0; j < MAXC; ++j) T[j] = (j < cs.nsel) ? __ldcg(&sel[row].T[j]) : 0u;
   double aD = 0, aE = 0, aB[MAXC];
   u32 mxw = 0, dfl = 0;
 #pragma unroll
@@ -146,7 +156,7 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
   const float* gr = G + (long long)row * d;
   const float* yr = Y + (long long)row * d;
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+  for (long long t = bx; t < ntile; t += gx) {
     const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
     if (c0 >= d) continue;
     float x[4], g[4], y[4];
@@ -191,9 +201,18 @@ __global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, con
     if (used) {
       double acc = 0;
       for (int w = 0; w < TPB / 32; ++w) acc += red[s][w];
-      partial[((long long)row * MAX_BLK_PER_ROW + blockIdx.x) * NSLOT + s] = acc;
+      partial[((long long)row * MAX_BLK_PER_ROW + bx) * NSLOT + s] = acc;
     }
   }
+}
+
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_energy(const float* __restrict__ X, const float* __restrict__ G,
+                                                const float* __restrict__ Y, long long d, CsetDev cs,
+                                                const SelRow* __restrict__ sel, double* __restrict__ partial,
+                                                const u32* __restrict__ rowflag, u32* __restrict__ diffflag) {
+  pdl_begin();
+  d_energy<ALIGNED>(blockIdx.x, blockIdx.y, gridDim.x, X, G, Y, d, cs, sel, partial, rowflag, diffflag);
 }
 
 
@@ -256,6 +275,17 @@ __global__ void __launch_bounds__(TPB) k_quant_err(const float* __restrict__ X, 
 }
 
 // `picked` (may be null): per-row ticket words; a row whose word 9 is set was already decided.
+// (rows decided here are not marked: nothing reads the mark after the level choice)
+__device__ __forceinline__ void picked_mark(const u32*, int) {}
+__device__ __forceinline__ void d_pick(int row, const CsetDev& cs, long long d, int nblk_main, int nblk_full, const u32* rowflag,
+                                       const double* partial, const SelRow* sel, const u32* maxkey, RowDec* dec, u32* flags,
+                                       const CompressOut& out, const u32* diffflag, const u32* picked, double tol) {
+  if (picked && __ldcg(&picked[row * NTICKET + 9])) return;
+  const int nblk = (rowflag && __ldcg(&rowflag[row])) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
+  pick_row(cs, d, row, nblk, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);  // k_quant_err: main grid
+  if (picked && threadIdx.x == 0) picked_mark(picked, row);
+}
+
 __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs_param, long long d, int nblk_main, int nblk_full,
                                              const u32* __restrict__ rowflag, const double* __restrict__ partial,
                                              const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
@@ -263,34 +293,30 @@ __global__ void __launch_bounds__(TPB) k_pick(CsetDev cs_param, long long d, int
                                              const u32* __restrict__ diffflag, const u32* __restrict__ picked,
                                              double tol) {
   pdl_begin();
-  const int row = blockIdx.x;
-  if (picked && picked[row * NTICKET + 9]) return;
   __shared__ CsetDev cs;   // indexed with run-time values below: a shared copy instead of a local one per thread
   if (threadIdx.x == 0) cs_copy_static(cs, cs_param);
   __syncthreads();
-  const int nblk = (rowflag && rowflag[row]) ? nblk_full : nblk_main;  // which pass produced this row's partial sums
-  pick_row(cs, d, row, nblk, nblk_main, partial, sel, maxkey, dec, flags, out, diffflag, tol);  // k_quant_err: main grid
+  d_pick(blockIdx.x, cs, d, nblk_main, nblk_full, rowflag, partial, sel, maxkey, dec, flags, out, diffflag, picked, tol);
 }
 
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X, const float* __restrict__ G,
-                                                    const float* __restrict__ Y, long long d, CsetDev cs,
-                                                    const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
-                                                    RowDec* __restrict__ dec, u64* __restrict__ limbs,
-                                                    u32* __restrict__ diffflag, long long d_full, CompressOut out,
-                                                    u32* __restrict__ tickets, u32* __restrict__ flags) {
-  pdl_begin();
-  const int row = blockIdx.y;
-  if (!dec[row].need_exact) return;
+__device__ __forceinline__ void d_exact_sums(int bx, int by, int gx, const float* __restrict__ X, const float* __restrict__ G,
+                                                    const float* __restrict__ Y, long long d, const CsetDev& cs,
+                                                    const SelRow* sel, const u32* maxkey,
+                                                    RowDec* dec, u64* limbs,
+                                                    u32* diffflag, long long d_full, const CompressOut& out,
+                                                    u32* tickets, u32* flags) {
+  const int row = by;
+  if (!__ldcg(&dec[row].need_exact)) return;
   __shared__ u64 sh[NSLOT * NLIMB];
   for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) sh[i] = 0;
   __syncthreads();
-  const float s = __uint_as_float(maxkey[row]);
+  const float s = __uint_as_float(__ldcg(&maxkey[row]));
   const float* xr = X + (long long)row * d;
   const float* gr = G + (long long)row * d;
   const float* yr = Y + (long long)row * d;
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
-  for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+  for (long long t = bx; t < ntile; t += gx) {
     const long long c0 = t * (TPB * 4) + threadIdx.x * 4;
     if (c0 >= d) continue;
     float x[4], g[4], y[4];
@@ -311,7 +337,7 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
       limb_add(sh + 1 * NLIMB, kk, p);
       const u32 key = key_of(v);
       for (int j = 0; j < cs.nsel; ++j)
-        if (key < sel[row].T[j]) limb_add(sh + (2 + cs.sel[j]) * NLIMB, kk, p);
+        if (key < __ldcg(&sel[row].T[j])) limb_add(sh + (2 + cs.sel[j]) * NLIMB, kk, p);
       for (int j = 0; j < cs.nquant; ++j) {
         const int c = cs.qsel[j];
         const float L = (float)((1 << ((int)cs.param[c] - 1)) - 1);
@@ -331,23 +357,33 @@ __global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X,
     if (vlo) atomicAdd(&gl[i], vlo);
     if (vhi && (i % NLIMB) + 1 < NLIMB) atomicAdd(&gl[i + 1], vhi);
   }
-  if (last_cta_of_row(&tickets[row * NTICKET + 7], gridDim.x) && threadIdx.x == 0)
+  if (last_cta_of_row(&tickets[row * NTICKET + 7], gx) && threadIdx.x == 0)
     pick_exact_row(cs, row, d_full, limbs + (long long)row * NSLOT * NLIMB, sel, maxkey, dec, out, diffflag, flags);
+}
+
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_exact_sums(const float* __restrict__ X, const float* __restrict__ G,
+                                                    const float* __restrict__ Y, long long d, CsetDev cs,
+                                                    const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
+                                                    RowDec* __restrict__ dec, u64* __restrict__ limbs,
+                                                    u32* __restrict__ diffflag, long long d_full, CompressOut out,
+                                                    u32* __restrict__ tickets, u32* __restrict__ flags) {
+  pdl_begin();
+  d_exact_sums<ALIGNED>(blockIdx.x, blockIdx.y, gridDim.x, X, G, Y, d, cs, sel, maxkey, dec, limbs, diffflag, d_full, out, tickets, flags);
 }
 
 // --------------------------------------------------------------------------
 // tie order, estimator update, server mean
 // --------------------------------------------------------------------------
 template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, const float* __restrict__ G,
-                                                  long long d, const RowDec* __restrict__ dec,
-                                                  u32* __restrict__ tiecnt, long long nchunk,
-                                                  u32* __restrict__ tickets) {
-  pdl_begin();
-  const int row = blockIdx.y;
-  if (!dec[row].need_tie) return;
-  const u32 T = dec[row].T;
-  for (long long chunk = blockIdx.x; chunk < nchunk; chunk += gridDim.x) {
+__device__ __forceinline__ void d_tiecount(int bx, int by, int gx, const float* __restrict__ X, const float* __restrict__ G,
+                                                  long long d, const RowDec* dec,
+                                                  u32* tiecnt, long long nchunk,
+                                                  u32* tickets) {
+  const int row = by;
+  if (!__ldcg(&dec[row].need_tie)) return;
+  const u32 T = __ldcg(&dec[row].T);
+  for (long long chunk = bx; chunk < nchunk; chunk += gx) {
     const long long c0 = chunk * UPD_COLS + threadIdx.x * 4;
     u32 cnt = 0;
     if (c0 < d) {
@@ -362,7 +398,7 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
     block_excl_scan(cnt, &total);
     if (threadIdx.x == 0) tiecnt[(long long)row * nchunk + chunk] = total;
   }
-  if (!last_cta_of_row(&tickets[row * NTICKET + 8], gridDim.x)) return;
+  if (!last_cta_of_row(&tickets[row * NTICKET + 8], gx)) return;
   // exclusive prefix over the row's chunks
   u32* t = tiecnt + (long long)row * nchunk;
   u32 carry = 0;
@@ -374,6 +410,15 @@ __global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, c
     if (i < nchunk) t[i] = carry + ex;
     carry += total;
   }
+}
+
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_tiecount(const float* __restrict__ X, const float* __restrict__ G,
+                                                  long long d, const RowDec* __restrict__ dec,
+                                                  u32* __restrict__ tiecnt, long long nchunk,
+                                                  u32* __restrict__ tickets) {
+  pdl_begin();
+  d_tiecount<ALIGNED>(blockIdx.x, blockIdx.y, gridDim.x, X, G, d, dec, tiecnt, nchunk, tickets);
 }
 
 // Thread owns 4 consecutive columns and walks the rows in order, so that the mean is
@@ -1535,19 +1580,17 @@ __device__ __noinline__ void lscan_row(const CsetDev& cs, int row, int nblk, int
 
 // Pass over the listed keys for digit level LEVEL (1, 2 or 3).
 template <int LEVEL>
-__global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __restrict__ sel,
-                                               const u64* __restrict__ list, const u32* __restrict__ lcount,
-                                               long long list_row, u32 segcap, u32* __restrict__ hist,
-                                               double* __restrict__ lepart2, double* __restrict__ lepart3,
-                                               u32* __restrict__ rowflag, u64* __restrict__ fl,
-                                               u32* __restrict__ flcnt, const u32* __restrict__ cntpart,
-                                               u32* __restrict__ tickets) {
-  pdl_begin();
-  extern __shared__ u32 sh[];
-  const int row = blockIdx.y;
+__device__ __forceinline__ void d_lhist(int bx, int by, int gx, u32* sh, const CsetDev& cs, int nseg, SelRow* sel,
+                                               const u64* list, const u32* lcount,
+                                               long long list_row, u32 segcap, u32* hist,
+                                               double* lepart2, double* lepart3,
+                                               u32* rowflag, u64* fl,
+                                               u32* flcnt, const u32* cntpart,
+                                               u32* tickets) {
+  const int row = by;
   const int nsel = cs.nsel;
-  if (rowflag[row] || !tickets[row * NTICKET + 13]) return;  // only rows whose first-digit bin is too full
-  if (LEVEL == 3 && !tickets[row * NTICKET + 10]) return;  // no bracket of this row needs a third digit
+  if (__ldcg(&rowflag[row]) || !__ldcg(&tickets[row * NTICKET + 13])) return;  // only rows whose first-digit bin is too full
+  if (LEVEL == 3 && !__ldcg(&tickets[row * NTICKET + 10])) return;  // no bracket of this row needs a third digit
   constexpr int NB = (LEVEL == 3) ? BINS3 : BINS1;
   for (int i = threadIdx.x; i < nsel * NB; i += TPB) sh[i] = 0;
   u32 lo[MAXC], hi[MAXC], sh1[MAXC], sh2[MAXC], b1[MAXC], b2[MAXC];
@@ -1558,12 +1601,12 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
     hi[j] = (j < nsel) ? sel[row].hi[j] : 0u;
     sh1[j] = (j < nsel) ? sel[row].sh1[j] : 0u;
     sh2[j] = (j < nsel) ? sel[row].sh2[j] : 0u;
-    b1[j] = (j < nsel && LEVEL >= 2) ? sel[row].b1[j] : 0u;
-    b2[j] = (j < nsel && LEVEL == 3) ? sel[row].p2[j] : 0u;
+    b1[j] = (j < nsel && LEVEL >= 2) ? __ldcg(&sel[row].b1[j]) : 0u;
+    b2[j] = (j < nsel && LEVEL == 3) ? __ldcg(&sel[row].p2[j]) : 0u;
     en[j] = 0.0;
   }
   __syncthreads();
-  for (int sg = blockIdx.x; sg < nseg; sg += gridDim.x) {
+  for (int sg = bx; sg < nseg; sg += gx) {
     const u32 n = lcount[(long long)row * MAX_BLK_PER_ROW + sg];
     const u64* seg = list + (long long)row * list_row + (long long)sg * segcap;
     for (u32 i = threadIdx.x; i < n; i += TPB) {
@@ -1615,12 +1658,13 @@ __global__ void __launch_bounds__(TPB) k_lhist(CsetDev cs, int nseg, SelRow* __r
       double a = 0;
       for (int w = 0; w < TPB / 32; ++w) a += red[threadIdx.x][w];
       double* lp = (LEVEL == 2) ? lepart2 : lepart3;
-      lp[((long long)row * LIST_BLK + blockIdx.x) * MAXC + threadIdx.x] = a;
+      lp[((long long)row * LIST_BLK + bx) * MAXC + threadIdx.x] = a;
     }
   }
-  if (last_cta_of_row(&tickets[row * NTICKET + LEVEL], gridDim.x))
-    lscan_row<LEVEL>(cs, row, nseg, (int)gridDim.x, hist, cntpart, lepart2, lepart3, sel, rowflag, fl, flcnt);
+  if (last_cta_of_row(&tickets[row * NTICKET + LEVEL], gx))
+    lscan_row<LEVEL>(cs, row, nseg, gx, hist, cntpart, lepart2, lepart3, sel, rowflag, fl, flcnt);
 }
+
 
 // ---- the usual case: the threshold's first-digit bin holds at most FINAL_CAP keys ----------------
 // Completes the brackets of a row from the keys collected out of each threshold's bin.  One warp
@@ -1814,6 +1858,128 @@ __global__ void __launch_bounds__(TPB) k_lcollect(CsetDev cs, int nseg, SelRow* 
   }
 }
 
+
+// --------------------------------------------------------------------------
+// the rarely needed steps of the single-pass route, one launch
+// --------------------------------------------------------------------------
+// After the streaming pass and the collection pass most calls have nothing left to decide.  What may remain:
+//   L  rows whose threshold bin holds more keys than the collection buffer: three digit levels over the key lists;
+//   F  rows whose bracket missed (or whose list overflowed): the full three-pass select and the energies;
+//   P  rows without a level yet (the two above, or every row when quantiser errors come from a separate pass);
+//   E  rows whose fast sums could not certify a trigger decision: exact integer sums;
+//   T  rows with more threshold-equal keys than the ranking buffers hold: per-chunk tie counts.
+// One cooperative grid looks at the per-row flags and returns at once when none is set; otherwise it walks the
+// phases in order, its CTAs standing in for the grids of the separate kernels (bx of gx per row), with a grid-wide
+// barrier wherever a phase reads what the one before wrote.  Every CTA derives the same phase mask from the same
+// memory: a barrier follows each look at the flags before anything that may change them runs.
+struct SideArgs {
+  const float *X, *G, *Y;
+  long long d;
+  int rows, nseg, lh_gx, f_gx, t_gx, nblk_main;
+  const CsetDev* cs_global;
+  SelRow* sel;
+  const u64* list;
+  const u32* lcount;
+  long long list_row;
+  u32 segcap;
+  u32 *lhist1, *hist1, *hist2, *hist3;
+  double *lepart, *lepart3, *partial;
+  u32 *rowflag, *flcnt, *tickets, *maxkey, *flags, *diffflag, *tiecnt;
+  const u32* cntpart;
+  u64 *fl, *limbs;
+  RowDec* dec;
+  long long nchunk;
+  CompressOut out;
+  double tol;
+};
+
+constexpr u32 SIDE_L = 1u, SIDE_F = 2u, SIDE_P = 4u, SIDE_E = 8u, SIDE_T = 16u;
+
+__device__ __forceinline__ u32 side_mask(const SideArgs& a) {
+  u32 m = 0;
+  for (int r = threadIdx.x; r < a.rows; r += TPB) {
+    if (__ldcg(&a.rowflag[r])) m |= SIDE_F;
+    else if (__ldcg(&a.tickets[r * NTICKET + 13])) m |= SIDE_L;
+    if (!__ldcg(&a.tickets[r * NTICKET + 9])) m |= SIDE_P;
+    if (__ldcg(&a.dec[r].need_exact)) m |= SIDE_E;
+    if (__ldcg(&a.dec[r].need_tie)) m |= SIDE_T;
+  }
+  // bitwise OR over the CTA
+  __shared__ u32 all;
+  if (threadIdx.x == 0) all = 0;
+  __syncthreads();
+  m = __reduce_or_sync(0xffffffffu, m);
+  if ((threadIdx.x & 31) == 0 && m) atomicOr(&all, m);
+  __syncthreads();
+  m = all;
+  __syncthreads();   // `all` may be cleared by the next call only after everyone has read it
+  return m;
+}
+
+template <bool ALIGNED>
+__global__ void __launch_bounds__(TPB) k_side(SideArgs a) {
+  namespace cg = cooperative_groups;
+  u32 m = side_mask(a);
+  if (!m) return;                                   // the usual call
+  cg::grid_group grid = cg::this_grid();
+  extern __shared__ u32 sh[];
+  __shared__ CsetDev cs;
+  if (threadIdx.x == 0) cs = *a.cs_global;
+  __syncthreads();
+  grid.sync();
+  const int G = (int)gridDim.x, b0 = (int)blockIdx.x;
+#define SIDE_PHASE(gx, call)                                   \
+  for (int v = b0; v < (gx) * a.rows; v += G) {                \
+    const int bx = v % (gx), by = v / (gx);                    \
+    call;                                                      \
+    __syncthreads();                                           \
+  }
+  if (m & SIDE_L) {
+    SIDE_PHASE(a.lh_gx, d_lhist<1>(bx, by, a.lh_gx, sh, cs, a.nseg, a.sel, a.list, a.lcount, a.list_row, a.segcap, a.lhist1,
+                                   a.lepart, a.lepart3, a.rowflag, a.fl, a.flcnt, a.cntpart, a.tickets))
+    grid.sync();
+    SIDE_PHASE(a.lh_gx, d_lhist<2>(bx, by, a.lh_gx, sh, cs, a.nseg, a.sel, a.list, a.lcount, a.list_row, a.segcap, a.hist2,
+                                   a.lepart, a.lepart3, a.rowflag, a.fl, a.flcnt, a.cntpart, a.tickets))
+    grid.sync();
+    SIDE_PHASE(a.lh_gx, d_lhist<3>(bx, by, a.lh_gx, sh, cs, a.nseg, a.sel, a.list, a.lcount, a.list_row, a.segcap, a.hist3,
+                                   a.lepart, a.lepart3, a.rowflag, a.fl, a.flcnt, a.cntpart, a.tickets))
+    grid.sync();
+    m = side_mask(a);                               // the first level may have found a bracket that missed
+    grid.sync();
+  }
+  if (m & SIDE_F) {
+    SIDE_PHASE(a.f_gx, (d_hist<1, ALIGNED>(bx, by, a.f_gx, sh, a.X, a.G, a.d, cs, a.sel, a.hist1, a.maxkey, a.rowflag, a.tickets, a.flags)))
+    grid.sync();
+    SIDE_PHASE(a.f_gx, (d_hist<2, ALIGNED>(bx, by, a.f_gx, sh, a.X, a.G, a.d, cs, a.sel, a.hist2, a.maxkey, a.rowflag, a.tickets, a.flags)))
+    grid.sync();
+    SIDE_PHASE(a.f_gx, (d_hist<3, ALIGNED>(bx, by, a.f_gx, sh, a.X, a.G, a.d, cs, a.sel, a.hist3, a.maxkey, a.rowflag, a.tickets, a.flags)))
+    grid.sync();
+    SIDE_PHASE(a.f_gx, d_energy<ALIGNED>(bx, by, a.f_gx, a.X, a.G, a.Y, a.d, cs, a.sel, a.partial, a.rowflag, a.diffflag))
+    grid.sync();
+  }
+  if (m & SIDE_P) {
+    for (int row = b0; row < a.rows; row += G) {
+      d_pick(row, cs, a.d, a.nblk_main, a.f_gx, a.rowflag, a.partial, a.sel, a.maxkey, a.dec, a.flags, a.out, a.diffflag, a.tickets,
+             a.tol);
+      __syncthreads();
+    }
+    grid.sync();
+    m = side_mask(a);
+    grid.sync();
+  }
+  if (m & SIDE_E) {
+    SIDE_PHASE(a.f_gx, d_exact_sums<ALIGNED>(bx, by, a.f_gx, a.X, a.G, a.Y, a.d, cs, a.sel, a.maxkey, a.dec, a.limbs, a.diffflag, a.d,
+                                             a.out, a.tickets, a.flags))
+    grid.sync();
+    m = side_mask(a);                               // the exact decision may pick another level
+    grid.sync();
+  }
+  if (m & SIDE_T) {
+    SIDE_PHASE(a.t_gx, d_tiecount<ALIGNED>(bx, by, a.t_gx, a.X, a.G, a.d, a.dec, a.tiecnt, a.nchunk, a.tickets))
+  }
+#undef SIDE_PHASE
+}
+
 // --------------------------------------------------------------------------
 // host side
 // --------------------------------------------------------------------------
@@ -1971,11 +2137,22 @@ adacgd_status make_cset(const adacgd_cset* in, long long d, CsetDev* out, const 
 }
 
 // Tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory.
+constexpr int SIDE_SHM = MAXC * BINS2 * 4;   // the largest table any phase of k_side keeps in shared memory
+static_assert(BINS2 >= BINS1 && BINS2 >= BINS3, "k_side sizes its shared memory by BINS2");
+
+// Co-resident CTAs per SM of the cooperative kernel (the smaller of its two instantiations); 0 on failure.
+int side_ctas_per_sm() {
+  int a = 0, b = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, k_side<true>, TPB, SIDE_SHM) != cudaSuccess) return 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, k_side<false>, TPB, SIDE_SHM) != cudaSuccess) return 0;
+  return a < b ? a : b;
+}
+
 void set_compress_kernel_attributes() {
   cudaFuncSetAttribute(k_hist<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
   cudaFuncSetAttribute(k_hist<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
-  cudaFuncSetAttribute(k_lhist<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS1 * 4);
-  cudaFuncSetAttribute(k_lhist<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * BINS2 * 4);
+  cudaFuncSetAttribute(k_side<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIDE_SHM);
+  cudaFuncSetAttribute(k_side<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIDE_SHM);
   cudaFuncSetAttribute(k_lcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, MAXC * FINISH_WORDS * 4);
   cudaFuncSetAttribute(k_sample<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
   cudaFuncSetAttribute(k_sample<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SBINS * 2);
@@ -2000,6 +2177,8 @@ const DevProps* current_device() {
     if (cudaGetLastError() != cudaSuccess) return nullptr;
     table[dev].ordinal = dev;
     table[dev].sms = sms;
+    table[dev].side_ctas = side_ctas_per_sm();
+    if (table[dev].side_ctas < 1) return nullptr;
     known[dev] = true;
   }
   return &table[dev];
@@ -2099,10 +2278,6 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
       launch_k(k_pass1<N, false, 1>, sgrid, dim3(TPB), 0, stream, pdl, P1_ARGS);                                    \
     }                                                                                                               \
     break;
-#define LIST_PASS(LEVEL, shm, hist)                                                                              \
-  TIMED(KID_LHIST, launch_k(k_lhist<LEVEL>, lhgrid, dim3(TPB), shm, stream, pdl, cs, nblk, s.sel, s.list,         \
-                            s.lcount, s.list_row, segcap, hist, s.lepart, s.lepart3, s.rowflag, s.fl, s.flcnt,   \
-                            s.cntpart, s.tickets))
 
   if (single) {
     // 1. brackets for every Top-K threshold from a sample of the row (the last CTA of a row derives them)
@@ -2154,11 +2329,26 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                                  s.list_row, segcap, s.lepart, s.rowflag, s.fl, s.flcnt, s.tickets,
                                  (cs.nquant == 0 || qinline) ? 1 : 0, d, nblk, s.partial, s.maxkey, s.dec, s.flags, out,
                                  s.diffflag, tol, (const CsetDev*)s.csdev));
-    // rows whose first-digit bin holds too many keys: three digit levels of 11, 11 and 9 bits (usually no row)
-    LIST_PASS(1, cs.nsel * BINS1 * 4, s.lhist1);
-    LIST_PASS(2, cs.nsel * BINS2 * 4, s.hist2);
-    LIST_PASS(3, cs.nsel * BINS3 * 4, s.hist3);
-  }
+    if (cs.nquant && !qinline) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
+    // everything that is only sometimes needed, in one cooperative launch: rows whose first-digit bin holds too many
+    // keys (three digit levels of 11, 11 and 9 bits over the lists), rows whose bracket failed (the full select),
+    // levels not chosen yet, exact sums, tie counts
+    SideArgs sa;
+    sa.X = X; sa.G = G; sa.Y = Y; sa.d = d; sa.rows = rows; sa.nseg = nblk;
+    sa.lh_gx = (int)(lgx < 16 ? lgx : 16);          // the lists are about 1 % of a row: a few CTAs per row do
+    sa.f_gx = nblk_full;
+    long long tgx = (SMS * 4 + rows - 1) / rows;
+    if (tgx > nchunk) tgx = nchunk;
+    sa.t_gx = (int)tgx;
+    sa.nblk_main = nblk; sa.cs_global = (const CsetDev*)s.csdev; sa.sel = s.sel; sa.list = s.list; sa.lcount = s.lcount;
+    sa.list_row = s.list_row; sa.segcap = segcap; sa.lhist1 = s.lhist1; sa.hist1 = s.hist1; sa.hist2 = s.hist2; sa.hist3 = s.hist3;
+    sa.lepart = s.lepart; sa.lepart3 = s.lepart3; sa.partial = s.partial; sa.rowflag = s.rowflag; sa.flcnt = s.flcnt;
+    sa.tickets = s.tickets; sa.maxkey = s.maxkey; sa.flags = s.flags; sa.diffflag = s.diffflag; sa.tiecnt = s.tiecnt;
+    sa.cntpart = s.cntpart; sa.fl = s.fl; sa.limbs = s.limbs; sa.dec = s.dec; sa.nchunk = nchunk; sa.out = out; sa.tol = tol;
+    int per_sm = dp->side_ctas < 4 ? dp->side_ctas : 4;
+    TIMED(KID_SIDE, if (al) launch_cooperative(k_side<true>, dim3((unsigned)(per_sm * SMS)), dim3(TPB), SIDE_SHM, stream, sa);
+                    else launch_cooperative(k_side<false>, dim3((unsigned)(per_sm * SMS)), dim3(TPB), SIDE_SHM, stream, sa));
+  } else {
   // the full radix select: every row, or (single-pass mode) only rows whose bracket failed
   if (cs.nsel || cs.nquant) TIMED_HIST(KID_HIST1, 1, BINS1 * 4, s.hist1);
   if (cs.nsel) {
@@ -2166,14 +2356,15 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     TIMED_HIST(KID_HIST3, 3, cs.nsel * BINS3 * 4, s.hist3);
   }
   TIMED_AL(KID_ENERGY, k_energy, fgrid, 0, X, G, Y, d, cs, s.sel, s.partial, only, s.diffflag);
-  if (cs.nquant && !qinline) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
+  if (cs.nquant) TIMED_AL(KID_QUANT_ERR, k_quant_err, sgrid, 0, X, G, d, cs, s.maxkey, s.partial);
   TIMED(KID_PICK, launch_k(k_pick, dim3(rows), dim3(TPB), 0, stream, pdl, cs, d, nblk, nblk_full, only, s.partial, s.sel, s.maxkey,
-                           s.dec, s.flags, out, s.diffflag, single ? s.tickets : nullptr, tol));
+                           s.dec, s.flags, out, s.diffflag, (const u32*)nullptr, tol));
   TIMED_AL(KID_EXACT, k_exact_sums, fgrid, 0, X, G, Y, d, cs, s.sel, s.maxkey, s.dec, s.limbs, s.diffflag, d, out, s.tickets, s.flags);
   if (cs.nsel) {
     long long tgx = (SMS * 4 + rows - 1) / rows;
     if (tgx > nchunk) tgx = nchunk;
     TIMED_AL(KID_TIE, k_tiecount, dim3((unsigned)tgx, rows), 0, X, G, d, s.dec, s.tiecnt, nchunk, s.tickets);
+  }
   }
   {
     // Not a programmatic dependent: launched as one, this persistent grid ran 400 us instead of 270 us on
@@ -2190,7 +2381,6 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     }
     TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, skip);
   }
-#undef LIST_PASS
 #undef PASS1_CASE
 #undef P1_ARGS
 #undef TIMED_HIST

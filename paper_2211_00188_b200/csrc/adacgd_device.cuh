@@ -448,4 +448,18 @@ inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t shm, 
   cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// Launches a kernel whose CTAs synchronise across the grid: the launch fails unless all of them can be resident
+// at once, so the grid is sized from the occupancy the runtime reports.
+template <typename... KArgs, typename... Args>
+inline void launch_cooperative(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t shm, cudaStream_t stream,
+                               Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = shm; cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;
+  at[0].val.cooperative = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 }  // namespace adacgd

@@ -33,7 +33,7 @@ constexpr int FLUSH_TILES = 16;     // binary32 chains are folded into binary64 
 enum KernelId {
   KID_MEMSET = 0, KID_HIST1, KID_HIST2, KID_HIST3, KID_SCAN, KID_ENERGY, KID_QUANT_ERR, KID_PICK,
   KID_EXACT, KID_TIE, KID_UPDATE, KID_GRAD_FWD, KID_GRAD_BWD, KID_GRAD_REDUCE, KID_LOSS, KID_AXPY,
-  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD, KID_CSR_RES, KID_DELTA, KID_INC, KID_INC_FINISH,
+  KID_LOG, KID_SAMPLE, KID_BRACKET, KID_PASS1, KID_LHIST, KID_LCOLLECT, KID_SMALL, KID_CSR_FWD, KID_CSC_BWD, KID_CSR_RES, KID_DELTA, KID_INC, KID_INC_FINISH, KID_SIDE,
   KID_COUNT
 };
 struct Prof {
@@ -55,6 +55,7 @@ inline void prof_end(Prof* p, cudaStream_t s) {
 struct DevProps {
   int ordinal;
   int sms;       // streaming multiprocessors: grids are sized in multiples of it
+  int side_ctas; // CTAs of the cooperative side-path kernel that fit on one SM
 };
 const DevProps* current_device();
 void set_compress_kernel_attributes();   // adacgd_compress.cu
