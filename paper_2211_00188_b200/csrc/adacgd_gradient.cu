@@ -351,12 +351,15 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd(const long long* __restrict__ c
 constexpr int CSR_BLK_MAX = 49152;   // columns of x per block: 192 KB of shared memory
 constexpr int CSR_FWD_TPB = 1024;
 constexpr int CSR_NB_MAX = 8;        // wider problems take the plain warp-per-row kernel
-constexpr int CSR_FWD_UNR = 6;       // entries a lane requests at once
+constexpr int CSR_FWD_UNR = 3;       // groups of four entries a lane requests at once
 
-__global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long* __restrict__ split, const int* __restrict__ col,
+__global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long* __restrict__ qptr, const u16* __restrict__ col16,
                                                                  const float* __restrict__ val, const float* __restrict__ x,
                                                                  long long rows, long long d, int blk,
                                                                  float* __restrict__ zpart) {
+  // val / col16: the entries regrouped at init, block-major, every (block, row) span padded with zero entries to a
+  // multiple of four so that a lane reads four values (16 bytes) and four 16-bit block-relative columns (8 bytes) per
+  // request: 6 bytes per stored entry.  qptr[b * rows + row]: first group of four of the span.
   extern __shared__ __align__(16) float xs[];
   const int b = blockIdx.y;
   const long long cbase = (long long)b * blk;
@@ -364,39 +367,53 @@ __global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long
   for (int i = threadIdx.x; i < ncol; i += CSR_FWD_TPB) xs[i] = x[cbase + i];
   __syncthreads();
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const long long* s0 = split + (long long)b * rows;
-  const long long* s1 = split + (long long)(b + 1) * rows;
-  const int cb = (int)cbase;
+  const long long* q = qptr + (long long)b * rows;
+  const float4* vq = (const float4*)val;
+  const uint2* cq = (const uint2*)col16;
   const long long stride = (long long)gridDim.x * (CSR_FWD_TPB / 32);
   long long row = (long long)blockIdx.x * (CSR_FWD_TPB / 32) + wid;
-  // the span of the next row is requested while the current one is summed
-  long long e0 = 0, e1 = 0;
-  if (row < rows) { e0 = s0[row]; e1 = s1[row]; }
+  // Two rows ahead the span is known, one row ahead its first CSR_FWD_UNR groups per lane are already requested
+  // while the current row is summed: a warp always has a row's worth of entries in flight.
+  struct Batch { uint2 c[CSR_FWD_UNR]; float4 v[CSR_FWD_UNR]; };
+  auto request = [&](long long e0, long long e1, int o, Batch& t) {
+    const float4* vp = vq + e0 + lane;                    // offsets are 32-bit and relative to the lane's first group
+    const uint2* cp = cq + e0 + lane;
+    const int cnt = (int)(e1 - e0) - lane;                // this lane owns groups 32 k with 32 k < cnt
+#pragma unroll
+    for (int k = 0; k < CSR_FWD_UNR; ++k) {
+      const bool ok = o + 32 * k < cnt;
+      t.c[k] = ok ? __ldcs(cp + o + 32 * k) : make_uint2(0u, 0u);
+      t.v[k] = ok ? __ldcs(vp + o + 32 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto add = [&](const Batch& t, float acc) {             // a lane adds its products in ascending entry order;
+#pragma unroll
+    for (int k = 0; k < CSR_FWD_UNR; ++k) {               // absent and padding entries add 0 * xs[0]
+      acc = fmaf(t.v[k].x, xs[t.c[k].x & 0xffffu], acc);
+      acc = fmaf(t.v[k].y, xs[t.c[k].x >> 16], acc);
+      acc = fmaf(t.v[k].z, xs[t.c[k].y & 0xffffu], acc);
+      acc = fmaf(t.v[k].w, xs[t.c[k].y >> 16], acc);
+    }
+    return acc;
+  };
+  long long e0 = 0, e1 = 0, n0 = 0, n1 = 0;
+  Batch cur, nxt;
+  if (row < rows) { e0 = q[row]; e1 = q[row + 1]; request(e0, e1, 0, cur); }
+  if (row + stride < rows) { n0 = q[row + stride]; n1 = q[row + stride + 1]; }
   for (; row < rows; row += stride) {
-    const long long nrow = row + stride;
-    long long n0 = 0, n1 = 0;
-    if (nrow < rows) { n0 = s0[nrow]; n1 = s1[nrow]; }
-    float acc = 0.f;
-    // CSR_FWD_UNR entries per lane in flight; a lane adds its products in ascending entry order.  Offsets
-    // are 32-bit and relative to the lane's first entry, so that a load is one instruction and its guard.
-    const int* cp = col + e0 + lane;
-    const float* vp = val + e0 + lane;
-    const int cnt = (int)(e1 - e0) - lane;               // this lane owns entries 32 k with 32 k < cnt
-    for (int o = 0; o < cnt; o += 32 * CSR_FWD_UNR) {
-      int c[CSR_FWD_UNR];
-      float v[CSR_FWD_UNR];
-#pragma unroll
-      for (int k = 0; k < CSR_FWD_UNR; ++k) {
-        const bool ok = o + 32 * k < cnt;
-        c[k] = ok ? __ldcs(cp + o + 32 * k) : cb;
-        v[k] = ok ? __ldcs(vp + o + 32 * k) : 0.f;
-      }
-#pragma unroll
-      for (int k = 0; k < CSR_FWD_UNR; ++k) acc = fmaf(v[k], xs[c[k] - cb], acc);   // absent entries add 0 * xs[0]
+    const long long nnrow = row + 2 * stride;
+    long long m0 = 0, m1 = 0;
+    if (nnrow < rows) { m0 = q[nnrow]; m1 = q[nnrow + 1]; }
+    if (row + stride < rows) request(n0, n1, 0, nxt);
+    float acc = add(cur, 0.f);
+    for (int o = 32 * CSR_FWD_UNR; o < (int)(e1 - e0); o += 32 * CSR_FWD_UNR) {   // the rest of a long span
+      request(e0, e1, o, cur);
+      acc = add(cur, acc);
     }
     acc = warp_sum_f32(acc);
     if (lane == 0) zpart[(long long)b * rows + row] = acc;
-    e0 = n0; e1 = n1;
+    e0 = n0; e1 = n1; n0 = m0; n1 = m1;
+    cur = nxt;
   }
 }
 
@@ -439,10 +456,11 @@ constexpr int CSC_WPCAP = 768;     // products parked per warp
 constexpr int CSC_UNR = 6;         // entries a lane requests at once
 constexpr int CSC_RCAP = 8192;     // residuals of a worker kept in shared memory
 __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restrict__ wbase, const u32* __restrict__ ptr32,
-                                                      const int* __restrict__ crow, const float* __restrict__ cval,
+                                                      const u16* __restrict__ crow, const float* __restrict__ cval,
                                                       const float* __restrict__ r, const float* __restrict__ x,
                                                       long long d, long long m_rows, int loss, float lambda,
                                                       float* __restrict__ grads) {
+  // crow: 16-bit sample indices (a worker has at most CSC_RCAP samples here)
   extern __shared__ __align__(16) float bsm[];   // [m_rows] residuals, then [TPB / 32][CSC_WPCAP] products
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   float* rs = bsm;
@@ -480,21 +498,21 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
     const long long c0 = grp * CSC_WCOLS;
     const long long c1 = (c0 + CSC_WCOLS < d) ? c0 + CSC_WCOLS : d;
     const u32 e0 = cur.e0, span = cur.e1 - cur.e0;
-    const int* er = crow + base + e0;
+    const u16* er = crow + base + e0;
     const float* ev = cval + base + e0;
     float acc[2] = {0.f, 0.f};
     if (span <= (u32)CSC_WPCAP) {
-      const int* erl = er + lane;
+      const u16* erl = er + lane;
       const float* evl = ev + lane;
       float* pl = prod + lane;
       const int cnt = (int)span - lane;                  // this lane owns entries 32 k with 32 k < cnt
       for (int o = 0; o < cnt; o += 32 * CSC_UNR) {
-        int rr[CSC_UNR];
+        u16 rr[CSC_UNR];
         float vv[CSC_UNR];
 #pragma unroll
         for (int k = 0; k < CSC_UNR; ++k) {
           const bool ok = o + 32 * k < cnt;
-          rr[k] = ok ? __ldcs(erl + o + 32 * k) : 0;
+          rr[k] = ok ? __ldcs(erl + o + 32 * k) : (u16)0;
           vv[k] = ok ? __ldcs(evl + o + 32 * k) : 0.f;
         }
 #pragma unroll
@@ -768,6 +786,10 @@ static int csr_block_cols(const adacgd_problem& p, int nb) {
   const long long blk = (p.d + nb - 1) / nb;
   return (int)((blk + 3) / 4 * 4);
 }
+// Entries of the regrouped forward copy: every (block, row) span padded to a multiple of four.
+static size_t csr_fwd_cap(const adacgd_problem& p, int nb) {
+  return (size_t)p.csr_nnz + 3 * (size_t)nb * (size_t)p.n * (size_t)p.m_rows + 4;
+}
 // Whether the backward pass walks spans (1) or takes one thread per column (0).
 static int csc_cols_per_cta(const adacgd_problem& p) {
   if (p.m_rows > CSC_RCAP) return 0;
@@ -809,11 +831,14 @@ size_t grad_scratch_bytes(const adacgd_problem& p, int flags) {
     const int nb = csr_blocks_of(p);
     const size_t rows = (size_t)p.n * p.m_rows;
     if (nb) {
-      o = align_up(o + (size_t)(nb + 1) * rows * 8, 256);
+      o = align_up(o + ((size_t)nb * rows + 1) * 8, 256);
       o = align_up(o + (size_t)nb * rows * 4, 256);
+      o = align_up(o + csr_fwd_cap(p, nb) * 4, 256);   // regrouped values
+      o = align_up(o + csr_fwd_cap(p, nb) * 2, 256);   // regrouped 16-bit columns
     }
     o = align_up(o + ((size_t)p.n + 1) * 8, 256);
     o = align_up(o + (size_t)p.n * ((size_t)p.d + 1) * 4, 256);
+    o = align_up(o + (size_t)p.csr_nnz * 2, 256);   // 16-bit sample indices of the transposed copy
   }
   return o;
 }
@@ -852,6 +877,7 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int
   o = align_up(o + g->ticket_bytes, 256);
   g->csc_ptr = nullptr; g->csc_row = nullptr; g->csc_val = nullptr;
   g->nb = 0; g->blk = 0; g->csr_split = nullptr; g->zpart = nullptr; g->ccols = 0; g->wbase = nullptr; g->ptr32 = nullptr;
+  g->csc_row16 = nullptr; g->csr_col16 = nullptr; g->fwd_val = nullptr;
   if (p.layout == ADACGD_LAYOUT_CSR) {
     g->csc_ptr = (long long*)(b + o); o = align_up(o + ((size_t)p.n * p.d + 1) * 8, 256);
     g->csc_row = (int*)(b + o); o = align_up(o + (size_t)p.csr_nnz * 4, 256);
@@ -860,12 +886,15 @@ void carve_grad_scratch(GradScratch* g, void* base, const adacgd_problem& p, int
     g->blk = csr_block_cols(p, g->nb);
     const size_t rows = (size_t)p.n * p.m_rows;
     if (g->nb) {
-      g->csr_split = (long long*)(b + o); o = align_up(o + (size_t)(g->nb + 1) * rows * 8, 256);
+      g->csr_split = (long long*)(b + o); o = align_up(o + ((size_t)g->nb * rows + 1) * 8, 256);
       g->zpart = (float*)(b + o); o = align_up(o + (size_t)g->nb * rows * 4, 256);
+      g->fwd_val = (float*)(b + o); o = align_up(o + csr_fwd_cap(p, g->nb) * 4, 256);
+      g->csr_col16 = (u16*)(b + o); o = align_up(o + csr_fwd_cap(p, g->nb) * 2, 256);
     }
     g->ccols = csc_cols_per_cta(p);
     g->wbase = (long long*)(b + o); o = align_up(o + ((size_t)p.n + 1) * 8, 256);
-    g->ptr32 = (u32*)(b + o);
+    g->ptr32 = (u32*)(b + o); o = align_up(o + (size_t)p.n * ((size_t)p.d + 1) * 4, 256);
+    g->csc_row16 = (u16*)(b + o);
   }
   g->prof = nullptr;
 }
@@ -884,7 +913,7 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
       if (gx > (rows + 31) / 32) gx = (rows + 31) / 32;
       prof_begin(g.prof, KID_CSR_FWD, stream);
       k_csr_fwd_blocked<<<dim3((unsigned)gx, g.nb), CSR_FWD_TPB, (size_t)g.blk * 4, stream>>>(
-          g.csr_split, p.csr_col, p.csr_val, x, rows, p.d, g.blk, g.zpart);
+          g.csr_split, g.csr_col16, g.fwd_val, x, rows, p.d, g.blk, g.zpart);
       prof_end(g.prof, stream);
       ++launches;
       loss_blocks = (int)((p.m_rows + TPB - 1) / TPB);
@@ -908,7 +937,7 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
       if (gx > (ngroups + TPB / 32 - 1) / (TPB / 32)) gx = (ngroups + TPB / 32 - 1) / (TPB / 32);
       if (gx < 1) gx = 1;
       k_csc_bwd_span<<<dim3((unsigned)gx, p.n), TPB, ((size_t)p.m_rows + (size_t)(TPB / 32) * CSC_WPCAP) * 4, stream>>>(
-          g.wbase, g.ptr32, g.csc_row, g.csc_val, g.r, x, p.d, p.m_rows, p.loss, p.lambda, grads);
+          g.wbase, g.ptr32, g.csc_row16, g.csc_val, g.r, x, p.d, p.m_rows, p.loss, p.lambda, grads);
     }
     else
       k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
@@ -1018,6 +1047,7 @@ const char* build_csc(const adacgd_problem& p, GradScratch* gp, cudaStream_t str
   std::vector<long long> rowptr((size_t)rows + 1), cptr((size_t)cols + 1, 0);
   std::vector<int> col((size_t)nnz), crow((size_t)nnz);
   std::vector<float> val((size_t)nnz), cval((size_t)nnz);
+  std::vector<u16> crow16, col16;
   if (cudaMemcpyAsync(rowptr.data(), p.csr_rowptr, (rows + 1) * 8, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       cudaMemcpyAsync(col.data(), p.csr_col, nnz * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
       cudaMemcpyAsync(val.data(), p.csr_val, nnz * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
@@ -1068,12 +1098,42 @@ const char* build_csc(const adacgd_problem& p, GradScratch* gp, cudaStream_t str
       }
     }
   }
+  // narrow copies of the indices for the two span kernels: what they read per stored entry drops from 8 to 6 bytes
+  if (g.ccols) {
+    crow16.resize((size_t)nnz);
+    for (long long e = 0; e < nnz; ++e) crow16[(size_t)e] = (u16)crow[(size_t)e];          // m_rows <= CSC_RCAP
+  }
+  std::vector<float> fval;
+  std::vector<long long> qptr;
+  if (g.nb) {
+    // the forward copy: block-major, spans padded with (0, column 0) to a multiple of four entries
+    const size_t cap = csr_fwd_cap(p, g.nb);
+    fval.assign(cap, 0.f);
+    col16.assign(cap, (u16)0);
+    qptr.resize((size_t)g.nb * (size_t)rows + 1);
+    long long at = 0;   // in entries, always a multiple of four
+    for (int b = 0; b < g.nb; ++b) {
+      for (long long r = 0; r < rows; ++r) {
+        qptr[(size_t)b * (size_t)rows + (size_t)r] = at / 4;
+        const long long e0 = split[(size_t)b * (size_t)rows + (size_t)r], e1 = split[(size_t)(b + 1) * (size_t)rows + (size_t)r];
+        for (long long e = e0; e < e1; ++e) {
+          fval[(size_t)(at + e - e0)] = val[(size_t)e];
+          col16[(size_t)(at + e - e0)] = (u16)(col[(size_t)e] - (long long)b * g.blk);     // blk <= CSR_BLK_MAX
+        }
+        at += (e1 - e0 + 3) / 4 * 4;
+      }
+    }
+    qptr[(size_t)g.nb * (size_t)rows] = at / 4;
+  }
   if (cudaMemcpyAsync(g.csc_ptr, cptr.data(), (cols + 1) * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.csc_row, crow.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.csc_val, cval.data(), nnz * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.wbase, wbase.data(), wbase.size() * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(g.ptr32, ptr32.data(), ptr32.size() * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      (g.nb && cudaMemcpyAsync(g.csr_split, split.data(), split.size() * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
+      (g.nb && cudaMemcpyAsync(g.csr_split, qptr.data(), qptr.size() * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
+      (g.nb && cudaMemcpyAsync(g.csr_col16, col16.data(), col16.size() * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
+      (g.nb && cudaMemcpyAsync(g.fwd_val, fval.data(), fval.size() * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
+      (g.ccols && cudaMemcpyAsync(g.csc_row16, crow16.data(), (size_t)nnz * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess) ||
       cudaStreamSynchronize(stream) != cudaSuccess)
     return "copying the transposed arrays to the device failed";
   if (g.nb) cudaFuncSetAttribute(k_csr_fwd_blocked, cudaFuncAttributeMaxDynamicSharedMemorySize, CSR_BLK_MAX * 4);

@@ -8,6 +8,7 @@
 
 namespace adacgd {
 
+typedef uint16_t u16;
 typedef uint32_t u32;
 typedef unsigned long long u64;
 
@@ -177,11 +178,15 @@ struct GradScratch {
   // is "row" i*d + c)
   long long* csc_ptr;   // [n*d + 1]
   int* csc_row;         // [nnz] sample row inside the worker
+  u16* csc_row16;       // the same in 16 bits (span kernel: at most 8192 samples per worker)
+  u16* csr_col16;       // blocked forward kernel: column index inside its column block, regrouped like fwd_val
+  float* fwd_val;       // values regrouped block-major, every (block, row) span padded to a multiple of four
   float* csc_val;       // [nnz]
-  // column-blocked forward: the entries of sample row g whose column lies in block b are
-  // [csr_split[b*rows + g], csr_split[(b+1)*rows + g]); zpart[b*rows + g] is that block's share of a_g . x
+  // column-blocked forward: the entries of sample row g whose column lies in block b are the groups of four
+  // [csr_split[b*rows + g], csr_split[b*rows + g + 1]) of fwd_val / csr_col16; zpart[b*rows + g] is that block's
+  // share of a_g . x
   int nb, blk;          // column blocks and columns per block (nb = 0: plain warp-per-row kernel)
-  long long* csr_split; // [(nb+1)][n*m_rows]
+  long long* csr_split; // [nb * n*m_rows + 1]
   float* zpart;         // [nb][n*m_rows]
   // span backward: column pointers relative to the worker's first entry
   int ccols;            // 1: contiguous spans per warp; 0: one thread per column on csc_ptr
