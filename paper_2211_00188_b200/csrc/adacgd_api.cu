@@ -23,6 +23,7 @@ struct Counters {  // device resident, cumulative
   unsigned long long bits_up, bits_down;
   unsigned int rechecks_seen;
   unsigned int log_pos;  // next free record of the step log; the host rewinds it before each batch
+  unsigned int pending;  // 1: the iteration that ran last has no record yet (written by the next x update or by k_log_step)
 };
 
 thread_local std::string g_err = "";
@@ -87,10 +88,11 @@ adacgd_status check_problem(const adacgd_problem* p, const char** msg) {
   return ADACGD_OK;
 }
 
-__global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned long long* __restrict__ bits,
-                           const int* __restrict__ mlevel, const unsigned long long* __restrict__ mbits,
-                           const double* __restrict__ loss, const unsigned int* __restrict__ flags,
-                           Counters* cnt, StepLog* log, int* loglevels) {
+// The record of the iteration that just ran: bits sent, levels, loss, exact rechecks.  Run by one CTA.
+__device__ void log_body(int n, const int* __restrict__ levels, const unsigned long long* __restrict__ bits,
+                         const int* __restrict__ mlevel, const unsigned long long* __restrict__ mbits,
+                         const double* __restrict__ loss, const unsigned int* __restrict__ flags,
+                         Counters* cnt, StepLog* log, int* loglevels) {
   __shared__ unsigned long long sh[32];
   const int slot = (int)cnt->log_pos;
   unsigned long long a = 0;
@@ -117,6 +119,34 @@ __global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned
     cnt->bits_down += r.bits_down;
     log[slot] = r;
   }
+}
+
+// Closes a batch of iterations: writes the record of the last one, if it has none yet.
+__global__ void k_log_step(int n, const int* __restrict__ levels, const unsigned long long* __restrict__ bits,
+                           const int* __restrict__ mlevel, const unsigned long long* __restrict__ mbits,
+                           const double* __restrict__ loss, const unsigned int* __restrict__ flags,
+                           Counters* cnt, StepLog* log, int* loglevels) {
+  if (!cnt->pending) return;
+  log_body(n, levels, bits, mlevel, mbits, loss, flags, cnt, log, loglevels);
+  __syncthreads();
+  if (threadIdx.x == 0) cnt->pending = 0u;
+}
+
+// Opens an iteration: x^{t+1} = x^t - gamma g^t (Algorithm 1).  Its first CTA also writes the record of the iteration
+// before, whose results (levels, bits, loss) stay in place until later kernels of this iteration overwrite them:
+// one launch per iteration less than a record kernel at the end of every iteration.
+__global__ void __launch_bounds__(256) k_axpy_log(float* __restrict__ x, const float* __restrict__ g, float gamma, long long d,
+                                                  int n, const int* __restrict__ levels,
+                                                  const unsigned long long* __restrict__ bits, const int* __restrict__ mlevel,
+                                                  const unsigned long long* __restrict__ mbits, const double* __restrict__ loss,
+                                                  const unsigned int* __restrict__ flags, Counters* cnt, StepLog* log,
+                                                  int* loglevels) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));   // two binary32 roundings: the product, then the difference
+  if (blockIdx.x != 0) return;
+  if (cnt->pending) log_body(n, levels, bits, mlevel, mbits, loss, flags, cnt, log, loglevels);
+  __syncthreads();
+  if (threadIdx.x == 0) cnt->pending = 1u;
 }
 
 __global__ void k_set_master_identity(int* mlevel, unsigned long long* mbits, long long d) {
@@ -476,9 +506,13 @@ static adacgd_status enqueue_iteration(adacgd_ctx* c, bool capturing = false) {
   const int n = c->p.n;
   const long long d = c->p.d;
   // a0: x^{t+1} = x^t - gamma g^t
-  int r = launch_axpy(c->x, c->gm, c->gamma, d, c->stream, c->prof);
-  if (r < 0) return cuda_fail(c, "x update");
-  c->launches += r;
+  prof_begin(c->prof, KID_AXPY, c->stream);
+  k_axpy_log<<<(unsigned)((d + 255) / 256), 256, 0, c->stream>>>(c->x, c->gm, c->gamma, d, n, c->levels, c->bits, c->mlevel, c->mbits,
+                                                                  c->gs.loss, c->scr.flags, c->counters, c->log, c->loglevels);
+  prof_end(c->prof, c->stream);
+  if (cudaGetLastError() != cudaSuccess) return cuda_fail(c, "x update");
+  c->launches += 1;
+  int r = 0;
   // a1: X_i = grad f_i(x^{t+1})
   if (c->gs.inc) {
     const bool refresh = !capturing && (c->inc_dirty || c->since_refresh + 1 >= c->refresh_period);
@@ -507,12 +541,16 @@ static adacgd_status enqueue_iteration(adacgd_ctx* c, bool capturing = false) {
   float* t2 = c->grad_cur;
   c->grad_cur = c->grad_nxt;
   c->grad_nxt = t2;
+  return ADACGD_OK;   // the iteration's record is written by the next x update, or by close_batch()
+}
+
+// The record of the last iteration enqueued, before the host reads the step log or other calls touch its inputs.
+static void close_batch(adacgd_ctx* c) {
   prof_begin(c->prof, KID_LOG, c->stream);
-  k_log_step<<<1, 256, 0, c->stream>>>(n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
+  k_log_step<<<1, 256, 0, c->stream>>>(c->p.n, c->levels, c->bits, c->mlevel, c->mbits, c->gs.loss, c->scr.flags,
                                        c->counters, c->log, c->loglevels);
   prof_end(c->prof, c->stream);
   c->launches += 1;
-  return ADACGD_OK;
 }
 
 // Captures two iterations into one graph: after two steps every ping-pong pointer is back where it
@@ -592,6 +630,7 @@ adacgd_status adacgd_step(adacgd_ctx* c, int32_t n_steps, adacgd_step_report* re
         ++t;
       }
     }
+    if (batch > 0) close_batch(c);
     if (report_host || levels_host) {
       hostlog.resize(batch);
       CK(c, cudaMemcpyAsync(hostlog.data(), c->log, sizeof(StepLog) * batch, cudaMemcpyDeviceToHost, c->stream), "adacgd_step (copy of the step log to the host)");
@@ -716,7 +755,7 @@ void adacgd_destroy(adacgd_ctx* ctx) {
 static const char* const kKernelNames[KID_COUNT] = {
     "memset", "k_hist<1>", "k_hist<2>", "k_hist<3>", "k_scan", "k_energy", "k_quant_err", "k_pick",
     "k_exact_sums+k_pick_exact", "k_tiecount+k_tiescan", "k_update", "k_dense_fwd", "k_dense_bwd",
-    "k_grad_reduce", "k_loss_reduce", "k_axpy", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows",
+    "k_grad_reduce", "k_loss_reduce", "k_axpy_log", "k_log_step", "k_sample", "k_bracket", "k_pass1", "k_lhist", "k_lcollect", "k_small_rows",
     "k_csr_fwd", "k_csc_bwd", "k_csr_residual", "k_delta_scan", "k_dense_inc", "k_inc_finish", "k_side"};
 
 int32_t adacgd_profile_kernel_count(void) { return KID_COUNT; }

@@ -2392,18 +2392,6 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
 // --------------------------------------------------------------------------
 // small vector kernels of the loop
 // --------------------------------------------------------------------------
-__global__ void k_axpy(float* __restrict__ x, const float* __restrict__ g, float gamma, long long d) {
-  pdl_begin();
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));
-}
-int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof) {
-  prof_begin(prof, KID_AXPY, stream);
-  k_axpy<<<(unsigned)((d + 255) / 256), 256, 0, stream>>>(x, g, gamma, d);
-  prof_end(prof, stream);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
-}
-
 __global__ void k_mean_rows(const float* __restrict__ G, int rows, long long d, float* __restrict__ out) {
   pdl_begin();
   const long long c = (long long)blockIdx.x * blockDim.x + threadIdx.x;

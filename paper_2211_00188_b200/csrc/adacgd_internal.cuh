@@ -220,8 +220,6 @@ int launch_gradient_incremental(const adacgd_problem& p, const GradScratch& g, c
 int build_transposed_features(const adacgd_problem& p, const GradScratch& g, cudaStream_t stream);
 const char* build_csc(const adacgd_problem& p, GradScratch* g, cudaStream_t stream);
 
-// x <- x - gamma * g  (two binary32 roundings: the product, then the difference)
-int launch_axpy(float* x, const float* g, float gamma, long long d, cudaStream_t stream, Prof* prof);
 int launch_mean_rows(const float* G, int rows, long long d, float* out, cudaStream_t stream);
 
 // Stores the message that adacgd_last_error(NULL) returns on this thread.
