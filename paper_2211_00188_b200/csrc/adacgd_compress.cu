@@ -6,7 +6,8 @@
 // Three routes to the same results, chosen by size in launch_compress():
 //   - large problems: thresholds are bracketed from a sample (k_sample), one streaming pass over
 //     X, G, Y (k_pass1) gathers the sums and lists the few keys inside a bracket, the exact
-//     selection runs on those lists (k_lcollect, k_lhist), k_update applies the chosen level;
+//     selection runs on those lists (k_lcollect), one cooperative launch holds what only some rows need
+//     (k_side), k_update applies the chosen level;
 //   - the three-pass radix select on the bit pattern of |v| (11 + 11 + 9 bits: k_hist, k_energy),
 //     shared by all Top-K candidates of a row: mid-size problems, and the per-row fallback of
 //     the first route;
