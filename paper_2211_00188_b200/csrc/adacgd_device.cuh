@@ -73,9 +73,10 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
   return v;
 }
 
-// Exclusive prefix sum of one u32 per thread over the CTA (TPB threads); also returns the total.
+// Exclusive prefix sum of one u32 per thread over the CTA (NT threads); also returns the total.
+template <int NT = TPB>
 __device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
-  __shared__ u32 wsum[TPB / 32];
+  __shared__ u32 wsum[NT / 32];
   __shared__ u32 wtot;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   u32 inc = v;
@@ -88,15 +89,15 @@ __device__ __forceinline__ u32 block_excl_scan(u32 v, u32* total) {
   if (lane == 31) wsum[wid] = inc;
   __syncthreads();
   if (wid == 0) {
-    u32 w = (lane < TPB / 32) ? wsum[lane] : 0;
+    u32 w = (lane < NT / 32) ? wsum[lane] : 0;
     u32 winc = w;
 #pragma unroll
-    for (int o = 1; o < TPB / 32; o <<= 1) {
+    for (int o = 1; o < NT / 32; o <<= 1) {
       u32 t = __shfl_up_sync(0xffffffffu, winc, o);
       if (lane >= o) winc += t;
     }
-    if (lane < TPB / 32) wsum[lane] = winc - w;
-    if (lane == TPB / 32 - 1) wtot = winc;
+    if (lane < NT / 32) wsum[lane] = winc - w;
+    if (lane == NT / 32 - 1) wtot = winc;
   }
   __syncthreads();
   if (total) *total = wtot;
@@ -203,15 +204,16 @@ inline __device__ void finalize_row(const CsetDev& cs, int row, int level, long 
     for (int j = 0; j <= cs.m; ++j) out.err[(long long)row * (cs.m + 1) + j] = e[j];
 }
 
-// Chooses the level of one row from its sums (Eq. 10 and 11); run by a whole CTA of TPB threads.
+// Chooses the level of one row from its sums (Eq. 10 and 11); run by a whole CTA of NT threads.
 // The per-CTA partial sums of the streaming pass are added in a fixed order: thread t takes
-// blocks t, t + TPB, ..., then lanes, then warps.  D, ||v||^2 and the Top-K slots hold nblk partial
+// blocks t, t + NT, ..., then lanes, then warps.  D, ||v||^2 and the Top-K slots hold nblk partial
 // sums per row, the quantiser slots nblk_q (their pass may run on another grid).
+template <int NT = TPB>
 inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nblk, int nblk_q, const double* __restrict__ partial,
                          const SelRow* __restrict__ sel, const u32* __restrict__ maxkey,
                          RowDec* __restrict__ dec, u32* __restrict__ flags, const CompressOut& out,
                          const u32* __restrict__ diffflag, double tol) {
-  __shared__ double ps[NSLOT][TPB / 32];
+  __shared__ double ps[NSLOT][NT / 32];
   __shared__ double p_extra[MAXC];
   __shared__ u32 p_T[MAXC], p_ntie[MAXC], p_q[MAXC], p_max, p_diff;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -230,7 +232,7 @@ inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nbl
   u32 qmask = 0;   // slots written by the quantiser pass
   for (int j = 0; j < cs.nquant; ++j) qmask |= 1u << (2 + cs.qsel[j]);
   const int nblk_max = nblk > nblk_q ? nblk : nblk_q;
-  for (int b = threadIdx.x; b < nblk_max; b += TPB) {
+  for (int b = threadIdx.x; b < nblk_max; b += NT) {
 #pragma unroll
     for (int s = 0; s < NSLOT; ++s)
       if (s < nslot && b < (((qmask >> s) & 1u) ? nblk_q : nblk)) a[s] += __ldcg(&p[(long long)b * NSLOT + s]);
@@ -246,7 +248,7 @@ inline __device__ void pick_row(const CsetDev& cs, long long d, int row, int nbl
 #pragma unroll
   for (int s = 0; s < NSLOT; ++s) {
     double t = 0.0;
-    for (int w = 0; w < TPB / 32; ++w) t += ps[s][w];
+    for (int w = 0; w < NT / 32; ++w) t += ps[s][w];
     sum[s] = t;
   }
   const double D = sum[0];

@@ -42,8 +42,18 @@ __device__ __forceinline__ void warp_find_kth_desc(const u32* hist, int nb, u32 
 }
 
 constexpr int SMALL_LIST = 4096;
-template <bool ALIGNED>
-__global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
+#ifndef SMALL_NT_LONG_N
+#define SMALL_NT_LONG_N 512
+#endif
+#ifndef SMALL_LONG_ROW_N
+#define SMALL_LONG_ROW_N 512
+#endif
+constexpr int SMALL_NT_LONG = SMALL_NT_LONG_N;   // threads per CTA for rows of at least SMALL_LONG_ROW elements
+constexpr int SMALL_LONG_ROW = SMALL_LONG_ROW_N;
+// NT threads per CTA: 256, or 512 for rows of at least SMALL_LONG_ROW elements (c2, 20 rows of 8000: 113 -> 94 us for the
+// two calls of an iteration; 1024 threads leave 64 registers per thread and measured 98 us).
+template <bool ALIGNED, int NT>
+__global__ void __launch_bounds__(NT) k_small_rows(const float* __restrict__ X, float* G, const float* __restrict__ Y,
                                                     int rows, long long d, CsetDev cs_param, SelRow* sel, RowDec* dec,
                                                     double* partial, u32* maxkey, u32* diffflag, u32* flags,
                                                     CompressOut out, double tol, u32* mean_ticket) {
@@ -58,8 +68,8 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   float* vs = reinterpret_cast<float*>(small_smem);                       // [d rounded up to 4]
   u32* tab = reinterpret_cast<u32*>(small_smem) + ((dn + 3) / 4) * 4;     // max(BINS1, nsel * BINS2) words
   u32* cl = tab + (cs.nsel > 1 ? cs.nsel : 1) * BINS2;                           // SMALL_LIST keys sharing a first digit with a threshold
-  __shared__ double redd[NSLOT][TPB / 32];
-  __shared__ u32 redu[3][TPB / 32];
+  __shared__ double redd[NSLOT][NT / 32];
+  __shared__ u32 redu[3][NT / 32];
   __shared__ u32 s_b1[MAXC], s_ab1[MAXC], s_p2[MAXC], s_ab2[MAXC], s_T[MAXC], s_above[MAXC], s_ntie[MAXC], s_q[MAXC], s_cut[MAXC];
   __shared__ u64 lsh[NSLOT * NLIMB];
   __shared__ u32 s_ncl;
@@ -73,12 +83,12 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   // ---- v into shared memory; D, ||v||^2, row maximum, |X-G| against |X-Y|
   double aD = 0.0, aE = 0.0;
   u32 mx = 0, mxw = 0, dfl = 0;
-  constexpr int SB = 4;   // tiles of TPB * 4 columns requested at once: the row is short, its latency is what counts
-  for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
+  constexpr int SB = 4;   // tiles of NT * 4 columns requested at once: the row is short, its latency is what counts
+  for (int base = threadIdx.x * 4; base < dn; base += SB * NT * 4) {
     float x[SB][4], g[SB][4], y[SB][4];
 #pragma unroll
     for (int u = 0; u < SB; ++u) {
-      const int c0 = base + u * TPB * 4;
+      const int c0 = base + u * NT * 4;
       if (c0 < dn) {
         load4<ALIGNED>(xr, c0, d, x[u]);
         load4<ALIGNED>(gr, c0, d, g[u]);
@@ -87,7 +97,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     }
 #pragma unroll
     for (int u = 0; u < SB; ++u) {
-      const int c0 = base + u * TPB * 4;
+      const int c0 = base + u * NT * 4;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         if (c0 + k >= dn) break;
@@ -113,15 +123,15 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   if (lane == 0) { redd[0][wid] = aD; redd[1][wid] = aE; redu[0][wid] = mx; redu[1][wid] = mxw; redu[2][wid] = dfl; }
   __syncthreads();
   mx = 0; mxw = 0; dfl = 0;
-  for (int w = 0; w < TPB / 32; ++w) { mx = max(mx, redu[0][w]); mxw = max(mxw, redu[1][w]); dfl |= redu[2][w]; }
+  for (int w = 0; w < NT / 32; ++w) { mx = max(mx, redu[0][w]); mxw = max(mxw, redu[1][w]); dfl |= redu[2][w]; }
   const float smax = __uint_as_float(mx);
 
   // ---- radix select, all candidates at once
   if (nsel) {
-    for (int i = threadIdx.x; i < BINS1; i += TPB) tab[i] = 0;
+    for (int i = threadIdx.x; i < BINS1; i += NT) tab[i] = 0;
     __syncthreads();
 #pragma unroll 4
-    for (int i = threadIdx.x; i < dn; i += TPB) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
+    for (int i = threadIdx.x; i < dn; i += NT) atomicAdd(&tab[key_of(vs[i]) >> 20], 1u);
     __syncthreads();
     if (wid < nsel) {   // one warp per candidate
       u32 bin, above;
@@ -132,10 +142,10 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     // The keys that share a first digit with some threshold (usually a few per cent of the row) are
     // compacted once, with warp votes; the second and third digit are then histogrammed from that list.
     // A list that does not fit sends the two passes over the whole row instead.
-    for (int i = threadIdx.x; i < nsel * BINS2; i += TPB) tab[i] = 0;
+    for (int i = threadIdx.x; i < nsel * BINS2; i += NT) tab[i] = 0;
     if (threadIdx.x == 0) s_ncl = 0;
     __syncthreads();
-    for (int i0 = 0; i0 < dn; i0 += TPB) {
+    for (int i0 = 0; i0 < dn; i0 += NT) {
       const int i = i0 + threadIdx.x;
       const u32 key = (i < dn) ? key_of(vs[i]) : 0xffffffffu;
       bool hit = false;
@@ -153,7 +163,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     const u32 ncl = s_ncl;
     const bool listed = ncl <= (u32)SMALL_LIST;
     const int nscan = listed ? (int)ncl : dn;
-    for (int i = threadIdx.x; i < nscan; i += TPB) {
+    for (int i = threadIdx.x; i < nscan; i += NT) {
       const u32 key = listed ? cl[i] : key_of(vs[i]);
       for (int j = 0; j < nsel; ++j)
         if ((key >> 20) == s_b1[j]) atomicAdd(&tab[j * BINS2 + ((key >> 9) & 0x7ffu)], 1u);
@@ -165,9 +175,9 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       if (lane == 0) { s_p2[wid] = (s_b1[wid] << 11) | bin; s_ab2[wid] = s_ab1[wid] + above; }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < nsel * BINS3; i += TPB) tab[i] = 0;
+    for (int i = threadIdx.x; i < nsel * BINS3; i += NT) tab[i] = 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < nscan; i += TPB) {
+    for (int i = threadIdx.x; i < nscan; i += NT) {
       const u32 key = listed ? cl[i] : key_of(vs[i]);
       for (int j = 0; j < nsel; ++j)
         if ((key >> 9) == s_p2[j]) atomicAdd(&tab[j * BINS3 + (key & 0x1ffu)], 1u);
@@ -191,11 +201,11 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     for (int j = 0; j < nsel; ++j) {
       if (s_q[j] >= s_ntie[j]) continue;
       const u32 T = s_T[j], q = s_q[j];
-      const int per = (dn + TPB - 1) / TPB;
+      const int per = (dn + NT - 1) / NT;
       const int i0 = threadIdx.x * per, i1 = (i0 + per < dn) ? i0 + per : dn;
       u32 cnt = 0;
       for (int i = i0; i < i1; ++i) cnt += (key_of(vs[i]) == T) ? 1u : 0u;
-      const u32 ex = block_excl_scan(cnt, nullptr);
+      const u32 ex = block_excl_scan<NT>(cnt, nullptr);
       if (ex < q && q <= ex + cnt) {
         u32 seen = ex;
         for (int i = i0; i < i1; ++i)
@@ -217,7 +227,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     }
   }
 #pragma unroll 2
-  for (int i = threadIdx.x; i < dn; i += TPB) {
+  for (int i = threadIdx.x; i < dn; i += NT) {
     const float v = vs[i];
     const u32 key = key_of(v);
     const double dv = (double)v;
@@ -245,7 +255,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     for (int j = 0; j < cs.nquant; ++j) used |= (sl == 2 + cs.qsel[j]);
     double acc = 0.0;
     if (used)
-      for (int w = 0; w < TPB / 32; ++w) acc += redd[sl][w];
+      for (int w = 0; w < NT / 32; ++w) acc += redd[sl][w];
     partial[(long long)row * MAX_BLK_PER_ROW * NSLOT + sl] = acc;
   }
   if (threadIdx.x >= 32 && threadIdx.x < 32 + nsel) {
@@ -259,11 +269,11 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     diffflag[row] = ((mxw >= 0x7f800000u) ? 0x80000000u : 0u) | (dfl & 0x7fffffffu);
   }
   __syncthreads();
-  pick_row(cs, d, row, 1, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
+  pick_row<NT>(cs, d, row, 1, 1, partial, sel, maxkey, dec, flags, out, diffflag, tol);
   __syncthreads();
   if (__ldcg(&dec[row].need_exact)) {
     // the comparison could not be certified: exact integer sums of the row, then the decision from them
-    for (int i = threadIdx.x; i < NSLOT * NLIMB; i += TPB) lsh[i] = 0;
+    for (int i = threadIdx.x; i < NSLOT * NLIMB; i += NT) lsh[i] = 0;
     __syncthreads();
     // A square is mant^2 * 2^off units of 2^-298.  Squares whose offset lies within 64 bits below the
     // largest one of the row are added in per-thread 128-bit integers anchored at bit `wb` (at most 128
@@ -289,24 +299,24 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
       limb_add(lsh + slot * NLIMB, kk, p);
     };
     // D needs X - Y again: four loads of each in flight per thread
-    for (int base = threadIdx.x; base < dn; base += 4 * TPB) {
+    for (int base = threadIdx.x; base < dn; base += 4 * NT) {
       float xw[4], yw[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int i = base + u * TPB;
+        const int i = base + u * NT;
         xw[u] = (i < dn) ? xr[i] : 0.f;
         yw[u] = (i < dn) ? yr[i] : 0.f;
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        if (base + u * TPB >= dn) break;
+        if (base + u * NT >= dn) break;
         const float w = __fsub_rn(xw[u], yw[u]);
         if (key_of(w) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
         unsigned __int128 tw;
         if (sq_term(w, &tw)) accD += tw; else slow_add(0, w);
       }
     }
-    for (int i = threadIdx.x; i < dn; i += TPB) {
+    for (int i = threadIdx.x; i < dn; i += NT) {
       const float v = vs[i];
       if (key_of(v) >= 0x7f800000u) { atomicOr(&diffflag[row], 0x80000000u); continue; }
       unsigned __int128 tv;
@@ -332,7 +342,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     // The per-thread integers are added up as four 32-bit pieces each: over the warp with shuffles, over the
     // warps through `wacc` (64-bit shared atomics are compare-and-swap loops: with every thread of the CTA on
     // the same few words they would take hundreds of microseconds), and only the totals go into the limbs.
-    __shared__ u64 wacc[TPB / 32][NSLOT][4];
+    __shared__ u64 wacc[NT / 32][NSLOT][4];
     auto stash = [&](unsigned __int128 acc, int slot) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -342,7 +352,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
         if (lane == 0) wacc[wid][slot][i] = piece;
       }
     };
-    for (int i = threadIdx.x; i < (TPB / 32) * NSLOT * 4; i += TPB) (&wacc[0][0][0])[i] = 0;
+    for (int i = threadIdx.x; i < (NT / 32) * NSLOT * 4; i += NT) (&wacc[0][0][0])[i] = 0;
     __syncthreads();
     stash(accD, 0);
     stash(accE, 1);
@@ -355,7 +365,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
     if (threadIdx.x < NSLOT * 4) {
       const int slot = threadIdx.x >> 2, i = threadIdx.x & 3;
       u64 tot = 0;                                     // < 2^32 * 256 threads = 2^40
-      for (int w = 0; w < TPB / 32; ++w) tot += wacc[w][slot][i];
+      for (int w = 0; w < NT / 32; ++w) tot += wacc[w][slot][i];
       const int k0 = (wb >> 5) + i, sh = wb & 31;
       const u64 lo = (tot & 0xffffffffull) << sh, hi = (tot >> 32) << sh;      // weights 2^(32 k0) and 2^(32 (k0 + 1))
       if (lo & 0xffffffffull) atomicAdd(&lsh[slot * NLIMB + k0], lo & 0xffffffffull);
@@ -377,14 +387,14 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   if (mode != 0) {
     const u32 T = __ldcg(&dec[row].T), cut = __ldcg(&dec[row].cut);
     const float L = __ldcg(&dec[row].qL), inv = __ldcg(&dec[row].qinv), step = __ldcg(&dec[row].qstep);
-    for (int base = threadIdx.x * 4; base < dn; base += SB * TPB * 4) {
+    for (int base = threadIdx.x * 4; base < dn; base += SB * NT * 4) {
       float gq[SB][4];
 #pragma unroll
       for (int u = 0; u < SB; ++u)
-        if (base + u * TPB * 4 < dn) load4<ALIGNED>(gr, base + u * TPB * 4, d, gq[u]);
+        if (base + u * NT * 4 < dn) load4<ALIGNED>(gr, base + u * NT * 4, d, gq[u]);
 #pragma unroll
       for (int u = 0; u < SB; ++u) {
-        const int c0 = base + u * TPB * 4;
+        const int c0 = base + u * NT * 4;
         if (c0 >= dn) break;
         bool any = false;
 #pragma unroll
@@ -421,7 +431,7 @@ __global__ void __launch_bounds__(TPB) k_small_rows(const float* __restrict__ X,
   if (!mean_last) return;
   __threadfence();
   const float nf = (float)rows;
-  for (int c = threadIdx.x; c < dn; c += TPB) {
+  for (int c = threadIdx.x; c < dn; c += NT) {
     float acc = -0.f;                    // -0 + g == g bit for bit
     for (int i = 0; i < rows; ++i) acc = __fadd_rn(acc, __ldcg(G + (long long)i * d + c));
     out.mean_out[c] = __fdiv_rn(acc, nf);
@@ -472,8 +482,11 @@ __global__ void __launch_bounds__(TPB) k_small_mean(const float* G, int rows, lo
 
 // The row and the tables of up to MAXC candidates exceed the default 48 KB of dynamic shared memory.
 void set_small_kernel_attributes() {
-  cudaFuncSetAttribute(k_small_rows<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
-  cudaFuncSetAttribute(k_small_rows<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST));
+  const int bytes = 4 * (SMALL_DMAX + MAXC * BINS2 + SMALL_LIST);
+  cudaFuncSetAttribute(k_small_rows<true, TPB>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaFuncSetAttribute(k_small_rows<false, TPB>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaFuncSetAttribute(k_small_rows<true, SMALL_NT_LONG>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaFuncSetAttribute(k_small_rows<false, SMALL_NT_LONG>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 // Enqueues k_small_rows and, if a mean is wanted, k_small_mean; returns the number of launches (< 0: CUDA error).
@@ -490,10 +503,12 @@ int launch_small_rows(const Scratch& s, const CsetDev& cs, const float* X, float
   // block, word 8, zero between calls)
   const bool tiny_mean = out.mean_out != nullptr && (long long)rows * d <= 16384;
   u32* mean_ticket = tiny_mean ? s.flags + 8 : nullptr;
-  if (al4) launch_k(k_small_rows<true>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                    s.maxkey, s.diffflag, s.flags, out, tol64, mean_ticket);
-  else launch_k(k_small_rows<false>, dim3(rows), dim3(TPB), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial,
-                s.maxkey, s.diffflag, s.flags, out, tol64, mean_ticket);
+#define SMALL_LAUNCH(AL, NT)                                                                                          \
+  launch_k(k_small_rows<AL, NT>, dim3(rows), dim3(NT), shm, stream, pdl, X, G, Y, rows, d, cs, s.sel, s.dec, s.partial, \
+           s.maxkey, s.diffflag, s.flags, out, tol64, mean_ticket)
+  if (d >= SMALL_LONG_ROW) { if (al4) SMALL_LAUNCH(true, SMALL_NT_LONG); else SMALL_LAUNCH(false, SMALL_NT_LONG); }
+  else { if (al4) SMALL_LAUNCH(true, TPB); else SMALL_LAUNCH(false, TPB); }
+#undef SMALL_LAUNCH
   prof_end(pf, stream);
   ++launches;
   if (out.mean_out && !tiny_mean) {
