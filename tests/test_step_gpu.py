@@ -154,6 +154,35 @@ def test_free_running_c1_loss_trajectory(torch):
     assert relerr(eng.get_state("x").cpu().numpy(), st["x"]) <= 1e-2
 
 
+def test_step_records_do_not_depend_on_how_steps_are_batched(torch):
+    # The record of an iteration is written by the next iteration's first kernel, or by a closing kernel at the end of a
+    # batch: one call of 300 steps (more than the 256 records the device holds, replayed as graphs of two), 300 calls of
+    # one step, and calls of 1, 2, 3, ... steps must give the same records, levels, counters and state, bit for bit.
+    W = S.WORKLOADS["c1"]
+    A, t = S.logistic_problem(W["n"], W["d"], W["m"], seed=5)
+    gamma = 0.5 / S.smoothness_estimate(A, W["loss"], W["lam"])
+    x0 = np.zeros(W["d"], F32)
+    T = 300
+    runs = []
+    for plan in ([T], [1] * T, list(range(1, 24)) + [T - sum(range(1, 24))]):
+        assert sum(plan) == T
+        eng = make_engine(torch, A, t, W["loss"], W["lam"], x0, gamma, W["worker"], 1.0)
+        recs, levels = [], []
+        for k in plan:
+            r, l = eng.step(k, report=True)
+            recs += r
+            levels += l
+        runs.append((recs, levels, eng.get_state("step"), eng.get_state("bits_up"), eng.get_state("x").cpu().numpy()))
+        eng.close()
+    ref = runs[0]
+    assert ref[2] == T and len(ref[0]) == T
+    assert len({r["loss"] for r in ref[0]}) > T // 2             # the records are those of different iterations
+    for other in runs[1:]:
+        assert other[0] == ref[0] and other[1] == ref[1]
+        assert other[2] == ref[2] and other[3] == ref[3]
+        assert np.array_equal(other[4].view(np.uint32), ref[4].view(np.uint32))
+
+
 def test_free_running_c2_bidirectional(torch):
     # workload c2 as benchmarked (20 x 8 000, 2 000 samples per worker, worker and master Top-K {8, 80, 800, 8000}),
     # both sides left to run on their own for as many of its 1 000 iterations as the oracle does in about two minutes
