@@ -282,6 +282,52 @@ def test_single_pass_falls_back_when_the_sample_misleads(torch):
     assert got["fallbacks"] == 1          # row 0 only; row 1 is homogeneous
 
 
+def side_path_rows():
+    """Five rows of 1e6 entries that need, in ONE call, every side path of the single-pass route: a row whose sample
+    misleads (full select), a row with a crowded threshold bin (list levels), a row of a few distinct magnitudes (list
+    overflow, tie groups far larger than the ranking buffers), a row whose skip trigger holds with equality at
+    zeta = 14.25 (exact sums), and an ordinary row."""
+    d = 1_000_000
+    X, G, Y = S.gaussian_rows(5, d, seed=61, drift=0.3, move=0.01)
+    # row 0: large entries only where the sampling kernel never looks
+    hidden = np.ones(d, dtype=bool)
+    seen = sampled_granules(d)
+    for k in range(16):
+        hidden[np.minimum(seen * 16 + k, d - 1)] = False
+    rng = np.random.Generator(np.random.PCG64(62))
+    bump = (5.0 * rng.standard_normal(int(hidden.sum()))).astype(F32)
+    X[0, hidden] += bump
+    Y[0, hidden] += bump                                  # D stays small: the row does not skip
+    # row 1: 30 000 magnitudes within a few units in the last place around the 1 % threshold
+    v = (X[1] - G[1]).astype(F32)
+    t = np.sort(np.abs(v))[-10_000]
+    where = rng.choice(d, 30_000, replace=False)
+    near = (F32(t) * (1.0 + 1e-7 * rng.integers(-3, 4, 30_000))).astype(F32) * rng.choice([-1.0, 1.0], 30_000).astype(F32)
+    G[1, where] = 0.0
+    X[1, where] = near
+    Y[1, where] = near
+    # row 2: small integers (seven magnitudes), Y equal to X but for 1000 entries
+    Xt, Gt, _ = S.tie_vectors(1, d, seed=63, levels=3)
+    X[2], G[2] = Xt[0], Gt[0]
+    Y[2] = X[2]
+    Y[2, :1000] += 1.0
+    # row 3: ||v||^2 = 14.25 and D = 1 exactly
+    X[3] = 0.0
+    X[3, :4] = [3, -1, 2, 0.5]
+    G[3] = 0.0
+    Y[3] = X[3]
+    Y[3, 0] -= 1.0
+    return X, G, Y, [(TOPK, 1000), (TOPK, 10_000), (TOPK, 100_000)], 14.25
+
+
+def test_all_side_paths_in_one_call(torch):
+    # the cooperative side-path kernel with every phase needed at once, each by another row
+    X, G, Y, cands, zeta = side_path_rows()
+    got, res = check_against_oracle(torch, X, G, Y, cands, zeta, both_update_paths=True)
+    assert [r["level"] for r in res] == [3, 3, 3, 0, 3]
+    assert got["fallbacks"] >= 2 and got["list_levels"] >= 1 and got["rechecks"] >= 1
+
+
 def test_block_scaled_rows_keep_the_single_pass(torch):
     # contiguous blocks of very different scale (the structure of the c5 workload) at a size where
     # each block is only a few dozen tiles long: the sample must still bracket every threshold
