@@ -2249,10 +2249,14 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   if (want < 1) want = 1;
   const int nblk = (int)want;
   const dim3 sgrid(nblk, rows);
-  // in single-pass mode the full select only serves rows whose bracket failed: a small grid keeps the
-  // usual no-op launches cheap
-  long long want_full = single ? (SMS * 2 + rows - 1) / rows : nblk;
-  if (want_full > nblk) want_full = nblk;
+  // in single-pass mode the full select only serves rows whose bracket failed, inside k_side, whose CTAs stand in
+  // for this many CTAs per flagged row: as many as the kernel has, so that a single such row still gets the whole
+  // machine (with 37 per row one 12.5e6-element row took 1.4 ms; rows that are not flagged cost one flag read each)
+  long long want_full = single ? SMS * 2 : nblk;
+  if (single && want_full > (ntile + 7) / 8) want_full = (ntile + 7) / 8;   // at least eight tiles per histogram flush
+  if (want_full > ntile) want_full = ntile;
+  if (want_full < 1) want_full = 1;
+  if (want_full > MAX_BLK_PER_ROW) want_full = MAX_BLK_PER_ROW;
   const int nblk_full = (int)want_full;
   const dim3 fgrid(nblk_full, rows);
   const u32* only = single ? s.rowflag : nullptr;  // in single-pass mode the full select serves flagged rows only
