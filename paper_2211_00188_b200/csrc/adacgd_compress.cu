@@ -2342,7 +2342,7 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     sa.X = X; sa.G = G; sa.Y = Y; sa.d = d; sa.rows = rows; sa.nseg = nblk;
     sa.lh_gx = (int)(lgx < 16 ? lgx : 16);          // the lists are about 1 % of a row: a few CTAs per row do
     sa.f_gx = nblk_full;
-    long long tgx = (SMS * 4 + rows - 1) / rows;
+    long long tgx = SMS * 2;                       // per row that needs the tie order, like the fallback grid
     if (tgx > nchunk) tgx = nchunk;
     sa.t_gx = (int)tgx;
     sa.nblk_main = nblk; sa.cs_global = (const CsetDev*)s.csdev; sa.sel = s.sel; sa.list = s.list; sa.lcount = s.lcount;
