@@ -1927,8 +1927,21 @@ __global__ void __launch_bounds__(TPB) k_side(SideArgs a) {
   __shared__ CsetDev cs;
   if (threadIdx.x == 0) cs = *a.cs_global;
   __syncthreads();
-  grid.sync();
   const int G = (int)gridDim.x, b0 = (int)blockIdx.x;
+  // The tables of the phases below are not cleared per call: the grid clears them here, for the rows that use them
+  // (the exact sums' limbs, which are small, for every row).  The barrier that follows separates this from their use.
+  {
+    const long long gtid = (long long)b0 * TPB + threadIdx.x, gsz = (long long)G * TPB;
+    for (int r = 0; r < a.rows; ++r) {
+      if (!__ldcg(&a.rowflag[r]) && !__ldcg(&a.tickets[r * NTICKET + 13])) continue;
+      for (long long i = gtid; i < BINS1; i += gsz) a.hist1[(long long)r * BINS1 + i] = 0u;
+      for (long long i = gtid; i < MAXC * BINS2; i += gsz) a.hist2[(long long)r * MAXC * BINS2 + i] = 0u;
+      for (long long i = gtid; i < MAXC * BINS3; i += gsz) a.hist3[(long long)r * MAXC * BINS3 + i] = 0u;
+      for (long long i = gtid; i < MAXC * BINS1; i += gsz) a.lhist1[(long long)r * MAXC * BINS1 + i] = 0u;
+    }
+    for (long long i = gtid; i < (long long)a.rows * NSLOT * NLIMB; i += gsz) a.limbs[i] = 0ull;
+  }
+  grid.sync();
 #define SIDE_PHASE(gx, call)                                   \
   for (int v = b0; v < (gx) * a.rows; v += G) {                \
     const int bx = v % (gx), by = v / (gx);                    \
@@ -1989,7 +2002,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; }
 
 struct Layout {
-  size_t hist1, hist2, hist3, maxkey, limbs, flags, csdev, zero_end, zero_noshist, sel, dec, partial, energy, tiecnt, total;
+  size_t hist1, hist2, hist3, maxkey, limbs, flags, csdev, zero_end, zero_noshist, zero_rare, sel, dec, partial, energy, tiecnt, total;
   size_t tickets, rowflag, diffflag, shist, lhist1, fhist, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
@@ -2003,20 +2016,24 @@ static long long list_row_of(long long d) {
 static Layout layout_of(int rows, long long d, bool single_pass) {
   Layout L;
   size_t o = 0;
+  // first the tables that only the side paths of the single-pass route use (k_side clears them itself, for the rows
+  // that need them), then what every call needs cleared
   L.hist1 = o; o = align_up(o + (size_t)rows * BINS1 * 4, 256);
   L.hist2 = o; o = align_up(o + (size_t)rows * MAXC * BINS2 * 4, 256);
   L.hist3 = o; o = align_up(o + (size_t)rows * MAXC * BINS3 * 4, 256);
-  L.maxkey = o; o = align_up(o + (size_t)rows * 4, 256);
   L.limbs = o; o = align_up(o + (size_t)rows * NSLOT * NLIMB * 8, 256);
+  L.lhist1 = o;
+  if (single_pass) o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
+  L.zero_rare = o;
+  L.maxkey = o; o = align_up(o + (size_t)rows * 4, 256);
   L.rowflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
-  L.shist = L.lhist1 = L.fhist = L.flcnt = L.cntpart = o;
+  L.shist = L.fhist = L.flcnt = L.cntpart = o;
   L.zero_noshist = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
-    L.lhist1 = o; o = align_up(o + (size_t)rows * MAXC * BINS1 * 4, 256);
     L.fhist = o; o = align_up(o + (size_t)rows * MAXC * LB1 * 4, 256);
     L.zero_noshist = o;   // the sample histogram comes last: calls that sample per row in shared memory do not clear it
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
@@ -2058,6 +2075,7 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->zero_begin = b;
   s->zero_bytes = L.zero_end;
   s->zero_bytes_noshist = L.zero_noshist;
+  s->zero_rare = L.zero_rare;
   s->sel = (SelRow*)(b + L.sel);
   s->dec = (RowDec*)(b + L.dec);
   s->partial = (double*)(b + L.partial);
@@ -2236,7 +2254,12 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
   // every element sampled and many rows: one CTA per row samples into shared memory (no global sample histogram)
   const long long ngran_all = (d + SAMP_G - 1) / SAMP_G;
   const bool row_sampler = single && ngran_all / 8192 < 2 && rows >= 32;
-  cudaMemsetAsync(s.zero_begin, 0, row_sampler ? s.zero_bytes_noshist : s.zero_bytes, stream);  // histograms, limbs, row flags
+  {
+    // row flags, tickets, first-digit tables; the three-pass route also needs its histograms and limbs cleared, which
+    // in the single-pass route only k_side uses, and clears for the rows that need them (160 KB per row)
+    const size_t skip = single ? s.zero_rare : 0;
+    cudaMemsetAsync((char*)s.zero_begin + skip, 0, (row_sampler ? s.zero_bytes_noshist : s.zero_bytes) - skip, stream);
+  }
   prof_end(pf, stream);
 
   const long long ntile = (d + TPB * 4 - 1) / (TPB * 4);
