@@ -1026,13 +1026,22 @@ constexpr int RS_SHIFT = 16;
 template <bool ALIGNED>
 __global__ void __launch_bounds__(SAMP_TPB) k_sample_row(const float* __restrict__ X, const float* __restrict__ G, long long d,
                                                          CsetDev cs, SelRow* __restrict__ sel, u32* __restrict__ tickets,
-                                                         u32* __restrict__ maxkey, CsetDev* __restrict__ cs_global) {
+                                                         u32* __restrict__ maxkey, CsetDev* __restrict__ cs_global,
+                                                         u32* __restrict__ rowflag, u32* __restrict__ diffflag,
+                                                         u32* __restrict__ flcnt, u32* __restrict__ cntpart,
+                                                         u32* __restrict__ fhist) {
   pdl_begin();
   if (blockIdx.x == 0 && threadIdx.x == 0) *cs_global = cs;   // for the last CTAs of the collection pass
   extern __shared__ __align__(16) u32 sh[];   // RS_BINS counts
   __shared__ u32 wsum[SAMP_TPB / 32];
   const int row = blockIdx.x;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  // This kernel is the first of its call and has one CTA per row: it clears the row's per-call words itself (flags,
+  // completion counts, first-digit tables; the row maximum is written below), so the call needs no memset.
+  for (int i = threadIdx.x; i < MAXC * LB1; i += SAMP_TPB) fhist[(long long)row * MAXC * LB1 + i] = 0u;
+  if (threadIdx.x < NTICKET) tickets[row * NTICKET + threadIdx.x] = 0u;
+  if (threadIdx.x >= 32 && threadIdx.x < 32 + MAXC) { flcnt[row * MAXC + threadIdx.x - 32] = 0u; cntpart[row * MAXC + threadIdx.x - 32] = 0u; }
+  if (threadIdx.x == 64) { rowflag[row] = 0u; diffflag[row] = 0u; }
   for (int i = threadIdx.x; i < RS_BINS / 4; i += SAMP_TPB) reinterpret_cast<uint4*>(sh)[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   const float* xr = X + (long long)row * d;
@@ -2002,7 +2011,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static long long nchunk_of(long long d) { return (d + UPD_COLS - 1) / UPD_COLS; }
 
 struct Layout {
-  size_t hist1, hist2, hist3, maxkey, limbs, flags, csdev, zero_end, zero_noshist, zero_rare, sel, dec, partial, energy, tiecnt, total;
+  size_t hist1, hist2, hist3, maxkey, limbs, flags, csdev, zero_end, zero_rare, sel, dec, partial, energy, tiecnt, total;
   size_t tickets, rowflag, diffflag, shist, lhist1, fhist, list, lcount, cntpart, lepart, lepart3, fl, flcnt;
   long long list_row;
 };
@@ -2030,12 +2039,10 @@ static Layout layout_of(int rows, long long d, bool single_pass) {
   L.diffflag = o; o = align_up(o + (size_t)rows * 4, 256);
   L.tickets = o; o = align_up(o + (size_t)rows * NTICKET * 4, 256);
   L.shist = L.fhist = L.flcnt = L.cntpart = o;
-  L.zero_noshist = o;
   if (single_pass) {
     L.flcnt = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.cntpart = o; o = align_up(o + (size_t)rows * MAXC * 4, 256);
     L.fhist = o; o = align_up(o + (size_t)rows * MAXC * LB1 * 4, 256);
-    L.zero_noshist = o;   // the sample histogram comes last: calls that sample per row in shared memory do not clear it
     L.shist = o; o = align_up(o + (size_t)rows * SBINS * 4, 256);
   }
   L.zero_end = o;
@@ -2074,7 +2081,6 @@ void carve_scratch(Scratch* s, void* base, int rows, long long d, bool single_pa
   s->csdev = (CsetDev*)(b + L.csdev);
   s->zero_begin = b;
   s->zero_bytes = L.zero_end;
-  s->zero_bytes_noshist = L.zero_noshist;
   s->zero_rare = L.zero_rare;
   s->sel = (SelRow*)(b + L.sel);
   s->dec = (RowDec*)(b + L.dec);
@@ -2258,7 +2264,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     // row flags, tickets, first-digit tables; the three-pass route also needs its histograms and limbs cleared, which
     // in the single-pass route only k_side uses, and clears for the rows that need them (160 KB per row)
     const size_t skip = single ? s.zero_rare : 0;
-    cudaMemsetAsync((char*)s.zero_begin + skip, 0, (row_sampler ? s.zero_bytes_noshist : s.zero_bytes) - skip, stream);
+    if (!row_sampler)   // the per-row sampler clears its row's words itself
+      cudaMemsetAsync((char*)s.zero_begin + skip, 0, s.zero_bytes - skip, stream);
   }
   prof_end(pf, stream);
 
@@ -2328,8 +2335,8 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
     u32* samp_max = qinline ? s.maxkey : nullptr;
     prof_begin(pf, KID_SAMPLE, stream);
     if (row_sampler) {
-      if (al) launch_k(k_sample_row<true>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev);
-      else launch_k(k_sample_row<false>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev);
+      if (al) launch_k(k_sample_row<true>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev, s.rowflag, s.diffflag, s.flcnt, s.cntpart, s.fhist);
+      else launch_k(k_sample_row<false>, dim3(rows), dim3(SAMP_TPB), RS_BINS * 4, stream, pdl, X, G, d, cs, s.sel, s.tickets, s.maxkey, s.csdev, s.rowflag, s.diffflag, s.flcnt, s.cntpart, s.fhist);
     } else if (al) launch_k(k_sample<true>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max, s.csdev);
     else launch_k(k_sample<false>, samp_grid, dim3(SAMP_TPB), SBINS * 2, stream, pdl, X, G, d, nwin, win, s.shist, cs, s.sel, s.tickets, samp_max, s.csdev);
     prof_end(pf, stream);

@@ -118,7 +118,6 @@ struct Scratch {
   u32* flags;      // [4]: 0 nonfinite seen, 1 #exact rechecks
   CsetDev* csdev;  // the call's candidate set, for code that indexes it with run-time values
   void* zero_begin; size_t zero_bytes;  // region cleared at the start of every call
-  size_t zero_bytes_noshist;            // the same without the sample histogram (its last part)
   size_t zero_rare;                     // its first part: tables that in the single-pass route only k_side uses (and clears)
   SelRow* sel;     // [rows]
   RowDec* dec;     // [rows]
