@@ -141,6 +141,7 @@ __global__ void __launch_bounds__(256) k_axpy_log(float* __restrict__ x, const f
                                                   const unsigned long long* __restrict__ mbits, const double* __restrict__ loss,
                                                   const unsigned int* __restrict__ flags, Counters* cnt, StepLog* log,
                                                   int* loglevels) {
+  pdl_trigger();   // the forward kernel may become resident; it waits for this grid before it reads x
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));   // two binary32 roundings: the product, then the difference
   if (blockIdx.x != 0) return;

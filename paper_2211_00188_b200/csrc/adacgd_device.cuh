@@ -18,6 +18,11 @@ __device__ __forceinline__ void pdl_begin() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// The two halves on their own.  A kernel whose successor is large waits first and lets the successor in only
+// afterwards (or not at all): CTAs that become resident early hold registers and shared memory while they wait.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // Number of SMs of the device the kernel runs on.
 __device__ __forceinline__ int sm_count() {
   u32 n;

@@ -4,7 +4,7 @@
 // A memory-bound GEMV pair per worker: z = A_i x (forward), X_i = A_i^T r(z) (backward).
 #include <vector>
 
-#include "adacgd_internal.cuh"
+#include "adacgd_device.cuh"
 
 namespace adacgd {
 
@@ -357,6 +357,7 @@ __global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long
                                                                  const float* __restrict__ val, const float* __restrict__ x,
                                                                  long long rows, long long d, int blk,
                                                                  float* __restrict__ zpart) {
+  pdl_begin();
   // val / col16: the entries regrouped at init, block-major, every (block, row) span padded with zero entries to a
   // multiple of four so that a lane reads four values (16 bytes) and four 16-bit block-relative columns (8 bytes) per
   // request: 6 bytes per stored entry.  qptr[b * rows + row]: first group of four of the span.
@@ -421,6 +422,8 @@ __global__ void __launch_bounds__(CSR_FWD_TPB) k_csr_fwd_blocked(const long long
 __global__ void __launch_bounds__(TPB) k_csr_residual(const float* __restrict__ zpart, int nb, long long rows,
                                                       const float* __restrict__ target, long long m_rows, int loss,
                                                       float* __restrict__ r, LossTail lt) {
+  pdl_wait();      // the large backward kernel that follows is let in once this one runs, not before
+  pdl_trigger();
   const int worker = blockIdx.y;
   const long long l = (long long)blockIdx.x * TPB + threadIdx.x;
   double ls = 0.0;
@@ -461,6 +464,7 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
                                                       long long d, long long m_rows, int loss, float lambda,
                                                       float* __restrict__ grads) {
   // crow: 16-bit sample indices (a worker has at most CSC_RCAP samples here)
+  pdl_wait();      // no early launch of the kernel after this one: its CTAs would take room from this grid
   extern __shared__ __align__(16) float bsm[];   // [m_rows] residuals, then [TPB / 32][CSC_WPCAP] products
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   float* rs = bsm;
@@ -906,20 +910,23 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
     const DevProps* dp = current_device();
     if (!dp) return -1;
     int loss_blocks = g.loss_blocks;
+    // chained as programmatic dependents (the x update before them lets the forward kernel in early); not under the
+    // per-kernel event timers, whose records would sit between the kernels
+    const bool pdl = g.prof == nullptr;
     if (g.nb) {
       const long long rows = (long long)p.n * p.m_rows;
       long long gx = dp->sms / g.nb;            // one 1024-thread CTA per SM over all column blocks
       if (gx < 1) gx = 1;
       if (gx > (rows + 31) / 32) gx = (rows + 31) / 32;
       prof_begin(g.prof, KID_CSR_FWD, stream);
-      k_csr_fwd_blocked<<<dim3((unsigned)gx, g.nb), CSR_FWD_TPB, (size_t)g.blk * 4, stream>>>(
-          g.csr_split, g.csr_col16, g.fwd_val, x, rows, p.d, g.blk, g.zpart);
+      launch_k(k_csr_fwd_blocked, dim3((unsigned)gx, g.nb), dim3(CSR_FWD_TPB), (size_t)g.blk * 4, stream, pdl,
+               (const long long*)g.csr_split, (const u16*)g.csr_col16, (const float*)g.fwd_val, x, rows, (long long)p.d, g.blk, g.zpart);
       prof_end(g.prof, stream);
       ++launches;
       loss_blocks = (int)((p.m_rows + TPB - 1) / TPB);
       prof_begin(g.prof, KID_CSR_RES, stream);
-      k_csr_residual<<<dim3((unsigned)loss_blocks, p.n), TPB, 0, stream>>>(g.zpart, g.nb, rows, p.target, p.m_rows, p.loss,
-                                                                           g.r, make_tail(p, g, x));
+      launch_k(k_csr_residual, dim3((unsigned)loss_blocks, p.n), dim3(TPB), 0, stream, pdl, (const float*)g.zpart, g.nb, rows,
+               (const float*)p.target, (long long)p.m_rows, (int)p.loss, g.r, make_tail(p, g, x));
       prof_end(g.prof, stream);
       ++launches;
     } else {
@@ -936,8 +943,9 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
       long long gx = (8ll * dp->sms + p.n - 1) / p.n;
       if (gx > (ngroups + TPB / 32 - 1) / (TPB / 32)) gx = (ngroups + TPB / 32 - 1) / (TPB / 32);
       if (gx < 1) gx = 1;
-      k_csc_bwd_span<<<dim3((unsigned)gx, p.n), TPB, ((size_t)p.m_rows + (size_t)(TPB / 32) * CSC_WPCAP) * 4, stream>>>(
-          g.wbase, g.ptr32, g.csc_row16, g.csc_val, g.r, x, p.d, p.m_rows, p.loss, p.lambda, grads);
+      launch_k(k_csc_bwd_span, dim3((unsigned)gx, p.n), dim3(TPB), ((size_t)p.m_rows + (size_t)(TPB / 32) * CSC_WPCAP) * 4, stream,
+               pdl && g.nb != 0, (const long long*)g.wbase, (const u32*)g.ptr32, (const u16*)g.csc_row16, (const float*)g.csc_val,
+               (const float*)g.r, x, (long long)p.d, (long long)p.m_rows, (int)p.loss, (float)p.lambda, grads);
     }
     else
       k_csc_bwd<<<dim3((unsigned)((p.d + TPB - 1) / TPB), p.n), TPB, 0, stream>>>(g.csc_ptr, g.csc_row, g.csc_val, g.r, x,
