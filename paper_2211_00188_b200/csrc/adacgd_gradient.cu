@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(TPB) k_dense_fwd(const float* __restrict__ A, 
                                                    float* __restrict__ zout, const u32* __restrict__ gate) {
   // r == nullptr: only the products z = A x are wanted (zout); gate != nullptr: the launch only runs when the
   // word is zero (the incremental pass found too many changed columns and leaves the products to this kernel)
+  pdl_wait();      // may be resident while the x update runs; the backward kernel is not let in early
   if (gate && *gate != 0u) return;
   const int worker = blockIdx.y;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -206,6 +207,7 @@ __global__ void __launch_bounds__(TPB) k_dense_bwd(const float* __restrict__ A, 
                                                    const float* __restrict__ x, long long d, long long m_rows,
                                                    int split, int loss, float lambda, float* __restrict__ grads,
                                                    float* __restrict__ part, int n, u32* __restrict__ tickets) {
+  pdl_wait();
   const int worker = blockIdx.y / split, s = blockIdx.y % split;
   const long long per = (m_rows + split - 1) / split;
   const long long l0 = s * per, l1 = (l0 + per < m_rows) ? l0 + per : m_rows;
@@ -546,6 +548,8 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
 __global__ void __launch_bounds__(1024) k_loss_reduce(const double* __restrict__ losspart, long long nparts, int n,
                                                       long long m_rows, const float* __restrict__ x, long long d,
                                                       int loss, float lambda, double* __restrict__ out) {
+  pdl_wait();
+  pdl_trigger();   // one CTA: the backward kernel may become resident beside it
   __shared__ double red[32];
   double a = 0.0;
   for (long long i = threadIdx.x; i < nparts; i += blockDim.x) a += losspart[i];
@@ -745,7 +749,7 @@ __global__ void __launch_bounds__(FIN_ROWS * FIN_SLICES) k_inc_finish(const floa
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout, cudaStream_t stream,
-                      const u32* gate = nullptr);
+                      const u32* gate = nullptr, bool pdl = false);
 // Above this many short CTAs (a few sample rows each) in a forward launch the loss is added up by k_loss_reduce
 // instead of the last CTA; a CTA that walks a whole long row does not notice the count at its end.
 constexpr long long FUSED_LOSS_MAX_CTAS = 1024;
@@ -758,7 +762,7 @@ static LossTail make_tail(const adacgd_problem& p, const GradScratch& g, const f
   return t;
 }
 int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks, bool al,
-                              cudaStream_t stream);
+                              cudaStream_t stream, bool pdl = false);
 
 // The split decides the size of the partial-sum buffer, so it is part of the workspace layout and must not
 // depend on the device a context later runs on: it is taken for a nominal 148 SMs.
@@ -956,15 +960,17 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
   }
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)x | (uintptr_t)grads) & 15) == 0;
   int launches = 0;
-  launch_dense_fwd(p, g, x, g.r, nullptr, stream);
+  const bool pdl = g.prof == nullptr;   // the kernels of the pass as programmatic dependents of one another
+  launch_dense_fwd(p, g, x, g.r, nullptr, stream, nullptr, pdl);
   ++launches;
   if (dense_fwd_short_ctas(p, g) > FUSED_LOSS_MAX_CTAS) {
     prof_begin(g.prof, KID_LOSS, stream);
-    k_loss_reduce<<<1, 1024, 0, stream>>>(g.losspart, (long long)p.n * g.loss_blocks, p.n, p.m_rows, x, p.d, p.loss, p.lambda, g.loss);
+    launch_k(k_loss_reduce, dim3(1), dim3(1024), 0, stream, pdl, (const double*)g.losspart, (long long)p.n * g.loss_blocks, (int)p.n,
+             (long long)p.m_rows, x, (long long)p.d, (int)p.loss, (float)p.lambda, g.loss);
     prof_end(g.prof, stream);
     ++launches;
   }
-  return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream);
+  return launches + launch_dense_bwd_and_loss(p, g, x, grads, g.loss_blocks, al, stream, pdl);
 }
 
 static long long dense_fwd_short_ctas(const adacgd_problem& p, const GradScratch& g) {
@@ -973,14 +979,16 @@ static long long dense_fwd_short_ctas(const adacgd_problem& p, const GradScratch
 
 // The forward kernel in the shape the problem calls for: z = A v for a d-vector v, residuals if r != nullptr.
 void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float* v, float* r, float* zout,
-                      cudaStream_t stream, const u32* gate) {
+                      cudaStream_t stream, const u32* gate, bool pdl) {
   const bool al = (p.d % 4 == 0) && (((uintptr_t)p.A | (uintptr_t)v) & 15) == 0;
   prof_begin(g.prof, KID_GRAD_FWD, stream);
   const long long fwd_ctas = dense_fwd_short_ctas(p, g);
   const LossTail lt = make_tail(p, g, v, fwd_ctas);
   const bool cta_row = cta_row_mode(p);
   const dim3 grid((unsigned)(cta_row ? p.m_rows : g.loss_blocks), p.n);
-#define FWD(CR, AL, FU) k_dense_fwd<CR, AL, FU><<<grid, TPB, 0, stream>>>(p.A, p.target, v, p.d, p.m_rows, p.loss, r, lt, zout, gate)
+#define FWD(CR, AL, FU)                                                                                                   \
+  launch_k(k_dense_fwd<CR, AL, FU>, grid, dim3(TPB), 0, stream, pdl && g.prof == nullptr, (const float*)p.A, (const float*)p.target, v, \
+           (long long)p.d, (long long)p.m_rows, (int)p.loss, r, lt, zout, gate)
   if (cta_row) { if (al) FWD(true, true, true); else FWD(true, false, true); }      // long CTAs always count themselves
   else if (lt.fused) { if (al) FWD(false, true, true); else FWD(false, false, true); }
   else { if (al) FWD(false, true, false); else FWD(false, false, false); }
@@ -990,12 +998,15 @@ void launch_dense_fwd(const adacgd_problem& p, const GradScratch& g, const float
 
 // X_i = A_i^T r + reg'(x) and the loss from `loss_blocks` partial sums per worker; returns the launches.
 int launch_dense_bwd_and_loss(const adacgd_problem& p, const GradScratch& g, const float* x, float* grads, int loss_blocks,
-                              bool al, cudaStream_t stream) {
+                              bool al, cudaStream_t stream, bool pdl) {
   int launches = 0;
   const dim3 bgrid((unsigned)((p.d + TPB * 4 - 1) / (TPB * 4)), p.n * g.split);
   prof_begin(g.prof, KID_GRAD_BWD, stream);
-  if (al) k_dense_bwd<true><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n, g.bwd_tickets);
-  else k_dense_bwd<false><<<bgrid, TPB, 0, stream>>>(p.A, g.r, x, p.d, p.m_rows, g.split, p.loss, p.lambda, grads, g.part, p.n, g.bwd_tickets);
+#define BWD(AL)                                                                                                              \
+  launch_k(k_dense_bwd<AL>, bgrid, dim3(TPB), 0, stream, pdl, (const float*)p.A, (const float*)g.r, x, (long long)p.d, (long long)p.m_rows, \
+           (int)g.split, (int)p.loss, (float)p.lambda, grads, g.part, (int)p.n, g.bwd_tickets)
+  if (al) BWD(true); else BWD(false);
+#undef BWD
   prof_end(g.prof, stream);
   ++launches;
   return cudaGetLastError() == cudaSuccess ? launches : -1;
