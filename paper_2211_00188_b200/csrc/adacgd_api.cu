@@ -141,7 +141,8 @@ __global__ void __launch_bounds__(256) k_axpy_log(float* __restrict__ x, const f
                                                   const unsigned long long* __restrict__ mbits, const double* __restrict__ loss,
                                                   const unsigned int* __restrict__ flags, Counters* cnt, StepLog* log,
                                                   int* loglevels) {
-  pdl_trigger();   // the forward kernel may become resident; it waits for this grid before it reads x
+  pdl_begin();     // the forward kernel may become resident (it waits for this grid before it reads x); this grid
+                   // itself may have become resident while the last kernel of the iteration before was running
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < d) x[i] = __fsub_rn(x[i], __fmul_rn(gamma, g[i]));   // two binary32 roundings: the product, then the difference
   if (blockIdx.x != 0) return;
@@ -508,8 +509,10 @@ static adacgd_status enqueue_iteration(adacgd_ctx* c, bool capturing = false) {
   const long long d = c->p.d;
   // a0: x^{t+1} = x^t - gamma g^t
   prof_begin(c->prof, KID_AXPY, c->stream);
-  k_axpy_log<<<(unsigned)((d + 255) / 256), 256, 0, c->stream>>>(c->x, c->gm, c->gamma, d, n, c->levels, c->bits, c->mlevel, c->mbits,
-                                                                  c->gs.loss, c->scr.flags, c->counters, c->log, c->loglevels);
+  launch_k(k_axpy_log, dim3((unsigned)((d + 255) / 256)), dim3(256), 0, c->stream, c->prof == nullptr, c->x, (const float*)c->gm, c->gamma,
+           (long long)d, n, (const int*)c->levels, (const unsigned long long*)c->bits, (const int*)c->mlevel,
+           (const unsigned long long*)c->mbits, (const double*)c->gs.loss, (const unsigned int*)c->scr.flags, c->counters, c->log,
+           c->loglevels);
   prof_end(c->prof, c->stream);
   if (cudaGetLastError() != cudaSuccess) return cuda_fail(c, "x update");
   c->launches += 1;
