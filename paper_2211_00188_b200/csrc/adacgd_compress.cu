@@ -2414,7 +2414,14 @@ int launch_compress(const Scratch& s, const CsetDev& cs, const float* X, float* 
                                  (const RowDec*)s.dec, out, done));
       skip = done;
     }
-    TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, skip);
+    if (skip) {
+      // the fallback of the kernel above: as its programmatic dependent it is resident by the time that one ends, reads
+      // the word and returns
+      const bool pdl = pf == nullptr;
+      TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, skip);
+    } else {
+      TIMED_AL(KID_UPDATE, k_update, ugrid, 0, X, G, rows, d, s.dec, s.tiecnt, nchunk, 0, out, skip);
+    }
   }
 #undef PASS1_CASE
 #undef P1_ARGS
