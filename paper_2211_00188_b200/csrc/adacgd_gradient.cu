@@ -460,14 +460,18 @@ constexpr int CSC_WCOLS = 64;      // columns a warp takes at a time (two per la
 constexpr int CSC_WPCAP = 768;     // products parked per warp
 constexpr int CSC_UNR = 6;         // entries a lane requests at once
 constexpr int CSC_RCAP = 8192;     // residuals of a worker kept in shared memory
-__global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restrict__ wbase, const u32* __restrict__ ptr32,
+#ifndef CSC_TPB_N
+#define CSC_TPB_N 64
+#endif
+constexpr int CSC_TPB = CSC_TPB_N;   // threads per CTA of the span kernel: small CTAs (c3: 512 threads 242 us, 256 117, 128 115, 64 113, 32 133)
+__global__ void __launch_bounds__(CSC_TPB) k_csc_bwd_span(const long long* __restrict__ wbase, const u32* __restrict__ ptr32,
                                                       const u16* __restrict__ crow, const float* __restrict__ cval,
                                                       const float* __restrict__ r, const float* __restrict__ x,
                                                       long long d, long long m_rows, int loss, float lambda,
                                                       float* __restrict__ grads) {
   // crow: 16-bit sample indices (a worker has at most CSC_RCAP samples here)
   pdl_wait();      // no early launch of the kernel after this one: its CTAs would take room from this grid
-  extern __shared__ __align__(16) float bsm[];   // [m_rows] residuals, then [TPB / 32][CSC_WPCAP] products
+  extern __shared__ __align__(16) float bsm[];   // [m_rows] residuals, then [CSC_TPB / 32][CSC_WPCAP] products
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   float* rs = bsm;
   float* prod = bsm + m_rows + (size_t)wid * CSC_WPCAP;
@@ -475,10 +479,10 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
   const u32* ptr = ptr32 + (long long)worker * (d + 1);
   const long long base = wbase[worker];
   const float* rw = r + (long long)worker * m_rows;
-  for (int i = threadIdx.x; i < (int)m_rows; i += TPB) rs[i] = rw[i];
+  for (int i = threadIdx.x; i < (int)m_rows; i += CSC_TPB) rs[i] = rw[i];
   __syncthreads();
   const long long ngroups = (d + CSC_WCOLS - 1) / CSC_WCOLS;
-  const long long gstride = (long long)gridDim.x * (TPB / 32);
+  const long long gstride = (long long)gridDim.x * (CSC_TPB / 32);
   // Column pointers and x of a group: this lane's columns c0 + lane and c0 + lane + 32, and the ends of the
   // warp's span.  The next group's are requested before the current group's entries.
   struct Grp { u32 pa[2], pb[2], e0, e1; float xv[2]; };
@@ -496,7 +500,7 @@ __global__ void __launch_bounds__(TPB) k_csc_bwd_span(const long long* __restric
     q.e0 = ptr[c0];
     q.e1 = ptr[c1];
   };
-  long long grp = (long long)blockIdx.x * (TPB / 32) + wid;
+  long long grp = (long long)blockIdx.x * (CSC_TPB / 32) + wid;
   Grp cur, nxt;
   if (grp < ngroups) fetch(grp, cur);
   for (; grp < ngroups; grp += gstride) {
@@ -944,10 +948,10 @@ int launch_gradient(const adacgd_problem& p, const GradScratch& g, const float* 
     if (g.ccols) {
       // about eight CTAs per SM over all workers, each walking groups of columns of its worker
       const long long ngroups = (p.d + CSC_WCOLS - 1) / CSC_WCOLS;
-      long long gx = (8ll * dp->sms + p.n - 1) / p.n;
-      if (gx > (ngroups + TPB / 32 - 1) / (TPB / 32)) gx = (ngroups + TPB / 32 - 1) / (TPB / 32);
+      long long gx = (8ll * (TPB / CSC_TPB) * dp->sms + p.n - 1) / p.n;
+      if (gx > (ngroups + CSC_TPB / 32 - 1) / (CSC_TPB / 32)) gx = (ngroups + CSC_TPB / 32 - 1) / (CSC_TPB / 32);
       if (gx < 1) gx = 1;
-      launch_k(k_csc_bwd_span, dim3((unsigned)gx, p.n), dim3(TPB), ((size_t)p.m_rows + (size_t)(TPB / 32) * CSC_WPCAP) * 4, stream,
+      launch_k(k_csc_bwd_span, dim3((unsigned)gx, p.n), dim3(CSC_TPB), ((size_t)p.m_rows + (size_t)(CSC_TPB / 32) * CSC_WPCAP) * 4, stream,
                pdl && g.nb != 0, (const long long*)g.wbase, (const u32*)g.ptr32, (const u16*)g.csc_row16, (const float*)g.csc_val,
                (const float*)g.r, x, (long long)p.d, (long long)p.m_rows, (int)p.loss, (float)p.lambda, grads);
     }
@@ -1156,7 +1160,7 @@ const char* build_csc(const adacgd_problem& p, GradScratch* gp, cudaStream_t str
       cudaStreamSynchronize(stream) != cudaSuccess)
     return "copying the transposed arrays to the device failed";
   if (g.nb) cudaFuncSetAttribute(k_csr_fwd_blocked, cudaFuncAttributeMaxDynamicSharedMemorySize, CSR_BLK_MAX * 4);
-  if (g.ccols) cudaFuncSetAttribute(k_csc_bwd_span, cudaFuncAttributeMaxDynamicSharedMemorySize, (CSC_RCAP + (TPB / 32) * CSC_WPCAP) * 4);
+  if (g.ccols) cudaFuncSetAttribute(k_csc_bwd_span, cudaFuncAttributeMaxDynamicSharedMemorySize, (CSC_RCAP + (CSC_TPB / 32) * CSC_WPCAP) * 4);
   return nullptr;
 }
 
